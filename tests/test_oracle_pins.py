@@ -1,0 +1,328 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests re-types the oracle's formulas to compare it with itself:
+each one is a hand-computed value, an invariant the paper states (ternary
+weights, 8-bit activations, four weights per byte: Section 2 and Section 5.1),
+a closed form, a special case that reduces to a textbook or library routine, or
+a brute-force evaluation of the definition in fp64 / int64.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2504_12285_b200 import workloads as wl
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def bf16_bits_of(values):
+    """Exact bf16 bit patterns of fp32 values that are representable in bf16."""
+    a = np.asarray(values, np.float32)
+    bits = a.view(np.uint32)
+    assert np.all((bits & 0xFFFF) == 0), "test value is not exactly representable in bf16"
+    return (bits >> 16).astype(np.uint16)
+
+
+# --------------------------------------------------------------------------- weights
+
+
+def test_weight_quant_hand_case():
+    # mean|W| = (0.3+0.1+0.05+0.55)/4 = 0.25; ratios 1.2, -0.4, 0.2, -2.2 -> round 1, 0, 0, -2 -> clip 1, 0, 0, -1
+    W = np.array([[0.3, -0.1, 0.05, -0.55]], np.float32)
+    for eps in (0.0, 1e-5):
+        s_w, _ = oracle.weight_scale(W, eps)
+        assert abs(float(s_w) - (0.25 + eps)) < 1e-7
+        assert oracle.weight_quant(W, s_w).tolist() == [[1, 0, 0, -1]]
+
+
+def test_weight_quant_ties_round_half_to_even():
+    # mean|W| = 1 exactly, eps 0: ratios 1, 1, 0.5, 1.5.  Half-to-even gives 0 and 2 (clipped to 1);
+    # half-away-from-zero would give 1 for the 0.5.  -0.5 and -1.5 mirror it.
+    W = np.array([[1.0, 1.0, 0.5, 1.5]], np.float32)
+    s_w, _ = oracle.weight_scale(W, 0.0)
+    assert float(s_w) == 1.0
+    assert oracle.weight_quant(W, s_w).tolist() == [[1, 1, 0, 1]]
+    Wn = np.array([[-1.0, -1.0, -0.5, -1.5]], np.float32)
+    assert oracle.weight_quant(Wn, np.float32(1.0)).tolist() == [[-1, -1, 0, -1]]
+    # 2.5 -> 2 -> clip 1 and -2.5 -> -2 -> clip -1: clipping works on both sides
+    assert oracle.weight_quant(np.array([[2.5, -2.5, 0.49, -0.51]], np.float32), np.float32(1.0)).tolist() == [
+        [1, -1, 0, -1]
+    ]
+
+
+def test_weight_quant_all_zero_matrix():
+    W = np.zeros((16, 256), np.float32)
+    s_w, _ = oracle.weight_scale(W, 1e-5)
+    assert float(s_w) == float(np.float32(1e-5))
+    wq = oracle.weight_quant(W, s_w)
+    assert not wq.any()
+
+
+def test_weight_scale_is_the_mean_absolute_value():
+    # 1, -2, 3, -4 ... mean of |.| over 1..64 is 32.5 (exact in fp32)
+    W = (np.arange(1, 65, dtype=np.float32) * np.where(np.arange(64) % 2, -1, 1)).reshape(4, 16)
+    s_w, fragile = oracle.weight_scale(W, 0.0)
+    assert float(s_w) == 32.5 and not fragile
+
+
+def test_weights_are_ternary_and_match_gaussian_closed_form():
+    # For W ~ N(0, sigma^2): mean|W| -> sigma*sqrt(2/pi); a weight quantises to 0 iff |W| < s_w/2,
+    # so P(0) = erf( s_w / (2*sqrt(2)*sigma) ) = 0.3101 and P(+1) = P(-1) = 0.3450.
+    sigma = wl.WEIGHT_STD
+    W = wl.latent_weights(2560, 2560, wl.seed_for(1, 0)).numpy()
+    s_w, _ = oracle.weight_scale(W, wl.WEIGHT_EPS)
+    s_theory = sigma * math.sqrt(2.0 / math.pi) + wl.WEIGHT_EPS
+    assert abs(float(s_w) - s_theory) / s_theory < 1e-3
+    wq = oracle.weight_quant(W, s_w)
+    assert set(np.unique(wq).tolist()) == {-1, 0, 1}
+    p0 = math.erf(s_theory / (2.0 * math.sqrt(2.0) * sigma))
+    assert abs(p0 - 0.3101) < 2e-4
+    assert abs(float((wq == 0).mean()) - p0) < 1e-3
+    assert abs(float((wq == 1).mean()) - (1 - p0) / 2) < 1e-3
+    assert abs(float((wq == -1).mean()) - (1 - p0) / 2) < 1e-3
+    # the quantiser is odd: W -> -W flips every trit
+    assert np.array_equal(oracle.weight_quant(-W, s_w), -wq)
+
+
+# --------------------------------------------------------------------------- activations
+
+
+def test_act_quant_hand_cases():
+    # a = 127 -> s = 1: values are rounded directly; ties go to even (0.5->0, 1.5->2, 2.5->2)
+    y = np.array([[127.0, 0.5, 1.5, 2.5, -0.5, -2.5]], np.float32)
+    q, d, xsum = oracle.absmax_quant(y)
+    assert q.tolist() == [[127, 0, 2, 2, 0, -2]]
+    assert float(d[0]) == 1.0 and int(xsum[0]) == 129
+    # a = 2 -> s = 63.5: 63.5 -> 64 (tie to even), -127, 31.75 -> 32, 0
+    y = np.array([[1.0, -2.0, 0.5, 0.0]], np.float32)
+    q, d, xsum = oracle.absmax_quant(y)
+    assert q.tolist() == [[64, -127, 32, 0]]
+    assert float(d[0]) == float(np.float32(2.0) / np.float32(127.0))
+    assert int(xsum[0]) == 64 - 127 + 32
+
+
+def test_act_quant_zero_row_is_safe():
+    q, d, xsum = oracle.absmax_quant(np.zeros((2, 8), np.float32))
+    assert not q.any() and not xsum.any()
+    assert np.all(d == np.float32(1e-5) / np.float32(127.0))
+
+
+def test_act_quant_range_invariants():
+    # 8-bit per-token absmax: every non-zero row reaches |q| = 127 and nothing reaches -128
+    for gen, cfg in ((wl.activations_normal, 2), (wl.activations_outlier, 4), (wl.activations_student_t, 5)):
+        x = gen(33, 2560, wl.seed_for(cfg, 0))
+        out = oracle.rmsnorm_quant(wl.bf16_bits(x), wl.bf16_bits(wl.gain_ones(2560)), wl.RMS_EPS)
+        q = out["q"].astype(np.int32)
+        assert q.min() >= -127 and q.max() <= 127
+        assert np.all(np.abs(q).max(axis=1) == 127)
+        assert np.array_equal(out["xsum"], q.sum(axis=1))
+
+
+def test_rmsnorm_constant_row_and_single_spike():
+    K = 256
+    # constant row c: y_i = c / sqrt(c^2 + eps), all equal -> every code is +-127
+    for c in (1.0, -3.0, 0.015625):
+        x = bf16_bits_of(np.full((1, K), c, np.float32))
+        out = oracle.rmsnorm_quant(x, None, 1e-5, want_norm=True)
+        assert np.all(out["q"] == (127 if c > 0 else -127))
+        expect = c / math.sqrt(c * c + 1e-5)
+        assert np.allclose(out["y_norm"], expect, rtol=3e-7, atol=0)
+        assert abs(float(out["d"][0]) - abs(expect) / 127.0) <= 3e-7 * abs(expect) / 127.0
+    # a single spike c at position 5: y_5 = c / sqrt(c^2/K + eps), the rest 0
+    x = np.zeros((1, K), np.float32)
+    x[0, 5] = -2.0
+    out = oracle.rmsnorm_quant(bf16_bits_of(x), None, 1e-5, want_norm=True)
+    q = out["q"][0]
+    assert q[5] == -127 and not np.delete(q, 5).any()
+    assert abs(float(out["y_norm"][0, 5]) - (-2.0 / math.sqrt(4.0 / K + 1e-5))) < 1e-5
+    # all-zero token
+    out = oracle.rmsnorm_quant(np.zeros((1, K), np.uint16), None, 1e-5)
+    assert not out["q"].any() and int(out["xsum"][0]) == 0
+
+
+def test_rmsnorm_matches_textbook_fp64():
+    K = 2560
+    x = wl.activations_normal(7, K, wl.seed_for(2, 3))
+    g = wl.gain_random(K, wl.seed_for(2, 3, 1))
+    out = oracle.rmsnorm_quant(wl.bf16_bits(x), wl.bf16_bits(g), wl.RMS_EPS, want_norm=True)
+    xd = x.double().numpy()
+    gd = g.double().numpy()
+    ref = xd / np.sqrt((xd * xd).mean(axis=1, keepdims=True) + wl.RMS_EPS) * gd
+    assert np.allclose(out["y_norm"], ref, rtol=3e-7, atol=1e-12)
+    # and the quantised row dequantises back to the normalised row within half a step
+    deq = out["q"].astype(np.float64) * out["d"][:, None].astype(np.float64)
+    assert np.all(np.abs(deq - ref) <= 0.5 * out["d"][:, None] * (1 + 1e-5))
+    assert not out["fragile"].any()
+
+
+def test_gain_is_applied_per_channel():
+    K = 256
+    x = bf16_bits_of(np.ones((1, K), np.float32))
+    g = np.ones(K, np.float32)
+    g[3] = 2.0
+    g[9] = -0.5
+    out = oracle.rmsnorm_quant(x, bf16_bits_of(g), 0.0)
+    q = out["q"][0]
+    # y = g exactly (r = 1): a = 2 -> s = 63.5 -> 63.5 rounds to 64 (tie to even), 127, -31.75 -> -32
+    assert q[3] == 127 and q[9] == -32 and q[0] == 64
+
+
+def test_bf16_rounding_is_nearest_even():
+    f = np.array([1.0, 1.00390625, 1.01171875, 1.0078125, -1.00390625, 3.0e38], np.float32)
+    # 1 + 2^-8 is a tie between 1.0 (even) and 1 + 2^-7 -> 1.0;  1 + 3*2^-8 is a tie -> 1 + 2^-6 (even)
+    bits = oracle.f32_to_bf16(f)
+    back = oracle.bf16_to_f32(bits)
+    assert back.tolist()[:5] == [1.0, 1.0, 1.015625, 1.0078125, -1.0]
+    assert np.isfinite(back[5])
+    # agrees with the library cast on random data
+    import torch
+
+    r = torch.randn(4096, generator=torch.Generator().manual_seed(7))
+    assert np.array_equal(oracle.f32_to_bf16(r.numpy()), wl.bf16_bits(r.to(torch.bfloat16)))
+
+
+# --------------------------------------------------------------------------- packing
+
+
+def _golden_positions():
+    rows = []
+    with open(os.path.join(GOLDEN, "pack_layout_positions.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(tuple(int(v) for v in line.split()))
+    return rows
+
+
+@pytest.mark.parametrize("n,k,byte,shift", _golden_positions())
+def test_pack_positions_match_hand_computed_layout(n, k, byte, shift):
+    N, K = 32, 512
+    for trit in (1, -1):
+        wq = np.zeros((N, K), np.int8)
+        wq[n, k] = trit
+        packed = oracle.pack(wq)
+        assert packed.size == N * K // 4  # four ternary values per byte, exactly
+        expect = np.full(N * K // 4, 0x55, np.uint8)  # code 1 (= trit 0) everywhere
+        expect[byte] = (0x55 & ~(3 << shift)) | ((trit + 1) << shift)
+        assert np.array_equal(packed, expect)
+
+
+def test_pack_roundtrip_all_byte_patterns_and_random():
+    # all 3^4 combinations of four neighbouring trits, at every position of one tile
+    N, K = 16, 256
+    combos = np.array(np.meshgrid(*[[-1, 0, 1]] * 4, indexing="ij")).reshape(4, -1).T  # 81 x 4
+    wq = np.zeros((N, K), np.int8)
+    flat = wq.reshape(-1, 4)
+    for r in range(flat.shape[0]):
+        flat[r] = combos[r % 81]
+    packed = oracle.pack(wq)
+    assert np.array_equal(oracle.unpack(packed, N, K), wq)
+    # the code 3 never appears in any 2-bit field
+    fields = np.stack([(packed >> s) & 3 for s in (0, 2, 4, 6)])
+    assert fields.max() == 2
+    rng = np.random.default_rng(3)
+    wq = rng.integers(-1, 2, size=(48, 768)).astype(np.int8)
+    packed = oracle.pack(wq)
+    assert packed.size == 48 * 768 // 4
+    assert np.array_equal(oracle.unpack(packed, 48, 768), wq)
+    # a 16-byte chunk is 64 consecutive columns of one row: flipping them touches only that chunk
+    wq2 = wq.copy()
+    wq2[17, 320:384] = -wq2[17, 320:384] + (wq2[17, 320:384] == 0)
+    diff = np.nonzero(oracle.pack(wq2) != packed)[0]
+    assert diff.size > 0 and diff.min() // 16 == diff.max() // 16
+    with pytest.raises(ValueError):
+        oracle.pack(np.zeros((8, 256), np.int8))
+    with pytest.raises(ValueError):
+        oracle.pack(np.full((16, 256), 2, np.int8))
+
+
+# --------------------------------------------------------------------------- contraction and epilogue
+
+
+def _rand_case(M, N, K, seed):
+    rng = np.random.default_rng(seed)
+    q = rng.integers(-127, 128, size=(M, K)).astype(np.int8)
+    wq = rng.integers(-1, 2, size=(N, K)).astype(np.int8)
+    return q, wq
+
+
+def test_matmul_matches_int64_library_matmul():
+    for (M, N, K) in ((1, 16, 256), (3, 48, 512), (4, 128, 256)):
+        q, wq = _rand_case(M, N, K, M * 1000 + N)
+        ref = q.astype(np.int64) @ wq.astype(np.int64).T
+        assert np.array_equal(oracle.matmul_i32(q, wq).astype(np.int64), ref)
+        # W -> -W negates every accumulator
+        assert np.array_equal(oracle.matmul_i32(q, -wq), -oracle.matmul_i32(q, wq))
+
+
+def test_matmul_structured_weights():
+    M, N, K = 3, 256, 256
+    q, _ = _rand_case(M, N, K, 5)
+    ones = np.ones((N, K), np.int8)
+    acc = oracle.matmul_i32(q, ones)
+    assert np.array_equal(acc, np.repeat(q.astype(np.int32).sum(axis=1, keepdims=True), N, axis=1))
+    eye = np.eye(N, K, dtype=np.int8)
+    assert np.array_equal(oracle.matmul_i32(q, eye), q.astype(np.int32))
+    # a transposed operand or a swapped index would break this asymmetric one-hot sweep
+    for (n, k) in ((0, 0), (5, 200), (255, 1), (100, 101)):
+        w = np.zeros((N, K), np.int8)
+        w[n, k] = -1
+        acc = oracle.matmul_i32(q, w)
+        expect = np.zeros((M, N), np.int32)
+        expect[:, n] = -q[:, k].astype(np.int32)
+        assert np.array_equal(acc, expect)
+    # extreme magnitudes do not overflow: 127 * K
+    big = oracle.matmul_i32(np.full((1, 6912), 127, np.int8), np.ones((16, 6912), np.int8))
+    assert np.all(big == 127 * 6912)
+
+
+def test_sampled_matmul_agrees_with_full():
+    q, wq = _rand_case(5, 64, 512, 11)
+    full = oracle.matmul_i32(q, wq)
+    m_idx = np.array([0, 4, 2, 3], np.int32)
+    n_idx = np.array([63, 0, 17, 40], np.int32)
+    assert np.array_equal(oracle.matmul_i32_sampled(q, wq, m_idx, n_idx), full[m_idx, n_idx])
+
+
+def test_forward_equals_fp64_product_of_dequantised_operands():
+    # "Lossless" reading (Section 5.2): the integer path times the two scales equals the product of
+    # the fake-quantised operands, here evaluated in fp64 by brute force.
+    for (M, N, K, seed) in ((1, 16, 256, 1), (4, 64, 512, 2), (3, 128, 256, 3)):
+        x = wl.activations_normal(M, K, seed)
+        W = wl.latent_weights(N, K, seed + 50).numpy()
+        wts = oracle.quantize_weights(W, wl.WEIGHT_EPS)
+        out = oracle.bitlinear_forward(wl.bf16_bits(x), None, wl.RMS_EPS, wts["wq"], wts["s_w"])
+        w_deq = wts["wq"].astype(np.float64) * float(wts["s_w"])
+        x_deq = out["q"].astype(np.float64) * out["d"].astype(np.float64)[:, None]
+        ref = x_deq @ w_deq.T
+        y = out["y"].astype(np.float64)
+        assert np.all(np.abs(y - ref) <= 1e-6 * np.abs(ref))
+        assert np.all(y[out["acc"] == 0] == 0.0)
+        # and the output tracks the unquantised layer as closely as ternary weights allow: for Gaussian W
+        # corr(W, W_q) = 2*phi(z0)/sqrt(1-p0) with z0 = sqrt(2/pi)/2, p0 = P(W_q = 0)  ->  0.887
+        xd = x.double().numpy()
+        yn = xd / np.sqrt((xd * xd).mean(axis=1, keepdims=True) + wl.RMS_EPS)
+        full = yn @ W.astype(np.float64).T
+        corr = np.corrcoef(full.ravel(), y.ravel())[0, 1]
+        z0 = 0.5 * math.sqrt(2.0 / math.pi)
+        p0 = math.erf(z0 / math.sqrt(2.0))
+        expect = 2.0 * math.exp(-0.5 * z0 * z0) / math.sqrt(2.0 * math.pi) / math.sqrt(1.0 - p0)
+        assert abs(expect - 0.887) < 2e-3
+        assert abs(corr - expect) < 0.06
+
+
+def test_dequant_hand_case():
+    acc = np.array([[3, -5, 0]], np.int32)
+    y = oracle.dequant(acc, np.float32(0.5), np.array([0.25], np.float32))
+    assert y.tolist() == [[0.375, -0.625, 0.0]]
+
+
+def test_packed_artifact_roundtrip_at_layer_shape():
+    W = wl.latent_weights(640, 2560, wl.seed_for(2, 1)).numpy()
+    wts = oracle.quantize_weights(W, wl.WEIGHT_EPS)
+    assert wts["packed"].size == 640 * 2560 // 4
+    assert np.array_equal(oracle.unpack(wts["packed"], 640, 2560), wts["wq"])
+    assert not wts["fragile"]
