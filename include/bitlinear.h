@@ -1,0 +1,178 @@
+/*
+ * bitlinear.h - C ABI of the B200 (sm_100a) W1.58A8 BitLinear library.
+ *
+ * The library computes the forward pass of one BitLinear layer of BitNet b1.58
+ * (paper Section 2: ternary absmean weights, per-token absmax int8 activations,
+ * subln normalisation in front of the projection, no bias; Section 5.1: weights
+ * stored packed, four ternary values per byte, unpacked on chip right before the
+ * integer matrix product with the 8-bit activations).
+ *
+ * Conventions for every entry point
+ *  - All pointers are DEVICE pointers owned by the caller unless a parameter is
+ *    documented as a host pointer.  The library allocates no device memory and
+ *    frees none; scratch space is passed in as a workspace.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  Calls only enqueue work on that stream and never synchronise,
+ *    except the *_host entry point, which says so.
+ *  - Matrices are row-major.  x is [M][K], weights are [N][K] (out x in), y is [M][N].
+ *  - Supported shapes: K a multiple of 256 with 256 <= K <= 16384; N a multiple
+ *    of 16; M >= 0 (M == 0 is a no-op that returns BITLINEAR_OK).
+ *  - Device pointers must be 16-byte aligned.
+ *  - Inputs must be finite; NaN/Inf propagate unspecified values but never fault.
+ *  - Host-detectable errors are returned before anything is launched.  A failed
+ *    launch is reported as BITLINEAR_ERR_CUDA.  Nothing throws, aborts or prints.
+ *
+ * Numerical definition (bit-exact integer stages; every fp32 operation is one
+ * IEEE round-to-nearest-even operation, "Round" is round-half-to-even):
+ *   r      = fl32( 1 / sqrt( mean_k(x^2) + rms_eps ) )      (sum of squares in fp64)
+ *   yn_k   = fl32( fl32(x_k * r) * g_k )
+ *   a      = max( max_k |yn_k|, 1e-5 )
+ *   xq_k   = clip( Round( fl32( yn_k * fl32(127 / a) ) ), -128, 127 ),   d = fl32(a / 127)
+ *   s_w    = fl32( fl32(mean |W|) + eps_w )                  (mean in fp64)
+ *   Wq_nk  = clip( Round( fl32(W_nk / s_w) ), -1, 1 )
+ *   acc_mn = sum_k xq_mk * Wq_nk                              (int32, exact)
+ *   y_mn   = fl32( fl32( (float)acc_mn * s_w ) * d_m )        (bf16 output: RN-even cast of that)
+ *
+ * Packed weight layout (2 bits per weight, code c = Wq + 1 in {0,1,2}; 3 is unused)
+ *   The [N][K] matrix is cut into tiles of 16 rows x 256 columns, 1024 bytes each,
+ *   stored row-block major: tile index = (n / 16) * (K / 256) + (k / 256).
+ *   Inside a tile, row r = 8*h + g (h in 0..1, g in 0..7) and column
+ *   c = 64*t + 16*i + 4*j + b (t, i, j, b in 0..3) live at
+ *       byte  512*h + 64*g + 16*t + 4*i + b,   bits 2*j and 2*j+1.
+ *   Hence a 16-byte chunk holds 64 consecutive columns of one row, the 32 lanes of
+ *   a warp loading 16 bytes each cover 8 rows x 256 columns of contiguous memory,
+ *   a little-endian 32-bit word holds 16 consecutive columns, and
+ *   (word >> 2*j) & 0x03030303 yields the codes of four consecutive columns, one
+ *   per byte - directly a dot-product-of-four or tensor-core operand.
+ *   Kernels accumulate sum_k c*xq and subtract sum_k xq (produced by the
+ *   activation quantiser) to recover sum_k Wq*xq.
+ */
+#ifndef BITLINEAR_H_
+#define BITLINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    BITLINEAR_OK = 0,
+    BITLINEAR_ERR_NULL = 1,      /* a required pointer is NULL */
+    BITLINEAR_ERR_SHAPE = 2,     /* unsupported M, N or K */
+    BITLINEAR_ERR_ALIGN = 3,     /* a pointer is not 16-byte aligned */
+    BITLINEAR_ERR_WORKSPACE = 4, /* workspace missing or too small */
+    BITLINEAR_ERR_DTYPE = 5,     /* unknown dtype code */
+    BITLINEAR_ERR_ARCH = 6,      /* the current device is not compute capability 10.x */
+    BITLINEAR_ERR_CUDA = 7,      /* a CUDA runtime call or a launch failed */
+    BITLINEAR_ERR_TIMEOUT = 8    /* a bounded device-side wait ran out (see bitlinear_poll_status) */
+} bitlinear_status;
+
+/* dtype codes */
+#define BITLINEAR_F32 0
+#define BITLINEAR_BF16 1
+
+/* Which contraction kernel bitlinear_matmul_q / bitlinear_forward use. */
+#define BITLINEAR_PATH_AUTO 0  /* decode kernel for M <= 16, tensor-core kernel above */
+#define BITLINEAR_PATH_GEMV 1  /* force the streaming decode kernel (any M, in chunks of 16 tokens) */
+#define BITLINEAR_PATH_GEMM 2  /* force the tcgen05 tensor-core kernel (needs N % 128 == 0) */
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* bitlinear_status_string(int status);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int bitlinear_version(void);
+
+/* Bytes of the packed form of an [N][K] ternary matrix: N*K/4 (Section 5.1: four values per
+ * byte).  Returns 0 for an unsupported shape. */
+size_t bitlinear_packed_bytes(int N, int K);
+
+/* Workspace bytes bitlinear_pack_weights needs for an [N][K] matrix (fp64 partial sums of the
+ * absmean reduction).  Returns 0 for an unsupported shape. */
+size_t bitlinear_pack_workspace_bytes(int N, int K);
+
+/* Workspace bytes bitlinear_forward needs: int8 activations [M][K], the per-token scale and
+ * code sum, and, when the tensor-core path can be taken (M > 16 or a forced path), an
+ * unpacked uint8 copy of the weight codes [N][K].  Returns 0 for an unsupported shape. */
+size_t bitlinear_workspace_bytes(int M, int N, int K);
+
+/* Workspace bytes bitlinear_matmul_q needs (the unpacked weight codes of the tensor-core path;
+ * 0 when only the decode kernel can be taken, i.e. M <= 16 and path AUTO or GEMV). */
+size_t bitlinear_matmul_workspace_bytes(int M, int N, int K, int path);
+
+/*
+ * Offline weight quantiser and packer (Section 2, "Weight Quantization": absmean scheme onto
+ * {-1,0,+1}; Section 5.1: four ternary values per byte kept in HBM).
+ *   W          in : [N][K] master weights, fp32 (w_dtype 0) or bf16 (w_dtype 1).
+ *   eps_w      in : added to mean|W| to form the scale s_w.
+ *   packed_out out: bitlinear_packed_bytes(N,K) bytes in the layout described above.
+ *   s_w_out    out: one fp32 on the device, the dequantisation scale mean|W| + eps_w.
+ *   ws / ws_bytes : scratch of at least bitlinear_pack_workspace_bytes(N,K).
+ * The reduction order is fixed, so the result is deterministic run to run.
+ */
+int bitlinear_pack_weights(const void* W, int w_dtype, int N, int K, float eps_w, void* packed_out,
+                           float* s_w_out, void* ws, size_t ws_bytes, void* stream);
+
+/* Test hook: expand a packed matrix back to int8 values in {-1,0,1}, [N][K] row-major. */
+int bitlinear_unpack_weights(const void* packed, int N, int K, int8_t* wq_out, void* stream);
+
+/*
+ * Fused RMSNorm + per-token absmax int8 quantiser (Section 2, "Activation Quantization" and
+ * "Normalization": the subln norm feeding each BitLinear, 8-bit absmax per token).
+ *   x_bf16   in : [M][K] bf16.
+ *   gain     in : [K] bf16 RMSNorm gain, or NULL for all ones.
+ *   xq_out   out: [M][K] int8 codes.
+ *   d_out    out: [M] fp32 dequantisation scale a/127 of each token.
+ *   xsum_out out: [M] int32 sum of each token's codes (the contraction kernels need it); nullable.
+ */
+int bitlinear_quant_act(const void* x_bf16, const void* gain, float rms_eps, int M, int K,
+                        int8_t* xq_out, float* d_out, int32_t* xsum_out, void* stream);
+
+/*
+ * Ternary x int8 contraction over packed weights with the dequantising epilogue
+ * (Section 5.1: packed weights are loaded from HBM, unpacked on chip and multiplied with the
+ * 8-bit activations; Section 2 fixes the two scales the epilogue undoes).
+ *   xq, d, xsum in : outputs of bitlinear_quant_act (all three required).
+ *   packed, s_w in : outputs of bitlinear_pack_weights (s_w on the device).
+ *   y_out      out : [M][N] fp32 (y_dtype 0) or bf16 (y_dtype 1).
+ *   acc_out    out : nullable; [M][N] int32 raw accumulators sum_k xq*Wq, for parity checks.
+ *   path           : BITLINEAR_PATH_*.
+ *   ws / ws_bytes  : scratch of at least bitlinear_matmul_workspace_bytes(M,N,K,path); may be
+ *                    NULL when that is 0.
+ */
+int bitlinear_matmul_q(const int8_t* xq, const float* d, const int32_t* xsum, const void* packed,
+                       const float* s_w, int M, int N, int K, void* y_out, int y_dtype,
+                       int32_t* acc_out, int path, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * The whole BitLinear forward: bitlinear_quant_act followed by bitlinear_matmul_q (path AUTO)
+ * on the same stream (Section 2: norm -> activation quantiser -> W1.58A8 product -> rescale).
+ *   ws / ws_bytes : scratch of at least bitlinear_workspace_bytes(M,N,K).
+ */
+int bitlinear_forward(const void* x_bf16, const void* gain, float rms_eps, const void* packed,
+                      const float* s_w, int M, int N, int K, void* y_out, int y_dtype, void* ws,
+                      size_t ws_bytes, void* stream);
+
+/*
+ * bitlinear_forward for callers whose activations live in HOST memory: copies x (host, ideally
+ * pinned) into the workspace, runs the forward, copies y back to the host buffer and
+ * SYNCHRONISES the stream before returning.
+ *   x_host  in : host pointer, [M][K] bf16.      y_host out: host pointer, [M][N] of y_dtype.
+ *   gain, packed, s_w, ws: device pointers as in bitlinear_forward;
+ *   ws_bytes >= bitlinear_workspace_bytes(M,N,K) + bitlinear_host_staging_bytes(M,N,K,y_dtype).
+ */
+size_t bitlinear_host_staging_bytes(int M, int N, int K, int y_dtype);
+int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, const void* packed,
+                           const float* s_w, int M, int N, int K, void* y_host, int y_dtype, void* ws,
+                           size_t ws_bytes, void* stream);
+
+/* Reads and clears the sticky device-side status word of the current device: BITLINEAR_OK, or
+ * BITLINEAR_ERR_TIMEOUT if a kernel gave up a bounded wait since the last poll.  Synchronises
+ * `stream` first. */
+int bitlinear_poll_status(void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITLINEAR_H_ */

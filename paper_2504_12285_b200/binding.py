@@ -1,0 +1,218 @@
+"""Thin ctypes binding of libbitlinear.so: argument marshalling only.
+
+Every function here has the name of the C entry point it calls (see
+include/bitlinear.h) and does nothing but check tensor dtypes/devices, take
+data pointers and the current CUDA stream, call into the library and raise on a
+non-zero status.  PyTorch is used for device memory and streams only.  There is
+no fallback: if the shared library is missing or a call fails, it raises.
+"""
+from __future__ import annotations
+
+import ctypes
+from pathlib import Path
+
+import torch
+
+from . import build as _build
+
+F32, BF16 = 0, 1
+PATH_AUTO, PATH_GEMV, PATH_GEMM = 0, 1, 2
+
+_lib = None
+_c_void_p, _c_int, _c_size_t, _c_float = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t, ctypes.c_float
+
+_SIGNATURES = {
+    "bitlinear_status_string": (ctypes.c_char_p, [_c_int]),
+    "bitlinear_version": (_c_int, []),
+    "bitlinear_packed_bytes": (_c_size_t, [_c_int, _c_int]),
+    "bitlinear_pack_workspace_bytes": (_c_size_t, [_c_int, _c_int]),
+    "bitlinear_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int]),
+    "bitlinear_matmul_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int]),
+    "bitlinear_host_staging_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int]),
+    "bitlinear_pack_weights": (_c_int, [_c_void_p, _c_int, _c_int, _c_int, _c_float, _c_void_p, _c_void_p,
+                                        _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_unpack_weights": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_void_p]),
+    "bitlinear_quant_act": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_int, _c_int, _c_void_p, _c_void_p,
+                                     _c_void_p, _c_void_p]),
+    "bitlinear_matmul_q": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
+                                    _c_void_p, _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_forward": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
+                                   _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
+                                        _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_poll_status": (_c_int, [_c_void_p]),
+}
+
+
+class BitLinearError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where} failed: status {status} ({status_string(status)})")
+
+
+def library_path() -> Path:
+    return _build.LIB
+
+
+def lib() -> ctypes.CDLL:
+    """Load libbitlinear.so (building it with nvcc if absent); raises if that is impossible."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        loaded = ctypes.CDLL(str(path))
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(loaded, name)  # AttributeError if an entry point is missing
+            fn.restype = res
+            fn.argtypes = args
+        _lib = loaded
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().bitlinear_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise BitLinearError(status, where)
+
+
+def _ptr(t: torch.Tensor | None) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> torch.Tensor:
+    if not t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous CUDA tensor of {dtype}")
+    return t
+
+
+def _ydt(dtype) -> int:
+    if dtype == torch.float32:
+        return F32
+    if dtype == torch.bfloat16:
+        return BF16
+    raise TypeError("output dtype must be float32 or bfloat16")
+
+
+def bitlinear_packed_bytes(N: int, K: int) -> int:
+    return int(lib().bitlinear_packed_bytes(N, K))
+
+
+def bitlinear_pack_workspace_bytes(N: int, K: int) -> int:
+    return int(lib().bitlinear_pack_workspace_bytes(N, K))
+
+
+def bitlinear_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().bitlinear_workspace_bytes(M, N, K))
+
+
+def bitlinear_matmul_workspace_bytes(M: int, N: int, K: int, path: int = PATH_AUTO) -> int:
+    return int(lib().bitlinear_matmul_workspace_bytes(M, N, K, path))
+
+
+def bitlinear_host_staging_bytes(M: int, N: int, K: int, y_dtype=torch.float32) -> int:
+    return int(lib().bitlinear_host_staging_bytes(M, N, K, _ydt(y_dtype)))
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 16), dtype=torch.uint8, device=device)
+
+
+def bitlinear_pack_weights(W: torch.Tensor, eps_w: float = 1e-5):
+    """W [N, K] fp32 or bf16 on the GPU -> (packed uint8 [N*K/4], s_w fp32 [1]), both on the GPU."""
+    if W.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("W must be float32 or bfloat16")
+    _dev(W, W.dtype, "W")
+    N, K = W.shape
+    nbytes = bitlinear_packed_bytes(N, K)
+    if nbytes == 0:
+        raise BitLinearError(2, "bitlinear_pack_weights")
+    packed = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    s_w = torch.empty(1, dtype=torch.float32, device=W.device)
+    ws = _workspace(bitlinear_pack_workspace_bytes(N, K), W.device)
+    rc = lib().bitlinear_pack_weights(_ptr(W), F32 if W.dtype == torch.float32 else BF16, N, K, eps_w, _ptr(packed),
+                                      _ptr(s_w), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_pack_weights")
+    return packed, s_w
+
+
+def bitlinear_unpack_weights(packed: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    _dev(packed, torch.uint8, "packed")
+    wq = torch.empty(N, K, dtype=torch.int8, device=packed.device)
+    _check(lib().bitlinear_unpack_weights(_ptr(packed), N, K, _ptr(wq), _stream()), "bitlinear_unpack_weights")
+    return wq
+
+
+def bitlinear_quant_act(x: torch.Tensor, gain: torch.Tensor | None, rms_eps: float = 1e-5):
+    """x [M, K] bf16 -> (xq int8 [M, K], d fp32 [M], xsum int32 [M])."""
+    _dev(x, torch.bfloat16, "x")
+    if gain is not None:
+        _dev(gain, torch.bfloat16, "gain")
+    M, K = x.shape
+    xq = torch.empty(M, K, dtype=torch.int8, device=x.device)
+    d = torch.empty(max(M, 1), dtype=torch.float32, device=x.device)[:M]
+    xsum = torch.empty(max(M, 1), dtype=torch.int32, device=x.device)[:M]
+    rc = lib().bitlinear_quant_act(_ptr(x), _ptr(gain), rms_eps, M, K, _ptr(xq), _ptr(d), _ptr(xsum), _stream())
+    _check(rc, "bitlinear_quant_act")
+    return xq, d, xsum
+
+
+def bitlinear_matmul_q(xq, d, xsum, packed, s_w, N: int, y_dtype=torch.float32, want_acc: bool = False,
+                       path: int = PATH_AUTO, ws: torch.Tensor | None = None):
+    """Contraction + epilogue on quantised activations -> y [M, N] (and the int32 accumulators)."""
+    _dev(xq, torch.int8, "xq")
+    _dev(d, torch.float32, "d")
+    _dev(xsum, torch.int32, "xsum")
+    _dev(packed, torch.uint8, "packed")
+    _dev(s_w, torch.float32, "s_w")
+    M, K = xq.shape
+    y = torch.empty(M, N, dtype=y_dtype, device=xq.device)
+    acc = torch.empty(M, N, dtype=torch.int32, device=xq.device) if want_acc else None
+    if ws is None:
+        ws = _workspace(bitlinear_matmul_workspace_bytes(M, N, K, path), xq.device)
+    rc = lib().bitlinear_matmul_q(_ptr(xq), _ptr(d), _ptr(xsum), _ptr(packed), _ptr(s_w), M, N, K, _ptr(y),
+                                  _ydt(y_dtype), _ptr(acc), path, _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_matmul_q")
+    return (y, acc) if want_acc else y
+
+
+def bitlinear_forward(x, gain, packed, s_w, N: int, rms_eps: float = 1e-5, y_dtype=torch.float32,
+                      ws: torch.Tensor | None = None, out: torch.Tensor | None = None) -> torch.Tensor:
+    """The whole BitLinear forward on device tensors -> y [M, N]."""
+    _dev(x, torch.bfloat16, "x")
+    if gain is not None:
+        _dev(gain, torch.bfloat16, "gain")
+    _dev(packed, torch.uint8, "packed")
+    _dev(s_w, torch.float32, "s_w")
+    M, K = x.shape
+    y = out if out is not None else torch.empty(M, N, dtype=y_dtype, device=x.device)
+    if ws is None:
+        ws = _workspace(bitlinear_workspace_bytes(M, N, K), x.device)
+    rc = lib().bitlinear_forward(_ptr(x), _ptr(gain), rms_eps, _ptr(packed), _ptr(s_w), M, N, K, _ptr(y),
+                                 _ydt(y.dtype), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_forward")
+    return y
+
+
+def bitlinear_forward_host(x_host, gain, packed, s_w, N: int, y_host, rms_eps: float = 1e-5,
+                           ws: torch.Tensor | None = None) -> torch.Tensor:
+    """Forward with HOST activations in and HOST result out (copies inside; synchronises)."""
+    if x_host.is_cuda or y_host.is_cuda or x_host.dtype != torch.bfloat16:
+        raise TypeError("x_host / y_host must be CPU tensors (x bf16)")
+    M, K = x_host.shape
+    if ws is None:
+        ws = _workspace(bitlinear_workspace_bytes(M, N, K) + bitlinear_host_staging_bytes(M, N, K, y_host.dtype),
+                        packed.device)
+    rc = lib().bitlinear_forward_host(_ptr(x_host), _ptr(gain), rms_eps, _ptr(packed), _ptr(s_w), M, N, K,
+                                      _ptr(y_host), _ydt(y_host.dtype), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_forward_host")
+    return y_host
+
+
+def bitlinear_poll_status() -> int:
+    return int(lib().bitlinear_poll_status(_stream()))

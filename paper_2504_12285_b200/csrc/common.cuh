@@ -1,0 +1,56 @@
+// Shared declarations of the BitLinear CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "bitlinear.h"
+
+namespace bitlinear {
+
+// Packed layout constants (see "Packed weight layout" in bitlinear.h).
+constexpr int kTileRows = 16;
+constexpr int kTileCols = 256;
+constexpr int kTileBytes = 1024;
+constexpr int kMaxK = 16384;
+constexpr int kGemvMaxTokens = 16;
+
+__host__ __device__ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+inline bool shape_ok(int N, int K) {
+    return N > 0 && K >= kTileCols && K <= kMaxK && (N % kTileRows) == 0 && (K % kTileCols) == 0;
+}
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Layout of the forward workspace: [xq M*K][d M floats][xsum M ints][tensor-core scratch].
+struct ForwardWorkspace {
+    size_t xq_off, d_off, xsum_off, mm_off, total;
+};
+ForwardWorkspace forward_workspace(int M, int N, int K, size_t mm_bytes);
+
+// ---- kernel launchers (each returns a cudaError_t from the launch) ---------------------------
+cudaError_t launch_absmean(const void* W, int w_dtype, size_t count, float eps_w, double* partials,
+                           int n_partials, float* s_w_out, cudaStream_t st);
+cudaError_t launch_quant_pack(const void* W, int w_dtype, int N, int K, const float* s_w, uint32_t* packed,
+                              cudaStream_t st);
+cudaError_t launch_unpack_i8(const uint32_t* packed, int N, int K, int8_t* wq, cudaStream_t st);
+cudaError_t launch_unpack_codes_u8(const uint32_t* packed, int N, int K, uint8_t* codes, cudaStream_t st);
+int absmean_num_partials(size_t count);
+
+cudaError_t launch_quant_act(const __nv_bfloat16* x, const __nv_bfloat16* gain, float eps, int M, int K,
+                             int8_t* xq, float* d, int32_t* xsum, cudaStream_t st);
+
+cudaError_t launch_gemv(const int8_t* xq, const float* d, const int32_t* xsum, const uint32_t* packed,
+                        const float* s_w, int M, int N, int K, void* y, int y_dtype, int32_t* acc_out,
+                        cudaStream_t st);
+
+// tcgen05 tensor-core GEMM on unpacked codes; returns a bitlinear_status.
+int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* codes, const float* s_w,
+                 int M, int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st);
+size_t gemm_scratch_bytes(int N, int K);
+
+// Sticky device-side status word (set by kernels whose bounded waits ran out).
+int* device_status_word();
+
+}  // namespace bitlinear

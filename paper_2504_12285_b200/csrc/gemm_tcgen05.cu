@@ -1,0 +1,375 @@
+// Prefill contraction (M > 16 tokens): int8 activations x uint8 weight codes on the 5th-generation
+// tensor cores (tcgen05.mma kind::i8, s8 x u8 -> s32) with accumulators in tensor memory.
+// (Paper Section 5.1: the packed weights are expanded to a form the matrix units can consume right
+// before the product with the 8-bit activations; here the expansion target is the code c = Wq + 1,
+// and the epilogue removes the offset with the per-token code sum.)
+//
+// Persistent, warp-specialised kernel, one CTA per SM:
+//   warp 0   : TMA producer  - 128B-swizzled tiles of A (tokens x K) and B (weight rows x K) into a
+//              4-stage shared-memory ring, completion on mbarriers
+//   warp 1   : MMA issuer    - one elected thread issues tcgen05.mma 128 x 256 x 32 and commits
+//   warps 2-5: epilogue      - tcgen05.ld of a finished 128 x 256 int32 accumulator, subtract the
+//              code sum, two fp32 multiplies, store; tensor memory is double buffered so the
+//              epilogue of tile i overlaps the main loop of tile i+1.
+// Every wait is bounded: if one runs out the CTA raises a sticky status word and leaves cleanly.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "common.cuh"
+
+namespace bitlinear {
+
+namespace {
+
+constexpr int BM = 128;   // tokens per tile (UMMA M, one per tensor-memory lane)
+constexpr int BN = 256;   // weight rows per tile (UMMA N, one per tensor-memory column)
+constexpr int BK = 128;   // bytes of K per pipeline stage = one 128-byte swizzle row
+constexpr int UMMA_K = 32;
+constexpr int STAGES = 4;
+constexpr uint32_t A_BYTES = BM * BK;
+constexpr uint32_t B_BYTES = BN * BK;
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr int THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;  // two accumulator buffers of 256 columns
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+
+// ---- thin PTX wrappers -------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done;
+}
+
+// Bounded wait: false if the CTA is aborting or the time limit ran out (which raises the abort flag).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                        uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes with the 128-byte
+// swizzle: 8-row groups are 1024 bytes apart (stride offset), descriptor version 1, layout type 2.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+    uint64_t desc = 0;
+    desc |= (uint64_t)((saddr & 0x3FFFFu) >> 4);  // start address, 16-byte units
+    desc |= (uint64_t)1 << 16;                    // leading byte offset (unused with swizzle): 1
+    desc |= (uint64_t)(1024 >> 4) << 32;          // stride byte offset between 8-row groups
+    desc |= (uint64_t)1 << 46;                    // descriptor version for this architecture
+    desc |= (uint64_t)2 << 61;                    // 128-byte swizzle
+    return desc;
+}
+
+// Instruction descriptor: D = s32, A = s8 (activations), B = u8 (weight codes), both K-major.
+__host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
+    return (2u << 4) | (1u << 7) | (0u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+struct TileCoord {
+    int m0, n0;
+};
+__device__ __forceinline__ TileCoord tile_coord(int tile, int m_tiles) {
+    // consecutive tiles share the weight tile and walk over the tokens
+    return TileCoord{(tile % m_tiles) * BM, (tile / m_tiles) * BN};
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const float* __restrict__ d, const int32_t* __restrict__ xsum, const float* __restrict__ s_w_ptr, int M,
+               int N, int K, void* __restrict__ y, int y_dtype, int32_t* __restrict__ acc_out, int* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
+    uint64_t* full_bar = bars;                 // [STAGES] TMA bytes landed
+    uint64_t* empty_bar = bars + STAGES;       // [STAGES] MMAs that read the stage retired
+    uint64_t* tfull_bar = bars + 2 * STAGES;   // [2] accumulator buffer complete
+    uint64_t* tempty_bar = tfull_bar + 2;      // [2] accumulator buffer drained by the epilogue
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m_tiles = (M + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
+    const int total_tiles = m_tiles * n_tiles;
+    const int k_blocks = K / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(full_bar + s), 1);
+            mbar_init(smem_u32(empty_bar + s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(tfull_bar + b), 1);
+            mbar_init(smem_u32(tempty_bar + b), 4);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
+                const TileCoord tc = tile_coord(tile, m_tiles);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = smem_u32(full_bar + stage);
+                    mbar_expect_tx(fb, STAGE_BYTES);
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+                    tma_load_2d(sa, &map_a, kb * BK, tc.m0, fb);
+                    tma_load_2d(sa + A_BYTES, &map_b, kb * BK, tc.n0, fb);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = make_idesc(BM, BN);
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            int iter = 0;
+            for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++iter) {
+                const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
+                if (!mbar_wait(smem_u32(tempty_bar + buf), bphase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(smem_u32(full_bar + stage), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
+                    const uint64_t a_desc = make_smem_desc(sa);
+                    const uint64_t b_desc = make_smem_desc(sa + A_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        // advance both operands by 32 bytes of K inside the swizzled row
+                        umma_i8(d_tmem, a_desc + (uint64_t)(k * UMMA_K / 16), b_desc + (uint64_t)(k * UMMA_K / 16), idesc,
+                                (uint32_t)((kb | k) != 0));
+                    }
+                    umma_commit(smem_u32(empty_bar + stage));  // frees the stage once these MMAs retire
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(smem_u32(tfull_bar + buf));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
+        const float s_w = *s_w_ptr;
+        bool ok = true;
+        int iter = 0;
+        for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++iter) {
+            const TileCoord tc = tile_coord(tile, m_tiles);
+            const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
+            if (!mbar_wait(smem_u32(tfull_bar + buf), bphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const int m = tc.m0 + quad * 32 + lane;
+            const bool row_ok = m < M;
+            const int xs = row_ok ? xsum[m] : 0;
+            const float dm = row_ok ? d[m] : 0.0f;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + c * 32, r);
+                tmem_ld_wait();
+                const int n = tc.n0 + c * 32;
+                if (row_ok && n < N) {
+                    const size_t off = (size_t)m * N + n;
+                    int a[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) a[i] = (int)r[i] - xs;
+                    if (acc_out != nullptr) {
+                        int4* dst = reinterpret_cast<int4*>(acc_out + off);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) dst[i] = make_int4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
+                    }
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __fmul_rn(__fmul_rn((float)a[i], s_w), dm);
+                    if (y_dtype == BITLINEAR_BF16) {
+                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(y) + off);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint32_t w[4];
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 p = __floats2bfloat162_rn(v[8 * i + 2 * e], v[8 * i + 2 * e + 1]);
+                                w[e] = *reinterpret_cast<const uint32_t*>(&p);
+                            }
+                            dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+                        }
+                    } else {
+                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(y) + off);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(tempty_bar + buf));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // give copies that may still be in flight time to land before shared memory is released
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+        if (threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side -----------------------------------------------------------------------------------
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_tiled_fn() {
+    static std::once_flag once;
+    static EncodeTiledFn fn = nullptr;
+    std::call_once(once, [] {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    });
+    return fn;
+}
+
+// 2-D map over a row-major [rows][K] byte matrix; box = box_rows x 128 bytes, 128-byte swizzle.
+bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+size_t gemm_scratch_bytes(int N, int K) { return (size_t)N * K; }
+
+int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* codes, const float* s_w, int M,
+                 int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st) {
+    static std::once_flag attr_once;
+    static cudaError_t attr_err = cudaSuccess;
+    static int sm_count = 0;
+    std::call_once(attr_once, [] {
+        attr_err = cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        int dev = 0;
+        if (attr_err == cudaSuccess) attr_err = cudaGetDevice(&dev);
+        if (attr_err == cudaSuccess) attr_err = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
+    });
+    if (attr_err != cudaSuccess || sm_count <= 0) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
+    CUtensorMap map_a, map_b;
+    if (!make_map(&map_a, xq, M, K, BM) || !make_map(&map_b, codes, N, K, BN)) return BITLINEAR_ERR_CUDA;
+    const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    const int grid = tiles < sm_count ? tiles : sm_count;
+    gemm_i8_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(map_a, map_b, d, xsum, s_w, M, N, K, y, y_dtype, acc_out,
+                                                      device_status_word());
+    return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+
+}  // namespace bitlinear
