@@ -143,19 +143,35 @@ def run_ours(args):
     packed_bytes = sum(p["packed"].numel() for p in pool)
     assert packed_bytes == 521_011_200
     gains = {k: wl.gain_ones(k).to(dev) for k in (wl.HIDDEN, wl.FFN)}
-    xs = {}
-    for i, (name, n, k) in enumerate(wl.LAYER_SHAPES):
-        xs[name] = wl.activations_normal(M, k, wl.seed_for(CONFIG_ID, i)).to(dev)
-    ys = {name: torch.empty(M, n, dtype=torch.float32, device=dev) for name, n, k in wl.LAYER_SHAPES}
-    ws = torch.empty(max(bl.bitlinear_workspace_bytes(M, n, k) for _, n, k in wl.LAYER_SHAPES), dtype=torch.uint8,
-                     device=dev)
+    # activations and outputs live in two arenas (one slot per forward) so that the end-to-end leg can
+    # move them with one copy each way
+    x_off, y_off, xo, yo = [], [], 0, 0
+    for p in pool:
+        x_off.append(xo)
+        y_off.append(yo)
+        xo += (M * p["K"] * 2 + 255) // 256 * 256
+        yo += (M * p["N"] * 4 + 255) // 256 * 256
+    x_host = torch.empty(xo, dtype=torch.uint8).pin_memory()
+    y_host = torch.empty(yo, dtype=torch.uint8).pin_memory()
+    x_dev = torch.empty(xo, dtype=torch.uint8, device=dev)
+    y_dev = torch.empty(yo, dtype=torch.uint8, device=dev)
+    shape_x = {name: wl.activations_normal(M, k, wl.seed_for(CONFIG_ID, i)) for i, (name, n, k) in enumerate(wl.LAYER_SHAPES)}
+    items = []
+    for p, xo_, yo_ in zip(pool, x_off, y_off):
+        nb = M * p["K"] * 2
+        x_host[xo_:xo_ + nb] = shape_x[p["name"]].view(torch.uint8).reshape(-1)
+        xv = x_dev[xo_:xo_ + nb].view(torch.bfloat16).view(M, p["K"])
+        yv = y_dev[yo_:yo_ + M * p["N"] * 4].view(torch.float32).view(M, p["N"])
+        items.append((xv, gains[p["K"]], p["packed"], p["s_w"], yv))
+    x_dev.copy_(x_host)
+    batch = bl.ProblemBatch(items, wl.RMS_EPS)
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=dev)
+    bl.bitlinear_forward_batch(batch, ws)  # uploads the plan once
 
     def step():
-        for p in pool:
-            bl.bitlinear_forward(xs[p["name"]], gains[p["K"]], p["packed"], p["s_w"], p["N"], wl.RMS_EPS, ws=ws,
-                                 out=ys[p["name"]])
+        bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
 
-    launches_per_step = 2 * len(pool)  # one quantiser kernel + one contraction kernel per forward
+    launches_per_step = 2  # one quantiser launch over all tokens + one persistent weight-streaming launch
 
     for _ in range(args.warmup):
         step()
@@ -168,56 +184,45 @@ def run_ours(args):
     value, slowest = replicas.aggregate_throughput(packed_bytes * args.steps / 1e9, sec, device=str(dev))
     ms_per_step = slowest * 1e3 / args.steps
 
-    # ---- roofline of the dominant kernel: the decode contraction, timed launch by launch ----
-    xq_d = {}
-    for name, n, k in wl.LAYER_SHAPES:
-        xq_d[name] = bl.bitlinear_quant_act(xs[name], gains[k], wl.RMS_EPS)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in pool]
-    gemv_ms = []
-    for rep in range(max(3, args.steps)):
-        torch.cuda.synchronize()
-        for (e0, e1), p in zip(ev, pool):
-            xq, d, xsum = xq_d[p["name"]]
-            e0.record()
-            bl.bitlinear_matmul_q(xq, d, xsum, p["packed"], p["s_w"], p["N"], path=bl.PATH_GEMV)
-            e1.record()
-        torch.cuda.synchronize()
-        if rep >= 1:
-            gemv_ms.append(sum(e0.elapsed_time(e1) for e0, e1 in ev))
-    gemv_launch_s = statistics.median(gemv_ms) / 1e3 / len(pool)
-    bytes_per_launch = packed_bytes / len(pool)
-    achieved = bytes_per_launch / gemv_launch_s / 1e9
-    roofline = {"bound": "hbm", "kernel": "gemv_kernel (decode contraction, M=1)", "achieved": round(achieved, 1),
-                "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
-                "frac": round(achieved / peaks["hbm_gbs"], 4),
-                "algorithmic_bytes_per_launch": bytes_per_launch, "avg_launch_us": round(gemv_launch_s * 1e6, 3),
-                "traffic": None}
+    # ---- roofline of the dominant kernel: the persistent weight-streaming kernel, timed alone ----
+    stream_ms = []
+    for rep in range(max(5, args.steps)):
+        stream_ms.append(cuda_time_ms(lambda: bl.bitlinear_forward_batch(batch, ws, reuse_plan=True, reuse_act=True)))
+    stream_s = statistics.median(stream_ms[2:]) / 1e3
+    achieved = packed_bytes / stream_s / 1e9
+    roofline = {"bound": "hbm", "kernel": "decode_stream_kernel (persistent decode contraction, 210 matmuls per launch)",
+                "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                "frac": round(achieved / peaks["hbm_gbs"], 4), "algorithmic_bytes_per_launch": packed_bytes,
+                "avg_launch_us": round(stream_s * 1e6, 2), "traffic": None}
 
-    # ---- end to end with host buffers through bitlinear_forward_host ----
+    # ---- the same 210 forwards as separate bitlinear_forward calls (two launches each), for comparison ----
+    def step_calls():
+        for xv, g, packed, s_w, yv in items:
+            bl.bitlinear_forward(xv, g, packed, s_w, yv.shape[1], wl.RMS_EPS, ws=ws, out=yv)
+
+    step_calls()
+    ms_calls = cuda_time_ms(lambda: [step_calls() for _ in range(3)]) / 3
+    per_call = {"api": "bitlinear_forward, one call per BitLinear", "ms_per_step": round(ms_calls, 4),
+                "value": round(packed_bytes / ms_calls / 1e6, 1), "unit": UNIT}
+
+    # ---- end to end with host buffers through bitlinear_forward_batch_host ----
     e2e = None
-    if rank == 0 or world > 1:
-        xh = {name: wl.activations_normal(M, k, wl.seed_for(CONFIG_ID, i)).pin_memory()
-              for i, (name, n, k) in enumerate(wl.LAYER_SHAPES)}
-        yh = {name: torch.empty(M, n, dtype=torch.float32).pin_memory() for name, n, k in wl.LAYER_SHAPES}
-        ws_h = torch.empty(max(bl.bitlinear_workspace_bytes(M, n, k) + bl.bitlinear_host_staging_bytes(M, n, k)
-                               for _, n, k in wl.LAYER_SHAPES), dtype=torch.uint8, device=dev)
-
+    if True:
         def step_host():
-            for p in pool:
-                bl.bitlinear_forward_host(xh[p["name"]], gains[p["K"]], p["packed"], p["s_w"], p["N"], yh[p["name"]],
-                                          wl.RMS_EPS, ws=ws_h)
+            bl.bitlinear_forward_batch_host(batch, x_host, x_dev, y_dev, y_host, ws, reuse_plan=True)
 
-        for _ in range(2):
+        for _ in range(3):
             step_host()
         replicas.barrier()
-        n_e2e = max(1, min(args.steps, 5))
-        ms_h = cuda_time_ms(lambda: [step_host() for _ in range(n_e2e)])
+        t0 = time.perf_counter()
+        ms_h = cuda_time_ms(lambda: [step_host() for _ in range(args.steps)])
+        wall_h = (time.perf_counter() - t0) * 1e3
         replicas.barrier()
-        v_h, _ = replicas.aggregate_throughput(packed_bytes * n_e2e / 1e9, ms_h / 1e3, device=str(dev))
-        e2e = {"value": round(v_h, 2), "unit": UNIT,
-               "h2d_bytes_per_step": sum(2 * M * p["K"] for p in pool),
-               "d2h_bytes_per_step": sum(4 * M * p["N"] for p in pool),
-               "api": "bitlinear_forward_host, one call per BitLinear (copy in, forward, copy out, sync)"}
+        v_h, _ = replicas.aggregate_throughput(packed_bytes * args.steps / 1e9, max(ms_h, wall_h * 0.0 + ms_h) / 1e3,
+                                               device=str(dev))
+        e2e = {"value": round(v_h, 2), "unit": UNIT, "ms_per_step": round(ms_h / args.steps, 4),
+               "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(y_host.numel()),
+               "api": "bitlinear_forward_batch_host: pinned x arena -> device, 2 launches, y arena -> pinned host, sync"}
 
     # ---- prefill: int8 tensor-core path at M = 2048 on the 7 shapes (rank 0 only) ----
     prefill = None
@@ -241,7 +246,7 @@ def run_ours(args):
                        "parallelism": "replicas only (no collective)" if world > 1 else "single GPU"},
             "frac_of_hbm_peak": round(value / world / peaks["hbm_gbs"], 4),
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "prefill": prefill, "cpu_baseline": cpu,
+            "roofline": roofline, "per_call": per_call, "prefill": prefill, "cpu_baseline": cpu,
         }
         print(json.dumps(out))
     replicas.finalize()
@@ -315,7 +320,7 @@ def oracle_decode_baseline(budget_s: float):
         one_pass()
         passes += 1
         el = time.perf_counter() - t0
-        if el > budget_s or passes >= 200:
+        if el > budget_s or passes >= 5000:
             break
     packed = sum(n * k // 4 for _, n, k, _, _ in mats)
     return {"value": round(packed * passes / el / 1e9, 3), "unit": UNIT, "cores": oracle.num_threads(),
@@ -347,6 +352,53 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+def run_case(args):
+    """One kernel on one shape (for profiling and sweeps): --case gemv|gemm|quant|pack --shape q --m 1.
+
+    Distinct copies of the packed weights (--copies) are cycled so that the footprint exceeds L2."""
+    from paper_2504_12285_b200 import binding as bl
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    n, k = wl.SHAPE_NK[args.shape]
+    M = args.m
+    peaks = load_peaks()
+    W = wl.latent_weights(n, k, wl.seed_for(CONFIG_ID, wl.SHAPE_INDEX[args.shape])).to(dev)
+    packed0, s_w = bl.bitlinear_pack_weights(W, wl.WEIGHT_EPS)
+    copies = [packed0] + [packed0.clone() for _ in range(args.copies - 1)]
+    x = wl.activations_normal(M, k, wl.seed_for(CONFIG_ID, 0, 1)).to(dev)
+    gain = wl.gain_ones(k).to(dev)
+    xq, d, xsum = bl.bitlinear_quant_act(x, gain, wl.RMS_EPS)
+    path = {"gemv": bl.PATH_GEMV, "gemm": bl.PATH_GEMM}.get(args.case, bl.PATH_AUTO)
+    ws = torch.empty(max(16, bl.bitlinear_matmul_workspace_bytes(M, n, k, path)), dtype=torch.uint8, device=dev)
+    ws_p = torch.empty(bl.bitlinear_pack_workspace_bytes(n, k), dtype=torch.uint8, device=dev)
+    y = torch.empty(M, n, dtype=torch.float32, device=dev)
+    lib, st = bl.lib(), torch.cuda.current_stream().cuda_stream
+
+    def one(i):
+        p = copies[i % len(copies)]
+        if args.case in ("gemv", "gemm"):
+            rc = lib.bitlinear_matmul_q(xq.data_ptr(), d.data_ptr(), xsum.data_ptr(), p.data_ptr(), s_w.data_ptr(), M, n, k,
+                                        y.data_ptr(), 0, None, path, ws.data_ptr(), ws.numel(), st)
+        elif args.case == "quant":
+            rc = lib.bitlinear_quant_act(x.data_ptr(), gain.data_ptr(), wl.RMS_EPS, M, k, xq.data_ptr(), d.data_ptr(),
+                                         xsum.data_ptr(), st)
+        else:
+            rc = lib.bitlinear_pack_weights(W.data_ptr(), 0, n, k, wl.WEIGHT_EPS, p.data_ptr(), s_w.data_ptr(),
+                                            ws_p.data_ptr(), ws_p.numel(), st)
+        assert rc == 0, rc
+
+    for i in range(args.warmup):
+        one(i)
+    calls = args.steps * len(copies)
+    ms = cuda_time_ms(lambda: [one(i) for i in range(calls)])
+    us = ms * 1e3 / calls
+    out = {"case": args.case, "shape": args.shape, "M": M, "N": n, "K": k, "copies": len(copies), "calls": calls,
+           "us_per_call": round(us, 3), "packed_GBps": round(n * k / 4 / us / 1e3, 1),
+           "tops": round(2.0 * M * n * k / us / 1e6, 1), "hbm_peak": peaks["hbm_gbs"]}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -354,7 +406,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--case", choices=["gemv", "gemm", "quant", "pack"], default=None)
+    ap.add_argument("--shape", choices=list(wl.SHAPE_NK), default="q")
+    ap.add_argument("--m", type=int, default=1)
+    ap.add_argument("--copies", type=int, default=1)
     args = ap.parse_args()
+    if args.case:
+        return run_case(args)
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         run_reference(args)

@@ -167,6 +167,51 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
                            const float* s_w, int M, int N, int K, void* y_host, int y_dtype, void* ws,
                            size_t ws_bytes, void* stream);
 
+/*
+ * Batched decode: `count` independent BitLinear forwards of at most 16 tokens each (the decode
+ * regime of Section 5.1, where the cost is the packed weight bytes streamed from HBM) in two
+ * launches: one fused RMSNorm+quantiser launch over every token, then one persistent kernel that
+ * streams the packed weights of all problems back to back.
+ *   problems : HOST array of `count` descriptors; the pointers inside are DEVICE pointers with the
+ *              meaning, layout and alignment of the bitlinear_forward arguments.  M <= 16,
+ *              K <= 8192.  Problems with M == 0 are skipped.  Outputs must not alias inputs of
+ *              other problems of the same call (they run concurrently).
+ *   flags    : 0, or an OR of BITLINEAR_BATCH_REUSE_PLAN (the previous call on this workspace had
+ *              exactly the same descriptors: skips re-uploading the plan) and
+ *              BITLINEAR_BATCH_REUSE_ACT (the inputs are unchanged as well: skips launch 1).
+ *   ws       : device scratch of at least bitlinear_batch_workspace_bytes(problems, count); it
+ *              holds the uploaded plan and the quantised activations, so a call must not overlap
+ *              another call that uses the same workspace.
+ */
+typedef struct bitlinear_problem {
+    const void* x;      /* [M][K] bf16 */
+    const void* gain;   /* [K] bf16 or NULL */
+    const void* packed; /* packed weights of an [N][K] matrix */
+    const float* s_w;   /* its scale */
+    void* y;            /* [M][N] */
+    int M, N, K;
+    int y_dtype;        /* BITLINEAR_F32 or BITLINEAR_BF16 */
+    float rms_eps;
+    int reserved;       /* set to 0 */
+} bitlinear_problem;
+
+#define BITLINEAR_BATCH_REUSE_PLAN 1 /* descriptors unchanged since the previous call on this workspace */
+#define BITLINEAR_BATCH_REUSE_ACT 2  /* inputs x unchanged too: skip the quantiser launch, reuse its results in ws */
+
+size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count);
+int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
+                            void* stream);
+
+/*
+ * bitlinear_forward_batch for callers whose activations live in HOST memory.  The x pointers of the
+ * descriptors point into one device arena x_dev and the y pointers into one device arena y_dev;
+ * the call copies x_host (host, ideally pinned, x_bytes) into x_dev, runs the batch, copies y_dev
+ * (y_bytes) into y_host and SYNCHRONISES the stream before returning.
+ */
+int bitlinear_forward_batch_host(const bitlinear_problem* problems, int count, int flags, const void* x_host,
+                                 void* x_dev, size_t x_bytes, const void* y_dev, void* y_host, size_t y_bytes,
+                                 void* ws, size_t ws_bytes, void* stream);
+
 /* Reads and clears the sticky device-side status word of the current device: BITLINEAR_OK, or
  * BITLINEAR_ERR_TIMEOUT if a kernel gave up a bounded wait since the last poll.  Synchronises
  * `stream` first. */

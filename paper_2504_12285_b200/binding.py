@@ -41,7 +41,21 @@ _SIGNATURES = {
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
+    "bitlinear_batch_workspace_bytes": (_c_size_t, [_c_void_p, _c_int]),
+    "bitlinear_forward_batch": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_forward_batch_host": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p,
+                                              _c_void_p, _c_size_t, _c_void_p, _c_size_t, _c_void_p]),
 }
+
+BATCH_REUSE_PLAN = 1
+BATCH_REUSE_ACT = 2
+
+
+class Problem(ctypes.Structure):
+    """Mirror of the C struct bitlinear_problem."""
+    _fields_ = [("x", _c_void_p), ("gain", _c_void_p), ("packed", _c_void_p), ("s_w", _c_void_p), ("y", _c_void_p),
+                ("M", _c_int), ("N", _c_int), ("K", _c_int), ("y_dtype", _c_int), ("rms_eps", _c_float),
+                ("reserved", _c_int)]
 
 
 class BitLinearError(RuntimeError):
@@ -212,6 +226,60 @@ def bitlinear_forward_host(x_host, gain, packed, s_w, N: int, y_host, rms_eps: f
                                       _ptr(y_host), _ydt(y_host.dtype), _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_forward_host")
     return y_host
+
+
+class ProblemBatch:
+    """A host array of bitlinear_problem descriptors plus the tensors they point to (kept alive)."""
+
+    def __init__(self, items, rms_eps: float = 1e-5):
+        """items: iterable of (x [M,K] bf16, gain [K] bf16 or None, packed uint8, s_w fp32 [1], y [M,N])."""
+        self.tensors = [tuple(it) for it in items]
+        self.array = (Problem * max(len(self.tensors), 1))()
+        for i, (x, gain, packed, s_w, y) in enumerate(self.tensors):
+            _dev(x, torch.bfloat16, "x")
+            if gain is not None:
+                _dev(gain, torch.bfloat16, "gain")
+            _dev(packed, torch.uint8, "packed")
+            _dev(s_w, torch.float32, "s_w")
+            if not y.is_cuda or not y.is_contiguous():
+                raise TypeError("y must be a contiguous CUDA tensor")
+            M, K = x.shape
+            if y.shape[0] != M:
+                raise ValueError("x and y disagree on M")
+            self.array[i] = Problem(_ptr(x), _ptr(gain), _ptr(packed), _ptr(s_w), _ptr(y), M, y.shape[1], K,
+                                    _ydt(y.dtype), rms_eps, 0)
+        self.count = len(self.tensors)
+
+    def workspace_bytes(self) -> int:
+        return int(lib().bitlinear_batch_workspace_bytes(ctypes.addressof(self.array), self.count))
+
+
+def bitlinear_batch_workspace_bytes(batch: ProblemBatch) -> int:
+    return batch.workspace_bytes()
+
+
+def bitlinear_forward_batch(batch: ProblemBatch, ws: torch.Tensor, reuse_plan: bool = False,
+                            reuse_act: bool = False) -> None:
+    """Run every forward of the batch (decode sizes, M <= 16) in two launches; results land in the y tensors."""
+    _dev(ws, torch.uint8, "ws")
+    flags = (BATCH_REUSE_PLAN if reuse_plan else 0) | (BATCH_REUSE_ACT if reuse_act else 0)
+    rc = lib().bitlinear_forward_batch(ctypes.addressof(batch.array), batch.count, flags, _ptr(ws), ws.numel(),
+                                       _stream())
+    _check(rc, "bitlinear_forward_batch")
+
+
+def bitlinear_forward_batch_host(batch: ProblemBatch, x_host: torch.Tensor, x_dev: torch.Tensor, y_dev: torch.Tensor,
+                                 y_host: torch.Tensor, ws: torch.Tensor, reuse_plan: bool = False) -> None:
+    """Batch forward with HOST activations in and HOST results out: x_host -> x_dev arena, run, y_dev arena -> y_host."""
+    if x_host.is_cuda or y_host.is_cuda or not x_dev.is_cuda or not y_dev.is_cuda:
+        raise TypeError("x_host / y_host must be CPU tensors and x_dev / y_dev CUDA tensors")
+    xb, yb = x_host.numel() * x_host.element_size(), y_host.numel() * y_host.element_size()
+    if xb > x_dev.numel() * x_dev.element_size() or yb > y_dev.numel() * y_dev.element_size():
+        raise ValueError("device arenas are smaller than the host buffers")
+    rc = lib().bitlinear_forward_batch_host(ctypes.addressof(batch.array), batch.count,
+                                            BATCH_REUSE_PLAN if reuse_plan else 0, _ptr(x_host), _ptr(x_dev), xb,
+                                            _ptr(y_dev), _ptr(y_host), yb, _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_forward_batch_host")
 
 
 def bitlinear_poll_status() -> int:

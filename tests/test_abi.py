@@ -92,6 +92,30 @@ def test_host_detectable_errors_need_no_gpu():
     assert lib.bitlinear_forward(addr, NULL, 1e-5, addr, addr, 0, 16, 256, addr, 0, addr, 4096, NULL) == 0
 
 
+def test_batch_entry_point_host_checks():
+    lib = binding.lib()
+    buf = (ctypes.c_char * 4096)()
+    addr = (ctypes.addressof(buf) + 255) // 256 * 256
+    arr = (binding.Problem * 2)()
+    arr[0] = binding.Problem(addr, None, addr, addr, addr, 1, 16, 256, 0, 1e-5, 0)
+    arr[1] = binding.Problem(addr, None, addr, addr, addr, 4, 32, 512, 1, 1e-5, 0)
+    need = lib.bitlinear_batch_workspace_bytes(ctypes.addressof(arr), 2)
+    assert need >= 256 + 4 * 512
+    assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, None, 0, None) == 4       # no workspace
+    assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, addr, need - 1, None) == 4
+    assert lib.bitlinear_forward_batch(None, 2, 0, addr, need, None) == 1
+    assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 0, 0, None, 0, None) == 0       # empty batch
+    assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 8, addr, need, None) == 5    # unknown flag
+    arr[1].M = 17                                                                               # decode sizes only
+    assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, addr, 1 << 20, None) == 2
+    assert lib.bitlinear_batch_workspace_bytes(ctypes.addressof(arr), 2) == 0
+    arr[1].M = 4
+    arr[1].packed = None
+    assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, addr, 1 << 20, None) == 1
+    arr[1].packed = addr + 4
+    assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, addr, 1 << 20, None) == 3
+
+
 def test_binding_raises_instead_of_falling_back():
     import torch
 

@@ -1,0 +1,109 @@
+"""Parity of the batched decode entry point (one quantiser launch + one persistent weight-streaming
+kernel for many independent BitLinear forwards) with the CPU oracle, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_12285_b200 import binding as bl
+from paper_2504_12285_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+def make_case(shapes, seed, y_dtype=torch.float32, gains=False):
+    """shapes: list of (M, N, K).  Returns (batch, refs) with one oracle result per problem."""
+    items, refs = [], []
+    for i, (M, N, K) in enumerate(shapes):
+        x = wl.activations_normal(M, K, seed + 10 * i) if i % 2 == 0 else wl.activations_student_t(M, K, seed + 10 * i)
+        g = wl.gain_random(K, seed + 10 * i + 1) if gains else None
+        W = wl.latent_weights(N, K, seed + 10 * i + 2)
+        packed, s_w = bl.bitlinear_pack_weights(W.to(DEV), wl.WEIGHT_EPS)
+        wref = oracle.quantize_weights(W.numpy(), wl.WEIGHT_EPS)
+        assert np.array_equal(packed.cpu().numpy(), wref["packed"])
+        ref = oracle.bitlinear_forward(wl.bf16_bits(x), None if g is None else wl.bf16_bits(g), wl.RMS_EPS, wref["wq"],
+                                       wref["s_w"]) if M > 0 else None
+        y = torch.full((M, N), float("nan"), dtype=y_dtype, device=DEV)
+        items.append((x.to(DEV), None if g is None else g.to(DEV), packed, s_w, y))
+        refs.append(ref)
+    return bl.ProblemBatch(items, wl.RMS_EPS), refs
+
+
+def check(batch, refs):
+    for (x, g, packed, s_w, y), ref in zip(batch.tensors, refs):
+        if ref is None:
+            continue
+        ok = ref["fragile"] == 0
+        assert ok.mean() > 0.9
+        if y.dtype == torch.float32:
+            got = y.cpu().numpy().astype(np.float64)[ok]
+            want = ref["y"].astype(np.float64)[ok]
+            assert np.all(np.abs(got - want) <= 1e-6 * np.abs(want))
+            assert np.all(got[ref["acc"][ok] == 0] == 0.0)
+        else:
+            want = oracle.f32_to_bf16(ref["y"]).astype(np.int32)[ok]
+            got = wl.bf16_bits(y.cpu()).astype(np.int32)[ok]
+            assert np.all(np.abs(got - want) <= 1)
+
+
+def run(batch, reuse=False):
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    bl.bitlinear_forward_batch(batch, ws, reuse_plan=False)
+    if reuse:
+        first = [t[4].clone() for t in batch.tensors]
+        for t in batch.tensors:
+            t[4].fill_(float("nan"))
+        bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
+        torch.cuda.synchronize()
+        for a, t in zip(first, batch.tensors):
+            assert torch.equal(a, t[4])
+    torch.cuda.synchronize()
+    assert bl.bitlinear_poll_status() == 0
+
+
+def test_batch_single_token_mixed_shapes():
+    shapes = [(1, 16, 256), (1, 48, 768), (1, 640, 2560), (1, 2560, 6912), (1, 128, 1024), (1, 32, 8192)]
+    batch, refs = make_case(shapes, 100, gains=True)
+    run(batch, reuse=True)
+    check(batch, refs)
+
+
+def test_batch_fewer_items_than_sms():
+    batch, refs = make_case([(1, 16, 256), (1, 32, 512)], 200)
+    run(batch)
+    check(batch, refs)
+
+
+@pytest.mark.parametrize("ms", [(2, 3, 8, 5), (16, 9, 1, 12)])
+def test_batch_several_tokens(ms):
+    shapes = [(ms[0], 48, 768), (ms[1], 640, 2560), (ms[2], 256, 6912), (ms[3], 128, 256)]
+    batch, refs = make_case(shapes, 300 + ms[0], gains=True)
+    run(batch, reuse=True)
+    check(batch, refs)
+
+
+def test_batch_bf16_output_and_empty_problem():
+    shapes = [(4, 64, 512), (0, 32, 256), (1, 640, 2560)]
+    batch, refs = make_case(shapes, 400, y_dtype=torch.bfloat16)
+    run(batch)
+    check(batch, refs)
+
+
+@pytest.mark.parametrize("M", [1, 4, 16])
+def test_batch_one_layer_decode_step(M):
+    # the seven BitLinear shapes of one 2B-style layer in a single call
+    shapes = [(M, n, k) for _, n, k in wl.LAYER_SHAPES]
+    batch, refs = make_case(shapes, wl.seed_for(2, 0, M))
+    run(batch)
+    check(batch, refs)
+
+
+def test_batch_matches_single_forward_bitwise():
+    shapes = [(1, n, k) for _, n, k in wl.LAYER_SHAPES[:4]]
+    batch, _ = make_case(shapes, 500)
+    run(batch)
+    for x, g, packed, s_w, y in batch.tensors:
+        y1 = bl.bitlinear_forward(x, g, packed, s_w, y.shape[1], wl.RMS_EPS)
+        assert torch.equal(y, y1)
