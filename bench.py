@@ -196,9 +196,12 @@ def run_ours(args):
                 "avg_launch_us": round(stream_s * 1e6, 2), "traffic": None}
 
     # ---- the same 210 forwards as separate bitlinear_forward calls (two launches each), for comparison ----
+    ws_call = torch.empty(max(bl.bitlinear_workspace_bytes(M, n, k) for _, n, k in wl.LAYER_SHAPES), dtype=torch.uint8,
+                          device=dev)
+
     def step_calls():
         for xv, g, packed, s_w, yv in items:
-            bl.bitlinear_forward(xv, g, packed, s_w, yv.shape[1], wl.RMS_EPS, ws=ws, out=yv)
+            bl.bitlinear_forward(xv, g, packed, s_w, yv.shape[1], wl.RMS_EPS, ws=ws_call, out=yv)
 
     step_calls()
     ms_calls = cuda_time_ms(lambda: [step_calls() for _ in range(3)]) / 3
@@ -352,14 +355,41 @@ def run_reference(args):
     print(json.dumps(out))
 
 
+def run_case_batch(args, bl, dev):
+    """The batched decode call on --layers layers of the 7 shapes at --m tokens (a smaller copy of the headline step)."""
+    M = args.m
+    pool = build_decode_pool(bl, dev, args.layers)
+    packed_bytes = sum(p["packed"].numel() for p in pool)
+    gains = {k: wl.gain_ones(k).to(dev) for k in (wl.HIDDEN, wl.FFN)}
+    items = []
+    for i, p in enumerate(pool):
+        x = wl.activations_normal(M, p["K"], wl.seed_for(CONFIG_ID, i % 7, M)).to(dev)
+        items.append((x, gains[p["K"]], p["packed"], p["s_w"], torch.empty(M, p["N"], dtype=torch.float32, device=dev)))
+    batch = bl.ProblemBatch(items, wl.RMS_EPS)
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=dev)
+    bl.bitlinear_forward_batch(batch, ws)
+    for _ in range(args.warmup):
+        bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
+    ms = cuda_time_ms(lambda: [bl.bitlinear_forward_batch(batch, ws, reuse_plan=True) for _ in range(args.steps)]) / args.steps
+    ms_s = statistics.median(cuda_time_ms(lambda: bl.bitlinear_forward_batch(batch, ws, reuse_plan=True, reuse_act=True))
+                             for _ in range(max(3, args.steps)))
+    print(json.dumps({"case": "batch", "M": M, "layers": args.layers, "forwards": len(pool), "packed_bytes": packed_bytes,
+                      "us_per_step": round(ms * 1e3, 2), "packed_GBps": round(packed_bytes / ms / 1e6, 1),
+                      "stream_kernel_us": round(ms_s * 1e3, 2), "stream_kernel_GBps": round(packed_bytes / ms_s / 1e6, 1),
+                      "hbm_peak": load_peaks()["hbm_gbs"]}))
+
+
 def run_case(args):
-    """One kernel on one shape (for profiling and sweeps): --case gemv|gemm|quant|pack --shape q --m 1.
+    """One kernel on one shape (for profiling and sweeps): --case gemv|gemm|quant|pack --shape q --m 1,
+    or --case batch --layers L --m M.
 
     Distinct copies of the packed weights (--copies) are cycled so that the footprint exceeds L2."""
     from paper_2504_12285_b200 import binding as bl
 
     dev = torch.device("cuda", 0)
     torch.cuda.set_device(0)
+    if args.case == "batch":
+        return run_case_batch(args, bl, dev)
     n, k = wl.SHAPE_NK[args.shape]
     M = args.m
     peaks = load_peaks()
@@ -406,7 +436,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", choices=["gemv", "gemm", "quant", "pack"], default=None)
+    ap.add_argument("--case", choices=["gemv", "gemm", "quant", "pack", "batch"], default=None)
+    ap.add_argument("--layers", type=int, default=10)
     ap.add_argument("--shape", choices=list(wl.SHAPE_NK), default="q")
     ap.add_argument("--m", type=int, default=1)
     ap.add_argument("--copies", type=int, default=1)

@@ -212,9 +212,11 @@ int bitlinear_forward_batch_host(const bitlinear_problem* problems, int count, i
                                  void* x_dev, size_t x_bytes, const void* y_dev, void* y_host, size_t y_bytes,
                                  void* ws, size_t ws_bytes, void* stream);
 
-/* Reads and clears the sticky device-side status word of the current device: BITLINEAR_OK, or
- * BITLINEAR_ERR_TIMEOUT if a kernel gave up a bounded wait since the last poll.  Synchronises
- * `stream` first. */
+/* Reads and clears the sticky device-side status word of the current device: BITLINEAR_OK,
+ * BITLINEAR_ERR_TIMEOUT if a kernel gave up a bounded wait since the last poll, or
+ * BITLINEAR_ERR_WORKSPACE if a batch call with BITLINEAR_BATCH_REUSE_PLAN found that the plan in
+ * its workspace was no longer the one it had uploaded (the call then computed nothing).
+ * Synchronises `stream` first. */
 int bitlinear_poll_status(void* stream);
 
 #ifdef __cplusplus

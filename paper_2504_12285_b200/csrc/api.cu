@@ -244,7 +244,7 @@ int bitlinear_poll_status(void* stream) {
             cudaGetLastError();
             return BITLINEAR_ERR_CUDA;
         }
-        return BITLINEAR_ERR_TIMEOUT;
+        return host == BITLINEAR_ERR_WORKSPACE ? BITLINEAR_ERR_WORKSPACE : BITLINEAR_ERR_TIMEOUT;
     }
     return BITLINEAR_OK;
 }

@@ -38,23 +38,46 @@ struct DevProblem {
     int M, N, K, y_dtype;
     float eps;
     int k_tiles;
+    int rb_per_item;  // 16-row blocks per work item (the last item of a problem may hold fewer)
     int item_begin;  // index of this problem's first item in the global work list
     int row_begin;   // index of this problem's first token in the global token list
 };
 
+// First bytes of the uploaded plan.  The kernels compare it with the values the host passes at
+// launch, so a workspace that was overwritten between calls (with BITLINEAR_BATCH_REUSE_PLAN) is
+// detected and reported instead of being followed into stale pointers.
+struct PlanHeader {
+    unsigned magic;
+    int count, total_items, grid, rows;
+    int pad[3];
+};
+constexpr unsigned kPlanMagic = 0xB171A9E5u;
+
 namespace {
+
+__device__ __forceinline__ bool plan_matches(const PlanHeader* h, int count, int total_items, int grid, int rows) {
+    return h->magic == kPlanMagic && h->count == count && h->total_items == total_items && h->grid == grid &&
+           h->rows == rows;
+}
 
 constexpr int kConsumers = 10;
 constexpr int kStreamThreads = (kConsumers + 2) * 32;
 constexpr int kMaxStages = 16;            // ring slots; a slot holds one item (16 rows x K/4 bytes, K <= 8192)
-constexpr int kRedBufs = 4;
+constexpr int kRedBufs = 2;
+constexpr int kItemBytesCap = 32 * 1024;  // an item is as many 16-row blocks as fit in this many packed bytes
 constexpr int kBatchMaxK = 8192;
 
 // ------------------------------------------------------------------------------------ launch 1
 
 template <int VPT>
-__global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const DevProblem* __restrict__ probs, int count) {
+__global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHeader* __restrict__ hdr,
+                                                                    const DevProblem* __restrict__ probs, int count,
+                                                                    int total_items, int grid, int* status_word) {
     __shared__ RowReduceSmem sm;
+    if (!plan_matches(hdr, count, total_items, grid, (int)gridDim.x)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
+        return;
+    }
     const int row = blockIdx.x;
     int lo = 0, hi = count - 1;  // last problem whose row_begin <= row
     while (lo < hi) {
@@ -93,30 +116,110 @@ struct StreamParams {
     const DevProblem* probs;
     const int* item_begin;  // [count + 1]
     const int* cta_begin;   // [gridDim.x + 1]
-    int count;
+    const PlanHeader* hdr;
+    int count, total_items, rows;
     int stages;
+    int rb_max;       // largest rb_per_item of the batch
     int stage_bytes;  // size of a ring slot: the largest item of the batch, a multiple of 1024
     int* status_word;
 };
+
+// Compute the partial sums of one 16-row block for this warp's tiles and write them to `rbuf`
+// ([16 rows][MP tokens]).  NT = 0: one token, dp4a.  NT = 1 / 2: up to 8 / 16 tokens, mma.sync.
+template <int NT, int TPW>
+__device__ __forceinline__ void row_block_partials(const uint4 (&wv)[TPW][2],
+                                                   const uint32_t (&xr)[TPW][NT == 0 ? 1 : NT][16], int* rbuf, int g,
+                                                   int t) {
+    constexpr int MP = NT == 0 ? 1 : 8 * NT;
+    constexpr int XT = NT == 0 ? 1 : NT;
+    if constexpr (NT == 0) {
+        // accumulators per row and per bit position j hold 4^j x the true partial sum
+        int acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+#pragma unroll
+        for (int i = 0; i < TPW; ++i) {
+            const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
+            const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t mask = 0x03030303u << (2 * j);
+                    acc[0][j] = dp4a_u8_s8(w0[q] & mask, xr[i][0][4 * q + j], acc[0][j]);
+                    acc[1][j] = dp4a_u8_s8(w1[q] & mask, xr[i][0][4 * q + j], acc[1][j]);
+                }
+        }
+        int v0 = acc[0][0] + (acc[0][1] >> 2) + (acc[0][2] >> 4) + (acc[0][3] >> 6);
+        int v1 = acc[1][0] + (acc[1][1] >> 2) + (acc[1][2] >> 4) + (acc[1][3] >> 6);
+        v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
+        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
+        v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
+        v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
+        if (t == 0) {
+            rbuf[g] = v0;
+            rbuf[8 + g] = v1;
+        }
+    } else {
+        int acc[4][XT][4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+#pragma unroll
+            for (int nt = 0; nt < XT; ++nt)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) acc[j][nt][r] = 0;
+#pragma unroll
+        for (int i = 0; i < TPW; ++i) {
+            const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
+            const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
+#pragma unroll
+            for (int q2 = 0; q2 < 2; ++q2)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t mask = 0x03030303u << (2 * j);
+                    const int qa = 2 * q2, qb = 2 * q2 + 1;
+                    const uint32_t a0 = w0[qa] & mask, a1 = w1[qa] & mask, a2 = w0[qb] & mask, a3 = w1[qb] & mask;
+#pragma unroll
+                    for (int nt = 0; nt < XT; ++nt)
+                        mma_u8s8(acc[j][nt], a0, a1, a2, a3, xr[i][nt][4 * qa + j], xr[i][nt][4 * qb + j]);
+                }
+        }
+#pragma unroll
+        for (int nt = 0; nt < XT; ++nt) {
+            int v[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                v[r] = acc[0][nt][r] + (acc[1][nt][r] >> 2) + (acc[2][nt][r] >> 4) + (acc[3][nt][r] >> 6);
+            // fragment layout: r0 (row g, token 2t), r1 (g, 2t+1), r2 (g+8, 2t), r3 (g+8, 2t+1)
+            const int tok = 8 * nt + 2 * t;
+            *reinterpret_cast<int2*>(rbuf + g * MP + tok) = make_int2(v[0], v[1]);
+            *reinterpret_cast<int2*>(rbuf + (g + 8) * MP + tok) = make_int2(v[2], v[3]);
+        }
+    }
+}
 
 // NT = 0: one token, dp4a.  NT = 1 / 2: up to 8 / 16 tokens, mma.sync with NT token tiles.
 template <int NT, int TPW>
 __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const StreamParams prm) {
     constexpr int MP = NT == 0 ? 1 : 8 * NT;  // padded token count of the partial-sum buffers
     constexpr int XT = NT == 0 ? 1 : NT;
+    constexpr int RB_INTS = kConsumers * 16 * MP;  // partial sums of one row block
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int stages = prm.stages;
-    const int kStageBytes = prm.stage_bytes;
-    int* red = reinterpret_cast<int*>(smem + (size_t)stages * kStageBytes);  // [kRedBufs][kConsumers][16][MP]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(red + kRedBufs * kConsumers * 16 * MP);
+    const int stage_bytes = prm.stage_bytes;
+    int* red = reinterpret_cast<int*>(smem + (size_t)stages * stage_bytes);  // [kRedBufs][rb_max][kConsumers][16][MP]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(red + kRedBufs * prm.rb_max * RB_INTS);
     uint64_t* full_bar = bars;                       // [stages]  bytes of the item landed
-    uint64_t* empty_bar = bars + kMaxStages;         // [stages]  all consumers have the item in registers
+    uint64_t* empty_bar = bars + kMaxStages;         // [stages]  all consumers are done reading the item
     uint64_t* redfull_bar = bars + 2 * kMaxStages;   // [kRedBufs] all consumers wrote their partial sums
     uint64_t* redfree_bar = redfull_bar + kRedBufs;  // [kRedBufs] the epilogue is done with the buffer
     volatile int* abort_flag = reinterpret_cast<volatile int*>(redfree_bar + kRedBufs);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (!plan_matches(prm.hdr, prm.count, prm.total_items, (int)gridDim.x, prm.rows)) {  // uniform over the grid
+        if (blockIdx.x == 0 && threadIdx.x == 0 && prm.status_word != nullptr)
+            atomicExch(prm.status_word, BITLINEAR_ERR_WORKSPACE);
+        return;
+    }
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
             mbar_init(smem_u32(full_bar + s), 1);
@@ -147,23 +250,30 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
         if (lane == 0) {
-            int next_begin = prm.item_begin[p + 1];
-            const uint8_t* base = reinterpret_cast<const uint8_t*>(prm.probs[p].packed);
-            uint32_t bytes = (uint32_t)prm.probs[p].k_tiles * kTileBytes;
-            int first = prm.item_begin[p];
+            int next_begin = prm.item_begin[p];  // forces the first refresh
+            const uint8_t* base = nullptr;
+            int first = 0, rbpi = 1, n_rb = 0;
+            uint32_t rb_bytes = 0;
+            --p;
             uint32_t stage = 0, phase = 0;
             for (int it = item_lo; it < item_hi; ++it) {
                 while (it >= next_begin) {
                     ++p;
                     next_begin = prm.item_begin[p + 1];
-                    base = reinterpret_cast<const uint8_t*>(prm.probs[p].packed);
-                    bytes = (uint32_t)prm.probs[p].k_tiles * kTileBytes;
-                    first = prm.item_begin[p];
+                    const DevProblem& pr = prm.probs[p];
+                    base = reinterpret_cast<const uint8_t*>(pr.packed);
+                    rb_bytes = (uint32_t)pr.k_tiles * kTileBytes;
+                    first = pr.item_begin;
+                    rbpi = pr.rb_per_item;
+                    n_rb = pr.N / kTileRows;
                 }
+                const int rb0 = (it - first) * rbpi;
+                const int nrb = (n_rb - rb0) < rbpi ? (n_rb - rb0) : rbpi;
+                const uint32_t bytes = (uint32_t)nrb * rb_bytes;
                 if (!mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag)) break;
                 const uint32_t fb = smem_u32(full_bar + stage);
                 mbar_expect_tx(fb, bytes);
-                bulk_load(smem_u32(smem + (size_t)stage * kStageBytes), base + (size_t)(it - first) * bytes, bytes, fb);
+                bulk_load(smem_u32(smem + (size_t)stage * stage_bytes), base + (size_t)rb0 * rb_bytes, bytes, fb);
                 if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
             }
         }
@@ -172,17 +282,22 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         // ---------------------------------------------------------------- consumers
         const int w = warp - 1;
         const int g = lane >> 2, t = lane & 3;
-        int cur = -1, next_begin = 0, k_tiles = 0;
+        int next_begin = prm.item_begin[p], k_tiles = 0, first = 0, rbpi = 1, n_rb = 0;
+        --p;
         uint32_t xr[TPW][XT][16];  // this lane's activation bytes: tile, token tile, 16 words = 64 columns
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
-            if (cur < 0 || it >= next_begin) {
-                if (cur >= 0) { while (it >= prm.item_begin[p + 1]) ++p; }
-                cur = p;
-                next_begin = prm.item_begin[p + 1];
+            if (it >= next_begin) {
+                while (it >= next_begin) {
+                    ++p;
+                    next_begin = prm.item_begin[p + 1];
+                }
                 const DevProblem& pr = prm.probs[p];
                 k_tiles = pr.k_tiles;
+                first = pr.item_begin;
+                rbpi = pr.rb_per_item;
+                n_rb = pr.N / kTileRows;
 #pragma unroll
                 for (int i = 0; i < TPW; ++i) {
                     const int kt = w + i * kConsumers;
@@ -206,124 +321,73 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                 }
             }
             const int c = it - item_lo;
+            const int rb0 = (it - first) * rbpi;
+            const int nrb = (n_rb - rb0) < rbpi ? (n_rb - rb0) : rbpi;
             if (!mbar_wait(smem_u32(full_bar + stage), phase, abort_flag)) { ok = false; break; }
-            const uint32_t sbase = smem_u32(smem + (size_t)stage * kStageBytes) + lane * 16;
-            uint4 wv[TPW][2];
-#pragma unroll
-            for (int i = 0; i < TPW; ++i) {
-                const int kt = w + i * kConsumers;
-                if (kt < k_tiles) {
-                    wv[i][0] = lds128(sbase + kt * kTileBytes);
-                    wv[i][1] = lds128(sbase + kt * kTileBytes + 512);
-                } else {
-                    wv[i][0] = make_uint4(0, 0, 0, 0);
-                    wv[i][1] = make_uint4(0, 0, 0, 0);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(empty_bar + stage));
-            if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
-
-            int* rbuf = red + ((c % kRedBufs) * kConsumers + w) * 16 * MP;
             const uint32_t rphase = (uint32_t)(c / kRedBufs) & 1u;
-            if constexpr (NT == 0) {
-                // accumulators per row and per bit position j hold 4^j x the true partial sum
-                int acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+            if (!mbar_wait(smem_u32(redfree_bar + c % kRedBufs), rphase ^ 1u, abort_flag)) { ok = false; break; }
+            const uint32_t sbase = smem_u32(smem + (size_t)stage * stage_bytes) + lane * 16;
+            int* rbase = red + (c % kRedBufs) * prm.rb_max * RB_INTS + w * 16 * MP;
+            for (int r = 0; r < nrb; ++r) {
+                uint4 wv[TPW][2];
 #pragma unroll
                 for (int i = 0; i < TPW; ++i) {
-                    const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
-                    const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q)
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t mask = 0x03030303u << (2 * j);
-                            acc[0][j] = dp4a_u8_s8(w0[q] & mask, xr[i][0][4 * q + j], acc[0][j]);
-                            acc[1][j] = dp4a_u8_s8(w1[q] & mask, xr[i][0][4 * q + j], acc[1][j]);
-                        }
+                    const int kt = w + i * kConsumers;
+                    if (kt < k_tiles) {
+                        wv[i][0] = lds128(sbase + (r * k_tiles + kt) * kTileBytes);
+                        wv[i][1] = lds128(sbase + (r * k_tiles + kt) * kTileBytes + 512);
+                    } else {
+                        wv[i][0] = make_uint4(0, 0, 0, 0);
+                        wv[i][1] = make_uint4(0, 0, 0, 0);
+                    }
                 }
-                int v0 = acc[0][0] + (acc[0][1] >> 2) + (acc[0][2] >> 4) + (acc[0][3] >> 6);
-                int v1 = acc[1][0] + (acc[1][1] >> 2) + (acc[1][2] >> 4) + (acc[1][3] >> 6);
-                v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
-                v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-                v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
-                v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
-                if (!mbar_wait(smem_u32(redfree_bar + c % kRedBufs), rphase ^ 1u, abort_flag)) { ok = false; break; }
-                if (t == 0) {
-                    rbuf[g] = v0;
-                    rbuf[8 + g] = v1;
-                }
-            } else {
-                int acc[4][XT][4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-#pragma unroll
-                    for (int nt = 0; nt < XT; ++nt)
-#pragma unroll
-                        for (int r = 0; r < 4; ++r) acc[j][nt][r] = 0;
-#pragma unroll
-                for (int i = 0; i < TPW; ++i) {
-                    const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
-                    const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
-#pragma unroll
-                    for (int q2 = 0; q2 < 2; ++q2)
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t mask = 0x03030303u << (2 * j);
-                            const int qa = 2 * q2, qb = 2 * q2 + 1;
-                            const uint32_t a0 = w0[qa] & mask, a1 = w1[qa] & mask, a2 = w0[qb] & mask, a3 = w1[qb] & mask;
-#pragma unroll
-                            for (int nt = 0; nt < XT; ++nt)
-                                mma_u8s8(acc[j][nt], a0, a1, a2, a3, xr[i][nt][4 * qa + j], xr[i][nt][4 * qb + j]);
-                        }
-                }
-                if (!mbar_wait(smem_u32(redfree_bar + c % kRedBufs), rphase ^ 1u, abort_flag)) { ok = false; break; }
-#pragma unroll
-                for (int nt = 0; nt < XT; ++nt) {
-                    int v[4];
-#pragma unroll
-                    for (int r = 0; r < 4; ++r)
-                        v[r] = acc[0][nt][r] + (acc[1][nt][r] >> 2) + (acc[2][nt][r] >> 4) + (acc[3][nt][r] >> 6);
-                    // fragment layout: r0 (row g, token 2t), r1 (g, 2t+1), r2 (g+8, 2t), r3 (g+8, 2t+1)
-                    const int tok = 8 * nt + 2 * t;
-                    *reinterpret_cast<int2*>(rbuf + g * MP + tok) = make_int2(v[0], v[1]);
-                    *reinterpret_cast<int2*>(rbuf + (g + 8) * MP + tok) = make_int2(v[2], v[3]);
-                }
+                row_block_partials<NT, TPW>(wv, xr, rbase + r * RB_INTS, g, t);
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(redfull_bar + c % kRedBufs));
+            if (lane == 0) {
+                mbar_arrive(smem_u32(empty_bar + stage));
+                mbar_arrive(smem_u32(redfull_bar + c % kRedBufs));
+            }
+            if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
         }
     } else {
         // ---------------------------------------------------------------- epilogue
-        int cur = -1, next_begin = 0, first = 0, active = 0, M = 0, N = 0, y_dtype = 0;
+        int next_begin = prm.item_begin[p], first = 0, active = 0, M = 0, N = 0, y_dtype = 0, rbpi = 1, n_rb = 0;
+        --p;
         float s_w = 0.0f;
         void* y = nullptr;
         const float* dptr = nullptr;
         const int32_t* xsptr = nullptr;
         for (int it = item_lo; it < item_hi; ++it) {
-            if (cur < 0 || it >= next_begin) {
-                if (cur >= 0) { while (it >= prm.item_begin[p + 1]) ++p; }
-                cur = p;
-                next_begin = prm.item_begin[p + 1];
+            if (it >= next_begin) {
+                while (it >= next_begin) {
+                    ++p;
+                    next_begin = prm.item_begin[p + 1];
+                }
                 const DevProblem& pr = prm.probs[p];
                 first = pr.item_begin;
                 active = pr.k_tiles < kConsumers ? pr.k_tiles : kConsumers;
                 M = pr.M; N = pr.N; y_dtype = pr.y_dtype;
+                rbpi = pr.rb_per_item;
+                n_rb = pr.N / kTileRows;
                 s_w = *pr.s_w;
                 y = pr.y; dptr = pr.d; xsptr = pr.xsum;
             }
             const int c = it - item_lo;
+            const int rb0 = (it - first) * rbpi;
+            const int nrb = (n_rb - rb0) < rbpi ? (n_rb - rb0) : rbpi;
             const uint32_t rphase = (uint32_t)(c / kRedBufs) & 1u;
             if (!mbar_wait(smem_u32(redfull_bar + c % kRedBufs), rphase, abort_flag)) break;
-            const int* rb = red + (c % kRedBufs) * kConsumers * 16 * MP;
-            const int n0 = (it - first) * kTileRows;
-            for (int o = lane; o < 16 * M; o += 32) {
-                const int m = o >> 4, r = o & 15;
+            const int* rb = red + (c % kRedBufs) * prm.rb_max * RB_INTS;
+            const int rows = nrb * 16;
+            for (int o = lane; o < rows * M; o += 32) {
+                const int m = o / rows, rr = o - m * rows;  // consecutive lanes -> consecutive output rows
+                const int r = rr >> 4, row = rr & 15;
                 int total = 0;
-                for (int w = 0; w < active; ++w) total += rb[(w * 16 + r) * MP + m];
+                for (int w = 0; w < active; ++w) total += rb[r * RB_INTS + (w * 16 + row) * MP + m];
                 total -= xsptr[m];
                 const float val = __fmul_rn(__fmul_rn((float)total, s_w), dptr[m]);
-                const size_t idx = (size_t)m * N + n0 + r;
+                const size_t idx = (size_t)m * N + (size_t)rb0 * kTileRows + rr;
                 if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
                 else reinterpret_cast<float*>(y)[idx] = val;
             }
@@ -364,7 +428,7 @@ struct PlanLayout {
 
 PlanLayout plan_layout(int count, int grid, size_t xq_bytes, size_t rows) {
     PlanLayout L;
-    size_t off = 0;
+    size_t off = 256;  // the PlanHeader sits at offset 0
     L.probs_off = off;
     off = align_up(off + (size_t)count * sizeof(DevProblem), 256);
     L.item_off = off;
@@ -444,6 +508,7 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     char* base = static_cast<char*>(ws);
 
     // ---- host plan: device descriptors, item prefix, byte-balanced CTA ranges ----
+    int rb_max = 1, stage_bytes = 0;
     std::vector<DevProblem> dp;
     std::vector<int> item_begin;
     dp.reserve(count);
@@ -468,11 +533,20 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
             v.M = q.M; v.N = q.N; v.K = q.K; v.y_dtype = q.y_dtype;
             v.eps = q.rms_eps;
             v.k_tiles = q.K / kTileCols;
+            {
+                int rb = kItemBytesCap / (v.k_tiles * kTileBytes);
+                const int rb_cap = max_m <= 8 ? 4 : 2;  // bounds the partial-sum buffers
+                if (rb > rb_cap) rb = rb_cap;
+                if (rb < 1) rb = 1;
+                v.rb_per_item = rb;
+                if (rb > rb_max) rb_max = rb;
+                if (rb * v.k_tiles * kTileBytes > stage_bytes) stage_bytes = rb * v.k_tiles * kTileBytes;
+            }
             v.item_begin = items;
             v.row_begin = row;
             dp.push_back(v);
             item_begin.push_back(items);
-            items += q.N / kTileRows;
+            items += (q.N / kTileRows + v.rb_per_item - 1) / v.rb_per_item;
             row += q.M;
             xq_ptr += align_up((size_t)q.M * q.K, 16);
         }
@@ -484,17 +558,18 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     std::vector<int> cta_begin(grid + 1);
     {
         double total_bytes = 0.0;
-        for (int i = 0; i < n_prob; ++i) total_bytes += (double)(item_begin[i + 1] - item_begin[i]) * dp[i].k_tiles;
+        for (int i = 0; i < n_prob; ++i) total_bytes += (double)(item_begin[i + 1] - item_begin[i]) * dp[i].k_tiles * dp[i].rb_per_item;
         int pi = 0;
         double before = 0.0;  // tile-KB before problem pi
         cta_begin[0] = 0;
         for (int c = 1; c < grid; ++c) {
             const double target = total_bytes * c / grid;
-            while (pi < n_prob - 1 && before + (double)(item_begin[pi + 1] - item_begin[pi]) * dp[pi].k_tiles <= target) {
-                before += (double)(item_begin[pi + 1] - item_begin[pi]) * dp[pi].k_tiles;
+            while (pi < n_prob - 1 &&
+                   before + (double)(item_begin[pi + 1] - item_begin[pi]) * dp[pi].k_tiles * dp[pi].rb_per_item <= target) {
+                before += (double)(item_begin[pi + 1] - item_begin[pi]) * dp[pi].k_tiles * dp[pi].rb_per_item;
                 ++pi;
             }
-            int it = item_begin[pi] + (int)((target - before) / dp[pi].k_tiles + 0.5);
+            int it = item_begin[pi] + (int)((target - before) / ((double)dp[pi].k_tiles * dp[pi].rb_per_item) + 0.5);
             if (it > item_begin[pi + 1]) it = item_begin[pi + 1];
             if (it < cta_begin[c - 1]) it = cta_begin[c - 1];
             cta_begin[c] = it;
@@ -502,8 +577,16 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
         cta_begin[grid] = total_items;
     }
 
+    PlanHeader hdr_host;
+    hdr_host.magic = kPlanMagic;
+    hdr_host.count = n_prob;
+    hdr_host.total_items = total_items;
+    hdr_host.grid = grid;
+    hdr_host.rows = (int)rows;
+    hdr_host.pad[0] = hdr_host.pad[1] = hdr_host.pad[2] = 0;
     if (!(flags & BITLINEAR_BATCH_REUSE_PLAN)) {
-        if (cudaMemcpyAsync(base + L.probs_off, dp.data(), dp.size() * sizeof(DevProblem), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        if (cudaMemcpyAsync(base, &hdr_host, sizeof(hdr_host), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(base + L.probs_off, dp.data(), dp.size() * sizeof(DevProblem), cudaMemcpyHostToDevice, st) != cudaSuccess ||
             cudaMemcpyAsync(base + L.item_off, item_begin.data(), item_begin.size() * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess ||
             cudaMemcpyAsync(base + L.cta_off, cta_begin.data(), cta_begin.size() * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess) {
             cudaGetLastError();
@@ -516,9 +599,11 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     if (!(flags & BITLINEAR_BATCH_REUSE_ACT)) {
         const int vpt = (max_k / 8 + kQuantThreads - 1) / kQuantThreads;
         const dim3 g((unsigned)rows), b(kQuantThreads);
-        if (vpt <= 1) batch_quant_kernel<1><<<g, b, 0, st>>>(probs_dev, n_prob);
-        else if (vpt <= 2) batch_quant_kernel<2><<<g, b, 0, st>>>(probs_dev, n_prob);
-        else batch_quant_kernel<4><<<g, b, 0, st>>>(probs_dev, n_prob);
+        const PlanHeader* h = reinterpret_cast<const PlanHeader*>(base);
+        int* sw = device_status_word();
+        if (vpt <= 1) batch_quant_kernel<1><<<g, b, 0, st>>>(h, probs_dev, n_prob, total_items, grid, sw);
+        else if (vpt <= 2) batch_quant_kernel<2><<<g, b, 0, st>>>(h, probs_dev, n_prob, total_items, grid, sw);
+        else batch_quant_kernel<4><<<g, b, 0, st>>>(h, probs_dev, n_prob, total_items, grid, sw);
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
 
@@ -527,17 +612,21 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     prm.probs = probs_dev;
     prm.item_begin = reinterpret_cast<const int*>(base + L.item_off);
     prm.cta_begin = reinterpret_cast<const int*>(base + L.cta_off);
+    prm.hdr = reinterpret_cast<const PlanHeader*>(base);
     prm.count = n_prob;
+    prm.total_items = total_items;
+    prm.rows = (int)rows;
     prm.status_word = device_status_word();
     const int nt = max_m <= 1 ? 0 : (max_m <= 8 ? 1 : 2);
     const int mp = nt == 0 ? 1 : 8 * nt;
     const int tpw = (max_ktiles + kConsumers - 1) / kConsumers;  // <= 4 since K <= 8192
-    const size_t fixed = 1024 + (size_t)kRedBufs * kConsumers * 16 * mp * sizeof(int) + (2 * kMaxStages + 2 * kRedBufs) * 8 + 64;
-    const int stage_bytes = max_ktiles * kTileBytes;
+    const size_t fixed = 1024 + (size_t)kRedBufs * rb_max * kConsumers * 16 * mp * sizeof(int) +
+                         (2 * kMaxStages + 2 * kRedBufs) * 8 + 64;
     int stages = (int)((227 * 1024 - fixed) / stage_bytes);
     if (stages > kMaxStages) stages = kMaxStages;
     prm.stages = stages;
     prm.stage_bytes = stage_bytes;
+    prm.rb_max = rb_max;
     const size_t smem = fixed + (size_t)stages * stage_bytes;
     cudaError_t e;
     if (nt == 0) e = launch_stream_nt<0>(tpw, prm, grid, smem, st);

@@ -107,3 +107,24 @@ def test_batch_matches_single_forward_bitwise():
     for x, g, packed, s_w, y in batch.tensors:
         y1 = bl.bitlinear_forward(x, g, packed, s_w, y.shape[1], wl.RMS_EPS)
         assert torch.equal(y, y1)
+
+
+def test_batch_detects_an_overwritten_plan():
+    # REUSE_PLAN trusts the workspace; if something else wrote over it, the kernels must notice and
+    # compute nothing instead of following stale pointers
+    batch, refs = make_case([(1, 48, 768), (2, 32, 256)], 600)
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    bl.bitlinear_forward_batch(batch, ws)
+    torch.cuda.synchronize()
+    check(batch, refs)
+    ws[:256].zero_()
+    for t in batch.tensors:
+        t[4].fill_(7.0)
+    bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
+    assert bl.bitlinear_poll_status() == 4  # workspace error, reported through the sticky status word
+    for t in batch.tensors:
+        assert torch.all(t[4] == 7.0)
+    assert bl.bitlinear_poll_status() == 0
+    bl.bitlinear_forward_batch(batch, ws)  # a fresh upload repairs it
+    torch.cuda.synchronize()
+    check(batch, refs)
