@@ -128,8 +128,8 @@ struct StreamParams {
 // ([16 rows][MP tokens]).  NT = 0: one token, dp4a.  NT = 1 / 2: up to 8 / 16 tokens, mma.sync.
 template <int NT, int TPW>
 __device__ __forceinline__ void row_block_partials(const uint4 (&wv)[TPW][2],
-                                                   const uint32_t (&xr)[TPW][NT == 0 ? 1 : NT][16], int* rbuf, int g,
-                                                   int t) {
+                                                   const uint32_t (&xr)[TPW][NT == 0 ? 1 : NT][16], int n_act,
+                                                   int* rbuf, int g, int t) {
     constexpr int MP = NT == 0 ? 1 : 8 * NT;
     constexpr int XT = NT == 0 ? 1 : NT;
     if constexpr (NT == 0) {
@@ -137,6 +137,7 @@ __device__ __forceinline__ void row_block_partials(const uint4 (&wv)[TPW][2],
         int acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
 #pragma unroll
         for (int i = 0; i < TPW; ++i) {
+            if (i >= n_act) break;  // warp-uniform: this warp owns n_act tiles of the row block
             const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
             const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
 #pragma unroll
@@ -168,6 +169,7 @@ __device__ __forceinline__ void row_block_partials(const uint4 (&wv)[TPW][2],
                 for (int r = 0; r < 4; ++r) acc[j][nt][r] = 0;
 #pragma unroll
         for (int i = 0; i < TPW; ++i) {
+            if (i >= n_act) break;  // warp-uniform
             const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
             const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
 #pragma unroll
@@ -282,7 +284,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         // ---------------------------------------------------------------- consumers
         const int w = warp - 1;
         const int g = lane >> 2, t = lane & 3;
-        int next_begin = prm.item_begin[p], k_tiles = 0, first = 0, rbpi = 1, n_rb = 0;
+        int next_begin = prm.item_begin[p], k_tiles = 0, first = 0, rbpi = 1, n_rb = 0, n_act = 0;
         --p;
         uint32_t xr[TPW][XT][16];  // this lane's activation bytes: tile, token tile, 16 words = 64 columns
         uint32_t stage = 0, phase = 0;
@@ -298,6 +300,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                 first = pr.item_begin;
                 rbpi = pr.rb_per_item;
                 n_rb = pr.N / kTileRows;
+                n_act = w < k_tiles ? (k_tiles - w + kConsumers - 1) / kConsumers : 0;  // tiles w, w+10, ... < k_tiles
 #pragma unroll
                 for (int i = 0; i < TPW; ++i) {
                     const int kt = w + i * kConsumers;
@@ -333,15 +336,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
 #pragma unroll
                 for (int i = 0; i < TPW; ++i) {
                     const int kt = w + i * kConsumers;
-                    if (kt < k_tiles) {
+                    if (i < n_act) {
                         wv[i][0] = lds128(sbase + (r * k_tiles + kt) * kTileBytes);
                         wv[i][1] = lds128(sbase + (r * k_tiles + kt) * kTileBytes + 512);
-                    } else {
-                        wv[i][0] = make_uint4(0, 0, 0, 0);
-                        wv[i][1] = make_uint4(0, 0, 0, 0);
                     }
                 }
-                row_block_partials<NT, TPW>(wv, xr, rbase + r * RB_INTS, g, t);
+                row_block_partials<NT, TPW>(wv, xr, n_act, rbase + r * RB_INTS, g, t);
             }
             __syncwarp();
             if (lane == 0) {
@@ -356,8 +356,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         --p;
         float s_w = 0.0f;
         void* y = nullptr;
-        const float* dptr = nullptr;
-        const int32_t* xsptr = nullptr;
+        int xs_lane = 0;       // lane m holds the code sum and the scale of token m of the current problem
+        float d_lane = 0.0f;
         for (int it = item_lo; it < item_hi; ++it) {
             if (it >= next_begin) {
                 while (it >= next_begin) {
@@ -371,7 +371,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                 rbpi = pr.rb_per_item;
                 n_rb = pr.N / kTileRows;
                 s_w = *pr.s_w;
-                y = pr.y; dptr = pr.d; xsptr = pr.xsum;
+                y = pr.y;
+                xs_lane = lane < M ? pr.xsum[lane] : 0;
+                d_lane = lane < M ? pr.d[lane] : 0.0f;
             }
             const int c = it - item_lo;
             const int rb0 = (it - first) * rbpi;
@@ -380,16 +382,19 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             if (!mbar_wait(smem_u32(redfull_bar + c % kRedBufs), rphase, abort_flag)) break;
             const int* rb = red + (c % kRedBufs) * prm.rb_max * RB_INTS;
             const int rows = nrb * 16;
-            for (int o = lane; o < rows * M; o += 32) {
-                const int m = o / rows, rr = o - m * rows;  // consecutive lanes -> consecutive output rows
-                const int r = rr >> 4, row = rr & 15;
-                int total = 0;
-                for (int w = 0; w < active; ++w) total += rb[r * RB_INTS + (w * 16 + row) * MP + m];
-                total -= xsptr[m];
-                const float val = __fmul_rn(__fmul_rn((float)total, s_w), dptr[m]);
-                const size_t idx = (size_t)m * N + (size_t)rb0 * kTileRows + rr;
-                if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
-                else reinterpret_cast<float*>(y)[idx] = val;
+            for (int m = 0; m < M; ++m) {
+                const int xs = __shfl_sync(0xffffffffu, xs_lane, m);
+                const float dm = __shfl_sync(0xffffffffu, d_lane, m);
+                for (int rr = lane; rr < rows; rr += 32) {  // consecutive lanes -> consecutive output rows
+                    const int r = rr >> 4, row = rr & 15;
+                    int total = 0;
+                    for (int w = 0; w < active; ++w) total += rb[r * RB_INTS + (w * 16 + row) * MP + m];
+                    total -= xs;
+                    const float val = __fmul_rn(__fmul_rn((float)total, s_w), dm);
+                    const size_t idx = (size_t)m * N + (size_t)rb0 * kTileRows + rr;
+                    if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
+                    else reinterpret_cast<float*>(y)[idx] = val;
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(redfree_bar + c % kRedBufs));
