@@ -212,6 +212,32 @@ int bitlinear_forward_batch_host(const bitlinear_problem* problems, int count, i
                                  void* x_dev, size_t x_bytes, const void* y_dev, void* y_host, size_t y_bytes,
                                  void* ws, size_t ws_bytes, void* stream);
 
+/*
+ * bitlinear_forward for decode-sized calls by code that cannot allocate device memory.
+ * (No counterpart in the paper: this is a convenience of the library.)
+ *
+ * Who needs it: an operator plug-in that receives only its input and output buffers, code that
+ * runs after a framework's pool has claimed the whole device, a serving loop whose steady state
+ * must not touch an allocator.  Such callers cannot provide the workspace bitlinear_forward asks
+ * for, and the library itself never calls cudaMalloc.  Here the workspace is a fixed array inside
+ * the library image instead: bitlinear_static_scratch_bytes() bytes (262,656) that every GPU which
+ * loads the library holds until the process exits.  The call allocates and frees nothing.
+ *
+ *   Arguments as bitlinear_forward, without ws.  Limits: M <= BITLINEAR_STATIC_MAX_TOKENS and
+ *   K <= BITLINEAR_STATIC_MAX_K; anything larger returns BITLINEAR_ERR_WORKSPACE before a launch.
+ *   The result is the same as bitlinear_forward's for the same arguments (same kernels).
+ *   The first call on each device looks up the array's device address (with that device current)
+ *   and caches it; make that first call outside any stream capture.
+ *   All calls on a device share the one array.  Each call rewrites every element it later reads,
+ *   so leftovers of earlier calls are harmless, but two calls that overlap on the GPU (different
+ *   streams, no ordering between them) race on it: serialise them.
+ */
+#define BITLINEAR_STATIC_MAX_TOKENS 16
+#define BITLINEAR_STATIC_MAX_K 16384
+size_t bitlinear_static_scratch_bytes(void);
+int bitlinear_forward_static(const void* x_bf16, const void* gain, float rms_eps, const void* packed,
+                             const float* s_w, int M, int N, int K, void* y_out, int y_dtype, void* stream);
+
 /* Reads and clears the sticky device-side status word of the current device: BITLINEAR_OK,
  * BITLINEAR_ERR_TIMEOUT if a kernel gave up a bounded wait since the last poll, or
  * BITLINEAR_ERR_WORKSPACE if a batch call with BITLINEAR_BATCH_REUSE_PLAN found that the plan in

@@ -41,6 +41,9 @@ _SIGNATURES = {
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
+    "bitlinear_static_scratch_bytes": (_c_size_t, []),
+    "bitlinear_forward_static": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
+                                          _c_void_p, _c_int, _c_void_p]),
     "bitlinear_batch_workspace_bytes": (_c_size_t, [_c_void_p, _c_int]),
     "bitlinear_forward_batch": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_forward_batch_host": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p,
@@ -226,6 +229,27 @@ def bitlinear_forward_host(x_host, gain, packed, s_w, N: int, y_host, rms_eps: f
                                       _ptr(y_host), _ydt(y_host.dtype), _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_forward_host")
     return y_host
+
+
+def bitlinear_static_scratch_bytes() -> int:
+    return int(lib().bitlinear_static_scratch_bytes())
+
+
+def bitlinear_forward_static(x, gain, packed, s_w, N: int, rms_eps: float = 1e-5, y_dtype=torch.float32,
+                             out: torch.Tensor | None = None) -> torch.Tensor:
+    """Decode-sized forward (M <= 16) that takes no workspace: for callers that cannot allocate device
+    memory, the scratch is a fixed array inside the library.  Calls on one device must not overlap."""
+    _dev(x, torch.bfloat16, "x")
+    if gain is not None:
+        _dev(gain, torch.bfloat16, "gain")
+    _dev(packed, torch.uint8, "packed")
+    _dev(s_w, torch.float32, "s_w")
+    M, K = x.shape
+    y = out if out is not None else torch.empty(M, N, dtype=y_dtype, device=x.device)
+    rc = lib().bitlinear_forward_static(_ptr(x), _ptr(gain), rms_eps, _ptr(packed), _ptr(s_w), M, N, K, _ptr(y),
+                                        _ydt(y.dtype), _stream())
+    _check(rc, "bitlinear_forward_static")
+    return y
 
 
 class ProblemBatch:
