@@ -4,21 +4,23 @@
 // whole batch of matmuls are streamed back to back by one persistent kernel.)
 //
 //   launch 1  batch_quant_kernel : one CTA per token of every problem - fused RMSNorm + absmax
-//             int8 quantiser into the workspace.
-//   launch 2  decode_stream_kernel : one persistent CTA per SM.  The work list is every block of
-//             16 weight rows of every problem ("item": 16 x K/4 contiguous packed bytes); each CTA
-//             owns a contiguous, byte-balanced range of it.
-//               warp 0      producer : one thread issues a linear bulk copy per item into a ring of
-//                                      shared-memory stages (mbarrier completion)
-//               warps 1-10  consumers: warp w owns the 16x256 tiles w, w+10, ... of every item; its
-//                                      slice of the quantised activations stays in registers for
-//                                      the whole problem.  M = 1: dot-product-of-four accumulation;
-//                                      M > 1: legacy mma.sync m16n8k32 (u8 codes x s8 activations),
-//                                      weights are the 16-row operand, tokens the 8-wide one.
-//               warp 11     epilogue : folds the consumers' partial sums, subtracts the code offset,
-//                                      applies the two scales and stores y.
-//             Stages, partial-sum buffers and activations hand over through mbarriers only, so the
-//             copy engine keeps streaming while consumers and epilogue work on earlier items.
+//             int8 quantiser into the workspace (codes stored in the lane-interleaved order the
+//             stream kernel reads, see quant_row).
+//   launch 2  decode_stream_kernel : one persistent CTA of 16 warps per SM.  The work list is every
+//             block of 16 weight rows of every problem; each CTA owns a contiguous, byte-balanced
+//             range of it.  A row block belongs to ONE group of G warps (G = 1 for up to four tokens;
+//             each warp of a group takes up to four tokens), so 16/G row blocks are in progress per
+//             CTA and no partial sum ever crosses a warp.  Each warp runs its own pipeline: lane 0
+//             issues a linear bulk copy (cp.async.bulk, a few contiguous 16x256 tiles) into one of
+//             the warp's two shared-memory slots and the warp waits on that slot's mbarrier,
+//             multiplies, and refills the slot it has just read - across row-block and matrix
+//             boundaries, so HBM requests are always in flight (16 issuing threads, ~80 KiB in flight
+//             per SM).  Nothing is handed from warp to warp.
+//             Before the stream starts the CTA copies the descriptors of the few problems its range
+//             touches, and their quantised activations, into shared memory once.
+//             Unpack: word & (0x03030303 << 2j) is 4^j x the codes of four consecutive columns, fed
+//             to a dot-product-of-four with the int8 activations; one accumulator per j keeps the
+//             scale uniform and the four are folded once per row block.
 #include <vector>
 
 #include "quant_row.cuh"
@@ -27,7 +29,7 @@
 namespace bitlinear {
 
 struct DevProblem {
-    const uint32_t* packed;
+    const uint8_t* packed;
     const float* s_w;
     void* y;
     const __nv_bfloat16* x;
@@ -38,9 +40,9 @@ struct DevProblem {
     int M, N, K, y_dtype;
     float eps;
     int k_tiles;
-    int rb_per_item;  // 16-row blocks per work item (the last item of a problem may hold fewer)
-    int item_begin;  // index of this problem's first item in the global work list
-    int row_begin;   // index of this problem's first token in the global token list
+    int rb_begin;   // index of this problem's first row block in the global row-block list
+    int rb_end;     // one past its last
+    int row_begin;  // index of its first token in the global token list
 };
 
 // First bytes of the uploaded plan.  The kernels compare it with the values the host passes at
@@ -48,46 +50,41 @@ struct DevProblem {
 // detected and reported instead of being followed into stale pointers.
 struct PlanHeader {
     unsigned magic;
-    int count, total_items, grid, rows;
+    int count, total_rb, grid, rows;
     int pad[3];
 };
-constexpr unsigned kPlanMagic = 0xB171A9E5u;
+constexpr unsigned kPlanMagic = 0xB171A9E6u;
 
 namespace {
 
-__device__ __forceinline__ bool plan_matches(const PlanHeader* h, int count, int total_items, int grid, int rows) {
-    return h->magic == kPlanMagic && h->count == count && h->total_items == total_items && h->grid == grid &&
-           h->rows == rows;
+__device__ __forceinline__ bool plan_matches(const PlanHeader* h, int count, int total_rb, int grid, int rows) {
+    return h->magic == kPlanMagic && h->count == count && h->total_rb == total_rb && h->grid == grid && h->rows == rows;
 }
 
-constexpr int kConsumers = 10;
-constexpr int kStreamThreads = (kConsumers + 2) * 32;
-constexpr int kMaxStages = 16;            // ring slots; a slot holds one item (16 rows x K/4 bytes, K <= 8192)
-constexpr int kRedBufs = 2;
-constexpr int kItemBytesCap = 32 * 1024;  // an item is as many 16-row blocks as fit in this many packed bytes
+constexpr int kStreamWarps = 16;
+constexpr int kStreamThreads = kStreamWarps * 32;
+constexpr int kRing = 2;  // chunk slots per warp
 constexpr int kBatchMaxK = 8192;
+constexpr size_t ring_bytes(int chunk_tiles) {
+    return (size_t)kStreamWarps * kRing * chunk_tiles * kTileBytes + kStreamWarps * kRing * 8 + 128;
+}
 
 // ------------------------------------------------------------------------------------ launch 1
 
 template <int VPT>
 __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHeader* __restrict__ hdr,
-                                                                    const DevProblem* __restrict__ probs, int count,
-                                                                    int total_items, int grid, int* status_word) {
+                                                                    const DevProblem* __restrict__ probs,
+                                                                    const int* __restrict__ row_prob, int count,
+                                                                    int total_rb, int grid, int* status_word) {
     __shared__ RowReduceSmem sm;
-    if (!plan_matches(hdr, count, total_items, grid, (int)gridDim.x)) {
+    if (!plan_matches(hdr, count, total_rb, grid, (int)gridDim.x)) {
         if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
         return;
     }
     const int row = blockIdx.x;
-    int lo = 0, hi = count - 1;  // last problem whose row_begin <= row
-    while (lo < hi) {
-        const int mid = (lo + hi + 1) >> 1;
-        if (probs[mid].row_begin <= row) lo = mid;
-        else hi = mid - 1;
-    }
-    const DevProblem& p = probs[lo];
+    const DevProblem& p = probs[row_prob[row]];
     const int m = row - p.row_begin;
-    quant_row<VPT>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq + (size_t)m * p.K, p.d + m, p.xsum + m, sm);
+    quant_row<VPT, true>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq + (size_t)m * p.K, p.d + m, p.xsum + m, sm);
 }
 
 // ------------------------------------------------------------------------------------ launch 2
@@ -98,337 +95,343 @@ __device__ __forceinline__ int dp4a_u8_s8(uint32_t a_u8x4, uint32_t b_s8x4, int 
     return d;
 }
 
-__device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+r"(c[0]), "+r"(c[1]), "+r"(c[2]), "+r"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
 
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+
 struct StreamParams {
     const DevProblem* probs;
-    const int* item_begin;  // [count + 1]
-    const int* cta_begin;   // [gridDim.x + 1]
+    const int4* cta_range;  // [grid] {first row block, one past the last, first problem, last problem} of each CTA
     const PlanHeader* hdr;
-    int count, total_items, rows;
-    int stages;
-    int rb_max;       // largest rb_per_item of the batch
-    int stage_bytes;  // size of a ring slot: the largest item of the batch, a multiple of 1024
+    int count, total_rb, rows;
+    int groups;     // G: warps that share a row block, each taking MT tokens
+    int table_cap;  // problems of a CTA whose descriptors are cached in shared memory
     int* status_word;
 };
 
-// Compute the partial sums of one 16-row block for this warp's tiles and write them to `rbuf`
-// ([16 rows][MP tokens]).  NT = 0: one token, dp4a.  NT = 1 / 2: up to 8 / 16 tokens, mma.sync.
-template <int NT, int TPW>
-__device__ __forceinline__ void row_block_partials(const uint4 (&wv)[TPW][2],
-                                                   const uint32_t (&xr)[TPW][NT == 0 ? 1 : NT][16], int n_act,
-                                                   int* rbuf, int g, int t) {
-    constexpr int MP = NT == 0 ? 1 : 8 * NT;
-    constexpr int XT = NT == 0 ? 1 : NT;
-    if constexpr (NT == 0) {
-        // accumulators per row and per bit position j hold 4^j x the true partial sum
-        int acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
-#pragma unroll
-        for (int i = 0; i < TPW; ++i) {
-            if (i >= n_act) break;  // warp-uniform: this warp owns n_act tiles of the row block
-            const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
-            const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t mask = 0x03030303u << (2 * j);
-                    acc[0][j] = dp4a_u8_s8(w0[q] & mask, xr[i][0][4 * q + j], acc[0][j]);
-                    acc[1][j] = dp4a_u8_s8(w1[q] & mask, xr[i][0][4 * q + j], acc[1][j]);
-                }
-        }
-        int v0 = acc[0][0] + (acc[0][1] >> 2) + (acc[0][2] >> 4) + (acc[0][3] >> 6);
-        int v1 = acc[1][0] + (acc[1][1] >> 2) + (acc[1][2] >> 4) + (acc[1][3] >> 6);
-        v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
-        v1 += __shfl_xor_sync(0xffffffffu, v1, 1);
-        v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
-        v1 += __shfl_xor_sync(0xffffffffu, v1, 2);
-        if (t == 0) {
-            rbuf[g] = v0;
-            rbuf[8 + g] = v1;
-        }
-    } else {
-        int acc[4][XT][4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-#pragma unroll
-            for (int nt = 0; nt < XT; ++nt)
-#pragma unroll
-                for (int r = 0; r < 4; ++r) acc[j][nt][r] = 0;
-#pragma unroll
-        for (int i = 0; i < TPW; ++i) {
-            if (i >= n_act) break;  // warp-uniform
-            const uint32_t w0[4] = {wv[i][0].x, wv[i][0].y, wv[i][0].z, wv[i][0].w};
-            const uint32_t w1[4] = {wv[i][1].x, wv[i][1].y, wv[i][1].z, wv[i][1].w};
-#pragma unroll
-            for (int q2 = 0; q2 < 2; ++q2)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t mask = 0x03030303u << (2 * j);
-                    const int qa = 2 * q2, qb = 2 * q2 + 1;
-                    const uint32_t a0 = w0[qa] & mask, a1 = w1[qa] & mask, a2 = w0[qb] & mask, a3 = w1[qb] & mask;
-#pragma unroll
-                    for (int nt = 0; nt < XT; ++nt)
-                        mma_u8s8(acc[j][nt], a0, a1, a2, a3, xr[i][nt][4 * qa + j], xr[i][nt][4 * qb + j]);
-                }
-        }
-#pragma unroll
-        for (int nt = 0; nt < XT; ++nt) {
-            int v[4];
-#pragma unroll
-            for (int r = 0; r < 4; ++r)
-                v[r] = acc[0][nt][r] + (acc[1][nt][r] >> 2) + (acc[2][nt][r] >> 4) + (acc[3][nt][r] >> 6);
-            // fragment layout: r0 (row g, token 2t), r1 (g, 2t+1), r2 (g+8, 2t), r3 (g+8, 2t+1)
-            const int tok = 8 * nt + 2 * t;
-            *reinterpret_cast<int2*>(rbuf + g * MP + tok) = make_int2(v[0], v[1]);
-            *reinterpret_cast<int2*>(rbuf + (g + 8) * MP + tok) = make_int2(v[2], v[3]);
-        }
-    }
-}
+// Shared-memory copy of what the stream kernel needs of one problem (filled once per CTA).
+struct alignas(16) SProb {
+    const uint8_t* packed;
+    void* y;
+    const int8_t* xq;
+    int rb_begin, rb_end, k_tiles, M, N, K, y_dtype;
+    int x_off;  // byte offset of token 0's codes in the CTA's activation arena
+    float s_w;
+    int pad[3];
+    float d[kGemvMaxTokens];
+    int xsum[kGemvMaxTokens];
+};
 
-// NT = 0: one token, dp4a.  NT = 1 / 2: up to 8 / 16 tokens, mma.sync with NT token tiles.
-template <int NT, int TPW>
+// Position of a warp in its sequence of weight chunks: row blocks rb, rb + par, ... of the CTA's range,
+// every chunk (a few 16x256 tiles, contiguous in memory) of each.  Two of these walk the same
+// sequence: one issues the bulk copies, one (kRing chunks behind) does the arithmetic.
+struct ChunkCursor {
+    int rb, c, p, rb_begin, rb_end, k_tiles, nc, ct;  // ct tiles per chunk, nc chunks per row block
+    const uint8_t* base;                              // the current problem's packed matrix
+    __device__ __forceinline__ void set_problem(int rb_begin_, int rb_end_, int k_tiles_, const void* packed,
+                                                int chunk_tiles) {
+        rb_begin = rb_begin_; rb_end = rb_end_; k_tiles = k_tiles_;
+        nc = (k_tiles + chunk_tiles - 1) / chunk_tiles;
+        ct = (k_tiles + nc - 1) / nc;
+        base = static_cast<const uint8_t*>(packed);
+    }
+    __device__ __forceinline__ int tiles() const { return (k_tiles - c * ct) < ct ? (k_tiles - c * ct) : ct; }
+    __device__ __forceinline__ const uint8_t* src() const {
+        return base + ((size_t)(rb - rb_begin) * k_tiles + (size_t)c * ct) * kTileBytes;
+    }
+};
+
+// MT = tokens per warp (1 or 4).  kChunkTiles = 16x256 tiles (1 KiB each) per bulk copy at most.
+// XS = the quantised activations of every problem the CTA touches are staged in shared memory once
+// (otherwise they are read through L1, which is slower).
+template <int MT, int kChunkTiles, bool XS>
 __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const StreamParams prm) {
-    constexpr int MP = NT == 0 ? 1 : 8 * NT;  // padded token count of the partial-sum buffers
-    constexpr int XT = NT == 0 ? 1 : NT;
-    constexpr int RB_INTS = kConsumers * 16 * MP;  // partial sums of one row block
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const int stages = prm.stages;
-    const int stage_bytes = prm.stage_bytes;
-    int* red = reinterpret_cast<int*>(smem + (size_t)stages * stage_bytes);  // [kRedBufs][rb_max][kConsumers][16][MP]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(red + kRedBufs * prm.rb_max * RB_INTS);
-    uint64_t* full_bar = bars;                       // [stages]  bytes of the item landed
-    uint64_t* empty_bar = bars + kMaxStages;         // [stages]  all consumers are done reading the item
-    uint64_t* redfull_bar = bars + 2 * kMaxStages;   // [kRedBufs] all consumers wrote their partial sums
-    uint64_t* redfree_bar = redfull_bar + kRedBufs;  // [kRedBufs] the epilogue is done with the buffer
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(redfree_bar + kRedBufs);
+    extern __shared__ __align__(128) uint8_t smem[];
+    // [ring: warps x kRing slots][barriers][abort flag][descriptor table][activation arena]
+    constexpr uint32_t kSlotBytes = kChunkTiles * kTileBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStreamWarps * kRing * kSlotBytes);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kStreamWarps * kRing);
+    SProb* table = reinterpret_cast<SProb*>(reinterpret_cast<uint8_t*>(bars) + kStreamWarps * kRing * 8 + 128);
+    uint8_t* arena = reinterpret_cast<uint8_t*>(table) + (size_t)prm.table_cap * sizeof(SProb);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (!plan_matches(prm.hdr, prm.count, prm.total_items, (int)gridDim.x, prm.rows)) {  // uniform over the grid
+    const int G = prm.groups;
+    if (!plan_matches(prm.hdr, prm.count, prm.total_rb, (int)gridDim.x, prm.rows)) {  // uniform over the grid
         if (blockIdx.x == 0 && threadIdx.x == 0 && prm.status_word != nullptr)
             atomicExch(prm.status_word, BITLINEAR_ERR_WORKSPACE);
         return;
     }
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < stages; ++s) {
-            mbar_init(smem_u32(full_bar + s), 1);
-            mbar_init(smem_u32(empty_bar + s), kConsumers);
-        }
-        for (int b = 0; b < kRedBufs; ++b) {
-            mbar_init(smem_u32(redfull_bar + b), kConsumers);
-            mbar_init(smem_u32(redfree_bar + b), 1);
-        }
-        *abort_flag = 0;
+    if (lane == 0) {
+        for (int r = 0; r < kRing; ++r) mbar_init(smem_u32(bars + warp * kRing + r), 1);
+        if (warp == 0) *abort_flag = 0;
         mbar_init_fence();
     }
     __syncthreads();
+    const int4 range = prm.cta_range[blockIdx.x];
+    const int rb_lo = range.x, rb_hi = range.y, p_lo = range.z;
+    const int n_local = rb_lo < rb_hi ? range.w - p_lo + 1 : 0;
+    const int n_tab = n_local < prm.table_cap ? n_local : prm.table_cap;
+    const DevProblem* probs = prm.probs;
+    const int par = kStreamWarps / G;             // row blocks in progress at a time in this CTA
+    const int rl = warp / G, tg = warp - rl * G;  // which of them this warp works on, and its token group
+    const bool mine = rl < par && rb_lo + rl < rb_hi;
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t ring_s = smem_u32(smem) + (uint32_t)warp * kRing * kSlotBytes;
+    const uint32_t bar_s = smem_u32(bars + warp * kRing);
 
-    const int item_lo = prm.cta_begin[blockIdx.x], item_hi = prm.cta_begin[blockIdx.x + 1];
-    // problem that holds item_lo
-    int p = 0;
-    {
-        int lo = 0, hi = prm.count - 1;
-        while (lo < hi) {
-            const int mid = (lo + hi + 1) >> 1;
-            if (prm.item_begin[mid] <= item_lo) lo = mid;
-            else hi = mid - 1;
-        }
-        p = lo;
-    }
-
-    if (warp == 0) {
-        // ---------------------------------------------------------------- producer
-        if (lane == 0) {
-            int next_begin = prm.item_begin[p];  // forces the first refresh
-            const uint8_t* base = nullptr;
-            int first = 0, rbpi = 1, n_rb = 0;
-            uint32_t rb_bytes = 0;
-            --p;
-            uint32_t stage = 0, phase = 0;
-            for (int it = item_lo; it < item_hi; ++it) {
-                while (it >= next_begin) {
-                    ++p;
-                    next_begin = prm.item_begin[p + 1];
-                    const DevProblem& pr = prm.probs[p];
-                    base = reinterpret_cast<const uint8_t*>(pr.packed);
-                    rb_bytes = (uint32_t)pr.k_tiles * kTileBytes;
-                    first = pr.item_begin;
-                    rbpi = pr.rb_per_item;
-                    n_rb = pr.N / kTileRows;
+    // descriptor of the next problem that holds row block c.rb: from the shared-memory table when it is there
+    auto enter = [&](ChunkCursor& c) {
+        for (;;) {
+            ++c.p;
+            const int i = c.p - p_lo;
+            if (i < n_tab) {
+                if (c.rb < table[i].rb_end) {
+                    c.set_problem(table[i].rb_begin, table[i].rb_end, table[i].k_tiles, table[i].packed, kChunkTiles);
+                    return;
                 }
-                const int rb0 = (it - first) * rbpi;
-                const int nrb = (n_rb - rb0) < rbpi ? (n_rb - rb0) : rbpi;
-                const uint32_t bytes = (uint32_t)nrb * rb_bytes;
-                if (!mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag)) break;
-                const uint32_t fb = smem_u32(full_bar + stage);
-                mbar_expect_tx(fb, bytes);
-                bulk_load(smem_u32(smem + (size_t)stage * stage_bytes), base + (size_t)rb0 * rb_bytes, bytes, fb);
-                if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
+            } else if (c.rb < probs[c.p].rb_end) {
+                c.set_problem(probs[c.p].rb_begin, probs[c.p].rb_end, probs[c.p].k_tiles, probs[c.p].packed, kChunkTiles);
+                return;
             }
         }
-        __syncwarp();
-    } else if (warp <= kConsumers) {
-        // ---------------------------------------------------------------- consumers
-        const int w = warp - 1;
-        const int g = lane >> 2, t = lane & 3;
-        int next_begin = prm.item_begin[p], k_tiles = 0, first = 0, rbpi = 1, n_rb = 0, n_act = 0;
-        --p;
-        uint32_t xr[TPW][XT][16];  // this lane's activation bytes: tile, token tile, 16 words = 64 columns
-        uint32_t stage = 0, phase = 0;
+    };
+
+    // ---- start the weight stream before anything else: the first chunks come from one problem ----
+    // Every warp of a token group issues its own copy of the chunk (the later readers hit L2).
+    ChunkCursor ld;  // where the next copy comes from
+    ld.rb = rb_lo + rl; ld.c = 0; ld.p = p_lo;
+    ld.rb_begin = 0; ld.rb_end = 0; ld.k_tiles = 1; ld.nc = 1; ld.ct = 1; ld.base = nullptr;
+    bool ld_valid = mine;
+    if (mine) {
+        while (ld.rb >= probs[ld.p].rb_end) ++ld.p;
+        ld.set_problem(probs[ld.p].rb_begin, probs[ld.p].rb_end, probs[ld.p].k_tiles, probs[ld.p].packed, kChunkTiles);
+    }
+    ChunkCursor cp = ld;  // where the arithmetic is
+    auto issue = [&](int slot) {  // lane 0 only
+        const uint32_t bytes = (uint32_t)ld.tiles() * kTileBytes;
+        mbar_expect_tx(bar_s + 8u * slot, bytes);
+        bulk_load(ring_s + (uint32_t)slot * kSlotBytes, ld.src(), bytes, bar_s + 8u * slot);
+    };
+    auto advance_ld = [&](bool may_enter) {
+        if (++ld.c == ld.nc) {
+            ld.c = 0;
+            ld.rb += par;
+            if (ld.rb >= rb_hi) ld_valid = false;
+            else if (may_enter && ld.rb >= ld.rb_end) enter(ld);
+        }
+    };
+    int primed = 0;  // the first copies stay inside the first problem (the table is not there yet)
+#pragma unroll
+    for (int r = 0; r < kRing; ++r)
+        if (ld_valid && ld.rb < ld.rb_end) {
+            if (lane == 0) issue(r);
+            primed = r + 1;
+            advance_ld(false);
+        }
+
+    // ---- fill the descriptor table (one warp per problem), then stage the activations ----
+    for (int i = warp; i < n_tab; i += kStreamWarps) {
+        const DevProblem& pr = probs[p_lo + i];
+        if (lane == 0) {
+            SProb& e = table[i];
+            e.packed = pr.packed;
+            e.y = pr.y; e.xq = pr.xq;
+            e.rb_begin = pr.rb_begin; e.rb_end = pr.rb_end; e.k_tiles = pr.k_tiles;
+            e.M = pr.M; e.N = pr.N; e.K = pr.K; e.y_dtype = pr.y_dtype;
+            e.x_off = 0;
+            e.s_w = *pr.s_w;
+        }
+        if (lane < kGemvMaxTokens) {
+            table[i].d[lane] = lane < pr.M ? pr.d[lane] : 0.0f;
+            table[i].xsum[lane] = lane < pr.M ? pr.xsum[lane] : 0;
+        }
+    }
+    __syncthreads();
+    if (XS) {
+        if (threadIdx.x == 0) {
+            int off = 0;
+            for (int i = 0; i < n_tab; ++i) {
+                table[i].x_off = off;
+                off += table[i].M * table[i].K;  // a multiple of 256
+            }
+        }
+        __syncthreads();
+        const uint32_t arena_s = smem_u32(arena);
+        for (int i = 0; i < n_tab; ++i) {
+            const int bytes = table[i].M * table[i].K;
+            const int8_t* src = table[i].xq;
+            const uint32_t dst = arena_s + (uint32_t)table[i].x_off;
+            for (int o = threadIdx.x * 16; o < bytes; o += kStreamThreads * 16) cp_async16(dst + o, src + o);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+    }
+
+    if (mine) {
+        // top up the ring now that the cursor may cross into later problems
+        if (ld_valid && ld.rb >= ld.rb_end) enter(ld);
+#pragma unroll
+        for (int r = 0; r < kRing; ++r)
+            if (r >= primed && ld_valid) {
+                if (lane == 0) issue(r);
+                advance_ld(true);
+            }
+
+        // per-problem state of the arithmetic side
+        int M = 0, N = 0, y_dtype = 0, xs_lane = 0;
+        void* y = nullptr;
+        float s_w = 0.0f, d_lane = 0.0f;
+        bool active = false;
+        const int8_t* xrow_g[MT];  // !XS: token rows in global memory
+        uint32_t xrow_s[MT];       //  XS: token rows in the shared-memory arena
+        auto load_problem_state = [&]() {
+            const int i = cp.p - p_lo;
+            const int my_tok = tg * MT + (MT == 1 ? 0 : t);  // lane t finishes token tg*MT + t
+            int K = 0, x_off = 0;
+            const int8_t* xq = nullptr;
+            if (i < n_tab) {
+                const SProb& e = table[i];
+                M = e.M; N = e.N; y_dtype = e.y_dtype; y = e.y; s_w = e.s_w; K = e.K; x_off = e.x_off; xq = e.xq;
+                d_lane = my_tok < M ? e.d[my_tok] : 0.0f;
+                xs_lane = my_tok < M ? e.xsum[my_tok] : 0;
+            } else {
+                const DevProblem& pr = probs[cp.p];
+                M = pr.M; N = pr.N; y_dtype = pr.y_dtype; y = pr.y; s_w = *pr.s_w; K = pr.K; xq = pr.xq;
+                d_lane = my_tok < M ? pr.d[my_tok] : 0.0f;
+                xs_lane = my_tok < M ? pr.xsum[my_tok] : 0;
+            }
+            active = tg * MT < M;  // warp-uniform: this token group holds real tokens
+#pragma unroll
+            for (int m = 0; m < MT; ++m) {
+                int tok = tg * MT + m;
+                if (tok > M - 1) tok = M - 1;  // padding tokens re-read a real row; their sums are dropped
+                xrow_g[m] = xq + (size_t)tok * K + t * 16;
+                xrow_s[m] = smem_u32(arena) + (uint32_t)(x_off + tok * K + t * 16);
+            }
+        };
+        load_problem_state();
+
+        int acc[2][4][MT];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int m = 0; m < MT; ++m) acc[h][j][m] = 0;
+
+        uint32_t n_chunk = 0;  // chunks consumed: slot = n_chunk % kRing, phase = (n_chunk / kRing) & 1
         bool ok = true;
-        for (int it = item_lo; ok && it < item_hi; ++it) {
-            if (it >= next_begin) {
-                while (it >= next_begin) {
-                    ++p;
-                    next_begin = prm.item_begin[p + 1];
-                }
-                const DevProblem& pr = prm.probs[p];
-                k_tiles = pr.k_tiles;
-                first = pr.item_begin;
-                rbpi = pr.rb_per_item;
-                n_rb = pr.N / kTileRows;
-                n_act = w < k_tiles ? (k_tiles - w + kConsumers - 1) / kConsumers : 0;  // tiles w, w+10, ... < k_tiles
+        for (;;) {
+            const uint32_t slot = n_chunk % kRing, phase = (n_chunk / kRing) & 1u;
+            if (!mbar_wait(bar_s + 8u * slot, phase, abort_flag)) { ok = false; break; }
+            const int tiles = cp.tiles();
+            if (active) {
+                uint32_t wa = ring_s + slot * kSlotBytes + (uint32_t)lane * 16u;
+                uint32_t xo = (uint32_t)(cp.c * cp.ct) * kTileCols;
+#pragma unroll 2
+                for (int tile = 0; tile < tiles; ++tile, wa += kTileBytes, xo += kTileCols) {
+                    const uint4 w0v = lds128(wa), w1v = lds128(wa + 512);
+                    const uint32_t w0[4] = {w0v.x, w0v.y, w0v.z, w0v.w};
+                    const uint32_t w1[4] = {w1v.x, w1v.y, w1v.z, w1v.w};
+                    // the token rows are stored with the four 16-byte pieces of each lane's 64 columns interleaved
+                    // (piece q of lane t at 64q + 16t inside the tile), so the four t lanes read 64 contiguous bytes
 #pragma unroll
-                for (int i = 0; i < TPW; ++i) {
-                    const int kt = w + i * kConsumers;
+                    for (int q = 0; q < 4; ++q) {
+                        uint32_t xw[MT][4];
 #pragma unroll
-                    for (int nt = 0; nt < XT; ++nt) {
-                        const int tok = NT == 0 ? 0 : g + 8 * nt;
-                        if (kt < k_tiles && tok < pr.M) {
-                            const uint4* src =
-                                reinterpret_cast<const uint4*>(pr.xq + (size_t)tok * pr.K + (size_t)kt * kTileCols + 64 * t);
+                        for (int m = 0; m < MT; ++m) {
+                            uint4 v;
+                            if (XS) v = lds128(xrow_s[m] + xo + 64u * q);
+                            else v = *reinterpret_cast<const uint4*>(xrow_g[m] + xo + 64 * q);
+                            xw[m][0] = v.x; xw[m][1] = v.y; xw[m][2] = v.z; xw[m][3] = v.w;
+                        }
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const uint4 v = src[q];
-                                xr[i][nt][4 * q] = v.x; xr[i][nt][4 * q + 1] = v.y;
-                                xr[i][nt][4 * q + 2] = v.z; xr[i][nt][4 * q + 3] = v.w;
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t mask = 0x03030303u << (2 * j);
+                            const uint32_t a0 = w0[q] & mask, a1 = w1[q] & mask;
+#pragma unroll
+                            for (int m = 0; m < MT; ++m) {
+                                acc[0][j][m] = dp4a_u8_s8(a0, xw[m][j], acc[0][j][m]);
+                                acc[1][j][m] = dp4a_u8_s8(a1, xw[m][j], acc[1][j][m]);
                             }
-                        } else {
-#pragma unroll
-                            for (int q = 0; q < 16; ++q) xr[i][nt][q] = 0u;
                         }
                     }
                 }
             }
-            const int c = it - item_lo;
-            const int rb0 = (it - first) * rbpi;
-            const int nrb = (n_rb - rb0) < rbpi ? (n_rb - rb0) : rbpi;
-            if (!mbar_wait(smem_u32(full_bar + stage), phase, abort_flag)) { ok = false; break; }
-            const uint32_t rphase = (uint32_t)(c / kRedBufs) & 1u;
-            if (!mbar_wait(smem_u32(redfree_bar + c % kRedBufs), rphase ^ 1u, abort_flag)) { ok = false; break; }
-            const uint32_t sbase = smem_u32(smem + (size_t)stage * stage_bytes) + lane * 16;
-            int* rbase = red + (c % kRedBufs) * prm.rb_max * RB_INTS + w * 16 * MP;
-            for (int r = 0; r < nrb; ++r) {
-                uint4 wv[TPW][2];
+            __syncwarp();  // every lane has read the slot: it may be refilled
+            if (ld_valid) {
+                if (lane == 0) issue((int)slot);
+                advance_ld(true);
+            }
+            ++n_chunk;
+            if (++cp.c == cp.nc) {
+                // ---- end of a row block: fold the four scales (accumulator j holds 4^j x its share), the four
+                //      column lanes, subtract the code offset, dequantise, store ----
+                if (active) {
+                    int v[2][MT];
 #pragma unroll
-                for (int i = 0; i < TPW; ++i) {
-                    const int kt = w + i * kConsumers;
-                    if (i < n_act) {
-                        wv[i][0] = lds128(sbase + (r * k_tiles + kt) * kTileBytes);
-                        wv[i][1] = lds128(sbase + (r * k_tiles + kt) * kTileBytes + 512);
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int m = 0; m < MT; ++m) {
+                            // 64 x the sum: ((a0*4 + a1)*4 + a2)*4 + a3; |sum| <= 254*K/4 per lane: no overflow for K <= 8192
+                            int sum = acc[h][0][m] * 4 + acc[h][1][m];
+                            sum = sum * 4 + acc[h][2][m];
+                            sum = sum * 4 + acc[h][3][m];
+                            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                            v[h][m] = sum >> 6;  // exact: a multiple of 64
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) acc[h][j][m] = 0;
+                        }
+                    const int n0 = (cp.rb - cp.rb_begin) * kTileRows + g;
+                    const int tok = tg * MT + (MT == 1 ? 0 : t);
+                    if (tok < M && (MT > 1 || t == 0)) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            int sel = v[h][0];
+#pragma unroll
+                            for (int m = 1; m < MT; ++m) sel = (t == m) ? v[h][m] : sel;
+                            const int total = sel - xs_lane;
+                            const float val = __fmul_rn(__fmul_rn((float)total, s_w), d_lane);
+                            const size_t idx = (size_t)tok * N + n0 + 8 * h;
+                            if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
+                            else reinterpret_cast<float*>(y)[idx] = val;
+                        }
                     }
                 }
-                row_block_partials<NT, TPW>(wv, xr, n_act, rbase + r * RB_INTS, g, t);
-            }
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(smem_u32(empty_bar + stage));
-                mbar_arrive(smem_u32(redfull_bar + c % kRedBufs));
-            }
-            if (++stage == (uint32_t)stages) { stage = 0; phase ^= 1u; }
-        }
-    } else {
-        // ---------------------------------------------------------------- epilogue
-        int next_begin = prm.item_begin[p], first = 0, active = 0, M = 0, N = 0, y_dtype = 0, rbpi = 1, n_rb = 0;
-        --p;
-        float s_w = 0.0f;
-        void* y = nullptr;
-        int xs_lane = 0;       // lane m holds the code sum and the scale of token m of the current problem
-        float d_lane = 0.0f;
-        for (int it = item_lo; it < item_hi; ++it) {
-            if (it >= next_begin) {
-                while (it >= next_begin) {
-                    ++p;
-                    next_begin = prm.item_begin[p + 1];
-                }
-                const DevProblem& pr = prm.probs[p];
-                first = pr.item_begin;
-                active = pr.k_tiles < kConsumers ? pr.k_tiles : kConsumers;
-                M = pr.M; N = pr.N; y_dtype = pr.y_dtype;
-                rbpi = pr.rb_per_item;
-                n_rb = pr.N / kTileRows;
-                s_w = *pr.s_w;
-                y = pr.y;
-                xs_lane = lane < M ? pr.xsum[lane] : 0;
-                d_lane = lane < M ? pr.d[lane] : 0.0f;
-            }
-            const int c = it - item_lo;
-            const int rb0 = (it - first) * rbpi;
-            const int nrb = (n_rb - rb0) < rbpi ? (n_rb - rb0) : rbpi;
-            const uint32_t rphase = (uint32_t)(c / kRedBufs) & 1u;
-            if (!mbar_wait(smem_u32(redfull_bar + c % kRedBufs), rphase, abort_flag)) break;
-            const int* rb = red + (c % kRedBufs) * prm.rb_max * RB_INTS;
-            const int rows = nrb * 16;
-            for (int m = 0; m < M; ++m) {
-                const int xs = __shfl_sync(0xffffffffu, xs_lane, m);
-                const float dm = __shfl_sync(0xffffffffu, d_lane, m);
-                for (int rr = lane; rr < rows; rr += 32) {  // consecutive lanes -> consecutive output rows
-                    const int r = rr >> 4, row = rr & 15;
-                    int total = 0;
-                    for (int w = 0; w < active; ++w) total += rb[r * RB_INTS + (w * 16 + row) * MP + m];
-                    total -= xs;
-                    const float val = __fmul_rn(__fmul_rn((float)total, s_w), dm);
-                    const size_t idx = (size_t)m * N + (size_t)rb0 * kTileRows + rr;
-                    if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
-                    else reinterpret_cast<float*>(y)[idx] = val;
+                cp.c = 0;
+                cp.rb += par;
+                if (cp.rb >= rb_hi) break;
+                if (cp.rb >= cp.rb_end) {
+                    enter(cp);
+                    load_problem_state();
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(redfree_bar + c % kRedBufs));
         }
+        if (!ok) abort_drain();  // copies of this warp may still be in flight
     }
-
     __syncthreads();
-    if (*abort_flag) {
-        abort_drain();
-        if (threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
-    }
+    if (*abort_flag && threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
 }
 
-template <int NT, int TPW>
+template <int MT, int kChunkTiles, bool XS>
 cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<NT, TPW>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<MT, kChunkTiles, XS>,
+                                         cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    decode_stream_kernel<NT, TPW><<<grid, kStreamThreads, smem, st>>>(prm);
+    decode_stream_kernel<MT, kChunkTiles, XS><<<grid, kStreamThreads, smem, st>>>(prm);
     return cudaGetLastError();
 }
 
-template <int NT>
-cudaError_t launch_stream_nt(int tpw, const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
-    switch (tpw) {
-        case 1: return launch_stream<NT, 1>(prm, grid, smem, st);
-        case 2: return launch_stream<NT, 2>(prm, grid, smem, st);
-        case 3: return launch_stream<NT, 3>(prm, grid, smem, st);
-        default: return launch_stream<NT, 4>(prm, grid, smem, st);
-    }
-}
-
 struct PlanLayout {
-    size_t probs_off, item_off, cta_off, xq_off, total;
+    size_t probs_off, cta_range_off, row_prob_off, xq_off, total;
 };
 
 PlanLayout plan_layout(int count, int grid, size_t xq_bytes, size_t rows) {
@@ -436,10 +439,10 @@ PlanLayout plan_layout(int count, int grid, size_t xq_bytes, size_t rows) {
     size_t off = 256;  // the PlanHeader sits at offset 0
     L.probs_off = off;
     off = align_up(off + (size_t)count * sizeof(DevProblem), 256);
-    L.item_off = off;
-    off = align_up(off + (size_t)(count + 1) * sizeof(int), 256);
-    L.cta_off = off;
-    off = align_up(off + (size_t)(grid + 1) * sizeof(int), 256);
+    L.cta_range_off = off;
+    off = align_up(off + (size_t)(grid + 1) * sizeof(int4), 256);
+    L.row_prob_off = off;
+    off = align_up(off + (rows + 1) * sizeof(int), 256);
     L.xq_off = off;
     off = align_up(off + xq_bytes, 256);                   // int8 activations of every problem
     off = align_up(off + rows * sizeof(float), 256);       // d
@@ -477,7 +480,7 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     if (!problems) return BITLINEAR_ERR_NULL;
     if (flags & ~(BITLINEAR_BATCH_REUSE_PLAN | BITLINEAR_BATCH_REUSE_ACT)) return BITLINEAR_ERR_DTYPE;
     size_t xq_bytes = 0, rows = 0;
-    int max_m = 0, max_ktiles = 0, max_k = 0;
+    int max_m = 0, max_k = 0;
     for (int i = 0; i < count; ++i) {
         const bitlinear_problem& q = problems[i];
         if (q.y_dtype != BITLINEAR_F32 && q.y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
@@ -490,7 +493,6 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
         xq_bytes += align_up((size_t)q.M * q.K, 16);
         rows += (size_t)q.M;
         if (q.M > max_m) max_m = q.M;
-        if (q.K / kTileCols > max_ktiles) max_ktiles = q.K / kTileCols;
         if (q.K > max_k) max_k = q.K;
     }
     const PlanLayout L = plan_layout(count, kPlanGrid, xq_bytes, rows);
@@ -512,22 +514,22 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ws);
 
-    // ---- host plan: device descriptors, item prefix, byte-balanced CTA ranges ----
-    int rb_max = 1, stage_bytes = 0;
+    // ---- host plan: device descriptors, token -> problem table, byte-balanced CTA ranges ----
     std::vector<DevProblem> dp;
-    std::vector<int> item_begin;
+    std::vector<int> row_prob;
     dp.reserve(count);
-    item_begin.reserve(count + 1);
+    row_prob.reserve(rows + 1);
+    int total_rb = 0;
     {
         char* xq_ptr = base + L.xq_off;
         float* d_ptr = reinterpret_cast<float*>(base + align_up(L.xq_off + xq_bytes, 256));
         int32_t* xs_ptr = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(d_ptr) + align_up(rows * sizeof(float), 256));
-        int items = 0, row = 0;
+        int row = 0;
         for (int i = 0; i < count; ++i) {
             const bitlinear_problem& q = problems[i];
             if (q.M == 0) continue;
             DevProblem v;
-            v.packed = static_cast<const uint32_t*>(q.packed);
+            v.packed = static_cast<const uint8_t*>(q.packed);
             v.s_w = q.s_w;
             v.y = q.y;
             v.x = static_cast<const __nv_bfloat16*>(q.x);
@@ -538,62 +540,80 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
             v.M = q.M; v.N = q.N; v.K = q.K; v.y_dtype = q.y_dtype;
             v.eps = q.rms_eps;
             v.k_tiles = q.K / kTileCols;
-            {
-                int rb = kItemBytesCap / (v.k_tiles * kTileBytes);
-                const int rb_cap = max_m <= 8 ? 4 : 2;  // bounds the partial-sum buffers
-                if (rb > rb_cap) rb = rb_cap;
-                if (rb < 1) rb = 1;
-                v.rb_per_item = rb;
-                if (rb > rb_max) rb_max = rb;
-                if (rb * v.k_tiles * kTileBytes > stage_bytes) stage_bytes = rb * v.k_tiles * kTileBytes;
-            }
-            v.item_begin = items;
+            v.rb_begin = total_rb;
+            v.rb_end = total_rb + q.N / kTileRows;
             v.row_begin = row;
+            for (int m = 0; m < q.M; ++m) row_prob.push_back((int)dp.size());
             dp.push_back(v);
-            item_begin.push_back(items);
-            items += (q.N / kTileRows + v.rb_per_item - 1) / v.rb_per_item;
+            total_rb = v.rb_end;
             row += q.M;
             xq_ptr += align_up((size_t)q.M * q.K, 16);
         }
-        item_begin.push_back(items);
+        row_prob.push_back(0);
     }
     const int n_prob = (int)dp.size();
-    const int total_items = item_begin.back();
-    int grid = sm_count < total_items ? sm_count : total_items;
-    std::vector<int> cta_begin(grid + 1);
+    const int grid = sm_count < total_rb ? sm_count : total_rb;
+    std::vector<int4> cta_range(grid);
+    int table_cap = 1;     // most problems any CTA touches
+    size_t arena_max = 0;  // most activation bytes any CTA needs
     {
-        double total_bytes = 0.0;
-        for (int i = 0; i < n_prob; ++i) total_bytes += (double)(item_begin[i + 1] - item_begin[i]) * dp[i].k_tiles * dp[i].rb_per_item;
+        std::vector<int> cta_rb(grid + 1);
+        double total_tiles = 0.0;
+        for (int i = 0; i < n_prob; ++i) total_tiles += (double)(dp[i].rb_end - dp[i].rb_begin) * dp[i].k_tiles;
         int pi = 0;
-        double before = 0.0;  // tile-KB before problem pi
-        cta_begin[0] = 0;
+        double before = 0.0;  // tiles before problem pi
+        cta_rb[0] = 0;
         for (int c = 1; c < grid; ++c) {
-            const double target = total_bytes * c / grid;
-            while (pi < n_prob - 1 &&
-                   before + (double)(item_begin[pi + 1] - item_begin[pi]) * dp[pi].k_tiles * dp[pi].rb_per_item <= target) {
-                before += (double)(item_begin[pi + 1] - item_begin[pi]) * dp[pi].k_tiles * dp[pi].rb_per_item;
+            const double target = total_tiles * c / grid;
+            while (pi < n_prob - 1 && before + (double)(dp[pi].rb_end - dp[pi].rb_begin) * dp[pi].k_tiles <= target) {
+                before += (double)(dp[pi].rb_end - dp[pi].rb_begin) * dp[pi].k_tiles;
                 ++pi;
             }
-            int it = item_begin[pi] + (int)((target - before) / ((double)dp[pi].k_tiles * dp[pi].rb_per_item) + 0.5);
-            if (it > item_begin[pi + 1]) it = item_begin[pi + 1];
-            if (it < cta_begin[c - 1]) it = cta_begin[c - 1];
-            cta_begin[c] = it;
+            int rb = dp[pi].rb_begin + (int)((target - before) / (double)dp[pi].k_tiles + 0.5);
+            if (rb > dp[pi].rb_end) rb = dp[pi].rb_end;
+            if (rb < cta_rb[c - 1]) rb = cta_rb[c - 1];
+            cta_rb[c] = rb;
         }
-        cta_begin[grid] = total_items;
+        cta_rb[grid] = total_rb;
+        int pf = 0;
+        for (int c = 0; c < grid; ++c) {
+            const int lo = cta_rb[c], hi = cta_rb[c + 1];
+            while (pf < n_prob - 1 && lo >= dp[pf].rb_end) ++pf;
+            int pl = pf;
+            while (pl < n_prob - 1 && hi - 1 >= dp[pl].rb_end) ++pl;
+            cta_range[c] = make_int4(lo, hi, pf, pl);
+            if (lo < hi) {
+                if (pl - pf + 1 > table_cap) table_cap = pl - pf + 1;
+                size_t a = 0;
+                for (int i = pf; i <= pl; ++i) a += (size_t)dp[i].M * dp[i].K;
+                if (a > arena_max) arena_max = a;
+            }
+        }
+    }
+    // shared memory: chunk ring + descriptor table + activation arena; when that does not fit, the activations
+    // are read through L1 instead and only as many descriptors as fit are cached
+    const int mt = max_m <= 1 ? 1 : 4;
+    const int chunk_tiles = mt == 1 ? 5 : 4;
+    const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles) - 128;
+    bool stage_x = true;
+    if ((size_t)table_cap * sizeof(SProb) + arena_max > smem_limit) {
+        stage_x = false;
+        arena_max = 0;
+        if ((size_t)table_cap * sizeof(SProb) > smem_limit) table_cap = (int)(smem_limit / sizeof(SProb));
     }
 
     PlanHeader hdr_host;
     hdr_host.magic = kPlanMagic;
     hdr_host.count = n_prob;
-    hdr_host.total_items = total_items;
+    hdr_host.total_rb = total_rb;
     hdr_host.grid = grid;
     hdr_host.rows = (int)rows;
     hdr_host.pad[0] = hdr_host.pad[1] = hdr_host.pad[2] = 0;
     if (!(flags & BITLINEAR_BATCH_REUSE_PLAN)) {
         if (cudaMemcpyAsync(base, &hdr_host, sizeof(hdr_host), cudaMemcpyHostToDevice, st) != cudaSuccess ||
             cudaMemcpyAsync(base + L.probs_off, dp.data(), dp.size() * sizeof(DevProblem), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-            cudaMemcpyAsync(base + L.item_off, item_begin.data(), item_begin.size() * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess ||
-            cudaMemcpyAsync(base + L.cta_off, cta_begin.data(), cta_begin.size() * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            cudaMemcpyAsync(base + L.cta_range_off, cta_range.data(), cta_range.size() * sizeof(int4), cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(base + L.row_prob_off, row_prob.data(), row_prob.size() * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess) {
             cudaGetLastError();
             return BITLINEAR_ERR_CUDA;
         }
@@ -605,38 +625,29 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
         const int vpt = (max_k / 8 + kQuantThreads - 1) / kQuantThreads;
         const dim3 g((unsigned)rows), b(kQuantThreads);
         const PlanHeader* h = reinterpret_cast<const PlanHeader*>(base);
+        const int* rp = reinterpret_cast<const int*>(base + L.row_prob_off);
         int* sw = device_status_word();
-        if (vpt <= 1) batch_quant_kernel<1><<<g, b, 0, st>>>(h, probs_dev, n_prob, total_items, grid, sw);
-        else if (vpt <= 2) batch_quant_kernel<2><<<g, b, 0, st>>>(h, probs_dev, n_prob, total_items, grid, sw);
-        else batch_quant_kernel<4><<<g, b, 0, st>>>(h, probs_dev, n_prob, total_items, grid, sw);
+        if (vpt <= 1) batch_quant_kernel<1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+        else if (vpt <= 2) batch_quant_kernel<2><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+        else batch_quant_kernel<4><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
 
     // ---- launch 2: stream the weights ----
     StreamParams prm;
     prm.probs = probs_dev;
-    prm.item_begin = reinterpret_cast<const int*>(base + L.item_off);
-    prm.cta_begin = reinterpret_cast<const int*>(base + L.cta_off);
+    prm.cta_range = reinterpret_cast<const int4*>(base + L.cta_range_off);
     prm.hdr = reinterpret_cast<const PlanHeader*>(base);
     prm.count = n_prob;
-    prm.total_items = total_items;
+    prm.total_rb = total_rb;
     prm.rows = (int)rows;
     prm.status_word = device_status_word();
-    const int nt = max_m <= 1 ? 0 : (max_m <= 8 ? 1 : 2);
-    const int mp = nt == 0 ? 1 : 8 * nt;
-    const int tpw = (max_ktiles + kConsumers - 1) / kConsumers;  // <= 4 since K <= 8192
-    const size_t fixed = 1024 + (size_t)kRedBufs * rb_max * kConsumers * 16 * mp * sizeof(int) +
-                         (2 * kMaxStages + 2 * kRedBufs) * 8 + 64;
-    int stages = (int)((227 * 1024 - fixed) / stage_bytes);
-    if (stages > kMaxStages) stages = kMaxStages;
-    prm.stages = stages;
-    prm.stage_bytes = stage_bytes;
-    prm.rb_max = rb_max;
-    const size_t smem = fixed + (size_t)stages * stage_bytes;
+    prm.groups = (max_m + mt - 1) / mt;  // 1 .. 4
+    prm.table_cap = table_cap;
+    const size_t smem = ring_bytes(chunk_tiles) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
     cudaError_t e;
-    if (nt == 0) e = launch_stream_nt<0>(tpw, prm, grid, smem, st);
-    else if (nt == 1) e = launch_stream_nt<1>(tpw, prm, grid, smem, st);
-    else e = launch_stream_nt<2>(tpw, prm, grid, smem, st);
+    if (mt == 1) e = stage_x ? launch_stream<1, 5, true>(prm, grid, smem, st) : launch_stream<1, 5, false>(prm, grid, smem, st);
+    else e = stage_x ? launch_stream<4, 4, true>(prm, grid, smem, st) : launch_stream<4, 4, false>(prm, grid, smem, st);
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 

@@ -30,7 +30,10 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& u, float (&f)[8]) {
 }
 
 // Quantises one row with the kQuantThreads threads of the calling CTA (all must call it).
-template <int VPT>  // 16-byte vectors (8 bf16) per thread
+// PERM = false: codes are stored in column order.  PERM = true: inside every block of 256 columns the
+// sixteen 16-byte pieces are stored transposed (piece 4t+q, columns 64t+16q .. +15, at byte 64q+16t), the
+// order in which the four column lanes of the batched decode kernel read them.
+template <int VPT, bool PERM = false>  // VPT = 16-byte vectors (8 bf16) per thread
 __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_row,
                                           const __nv_bfloat16* __restrict__ gain, float eps, int K,
                                           int8_t* __restrict__ xq_row, float* __restrict__ d_out,
@@ -112,7 +115,12 @@ __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_ro
             csum += q;
             packed[e >> 2] |= (uint32_t)(q & 0xff) << (8 * (e & 3));
         }
-        if (v < n_vec) qrow[v] = make_uint2(packed[0], packed[1]);
+        int dst = v;  // in units of 8 codes
+        if (PERM) {
+            const int piece = (v >> 1) & 15;  // 16-byte piece inside the 256-column block: 4t + q
+            dst = (v & ~31) | ((((piece & 3) << 2) | (piece >> 2)) << 1) | (v & 1);
+        }
+        if (v < n_vec) qrow[dst] = make_uint2(packed[0], packed[1]);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xffffffffu, csum, o);
