@@ -5,8 +5,9 @@
 // and the epilogue removes the offset with the per-token code sum.)
 //
 // Persistent, warp-specialised kernel, one CTA per SM:
-//   warp 0   : TMA producer  - 128B-swizzled tiles of A (tokens x K) and B (weight rows x K) into a
-//              4-stage shared-memory ring, completion on mbarriers
+//   warp 0   : producer      - per stage a 128B-swizzled TMA tile of A (tokens x K) and one linear 32 KiB
+//              bulk copy of B (the weight codes are laid out in global memory as the shared-memory images
+//              of their 256 x 128 tiles) into a 4-stage shared-memory ring, completion on mbarriers
 //   warp 1   : MMA issuer    - one elected thread issues tcgen05.mma 128 x 256 x 32 and commits
 //   warps 2-5: epilogue      - tcgen05.ld of a finished 128 x 256 int32 accumulator, subtract the
 //              code sum, two fp32 multiplies, store; tensor memory is double buffered so the
@@ -88,6 +89,13 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// Linear bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -144,7 +152,7 @@ __device__ __forceinline__ TileCoord tile_coord(int tile, int m_tiles) {
 }
 
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restrict__ codes,
                const float* __restrict__ d, const int32_t* __restrict__ xsum, const float* __restrict__ s_w_ptr, int M,
                int N, int K, void* __restrict__ y, int y_dtype, int32_t* __restrict__ acc_out, int* status_word) {
     extern __shared__ uint8_t smem_raw[];
@@ -199,7 +207,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     mbar_expect_tx(fb, STAGE_BYTES);
                     const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
                     tma_load_2d(sa, &map_a, kb * BK, tc.m0, fb);
-                    tma_load_2d(sa + A_BYTES, &map_b, kb * BK, tc.n0, fb);
+                    bulk_load(sa + A_BYTES, codes + ((size_t)(tc.n0 / BN) * k_blocks + kb) * B_BYTES, B_BYTES, fb);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -346,7 +354,7 @@ bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows)
 
 }  // namespace
 
-size_t gemm_scratch_bytes(int N, int K) { return (size_t)N * K; }
+size_t gemm_scratch_bytes(int N, int K) { return (size_t)((N + BN - 1) / BN) * BN * K; }  // whole 256-row tiles
 
 int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* codes, const float* s_w, int M,
                  int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st) {
@@ -363,11 +371,11 @@ int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const ui
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
-    CUtensorMap map_a, map_b;
-    if (!make_map(&map_a, xq, M, K, BM) || !make_map(&map_b, codes, N, K, BN)) return BITLINEAR_ERR_CUDA;
+    CUtensorMap map_a;
+    if (!make_map(&map_a, xq, M, K, BM)) return BITLINEAR_ERR_CUDA;
     const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
     const int grid = tiles < sm_count ? tiles : sm_count;
-    gemm_i8_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(map_a, map_b, d, xsum, s_w, M, N, K, y, y_dtype, acc_out,
+    gemm_i8_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(map_a, codes, d, xsum, s_w, M, N, K, y, y_dtype, acc_out,
                                                       device_status_word());
     return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }

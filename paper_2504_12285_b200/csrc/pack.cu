@@ -113,6 +113,25 @@ __global__ void __launch_bounds__(256) quant_pack_kernel(const T* __restrict__ W
     packed[word] = out;
 }
 
+// Tensor-core staging order of the unpacked codes (see launch_unpack_codes_u8): one thread expands one
+// packed word into the 16-byte piece of its 256-row x 128-column tile.
+__global__ void __launch_bounds__(256) unpack_codes_tiled_kernel(const uint32_t* __restrict__ packed, int N, int K,
+                                                                 uint8_t* __restrict__ out) {
+    const size_t n_words = (size_t)N * K / 16;
+    const size_t word = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (word >= n_words) return;
+    int n, k0;
+    word_to_row_col(word, K / kTileCols, n, k0);
+    const uint32_t p = packed[word];
+    uint32_t v[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[j] = (p >> (2 * j)) & 0x03030303u;
+    const int r = n & 255, piece = (k0 & 127) >> 4;
+    const size_t tile = (size_t)(n >> 8) * (K / 128) + (k0 >> 7);
+    *reinterpret_cast<uint4*>(out + tile * 32768 + (size_t)r * 128 + ((piece ^ (r & 7)) << 4)) =
+        make_uint4(v[0], v[1], v[2], v[3]);
+}
+
 // One thread expands one packed word into 16 bytes.  SIGNED: values -1/0/1, else codes 0/1/2.
 template <bool SIGNED>
 __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict__ packed, int N, int K,
@@ -175,9 +194,13 @@ cudaError_t launch_unpack_i8(const uint32_t* packed, int N, int K, int8_t* wq, c
     return cudaGetLastError();
 }
 
+// Codes 0/1/2 as bytes, in the order the tensor-core kernel stages them: the [N][K] matrix is cut into tiles of
+// 256 rows x 128 columns, 32 KiB each, stored row-tile major; inside a tile row r keeps its eight 16-byte pieces at
+// r*128 + ((piece ^ (r & 7)) * 16), which is the 128-byte shared-memory swizzle.  A tile is therefore the exact
+// shared-memory image of one pipeline stage of the weight operand and is fetched with one linear bulk copy.
 cudaError_t launch_unpack_codes_u8(const uint32_t* packed, int N, int K, uint8_t* codes, cudaStream_t st) {
     const size_t n_words = (size_t)N * K / 16;
-    unpack_kernel<false><<<(unsigned)((n_words + 255) / 256), 256, 0, st>>>(packed, N, K, codes);
+    unpack_codes_tiled_kernel<<<(unsigned)((n_words + 255) / 256), 256, 0, st>>>(packed, N, K, codes);
     return cudaGetLastError();
 }
 
