@@ -33,7 +33,7 @@ constexpr uint32_t B_BYTES = BN * BK;
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;  // two accumulator buffers of 256 columns
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256;
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256 /*barriers*/ + 4 * 32 * 144 /*epilogue staging*/;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 
 // ---- thin PTX wrappers -------------------------------------------------------------------------
@@ -143,6 +143,57 @@ __host__ __device__ constexpr uint32_t make_idesc(int m, int n) {
     return (2u << 4) | (1u << 7) | (0u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// Epilogue staging: a warp holds a 32-row x 32-column block with one row per lane.  It is written to shared
+// memory (row stride 144 bytes keeps the eight 16-byte stores of a quarter warp on distinct banks), read back with
+// eight lanes per row, and stored with each instruction covering four whole 128-byte row segments.
+constexpr uint32_t STAGE_ROW_B32 = 144;
+constexpr uint32_t STAGE_ROW_B16 = 80;
+constexpr uint32_t STAGE_OUT_BYTES = 32 * STAGE_ROW_B32;  // per epilogue warp
+
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+// vals: this lane's row (32 x 32-bit).  dst: element (row 0, column 0) of the block in a row-major matrix of
+// leading dimension ld (elements); rows >= rows_ok are not stored.
+__device__ __forceinline__ void store_block_b32(const uint32_t (&vals)[32], uint32_t stage_s, uint32_t* dst, int ld,
+                                                int rows_ok, int lane) {
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+        sts128(stage_s + lane * STAGE_ROW_B32 + 16 * i, vals[4 * i], vals[4 * i + 1], vals[4 * i + 2], vals[4 * i + 3]);
+    __syncwarp();
+    const int sub = lane >> 3, piece = lane & 7;
+#pragma unroll
+    for (int it = 0; it < 8; ++it) {
+        const int row = 4 * it + sub;
+        const uint4 v = lds128(stage_s + row * STAGE_ROW_B32 + 16 * piece);
+        if (row < rows_ok) *reinterpret_cast<uint4*>(dst + (size_t)row * ld + 4 * piece) = v;
+    }
+    __syncwarp();
+}
+
+// Same for 16-bit elements: vals holds this lane's 32 columns as 16 packed words (64 bytes per row).
+__device__ __forceinline__ void store_block_b16(const uint32_t (&vals)[16], uint32_t stage_s, uint16_t* dst, int ld,
+                                                int rows_ok, int lane) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        sts128(stage_s + lane * STAGE_ROW_B16 + 16 * i, vals[4 * i], vals[4 * i + 1], vals[4 * i + 2], vals[4 * i + 3]);
+    __syncwarp();
+    const int sub = lane >> 2, piece = lane & 3;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+        const int row = 8 * it + sub;
+        const uint4 v = lds128(stage_s + row * STAGE_ROW_B16 + 16 * piece);
+        if (row < rows_ok) *reinterpret_cast<uint4*>(dst + (size_t)row * ld + 8 * piece) = v;
+    }
+    __syncwarp();
+}
+
 struct TileCoord {
     int m0, n0;
 };
@@ -247,6 +298,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
     } else {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
+        const uint32_t stage_s = smem_u32(smem + (size_t)STAGES * STAGE_BYTES + 256) + (uint32_t)quad * STAGE_OUT_BYTES;
         const float s_w = *s_w_ptr;
         bool ok = true;
         int iter = 0;
@@ -255,45 +307,40 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
             const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
             if (!mbar_wait(smem_u32(tfull_bar + buf), bphase, abort_flag)) { ok = false; break; }
             tc_fence_after();
-            const int m = tc.m0 + quad * 32 + lane;
+            const int m_warp = tc.m0 + quad * 32;  // first token row of this warp's 32 tensor-memory lanes
+            const int m = m_warp + lane;
             const bool row_ok = m < M;
             const int xs = row_ok ? xsum[m] : 0;
             const float dm = row_ok ? d[m] : 0.0f;
+            const int rows_ok = (M - m_warp) < 32 ? (M - m_warp) : 32;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + c * 32, r);
                 tmem_ld_wait();
                 const int n = tc.n0 + c * 32;
-                if (row_ok && n < N) {
-                    const size_t off = (size_t)m * N + n;
-                    int a[32];
+                if (n < N) {  // warp-uniform
+                    // Each lane holds 32 consecutive columns of ONE row.  The block goes through this warp's
+                    // shared-memory staging area so that every global store covers whole 128-byte row segments.
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) a[i] = (int)r[i] - xs;
-                    if (acc_out != nullptr) {
-                        int4* dst = reinterpret_cast<int4*>(acc_out + off);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) dst[i] = make_int4(a[4 * i], a[4 * i + 1], a[4 * i + 2], a[4 * i + 3]);
-                    }
-                    float v[32];
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __fmul_rn(__fmul_rn((float)a[i], s_w), dm);
+                    for (int i = 0; i < 32; ++i) r[i] = (uint32_t)((int)r[i] - xs);
+                    if (acc_out != nullptr)
+                        store_block_b32(r, stage_s, reinterpret_cast<uint32_t*>(acc_out) + (size_t)m_warp * N + n, N, rows_ok,
+                                        lane);
                     if (y_dtype == BITLINEAR_BF16) {
-                        uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(y) + off);
+                        uint32_t w[16];
 #pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            uint32_t w[4];
-#pragma unroll
-                            for (int e = 0; e < 4; ++e) {
-                                const __nv_bfloat162 p = __floats2bfloat162_rn(v[8 * i + 2 * e], v[8 * i + 2 * e + 1]);
-                                w[e] = *reinterpret_cast<const uint32_t*>(&p);
-                            }
-                            dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+                        for (int i = 0; i < 16; ++i) {
+                            const float v0 = __fmul_rn(__fmul_rn((float)(int)r[2 * i], s_w), dm);
+                            const float v1 = __fmul_rn(__fmul_rn((float)(int)r[2 * i + 1], s_w), dm);
+                            const __nv_bfloat162 p = __floats2bfloat162_rn(v0, v1);
+                            w[i] = *reinterpret_cast<const uint32_t*>(&p);
                         }
+                        store_block_b16(w, stage_s, reinterpret_cast<uint16_t*>(y) + (size_t)m_warp * N + n, N, rows_ok, lane);
                     } else {
-                        float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(y) + off);
 #pragma unroll
-                        for (int i = 0; i < 8; ++i) dst[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__fmul_rn((float)(int)r[i], s_w), dm));
+                        store_block_b32(r, stage_s, reinterpret_cast<uint32_t*>(y) + (size_t)m_warp * N + n, N, rows_ok, lane);
                     }
                 }
             }
