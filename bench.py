@@ -431,14 +431,16 @@ def run_case(args):
     path = {"gemv": bl.PATH_GEMV, "gemm": bl.PATH_GEMM}.get(args.case, bl.PATH_AUTO)
     ws = torch.empty(max(16, bl.bitlinear_matmul_workspace_bytes(M, n, k, path)), dtype=torch.uint8, device=dev)
     ws_p = torch.empty(bl.bitlinear_pack_workspace_bytes(n, k), dtype=torch.uint8, device=dev)
-    y = torch.empty(M, n, dtype=torch.float32, device=dev)
+    ydt = torch.bfloat16 if args.ydtype == "bf16" else torch.float32
+    y = torch.empty(M, n, dtype=ydt, device=dev)
     lib, st = bl.lib(), torch.cuda.current_stream().cuda_stream
 
     def one(i):
         p = copies[i % len(copies)]
         if args.case in ("gemv", "gemm"):
             rc = lib.bitlinear_matmul_q(xq.data_ptr(), d.data_ptr(), xsum.data_ptr(), p.data_ptr(), s_w.data_ptr(), M, n, k,
-                                        y.data_ptr(), 0, None, path, ws.data_ptr(), ws.numel(), st)
+                                        y.data_ptr(), 1 if args.ydtype == "bf16" else 0, None, path, ws.data_ptr(),
+                                        ws.numel(), st)
         elif args.case == "quant":
             rc = lib.bitlinear_quant_act(x.data_ptr(), gain.data_ptr(), wl.RMS_EPS, M, k, xq.data_ptr(), d.data_ptr(),
                                          xsum.data_ptr(), st)
@@ -470,6 +472,7 @@ def main():
     ap.add_argument("--shape", choices=list(wl.SHAPE_NK), default="q")
     ap.add_argument("--m", type=int, default=1)
     ap.add_argument("--copies", type=int, default=1)
+    ap.add_argument("--ydtype", choices=["f32", "bf16"], default="f32")
     args = ap.parse_args()
     if args.case:
         return run_case(args)

@@ -45,6 +45,33 @@ cudaError_t launch_gemv(const int8_t* xq, const float* d, const int32_t* xsum, c
                         const float* s_w, int M, int N, int K, void* y, int y_dtype, int32_t* acc_out,
                         cudaStream_t st);
 
+// One matmul of a group (device copy, read by the kernel through shared memory).
+struct GemmProblem {
+    const uint8_t* a_tiles;  // activations as 128 x 128 shared-memory tile images (A_TILED), else unused
+    const uint8_t* codes;    // weight codes as 256 x 128 shared-memory tile images
+    const float* d;
+    const int32_t* xsum;
+    const float* s_w;
+    void* y;
+    int32_t* acc_out;
+    int M, N, K, y_dtype;
+    int m_tiles;     // ceil(M / 128)
+    int tile_begin;  // tiles of the problems before this one
+};
+constexpr int kMaxGroup = 32;
+struct GemmGroupHeader {
+    int count, total_tiles, pad0, pad1;
+};
+// layout of the uploaded group table: GemmGroupHeader, then count x GemmProblem
+constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof(GemmProblem);
+
+// Grouped launch: fills m_tiles / tile_begin, uploads the table to table_dev (kGroupTableBytes) and runs every tile of
+// every problem in one persistent kernel.  a_tiled = activations given as tile images (any count), else one problem with
+// row-major activations.  Returns a bitlinear_status.
+int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev, cudaStream_t st);
+size_t gemm_codes_bytes(int N, int K);
+size_t gemm_a_tiles_bytes(int M, int K);
+
 // tcgen05 tensor-core GEMM on unpacked codes; returns a bitlinear_status.
 int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* codes, const float* s_w,
                  int M, int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st);

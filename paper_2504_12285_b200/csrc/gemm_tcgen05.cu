@@ -15,6 +15,7 @@
 // Every wait is bounded: if one runs out the CTA raises a sticky status word and leaves cleanly.
 #include <cuda.h>
 
+#include <cstring>
 #include <mutex>
 
 #include "common.cuh"
@@ -33,7 +34,7 @@ constexpr uint32_t B_BYTES = BN * BK;
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;  // two accumulator buffers of 256 columns
-constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256 /*barriers*/ + 4 * 32 * 144 /*epilogue staging*/;
+constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256 /*barriers*/ + 4 * 32 * 144 /*epilogue staging*/ + 3072 /*group table*/;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 
 // ---- thin PTX wrappers -------------------------------------------------------------------------
@@ -194,18 +195,22 @@ __device__ __forceinline__ void store_block_b16(const uint32_t (&vals)[16], uint
     __syncwarp();
 }
 
-struct TileCoord {
-    int m0, n0;
+// Tile -> (problem, token rows, weight rows).  Tiles of one problem are numbered with the token tile
+// fastest, so CTAs that run side by side share the weight tile; problems follow each other in table order.
+struct TileWalk {
+    const GemmProblem* probs;
+    int count, pi;
+    __device__ __forceinline__ const GemmProblem& find(int tile) {
+        while (pi + 1 < count && tile >= probs[pi + 1].tile_begin) ++pi;
+        return probs[pi];
+    }
 };
-__device__ __forceinline__ TileCoord tile_coord(int tile, int m_tiles) {
-    // consecutive tiles share the weight tile and walk over the tokens
-    return TileCoord{(tile % m_tiles) * BM, (tile / m_tiles) * BN};
-}
 
+// A_TILED: the activations come as tile images and are fetched with linear bulk copies (any group size);
+// otherwise the group holds one problem whose row-major activations are fetched through the tensor map.
+template <bool A_TILED>
 __global__ void __launch_bounds__(THREADS, 1)
-gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restrict__ codes,
-               const float* __restrict__ d, const int32_t* __restrict__ xsum, const float* __restrict__ s_w_ptr, int M,
-               int N, int K, void* __restrict__ y, int y_dtype, int32_t* __restrict__ acc_out, int* status_word) {
+gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restrict__ table_g, int* status_word) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)STAGES * STAGE_BYTES);
@@ -215,11 +220,12 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
     uint64_t* tempty_bar = tfull_bar + 2;      // [2] accumulator buffer drained by the epilogue
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint8_t* table_s = smem + (size_t)STAGES * STAGE_BYTES + 256 + 4 * STAGE_OUT_BYTES;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int m_tiles = (M + BM - 1) / BM, n_tiles = (N + BN - 1) / BN;
-    const int total_tiles = m_tiles * n_tiles;
-    const int k_blocks = K / BK;
+    // the group table goes to shared memory once; every role walks it on its own
+    for (int o = threadIdx.x * 16; o < (int)kGroupTableBytes; o += THREADS * 16)
+        *reinterpret_cast<uint4*>(table_s + o) = *reinterpret_cast<const uint4*>(table_g + o);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -244,21 +250,29 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    const GemmGroupHeader hdr = *reinterpret_cast<const GemmGroupHeader*>(table_s);
+    const int total_tiles = hdr.total_tiles;
+    TileWalk walk{reinterpret_cast<const GemmProblem*>(table_s + sizeof(GemmGroupHeader)), hdr.count, 0};
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ TMA producer
+        // ------------------------------------------------------------------ producer
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x) {
-                const TileCoord tc = tile_coord(tile, m_tiles);
+                const GemmProblem& p = walk.find(tile);
+                const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
+                const int k_blocks = p.K / BK;
+                const uint8_t* a_src = A_TILED ? p.a_tiles + (size_t)mt * k_blocks * A_BYTES : nullptr;
+                const uint8_t* b_src = p.codes + (size_t)nt * k_blocks * B_BYTES;
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = smem_u32(full_bar + stage);
                     mbar_expect_tx(fb, STAGE_BYTES);
                     const uint32_t sa = smem_u32(smem + (size_t)stage * STAGE_BYTES);
-                    tma_load_2d(sa, &map_a, kb * BK, tc.m0, fb);
-                    bulk_load(sa + A_BYTES, codes + ((size_t)(tc.n0 / BN) * k_blocks + kb) * B_BYTES, B_BYTES, fb);
+                    if (A_TILED) bulk_load(sa, a_src + (size_t)kb * A_BYTES, A_BYTES, fb);
+                    else tma_load_2d(sa, &map_a, kb * BK, mt * BM, fb);
+                    bulk_load(sa + A_BYTES, b_src + (size_t)kb * B_BYTES, B_BYTES, fb);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -272,6 +286,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
             bool ok = true;
             int iter = 0;
             for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++iter) {
+                const int k_blocks = walk.find(tile).K / BK;
                 const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
                 if (!mbar_wait(smem_u32(tempty_bar + buf), bphase ^ 1u, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -299,27 +314,31 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
         const uint32_t stage_s = smem_u32(smem + (size_t)STAGES * STAGE_BYTES + 256) + (uint32_t)quad * STAGE_OUT_BYTES;
-        const float s_w = *s_w_ptr;
         bool ok = true;
         int iter = 0;
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++iter) {
-            const TileCoord tc = tile_coord(tile, m_tiles);
+            const GemmProblem& p = walk.find(tile);
+            const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
+            const int M = p.M, N = p.N, y_dtype = p.y_dtype;
+            void* y = p.y;
+            int32_t* acc_out = p.acc_out;
+            const float s_w = *p.s_w;
             const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
-            if (!mbar_wait(smem_u32(tfull_bar + buf), bphase, abort_flag)) { ok = false; break; }
-            tc_fence_after();
-            const int m_warp = tc.m0 + quad * 32;  // first token row of this warp's 32 tensor-memory lanes
+            const int m_warp = mt * BM + quad * 32;  // first token row of this warp's 32 tensor-memory lanes
             const int m = m_warp + lane;
             const bool row_ok = m < M;
-            const int xs = row_ok ? xsum[m] : 0;
-            const float dm = row_ok ? d[m] : 0.0f;
+            const int xs = row_ok ? p.xsum[m] : 0;
+            const float dm = row_ok ? p.d[m] : 0.0f;
             const int rows_ok = (M - m_warp) < 32 ? (M - m_warp) : 32;
+            if (!mbar_wait(smem_u32(tfull_bar + buf), bphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + c * 32, r);
                 tmem_ld_wait();
-                const int n = tc.n0 + c * 32;
-                if (n < N) {  // warp-uniform
+                const int n = nt * BN + c * 32;
+                if (n < N && rows_ok > 0) {  // warp-uniform
                     // Each lane holds 32 consecutive columns of ONE row.  The block goes through this warp's
                     // shared-memory staging area so that every global store covers whole 128-byte row segments.
 #pragma unroll
@@ -333,8 +352,8 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
                         for (int i = 0; i < 16; ++i) {
                             const float v0 = __fmul_rn(__fmul_rn((float)(int)r[2 * i], s_w), dm);
                             const float v1 = __fmul_rn(__fmul_rn((float)(int)r[2 * i + 1], s_w), dm);
-                            const __nv_bfloat162 p = __floats2bfloat162_rn(v0, v1);
-                            w[i] = *reinterpret_cast<const uint32_t*>(&p);
+                            const __nv_bfloat162 pk = __floats2bfloat162_rn(v0, v1);
+                            w[i] = *reinterpret_cast<const uint32_t*>(&pk);
                         }
                         store_block_b16(w, stage_s, reinterpret_cast<uint16_t*>(y) + (size_t)m_warp * N + n, N, rows_ok, lane);
                     } else {
@@ -401,15 +420,19 @@ bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows)
 
 }  // namespace
 
-size_t gemm_scratch_bytes(int N, int K) { return (size_t)((N + BN - 1) / BN) * BN * K; }  // whole 256-row tiles
+size_t gemm_codes_bytes(int N, int K) { return (size_t)((N + BN - 1) / BN) * BN * K; }  // whole 256-row tiles
+size_t gemm_a_tiles_bytes(int M, int K) { return (size_t)((M + BM - 1) / BM) * BM * K; }  // whole 128-row tiles
+size_t gemm_scratch_bytes(int N, int K) { return align_up(gemm_codes_bytes(N, K), 256) + align_up(kGroupTableBytes, 256); }
 
-int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* codes, const float* s_w, int M,
-                 int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st) {
+int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev,
+                cudaStream_t st) {
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     static int sm_count = 0;
     std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(gemm_i8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
         int dev = 0;
         if (attr_err == cudaSuccess) attr_err = cudaGetDevice(&dev);
         if (attr_err == cudaSuccess) attr_err = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
@@ -418,13 +441,41 @@ int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const ui
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
+    if (count < 1 || count > kMaxGroup || (!a_tiled && count != 1)) return BITLINEAR_ERR_SHAPE;
+    alignas(16) uint8_t host[kGroupTableBytes] = {};
+    GemmGroupHeader* hdr = reinterpret_cast<GemmGroupHeader*>(host);
+    GemmProblem* tab = reinterpret_cast<GemmProblem*>(host + sizeof(GemmGroupHeader));
+    int tiles = 0;
+    for (int i = 0; i < count; ++i) {
+        probs[i].m_tiles = (probs[i].M + BM - 1) / BM;
+        probs[i].tile_begin = tiles;
+        tiles += probs[i].m_tiles * ((probs[i].N + BN - 1) / BN);
+        tab[i] = probs[i];
+    }
+    hdr->count = count;
+    hdr->total_tiles = tiles;
+    if (cudaMemcpyAsync(table_dev, host, kGroupTableBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
     CUtensorMap map_a;
-    if (!make_map(&map_a, xq, M, K, BM)) return BITLINEAR_ERR_CUDA;
-    const int tiles = ((M + BM - 1) / BM) * ((N + BN - 1) / BN);
+    memset(&map_a, 0, sizeof(map_a));
+    if (!a_tiled && !make_map(&map_a, xq_row_major, probs[0].M, probs[0].K, BM)) return BITLINEAR_ERR_CUDA;
     const int grid = tiles < sm_count ? tiles : sm_count;
-    gemm_i8_kernel<<<grid, THREADS, SMEM_BYTES, st>>>(map_a, codes, d, xsum, s_w, M, N, K, y, y_dtype, acc_out,
-                                                      device_status_word());
+    if (a_tiled) gemm_i8_kernel<true><<<grid, THREADS, SMEM_BYTES, st>>>(map_a, table_dev, device_status_word());
+    else gemm_i8_kernel<false><<<grid, THREADS, SMEM_BYTES, st>>>(map_a, table_dev, device_status_word());
     return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+
+// One matmul on row-major int8 activations; `scratch` holds the code tiles followed by the group table.
+int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* scratch, const float* s_w, int M,
+                 int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st) {
+    GemmProblem p = {};
+    p.codes = scratch;
+    p.d = d; p.xsum = xsum; p.s_w = s_w; p.y = y; p.acc_out = acc_out;
+    p.M = M; p.N = N; p.K = K; p.y_dtype = y_dtype;
+    uint8_t* table_dev = const_cast<uint8_t*>(scratch) + align_up(gemm_codes_bytes(N, K), 256);
+    return gemm_launch(&p, 1, false, xq, table_dev, st);
 }
 
 }  // namespace bitlinear
