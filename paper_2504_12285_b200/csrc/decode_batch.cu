@@ -84,7 +84,7 @@ __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHe
     const int row = blockIdx.x;
     const DevProblem& p = probs[row_prob[row]];
     const int m = row - p.row_begin;
-    quant_row<VPT, true>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq + (size_t)m * p.K, p.d + m, p.xsum + m, sm);
+    quant_row<VPT, 1>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq + (size_t)m * p.K, p.d + m, p.xsum + m, sm);
 }
 
 // ------------------------------------------------------------------------------------ launch 2
@@ -457,11 +457,15 @@ constexpr int kPlanGrid = 148 * 2;  // upper bound on the persistent grid used f
 
 }  // namespace bitlinear
 
-using namespace bitlinear;
+namespace bitlinear {
 
-extern "C" {
+size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const int* idx, int n);
+int prefill_group_forward(const bitlinear_problem* problems, const int* idx, int n, void* ws, bool skip_quant,
+                          cudaStream_t st);
 
-size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
+namespace {
+
+size_t decode_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
     if (!problems || count <= 0) return 0;
     size_t xq = 0, rows = 0;
     for (int i = 0; i < count; ++i) {
@@ -473,12 +477,8 @@ size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int co
     return plan_layout(count, kPlanGrid, xq, rows).total;
 }
 
-int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
-                            void* stream) {
-    if (count < 0) return BITLINEAR_ERR_SHAPE;
-    if (count == 0) return BITLINEAR_OK;
-    if (!problems) return BITLINEAR_ERR_NULL;
-    if (flags & ~(BITLINEAR_BATCH_REUSE_PLAN | BITLINEAR_BATCH_REUSE_ACT)) return BITLINEAR_ERR_DTYPE;
+int decode_batch_forward(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
+                         void* stream) {
     size_t xq_bytes = 0, rows = 0;
     int max_m = 0, max_k = 0;
     for (int i = 0; i < count; ++i) {
@@ -649,6 +649,83 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     if (mt == 1) e = stage_x ? launch_stream<1, 5, true>(prm, grid, smem, st) : launch_stream<1, 5, false>(prm, grid, smem, st);
     else e = stage_x ? launch_stream<4, 4, true>(prm, grid, smem, st) : launch_stream<4, 4, false>(prm, grid, smem, st);
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+
+}  // namespace
+
+}  // namespace bitlinear
+
+using namespace bitlinear;
+
+extern "C" {
+
+size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
+    if (!problems || count <= 0) return 0;
+    std::vector<bitlinear_problem> dec;
+    std::vector<int> pre;
+    for (int i = 0; i < count; ++i) {
+        const bitlinear_problem& q = problems[i];
+        if (q.M < 0 || !shape_ok(q.N, q.K)) return 0;
+        if (q.M <= kGemvMaxTokens) {
+            if (q.K > kBatchMaxK) return 0;
+            dec.push_back(q);
+        } else {
+            if (q.N % 128) return 0;
+            pre.push_back(i);
+        }
+    }
+    size_t total = 0;
+    if (!dec.empty()) total += align_up(decode_batch_workspace_bytes(dec.data(), (int)dec.size()), 1024);
+    if (!pre.empty()) total += prefill_group_workspace_bytes(problems, pre.data(), (int)pre.size());
+    return total;
+}
+
+int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
+                            void* stream) {
+    if (count < 0) return BITLINEAR_ERR_SHAPE;
+    if (count == 0) return BITLINEAR_OK;
+    if (!problems) return BITLINEAR_ERR_NULL;
+    if (flags & ~(BITLINEAR_BATCH_REUSE_PLAN | BITLINEAR_BATCH_REUSE_ACT)) return BITLINEAR_ERR_DTYPE;
+    std::vector<bitlinear_problem> dec;
+    std::vector<int> pre;
+    for (int i = 0; i < count; ++i) {
+        const bitlinear_problem& q = problems[i];
+        if (q.y_dtype != BITLINEAR_F32 && q.y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
+        if (q.M < 0 || !shape_ok(q.N, q.K)) return BITLINEAR_ERR_SHAPE;
+        if (q.M <= kGemvMaxTokens) {
+            if (q.K > kBatchMaxK) return BITLINEAR_ERR_SHAPE;
+            dec.push_back(q);
+            continue;
+        }
+        if (q.N % 128) return BITLINEAR_ERR_SHAPE;
+        if (!q.x || !q.packed || !q.s_w || !q.y) return BITLINEAR_ERR_NULL;
+        if (!aligned16(q.x) || !aligned16(q.packed) || !aligned16(q.y) || (q.gain && !aligned16(q.gain)) ||
+            (reinterpret_cast<uintptr_t>(q.s_w) & 3u))
+            return BITLINEAR_ERR_ALIGN;
+        pre.push_back(i);
+    }
+    const size_t dec_bytes = dec.empty() ? 0 : align_up(decode_batch_workspace_bytes(dec.data(), (int)dec.size()), 1024);
+    const size_t pre_bytes = pre.empty() ? 0 : prefill_group_workspace_bytes(problems, pre.data(), (int)pre.size());
+    if (!ws || !aligned16(ws) || ws_bytes < dec_bytes + pre_bytes) return BITLINEAR_ERR_WORKSPACE;
+    if (!dec.empty()) {
+        const int rc = decode_batch_forward(dec.data(), (int)dec.size(), flags, ws, dec_bytes, stream);
+        if (rc != BITLINEAR_OK) return rc;
+    }
+    if (!pre.empty()) {
+        if (int rc = [] {
+                int dev = 0, major = 0;
+                if (cudaGetDevice(&dev) != cudaSuccess ||
+                    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+                    cudaGetLastError();
+                    return (int)BITLINEAR_ERR_CUDA;
+                }
+                return major == 10 ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_ARCH;
+            }())
+            return rc;
+        return prefill_group_forward(problems, pre.data(), (int)pre.size(), static_cast<char*>(ws) + dec_bytes,
+                                     (flags & BITLINEAR_BATCH_REUSE_ACT) != 0, static_cast<cudaStream_t>(stream));
+    }
+    return BITLINEAR_OK;
 }
 
 int bitlinear_forward_batch_host(const bitlinear_problem* problems, int count, int flags, const void* x_host,

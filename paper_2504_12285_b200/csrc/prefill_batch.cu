@@ -1,0 +1,193 @@
+// Grouped prefill: several BitLinear forwards of more than 16 tokens each in three launches.
+// (Paper Section 5.1: packed weights are expanded on chip to a form the matrix units consume, then multiplied with
+// the 8-bit activations; here the expansion and the activation quantiser write directly the shared-memory images of
+// the tensor-core kernel's tiles, and one persistent kernel runs the tiles of every matmul of the group.)
+//
+//   launch 1  group_quant_kernel  : one warp per token - fused RMSNorm + absmax int8 quantiser; codes go into
+//                                   128 x 128 tile images (128-byte swizzle) of the activation operand.  Problems
+//                                   that read the same activations share one quantised copy.
+//   launch 2  group_unpack_kernel : packed 2-bit weights -> byte codes in 256 x 128 tile images.
+//   launch 3  gemm_i8_kernel<true>: every tile of every matmul, operands fetched with linear bulk copies.
+// Problems are ordered by decreasing K so that the long tiles are scheduled first and the tail is made of short ones.
+#include <algorithm>
+#include <vector>
+
+#include "quant_row.cuh"
+
+namespace bitlinear {
+
+namespace {
+
+struct PrefillItem {
+    const __nv_bfloat16* x;
+    const __nv_bfloat16* gain;
+    const uint32_t* packed;
+    uint8_t* a_tiles;
+    uint8_t* codes;
+    float* d;
+    int32_t* xsum;
+    long long word_begin;  // packed 32-bit words of the problems before this one
+    float eps;
+    int M, N, K;
+    int row_begin;  // tokens of the problems before this one
+    int pad;
+};
+constexpr size_t kItemTableBytes = kMaxGroup * sizeof(PrefillItem);
+
+template <int VPT>
+__global__ void __launch_bounds__(kQuantThreads) group_quant_kernel(const PrefillItem* __restrict__ items, int count) {
+    __shared__ RowReduceSmem sm;
+    const int row = blockIdx.x;
+    int i = 0;
+    while (i + 1 < count && row >= items[i + 1].row_begin) ++i;
+    const PrefillItem& p = items[i];
+    const int m = row - p.row_begin;
+    uint8_t* dst = p.a_tiles + (size_t)(m >> 7) * (p.K >> 7) * (128 * 128) + (size_t)(m & 127) * 128;
+    quant_row<VPT, 2>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, reinterpret_cast<int8_t*>(dst), p.d + m, p.xsum + m, sm,
+                      m & 7);
+}
+
+// Warp-per-row variant (eight rows per CTA).
+__global__ void __launch_bounds__(kQuantThreads) group_quant_warp_kernel(const PrefillItem* __restrict__ items, int count,
+                                                                         int rows) {
+    const int row = blockIdx.x * kQuantWarps + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    int i = 0;
+    while (i + 1 < count && row >= items[i + 1].row_begin) ++i;
+    const PrefillItem& p = items[i];
+    const int m = row - p.row_begin;
+    uint8_t* dst = p.a_tiles + (size_t)(m >> 7) * (p.K >> 7) * (128 * 128) + (size_t)(m & 127) * 128;
+    quant_row_warp<2>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, reinterpret_cast<int8_t*>(dst), p.d + m, p.xsum + m,
+                      m & 7);
+}
+
+// One thread expands one packed word (16 codes) into its 16-byte piece of a 256 x 128 tile image.
+__global__ void __launch_bounds__(256) group_unpack_kernel(const PrefillItem* __restrict__ items, int count,
+                                                           long long total_words) {
+    const long long word = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (word >= total_words) return;
+    int i = 0;
+    while (i + 1 < count && word >= items[i + 1].word_begin) ++i;
+    const PrefillItem& p = items[i];
+    const size_t w = (size_t)(word - p.word_begin);
+    const int k_tiles = p.K / kTileCols;
+    // position of packed word w (see "Packed weight layout" in bitlinear.h)
+    const size_t tile = w >> 8;
+    const int wo = (int)(w & 255);
+    const int h = wo >> 7, g = (wo >> 4) & 7, t = (wo >> 2) & 3, q = wo & 3;
+    const int n = (int)(tile / k_tiles) * kTileRows + 8 * h + g;
+    const int k0 = (int)(tile % k_tiles) * kTileCols + 64 * t + 16 * q;
+    const uint32_t v = p.packed[w];
+    const int r = n & 255, piece = (k0 & 127) >> 4;
+    const size_t img = (size_t)(n >> 8) * (p.K / 128) + (k0 >> 7);
+    *reinterpret_cast<uint4*>(p.codes + img * 32768 + (size_t)r * 128 + ((piece ^ (r & 7)) << 4)) =
+        make_uint4(v & 0x03030303u, (v >> 2) & 0x03030303u, (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
+}
+
+struct GroupLayout {
+    size_t table_off, items_off, total;
+    std::vector<size_t> a_off, codes_off, d_off, xsum_off;
+};
+
+GroupLayout group_layout(const bitlinear_problem* problems, const int* idx, int n) {
+    GroupLayout L;
+    size_t off = 0;
+    L.table_off = off;
+    off = align_up(off + kGroupTableBytes, 256);
+    L.items_off = off;
+    off = align_up(off + kItemTableBytes, 256);
+    for (int i = 0; i < n; ++i) {
+        const bitlinear_problem& q = problems[idx[i]];
+        L.a_off.push_back(off);
+        off = align_up(off + gemm_a_tiles_bytes(q.M, q.K), 1024);
+        L.codes_off.push_back(off);
+        off = align_up(off + gemm_codes_bytes(q.N, q.K), 1024);
+        L.d_off.push_back(off);
+        off = align_up(off + (size_t)q.M * sizeof(float), 256);
+        L.xsum_off.push_back(off);
+        off = align_up(off + (size_t)q.M * sizeof(int32_t), 256);
+    }
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+// Workspace of a group of prefill problems (problems[idx[0..n)], every M > 16); at most kMaxGroup per launch group,
+// larger sets are run as consecutive groups over the same layout.
+size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const int* idx, int n) {
+    size_t total = 0;
+    for (int b = 0; b < n; b += kMaxGroup) total += group_layout(problems, idx + b, std::min(kMaxGroup, n - b)).total;
+    return total;
+}
+
+int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, int n_in, void* ws, bool skip_quant,
+                          cudaStream_t st) {
+    char* base_all = static_cast<char*>(ws);
+    for (int b = 0; b < n_in; b += kMaxGroup) {
+        const int n = std::min(kMaxGroup, n_in - b);
+        std::vector<int> idx(idx_in + b, idx_in + b + n);
+        std::stable_sort(idx.begin(), idx.end(), [&](int l, int r) { return problems[l].K > problems[r].K; });
+        const GroupLayout L = group_layout(problems, idx.data(), n);
+        char* base = base_all;
+        base_all += L.total;
+
+        PrefillItem items[kMaxGroup] = {};
+        GemmProblem gp[kMaxGroup] = {};
+        long long words = 0;
+        int rows = 0, max_k = 0;
+        for (int i = 0; i < n; ++i) {
+            const bitlinear_problem& q = problems[idx[i]];
+            PrefillItem& it = items[i];
+            it.x = static_cast<const __nv_bfloat16*>(q.x);
+            it.gain = static_cast<const __nv_bfloat16*>(q.gain);
+            it.packed = static_cast<const uint32_t*>(q.packed);
+            it.a_tiles = reinterpret_cast<uint8_t*>(base + L.a_off[i]);
+            it.codes = reinterpret_cast<uint8_t*>(base + L.codes_off[i]);
+            it.d = reinterpret_cast<float*>(base + L.d_off[i]);
+            it.xsum = reinterpret_cast<int32_t*>(base + L.xsum_off[i]);
+            it.word_begin = words;
+            it.eps = q.rms_eps;
+            it.M = q.M; it.N = q.N; it.K = q.K;
+            it.row_begin = rows;
+            words += (long long)q.N * q.K / 16;
+            // problems that read the same activations (q/k/v, gate/up of a layer) share one quantised copy
+            int same = -1;
+            for (int j = 0; j < i && same < 0; ++j) {
+                const bitlinear_problem& o = problems[idx[j]];
+                if (o.x == q.x && o.gain == q.gain && o.rms_eps == q.rms_eps && o.M == q.M && o.K == q.K) same = j;
+            }
+            if (same >= 0) {
+                it.a_tiles = items[same].a_tiles; it.d = items[same].d; it.xsum = items[same].xsum;
+            } else {
+                rows += q.M;
+            }
+            if (q.K > max_k) max_k = q.K;
+            GemmProblem& g = gp[i];
+            g.a_tiles = it.a_tiles; g.codes = it.codes; g.d = it.d; g.xsum = it.xsum; g.s_w = q.s_w;
+            g.y = q.y; g.acc_out = nullptr;
+            g.M = q.M; g.N = q.N; g.K = q.K; g.y_dtype = q.y_dtype;
+        }
+        PrefillItem* items_dev = reinterpret_cast<PrefillItem*>(base + L.items_off);
+        if (cudaMemcpyAsync(items_dev, items, sizeof(PrefillItem) * n, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return BITLINEAR_ERR_CUDA;
+        }
+        const int vpt = (max_k / 8 + kQuantThreads - 1) / kQuantThreads;
+        const dim3 g((unsigned)rows), blk(kQuantThreads), gw((unsigned)((rows + kQuantWarps - 1) / kQuantWarps));
+        if (skip_quant) {
+        } else if (true) group_quant_warp_kernel<<<gw, blk, 0, st>>>(items_dev, n, rows);
+        else if (vpt <= 1) group_quant_kernel<1><<<g, blk, 0, st>>>(items_dev, n);
+        else if (vpt <= 2) group_quant_kernel<2><<<g, blk, 0, st>>>(items_dev, n);
+        else if (vpt <= 4) group_quant_kernel<4><<<g, blk, 0, st>>>(items_dev, n);
+        else group_quant_kernel<8><<<g, blk, 0, st>>>(items_dev, n);
+        if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+        group_unpack_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(items_dev, n, words);
+        if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+        const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st);
+        if (rc != BITLINEAR_OK) return rc;
+    }
+    return BITLINEAR_OK;
+}
+
+}  // namespace bitlinear

@@ -16,13 +16,28 @@ __global__ void __launch_bounds__(kQuantThreads) quant_act_kernel(const __nv_bfl
     quant_row<VPT>(x + row * K, gain, eps, K, xq + row * K, d_out + row, xsum_out ? xsum_out + row : nullptr, sm);
 }
 
+// Many tokens: one warp per token, eight tokens per CTA.
+__global__ void __launch_bounds__(kQuantThreads) quant_act_warp_kernel(const __nv_bfloat16* __restrict__ x,
+                                                                       const __nv_bfloat16* __restrict__ gain, float eps,
+                                                                       int M, int K, int8_t* __restrict__ xq,
+                                                                       float* __restrict__ d_out,
+                                                                       int32_t* __restrict__ xsum_out) {
+    const size_t row = (size_t)blockIdx.x * kQuantWarps + (threadIdx.x >> 5);
+    if (row >= (size_t)M) return;
+    quant_row_warp<0>(x + row * K, gain, eps, K, xq + row * K, d_out + row, xsum_out ? xsum_out + row : nullptr);
+}
+
 }  // namespace
 
 cudaError_t launch_quant_act(const __nv_bfloat16* x, const __nv_bfloat16* gain, float eps, int M, int K,
                              int8_t* xq, float* d, int32_t* xsum, cudaStream_t st) {
     const int n_vec = K / 8;
     const int vpt = (n_vec + kQuantThreads - 1) / kQuantThreads;
-    const dim3 grid((unsigned)M), block(kQuantThreads);
+    const dim3 grid((unsigned)M), block(kQuantThreads), gw((unsigned)((M + kQuantWarps - 1) / kQuantWarps));
+    if (M >= 64) {
+        quant_act_warp_kernel<<<gw, block, 0, st>>>(x, gain, eps, M, K, xq, d, xsum);
+        return cudaGetLastError();
+    }
     if (vpt <= 1) quant_act_kernel<1><<<grid, block, 0, st>>>(x, gain, eps, K, xq, d, xsum);
     else if (vpt <= 2) quant_act_kernel<2><<<grid, block, 0, st>>>(x, gain, eps, K, xq, d, xsum);
     else if (vpt <= 4) quant_act_kernel<4><<<grid, block, 0, st>>>(x, gain, eps, K, xq, d, xsum);

@@ -16,6 +16,7 @@ constexpr int kQuantWarps = kQuantThreads / 32;
 
 struct RowReduceSmem {
     double sq[kQuantWarps];
+    float r;
     float mx[kQuantWarps];
     int sum[kQuantWarps];
 };
@@ -29,15 +30,31 @@ __device__ __forceinline__ void unpack_bf16x8(const uint4& u, float (&f)[8]) {
     }
 }
 
+// Round-half-even of a float with |v| < 2^22 to an integer whose low byte is the int8 code: adding 1.5 * 2^23 leaves
+// the rounded integer in the low mantissa bits (one full-rate add instead of a conversion).  |v| <= 127 * (1 + 2^-24)
+// by construction of the absmax scale, so the clip to [-128, 127] of the definition is the identity and is not coded.
+__device__ __forceinline__ uint32_t round_code(float v) { return __float_as_uint(__fadd_rn(v, 12582912.0f)); }
+
+// Packs the low bytes of four round_code results into one word and adds their (signed) sum to csum.
+__device__ __forceinline__ uint32_t pack_codes4(uint32_t a, uint32_t b, uint32_t c, uint32_t d, int& csum) {
+    const uint32_t w = __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+    asm("dp4a.s32.s32 %0, %1, %2, %0;" : "+r"(csum) : "r"(w), "r"(0x01010101));
+    return w;
+}
+
 // Quantises one row with the kQuantThreads threads of the calling CTA (all must call it).
-// PERM = false: codes are stored in column order.  PERM = true: inside every block of 256 columns the
-// sixteen 16-byte pieces are stored transposed (piece 4t+q, columns 64t+16q .. +15, at byte 64q+16t), the
-// order in which the four column lanes of the batched decode kernel read them.
-template <int VPT, bool PERM = false>  // VPT = 16-byte vectors (8 bf16) per thread
+// LAYOUT 0: codes are stored in column order.
+// LAYOUT 1: inside every block of 256 columns the sixteen 16-byte pieces are stored transposed (piece 4t+q,
+//           columns 64t+16q .. +15, at byte 64q+16t), the order in which the four column lanes of the batched
+//           decode kernel read them.
+// LAYOUT 2: tensor-core tile images: xq_row points at this row inside the first 128-row x 128-column tile of its
+//           row tile (tiles of 16 KiB follow each other along K); 16-byte piece p of a row sits at (p ^ swz) * 16,
+//           swz = row & 7 - the 128-byte shared-memory swizzle.
+template <int VPT, int LAYOUT = 0>  // VPT = 16-byte vectors (8 bf16) per thread
 __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_row,
                                           const __nv_bfloat16* __restrict__ gain, float eps, int K,
                                           int8_t* __restrict__ xq_row, float* __restrict__ d_out,
-                                          int32_t* __restrict__ xsum_out, RowReduceSmem& sm) {
+                                          int32_t* __restrict__ xsum_out, RowReduceSmem& sm, int swz = 0) {
     const int n_vec = K >> 3;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint4* xrow = reinterpret_cast<const uint4*>(x_row);
@@ -58,18 +75,22 @@ __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_ro
         unpack_bf16x8(xv[i], f);
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
-            const double v = (double)f[e];
-            sq += v * v;
+            const double t = (double)f[e];
+            sq += t * t;  // each square of a bf16 value is exact
         }
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
     if (lane == 0) sm.sq[warp] = sq;
     __syncthreads();
-    double S = 0.0;
+    if (tid == 0) {  // one thread does the fp64 divide and square root
+        double S = 0.0;
 #pragma unroll
-    for (int w = 0; w < kQuantWarps; ++w) S += sm.sq[w];
-    const float r = (float)(1.0 / sqrt(S / (double)K + (double)eps));
+        for (int w = 0; w < kQuantWarps; ++w) S += sm.sq[w];
+        sm.r = (float)(1.0 / sqrt(S / (double)K + (double)eps));
+    }
+    __syncthreads();
+    const float r = sm.r;
 
     // ---- normalise (kept in registers) and find the absolute maximum ----
     float y[VPT][8];
@@ -107,18 +128,18 @@ __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_ro
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int v = tid + i * kQuantThreads;
-        uint32_t packed[2] = {0u, 0u};
+        uint32_t c[8], packed[2];
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            int q = __float2int_rn(__fmul_rn(y[i][e], s));
-            q = max(-128, min(127, q));
-            csum += q;
-            packed[e >> 2] |= (uint32_t)(q & 0xff) << (8 * (e & 3));
-        }
+        for (int e = 0; e < 8; ++e) c[e] = round_code(__fmul_rn(y[i][e], s));
+        packed[0] = pack_codes4(c[0], c[1], c[2], c[3], csum);
+        packed[1] = pack_codes4(c[4], c[5], c[6], c[7], csum);
         int dst = v;  // in units of 8 codes
-        if (PERM) {
+        if (LAYOUT == 1) {
             const int piece = (v >> 1) & 15;  // 16-byte piece inside the 256-column block: 4t + q
             dst = (v & ~31) | ((((piece & 3) << 2) | (piece >> 2)) << 1) | (v & 1);
+        } else if (LAYOUT == 2) {
+            const int kb = v >> 4, piece = (v >> 1) & 7;  // 128-column tile along K, 16-byte piece in the row
+            dst = kb * (128 * 128 / 8) + (((piece ^ swz) << 1) | (v & 1));
         }
         if (v < n_vec) qrow[dst] = make_uint2(packed[0], packed[1]);
     }
@@ -135,5 +156,90 @@ __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_ro
     }
 }
 
+
+// Warp-per-row variant for many-token calls: the same arithmetic with one warp owning a whole row (16-byte
+// vector v of the row belongs to lane v % 32), so a CTA of kQuantThreads threads quantises eight rows with no
+// block-wide barrier.  The row is read from HBM once; the second and third pass read it again (it is still in
+// L1 / L2), which keeps the register count low and no shared memory is needed, so many rows are in flight per SM.
+template <int LAYOUT = 0>
+__device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__ x_row,
+                                               const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                               int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                               int32_t* __restrict__ xsum_out, int swz = 0) {
+    const int n_vec = K >> 3;
+    const int lane = threadIdx.x & 31;
+    const uint4* xrow = reinterpret_cast<const uint4*>(x_row);
+    const uint4* grow = reinterpret_cast<const uint4*>(gain);
+    double sq = 0.0;
+#pragma unroll 4
+    for (int v = lane; v < n_vec; v += 32) {
+        const uint4 u = xrow[v];
+        float f[8];
+        unpack_bf16x8(u, f);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const double t = (double)f[e];
+            sq += t * t;  // each square of a bf16 value is exact
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    float r = 0.0f;
+    if (lane == 0) r = (float)(1.0 / sqrt(sq / (double)K + (double)eps));  // one lane does the fp64 divide and root
+    r = __shfl_sync(0xffffffffu, r, 0);
+
+    float amax = 0.0f;
+#pragma unroll 2
+    for (int v = lane; v < n_vec; v += 32) {
+        float f[8], g[8];
+        unpack_bf16x8(xrow[v], f);
+        if (gain != nullptr) {
+            unpack_bf16x8(grow[v], g);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = 1.0f;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(__fmul_rn(__fmul_rn(f[e], r), g[e])));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    const float a = fmaxf(amax, 1e-5f);
+    const float s = __fdiv_rn(127.0f, a);
+
+    int csum = 0;
+    uint2* qrow = reinterpret_cast<uint2*>(xq_row);
+#pragma unroll 2
+    for (int v = lane; v < n_vec; v += 32) {
+        float f[8], g[8];
+        unpack_bf16x8(xrow[v], f);
+        if (gain != nullptr) {
+            unpack_bf16x8(grow[v], g);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = 1.0f;
+        }
+        uint32_t c[8], packed[2];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) c[e] = round_code(__fmul_rn(__fmul_rn(__fmul_rn(f[e], r), g[e]), s));
+        packed[0] = pack_codes4(c[0], c[1], c[2], c[3], csum);
+        packed[1] = pack_codes4(c[4], c[5], c[6], c[7], csum);
+        int dst = v;  // in units of 8 codes
+        if (LAYOUT == 1) {
+            const int piece = (v >> 1) & 15;
+            dst = (v & ~31) | ((((piece & 3) << 2) | (piece >> 2)) << 1) | (v & 1);
+        } else if (LAYOUT == 2) {
+            const int kb = v >> 4, piece = (v >> 1) & 7;
+            dst = kb * (128 * 128 / 8) + (((piece ^ swz) << 1) | (v & 1));
+        }
+        qrow[dst] = make_uint2(packed[0], packed[1]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xffffffffu, csum, o);
+    if (lane == 0) {
+        *d_out = __fdiv_rn(a, 127.0f);
+        if (xsum_out != nullptr) *xsum_out = csum;
+    }
+}
 
 }  // namespace bitlinear

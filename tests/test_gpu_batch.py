@@ -128,3 +128,31 @@ def test_batch_detects_an_overwritten_plan():
     bl.bitlinear_forward_batch(batch, ws)  # a fresh upload repairs it
     torch.cuda.synchronize()
     check(batch, refs)
+
+
+# ---- problems of more than 16 tokens in the same entry point: grouped tensor-core path ----
+
+
+def test_batch_prefill_group_small_mixed_shapes():
+    # ragged token counts (not multiples of the 128-row tile), several tiles along N and K, different K per problem
+    shapes = [(96, 256, 512), (130, 640, 2560), (17, 128, 256), (300, 384, 768)]
+    batch, refs = make_case(shapes, 700, gains=True)
+    run(batch)
+    check(batch, refs)
+
+
+def test_batch_prefill_group_bf16_and_decode_problems_together():
+    # decode-sized and prefill-sized problems in one call: each goes to its own kernel
+    shapes = [(1, 640, 2560), (64, 256, 1024), (4, 48, 768), (200, 128, 512)]
+    batch, refs = make_case(shapes, 800, y_dtype=torch.bfloat16)
+    run(batch, reuse=True)
+    check(batch, refs)
+
+
+def test_batch_prefill_group_matches_single_forward_bitwise():
+    shapes = [(256, 640, 2560), (256, 2560, 2560)]
+    batch, _ = make_case(shapes, 900)
+    run(batch)
+    for x, g, packed, s_w, y in batch.tensors:
+        y1 = bl.bitlinear_forward(x, g, packed, s_w, y.shape[1], wl.RMS_EPS)
+        assert torch.equal(y, y1)
