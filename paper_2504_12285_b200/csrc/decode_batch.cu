@@ -10,17 +10,18 @@
 //             block of 16 weight rows of every problem; each CTA owns a contiguous, byte-balanced
 //             range of it.  A row block belongs to ONE group of G warps (G = 1 for up to four tokens;
 //             each warp of a group takes up to four tokens), so 16/G row blocks are in progress per
-//             CTA and no partial sum ever crosses a warp.  Each warp runs its own pipeline: lane 0
-//             issues a linear bulk copy (cp.async.bulk, a few contiguous 16x256 tiles) into one of
-//             the warp's two shared-memory slots and the warp waits on that slot's mbarrier,
-//             multiplies, and refills the slot it has just read - across row-block and matrix
-//             boundaries, so HBM requests are always in flight (16 issuing threads, ~80 KiB in flight
-//             per SM).  Nothing is handed from warp to warp.
+//             CTA and no partial sum ever crosses a warp.  Each group runs its own pipeline: one
+//             thread issues a linear bulk copy (cp.async.bulk, a few contiguous 16x256 tiles) into one
+//             of the group's two shared-memory slots; its warps wait on that slot's mbarrier, multiply,
+//             and the slot is refilled once they have all read it - across row-block and matrix
+//             boundaries, so HBM requests are always in flight (with G = 1: 16 issuing threads, ~80 KiB
+//             in flight per SM, and nothing is handed from warp to warp).
 //             Before the stream starts the CTA copies the descriptors of the few problems its range
 //             touches, and their quantised activations, into shared memory once.
 //             Unpack: word & (0x03030303 << 2j) is 4^j x the codes of four consecutive columns, fed
 //             to a dot-product-of-four with the int8 activations; one accumulator per j keeps the
 //             scale uniform and the four are folded once per row block.
+#include <type_traits>
 #include <vector>
 
 #include "quant_row.cuh"
@@ -63,10 +64,11 @@ __device__ __forceinline__ bool plan_matches(const PlanHeader* h, int count, int
 
 constexpr int kStreamWarps = 16;
 constexpr int kStreamThreads = kStreamWarps * 32;
-constexpr int kRing = 2;  // chunk slots per warp
+constexpr int kRing = 2;  // chunk slots per group of warps that share a row block
 constexpr int kBatchMaxK = 8192;
-constexpr size_t ring_bytes(int chunk_tiles) {
-    return (size_t)kStreamWarps * kRing * chunk_tiles * kTileBytes + kStreamWarps * kRing * 8 + 128;
+constexpr size_t kBarBytes = (size_t)kStreamWarps * kRing * 2 * 8 + 128;  // full + empty barriers, abort flag
+constexpr size_t ring_bytes(int chunk_tiles, int groups) {
+    return (size_t)(kStreamWarps / groups) * kRing * chunk_tiles * kTileBytes + kBarBytes;
 }
 
 // ------------------------------------------------------------------------------------ launch 1
@@ -112,6 +114,7 @@ struct StreamParams {
     int count, total_rb, rows;
     int groups;     // G: warps that share a row block, each taking MT tokens
     int table_cap;  // problems of a CTA whose descriptors are cached in shared memory
+    int arena_bytes;  // shared memory available for staged activations
     int* status_word;
 };
 
@@ -148,27 +151,32 @@ struct ChunkCursor {
 };
 
 // MT = tokens per warp (1 or 4).  kChunkTiles = 16x256 tiles (1 KiB each) per bulk copy at most.
-// XS = the quantised activations of every problem the CTA touches are staged in shared memory once
-// (otherwise they are read through L1, which is slower).
-template <int MT, int kChunkTiles, bool XS>
+// The quantised activations of the problems the CTA touches are staged in shared memory once, as far as the arena
+// reaches; those of the remaining problems are read through L1, which is slower.
+template <int MT, int kChunkTiles>
 __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const StreamParams prm) {
     extern __shared__ __align__(128) uint8_t smem[];
-    // [ring: warps x kRing slots][barriers][abort flag][descriptor table][activation arena]
+    // [ring: (16 / G) row-block lanes x kRing slots][full barriers][empty barriers][abort flag][descriptor table]
+    // [activation arena]
     constexpr uint32_t kSlotBytes = kChunkTiles * kTileBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kStreamWarps * kRing * kSlotBytes);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kStreamWarps * kRing);
-    SProb* table = reinterpret_cast<SProb*>(reinterpret_cast<uint8_t*>(bars) + kStreamWarps * kRing * 8 + 128);
+    const int G = prm.groups;
+    const int par = kStreamWarps / G;  // row blocks in progress at a time in this CTA
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)par * kRing * kSlotBytes);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStreamWarps * kRing);
+    SProb* table = reinterpret_cast<SProb*>(reinterpret_cast<uint8_t*>(bars) + kBarBytes);
     uint8_t* arena = reinterpret_cast<uint8_t*>(table) + (size_t)prm.table_cap * sizeof(SProb);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int G = prm.groups;
     if (!plan_matches(prm.hdr, prm.count, prm.total_rb, (int)gridDim.x, prm.rows)) {  // uniform over the grid
         if (blockIdx.x == 0 && threadIdx.x == 0 && prm.status_word != nullptr)
             atomicExch(prm.status_word, BITLINEAR_ERR_WORKSPACE);
         return;
     }
-    if (lane == 0) {
-        for (int r = 0; r < kRing; ++r) mbar_init(smem_u32(bars + warp * kRing + r), 1);
+    if (lane == 0 && warp < par) {  // warp i sets up the barriers of row-block lane i
+        for (int r = 0; r < kRing; ++r) {
+            mbar_init(smem_u32(bars + warp * kRing + r), 1);                          // full: the copy landed
+            mbar_init(smem_u32(bars + kStreamWarps * kRing + warp * kRing + r), G);   // empty: all G warps have read it
+        }
         if (warp == 0) *abort_flag = 0;
         mbar_init_fence();
     }
@@ -178,12 +186,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     const int n_local = rb_lo < rb_hi ? range.w - p_lo + 1 : 0;
     const int n_tab = n_local < prm.table_cap ? n_local : prm.table_cap;
     const DevProblem* probs = prm.probs;
-    const int par = kStreamWarps / G;             // row blocks in progress at a time in this CTA
-    const int rl = warp / G, tg = warp - rl * G;  // which of them this warp works on, and its token group
+    const int rl = warp / G, tg = warp - rl * G;  // the row-block lane this warp works on, and its token group
     const bool mine = rl < par && rb_lo + rl < rb_hi;
     const int g = lane >> 2, t = lane & 3;
-    const uint32_t ring_s = smem_u32(smem) + (uint32_t)warp * kRing * kSlotBytes;
-    const uint32_t bar_s = smem_u32(bars + warp * kRing);
+    const uint32_t ring_s = smem_u32(smem) + (uint32_t)rl * kRing * kSlotBytes;
+    const uint32_t bar_s = smem_u32(bars + rl * kRing);                            // full barriers of this lane
+    const uint32_t ebar_s = smem_u32(bars + kStreamWarps * kRing + rl * kRing);    // empty barriers
+    const bool issuer = tg == 0 && lane == 0;  // the one thread of the group that issues its copies
 
     // descriptor of the next problem that holds row block c.rb: from the shared-memory table when it is there
     auto enter = [&](ChunkCursor& c) {
@@ -203,7 +212,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     };
 
     // ---- start the weight stream before anything else: the first chunks come from one problem ----
-    // Every warp of a token group issues its own copy of the chunk (the later readers hit L2).
+    // The warps of a group share the lane's ring: one thread issues, every warp of the group reads.
     ChunkCursor ld;  // where the next copy comes from
     ld.rb = rb_lo + rl; ld.c = 0; ld.p = p_lo;
     ld.rb_begin = 0; ld.rb_end = 0; ld.k_tiles = 1; ld.nc = 1; ld.ct = 1; ld.base = nullptr;
@@ -230,7 +239,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
 #pragma unroll
     for (int r = 0; r < kRing; ++r)
         if (ld_valid && ld.rb < ld.rb_end) {
-            if (lane == 0) issue(r);
+            if (issuer) issue(r);
             primed = r + 1;
             advance_ld(false);
         }
@@ -253,17 +262,23 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         }
     }
     __syncthreads();
-    if (XS) {
+    {
         if (threadIdx.x == 0) {
             int off = 0;
             for (int i = 0; i < n_tab; ++i) {
-                table[i].x_off = off;
-                off += table[i].M * table[i].K;  // a multiple of 256
+                const int bytes = table[i].M * table[i].K;  // a multiple of 256
+                if (off + bytes <= prm.arena_bytes) {
+                    table[i].x_off = off;
+                    off += bytes;
+                } else {
+                    table[i].x_off = -1;  // does not fit: read through L1
+                }
             }
         }
         __syncthreads();
         const uint32_t arena_s = smem_u32(arena);
         for (int i = 0; i < n_tab; ++i) {
+            if (table[i].x_off < 0) continue;
             const int bytes = table[i].M * table[i].K;
             const int8_t* src = table[i].xq;
             const uint32_t dst = arena_s + (uint32_t)table[i].x_off;
@@ -280,7 +295,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
 #pragma unroll
         for (int r = 0; r < kRing; ++r)
             if (r >= primed && ld_valid) {
-                if (lane == 0) issue(r);
+                if (issuer) issue(r);
                 advance_ld(true);
             }
 
@@ -288,13 +303,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         int M = 0, N = 0, y_dtype = 0, xs_lane = 0;
         void* y = nullptr;
         float s_w = 0.0f, d_lane = 0.0f;
-        bool active = false;
-        const int8_t* xrow_g[MT];  // !XS: token rows in global memory
-        uint32_t xrow_s[MT];       //  XS: token rows in the shared-memory arena
+        bool active = false, x_staged = false;
+        const int8_t* xrow_g[MT];  // token rows in global memory
+        uint32_t xrow_s[MT];       // token rows in the shared-memory arena (when staged)
         auto load_problem_state = [&]() {
             const int i = cp.p - p_lo;
             const int my_tok = tg * MT + (MT == 1 ? 0 : t);  // lane t finishes token tg*MT + t
-            int K = 0, x_off = 0;
+            int K = 0, x_off = -1;
             const int8_t* xq = nullptr;
             if (i < n_tab) {
                 const SProb& e = table[i];
@@ -308,12 +323,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                 xs_lane = my_tok < M ? pr.xsum[my_tok] : 0;
             }
             active = tg * MT < M;  // warp-uniform: this token group holds real tokens
+            x_staged = x_off >= 0;
 #pragma unroll
             for (int m = 0; m < MT; ++m) {
                 int tok = tg * MT + m;
                 if (tok > M - 1) tok = M - 1;  // padding tokens re-read a real row; their sums are dropped
                 xrow_g[m] = xq + (size_t)tok * K + t * 16;
-                xrow_s[m] = smem_u32(arena) + (uint32_t)(x_off + tok * K + t * 16);
+                xrow_s[m] = smem_u32(arena) + (uint32_t)((x_staged ? x_off : 0) + tok * K + t * 16);
             }
         };
         load_problem_state();
@@ -332,7 +348,8 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             const uint32_t slot = n_chunk % kRing, phase = (n_chunk / kRing) & 1u;
             if (!mbar_wait(bar_s + 8u * slot, phase, abort_flag)) { ok = false; break; }
             const int tiles = cp.tiles();
-            if (active) {
+            auto run_tiles = [&](auto staged) {
+                constexpr bool XS = decltype(staged)::value;  // activations of this problem are in the arena
                 uint32_t wa = ring_s + slot * kSlotBytes + (uint32_t)lane * 16u;
                 uint32_t xo = (uint32_t)(cp.c * cp.ct) * kTileCols;
 #pragma unroll 2
@@ -364,10 +381,16 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                         }
                     }
                 }
+            };
+            if (active) {
+                if (x_staged) run_tiles(std::true_type{});
+                else run_tiles(std::false_type{});
             }
-            __syncwarp();  // every lane has read the slot: it may be refilled
+            __syncwarp();  // every lane of this warp has read the slot
+            if (lane == 0) mbar_arrive(ebar_s + 8u * slot);
             if (ld_valid) {
-                if (lane == 0) issue((int)slot);
+                // refill once all G warps of the group have read it
+                if (issuer && mbar_wait(ebar_s + 8u * slot, phase, abort_flag)) issue((int)slot);
                 advance_ld(true);
             }
             ++n_chunk;
@@ -421,12 +444,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (*abort_flag && threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
 }
 
-template <int MT, int kChunkTiles, bool XS>
+template <int MT, int kChunkTiles>
 cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<MT, kChunkTiles, XS>,
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<MT, kChunkTiles>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    decode_stream_kernel<MT, kChunkTiles, XS><<<grid, kStreamThreads, smem, st>>>(prm);
+    decode_stream_kernel<MT, kChunkTiles><<<grid, kStreamThreads, smem, st>>>(prm);
     return cudaGetLastError();
 }
 
@@ -590,17 +613,15 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
             }
         }
     }
-    // shared memory: chunk ring + descriptor table + activation arena; when that does not fit, the activations
-    // are read through L1 instead and only as many descriptors as fit are cached
+    // shared memory: chunk ring + descriptor table + activation arena; activations that do not fit the arena are read
+    // through L1 instead, and only as many descriptors as fit a quarter of the space are cached
     const int mt = max_m <= 1 ? 1 : 4;
     const int chunk_tiles = mt == 1 ? 5 : 4;
-    const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles) - 128;
-    bool stage_x = true;
-    if ((size_t)table_cap * sizeof(SProb) + arena_max > smem_limit) {
-        stage_x = false;
-        arena_max = 0;
-        if ((size_t)table_cap * sizeof(SProb) > smem_limit) table_cap = (int)(smem_limit / sizeof(SProb));
-    }
+    const int groups = (max_m + mt - 1) / mt;  // 1 .. 4
+    const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles, groups) - 128;
+    if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
+    if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
+    arena_max &= ~(size_t)255;
 
     PlanHeader hdr_host;
     hdr_host.magic = kPlanMagic;
@@ -642,12 +663,13 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.total_rb = total_rb;
     prm.rows = (int)rows;
     prm.status_word = device_status_word();
-    prm.groups = (max_m + mt - 1) / mt;  // 1 .. 4
+    prm.groups = groups;
     prm.table_cap = table_cap;
-    const size_t smem = ring_bytes(chunk_tiles) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
+    prm.arena_bytes = (int)arena_max;
+    const size_t smem = ring_bytes(chunk_tiles, groups) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
     cudaError_t e;
-    if (mt == 1) e = stage_x ? launch_stream<1, 5, true>(prm, grid, smem, st) : launch_stream<1, 5, false>(prm, grid, smem, st);
-    else e = stage_x ? launch_stream<4, 4, true>(prm, grid, smem, st) : launch_stream<4, 4, false>(prm, grid, smem, st);
+    if (mt == 1) e = launch_stream<1, 5>(prm, grid, smem, st);
+    else e = launch_stream<4, 4>(prm, grid, smem, st);
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
