@@ -244,6 +244,11 @@ def run_ours(args):
                                   "frac_of_hbm_peak": round(packed_bytes / ms_m / 1e6 / peaks["hbm_gbs"], 4)}
             del its, bm, wm
 
+    # ---- the 30-layer stack as a dependent chain (configs[2]): 210 matmuls, glue in between, M = 1 (rank 0 only) ----
+    chain = None
+    if rank == 0:
+        chain = run_chain(bl, dev, pool, gains, peaks, packed_bytes, reps=max(5, args.steps))
+
     # ---- prefill: int8 tensor-core path at M = 2048 on the 7 shapes (rank 0 only) ----
     prefill = None
     if rank == 0:
@@ -266,11 +271,47 @@ def run_ours(args):
                        "parallelism": "replicas only (no collective)" if world > 1 else "single GPU"},
             "frac_of_hbm_peak": round(value / world / peaks["hbm_gbs"], 4),
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
-            "roofline": roofline, "per_call": per_call, "decode_more_tokens": decode_m, "prefill": prefill,
+            "roofline": roofline, "per_call": per_call, "decode_more_tokens": decode_m, "chain": chain, "prefill": prefill,
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))
     replicas.finalize()
+
+
+def run_chain(bl, dev, pool, gains, peaks, packed_bytes, reps):
+    """configs[2]: every matmul of the 30-layer stack depends on the one before (RMSNorm + quantiser per BitLinear
+    input, squared-ReLU gate, residuals, attention stand-in); one pass = one decoded token at M = 1."""
+    from paper_2504_12285_b200 import chain as gpu_chain
+
+    layers = []
+    for layer in range(wl.N_LAYERS):
+        mats = pool[layer * 7:(layer + 1) * 7]
+        layers.append({m["name"]: (m["packed"], m["s_w"], gains[m["K"]]) for m in mats})
+    ch = gpu_chain.DecodeChain(layers, 1, wl.HIDDEN, wl.FFN, wl.N_Q_HEADS, wl.N_KV_HEADS, wl.HEAD_DIM, wl.RMS_EPS, dev)
+    h0 = wl.activations_normal(1, wl.HIDDEN, wl.seed_for(3)).to(dev)
+    ch.step(h0)
+    eager_ms = cuda_time_ms(lambda: [ch.step(h0) for _ in range(reps)]) / reps
+    out = {"workload": "configs[2]: 30 layers x 7 BitLinear as a dependent chain at M=1 (210 matmuls, 120 fused "
+                       "RMSNorm+quantiser inputs, glue kernels in between)",
+           "launches_per_token": wl.N_LAYERS * ch.launches_per_layer + 1,
+           "eager_us_per_token": round(eager_ms * 1e3, 1),
+           "eager_value": round(packed_bytes / eager_ms / 1e6, 1), "unit": UNIT}
+    try:  # the same launches replayed from a CUDA graph (no host launch cost)
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            ch.step(h0)
+            with torch.cuda.graph(graph, stream=side):
+                ch.step(h0)
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        graph_ms = cuda_time_ms(lambda: [graph.replay() for _ in range(reps)]) / reps
+        out.update({"graph_us_per_token": round(graph_ms * 1e3, 1), "graph_value": round(packed_bytes / graph_ms / 1e6, 1),
+                    "graph_frac_of_hbm_peak": round(packed_bytes / graph_ms / 1e6 / peaks["hbm_gbs"], 4)})
+    except Exception as exc:  # capture refused: keep the eager number
+        out["graph"] = f"not captured: {type(exc).__name__}"
+    return out
 
 
 def timed_sequence(calls, blocker):

@@ -93,12 +93,14 @@ size_t bitlinear_packed_bytes(int N, int K);
 size_t bitlinear_pack_workspace_bytes(int N, int K);
 
 /* Workspace bytes bitlinear_forward needs: int8 activations [M][K], the per-token scale and
- * code sum, and, when the tensor-core path can be taken (M > 16 or a forced path), an
- * unpacked uint8 copy of the weight codes [N][K].  Returns 0 for an unsupported shape. */
+ * code sum, and, when the tensor-core path can be taken (M > 16 or a forced path), the scratch
+ * of bitlinear_matmul_workspace_bytes.  Returns 0 for an unsupported shape. */
 size_t bitlinear_workspace_bytes(int M, int N, int K);
 
-/* Workspace bytes bitlinear_matmul_q needs (the unpacked weight codes of the tensor-core path;
- * 0 when only the decode kernel can be taken, i.e. M <= 16 and path AUTO or GEMV). */
+/* Workspace bytes bitlinear_matmul_q needs: for the tensor-core path one byte per weight (the
+ * codes 0/1/2 expanded into the shared-memory images of the kernel's 256 x 128 tiles, N rounded up
+ * to whole tiles) plus a small launch table; 0 when only the decode kernel can be taken, i.e.
+ * M <= 16 and path AUTO or GEMV. */
 size_t bitlinear_matmul_workspace_bytes(int M, int N, int K, int path);
 
 /*
@@ -168,20 +170,28 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
                            size_t ws_bytes, void* stream);
 
 /*
- * Batched decode: `count` independent BitLinear forwards of at most 16 tokens each (the decode
- * regime of Section 5.1, where the cost is the packed weight bytes streamed from HBM) in two
- * launches: one fused RMSNorm+quantiser launch over every token, then one persistent kernel that
- * streams the packed weights of all problems back to back.
+ * Batched forward: `count` independent BitLinear forwards in a handful of launches.
+ *
+ * Problems of at most 16 tokens (the decode regime of Section 5.1, where the cost is the packed
+ * weight bytes streamed from HBM) take two launches together: one fused RMSNorm+quantiser launch
+ * over every token, then one persistent kernel that streams the packed weights of all of them
+ * back to back.  Problems of more than 16 tokens (prefill; N must be a multiple of 128) take three
+ * launches together: the quantiser, the expansion of the packed weights into tensor-core tile
+ * images, and one persistent tcgen05 kernel that runs every tile of every matmul; problems that
+ * name the same x, gain, rms_eps, M and K (q/k/v or gate/up of a layer) share one quantised copy.
+ * Both kinds may be mixed in one call.
  *   problems : HOST array of `count` descriptors; the pointers inside are DEVICE pointers with the
- *              meaning, layout and alignment of the bitlinear_forward arguments.  M <= 16,
- *              K <= 8192.  Problems with M == 0 are skipped.  Outputs must not alias inputs of
- *              other problems of the same call (they run concurrently).
+ *              meaning, layout and alignment of the bitlinear_forward arguments.  K <= 8192 for
+ *              problems of at most 16 tokens.  Problems with M == 0 are skipped.  Outputs must not
+ *              alias inputs of other problems of the same call (they run concurrently).
  *   flags    : 0, or an OR of BITLINEAR_BATCH_REUSE_PLAN (the previous call on this workspace had
- *              exactly the same descriptors: skips re-uploading the plan) and
- *              BITLINEAR_BATCH_REUSE_ACT (the inputs are unchanged as well: skips launch 1).
+ *              exactly the same descriptors: skips re-uploading the decode plan) and
+ *              BITLINEAR_BATCH_REUSE_ACT (the inputs are unchanged as well: skips the quantiser
+ *              launches and reuses their results in ws).
  *   ws       : device scratch of at least bitlinear_batch_workspace_bytes(problems, count); it
- *              holds the uploaded plan and the quantised activations, so a call must not overlap
- *              another call that uses the same workspace.
+ *              holds the uploaded plan, the quantised activations and the expanded weights of the
+ *              prefill problems, so a call must not overlap another call that uses the same
+ *              workspace.
  */
 typedef struct bitlinear_problem {
     const void* x;      /* [M][K] bf16 */
@@ -211,6 +221,22 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
 int bitlinear_forward_batch_host(const bitlinear_problem* problems, int count, int flags, const void* x_host,
                                  void* x_dev, size_t x_bytes, const void* y_dev, void* y_host, size_t y_bytes,
                                  void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Element-wise glue between the BitLinear matmuls of a decoder layer, for chained decode runs (Section 2: squared
+ * ReLU replaces SwiGLU in the feed-forward block; residual connections of the Transformer).  Inputs that come out of
+ * a BitLinear are fp32 [M][*]; every result is rounded once to bf16 (round to nearest even) because it feeds the next
+ * BitLinear.  Each arithmetic step is one fp32 operation.
+ *   relu2_mul    : u = bf16( fl32( fl32(r*r) * up ) ), r = max(gate, 0);          gate, up [M][F] -> u [M][F]
+ *   residual_add : h = bf16( fl32( float(h) + y ) ) in place;                       h bf16 [M][N], y fp32 [M][N]
+ *   attn_standin : NOT attention (attention is not a BitLinear and is outside this library): a fixed mixing of the
+ *                  q and v projections that keeps the data dependence of a layer,
+ *                  o_in[m][h*D + j] = bf16( fl32( q[m][h*D + j] + v[m][(h / (n_q/n_kv))*D + j] ) ).
+ */
+int bitlinear_glue_relu2_mul(const float* gate, const float* up, void* u_bf16, int M, int F, void* stream);
+int bitlinear_glue_residual_add(void* h_bf16, const float* y, int M, int N, void* stream);
+int bitlinear_glue_attn_standin(const float* q, const float* v, void* o_in_bf16, int M, int n_q_heads, int n_kv_heads,
+                                int head_dim, void* stream);
 
 /*
  * bitlinear_forward for decode-sized calls by code that cannot allocate device memory.

@@ -41,6 +41,9 @@ _SIGNATURES = {
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
+    "bitlinear_glue_relu2_mul": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
+    "bitlinear_glue_residual_add": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
+    "bitlinear_glue_attn_standin": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_void_p]),
     "bitlinear_static_scratch_bytes": (_c_size_t, []),
     "bitlinear_forward_static": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
                                           _c_void_p, _c_int, _c_void_p]),
@@ -229,6 +232,32 @@ def bitlinear_forward_host(x_host, gain, packed, s_w, N: int, y_host, rms_eps: f
                                       _ptr(y_host), _ydt(y_host.dtype), _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_forward_host")
     return y_host
+
+
+def bitlinear_glue_relu2_mul(gate: torch.Tensor, up: torch.Tensor, u: torch.Tensor) -> torch.Tensor:
+    """u (bf16) = relu(gate)^2 * up, gate / up fp32 [M, F]."""
+    _dev(gate, torch.float32, "gate"), _dev(up, torch.float32, "up"), _dev(u, torch.bfloat16, "u")
+    M, F = gate.shape
+    _check(lib().bitlinear_glue_relu2_mul(_ptr(gate), _ptr(up), _ptr(u), M, F, _stream()), "bitlinear_glue_relu2_mul")
+    return u
+
+
+def bitlinear_glue_residual_add(h: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    """h (bf16, in place) = h + y, y fp32 [M, N]."""
+    _dev(h, torch.bfloat16, "h"), _dev(y, torch.float32, "y")
+    M, N = h.shape
+    _check(lib().bitlinear_glue_residual_add(_ptr(h), _ptr(y), M, N, _stream()), "bitlinear_glue_residual_add")
+    return h
+
+
+def bitlinear_glue_attn_standin(q: torch.Tensor, v: torch.Tensor, o_in: torch.Tensor, n_q_heads: int, n_kv_heads: int,
+                                head_dim: int) -> torch.Tensor:
+    """o_in (bf16) = q + v of the matching KV head: a stand-in for attention that keeps a layer's data dependence."""
+    _dev(q, torch.float32, "q"), _dev(v, torch.float32, "v"), _dev(o_in, torch.bfloat16, "o_in")
+    rc = lib().bitlinear_glue_attn_standin(_ptr(q), _ptr(v), _ptr(o_in), q.shape[0], n_q_heads, n_kv_heads, head_dim,
+                                           _stream())
+    _check(rc, "bitlinear_glue_attn_standin")
+    return o_in
 
 
 def bitlinear_static_scratch_bytes() -> int:

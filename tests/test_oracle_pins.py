@@ -326,3 +326,52 @@ def test_packed_artifact_roundtrip_at_layer_shape():
     assert wts["packed"].size == 640 * 2560 // 4
     assert np.array_equal(oracle.unpack(wts["packed"], 640, 2560), wts["wq"])
     assert not wts["fragile"]
+
+
+# ---- chained decode: the glue between BitLinears (squared ReLU, residual, attention stand-in) ----
+
+
+def test_chain_glue_closed_forms():
+    """With every weight matrix all zeros each BitLinear returns 0, so the chain must leave h unchanged (residual
+    adds of zero); with gate weights that make g negative the squared-ReLU branch must contribute exactly nothing."""
+    from oracle import chain as oc
+
+    H, F, nq, nkv, hd = 256, 256, 2, 1, 128
+    zero = lambda n, k: dict(wq=np.zeros((n, k), np.int8), s_w=np.float32(1e-5))
+    layer = {"q": zero(H, H), "k": zero(nkv * hd, H), "v": zero(nkv * hd, H), "o": zero(H, H), "gate": zero(F, H),
+             "up": zero(F, H), "down": zero(H, F)}
+    h0 = wl.bf16_bits(wl.activations_normal(3, H, 321))
+    out = oc.decode_chain(h0, [layer, layer], nq, nkv, hd, 1e-5)
+    assert np.array_equal(out["h"], h0)
+    assert np.all(out["k"] == 0)
+
+
+def test_chain_attention_standin_and_relu2_by_hand():
+    """One layer with identity-like ternary weights, checked against the formulas written out in numpy fp64 on the
+    oracle's own integer stages: a = q + v[head // group], f = relu(g)^2 * u, both residuals."""
+    from oracle import chain as oc
+
+    H, F, nq, nkv, hd = 256, 256, 2, 1, 128
+    rng = np.random.default_rng(7)
+    mats = {}
+    for name, (n, k) in {"q": (H, H), "k": (nkv * hd, H), "v": (nkv * hd, H), "o": (H, H), "gate": (F, H), "up": (F, H),
+                         "down": (H, F)}.items():
+        mats[name] = dict(wq=rng.integers(-1, 2, size=(n, k)).astype(np.int8), s_w=np.float32(0.02))
+    h0 = wl.bf16_bits(wl.activations_normal(2, H, 654))
+    out = oc.decode_chain(h0, [mats], nq, nkv, hd, 1e-5)
+
+    def lin(bits, m):
+        return oracle.bitlinear_forward(bits, None, 1e-5, m["wq"], m["s_w"])["y"].astype(np.float64)
+
+    def bf(x64):  # fp64 values that are exactly representable in fp32 after one fp32 op are passed as float32
+        return oracle.f32_to_bf16(x64.astype(np.float32))
+
+    q, v = lin(h0, mats["q"]), lin(h0, mats["v"])
+    a = np.concatenate([q[:, :hd] + v[:, :hd], q[:, hd:] + v[:, :hd]], axis=1)
+    a_bits = bf(np.float32(q.astype(np.float32)[:, :]) * 0 + a.astype(np.float32))  # one fp32 rounding of the sum
+    h1 = bf((oracle.bf16_to_f32(h0).astype(np.float64) + lin(a_bits, mats["o"])).astype(np.float32))
+    g, u = lin(h1, mats["gate"]).astype(np.float32), lin(h1, mats["up"]).astype(np.float32)
+    r = np.maximum(g, 0)
+    f_bits = bf(((r * r).astype(np.float32) * u).astype(np.float32))
+    h2 = bf((oracle.bf16_to_f32(h1).astype(np.float64) + lin(f_bits, mats["down"])).astype(np.float32))
+    assert np.array_equal(out["h"], h2)
