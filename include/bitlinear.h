@@ -239,6 +239,35 @@ int bitlinear_glue_attn_standin(const float* q, const float* v, void* o_in_bf16,
                                 int head_dim, void* stream);
 
 /*
+ * One decoded token through a stack of decoder layers in ONE persistent cooperative kernel (Section 2: every linear
+ * map of a layer is a BitLinear; squared-ReLU feed-forward block; Section 5.1: decode is bound by the packed weight
+ * bytes).  Per layer, with the glue steps defined above:
+ *     q,k,v = BitLinear(h);  a = attn_standin(q, v);  h = residual_add(h, BitLinear_o(a));
+ *     g,u   = BitLinear_gate/up(h);  f = relu2_mul(g, u);  h = residual_add(h, BitLinear_down(f)).
+ * The result is bit-identical to issuing those calls one by one.  The kernel keeps every SM busy for the whole token:
+ * a level's weight rows are split over the SMs, prefetched into shared memory one level ahead, and levels are
+ * separated by grid barriers instead of kernel boundaries.
+ *   layers   : HOST array of n_layers descriptors; pointers inside are DEVICE pointers: packed / s_w of the seven
+ *              matrices in the order q,k,v,o,gate,up,down, and the bf16 RMSNorm gains of the four BitLinear inputs
+ *              (of {q,k,v}, o, {gate,up}, down; NULL = ones).
+ *   dims     : hidden = n_q_heads * head_dim; hidden and ffn multiples of 256, at most 8192; one token.
+ *   h_bf16   : [hidden] bf16, in and out.      k_out : nullable, [n_kv_heads*head_dim] fp32, the last layer's k.
+ *   flags    : 0 or BITLINEAR_BATCH_REUSE_PLAN (the layer table uploaded by the previous call on ws is still valid).
+ *   ws       : at least bitlinear_decode_chain_workspace_bytes(...); calls on one workspace must not overlap.
+ * Needs a device that supports cooperative launches with one CTA per SM free (else BITLINEAR_ERR_CUDA).
+ */
+typedef struct bitlinear_chain_layer {
+    const void* packed[7];
+    const float* s_w[7];
+    const void* gain[4];
+} bitlinear_chain_layer;
+size_t bitlinear_decode_chain_workspace_bytes(int n_layers, int hidden, int ffn, int n_q_heads, int n_kv_heads,
+                                              int head_dim);
+int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, int hidden, int ffn, int n_q_heads,
+                           int n_kv_heads, int head_dim, float rms_eps, void* h_bf16, float* k_out, int flags, void* ws,
+                           size_t ws_bytes, void* stream);
+
+/*
  * bitlinear_forward for decode-sized calls by code that cannot allocate device memory.
  * (No counterpart in the paper: this is a convenience of the library.)
  *

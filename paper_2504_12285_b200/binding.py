@@ -44,6 +44,9 @@ _SIGNATURES = {
     "bitlinear_glue_relu2_mul": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
     "bitlinear_glue_residual_add": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
     "bitlinear_glue_attn_standin": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_void_p]),
+    "bitlinear_decode_chain_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int, _c_int, _c_int]),
+    "bitlinear_decode_chain": (_c_int, [_c_void_p, _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_float, _c_void_p,
+                                        _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_static_scratch_bytes": (_c_size_t, []),
     "bitlinear_forward_static": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
                                           _c_void_p, _c_int, _c_void_p]),
@@ -258,6 +261,55 @@ def bitlinear_glue_attn_standin(q: torch.Tensor, v: torch.Tensor, o_in: torch.Te
                                            _stream())
     _check(rc, "bitlinear_glue_attn_standin")
     return o_in
+
+
+class ChainLayer(ctypes.Structure):
+    """Mirror of the C struct bitlinear_chain_layer."""
+    _fields_ = [("packed", _c_void_p * 7), ("s_w", _c_void_p * 7), ("gain", _c_void_p * 4)]
+
+
+CHAIN_MATRICES = ("q", "k", "v", "o", "gate", "up", "down")
+
+
+class ChainLayers:
+    """Host array of bitlinear_chain_layer plus the tensors it points to (kept alive).
+
+    layers: list of dicts with keys q,k,v,o,gate,up,down -> (packed uint8, s_w fp32 [1]) and "gains" -> four bf16 [K]
+    tensors or None (inputs of {q,k,v}, o, {gate,up}, down)."""
+
+    def __init__(self, layers):
+        self.keep = layers
+        self.count = len(layers)
+        self.array = (ChainLayer * max(self.count, 1))()
+        for i, layer in enumerate(layers):
+            for j, name in enumerate(CHAIN_MATRICES):
+                packed, s_w = layer[name]
+                _dev(packed, torch.uint8, name), _dev(s_w, torch.float32, name + ".s_w")
+                self.array[i].packed[j] = packed.data_ptr()
+                self.array[i].s_w[j] = s_w.data_ptr()
+            for j, gain in enumerate(layer["gains"]):
+                if gain is not None:
+                    _dev(gain, torch.bfloat16, "gain")
+                self.array[i].gain[j] = None if gain is None else gain.data_ptr()
+
+
+def bitlinear_decode_chain_workspace_bytes(n_layers: int, hidden: int, ffn: int, n_q_heads: int, n_kv_heads: int,
+                                           head_dim: int) -> int:
+    return int(lib().bitlinear_decode_chain_workspace_bytes(n_layers, hidden, ffn, n_q_heads, n_kv_heads, head_dim))
+
+
+def bitlinear_decode_chain(layers: ChainLayers, hidden: int, ffn: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                           h: torch.Tensor, ws: torch.Tensor, rms_eps: float = 1e-5, k_out: torch.Tensor | None = None,
+                           reuse_plan: bool = False) -> torch.Tensor:
+    """One token through the whole stack in one persistent kernel; h (bf16 [1, hidden] or [hidden]) is updated in place."""
+    _dev(h, torch.bfloat16, "h"), _dev(ws, torch.uint8, "ws")
+    if k_out is not None:
+        _dev(k_out, torch.float32, "k_out")
+    rc = lib().bitlinear_decode_chain(ctypes.addressof(layers.array), layers.count, hidden, ffn, n_q_heads, n_kv_heads,
+                                      head_dim, rms_eps, _ptr(h), _ptr(k_out), BATCH_REUSE_PLAN if reuse_plan else 0,
+                                      _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_decode_chain")
+    return h
 
 
 def bitlinear_static_scratch_bytes() -> int:

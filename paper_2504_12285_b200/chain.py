@@ -61,3 +61,26 @@ class DecodeChain:
             bl.bitlinear_forward_batch(down[0], down[1], reuse_plan=True)
             bl.bitlinear_glue_residual_add(self.h, self.dn)
         return self.h
+
+
+class PersistentChain:
+    """The same chain at one token through bitlinear_decode_chain: one cooperative kernel per token."""
+
+    def __init__(self, layers, hidden: int, ffn: int, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                 rms_eps: float = 1e-5, device="cuda:0"):
+        """layers: list of dicts q,k,v,o,gate,up,down -> (packed, s_w) and "gains" -> 4 x (bf16 [K] or None)."""
+        dev = torch.device(device)
+        self.dims = (hidden, ffn, n_q_heads, n_kv_heads, head_dim)
+        self.eps = rms_eps
+        self.table = bl.ChainLayers(layers)
+        self.h = torch.zeros(1, hidden, dtype=torch.bfloat16, device=dev)
+        self.k = torch.empty(n_kv_heads * head_dim, dtype=torch.float32, device=dev)
+        self.ws = torch.empty(bl.bitlinear_decode_chain_workspace_bytes(len(layers), *self.dims), dtype=torch.uint8, device=dev)
+        self.uploaded = False
+
+    def step(self, h0: torch.Tensor | None = None) -> torch.Tensor:
+        if h0 is not None:
+            self.h.copy_(h0)
+        bl.bitlinear_decode_chain(self.table, *self.dims, self.h, self.ws, self.eps, k_out=self.k, reuse_plan=self.uploaded)
+        self.uploaded = True
+        return self.h

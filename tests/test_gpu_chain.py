@@ -16,24 +16,34 @@ DEV = "cuda:0"
 NAMES = ("q", "k", "v", "o", "gate", "up", "down")
 
 
+INPUT_OF = {"q": 0, "k": 0, "v": 0, "o": 1, "gate": 2, "up": 2, "down": 3}  # which of the 4 normalised inputs
+
+
 def build(n_layers, hidden, ffn, n_q, n_kv, hd, seed, gains):
+    """Returns (per-level layers for DecodeChain, layers for PersistentChain, oracle layers).  One RMSNorm gain per
+    BitLinear INPUT (q/k/v share one, gate/up share one), as in a decoder layer."""
     shapes = {"q": (hidden, hidden), "k": (n_kv * hd, hidden), "v": (n_kv * hd, hidden), "o": (hidden, hidden),
               "gate": (ffn, hidden), "up": (ffn, hidden), "down": (hidden, ffn)}
-    gpu_layers, ref_layers = [], []
+    level_layers, chain_layers, ref_layers = [], [], []
     for layer in range(n_layers):
-        gl, rl = {}, {}
+        in_k = (hidden, hidden, hidden, ffn)
+        g_host = [wl.gain_random(in_k[j], seed + 100 * layer + 50 + j) if gains else None for j in range(4)]
+        g_dev = [None if g is None else g.to(DEV) for g in g_host]
+        gl, cl, rl = {}, {"gains": g_dev}, {}
         for i, name in enumerate(NAMES):
             n, k = shapes[name]
             W = wl.latent_weights(n, k, seed + 100 * layer + i)
             packed, s_w = bl.bitlinear_pack_weights(W.to(DEV), wl.WEIGHT_EPS)
             ref = oracle.quantize_weights(W.numpy(), wl.WEIGHT_EPS)
             assert np.array_equal(packed.cpu().numpy(), ref["packed"])
-            g = wl.gain_random(k, seed + 100 * layer + 50 + i) if gains else None
-            gl[name] = (packed, s_w, None if g is None else g.to(DEV))
-            rl[name] = dict(wq=ref["wq"], s_w=ref["s_w"], gain=None if g is None else wl.bf16_bits(g))
-        gpu_layers.append(gl)
+            j = INPUT_OF[name]
+            gl[name] = (packed, s_w, g_dev[j])
+            cl[name] = (packed, s_w)
+            rl[name] = dict(wq=ref["wq"], s_w=ref["s_w"], gain=None if g_host[j] is None else wl.bf16_bits(g_host[j]))
+        level_layers.append(gl)
+        chain_layers.append(cl)
         ref_layers.append(rl)
-    return gpu_layers, ref_layers
+    return level_layers, chain_layers, ref_layers
 
 
 @pytest.mark.parametrize("M,n_layers,hidden,ffn,n_q,n_kv,hd,gains", [
@@ -42,7 +52,7 @@ def build(n_layers, hidden, ffn, n_q, n_kv, hd, seed, gains):
     (1, 2, wl.HIDDEN, wl.FFN, wl.N_Q_HEADS, wl.N_KV_HEADS, wl.HEAD_DIM, False),  # two full-size layers
 ])
 def test_chain_matches_oracle_bitwise(M, n_layers, hidden, ffn, n_q, n_kv, hd, gains):
-    gpu_layers, ref_layers = build(n_layers, hidden, ffn, n_q, n_kv, hd, 5000 + M, gains)
+    gpu_layers, chain_layers, ref_layers = build(n_layers, hidden, ffn, n_q, n_kv, hd, 5000 + M, gains)
     h0 = wl.activations_normal(M, hidden, 5999)
     ch = gpu_chain.DecodeChain(gpu_layers, M, hidden, ffn, n_q, n_kv, hd, wl.RMS_EPS, DEV)
     h = ch.step(h0.to(DEV))
@@ -55,3 +65,12 @@ def test_chain_matches_oracle_bitwise(M, n_layers, hidden, ffn, n_q, n_kv, hd, g
     torch.cuda.synchronize()
     assert np.array_equal(wl.bf16_bits(h2.cpu()), ref["h"])
     assert bl.bitlinear_poll_status() == 0
+    if M == 1:
+        # the same token through the single persistent kernel
+        pc = gpu_chain.PersistentChain(chain_layers, hidden, ffn, n_q, n_kv, hd, wl.RMS_EPS, DEV)
+        for _ in range(2):  # the second call reuses the uploaded layer table
+            hp = pc.step(h0.to(DEV))
+            torch.cuda.synchronize()
+            assert bl.bitlinear_poll_status() == 0
+            assert np.array_equal(wl.bf16_bits(hp.cpu()), ref["h"])
+            assert np.array_equal(pc.k.cpu().numpy(), ref["k"].reshape(-1))
