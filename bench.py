@@ -314,6 +314,18 @@ def run_chain(bl, dev, pool, gains, peaks, packed_bytes, reps):
                     "graph_frac_of_hbm_peak": round(packed_bytes / graph_ms / 1e6 / peaks["hbm_gbs"], 4)})
     except Exception as exc:  # capture refused: keep the eager number
         out["graph"] = f"not captured: {type(exc).__name__}"
+    # the same token through ONE persistent cooperative kernel (grid barriers instead of kernel boundaries)
+    pl = [dict({m["name"]: (m["packed"], m["s_w"]) for m in pool[layer * 7:(layer + 1) * 7]},
+               gains=[gains[wl.HIDDEN], gains[wl.HIDDEN], gains[wl.HIDDEN], gains[wl.FFN]]) for layer in range(wl.N_LAYERS)]
+    pc = gpu_chain.PersistentChain(pl, wl.HIDDEN, wl.FFN, wl.N_Q_HEADS, wl.N_KV_HEADS, wl.HEAD_DIM, wl.RMS_EPS, dev)
+    h_ref = ch.step(h0).clone()
+    h_p = pc.step(h0).clone()
+    torch.cuda.synchronize()
+    pers_ms = cuda_time_ms(lambda: [pc.step(h0) for _ in range(reps)]) / reps
+    out.update({"persistent_us_per_token": round(pers_ms * 1e3, 1), "persistent_value": round(packed_bytes / pers_ms / 1e6, 1),
+                "persistent_frac_of_hbm_peak": round(packed_bytes / pers_ms / 1e6 / peaks["hbm_gbs"], 4),
+                "persistent_launches_per_token": 1,
+                "persistent_equals_per_level_calls": bool(torch.equal(h_ref, h_p))})
     return out
 
 

@@ -105,8 +105,10 @@ static float rms_scale(long double S, int K, float eps) {
  * x: [M][K] bf16 bit patterns; g: [K] bf16 bit patterns or NULL (all ones).
  * Outputs: q [M][K], d [M], xsum [M] (nullable), y_norm [M][K] fp32 (nullable: the
  * normalised row before quantisation), fragile [M] (nullable): 1 where the fp32
- * rounding of r would change if the sum of squares moved by K*2^-52 relative, i.e.
- * where another (equally valid) summation order could legitimately give another r.
+ * rounding of r would change if the sum of squares moved by max(K*2^-52, 2^-40)
+ * relative, i.e. where another (equally valid) way of summing the exact squares -
+ * another fp64 order, or partial sums carried as error-free pairs of fp32 - could
+ * legitimately give another r.
  */
 void oracle_rmsnorm_quant(const uint16_t *x, const uint16_t *g, float eps, int M, int K,
                           int8_t *q, float *d, int32_t *xsum, float *y_norm, int *fragile) {
@@ -121,6 +123,7 @@ void oracle_rmsnorm_quant(const uint16_t *x, const uint16_t *g, float eps, int M
         float r = rms_scale(S, K, eps);
         if (fragile) {
             long double rel = (long double)K * 2.220446049250313e-16L;
+            if (rel < 9.094947017729282e-13L) rel = 9.094947017729282e-13L; /* 2^-40 */
             float r_lo = rms_scale(S * (1.0L - rel), K, eps);
             float r_hi = rms_scale(S * (1.0L + rel), K, eps);
             fragile[m] = (r_lo != r || r_hi != r) ? 1 : 0;

@@ -16,15 +16,18 @@
 // Every wait is bounded; on a timeout an abort word makes every CTA leave and BITLINEAR_ERR_TIMEOUT is reported.
 #include <algorithm>
 
-#include "common.cuh"
+#include "quant_row.cuh"
 #include "sm100_sync.cuh"
 
 namespace bitlinear {
 
 namespace {
 
-constexpr int kChainThreads = 512;
+constexpr int kChainThreads = 512;  // compute threads; one more warp issues the weight copies
 constexpr int kChainWarps = kChainThreads / 32;
+constexpr int kChainLaunchThreads = kChainThreads + 32;
+// barrier of the compute threads only (the copy warp runs on its own)
+#define CSYNC() asm volatile("bar.sync 1, 512;" ::: "memory")
 constexpr int kMaxEpt = 16;  // input elements per thread: K <= 8192
 
 struct ChainLayerDev {
@@ -80,6 +83,7 @@ struct BlockScratch {
     float r, d;
     int xsum;
     int ok;
+    int desc_ready;  // highest layer whose descriptor is in shared memory
 };
 
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
@@ -93,7 +97,7 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
     return v;
 }
 
-__global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const ChainParams p) {
+__global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(const ChainParams p) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int kmax = p.hidden > p.ffn ? p.hidden : p.ffn;
     const int max_rb = p.buf_bytes / ((p.hidden / kTileCols) * kTileBytes);  // most row blocks a CTA can own in a level
@@ -103,8 +107,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
     int* acc_s = reinterpret_cast<int*>(h_s + p.hidden);                       // [max_rb][16]
     ChainLayerDev* desc_s = reinterpret_cast<ChainLayerDev*>(acc_s + (size_t)max_rb * 16);  // [2]
     float* sw_s = reinterpret_cast<float*>(desc_s + 2);                        // [2][8]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sw_s + 16);                   // [2] weight buffer landed
-    BlockScratch* sc = reinterpret_cast<BlockScratch*>(bars + 2);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sw_s + 16);                   // [2] weight buffer landed, [2] buffer read
+    BlockScratch* sc = reinterpret_cast<BlockScratch*>(bars + 4);
     volatile int* abort_s = reinterpret_cast<volatile int*>(&sc->ok);  // CTA-local abort flag for the mbarrier waits
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -115,17 +119,17 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
 
     // ---- prologue: barriers, first descriptor, its scales, the hidden state ----
     if (tid == 0) {
-        mbar_init(smem_u32(bars + 0), 1);
-        mbar_init(smem_u32(bars + 1), 1);
+        for (int b = 0; b < 4; ++b) mbar_init(smem_u32(bars + b), 1);
         sc->ok = 0;
+        sc->desc_ready = 0;
         mbar_init_fence();
     }
     {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(p.layers);
         uint32_t* dst = reinterpret_cast<uint32_t*>(desc_s);
-        for (int i = tid; i < (int)(sizeof(ChainLayerDev) / 4); i += kChainThreads) dst[i] = src[i];
+        for (int i = tid; i < (int)(sizeof(ChainLayerDev) / 4); i += kChainLaunchThreads) dst[i] = src[i];
     }
-    for (int i = tid; i < p.hidden; i += kChainThreads) h_s[i] = p.h[i];
+    for (int i = tid; i < p.hidden; i += kChainLaunchThreads) h_s[i] = p.h[i];
     __syncthreads();
     if (tid < 7) sw_s[tid] = *desc_s[0].s_w[tid];
     __syncthreads();
@@ -148,9 +152,22 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                       dsc.packed[s.first + m] + (size_t)(row / kTileRows) * rb_bytes, rb_bytes, bar);
         }
     };
-    if (warp == 0) issue_level(0);
-
     bool ok = true;
+    if (warp == kChainWarps) {
+        // ---- copy warp: one level ahead of the arithmetic, as soon as the buffer has been read and the layer's
+        //      descriptor is in shared memory ----
+        for (int L = 0; L < total_levels; ++L) {
+            const int layer = L >> 2;
+            if (L >= 2 && !mbar_wait(smem_u32(bars + 2 + (L & 1)), (uint32_t)((L >> 1) - 1) & 1u, abort_s)) break;
+            const unsigned long long t0 = globaltimer_ns();
+            bool ready = true;
+            while (*reinterpret_cast<volatile int*>(&sc->desc_ready) < layer) {
+                if (*abort_s || globaltimer_ns() - t0 > kWaitLimitNs) { ready = false; break; }
+            }
+            if (!ready) { *abort_s = 1; break; }
+            issue_level(L);
+        }
+    } else
     for (int L = 0; L < total_levels && ok; ++L) {
         const int layer = L >> 2, level = L & 3;
         const LevelShape s = level_shape(level, p);
@@ -162,7 +179,11 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         // ---- descriptor / scale prefetch for the next layer, weight prefetch for the next level ----
         if (level == 3 || level == 0) {  // level 3 needs the next layer's descriptor, level 0 this layer's scales
             asm volatile("cp.async.wait_group 0;" ::: "memory");
-            __syncthreads();
+            CSYNC();
+            if (level == 3 && tid == 0) {
+                __threadfence_block();
+                *reinterpret_cast<volatile int*>(&sc->desc_ready) = layer + 1;  // the copy warp may go on to the next layer
+            }
         }
         if (level == 0 && layer + 1 < p.n_layers && tid < (int)(sizeof(ChainLayerDev) / 16)) {
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(&desc_s[(layer + 1) & 1]) + 16u * tid),
@@ -176,7 +197,6 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                          : "memory");
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        if (warp == 0 && L + 1 < total_levels) issue_level(L + 1);
 
         // ---- wait for the outputs of the previous level (grid barrier, bounded) ----
         if (L > 0) {
@@ -195,7 +215,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                     }
                 }
             }
-            __syncthreads();
+            CSYNC();
             if (sc->ok) { ok = false; break; }
         }
 
@@ -203,6 +223,32 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
         for (int i = tid; i < n_rb * 16; i += kChainThreads) acc_s[i] = 0;
         const __nv_bfloat16* gain = desc_s[layer & 1].gain[level];
         float xv[kMaxEpt], gv[kMaxEpt];
+        // every load of the stage is issued before anything is computed, so the L2 round trips overlap
+        float ra[kMaxEpt], rb[kMaxEpt];
+#pragma unroll
+        for (int e = 0; e < kMaxEpt; ++e) {
+            const int i = tid + e * kChainThreads;
+            const bool in = i < K;
+            ra[e] = 0.0f;
+            rb[e] = 0.0f;
+            if (level == 0) {
+                if (in && layer > 0) ra[e] = ldcg_f32(p.dn + i);
+            } else if (level == 1) {
+                if (in) {
+                    const int head = i / p.head_dim, j = i - head * p.head_dim;
+                    ra[e] = ldcg_f32(p.q + i);
+                    rb[e] = ldcg_f32(p.v + (head / group) * p.head_dim + j);
+                }
+            } else if (level == 2) {
+                if (in) ra[e] = ldcg_f32(p.o + i);
+            } else {
+                if (in) {
+                    ra[e] = ldcg_f32(p.g + i);
+                    rb[e] = ldcg_f32(p.u + i);
+                }
+            }
+            gv[e] = (gain != nullptr && in) ? __bfloat162float(gain[i]) : 1.0f;
+        }
         double sq = 0.0;
 #pragma unroll
         for (int e = 0; e < kMaxEpt; ++e) {
@@ -212,35 +258,39 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                 if (level == 0) {
                     x = __bfloat162float(h_s[i]);
                     if (layer > 0) {
-                        x = bf16_round(__fadd_rn(x, ldcg_f32(p.dn + i)));
+                        x = bf16_round(__fadd_rn(x, ra[e]));
                         h_s[i] = __float2bfloat16_rn(x);
                     }
                 } else if (level == 1) {
-                    const int head = i / p.head_dim, j = i - head * p.head_dim;
-                    x = bf16_round(__fadd_rn(ldcg_f32(p.q + i), ldcg_f32(p.v + (head / group) * p.head_dim + j)));
+                    x = bf16_round(__fadd_rn(ra[e], rb[e]));
                 } else if (level == 2) {
-                    x = bf16_round(__fadd_rn(__bfloat162float(h_s[i]), ldcg_f32(p.o + i)));
+                    x = bf16_round(__fadd_rn(__bfloat162float(h_s[i]), ra[e]));
                     h_s[i] = __float2bfloat16_rn(x);
                 } else {
-                    const float r = fmaxf(ldcg_f32(p.g + i), 0.0f);
-                    x = bf16_round(__fmul_rn(__fmul_rn(r, r), ldcg_f32(p.u + i)));
+                    const float r = fmaxf(ra[e], 0.0f);
+                    x = bf16_round(__fmul_rn(__fmul_rn(r, r), rb[e]));
                 }
             }
             xv[e] = x;
-            gv[e] = (gain != nullptr && i < K) ? __bfloat162float(gain[i]) : 1.0f;
-            sq += (double)x * (double)x;
+        }
+        {   // sum of squares: error-free fp32 chains of eight, then fp64 (see sum_squares8)
+            float lo8[8], hi8[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) { lo8[e] = xv[e]; hi8[e] = xv[8 + e]; }
+            sq = sum_squares8(lo8);
+            if (K > 8 * kChainThreads) sq += sum_squares8(hi8);
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
         if (lane == 0) sc->sq[warp] = sq;
-        __syncthreads();
+        CSYNC();
         if (tid == 0) {
             double S = 0.0;
 #pragma unroll
             for (int w = 0; w < kChainWarps; ++w) S += sc->sq[w];
             sc->r = (float)(1.0 / sqrt(S / (double)K + (double)p.eps));
         }
-        __syncthreads();
+        CSYNC();
         const float r = sc->r;
         float amax = 0.0f;
 #pragma unroll
@@ -251,7 +301,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
         if (lane == 0) sc->mx[warp] = amax;
-        __syncthreads();
+        CSYNC();
         float a = 1e-5f;
 #pragma unroll
         for (int w = 0; w < kChainWarps; ++w) a = fmaxf(a, sc->mx[w]);
@@ -271,14 +321,14 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xffffffffu, csum, o);
         if (lane == 0) sc->sum[warp] = csum;
-        __syncthreads();
+        CSYNC();
         int xsum = 0;
 #pragma unroll
         for (int w = 0; w < kChainWarps; ++w) xsum += sc->sum[w];
 
         // ---- the level's weights: wait for the prefetched share, multiply ----
         mbar_wait(smem_u32(bars + (L & 1)), (uint32_t)(L >> 1) & 1u, abort_s);
-        __syncthreads();
+        CSYNC();
         if (sc->ok) {  // the copy did not land in time: tell the other CTAs and leave
             if (tid == 0) atomicExch(p.abort_word, 1);
             ok = false;
@@ -314,7 +364,8 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                 if (t == 0) atomicAdd(&acc_s[rbl * 16 + 8 * hh + g], sum >> 6);
             }
         }
-        __syncthreads();
+        CSYNC();
+        if (tid == 0) mbar_arrive(smem_u32(bars + 2 + (L & 1)));  // the buffer has been read: it may be refilled
 
         // ---- dequantising epilogue: this CTA's rows of the level's output ----
         for (int o = tid; o < n_rb * 16; o += kChainThreads) {
@@ -328,7 +379,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
             const float s_w = sw_s[8 * (layer & 1) + s.first + m];
             y[row] = __fmul_rn(__fmul_rn((float)(acc_s[o] - xsum), s_w), d);
         }
-        __syncthreads();
+        CSYNC();
         if (tid == 0) {
             __threadfence();
             atomicAdd(p.barrier, 1u);
@@ -336,7 +387,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
     }
 
     // ---- after the last level: the final residual, written by CTA 0 ----
-    if (ok && cta == 0) {
+    if (warp < kChainWarps && ok && cta == 0) {
         if (tid == 0) {
             const unsigned target = (unsigned)grid * (unsigned)total_levels;
             const unsigned long long t0 = globaltimer_ns();
@@ -349,7 +400,7 @@ __global__ void __launch_bounds__(kChainThreads, 1) decode_chain_kernel(const Ch
                 }
             }
         }
-        __syncthreads();
+        CSYNC();
         if (!sc->ok)
             for (int i = tid; i < p.hidden; i += kChainThreads)
                 p.h[i] = __float2bfloat16_rn(__fadd_rn(__bfloat162float(h_s[i]), ldcg_f32(p.dn + i)));
@@ -464,7 +515,7 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
     prm.buf_bytes = (int)buf;
     const int kmax = hidden > ffn ? hidden : ffn;
     const size_t max_rb = buf / ((size_t)(hidden / kTileCols) * kTileBytes);
-    const size_t smem = 2 * buf + kmax + (size_t)hidden * 2 + max_rb * 64 + 2 * sizeof(ChainLayerDev) + 64 + 16 +
+    const size_t smem = 2 * buf + kmax + (size_t)hidden * 2 + max_rb * 64 + 2 * sizeof(ChainLayerDev) + 64 + 32 +
                         sizeof(BlockScratch) + 1024;
     if (smem > 227 * 1024) return BITLINEAR_ERR_SHAPE;
     if (cudaFuncSetAttribute(decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
@@ -472,7 +523,7 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
         return BITLINEAR_ERR_CUDA;
     }
     void* args[] = {&prm};
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_chain_kernel), dim3(grid), dim3(kChainThreads), args, smem,
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(decode_chain_kernel), dim3(grid), dim3(kChainLaunchThreads), args, smem,
                                     st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
