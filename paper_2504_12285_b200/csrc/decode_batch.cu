@@ -79,6 +79,9 @@ __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHe
                                                                     const int* __restrict__ row_prob, int count,
                                                                     int total_rb, int grid, int* status_word) {
     __shared__ RowReduceSmem sm;
+    // the stream kernel that follows may start now: it fetches weights first and waits for this grid before it reads
+    // anything written here (programmatic dependent launch)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (!plan_matches(hdr, count, total_rb, grid, (int)gridDim.x)) {
         if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
         return;
@@ -243,6 +246,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             primed = r + 1;
             advance_ld(false);
         }
+
+    // the quantiser launch that precedes this kernel must be complete before its results are read
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     // ---- fill the descriptor table (one warp per problem), then stage the activations ----
     for (int i = warp; i < n_tab; i += kStreamWarps) {
@@ -449,8 +455,19 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
     cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<MT, kChunkTiles>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    decode_stream_kernel<MT, kChunkTiles><<<grid, kStreamThreads, smem, st>>>(prm);
-    return cudaGetLastError();
+    // programmatic dependent launch: the kernel may begin (barrier set-up, first weight copies) while the quantiser
+    // launch before it is still running; it calls griddepcontrol.wait before touching that launch's results
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<MT, kChunkTiles>, prm);
 }
 
 struct PlanLayout {
