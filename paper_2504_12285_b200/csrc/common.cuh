@@ -60,7 +60,8 @@ struct GemmProblem {
 };
 constexpr int kMaxGroup = 32;
 struct GemmGroupHeader {
-    int count, total_tiles, pad0, pad1;
+    int count, total_tiles;
+    unsigned long long region_base;  // CTA-pair kernel: address its tensor map starts at (tile images are addressed as rows of 128 B)
 };
 // layout of the uploaded group table: GemmGroupHeader, then count x GemmProblem
 constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof(GemmProblem);
@@ -68,7 +69,8 @@ constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof
 // Grouped launch: fills m_tiles / tile_begin, uploads the table to table_dev (kGroupTableBytes) and runs every tile of
 // every problem in one persistent kernel.  a_tiled = activations given as tile images (any count), else one problem with
 // row-major activations.  Returns a bitlinear_status.
-int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev, cudaStream_t st);
+int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev, cudaStream_t st,
+                const void* region_base = nullptr, size_t region_bytes = 0);
 size_t gemm_codes_bytes(int N, int K);
 size_t gemm_a_tiles_bytes(int M, int K);
 

@@ -195,6 +195,51 @@ __device__ __forceinline__ void store_block_b16(const uint32_t (&vals)[16], uint
     __syncwarp();
 }
 
+// Epilogue of one warp for one accumulator: 32 tensor-memory lanes (token rows m_warp .. m_warp+31) x 256 columns
+// (weight rows n0 .. n0+255) starting at tensor-memory address taddr.  Subtracts the code offset, dequantises, stores.
+__device__ __forceinline__ void drain_accumulator(const GemmProblem& p, uint32_t taddr, int m_warp, int n0, uint32_t stage_s,
+                                                  int lane) {
+    const int M = p.M, N = p.N, y_dtype = p.y_dtype;
+    void* y = p.y;
+    int32_t* acc_out = p.acc_out;
+    const float s_w = *p.s_w;
+    const int m = m_warp + lane;
+    const bool row_ok = m < M;
+    const int xs = row_ok ? p.xsum[m] : 0;
+    const float dm = row_ok ? p.d[m] : 0.0f;
+    const int rows_ok = (M - m_warp) < 32 ? (M - m_warp) : 32;
+#pragma unroll 1
+    for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32(taddr + c * 32, r);
+        tmem_ld_wait();
+        const int n = n0 + c * 32;
+        if (n < N && rows_ok > 0) {  // warp-uniform
+            // Each lane holds 32 consecutive columns of ONE row.  The block goes through this warp's
+            // shared-memory staging area so that every global store covers whole 128-byte row segments.
+#pragma unroll
+            for (int i = 0; i < 32; ++i) r[i] = (uint32_t)((int)r[i] - xs);
+            if (acc_out != nullptr)
+                store_block_b32(r, stage_s, reinterpret_cast<uint32_t*>(acc_out) + (size_t)m_warp * N + n, N, rows_ok, lane);
+            if (y_dtype == BITLINEAR_BF16) {
+                uint32_t w[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float v0 = __fmul_rn(__fmul_rn((float)(int)r[2 * i], s_w), dm);
+                    const float v1 = __fmul_rn(__fmul_rn((float)(int)r[2 * i + 1], s_w), dm);
+                    const __nv_bfloat162 pk = __floats2bfloat162_rn(v0, v1);
+                    w[i] = *reinterpret_cast<const uint32_t*>(&pk);
+                }
+                store_block_b16(w, stage_s, reinterpret_cast<uint16_t*>(y) + (size_t)m_warp * N + n, N, rows_ok, lane);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__fmul_rn((float)(int)r[i], s_w), dm));
+                store_block_b32(r, stage_s, reinterpret_cast<uint32_t*>(y) + (size_t)m_warp * N + n, N, rows_ok, lane);
+            }
+        }
+    }
+}
+
 // Tile -> (problem, token rows, weight rows).  Tiles of one problem are numbered with the token tile
 // fastest, so CTAs that run side by side share the weight tile; problems follow each other in table order.
 struct TileWalk {
@@ -319,50 +364,11 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
         for (int tile = blockIdx.x; ok && tile < total_tiles; tile += gridDim.x, ++iter) {
             const GemmProblem& p = walk.find(tile);
             const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
-            const int M = p.M, N = p.N, y_dtype = p.y_dtype;
-            void* y = p.y;
-            int32_t* acc_out = p.acc_out;
-            const float s_w = *p.s_w;
             const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
             const int m_warp = mt * BM + quad * 32;  // first token row of this warp's 32 tensor-memory lanes
-            const int m = m_warp + lane;
-            const bool row_ok = m < M;
-            const int xs = row_ok ? p.xsum[m] : 0;
-            const float dm = row_ok ? p.d[m] : 0.0f;
-            const int rows_ok = (M - m_warp) < 32 ? (M - m_warp) : 32;
             if (!mbar_wait(smem_u32(tfull_bar + buf), bphase, abort_flag)) { ok = false; break; }
             tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN + c * 32, r);
-                tmem_ld_wait();
-                const int n = nt * BN + c * 32;
-                if (n < N && rows_ok > 0) {  // warp-uniform
-                    // Each lane holds 32 consecutive columns of ONE row.  The block goes through this warp's
-                    // shared-memory staging area so that every global store covers whole 128-byte row segments.
-#pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = (uint32_t)((int)r[i] - xs);
-                    if (acc_out != nullptr)
-                        store_block_b32(r, stage_s, reinterpret_cast<uint32_t*>(acc_out) + (size_t)m_warp * N + n, N, rows_ok,
-                                        lane);
-                    if (y_dtype == BITLINEAR_BF16) {
-                        uint32_t w[16];
-#pragma unroll
-                        for (int i = 0; i < 16; ++i) {
-                            const float v0 = __fmul_rn(__fmul_rn((float)(int)r[2 * i], s_w), dm);
-                            const float v1 = __fmul_rn(__fmul_rn((float)(int)r[2 * i + 1], s_w), dm);
-                            const __nv_bfloat162 pk = __floats2bfloat162_rn(v0, v1);
-                            w[i] = *reinterpret_cast<const uint32_t*>(&pk);
-                        }
-                        store_block_b16(w, stage_s, reinterpret_cast<uint16_t*>(y) + (size_t)m_warp * N + n, N, rows_ok, lane);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__fmul_rn(__fmul_rn((float)(int)r[i], s_w), dm));
-                        store_block_b32(r, stage_s, reinterpret_cast<uint32_t*>(y) + (size_t)m_warp * N + n, N, rows_ok, lane);
-                    }
-                }
-            }
+            drain_accumulator(p, tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN, m_warp, nt * BN, stage_s, lane);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(tempty_bar + buf));
@@ -381,6 +387,196 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ================================================================================================
+// CTA-pair variant (cta_group::2): two CTAs of a cluster share one 256 x 256 tile.  Each CTA stages its
+// own 128 token rows of A and HALF of the weight tile (128 rows of B) per k-block, so a CTA ingests 32 KB
+// per 512 tensor-pipe cycles (64 B/clk) instead of 48 KB; the leader CTA (cluster rank 0) issues the MMAs
+// for both, each CTA drains its own 128 x 256 accumulator.  Operands are tile images (the grouped path);
+// they are fetched with tensor-map copies in the .cta_group::2 form, which may signal the leader's
+// mbarrier from either CTA: the tensor map views the whole workspace region as rows of 128 bytes, no
+// swizzle (the images are stored swizzled).
+// ================================================================================================
+constexpr int P_STAGES = 6;
+constexpr uint32_t P_HALF_BYTES = 128 * BK;              // 128 rows x 128 bytes
+constexpr uint32_t P_STAGE_BYTES = 2 * P_HALF_BYTES;     // A rows of this CTA + its half of B
+constexpr size_t P_SMEM_BYTES = 1024 + (size_t)P_STAGES * P_STAGE_BYTES + 256 + 4 * 32 * 144 + 3072;
+constexpr uint32_t kPeerMask = 0xFEFFFFFFu;  // clears the cluster-rank bit of a shared::cluster address: the pair's rank-0 CTA
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// tensor-map copy whose completion bytes are counted on the LEADER CTA's mbarrier (same offset, rank bit cleared)
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar_local) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar_local & kPeerMask)
+        : "memory");
+}
+__device__ __forceinline__ void umma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrives (once the MMAs issued so far have retired) on the barrier at this offset in BOTH CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"((uint16_t)3)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar_local) {
+    asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_local & kPeerMask) : "memory");
+}
+
+__global__ void __launch_bounds__(THREADS, 1)
+gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __restrict__ table_g, int* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    // the rounding of the base is the same in both CTAs (same launch, same dynamic offset), so operand offsets match
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)P_STAGES * P_STAGE_BYTES);
+    uint64_t* full_bar = bars;                    // [P_STAGES] leader: both CTAs' operand bytes landed
+    uint64_t* empty_bar = bars + P_STAGES;        // [P_STAGES] each CTA: the MMAs that read the stage retired
+    uint64_t* tfull_bar = bars + 2 * P_STAGES;    // [2] each CTA: accumulator buffer complete
+    uint64_t* tempty_bar = tfull_bar + 2;         // [2] leader: drained by the 8 epilogue warps of the pair
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint8_t* table_s = smem + (size_t)P_STAGES * P_STAGE_BYTES + 256 + 4 * STAGE_OUT_BYTES;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const bool leader = rank == 0;
+    const int pair = (int)blockIdx.x >> 1, n_pairs = (int)gridDim.x >> 1;
+    for (int o = threadIdx.x * 16; o < (int)kGroupTableBytes; o += THREADS * 16)
+        *reinterpret_cast<uint4*>(table_s + o) = *reinterpret_cast<const uint4*>(table_g + o);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < P_STAGES; ++s) {
+            mbar_init(smem_u32(full_bar + s), 1);
+            mbar_init(smem_u32(empty_bar + s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(tfull_bar + b), 1);
+            mbar_init(smem_u32(tempty_bar + b), 8);
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {  // the same warp of both CTAs allocates for the pair
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();  // the peer's barriers are initialised before anything arrives on them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const GemmGroupHeader hdr = *reinterpret_cast<const GemmGroupHeader*>(table_s);
+    const int total_tiles = hdr.total_tiles;  // counted in 256 x 256 pair tiles (m_tiles = ceil(M / 256))
+    TileWalk walk{reinterpret_cast<const GemmProblem*>(table_s + sizeof(GemmGroupHeader)), hdr.count, 0};
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer (both CTAs)
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+                const GemmProblem& p = walk.find(tile);
+                const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
+                const int k_blocks = p.K / BK;
+                // rows (of 128 bytes) of this CTA's operand images inside the mapped region
+                const int a_row = (int)((reinterpret_cast<unsigned long long>(p.a_tiles) - hdr.region_base) >> 7) +
+                                  (2 * mt + (int)rank) * k_blocks * 128;
+                const int b_row = (int)((reinterpret_cast<unsigned long long>(p.codes) - hdr.region_base) >> 7) +
+                                  nt * k_blocks * 256 + (int)rank * 128;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t fb = smem_u32(full_bar + stage);
+                    if (leader) mbar_expect_tx(fb, 2 * P_STAGE_BYTES);  // its own copies and the peer's
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * P_STAGE_BYTES);
+                    tma_load_2d_pair(sa, &map, 0, a_row + kb * 128, fb);
+                    tma_load_2d_pair(sa + P_HALF_BYTES, &map, 0, b_row + kb * 256, fb);
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader CTA only)
+        if (leader && lane == 0) {
+            constexpr uint32_t idesc = make_idesc(256, BN);
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            int iter = 0;
+            for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++iter) {
+                const int k_blocks = walk.find(tile).K / BK;
+                const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
+                if (!mbar_wait(smem_u32(tempty_bar + buf), bphase ^ 1u, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * BN;
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!mbar_wait(smem_u32(full_bar + stage), phase, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + (size_t)stage * P_STAGE_BYTES);
+                    const uint64_t a_desc = make_smem_desc(sa);
+                    const uint64_t b_desc = make_smem_desc(sa + P_HALF_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k)
+                        umma_i8_pair(d_tmem, a_desc + (uint64_t)(k * UMMA_K / 16), b_desc + (uint64_t)(k * UMMA_K / 16), idesc,
+                                     (uint32_t)((kb | k) != 0));
+                    umma_commit_pair(smem_u32(empty_bar + stage));  // frees the stage in both CTAs
+                    if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit_pair(smem_u32(tfull_bar + buf));
+            }
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
+        const int quad = warp & 3;
+        const uint32_t stage_s = smem_u32(smem + (size_t)P_STAGES * P_STAGE_BYTES + 256) + (uint32_t)quad * STAGE_OUT_BYTES;
+        bool ok = true;
+        int iter = 0;
+        for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++iter) {
+            const GemmProblem& p = walk.find(tile);
+            const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
+            const uint32_t buf = (uint32_t)iter & 1u, bphase = ((uint32_t)iter >> 1) & 1u;
+            const int m_warp = mt * 256 + (int)rank * 128 + quad * 32;
+            if (!mbar_wait(smem_u32(tfull_bar + buf), bphase, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            drain_accumulator(p, tmem_base + ((uint32_t)(quad * 32) << 16) + buf * BN, m_warp, nt * BN, stage_s, lane);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_leader(smem_u32(tempty_bar + buf));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+        if (threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
+        __syncthreads();
+    }
+    cluster_sync_all();  // neither CTA frees tensor memory or leaves while the other may still use the pair's resources
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
 }
 
@@ -421,11 +617,25 @@ bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows)
 }  // namespace
 
 size_t gemm_codes_bytes(int N, int K) { return (size_t)((N + BN - 1) / BN) * BN * K; }  // whole 256-row tiles
-size_t gemm_a_tiles_bytes(int M, int K) { return (size_t)((M + BM - 1) / BM) * BM * K; }  // whole 128-row tiles
+size_t gemm_a_tiles_bytes(int M, int K) { return (size_t)((M + 255) / 256) * 256 * K; }  // whole pairs of 128-row tiles
 size_t gemm_scratch_bytes(int N, int K) { return align_up(gemm_codes_bytes(N, K), 256) + align_up(kGroupTableBytes, 256); }
 
+// The whole region [base, base + bytes) as a matrix of 128-byte rows, box = 128 rows, no swizzle: a tile image (stored
+// swizzled) is copied as it is.
+bool make_map_rows128(CUtensorMap* map, const void* base, size_t bytes) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || (reinterpret_cast<uintptr_t>(base) & 127u) || bytes < 128 * 128) return false;
+    const cuuint64_t dims[2] = {128, (cuuint64_t)(bytes / 128)};
+    const cuuint64_t strides[1] = {128};
+    const cuuint32_t box[2] = {128, 128};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev,
-                cudaStream_t st) {
+                cudaStream_t st, const void* region_base, size_t region_bytes) {
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     static int sm_count = 0;
@@ -433,6 +643,8 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
         attr_err = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
         if (attr_err == cudaSuccess)
             attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
+        if (attr_err == cudaSuccess)
+            attr_err = cudaFuncSetAttribute(gemm_i8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P_SMEM_BYTES);
         int dev = 0;
         if (attr_err == cudaSuccess) attr_err = cudaGetDevice(&dev);
         if (attr_err == cudaSuccess) attr_err = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
@@ -445,21 +657,44 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     alignas(16) uint8_t host[kGroupTableBytes] = {};
     GemmGroupHeader* hdr = reinterpret_cast<GemmGroupHeader*>(host);
     GemmProblem* tab = reinterpret_cast<GemmProblem*>(host + sizeof(GemmGroupHeader));
+    // CTA pairs (256 x 256 tiles) when the operands are tile images inside one mapped region and the SMs pair up
+    const bool pairs = a_tiled && region_base != nullptr && (sm_count % 2) == 0;
+    const int tile_m = pairs ? 256 : BM;
     int tiles = 0;
     for (int i = 0; i < count; ++i) {
-        probs[i].m_tiles = (probs[i].M + BM - 1) / BM;
+        probs[i].m_tiles = (probs[i].M + tile_m - 1) / tile_m;
         probs[i].tile_begin = tiles;
         tiles += probs[i].m_tiles * ((probs[i].N + BN - 1) / BN);
         tab[i] = probs[i];
     }
     hdr->count = count;
     hdr->total_tiles = tiles;
+    hdr->region_base = reinterpret_cast<unsigned long long>(region_base);
     if (cudaMemcpyAsync(table_dev, host, kGroupTableBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
     CUtensorMap map_a;
     memset(&map_a, 0, sizeof(map_a));
+    if (pairs) {
+        if (!make_map_rows128(&map_a, region_base, region_bytes)) return BITLINEAR_ERR_CUDA;
+        int n_pairs = tiles < sm_count / 2 ? tiles : sm_count / 2;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(2 * n_pairs));
+        cfg.blockDim = dim3(THREADS);
+        cfg.dynamicSmemBytes = P_SMEM_BYTES;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_i8_pair_kernel, map_a, (const uint8_t*)table_dev, device_status_word());
+        if (e != cudaSuccess) cudaGetLastError();
+        return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+    }
     if (!a_tiled && !make_map(&map_a, xq_row_major, probs[0].M, probs[0].K, BM)) return BITLINEAR_ERR_CUDA;
     const int grid = tiles < sm_count ? tiles : sm_count;
     if (a_tiled) gemm_i8_kernel<true><<<grid, THREADS, SMEM_BYTES, st>>>(map_a, table_dev, device_status_word());

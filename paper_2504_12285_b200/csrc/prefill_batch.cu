@@ -184,7 +184,7 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
         group_unpack_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(items_dev, n, words);
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
-        const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st);
+        const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st, base, L.total);
         if (rc != BITLINEAR_OK) return rc;
     }
     return BITLINEAR_OK;
