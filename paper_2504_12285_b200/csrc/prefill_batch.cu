@@ -3,11 +3,12 @@
 // the 8-bit activations; here the expansion and the activation quantiser write directly the shared-memory images of
 // the tensor-core kernel's tiles, and one persistent kernel runs the tiles of every matmul of the group.)
 //
-//   launch 1  group_quant_kernel  : one warp per token - fused RMSNorm + absmax int8 quantiser; codes go into
+//   launch 1  group_quant_warp_kernel : one warp per token - fused RMSNorm + absmax int8 quantiser; codes go into
 //                                   128 x 128 tile images (128-byte swizzle) of the activation operand.  Problems
 //                                   that read the same activations share one quantised copy.
 //   launch 2  group_unpack_kernel : packed 2-bit weights -> byte codes in 256 x 128 tile images.
-//   launch 3  gemm_i8_kernel<true>: every tile of every matmul, operands fetched with linear bulk copies.
+//   launch 3  gemm_i8_pair_kernel : every tile of every matmul on CTA pairs (gemm_i8_kernel<true> when the SMs do not
+//                                   pair up), operands fetched as whole tile images.
 // Problems are ordered by decreasing K so that the long tiles are scheduled first and the tail is made of short ones.
 #include <algorithm>
 #include <vector>
@@ -34,20 +35,7 @@ struct PrefillItem {
 };
 constexpr size_t kItemTableBytes = kMaxGroup * sizeof(PrefillItem);
 
-template <int VPT>
-__global__ void __launch_bounds__(kQuantThreads) group_quant_kernel(const PrefillItem* __restrict__ items, int count) {
-    __shared__ RowReduceSmem sm;
-    const int row = blockIdx.x;
-    int i = 0;
-    while (i + 1 < count && row >= items[i + 1].row_begin) ++i;
-    const PrefillItem& p = items[i];
-    const int m = row - p.row_begin;
-    uint8_t* dst = p.a_tiles + (size_t)(m >> 7) * (p.K >> 7) * (128 * 128) + (size_t)(m & 127) * 128;
-    quant_row<VPT, 2>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, reinterpret_cast<int8_t*>(dst), p.d + m, p.xsum + m, sm,
-                      m & 7);
-}
-
-// Warp-per-row variant (eight rows per CTA).
+// One warp per token, eight tokens per CTA.
 __global__ void __launch_bounds__(kQuantThreads) group_quant_warp_kernel(const PrefillItem* __restrict__ items, int count,
                                                                          int rows) {
     const int row = blockIdx.x * kQuantWarps + (threadIdx.x >> 5);
@@ -135,7 +123,7 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
         PrefillItem items[kMaxGroup] = {};
         GemmProblem gp[kMaxGroup] = {};
         long long words = 0;
-        int rows = 0, max_k = 0;
+        int rows = 0;
         for (int i = 0; i < n; ++i) {
             const bitlinear_problem& q = problems[idx[i]];
             PrefillItem& it = items[i];
@@ -162,7 +150,6 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             } else {
                 rows += q.M;
             }
-            if (q.K > max_k) max_k = q.K;
             GemmProblem& g = gp[i];
             g.a_tiles = it.a_tiles; g.codes = it.codes; g.d = it.d; g.xsum = it.xsum; g.s_w = q.s_w;
             g.y = q.y; g.acc_out = nullptr;
@@ -173,15 +160,11 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             cudaGetLastError();
             return BITLINEAR_ERR_CUDA;
         }
-        const int vpt = (max_k / 8 + kQuantThreads - 1) / kQuantThreads;
-        const dim3 g((unsigned)rows), blk(kQuantThreads), gw((unsigned)((rows + kQuantWarps - 1) / kQuantWarps));
-        if (skip_quant) {
-        } else if (true) group_quant_warp_kernel<<<gw, blk, 0, st>>>(items_dev, n, rows);
-        else if (vpt <= 1) group_quant_kernel<1><<<g, blk, 0, st>>>(items_dev, n);
-        else if (vpt <= 2) group_quant_kernel<2><<<g, blk, 0, st>>>(items_dev, n);
-        else if (vpt <= 4) group_quant_kernel<4><<<g, blk, 0, st>>>(items_dev, n);
-        else group_quant_kernel<8><<<g, blk, 0, st>>>(items_dev, n);
-        if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+        if (!skip_quant) {
+            const unsigned blocks = (unsigned)((rows + kQuantWarps - 1) / kQuantWarps);
+            group_quant_warp_kernel<<<blocks, kQuantThreads, 0, st>>>(items_dev, n, rows);
+            if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+        }
         group_unpack_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(items_dev, n, words);
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
         const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st, base, L.total);
