@@ -502,18 +502,25 @@ namespace bitlinear {
 size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const int* idx, int n);
 int prefill_group_forward(const bitlinear_problem* problems, const int* idx, int n, void* ws, bool skip_quant,
                           cudaStream_t st);
+// Sub-batches with a problem of more than kDp4aMaxTokens tokens run on the tensor cores (decode_mma.cu).
+size_t decode_mma_workspace_bytes(const bitlinear_problem* problems, int count);
+int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes, void* stream);
+constexpr int kDp4aMaxTokens = 4;
 
 namespace {
 
 size_t decode_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
     if (!problems || count <= 0) return 0;
     size_t xq = 0, rows = 0;
+    int max_m = 0;
     for (int i = 0; i < count; ++i) {
         const bitlinear_problem& q = problems[i];
         if (q.M < 0 || q.M > kGemvMaxTokens || !shape_ok(q.N, q.K) || q.K > kBatchMaxK) return 0;
         xq += align_up((size_t)q.M * q.K, 16);
         rows += (size_t)q.M;
+        if (q.M > max_m) max_m = q.M;
     }
+    if (max_m > kDp4aMaxTokens) return decode_mma_workspace_bytes(problems, count);
     return plan_layout(count, kPlanGrid, xq, rows).total;
 }
 
@@ -535,6 +542,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         if (q.M > max_m) max_m = q.M;
         if (q.K > max_k) max_k = q.K;
     }
+    if (max_m > kDp4aMaxTokens) return decode_mma_forward(problems, count, flags, ws, ws_bytes, stream);
     const PlanLayout L = plan_layout(count, kPlanGrid, xq_bytes, rows);
     if (!ws || !aligned16(ws) || ws_bytes < L.total) return BITLINEAR_ERR_WORKSPACE;
     if (rows == 0) return BITLINEAR_OK;

@@ -68,6 +68,8 @@ __device__ __forceinline__ double sum_squares8(const float (&f)[8]) {
 // LAYOUT 2: tensor-core tile images: xq_row points at this row inside the first 128-row x 128-column tile of its
 //           row tile (tiles of 16 KiB follow each other along K); 16-byte piece p of a row sits at (p ^ swz) * 16,
 //           swz = row & 7 - the 128-byte shared-memory swizzle.
+// LAYOUT 3: the same with tiles of 16 rows x 128 columns (2 KiB): the token-side operand of the decode kernel that
+//           runs on the tensor cores with the tokens as the narrow dimension.
 template <int VPT, int LAYOUT = 0>  // VPT = 16-byte vectors (8 bf16) per thread
 __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_row,
                                           const __nv_bfloat16* __restrict__ gain, float eps, int K,
@@ -151,9 +153,9 @@ __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_ro
         if (LAYOUT == 1) {
             const int piece = (v >> 1) & 15;  // 16-byte piece inside the 256-column block: 4t + q
             dst = (v & ~31) | ((((piece & 3) << 2) | (piece >> 2)) << 1) | (v & 1);
-        } else if (LAYOUT == 2) {
+        } else if (LAYOUT == 2 || LAYOUT == 3) {
             const int kb = v >> 4, piece = (v >> 1) & 7;  // 128-column tile along K, 16-byte piece in the row
-            dst = kb * (128 * 128 / 8) + (((piece ^ swz) << 1) | (v & 1));
+            dst = kb * ((LAYOUT == 2 ? 128 : 16) * 128 / 8) + (((piece ^ swz) << 1) | (v & 1));
         }
         if (v < n_vec) qrow[dst] = make_uint2(packed[0], packed[1]);
     }
@@ -238,9 +240,9 @@ __device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__
         if (LAYOUT == 1) {
             const int piece = (v >> 1) & 15;
             dst = (v & ~31) | ((((piece & 3) << 2) | (piece >> 2)) << 1) | (v & 1);
-        } else if (LAYOUT == 2) {
+        } else if (LAYOUT == 2 || LAYOUT == 3) {
             const int kb = v >> 4, piece = (v >> 1) & 7;
-            dst = kb * (128 * 128 / 8) + (((piece ^ swz) << 1) | (v & 1));
+            dst = kb * ((LAYOUT == 2 ? 128 : 16) * 128 / 8) + (((piece ^ swz) << 1) | (v & 1));
         }
         qrow[dst] = make_uint2(packed[0], packed[1]);
     }

@@ -130,6 +130,36 @@ def test_batch_detects_an_overwritten_plan():
     check(batch, refs)
 
 
+def test_batch_many_tokens_bf16_ragged_rows_and_overwritten_plan():
+    # 5 to 16 tokens: the tensor-core decode kernel; weight-row counts that are not multiples of 128,
+    # one K that is a single 256-column step and one that ends in a partial ring slot (27 steps)
+    shapes = [(7, 16, 256), (16, 144, 6912), (0, 32, 256), (5, 2560, 1280), (11, 272, 2560), (1, 96, 512)]
+    batch, refs = make_case(shapes, 700, y_dtype=torch.bfloat16, gains=True)
+    run(batch, reuse=True)
+    check(batch, refs)
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    bl.bitlinear_forward_batch(batch, ws)
+    torch.cuda.synchronize()
+    ws[:256].zero_()
+    for t in batch.tensors:
+        t[4].fill_(7.0)
+    bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
+    assert bl.bitlinear_poll_status() == 4
+    for t in batch.tensors:
+        assert torch.all(t[4] == 7.0)
+    assert bl.bitlinear_poll_status() == 0
+
+
+@pytest.mark.parametrize("M", [5, 8, 16])
+def test_batch_many_tokens_match_single_forward_bitwise(M):
+    shapes = [(M, n, k) for _, n, k in wl.LAYER_SHAPES[:4]]
+    batch, _ = make_case(shapes, 800 + M)
+    run(batch)
+    for x, g, packed, s_w, y in batch.tensors:
+        y1 = bl.bitlinear_forward(x, g, packed, s_w, y.shape[1], wl.RMS_EPS)
+        assert torch.equal(y, y1)
+
+
 # ---- problems of more than 16 tokens in the same entry point: grouped tensor-core path ----
 
 
