@@ -8,7 +8,7 @@
 //   warp 0      producer : bulk copies of packed weights (eight 16-row blocks x up to four 16x256 tiles, 4 KiB each)
 //                          and of the matching slice of the quantised tokens (16-row tile images) into a 2-slot ring
 //   warps 1-8   unpack   : warp w expands row block w of the current 256-column step: 2-bit codes -> bytes, written
-//                          as the 128-byte-swizzled K-major operand image the tensor core reads (2 stages of 32 KiB)
+//                          as the 128-byte-swizzled K-major operand image the tensor core reads (4 stages of 32 KiB)
 //   warp 9      MMA      : one thread issues 8 tcgen05.mma (128 x 16 x 32) per 256-column step and commits
 //   warps 10-13 epilogue : tcgen05.ld of the finished 128 x 16 accumulator (double buffered), minus the code sum,
 //                          two fp32 multiplies, stores coalesced along the weight rows
@@ -31,8 +31,10 @@ constexpr int kMmaThreads = (1 + kUnpackWarps + 1 + 4) * 32;
 constexpr uint32_t kPackedSlot = 8 * kStepTiles * kTileBytes;  // 32 KiB of packed weights
 constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;       // 16 KiB: 8 k-blocks of 16 x 128 token images
 constexpr uint32_t kAStage = 2 * kRows * 128;                  // 32 KiB: two k-blocks of 128 x 128 weight codes
-constexpr uint32_t kTmemCols = 32;                             // two accumulators of 16 columns
-constexpr size_t kMmaSmem = 1024 + 2 * (size_t)(kPackedSlot + kXSlot) + 2 * (size_t)kAStage + 256;
+constexpr int kSplit = 8;        // partial accumulators per item: the 8 MMAs of a step do not wait on each other
+constexpr uint32_t kTmemCols = 2 * kSplit * kTok;              // two buffers of kSplit accumulators of 16 columns
+constexpr int kStages = 4;       // operand images of the weights in flight between unpack and MMA
+constexpr size_t kMmaSmem = 1024 + 2 * (size_t)(kPackedSlot + kXSlot) + kStages * (size_t)kAStage + 256;
 
 struct MmaProblem {
     const uint8_t* packed;
@@ -139,14 +141,14 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
 __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t a_s = smem_u32(smem);                          // [2] operand images of the weights
-    const uint32_t x_s = a_s + 2 * kAStage;                       // [2] token images
+    const uint32_t a_s = smem_u32(smem);                          // [kStages] operand images of the weights
+    const uint32_t x_s = a_s + kStages * kAStage;                 // [2] token images
     const uint32_t p_s = x_s + 2 * kXSlot;                        // [2] packed weights
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * (size_t)(kAStage + kXSlot + kPackedSlot));
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * (size_t)kAStage + 2 * (size_t)(kXSlot + kPackedSlot));
     const uint32_t pfull = smem_u32(bars + 0), pempty = smem_u32(bars + 2), xempty = smem_u32(bars + 4);
-    const uint32_t afull = smem_u32(bars + 6), aempty = smem_u32(bars + 8);
-    const uint32_t tfull = smem_u32(bars + 10), tempty = smem_u32(bars + 12);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 14);
+    const uint32_t tfull = smem_u32(bars + 6), tempty = smem_u32(bars + 8);
+    const uint32_t afull = smem_u32(bars + 10), aempty = smem_u32(bars + 10 + kStages);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10 + 2 * kStages);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -160,10 +162,12 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             mbar_init(pfull + 8 * b, 1);
             mbar_init(pempty + 8 * b, kUnpackWarps);
             mbar_init(xempty + 8 * b, 1);
-            mbar_init(afull + 8 * b, kUnpackWarps);
-            mbar_init(aempty + 8 * b, 1);
             mbar_init(tfull + 8 * b, 1);
             mbar_init(tempty + 8 * b, 4);
+        }
+        for (int b = 0; b < kStages; ++b) {
+            mbar_init(afull + 8 * b, kUnpackWarps);
+            mbar_init(aempty + 8 * b, 1);
         }
         *abort_flag = 0;
         mbar_init_fence();
@@ -222,23 +226,31 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 const uint32_t slot = sc_idx & 1u, phase = (sc_idx >> 1) & 1u;
                 if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
                 for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                    const uint32_t stage = st_idx & 1u, sphase = (st_idx >> 1) & 1u;
-                    if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t stage = st_idx % kStages, sphase = (st_idx / kStages) & 1u;
+                    uint4 pv[2] = {};
                     if (w < n_rb) {
                         const uint32_t src = p_s + slot * kPackedSlot + (uint32_t)w * (kStepTiles * kTileBytes) +
                                              (uint32_t)kt * kTileBytes + (uint32_t)lane * 16u;
+                        pv[0] = lds128(src);
+                        pv[1] = lds128(src + 512u);
+                    }
+                    if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (w < n_rb) {
                         // lane (g, t) holds rows g and 8+g of the 16-row block, columns 64t .. 64t+63 of the 256:
                         // k-block t >> 1, 16-byte pieces 4*(t & 1) + q of the 128-byte operand row
                         const uint32_t dst = a_s + stage * kAStage + (uint32_t)(t >> 1) * (kRows * 128) +
                                              (uint32_t)(w * 16 + g) * 128u;
+                        // lanes of the upper k-block take their words in the order 2, 3, 0, 1: the eight lanes
+                        // that store together then hit eight different 16-byte bank groups
+                        const bool up = (t & 2) != 0;
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            const uint4 pv = lds128(src + 512u * h);
-                            const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
+                            const uint32_t pw[4] = {up ? pv[h].z : pv[h].x, up ? pv[h].w : pv[h].y, up ? pv[h].x : pv[h].z,
+                                                    up ? pv[h].y : pv[h].w};
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
                                 const uint32_t v = pw[q];
-                                const uint32_t piece = (uint32_t)(4 * (t & 1) + q) ^ (uint32_t)g;  // row & 7 == g
+                                const uint32_t piece = (uint32_t)(4 * (t & 1) + (q ^ (t & 2))) ^ (uint32_t)g;  // row & 7 == g
                                 sts128(dst + 1024u * h + (piece << 4), v & 0x03030303u, (v >> 2) & 0x03030303u,
                                        (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
                             }
@@ -263,13 +275,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
                 if (!mbar_wait(tempty + 8 * buf, bphase ^ 1u, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * kTok;
+                const uint32_t d_tmem = tmem_base + buf * (kSplit * kTok);
                 for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                     const int tiles = min(kStepTiles, k_tiles - t0);
                     const uint32_t slot = sc_idx & 1u, phase = (sc_idx >> 1) & 1u;
                     if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }  // the token images landed
                     for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                        const uint32_t stage = st_idx & 1u, sphase = (st_idx >> 1) & 1u;
+                        const uint32_t stage = st_idx % kStages, sphase = (st_idx / kStages) & 1u;
                         if (!mbar_wait(afull + 8 * stage, sphase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
 #pragma unroll
@@ -278,8 +290,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                             const uint64_t b_desc = smem_desc_sw128(x_s + slot * kXSlot + (uint32_t)(kt * 2 + kb) * (kTok * 128));
 #pragma unroll
                             for (int k = 0; k < 4; ++k)
-                                umma_i8(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), kIdesc,
-                                        (uint32_t)((t0 | kt | kb | k) != 0));
+                                umma_i8(d_tmem + (uint32_t)((kb * 4 + k) * kTok), a_desc + (uint64_t)(2 * k),
+                                        b_desc + (uint64_t)(2 * k), kIdesc, (uint32_t)((t0 | kt) != 0));
                         }
                         umma_commit(aempty + 8 * stage);  // the stage may be rewritten once these MMAs retire
                     }
@@ -305,7 +317,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             if (!mbar_wait(tfull + 8 * buf, bphase, abort_flag)) break;
             tc_fence_after();
             uint32_t r[16];
-            tmem_ld_32x16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kTok, r);
+            tmem_ld_32x16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * (kSplit * kTok), r);
+#pragma unroll
+            for (int sp = 1; sp < kSplit; ++sp) {  // integer partial sums: any order gives the same total
+                uint32_t r2[16];
+                tmem_ld_32x16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * (kSplit * kTok) + sp * kTok, r2);
+#pragma unroll
+                for (int m = 0; m < kTok; ++m) r[m] += r2[m];
+            }
             const int n = item.y * kTileRows + quad * 32 + lane;  // this lane's weight row
 #pragma unroll
             for (int m = 0; m < kTok; ++m) {
