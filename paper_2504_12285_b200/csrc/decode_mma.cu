@@ -1,17 +1,18 @@
-// Batched decode for 5 to 16 tokens per matmul on the tensor cores, tokens as the NARROW operand.
+// Batched decode for 5 to 16 tokens per matmul on the tensor cores.
 // (Paper Section 5.1: packed weights are loaded from HBM into shared memory and unpacked there right before the
 // product with the 8-bit activations.  With more than a few tokens the dot-product-of-four kernel is bound by its
-// arithmetic - one instruction per token per four weights - so here the product runs on tcgen05: D[128 weight rows x
-// 16 tokens] += A[128 x 32 weight codes (u8)] x B[16 x 32 activations (s8)], accumulators in tensor memory.)
+// arithmetic - one instruction per token per four weights - so here the product runs on tcgen05.  The time of one
+// tcgen05.mma grows with the rows of its A operand and hardly with its N, so the weights are the wide, stationary
+// B operand: D[tokens (16 of M = 64 rows) x 256 weight rows] += A[tokens x 32 activations (s8)] x B[256 x 32 codes (u8)].)
 //
-// One persistent CTA per SM owns a contiguous, byte-balanced range of work items (128 weight rows of one matmul).
-//   warp 0      producer : bulk copies of packed weights (eight 16-row blocks x up to four 16x256 tiles, 4 KiB each)
-//                          and of the matching slice of the quantised tokens (16-row tile images) into a 2-slot ring
-//   warps 1-8   unpack   : warp w expands row block w of the current 256-column step: 2-bit codes -> bytes, written
-//                          as the 128-byte-swizzled K-major operand image the tensor core reads (4 stages of 32 KiB)
-//   warp 9      MMA      : one thread issues 8 tcgen05.mma (128 x 16 x 32) per 256-column step and commits
-//   warps 10-13 epilogue : tcgen05.ld of the finished 128 x 16 accumulator (double buffered), minus the code sum,
-//                          two fp32 multiplies, stores coalesced along the weight rows
+// One persistent CTA per SM owns a contiguous, byte-balanced range of work items (256 weight rows of one matmul).
+//   warp 0      epilogue : tcgen05.ld of the finished accumulator (token m in lane m; double buffered), minus the
+//                          code sum, two fp32 multiplies, 16-byte stores
+//   warp 1      producer : bulk copies of packed weights (sixteen 16-row blocks x up to two 16x256 tiles) and of the
+//                          matching slice of the quantised tokens (16-row tile images) into a 2-slot ring
+//   warp 2      MMA      : one thread issues 8 tcgen05.mma (64 x 256 x 32) per 256-column step and commits
+//   warps 3-10  unpack   : warp w expands row blocks 2w and 2w+1 of the current 256-column step: 2-bit codes -> bytes,
+//                          written as two 128-byte-swizzled K-major operand images of 256 rows (2 stages of 64 KiB)
 // Every wait is bounded; on a timeout the CTA raises the sticky status word and leaves.
 #include <algorithm>
 #include <vector>
@@ -23,18 +24,21 @@ namespace bitlinear {
 
 namespace {
 
-constexpr int kRows = 128;        // weight rows per work item = tensor-memory lanes
-constexpr int kTok = 16;          // tokens per matmul, padded (UMMA N)
-constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1024 columns)
-constexpr int kUnpackWarps = 8;   // one per 16-row block of an item
-constexpr int kMmaThreads = (1 + kUnpackWarps + 1 + 4) * 32;
-constexpr uint32_t kPackedSlot = 8 * kStepTiles * kTileBytes;  // 32 KiB of packed weights
-constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;       // 16 KiB: 8 k-blocks of 16 x 128 token images
-constexpr uint32_t kAStage = 2 * kRows * 128;                  // 32 KiB: two k-blocks of 128 x 128 weight codes
-constexpr int kSplit = 8;        // partial accumulators per item: the 8 MMAs of a step do not wait on each other
-constexpr uint32_t kTmemCols = 2 * kSplit * kTok;              // two buffers of kSplit accumulators of 16 columns
-constexpr int kStages = 4;       // operand images of the weights in flight between unpack and MMA
-constexpr size_t kMmaSmem = 1024 + 2 * (size_t)(kPackedSlot + kXSlot) + kStages * (size_t)kAStage + 256;
+constexpr int kItemRb = 16;       // 16-row blocks per work item
+constexpr int kItemRows = kItemRb * kTileRows;  // 256 weight rows = UMMA N
+constexpr int kTok = 16;          // tokens per matmul, padded; the MMA computes 64 rows of which 16 are read
+constexpr int kMmaM = 64;
+constexpr int kStepTiles = 2;     // 16x256 tiles per row block per ring slot (512 columns)
+constexpr int kUnpackWarps = 8;   // two row blocks each
+constexpr int kEpiWarp = 0, kProdWarp = 1, kMmaWarp = 2, kFirstUnpackWarp = 3;
+constexpr int kMmaThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;
+constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;              // 8 KiB: 4 k-blocks of 16 x 128 token images
+constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;   // 32 KiB of packed weights
+constexpr uint32_t kKbImage = kItemRows * 128;                        // 32 KiB: 256 rows x 128 codes
+constexpr uint32_t kStage = 2 * kKbImage;                             // one 256-column step
+constexpr int kStages = 2;
+constexpr uint32_t kTmemCols = 2 * kItemRows;                         // two accumulators of 256 columns
+constexpr size_t kMmaSmem = 1024 + 2 * (size_t)(kXSlot + kPackedSlot) + kStages * (size_t)kStage + 256;
 
 struct MmaProblem {
     const uint8_t* packed;
@@ -64,7 +68,7 @@ constexpr unsigned kMmaMagic = 0xB171A9E7u;
 struct MmaParams {
     const MmaHeader* hdr;
     const MmaProblem* probs;
-    const int2* items;      // {problem, first row block of the item (a multiple of 8)}
+    const int2* items;      // {problem, first row block of the item (a multiple of 16)}
     const int* cta_begin;   // [grid + 1]
     int count, total_items, rows;
     int* status_word;
@@ -89,6 +93,7 @@ __device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
+// Lane l of the warp receives 16 consecutive columns of tensor-memory lane (taddr lane + l).
 __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -109,8 +114,8 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
     desc |= (uint64_t)2 << 61;
     return desc;
 }
-// D = s32, A = u8 (weight codes), B = s8 (activations), both K-major, M = 128, N = 16.
-constexpr uint32_t kIdesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
+// D = s32, A = s8 (activations), B = u8 (weight codes), both K-major, M = 64, N = 256.
+constexpr uint32_t kIdesc = (2u << 4) | (1u << 7) | (0u << 10) | ((uint32_t)(kItemRows >> 3) << 17) | ((uint32_t)(kMmaM >> 4) << 24);
 
 template <int VPT>
 __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeader* __restrict__ hdr,
@@ -141,13 +146,15 @@ __device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, ui
 __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    const uint32_t a_s = smem_u32(smem);                          // [kStages] operand images of the weights
-    const uint32_t x_s = a_s + kStages * kAStage;                 // [2] token images
-    const uint32_t p_s = x_s + 2 * kXSlot;                        // [2] packed weights
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kStages * (size_t)kAStage + 2 * (size_t)(kXSlot + kPackedSlot));
+    // The token images come first: the MMA reads 64 operand rows where 16 are stored, and what it reads past them
+    // (rows whose results nobody looks at) must still be this CTA's shared memory.
+    const uint32_t x_s = smem_u32(smem);          // [2] token images
+    const uint32_t p_s = x_s + 2 * kXSlot;        // [2] packed weights
+    const uint32_t b_s = p_s + 2 * kPackedSlot;   // [kStages] operand images of the weights
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * (size_t)(kXSlot + kPackedSlot) + kStages * (size_t)kStage);
     const uint32_t pfull = smem_u32(bars + 0), pempty = smem_u32(bars + 2), xempty = smem_u32(bars + 4);
     const uint32_t tfull = smem_u32(bars + 6), tempty = smem_u32(bars + 8);
-    const uint32_t afull = smem_u32(bars + 10), aempty = smem_u32(bars + 10 + kStages);
+    const uint32_t bfull = smem_u32(bars + 10), bempty = smem_u32(bars + 10 + kStages);
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10 + 2 * kStages);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -163,16 +170,16 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             mbar_init(pempty + 8 * b, kUnpackWarps);
             mbar_init(xempty + 8 * b, 1);
             mbar_init(tfull + 8 * b, 1);
-            mbar_init(tempty + 8 * b, 4);
+            mbar_init(tempty + 8 * b, 1);
         }
         for (int b = 0; b < kStages; ++b) {
-            mbar_init(afull + 8 * b, kUnpackWarps);
-            mbar_init(aempty + 8 * b, 1);
+            mbar_init(bfull + 8 * b, kUnpackWarps);
+            mbar_init(bempty + 8 * b, 1);
         }
         *abort_flag = 0;
         mbar_init_fence();
     }
-    if (warp == 9) {
+    if (warp == kMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -183,14 +190,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t tmem_base = *tmem_slot;
     const int item_lo = prm.cta_begin[blockIdx.x], item_hi = prm.cta_begin[blockIdx.x + 1];
 
-    if (warp == 0) {
+    if (warp == kProdWarp) {
         // ------------------------------------------------------------------ producer
         uint32_t sc_idx = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
             const int2 item = prm.items[it];
             const MmaProblem& p = prm.probs[item.x];
-            const int k_tiles = p.K / kTileCols, n_rb = min(8, p.N / kTileRows - item.y);
+            const int k_tiles = p.K / kTileCols, n_rb = min(kItemRb, p.N / kTileRows - item.y);
             const uint8_t* packed = p.packed;
             const uint8_t* x_img = p.x_img;
             for (int t0 = 0; t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
@@ -206,65 +213,71 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     bulk_load(p_s + slot * kPackedSlot + lane * (kStepTiles * kTileBytes),
                               packed + ((size_t)(item.y + lane) * k_tiles + t0) * kTileBytes, (uint32_t)tiles * kTileBytes,
                               pfull + 8 * slot);
-                else if (lane == 8)
+                else if (lane == kItemRb)
                     bulk_load(x_s + slot * kXSlot, x_img + (size_t)t0 * 2 * kTok * 128, (uint32_t)tiles * 2 * kTok * 128,
                               pfull + 8 * slot);
             }
         }
-    } else if (warp <= kUnpackWarps) {
-        // ------------------------------------------------------------------ unpack: warp w expands row block w
-        const int w = warp - 1;
+    } else if (warp >= kFirstUnpackWarp) {
+        // ------------------------------------------------------------------ unpack: warp w expands row blocks 2w, 2w+1
+        const int w = warp - kFirstUnpackWarp;
         const int g = lane >> 2, t = lane & 3;
+        // lanes of the upper k-block take their words in the order 2, 3, 0, 1: the eight lanes that store together
+        // then hit eight different 16-byte bank groups
+        const bool up = (t & 2) != 0;
         uint32_t sc_idx = 0, st_idx = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
             const int2 item = prm.items[it];
             const MmaProblem& p = prm.probs[item.x];
-            const int k_tiles = p.K / kTileCols, n_rb = min(8, p.N / kTileRows - item.y);
+            const int k_tiles = p.K / kTileCols, n_rb = min(kItemRb, p.N / kTileRows - item.y);
             for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                 const int tiles = min(kStepTiles, k_tiles - t0);
                 const uint32_t slot = sc_idx & 1u, phase = (sc_idx >> 1) & 1u;
                 if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
                 for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
                     const uint32_t stage = st_idx % kStages, sphase = (st_idx / kStages) & 1u;
-                    uint4 pv[2] = {};
-                    if (w < n_rb) {
-                        const uint32_t src = p_s + slot * kPackedSlot + (uint32_t)w * (kStepTiles * kTileBytes) +
-                                             (uint32_t)kt * kTileBytes + (uint32_t)lane * 16u;
-                        pv[0] = lds128(src);
-                        pv[1] = lds128(src + 512u);
+                    uint4 pv[2][2] = {};
+#pragma unroll
+                    for (int r = 0; r < 2; ++r) {
+                        if (2 * w + r < n_rb) {
+                            const uint32_t src = p_s + slot * kPackedSlot + (uint32_t)(2 * w + r) * (kStepTiles * kTileBytes) +
+                                                 (uint32_t)kt * kTileBytes + (uint32_t)lane * 16u;
+                            pv[r][0] = lds128(src);
+                            pv[r][1] = lds128(src + 512u);
+                        }
                     }
-                    if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
-                    if (w < n_rb) {
-                        // lane (g, t) holds rows g and 8+g of the 16-row block, columns 64t .. 64t+63 of the 256:
-                        // k-block t >> 1, 16-byte pieces 4*(t & 1) + q of the 128-byte operand row
-                        const uint32_t dst = a_s + stage * kAStage + (uint32_t)(t >> 1) * (kRows * 128) +
-                                             (uint32_t)(w * 16 + g) * 128u;
-                        // lanes of the upper k-block take their words in the order 2, 3, 0, 1: the eight lanes
-                        // that store together then hit eight different 16-byte bank groups
-                        const bool up = (t & 2) != 0;
+                    if (!mbar_wait(bempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            const uint32_t pw[4] = {up ? pv[h].z : pv[h].x, up ? pv[h].w : pv[h].y, up ? pv[h].x : pv[h].z,
-                                                    up ? pv[h].y : pv[h].w};
+                    for (int r = 0; r < 2; ++r) {
+                        if (2 * w + r < n_rb) {
+                            // lane (g, t) holds rows g and 8+g of the 16-row block, columns 64t .. 64t+63 of the 256:
+                            // k-block t >> 1, 16-byte pieces 4*(t & 1) + q of the 128-byte operand row
+                            const uint32_t dst = b_s + stage * kStage + (uint32_t)(t >> 1) * kKbImage +
+                                                 (uint32_t)((2 * w + r) * kTileRows + g) * 128u;
 #pragma unroll
-                            for (int q = 0; q < 4; ++q) {
-                                const uint32_t v = pw[q];
-                                const uint32_t piece = (uint32_t)(4 * (t & 1) + (q ^ (t & 2))) ^ (uint32_t)g;  // row & 7 == g
-                                sts128(dst + 1024u * h + (piece << 4), v & 0x03030303u, (v >> 2) & 0x03030303u,
-                                       (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
+                            for (int h = 0; h < 2; ++h) {
+                                const uint4 v4 = pv[r][h];
+                                const uint32_t pw[4] = {up ? v4.z : v4.x, up ? v4.w : v4.y, up ? v4.x : v4.z, up ? v4.y : v4.w};
+#pragma unroll
+                                for (int q = 0; q < 4; ++q) {
+                                    const uint32_t v = pw[q];
+                                    const uint32_t piece = (uint32_t)(4 * (t & 1) + (q ^ (t & 2))) ^ (uint32_t)g;  // row & 7 == g
+                                    sts128(dst + 1024u * h + (piece << 4), v & 0x03030303u, (v >> 2) & 0x03030303u,
+                                           (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
+                                }
                             }
                         }
-                        fence_async_smem();  // the tensor core reads these bytes through the async proxy
                     }
+                    fence_async_smem();  // the tensor core reads these bytes through the async proxy
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(afull + 8 * stage);
+                    if (lane == 0) mbar_arrive(bfull + 8 * stage);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pempty + 8 * slot);
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             uint32_t sc_idx = 0, st_idx = 0, it_idx = 0;
@@ -275,25 +288,25 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
                 if (!mbar_wait(tempty + 8 * buf, bphase ^ 1u, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * (kSplit * kTok);
+                const uint32_t d_tmem = tmem_base + buf * kItemRows;
                 for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                     const int tiles = min(kStepTiles, k_tiles - t0);
                     const uint32_t slot = sc_idx & 1u, phase = (sc_idx >> 1) & 1u;
                     if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }  // the token images landed
                     for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
                         const uint32_t stage = st_idx % kStages, sphase = (st_idx / kStages) & 1u;
-                        if (!mbar_wait(afull + 8 * stage, sphase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(bfull + 8 * stage, sphase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
 #pragma unroll
                         for (int kb = 0; kb < 2; ++kb) {
-                            const uint64_t a_desc = smem_desc_sw128(a_s + stage * kAStage + (uint32_t)kb * (kRows * 128));
-                            const uint64_t b_desc = smem_desc_sw128(x_s + slot * kXSlot + (uint32_t)(kt * 2 + kb) * (kTok * 128));
+                            const uint64_t a_desc = smem_desc_sw128(x_s + slot * kXSlot + (uint32_t)(kt * 2 + kb) * (kTok * 128));
+                            const uint64_t b_desc = smem_desc_sw128(b_s + stage * kStage + (uint32_t)kb * kKbImage);
 #pragma unroll
                             for (int k = 0; k < 4; ++k)
-                                umma_i8(d_tmem + (uint32_t)((kb * 4 + k) * kTok), a_desc + (uint64_t)(2 * k),
-                                        b_desc + (uint64_t)(2 * k), kIdesc, (uint32_t)((t0 | kt) != 0));
+                                umma_i8(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), kIdesc,
+                                        (uint32_t)((t0 | kt | kb | k) != 0));
                         }
-                        umma_commit(aempty + 8 * stage);  // the stage may be rewritten once these MMAs retire
+                        umma_commit(bempty + 8 * stage);  // the stage may be rewritten once these MMAs retire
                     }
                     if (ok) umma_commit(xempty + 8 * slot);
                 }
@@ -302,39 +315,45 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ epilogue
-        const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
+        // ------------------------------------------------------------------ epilogue (warp 0: tensor-memory lanes 0 .. 31)
         uint32_t it_idx = 0;
         for (int it = item_lo; it < item_hi; ++it, ++it_idx) {
             const int2 item = prm.items[it];
             const MmaProblem& p = prm.probs[item.x];
             const int M = p.M, N = p.N, y_dtype = p.y_dtype;
-            void* y = p.y;
             const float s_w = *p.s_w;
-            const int xs_lane = lane < M ? p.xsum[lane] : 0;
-            const float d_lane = lane < M ? p.d[lane] : 0.0f;
+            const bool live = lane < M;  // accumulator row m of the 64 sits in tensor-memory lane m for m < 16
+            const int xs = live ? p.xsum[lane] : 0;
+            const float dm = live ? p.d[lane] : 0.0f;
+            float* y32 = reinterpret_cast<float*>(p.y) + (size_t)lane * N;
+            __nv_bfloat16* y16 = reinterpret_cast<__nv_bfloat16*>(p.y) + (size_t)lane * N;
             const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
             if (!mbar_wait(tfull + 8 * buf, bphase, abort_flag)) break;
             tc_fence_after();
-            uint32_t r[16];
-            tmem_ld_32x16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * (kSplit * kTok), r);
+            for (int c = 0; c < kItemRb; ++c) {
+                const int n0 = (item.y + c) * kTileRows;  // first weight row of these 16 columns
+                if (n0 >= N) break;
+                uint32_t r[16];
+                tmem_ld_32x16(tmem_base + buf * kItemRows + (uint32_t)c * kTileRows, r);
+                if (live) {
+                    float v[16];
 #pragma unroll
-            for (int sp = 1; sp < kSplit; ++sp) {  // integer partial sums: any order gives the same total
-                uint32_t r2[16];
-                tmem_ld_32x16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * (kSplit * kTok) + sp * kTok, r2);
+                    for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(__fmul_rn((float)((int)r[j] - xs), s_w), dm);
+                    if (y_dtype == BITLINEAR_BF16) {
+                        uint32_t h[8];
 #pragma unroll
-                for (int m = 0; m < kTok; ++m) r[m] += r2[m];
-            }
-            const int n = item.y * kTileRows + quad * 32 + lane;  // this lane's weight row
+                        for (int j = 0; j < 8; ++j) {
+                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
+                            h[j] = *reinterpret_cast<const uint32_t*>(&b2);
+                        }
+                        uint4* dst = reinterpret_cast<uint4*>(y16 + n0);
+                        dst[0] = make_uint4(h[0], h[1], h[2], h[3]);
+                        dst[1] = make_uint4(h[4], h[5], h[6], h[7]);
+                    } else {
+                        float4* dst = reinterpret_cast<float4*>(y32 + n0);
 #pragma unroll
-            for (int m = 0; m < kTok; ++m) {
-                const int xs = __shfl_sync(0xffffffffu, xs_lane, m);
-                const float dm = __shfl_sync(0xffffffffu, d_lane, m);
-                if (m < M && n < N) {
-                    const float val = __fmul_rn(__fmul_rn((float)((int)r[m] - xs), s_w), dm);
-                    const size_t idx = (size_t)m * N + n;
-                    if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
-                    else reinterpret_cast<float*>(y)[idx] = val;
+                        for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+                    }
                 }
             }
             tc_fence_before();
@@ -350,7 +369,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         if (threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
         __syncthreads();
     }
-    if (warp == 9) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
@@ -372,7 +391,7 @@ MmaLayout mma_layout(const bitlinear_problem* problems, int count) {
     for (int i = 0; i < count; ++i) {
         const bitlinear_problem& q = problems[i];
         if (q.M <= 0) continue;
-        items += (size_t)(q.N / kTileRows + 7) / 8;
+        items += (size_t)(q.N / kTileRows + kItemRb - 1) / kItemRb;
         rows += (size_t)q.M;
         x_bytes += (size_t)kTok * q.K;  // K / 128 images of 16 rows x 128 codes
     }
@@ -421,7 +440,7 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ws);
 
-    // ---- host plan: descriptors, work items of 128 weight rows, token -> problem table, balanced CTA ranges ----
+    // ---- host plan: descriptors, work items of 256 weight rows, token -> problem table, balanced CTA ranges ----
     std::vector<MmaProblem> mp;
     std::vector<int2> items;
     std::vector<double> weight;  // packed tiles of each item
@@ -451,9 +470,9 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
             v.eps = q.rms_eps;
             v.row_begin = row;
             const int n_rb = q.N / kTileRows;
-            for (int rb = 0; rb < n_rb; rb += 8) {
+            for (int rb = 0; rb < n_rb; rb += kItemRb) {
                 items.push_back(make_int2((int)mp.size(), rb));
-                weight.push_back((double)std::min(8, n_rb - rb) * (q.K / kTileCols));
+                weight.push_back((double)std::min(kItemRb, n_rb - rb) * (q.K / kTileCols));
             }
             for (int m = 0; m < q.M; ++m) row_prob.push_back((int)mp.size());
             mp.push_back(v);
