@@ -1,18 +1,20 @@
 // Batched decode for 5 to 16 tokens per matmul on the tensor cores.
-// (Paper Section 5.1: packed weights are loaded from HBM into shared memory and unpacked there right before the
-// product with the 8-bit activations.  With more than a few tokens the dot-product-of-four kernel is bound by its
-// arithmetic - one instruction per token per four weights - so here the product runs on tcgen05.  The time of one
-// tcgen05.mma grows with the rows of its A operand and hardly with its N, so the weights are the wide, stationary
-// B operand: D[tokens (16 of M = 64 rows) x 256 weight rows] += A[tokens x 32 activations (s8)] x B[256 x 32 codes (u8)].)
+// (Paper Section 5.1: packed weights are loaded from HBM into shared memory and unpacked right before the product
+// with the 8-bit activations.  With more than a few tokens the dot-product-of-four kernel is bound by its arithmetic
+// - one instruction per token per four weights - so here the product runs on tcgen05:
+// D[128 weight rows x 16 tokens] += A[128 x 32 weight codes (u8)] x B[16 x 32 activations (s8)].
+// The unpacked codes never touch shared memory: each unpack thread owns one weight row, expands its 2-bit codes in
+// registers and stores them with tcgen05.st into tensor memory, from where the MMA takes its A operand; shared
+// memory only carries the packed bytes and the token images, so the copy ring can be deep.)
 //
-// One persistent CTA per SM owns a contiguous, byte-balanced range of work items (256 weight rows of one matmul).
-//   warp 0      epilogue : tcgen05.ld of the finished accumulator (token m in lane m; double buffered), minus the
-//                          code sum, two fp32 multiplies, 16-byte stores
-//   warp 1      producer : bulk copies of packed weights (sixteen 16-row blocks x up to two 16x256 tiles) and of the
-//                          matching slice of the quantised tokens (16-row tile images) into a 2-slot ring
-//   warp 2      MMA      : one thread issues 8 tcgen05.mma (64 x 256 x 32) per 256-column step and commits
-//   warps 3-10  unpack   : warp w expands row blocks 2w and 2w+1 of the current 256-column step: 2-bit codes -> bytes,
-//                          written as two 128-byte-swizzled K-major operand images of 256 rows (2 stages of 64 KiB)
+// One persistent CTA per SM owns a contiguous, byte-balanced range of work items (128 weight rows of one matmul).
+//   warp 0      producer : bulk copies of packed weights (eight 16-row blocks x up to four 16x256 tiles, 4 KiB each)
+//                          and of the matching slice of the quantised tokens (16-row tile images) into a 4-slot ring
+//   warps 1-8   unpack   : two groups of four warps take alternate 256-column steps; the warp of tensor-memory lane
+//                          quarter q expands weight rows 32q .. 32q+31 (thread = row) into 64 columns of a 4-stage ring
+//   warp 9      MMA      : one thread issues 8 tcgen05.mma (128 x 16 x 32, A from tensor memory) per step and commits
+//   warps 10-13 epilogue : tcgen05.ld of the finished 128 x 16 accumulator (double buffered), minus the code sum,
+//                          two fp32 multiplies, stores coalesced along the weight rows
 // Every wait is bounded; on a timeout the CTA raises the sticky status word and leaves.
 #include <algorithm>
 #include <vector>
@@ -24,21 +26,21 @@ namespace bitlinear {
 
 namespace {
 
-constexpr int kItemRb = 16;       // 16-row blocks per work item
-constexpr int kItemRows = kItemRb * kTileRows;  // 256 weight rows = UMMA N
-constexpr int kTok = 16;          // tokens per matmul, padded; the MMA computes 64 rows of which 16 are read
-constexpr int kMmaM = 64;
-constexpr int kStepTiles = 2;     // 16x256 tiles per row block per ring slot (512 columns)
-constexpr int kUnpackWarps = 8;   // two row blocks each
-constexpr int kEpiWarp = 0, kProdWarp = 1, kMmaWarp = 2, kFirstUnpackWarp = 3;
-constexpr int kMmaThreads = (kFirstUnpackWarp + kUnpackWarps) * 32;
-constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;              // 8 KiB: 4 k-blocks of 16 x 128 token images
-constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;   // 32 KiB of packed weights
-constexpr uint32_t kKbImage = kItemRows * 128;                        // 32 KiB: 256 rows x 128 codes
-constexpr uint32_t kStage = 2 * kKbImage;                             // one 256-column step
-constexpr int kStages = 2;
-constexpr uint32_t kTmemCols = 2 * kItemRows;                         // two accumulators of 256 columns
-constexpr size_t kMmaSmem = 1024 + 2 * (size_t)(kXSlot + kPackedSlot) + kStages * (size_t)kStage + 256;
+constexpr int kRows = 128;        // weight rows per work item = tensor-memory lanes = UMMA M
+constexpr int kItemRb = kRows / kTileRows;
+constexpr int kTok = 16;          // tokens per matmul, padded (UMMA N)
+constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1024 columns)
+constexpr int kSlots = 4;         // ring slots of packed weights + token images
+constexpr int kUnpackWarps = 8;   // two groups of four (one warp per tensor-memory lane quarter)
+constexpr int kMmaWarp = 1 + kUnpackWarps;
+constexpr int kMmaThreads = (1 + kUnpackWarps + 1 + 4) * 32;
+constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;  // 32 KiB of packed weights
+constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;             // 16 KiB: 8 k-blocks of 16 x 128 token images
+constexpr int kAStages = 4;                                          // unpacked steps in flight in tensor memory
+constexpr uint32_t kAStageCols = kTileCols / 4;                      // 64 columns: 256 codes per row, 4 per column
+constexpr uint32_t kAColBase = 2 * kTok;                             // after the two accumulators
+constexpr uint32_t kTmemCols = 512;                                  // power of two >= 32 + 4 * 64
+constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + 256;
 
 struct MmaProblem {
     const uint8_t* packed;
@@ -68,7 +70,7 @@ constexpr unsigned kMmaMagic = 0xB171A9E7u;
 struct MmaParams {
     const MmaHeader* hdr;
     const MmaProblem* probs;
-    const int2* items;      // {problem, first row block of the item (a multiple of 16)}
+    const int2* items;      // {problem, first row block of the item (a multiple of 8)}
     const int* cta_begin;   // [grid + 1]
     int count, total_items, rows;
     int* status_word;
@@ -82,18 +84,31 @@ __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence:
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__device__ __forceinline__ void umma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+// A operand in tensor memory (lane = row, four 8-bit codes per 32-bit column), B operand in shared memory.
+__device__ __forceinline__ void umma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// Lane l of the warp writes 32 consecutive columns of tensor-memory lane (taddr lane + l).
+__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]),
+          "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]),
+          "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]),
+          "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// Lane l of the warp receives 16 consecutive columns of tensor-memory lane (taddr lane + l).
 __device__ __forceinline__ void tmem_ld_32x16(uint32_t taddr, uint32_t (&r)[16]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
@@ -114,8 +129,8 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
     desc |= (uint64_t)2 << 61;
     return desc;
 }
-// D = s32, A = s8 (activations), B = u8 (weight codes), both K-major, M = 64, N = 256.
-constexpr uint32_t kIdesc = (2u << 4) | (1u << 7) | (0u << 10) | ((uint32_t)(kItemRows >> 3) << 17) | ((uint32_t)(kMmaM >> 4) << 24);
+// D = s32, A = u8 (weight codes, tensor memory), B = s8 (activations, K-major shared memory), M = 128, N = 16.
+constexpr uint32_t kIdesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
 
 template <int VPT>
 __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeader* __restrict__ hdr,
@@ -139,23 +154,17 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ void sts128(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
 
 __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaParams prm) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    // The token images come first: the MMA reads 64 operand rows where 16 are stored, and what it reads past them
-    // (rows whose results nobody looks at) must still be this CTA's shared memory.
-    const uint32_t x_s = smem_u32(smem);          // [2] token images
-    const uint32_t p_s = x_s + 2 * kXSlot;        // [2] packed weights
-    const uint32_t b_s = p_s + 2 * kPackedSlot;   // [kStages] operand images of the weights
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + 2 * (size_t)(kXSlot + kPackedSlot) + kStages * (size_t)kStage);
-    const uint32_t pfull = smem_u32(bars + 0), pempty = smem_u32(bars + 2), xempty = smem_u32(bars + 4);
-    const uint32_t tfull = smem_u32(bars + 6), tempty = smem_u32(bars + 8);
-    const uint32_t bfull = smem_u32(bars + 10), bempty = smem_u32(bars + 10 + kStages);
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10 + 2 * kStages);
+    const uint32_t x_s = smem_u32(smem);            // [kSlots] token images
+    const uint32_t p_s = x_s + kSlots * kXSlot;     // [kSlots] packed weights
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSlots * (size_t)(kXSlot + kPackedSlot));
+    const uint32_t pfull = smem_u32(bars), pempty = pfull + 8 * kSlots, xempty = pempty + 8 * kSlots;
+    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kAStages;
+    const uint32_t tfull = aempty + 8 * kAStages, tempty = tfull + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kSlots + 2 * kAStages + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -165,16 +174,18 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         return;
     }
     if (threadIdx.x == 0) {
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < kSlots; ++b) {
             mbar_init(pfull + 8 * b, 1);
             mbar_init(pempty + 8 * b, kUnpackWarps);
             mbar_init(xempty + 8 * b, 1);
-            mbar_init(tfull + 8 * b, 1);
-            mbar_init(tempty + 8 * b, 1);
         }
-        for (int b = 0; b < kStages; ++b) {
-            mbar_init(bfull + 8 * b, kUnpackWarps);
-            mbar_init(bempty + 8 * b, 1);
+        for (int b = 0; b < kAStages; ++b) {
+            mbar_init(afull + 8 * b, kUnpackWarps / 2);
+            mbar_init(aempty + 8 * b, 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(tfull + 8 * b, 1);
+            mbar_init(tempty + 8 * b, 4);
         }
         *abort_flag = 0;
         mbar_init_fence();
@@ -190,7 +201,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t tmem_base = *tmem_slot;
     const int item_lo = prm.cta_begin[blockIdx.x], item_hi = prm.cta_begin[blockIdx.x + 1];
 
-    if (warp == kProdWarp) {
+    if (warp == 0) {
         // ------------------------------------------------------------------ producer
         uint32_t sc_idx = 0;
         bool ok = true;
@@ -202,7 +213,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             const uint8_t* x_img = p.x_img;
             for (int t0 = 0; t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                 const int tiles = min(kStepTiles, k_tiles - t0);
-                const uint32_t slot = sc_idx & 1u, phase = (sc_idx >> 1) & 1u;
+                const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
                 if (!mbar_wait(pempty + 8 * slot, phase ^ 1u, abort_flag) || !mbar_wait(xempty + 8 * slot, phase ^ 1u, abort_flag)) {
                     ok = false;
                     break;
@@ -218,60 +229,58 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                               pfull + 8 * slot);
             }
         }
-    } else if (warp >= kFirstUnpackWarp) {
-        // ------------------------------------------------------------------ unpack: warp w expands row blocks 2w, 2w+1
-        const int w = warp - kFirstUnpackWarp;
-        const int g = lane >> 2, t = lane & 3;
-        // lanes of the upper k-block take their words in the order 2, 3, 0, 1: the eight lanes that store together
-        // then hit eight different 16-byte bank groups
-        const bool up = (t & 2) != 0;
+    } else if (warp <= kUnpackWarps) {
+        // ------------------------------------------------------------------ unpack: one thread per weight row
+        const int quarter = warp & 3;          // tensor-memory lanes 32*quarter .. +31 are the ones this warp may touch
+        const int group = (warp - 1) >> 2;     // takes the steps of this parity
+        const int rbl = 2 * quarter + (lane >> 4), r16 = lane & 15;  // row block of the item, row inside it
+        // the 256 codes of row r16 = 8h + g of a 16 x 256 tile are 64 consecutive packed bytes at 512h + 64g
+        const uint32_t row_off = (uint32_t)rbl * (kStepTiles * kTileBytes) + (uint32_t)(r16 >> 3) * 512u + (uint32_t)(r16 & 7) * 64u;
+        const uint32_t a_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + kAColBase;
         uint32_t sc_idx = 0, st_idx = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
             const int2 item = prm.items[it];
             const MmaProblem& p = prm.probs[item.x];
             const int k_tiles = p.K / kTileCols, n_rb = min(kItemRb, p.N / kTileRows - item.y);
+            const bool have_row = rbl < n_rb;
             for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                 const int tiles = min(kStepTiles, k_tiles - t0);
-                const uint32_t slot = sc_idx & 1u, phase = (sc_idx >> 1) & 1u;
+                const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
+                // every warp waits for every slot, also one in which it has no step: a warp can then never be a whole
+                // ring lap ahead of another and arrive twice on pempty in one phase
                 if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
                 for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                    const uint32_t stage = st_idx % kStages, sphase = (st_idx / kStages) & 1u;
-                    uint4 pv[2][2] = {};
+                    if ((int)(st_idx & 1u) != group) continue;
+                    const uint32_t stage = st_idx % kAStages, sphase = (st_idx / kAStages) & 1u;
+                    uint4 pw[4] = {};
+                    if (have_row) {
+                        const uint32_t src = p_s + slot * kPackedSlot + row_off + (uint32_t)kt * kTileBytes;
 #pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        if (2 * w + r < n_rb) {
-                            const uint32_t src = p_s + slot * kPackedSlot + (uint32_t)(2 * w + r) * (kStepTiles * kTileBytes) +
-                                                 (uint32_t)kt * kTileBytes + (uint32_t)lane * 16u;
-                            pv[r][0] = lds128(src);
-                            pv[r][1] = lds128(src + 512u);
-                        }
+                        for (int t = 0; t < 4; ++t) pw[t] = lds128(src + 16u * t);
                     }
-                    if (!mbar_wait(bempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    // word i of piece t, bit plane j, byte b = column 64t + 16i + 4j + b: tensor-memory column 16t + 4i + j
 #pragma unroll
-                    for (int r = 0; r < 2; ++r) {
-                        if (2 * w + r < n_rb) {
-                            // lane (g, t) holds rows g and 8+g of the 16-row block, columns 64t .. 64t+63 of the 256:
-                            // k-block t >> 1, 16-byte pieces 4*(t & 1) + q of the 128-byte operand row
-                            const uint32_t dst = b_s + stage * kStage + (uint32_t)(t >> 1) * kKbImage +
-                                                 (uint32_t)((2 * w + r) * kTileRows + g) * 128u;
+                    for (int half = 0; half < 2; ++half) {
+                        uint32_t v[32];
 #pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                const uint4 v4 = pv[r][h];
-                                const uint32_t pw[4] = {up ? v4.z : v4.x, up ? v4.w : v4.y, up ? v4.x : v4.z, up ? v4.y : v4.w};
+                        for (int tt = 0; tt < 2; ++tt) {
+                            const uint4 q4 = pw[2 * half + tt];
+                            const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
 #pragma unroll
-                                for (int q = 0; q < 4; ++q) {
-                                    const uint32_t v = pw[q];
-                                    const uint32_t piece = (uint32_t)(4 * (t & 1) + (q ^ (t & 2))) ^ (uint32_t)g;  // row & 7 == g
-                                    sts128(dst + 1024u * h + (piece << 4), v & 0x03030303u, (v >> 2) & 0x03030303u,
-                                           (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
-                                }
+                            for (int i = 0; i < 4; ++i) {
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) v[16 * tt + 4 * i + j] = (w4[i] >> (2 * j)) & 0x03030303u;
                             }
                         }
+                        tmem_st_32x32(a_lane + stage * kAStageCols + 32u * half, v);
                     }
-                    fence_async_smem();  // the tensor core reads these bytes through the async proxy
+                    tmem_st_wait();
+                    tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(bfull + 8 * stage);
+                    if (lane == 0) mbar_arrive(afull + 8 * stage);
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pempty + 8 * slot);
@@ -288,25 +297,24 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
                 if (!mbar_wait(tempty + 8 * buf, bphase ^ 1u, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * kItemRows;
+                const uint32_t d_tmem = tmem_base + buf * kTok;
                 for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                     const int tiles = min(kStepTiles, k_tiles - t0);
-                    const uint32_t slot = sc_idx & 1u, phase = (sc_idx >> 1) & 1u;
+                    const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
                     if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }  // the token images landed
+                    const uint64_t x_desc = smem_desc_sw128(x_s + slot * kXSlot);
                     for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                        const uint32_t stage = st_idx % kStages, sphase = (st_idx / kStages) & 1u;
-                        if (!mbar_wait(bfull + 8 * stage, sphase, abort_flag)) { ok = false; break; }
+                        const uint32_t stage = st_idx % kAStages, sphase = (st_idx / kAStages) & 1u;
+                        if (!mbar_wait(afull + 8 * stage, sphase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
+                        const uint32_t a_tmem = tmem_base + kAColBase + stage * kAStageCols;
+                        // k-block kb of the step: token image kt*2 + kb (2 KiB each); 32-byte slice k inside it
+                        const uint64_t b_desc = x_desc + (uint64_t)((kt * 2 * kTok * 128) >> 4);
 #pragma unroll
-                        for (int kb = 0; kb < 2; ++kb) {
-                            const uint64_t a_desc = smem_desc_sw128(x_s + slot * kXSlot + (uint32_t)(kt * 2 + kb) * (kTok * 128));
-                            const uint64_t b_desc = smem_desc_sw128(b_s + stage * kStage + (uint32_t)kb * kKbImage);
-#pragma unroll
-                            for (int k = 0; k < 4; ++k)
-                                umma_i8(d_tmem, a_desc + (uint64_t)(2 * k), b_desc + (uint64_t)(2 * k), kIdesc,
-                                        (uint32_t)((t0 | kt | kb | k) != 0));
-                        }
-                        umma_commit(bempty + 8 * stage);  // the stage may be rewritten once these MMAs retire
+                        for (int s = 0; s < 8; ++s)
+                            umma_i8_ts(d_tmem, a_tmem + 8u * s, b_desc + (uint64_t)((s >> 2) * ((kTok * 128) >> 4) + 2 * (s & 3)),
+                                       kIdesc, (uint32_t)((t0 | kt | s) != 0));
+                        umma_commit(aempty + 8 * stage);  // the stage may be rewritten once these MMAs retire
                     }
                     if (ok) umma_commit(xempty + 8 * slot);
                 }
@@ -315,45 +323,32 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         }
         __syncwarp();
     } else {
-        // ------------------------------------------------------------------ epilogue (warp 0: tensor-memory lanes 0 .. 31)
+        // ------------------------------------------------------------------ epilogue
+        const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
         uint32_t it_idx = 0;
         for (int it = item_lo; it < item_hi; ++it, ++it_idx) {
             const int2 item = prm.items[it];
             const MmaProblem& p = prm.probs[item.x];
             const int M = p.M, N = p.N, y_dtype = p.y_dtype;
+            void* y = p.y;
             const float s_w = *p.s_w;
-            const bool live = lane < M;  // accumulator row m of the 64 sits in tensor-memory lane m for m < 16
-            const int xs = live ? p.xsum[lane] : 0;
-            const float dm = live ? p.d[lane] : 0.0f;
-            float* y32 = reinterpret_cast<float*>(p.y) + (size_t)lane * N;
-            __nv_bfloat16* y16 = reinterpret_cast<__nv_bfloat16*>(p.y) + (size_t)lane * N;
+            const int xs_lane = lane < M ? p.xsum[lane] : 0;
+            const float d_lane = lane < M ? p.d[lane] : 0.0f;
             const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
             if (!mbar_wait(tfull + 8 * buf, bphase, abort_flag)) break;
             tc_fence_after();
-            for (int c = 0; c < kItemRb; ++c) {
-                const int n0 = (item.y + c) * kTileRows;  // first weight row of these 16 columns
-                if (n0 >= N) break;
-                uint32_t r[16];
-                tmem_ld_32x16(tmem_base + buf * kItemRows + (uint32_t)c * kTileRows, r);
-                if (live) {
-                    float v[16];
+            uint32_t r[16];
+            tmem_ld_32x16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kTok, r);
+            const int n = item.y * kTileRows + quad * 32 + lane;  // this lane's weight row
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) v[j] = __fmul_rn(__fmul_rn((float)((int)r[j] - xs), s_w), dm);
-                    if (y_dtype == BITLINEAR_BF16) {
-                        uint32_t h[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * j], v[2 * j + 1]);
-                            h[j] = *reinterpret_cast<const uint32_t*>(&b2);
-                        }
-                        uint4* dst = reinterpret_cast<uint4*>(y16 + n0);
-                        dst[0] = make_uint4(h[0], h[1], h[2], h[3]);
-                        dst[1] = make_uint4(h[4], h[5], h[6], h[7]);
-                    } else {
-                        float4* dst = reinterpret_cast<float4*>(y32 + n0);
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                    }
+            for (int m = 0; m < kTok; ++m) {
+                const int xs = __shfl_sync(0xffffffffu, xs_lane, m);
+                const float dm = __shfl_sync(0xffffffffu, d_lane, m);
+                if (m < M && n < N) {
+                    const float val = __fmul_rn(__fmul_rn((float)((int)r[m] - xs), s_w), dm);
+                    const size_t idx = (size_t)m * N + n;
+                    if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
+                    else reinterpret_cast<float*>(y)[idx] = val;
                 }
             }
             tc_fence_before();
@@ -440,7 +435,7 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ws);
 
-    // ---- host plan: descriptors, work items of 256 weight rows, token -> problem table, balanced CTA ranges ----
+    // ---- host plan: descriptors, work items of 128 weight rows, token -> problem table, balanced CTA ranges ----
     std::vector<MmaProblem> mp;
     std::vector<int2> items;
     std::vector<double> weight;  // packed tiles of each item
