@@ -10,11 +10,15 @@
 // One persistent CTA per SM owns a contiguous, byte-balanced range of work items (128 weight rows of one matmul).
 //   warp 0      producer : bulk copies of packed weights (eight 16-row blocks x up to four 16x256 tiles, 4 KiB each)
 //                          and of the matching slice of the quantised tokens (16-row tile images) into a 4-slot ring
-//   warps 1-8   unpack   : two groups of four warps take alternate 256-column steps; the warp of tensor-memory lane
-//                          quarter q expands weight rows 32q .. 32q+31 (thread = row) into 64 columns of a 4-stage ring
-//   warp 9      MMA      : one thread issues 8 tcgen05.mma (128 x 16 x 32, A from tensor memory) per step and commits
-//   warps 10-13 epilogue : tcgen05.ld of the finished 128 x 16 accumulator (double buffered), minus the code sum,
-//                          two fp32 multiplies, stores coalesced along the weight rows
+// The 256-column steps of a CTA's work are dealt round-robin to kLanes pipelines, each with its own unpack group, its
+// own 64 tensor-memory columns for the codes, its own MMA-issuing thread and its own partial accumulator (one thread
+// can start a tcgen05.mma only every ~55 cycles whatever its shape, several threads scale; the integer partial sums
+// are added in the epilogue, exactly):
+//   unpack groups  : four warps each, the warp of tensor-memory lane quarter q expands weight rows 32q .. 32q+31
+//                    (thread = row) into the pipeline's 64 columns
+//   MMA warps      : one thread each issues the 8 tcgen05.mma (128 x 16 x 32, A from tensor memory) of a step
+//   epilogue warps : tcgen05.ld of the finished partial accumulators (double buffered), their sum minus the code
+//                    sum, two fp32 multiplies, stores coalesced along the weight rows
 // Every wait is bounded; on a timeout the CTA raises the sticky status word and leaves.
 #include <algorithm>
 #include <vector>
@@ -31,15 +35,17 @@ constexpr int kItemRb = kRows / kTileRows;
 constexpr int kTok = 16;          // tokens per matmul, padded (UMMA N)
 constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1024 columns)
 constexpr int kSlots = 4;         // ring slots of packed weights + token images
-constexpr int kUnpackWarps = 8;   // two groups of four (one warp per tensor-memory lane quarter)
-constexpr int kMmaWarp = 1 + kUnpackWarps;
-constexpr int kMmaThreads = (1 + kUnpackWarps + 1 + 4) * 32;
+constexpr int kLanes = 4;         // pipelines: unpack group + tensor-memory stage + MMA issuer + partial accumulator
+constexpr int kUnpackWarps = 4 * kLanes;  // groups of four (one warp per tensor-memory lane quarter)
+constexpr int kFirstMmaWarp = 1 + kUnpackWarps;
+constexpr int kFirstEpiWarp = kFirstMmaWarp + kLanes;
+constexpr int kMmaThreads = (kFirstEpiWarp + 4) * 32;
 constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;  // 32 KiB of packed weights
 constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;             // 16 KiB: 8 k-blocks of 16 x 128 token images
-constexpr int kAStages = 4;                                          // unpacked steps in flight in tensor memory
 constexpr uint32_t kAStageCols = kTileCols / 4;                      // 64 columns: 256 codes per row, 4 per column
-constexpr uint32_t kAColBase = 2 * kTok;                             // after the two accumulators
-constexpr uint32_t kTmemCols = 512;                                  // power of two >= 32 + 4 * 64
+constexpr uint32_t kAColBase = 2 * kLanes * kTok;                    // after the two buffers of partial accumulators
+constexpr uint32_t kTmemCols = 512;                                  // power of two >= kAColBase + kLanes * 64
+static_assert(kAColBase + kLanes * kAStageCols <= kTmemCols, "tensor memory");
 constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + 256;
 
 struct MmaProblem {
@@ -162,9 +168,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t p_s = x_s + kSlots * kXSlot;     // [kSlots] packed weights
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSlots * (size_t)(kXSlot + kPackedSlot));
     const uint32_t pfull = smem_u32(bars), pempty = pfull + 8 * kSlots, xempty = pempty + 8 * kSlots;
-    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kAStages;
-    const uint32_t tfull = aempty + 8 * kAStages, tempty = tfull + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kSlots + 2 * kAStages + 4);
+    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kLanes;
+    const uint32_t tfull = aempty + 8 * kLanes, tempty = tfull + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kSlots + 2 * kLanes + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -177,20 +183,20 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         for (int b = 0; b < kSlots; ++b) {
             mbar_init(pfull + 8 * b, 1);
             mbar_init(pempty + 8 * b, kUnpackWarps);
-            mbar_init(xempty + 8 * b, 1);
+            mbar_init(xempty + 8 * b, kLanes);
         }
-        for (int b = 0; b < kAStages; ++b) {
-            mbar_init(afull + 8 * b, kUnpackWarps / 2);
+        for (int b = 0; b < kLanes; ++b) {
+            mbar_init(afull + 8 * b, 4);
             mbar_init(aempty + 8 * b, 1);
         }
         for (int b = 0; b < 2; ++b) {
-            mbar_init(tfull + 8 * b, 1);
+            mbar_init(tfull + 8 * b, kLanes);
             mbar_init(tempty + 8 * b, 4);
         }
         *abort_flag = 0;
         mbar_init_fence();
     }
-    if (warp == kMmaWarp) {
+    if (warp == kFirstMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -232,7 +238,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     } else if (warp <= kUnpackWarps) {
         // ------------------------------------------------------------------ unpack: one thread per weight row
         const int quarter = warp & 3;          // tensor-memory lanes 32*quarter .. +31 are the ones this warp may touch
-        const int group = (warp - 1) >> 2;     // takes the steps of this parity
+        const int group = (warp - 1) >> 2;     // this warp's pipeline: steps with st_idx % kLanes == group
         const int rbl = 2 * quarter + (lane >> 4), r16 = lane & 15;  // row block of the item, row inside it
         // the 256 codes of row r16 = 8h + g of a 16 x 256 tile are 64 consecutive packed bytes at 512h + 64g
         const uint32_t row_off = (uint32_t)rbl * (kStepTiles * kTileBytes) + (uint32_t)(r16 >> 3) * 512u + (uint32_t)(r16 & 7) * 64u;
@@ -251,8 +257,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 // ring lap ahead of another and arrive twice on pempty in one phase
                 if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
                 for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                    if ((int)(st_idx & 1u) != group) continue;
-                    const uint32_t stage = st_idx % kAStages, sphase = (st_idx / kAStages) & 1u;
+                    if ((int)(st_idx % kLanes) != group) continue;
+                    const uint32_t stage = (uint32_t)group, sphase = (st_idx / kLanes) & 1u;
                     uint4 pw[4] = {};
                     if (have_row) {
                         const uint32_t src = p_s + slot * kPackedSlot + row_off + (uint32_t)kt * kTileBytes;
@@ -286,9 +292,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 if (lane == 0) mbar_arrive(pempty + 8 * slot);
             }
         }
-    } else if (warp == kMmaWarp) {
-        // ------------------------------------------------------------------ MMA issuer
+    } else if (warp < kFirstEpiWarp) {
+        // ------------------------------------------------------------------ MMA issuers: one pipeline each
         if (lane == 0) {
+            const int me = warp - kFirstMmaWarp;
+            const uint32_t a_tmem = tmem_base + kAColBase + (uint32_t)me * kAStageCols;
             uint32_t sc_idx = 0, st_idx = 0, it_idx = 0;
             bool ok = true;
             for (int it = item_lo; ok && it < item_hi; ++it, ++it_idx) {
@@ -297,26 +305,29 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
                 if (!mbar_wait(tempty + 8 * buf, bphase ^ 1u, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + buf * kTok;
+                const uint32_t d_tmem = tmem_base + (buf * kLanes + (uint32_t)me) * kTok;
+                const uint32_t st_item = st_idx;  // this pipeline's first step of the item starts its partial sum
                 for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                     const int tiles = min(kStepTiles, k_tiles - t0);
                     const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
-                    if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }  // the token images landed
+                    // every issuer waits for every slot, also one in which it has no step (see the unpack warps)
+                    if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
                     const uint64_t x_desc = smem_desc_sw128(x_s + slot * kXSlot);
                     for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                        const uint32_t stage = st_idx % kAStages, sphase = (st_idx / kAStages) & 1u;
-                        if (!mbar_wait(afull + 8 * stage, sphase, abort_flag)) { ok = false; break; }
+                        if ((int)(st_idx % kLanes) != me) continue;
+                        const uint32_t sphase = (st_idx / kLanes) & 1u;
+                        if (!mbar_wait(afull + 8 * me, sphase, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        const uint32_t a_tmem = tmem_base + kAColBase + stage * kAStageCols;
                         // k-block kb of the step: token image kt*2 + kb (2 KiB each); 32-byte slice k inside it
                         const uint64_t b_desc = x_desc + (uint64_t)((kt * 2 * kTok * 128) >> 4);
+                        const bool first = st_idx - st_item < (uint32_t)kLanes;
 #pragma unroll
                         for (int s = 0; s < 8; ++s)
                             umma_i8_ts(d_tmem, a_tmem + 8u * s, b_desc + (uint64_t)((s >> 2) * ((kTok * 128) >> 4) + 2 * (s & 3)),
-                                       kIdesc, (uint32_t)((t0 | kt | s) != 0));
-                        umma_commit(aempty + 8 * stage);  // the stage may be rewritten once these MMAs retire
+                                       kIdesc, (uint32_t)(!first || s != 0));
+                        umma_commit(aempty + 8 * me);  // the codes may be overwritten once these MMAs retire
                     }
-                    if (ok) umma_commit(xempty + 8 * slot);
+                    if (ok) umma_commit(xempty + 8 * slot);  // counts kLanes arrivals: every issuer is done with the slot
                 }
                 if (ok) umma_commit(tfull + 8 * buf);
             }
@@ -325,25 +336,35 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     } else {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
-        uint32_t it_idx = 0;
+        uint32_t it_idx = 0, st_idx = 0;
         for (int it = item_lo; it < item_hi; ++it, ++it_idx) {
             const int2 item = prm.items[it];
             const MmaProblem& p = prm.probs[item.x];
             const int M = p.M, N = p.N, y_dtype = p.y_dtype;
+            const int k_tiles = p.K / kTileCols;
             void* y = p.y;
             const float s_w = *p.s_w;
             const int xs_lane = lane < M ? p.xsum[lane] : 0;
-            const float d_lane = lane < M ? p.d[lane] : 0.0f;
+            const float d_tok = lane < M ? p.d[lane] : 0.0f;
             const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
             if (!mbar_wait(tfull + 8 * buf, bphase, abort_flag)) break;
             tc_fence_after();
+            // the pipelines that had a step in this item hold its partial sums (integers: any order, same total)
+            const uint32_t d_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kLanes * kTok;
             uint32_t r[16];
-            tmem_ld_32x16(tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kTok, r);
+            tmem_ld_32x16(d_lane + (st_idx % kLanes) * kTok, r);
+            for (int j = 1; j < min(kLanes, k_tiles); ++j) {
+                uint32_t r2[16];
+                tmem_ld_32x16(d_lane + ((st_idx + j) % kLanes) * kTok, r2);
+#pragma unroll
+                for (int m = 0; m < kTok; ++m) r[m] += r2[m];
+            }
+            st_idx += (uint32_t)k_tiles;
             const int n = item.y * kTileRows + quad * 32 + lane;  // this lane's weight row
 #pragma unroll
             for (int m = 0; m < kTok; ++m) {
                 const int xs = __shfl_sync(0xffffffffu, xs_lane, m);
-                const float dm = __shfl_sync(0xffffffffu, d_lane, m);
+                const float dm = __shfl_sync(0xffffffffu, d_tok, m);
                 if (m < M && n < N) {
                     const float val = __fmul_rn(__fmul_rn((float)((int)r[m] - xs), s_w), dm);
                     const size_t idx = (size_t)m * N + n;
@@ -364,7 +385,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         if (threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
         __syncthreads();
     }
-    if (warp == kMmaWarp) {
+    if (warp == kFirstMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
     }
