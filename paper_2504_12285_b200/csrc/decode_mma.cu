@@ -46,7 +46,8 @@ constexpr uint32_t kAStageCols = kTileCols / 4;                      // 64 colum
 constexpr uint32_t kAColBase = 2 * kLanes * kTok;                    // after the two buffers of partial accumulators
 constexpr uint32_t kTmemCols = 512;                                  // power of two >= kAColBase + kLanes * 64
 static_assert(kAColBase + kLanes * kAStageCols <= kTmemCols, "tensor memory");
-constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + 256;
+constexpr int kItemCap = 192;     // work items and matmul descriptors of the CTA kept in shared memory; what does
+constexpr int kProbCap = 48;      // not fit is read from global memory where it is needed (slow, still correct)
 
 struct MmaProblem {
     const uint8_t* packed;
@@ -81,6 +82,26 @@ struct MmaParams {
     int count, total_items, rows;
     int* status_word;
 };
+
+// What the kernel's roles need of a matmul, copied to shared memory once: a descriptor fetched from global memory
+// at every item boundary costs two dependent loads at loaded-HBM latency in every role, and the pipeline drains.
+struct alignas(16) SProb {
+    const uint8_t* packed;
+    const uint8_t* x_img;
+    const float* s_w;
+    const float* d;
+    const int32_t* xsum;
+    void* y;
+    int M, N, K, y_dtype;
+};
+constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + 256 + kItemCap * sizeof(int2) + kProbCap * sizeof(SProb);
+
+__device__ __forceinline__ SProb load_prob(const MmaProblem& q) {
+    SProb v;
+    v.packed = q.packed; v.x_img = q.x_img; v.s_w = q.s_w; v.d = q.d; v.xsum = q.xsum; v.y = q.y;
+    v.M = q.M; v.N = q.N; v.K = q.K; v.y_dtype = q.y_dtype;
+    return v;
+}
 
 __device__ __forceinline__ bool mma_plan_matches(const MmaHeader* h, int count, int total_items, int grid, int rows) {
     return h->magic == kMmaMagic && h->count == count && h->total_items == total_items && h->grid == grid && h->rows == rows;
@@ -135,7 +156,7 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
     desc |= (uint64_t)2 << 61;
     return desc;
 }
-// D = s32, A = u8 (weight codes, tensor memory), B = s8 (activations, K-major shared memory), M = 128, N = 16.
+// D = s32, A = u8 (64 x weight code, tensor memory), B = s8 (activations, K-major shared memory), M = 128, N = 16.
 constexpr uint32_t kIdesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
 
 template <int VPT>
@@ -172,6 +193,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t tfull = aempty + 8 * kLanes, tempty = tfull + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kSlots + 2 * kLanes + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    int2* items_s = reinterpret_cast<int2*>(reinterpret_cast<uint8_t*>(bars) + 256);
+    SProb* probs_s = reinterpret_cast<SProb*>(items_s + kItemCap);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (!mma_plan_matches(prm.hdr, prm.count, prm.total_items, (int)gridDim.x, prm.rows)) {  // uniform over the grid
@@ -201,19 +224,25 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    const int item_lo = prm.cta_begin[blockIdx.x], item_hi = prm.cta_begin[blockIdx.x + 1];
+    const int prob_lo = item_lo < item_hi ? prm.items[item_lo].x : 0;  // items are sorted by matmul
+    for (int i = threadIdx.x; i < min(item_hi - item_lo, kItemCap); i += kMmaThreads) items_s[i] = prm.items[item_lo + i];
+    for (int i = threadIdx.x; i < min(prm.count - prob_lo, kProbCap); i += kMmaThreads) probs_s[i] = load_prob(prm.probs[prob_lo + i]);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const int item_lo = prm.cta_begin[blockIdx.x], item_hi = prm.cta_begin[blockIdx.x + 1];
+    // item it of this CTA and its matmul, from shared memory when cached
+    auto item_at = [&](int it) -> int2 { return it - item_lo < kItemCap ? items_s[it - item_lo] : prm.items[it]; };
+    auto prob_at = [&](int pi) -> SProb { return pi - prob_lo < kProbCap ? probs_s[pi - prob_lo] : load_prob(prm.probs[pi]); };
 
     if (warp == 0) {
         // ------------------------------------------------------------------ producer
         uint32_t sc_idx = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
-            const int2 item = prm.items[it];
-            const MmaProblem& p = prm.probs[item.x];
+            const int2 item = item_at(it);
+            const SProb p = prob_at(item.x);
             const int k_tiles = p.K / kTileCols, n_rb = min(kItemRb, p.N / kTileRows - item.y);
             const uint8_t* packed = p.packed;
             const uint8_t* x_img = p.x_img;
@@ -246,8 +275,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         uint32_t sc_idx = 0, st_idx = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
-            const int2 item = prm.items[it];
-            const MmaProblem& p = prm.probs[item.x];
+            const int2 item = item_at(it);
+            const SProb p = prob_at(item.x);
             const int k_tiles = p.K / kTileCols, n_rb = min(kItemRb, p.N / kTileRows - item.y);
             const bool have_row = rbl < n_rb;
             for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
@@ -267,7 +296,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     }
                     if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    // word i of piece t, bit plane j, byte b = column 64t + 16i + 4j + b: tensor-memory column 16t + 4i + j
+                    // word i of piece t, bit plane j, byte b = column 64t + 16i + 4j + b: tensor-memory column 16t + 4i + j.
+                    // The 2-bit codes are moved to the TOP of their bytes (value 64 * code, still an unsigned byte):
+                    // that takes a left shift, which the multiplier pipe executes, and one AND, where a right shift
+                    // and an AND would both go to the logic pipe that bounds this loop; the epilogue divides by 64.
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         uint32_t v[32];
@@ -278,7 +310,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
 #pragma unroll
                             for (int i = 0; i < 4; ++i) {
 #pragma unroll
-                                for (int j = 0; j < 4; ++j) v[16 * tt + 4 * i + j] = (w4[i] >> (2 * j)) & 0x03030303u;
+                                for (int j = 0; j < 4; ++j) v[16 * tt + 4 * i + j] = (w4[i] * (64u >> (2 * j))) & 0xC0C0C0C0u;
                             }
                         }
                         tmem_st_32x32(a_lane + stage * kAStageCols + 32u * half, v);
@@ -300,8 +332,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             uint32_t sc_idx = 0, st_idx = 0, it_idx = 0;
             bool ok = true;
             for (int it = item_lo; ok && it < item_hi; ++it, ++it_idx) {
-                const int2 item = prm.items[it];
-                const int k_tiles = prm.probs[item.x].K / kTileCols;
+                const int2 item = item_at(it);
+                const int k_tiles = prob_at(item.x).K / kTileCols;
                 const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
                 if (!mbar_wait(tempty + 8 * buf, bphase ^ 1u, abort_flag)) break;
                 tc_fence_after();
@@ -338,8 +370,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
         uint32_t it_idx = 0, st_idx = 0;
         for (int it = item_lo; it < item_hi; ++it, ++it_idx) {
-            const int2 item = prm.items[it];
-            const MmaProblem& p = prm.probs[item.x];
+            const int2 item = item_at(it);
+            const SProb p = prob_at(item.x);
             const int M = p.M, N = p.N, y_dtype = p.y_dtype;
             const int k_tiles = p.K / kTileCols;
             void* y = p.y;
@@ -359,6 +391,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
 #pragma unroll
                 for (int m = 0; m < kTok; ++m) r[m] += r2[m];
             }
+#pragma unroll
+            for (int m = 0; m < kTok; ++m) r[m] = (uint32_t)((int)r[m] >> 6);  // exact: the sums are multiples of 64
             st_idx += (uint32_t)k_tiles;
             const int n = item.y * kTileRows + quad * 32 + lane;  // this lane's weight row
 #pragma unroll
