@@ -37,7 +37,8 @@ constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1
 constexpr int kSlots = 4;         // ring slots of packed weights + token images
 constexpr int kLanes = 4;         // pipelines: unpack group + tensor-memory stage + MMA issuer + partial accumulator
 constexpr int kUnpackWarps = 4 * kLanes;  // groups of four (one warp per tensor-memory lane quarter)
-constexpr int kFirstMmaWarp = 1 + kUnpackWarps;
+constexpr int kProdWarps = 3, kCopiesPerWarp = 3;  // 8 packed row blocks + the token images
+constexpr int kFirstMmaWarp = kProdWarps + kUnpackWarps;
 constexpr int kFirstEpiWarp = kFirstMmaWarp + kLanes;
 constexpr int kMmaThreads = (kFirstEpiWarp + 4) * 32;
 constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;  // 32 KiB of packed weights
@@ -204,7 +205,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     }
     if (threadIdx.x == 0) {
         for (int b = 0; b < kSlots; ++b) {
-            mbar_init(pfull + 8 * b, 1);
+            mbar_init(pfull + 8 * b, kProdWarps);
             mbar_init(pempty + 8 * b, kUnpackWarps);
             mbar_init(xempty + 8 * b, kLanes);
         }
@@ -236,16 +237,17 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     auto item_at = [&](int it) -> int2 { return it - item_lo < kItemCap ? items_s[it - item_lo] : prm.items[it]; };
     auto prob_at = [&](int pi) -> SProb { return pi - prob_lo < kProbCap ? probs_s[pi - prob_lo] : load_prob(prm.probs[pi]); };
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ producer
+    if (warp < kProdWarps) {
+        // ------------------------------------------------------------------ producers: three copies per warp
+        // (a thread starts a bulk copy only every ~200 cycles, and the lanes of a warp take turns)
+        const int c = warp * kCopiesPerWarp + lane;  // copy 0 .. 7: packed row block c of the item; copy 8: token images
         uint32_t sc_idx = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
             const int2 item = item_at(it);
             const SProb p = prob_at(item.x);
             const int k_tiles = p.K / kTileCols, n_rb = min(kItemRb, p.N / kTileRows - item.y);
-            const uint8_t* packed = p.packed;
-            const uint8_t* x_img = p.x_img;
+            const uint8_t* src_row = p.packed + (size_t)(item.y + c) * k_tiles * kTileBytes;
             for (int t0 = 0; t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                 const int tiles = min(kStepTiles, k_tiles - t0);
                 const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
@@ -253,53 +255,57 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     ok = false;
                     break;
                 }
-                if (lane == 0) mbar_expect_tx(pfull + 8 * slot, (uint32_t)(n_rb * tiles * kTileBytes + tiles * 2 * kTok * 128));
+                if (lane == 0) {  // this warp's share of the slot's bytes
+                    const int c0 = warp * kCopiesPerWarp;
+                    const int n_packed = max(0, min(n_rb, c0 + kCopiesPerWarp) - c0);
+                    const int has_x = (c0 <= kItemRb && kItemRb < c0 + kCopiesPerWarp) ? 1 : 0;
+                    mbar_expect_tx(pfull + 8 * slot, (uint32_t)(n_packed * tiles * kTileBytes + has_x * tiles * 2 * kTok * 128));
+                }
                 __syncwarp();
-                if (lane < n_rb)
-                    bulk_load(p_s + slot * kPackedSlot + lane * (kStepTiles * kTileBytes),
-                              packed + ((size_t)(item.y + lane) * k_tiles + t0) * kTileBytes, (uint32_t)tiles * kTileBytes,
-                              pfull + 8 * slot);
-                else if (lane == kItemRb)
-                    bulk_load(x_s + slot * kXSlot, x_img + (size_t)t0 * 2 * kTok * 128, (uint32_t)tiles * 2 * kTok * 128,
-                              pfull + 8 * slot);
+                if (lane < kCopiesPerWarp) {
+                    if (c < n_rb)
+                        bulk_load(p_s + slot * kPackedSlot + c * (kStepTiles * kTileBytes), src_row + (size_t)t0 * kTileBytes,
+                                  (uint32_t)tiles * kTileBytes, pfull + 8 * slot);
+                    else if (c == kItemRb)
+                        bulk_load(x_s + slot * kXSlot, p.x_img + (size_t)t0 * 2 * kTok * 128, (uint32_t)tiles * 2 * kTok * 128,
+                                  pfull + 8 * slot);
+                }
             }
         }
-    } else if (warp <= kUnpackWarps) {
+    } else if (warp < kFirstMmaWarp) {
         // ------------------------------------------------------------------ unpack: one thread per weight row
-        const int quarter = warp & 3;          // tensor-memory lanes 32*quarter .. +31 are the ones this warp may touch
-        const int group = (warp - 1) >> 2;     // this warp's pipeline: steps with st_idx % kLanes == group
+        const int quarter = warp & 3;                   // tensor-memory lanes 32*quarter .. +31 are the ones this warp may touch
+        const int g = (warp - kProdWarps) >> 2;         // this warp's pipeline: tile g of every slot
         const int rbl = 2 * quarter + (lane >> 4), r16 = lane & 15;  // row block of the item, row inside it
         // the 256 codes of row r16 = 8h + g of a 16 x 256 tile are 64 consecutive packed bytes at 512h + 64g
-        const uint32_t row_off = (uint32_t)rbl * (kStepTiles * kTileBytes) + (uint32_t)(r16 >> 3) * 512u + (uint32_t)(r16 & 7) * 64u;
-        const uint32_t a_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + kAColBase;
-        uint32_t sc_idx = 0, st_idx = 0;
+        const uint32_t row_off = (uint32_t)rbl * (kStepTiles * kTileBytes) + (uint32_t)(r16 >> 3) * 512u + (uint32_t)(r16 & 7) * 64u +
+                                 (uint32_t)g * kTileBytes;
+        const uint32_t a_dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + kAColBase + (uint32_t)g * kAStageCols;
+        uint32_t sc_idx = 0, n_own = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
             const int2 item = item_at(it);
             const SProb p = prob_at(item.x);
-            const int k_tiles = p.K / kTileCols, n_rb = min(kItemRb, p.N / kTileRows - item.y);
-            const bool have_row = rbl < n_rb;
-            for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
-                const int tiles = min(kStepTiles, k_tiles - t0);
+            const int k_tiles = p.K / kTileCols;
+            const bool have_row = rbl < min(kItemRb, p.N / kTileRows - item.y);
+            for (int t0 = 0; t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                 const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
                 // every warp waits for every slot, also one in which it has no step: a warp can then never be a whole
                 // ring lap ahead of another and arrive twice on pempty in one phase
                 if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
-                for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                    if ((int)(st_idx % kLanes) != group) continue;
-                    const uint32_t stage = (uint32_t)group, sphase = (st_idx / kLanes) & 1u;
+                if (g < k_tiles - t0) {
                     uint4 pw[4] = {};
                     if (have_row) {
-                        const uint32_t src = p_s + slot * kPackedSlot + row_off + (uint32_t)kt * kTileBytes;
+                        const uint32_t src = p_s + slot * kPackedSlot + row_off;
 #pragma unroll
                         for (int t = 0; t < 4; ++t) pw[t] = lds128(src + 16u * t);
                     }
-                    if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(aempty + 8 * g, (n_own & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     // word i of piece t, bit plane j, byte b = column 64t + 16i + 4j + b: tensor-memory column 16t + 4i + j.
                     // The 2-bit codes are moved to the TOP of their bytes (value 64 * code, still an unsigned byte):
                     // that takes a left shift, which the multiplier pipe executes, and one AND, where a right shift
-                    // and an AND would both go to the logic pipe that bounds this loop; the epilogue divides by 64.
+                    // and an AND would both go to the logic pipe; the epilogue divides by 64.
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
                         uint32_t v[32];
@@ -313,12 +319,13 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                                 for (int j = 0; j < 4; ++j) v[16 * tt + 4 * i + j] = (w4[i] * (64u >> (2 * j))) & 0xC0C0C0C0u;
                             }
                         }
-                        tmem_st_32x32(a_lane + stage * kAStageCols + 32u * half, v);
+                        tmem_st_32x32(a_dst + 32u * half, v);
                     }
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(afull + 8 * stage);
+                    if (lane == 0) mbar_arrive(afull + 8 * g);
+                    ++n_own;
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pempty + 8 * slot);
@@ -327,39 +334,34 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     } else if (warp < kFirstEpiWarp) {
         // ------------------------------------------------------------------ MMA issuers: one pipeline each
         if (lane == 0) {
-            const int me = warp - kFirstMmaWarp;
-            const uint32_t a_tmem = tmem_base + kAColBase + (uint32_t)me * kAStageCols;
-            uint32_t sc_idx = 0, st_idx = 0, it_idx = 0;
+            const int g = warp - kFirstMmaWarp;
+            const uint32_t a_tmem = tmem_base + kAColBase + (uint32_t)g * kAStageCols;
+            // token images of tile g of a slot: k-block kb at 2 KiB * (2g + kb), 32-byte slice k inside it
+            const uint64_t x_desc = smem_desc_sw128(x_s) + (uint64_t)((g * 2 * kTok * 128) >> 4);
+            uint32_t sc_idx = 0, n_own = 0, it_idx = 0;
             bool ok = true;
             for (int it = item_lo; ok && it < item_hi; ++it, ++it_idx) {
-                const int2 item = item_at(it);
-                const int k_tiles = prob_at(item.x).K / kTileCols;
-                const uint32_t buf = it_idx & 1u, bphase = (it_idx >> 1) & 1u;
-                if (!mbar_wait(tempty + 8 * buf, bphase ^ 1u, abort_flag)) break;
+                const int k_tiles = prob_at(item_at(it).x).K / kTileCols;
+                const uint32_t buf = it_idx & 1u;
+                if (!mbar_wait(tempty + 8 * buf, ((it_idx >> 1) & 1u) ^ 1u, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (buf * kLanes + (uint32_t)me) * kTok;
-                const uint32_t st_item = st_idx;  // this pipeline's first step of the item starts its partial sum
-                for (int t0 = 0; ok && t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
-                    const int tiles = min(kStepTiles, k_tiles - t0);
+                const uint32_t d_tmem = tmem_base + (buf * kLanes + (uint32_t)g) * kTok;
+                for (int t0 = 0; t0 < k_tiles; t0 += kStepTiles, ++sc_idx) {
                     const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
                     // every issuer waits for every slot, also one in which it has no step (see the unpack warps)
                     if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
-                    const uint64_t x_desc = smem_desc_sw128(x_s + slot * kXSlot);
-                    for (int kt = 0; kt < tiles; ++kt, ++st_idx) {
-                        if ((int)(st_idx % kLanes) != me) continue;
-                        const uint32_t sphase = (st_idx / kLanes) & 1u;
-                        if (!mbar_wait(afull + 8 * me, sphase, abort_flag)) { ok = false; break; }
+                    if (g < k_tiles - t0) {
+                        if (!mbar_wait(afull + 8 * g, n_own & 1u, abort_flag)) { ok = false; break; }
                         tc_fence_after();
-                        // k-block kb of the step: token image kt*2 + kb (2 KiB each); 32-byte slice k inside it
-                        const uint64_t b_desc = x_desc + (uint64_t)((kt * 2 * kTok * 128) >> 4);
-                        const bool first = st_idx - st_item < (uint32_t)kLanes;
+                        const uint64_t b_desc = x_desc + (uint64_t)(slot * (kXSlot >> 4));
 #pragma unroll
                         for (int s = 0; s < 8; ++s)
                             umma_i8_ts(d_tmem, a_tmem + 8u * s, b_desc + (uint64_t)((s >> 2) * ((kTok * 128) >> 4) + 2 * (s & 3)),
-                                       kIdesc, (uint32_t)(!first || s != 0));
-                        umma_commit(aempty + 8 * me);  // the codes may be overwritten once these MMAs retire
+                                       kIdesc, (uint32_t)(t0 != 0 || s != 0));
+                        umma_commit(aempty + 8 * g);  // the codes may be overwritten once these MMAs retire
+                        ++n_own;
                     }
-                    if (ok) umma_commit(xempty + 8 * slot);  // counts kLanes arrivals: every issuer is done with the slot
+                    umma_commit(xempty + 8 * slot);  // counts kLanes arrivals: every issuer is done with the slot
                 }
                 if (ok) umma_commit(tfull + 8 * buf);
             }
@@ -368,7 +370,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     } else {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
-        uint32_t it_idx = 0, st_idx = 0;
+        uint32_t it_idx = 0;
         for (int it = item_lo; it < item_hi; ++it, ++it_idx) {
             const int2 item = item_at(it);
             const SProb p = prob_at(item.x);
@@ -384,16 +386,15 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             // the pipelines that had a step in this item hold its partial sums (integers: any order, same total)
             const uint32_t d_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + buf * kLanes * kTok;
             uint32_t r[16];
-            tmem_ld_32x16(d_lane + (st_idx % kLanes) * kTok, r);
+            tmem_ld_32x16(d_lane, r);
             for (int j = 1; j < min(kLanes, k_tiles); ++j) {
                 uint32_t r2[16];
-                tmem_ld_32x16(d_lane + ((st_idx + j) % kLanes) * kTok, r2);
+                tmem_ld_32x16(d_lane + (uint32_t)j * kTok, r2);
 #pragma unroll
                 for (int m = 0; m < kTok; ++m) r[m] += r2[m];
             }
 #pragma unroll
             for (int m = 0; m < kTok; ++m) r[m] = (uint32_t)((int)r[m] >> 6);  // exact: the sums are multiples of 64
-            st_idx += (uint32_t)k_tiles;
             const int n = item.y * kTileRows + quad * 32 + lane;  // this lane's weight row
 #pragma unroll
             for (int m = 0; m < kTok; ++m) {
