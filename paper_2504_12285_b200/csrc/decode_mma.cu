@@ -96,7 +96,10 @@ struct alignas(16) SProb {
     void* y;
     int M, N, K, y_dtype;
 };
-constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + 256 + kItemCap * sizeof(int2) + kProbCap * sizeof(SProb);
+constexpr int kNumBars = 3 * kSlots + 4 * kLanes + 4;               // pfull, pempty, xempty; afull, aempty; tfull, tempty
+constexpr size_t kBarBytes = 512;                                    // barriers, tensor-memory base, abort flag
+static_assert(kNumBars * 8 + 8 <= kBarBytes, "barrier block");
+constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + kBarBytes + kItemCap * sizeof(int2) + kProbCap * sizeof(SProb);
 
 __device__ __forceinline__ SProb load_prob(const MmaProblem& q) {
     SProb v;
@@ -193,9 +196,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t pfull = smem_u32(bars), pempty = pfull + 8 * kSlots, xempty = pempty + 8 * kSlots;
     const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * 2 * kLanes;  // [pipeline][half]
     const uint32_t tfull = aempty + 8 * 2 * kLanes, tempty = tfull + 16;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 3 * kSlots + 4 * kLanes + 4);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-    int2* items_s = reinterpret_cast<int2*>(reinterpret_cast<uint8_t*>(bars) + 256);
+    int2* items_s = reinterpret_cast<int2*>(reinterpret_cast<uint8_t*>(bars) + kBarBytes);
     SProb* probs_s = reinterpret_cast<SProb*>(items_s + kItemCap);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
