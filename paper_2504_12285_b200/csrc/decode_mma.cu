@@ -43,8 +43,7 @@ constexpr int kFirstEpiWarp = kFirstMmaWarp + kLanes;
 constexpr int kMmaThreads = (kFirstEpiWarp + 4) * 32;
 constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;  // 32 KiB of packed weights
 constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;             // 16 KiB: 8 k-blocks of 16 x 128 token images
-constexpr uint32_t kAStageCols = kTileCols / 4;                      // 64 columns: 256 codes per row, 4 per column;
-                                                                     // its two halves are handed over separately
+constexpr uint32_t kAStageCols = kTileCols / 4;                      // 64 columns: 256 codes per row, 4 per column
 constexpr uint32_t kAColBase = 2 * kLanes * kTok;                    // after the two buffers of partial accumulators
 constexpr uint32_t kTmemCols = 512;                                  // power of two >= kAColBase + kLanes * 64
 static_assert(kAColBase + kLanes * kAStageCols <= kTmemCols, "tensor memory");
@@ -96,8 +95,8 @@ struct alignas(16) SProb {
     void* y;
     int M, N, K, y_dtype;
 };
-constexpr int kNumBars = 3 * kSlots + 4 * kLanes + 4;               // pfull, pempty, xempty; afull, aempty; tfull, tempty
-constexpr size_t kBarBytes = 512;                                    // barriers, tensor-memory base, abort flag
+constexpr int kNumBars = 3 * kSlots + 2 * kLanes + 4;               // pfull, pempty, xempty; afull, aempty; tfull, tempty
+constexpr size_t kBarBytes = 256;                                    // barriers, tensor-memory base, abort flag
 static_assert(kNumBars * 8 + 8 <= kBarBytes, "barrier block");
 constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + kBarBytes + kItemCap * sizeof(int2) + kProbCap * sizeof(SProb);
 
@@ -194,8 +193,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t p_s = x_s + kSlots * kXSlot;     // [kSlots] packed weights
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSlots * (size_t)(kXSlot + kPackedSlot));
     const uint32_t pfull = smem_u32(bars), pempty = pfull + 8 * kSlots, xempty = pempty + 8 * kSlots;
-    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * 2 * kLanes;  // [pipeline][half]
-    const uint32_t tfull = aempty + 8 * 2 * kLanes, tempty = tfull + 16;
+    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kLanes;
+    const uint32_t tfull = aempty + 8 * kLanes, tempty = tfull + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int2* items_s = reinterpret_cast<int2*>(reinterpret_cast<uint8_t*>(bars) + kBarBytes);
@@ -213,7 +212,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             mbar_init(pempty + 8 * b, kUnpackWarps);
             mbar_init(xempty + 8 * b, kLanes);
         }
-        for (int b = 0; b < 2 * kLanes; ++b) {
+        for (int b = 0; b < kLanes; ++b) {
             mbar_init(afull + 8 * b, 4);
             mbar_init(aempty + 8 * b, 1);
         }
@@ -304,16 +303,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
 #pragma unroll
                         for (int t = 0; t < 4; ++t) pw[t] = lds128(src + 16u * t);
                     }
+                    if (!mbar_wait(aempty + 8 * g, (n_own & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
                     // word i of piece t, bit plane j, byte b = column 64t + 16i + 4j + b: tensor-memory column 16t + 4i + j.
                     // The 2-bit codes are moved to the TOP of their bytes (value 64 * code, still an unsigned byte):
                     // that takes a left shift, which the multiplier pipe executes, and one AND, where a right shift
                     // and an AND would both go to the logic pipe; the epilogue divides by 64.
-                    // The two 128-column halves of the step are handed to the issuer one by one, so that it multiplies
-                    // one half while the other is being expanded.
 #pragma unroll
                     for (int half = 0; half < 2; ++half) {
-                        if (!mbar_wait(aempty + 8 * (2 * g + half), (n_own & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
                         uint32_t v[32];
 #pragma unroll
                         for (int tt = 0; tt < 2; ++tt) {
@@ -326,12 +323,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                             }
                         }
                         tmem_st_32x32(a_dst + 32u * half, v);
-                        tmem_st_wait();
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(afull + 8 * (2 * g + half));
                     }
-                    if (!ok) break;
+                    tmem_st_wait();
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(afull + 8 * g);
                     ++n_own;
                 }
                 __syncwarp();
@@ -358,18 +354,14 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     // every issuer waits for every slot, also one in which it has no step (see the unpack warps)
                     if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
                     if (g < k_tiles - t0) {
+                        if (!mbar_wait(afull + 8 * g, n_own & 1u, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
                         const uint64_t b_desc = x_desc + (uint64_t)(slot * (kXSlot >> 4));
 #pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            if (!mbar_wait(afull + 8 * (2 * g + half), n_own & 1u, abort_flag)) { ok = false; break; }
-                            tc_fence_after();
-#pragma unroll
-                            for (int s = 4 * half; s < 4 * half + 4; ++s)
-                                umma_i8_ts(d_tmem, a_tmem + 8u * s, b_desc + (uint64_t)((s >> 2) * ((kTok * 128) >> 4) + 2 * (s & 3)),
-                                           kIdesc, (uint32_t)(t0 != 0 || s != 0));
-                            umma_commit(aempty + 8 * (2 * g + half));  // the codes may be overwritten once these MMAs retire
-                        }
-                        if (!ok) break;
+                        for (int s = 0; s < 8; ++s)
+                            umma_i8_ts(d_tmem, a_tmem + 8u * s, b_desc + (uint64_t)((s >> 2) * ((kTok * 128) >> 4) + 2 * (s & 3)),
+                                       kIdesc, (uint32_t)(t0 != 0 || s != 0));
+                        umma_commit(aempty + 8 * g);  // the codes may be overwritten once these MMAs retire
                         ++n_own;
                     }
                     umma_commit(xempty + 8 * slot);  // counts kLanes arrivals: every issuer is done with the slot
