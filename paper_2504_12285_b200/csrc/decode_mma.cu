@@ -113,7 +113,6 @@ __device__ __forceinline__ bool mma_plan_matches(const MmaHeader* h, int count, 
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // A operand in tensor memory (lane = row, four 8-bit codes per 32-bit column), B operand in shared memory.
 __device__ __forceinline__ void umma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -163,21 +162,24 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 // D = s32, A = u8 (64 x weight code, tensor memory), B = s8 (activations, K-major shared memory), M = 128, N = 16.
 constexpr uint32_t kIdesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
 
-template <int VPT>
+// One warp per token, eight tokens per CTA: few enough CTAs that all are resident at once, so the launch_dependents
+// below releases the weight-streaming kernel right away and the two overlap.
 __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeader* __restrict__ hdr,
                                                                   const MmaProblem* __restrict__ probs,
                                                                   const int* __restrict__ row_prob, int count, int total_items,
-                                                                  int grid, int* status_word) {
-    __shared__ RowReduceSmem sm;
-    if (!mma_plan_matches(hdr, count, total_items, grid, (int)gridDim.x)) {
+                                                                  int grid, int rows, int* status_word) {
+    // the kernel that follows may start now: it fetches weights first and waits for this grid before it reads
+    // anything written here (programmatic dependent launch)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!mma_plan_matches(hdr, count, total_items, grid, rows)) {
         if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
         return;
     }
-    const int row = blockIdx.x;
+    const int row = blockIdx.x * kQuantWarps + (threadIdx.x >> 5);
+    if (row >= rows) return;
     const MmaProblem& p = probs[row_prob[row]];
     const int m = row - p.row_begin;
-    quant_row<VPT, 3>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m, p.xsum_out + m, sm,
-                      m & 7);
+    quant_row_warp<3>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m, p.xsum_out + m, m & 7);
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
@@ -244,6 +246,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         // ------------------------------------------------------------------ producers: three copies per warp
         // (a thread starts a bulk copy only every ~200 cycles, and the lanes of a warp take turns)
         const int c = warp * kCopiesPerWarp + lane;  // copy 0 .. 7: packed row block c of the item; copy 8: token images
+        // the token images are written by the quantiser launch before this kernel; the weights are not
+        if (c == kItemRb) asm volatile("griddepcontrol.wait;" ::: "memory");
         uint32_t sc_idx = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
@@ -373,6 +377,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     } else {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;  // tensor-memory lanes 32*quad .. 32*quad+31 belong to this warp
+        asm volatile("griddepcontrol.wait;" ::: "memory");  // scales and code sums come from the quantiser launch
         uint32_t it_idx = 0;
         for (int it = item_lo; it < item_hi; ++it, ++it_idx) {
             const int2 item = item_at(it);
@@ -499,7 +504,6 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
     std::vector<int2> items;
     std::vector<double> weight;  // packed tiles of each item
     std::vector<int> row_prob;
-    int max_k = 0;
     {
         uint8_t* x_ptr = reinterpret_cast<uint8_t*>(base + L.x_off);
         float* d_ptr = reinterpret_cast<float*>(base + L.d_off);
@@ -532,7 +536,6 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
             mp.push_back(v);
             row += q.M;
             x_ptr += (size_t)kTok * q.K;
-            if (q.K > max_k) max_k = q.K;
         }
         row_prob.push_back(0);
     }
@@ -577,12 +580,9 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
 
     // ---- launch 1: quantise every token into the 16-row tile images ----
     if (!(flags & BITLINEAR_BATCH_REUSE_ACT)) {
-        const int vpt = (max_k / 8 + kQuantThreads - 1) / kQuantThreads;
-        const dim3 g((unsigned)rows), b(kQuantThreads);
         const int* rp = reinterpret_cast<const int*>(base + L.row_prob_off);
-        if (vpt <= 1) mma_quant_kernel<1><<<g, b, 0, st>>>(hdr, probs_dev, rp, n_prob, total_items, grid, sw);
-        else if (vpt <= 2) mma_quant_kernel<2><<<g, b, 0, st>>>(hdr, probs_dev, rp, n_prob, total_items, grid, sw);
-        else mma_quant_kernel<4><<<g, b, 0, st>>>(hdr, probs_dev, rp, n_prob, total_items, grid, sw);
+        mma_quant_kernel<<<(unsigned)((rows + kQuantWarps - 1) / kQuantWarps), kQuantThreads, 0, st>>>(hdr, probs_dev, rp, n_prob,
+                                                                                                   total_items, grid, rows, sw);
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
 
@@ -596,8 +596,23 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
     prm.total_items = total_items;
     prm.rows = rows;
     prm.status_word = sw;
-    decode_mma_kernel<<<grid, kMmaThreads, kMmaSmem, st>>>(prm);
-    return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+    // programmatic dependent launch: the kernel may begin (set-up, first weight copies) while the quantiser launch
+    // before it is still running; the threads that read that launch's results call griddepcontrol.wait first
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kMmaThreads);
+    cfg.dynamicSmemBytes = kMmaSmem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, decode_mma_kernel, prm) != cudaSuccess) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
+    return BITLINEAR_OK;
 }
 
 }  // namespace bitlinear
