@@ -8,17 +8,21 @@
 // memory only carries the packed bytes and the token images, so the copy ring can be deep.)
 //
 // One persistent CTA per SM owns a contiguous, byte-balanced range of work items (128 weight rows of one matmul).
-//   warp 0      producer : bulk copies of packed weights (eight 16-row blocks x up to four 16x256 tiles, 4 KiB each)
-//                          and of the matching slice of the quantised tokens (16-row tile images) into a 4-slot ring
-// The 256-column steps of a CTA's work are dealt round-robin to kLanes pipelines, each with its own unpack group, its
-// own 64 tensor-memory columns for the codes, its own MMA-issuing thread and its own partial accumulator (one thread
-// can start a tcgen05.mma only every ~55 cycles whatever its shape, several threads scale; the integer partial sums
-// are added in the epilogue, exactly):
+// Launch 1 (mma_quant_kernel, one warp per token) writes the quantised tokens as 16-row tile images; launch 2
+// (decode_mma_kernel) starts under programmatic dependent launch and streams weights while launch 1 still runs.
+//   producer warps : three warps, three bulk copies each (a thread starts a copy only every few hundred cycles):
+//                    eight packed 16-row blocks x up to four 16x256 tiles (4 KiB each) and the matching slice of
+//                    the token images, into a 4-slot ring of 48 KiB
+// Tile g of every ring slot belongs to pipeline g (kLanes = 4 pipelines), each with its own unpack group, its own 64
+// tensor-memory columns for the codes, its own MMA-issuing thread and its own partial accumulator (one thread can
+// start a tcgen05.mma only every ~55 cycles whatever its shape, several threads scale; the integer partial sums are
+// added in the epilogue, exactly):
 //   unpack groups  : four warps each, the warp of tensor-memory lane quarter q expands weight rows 32q .. 32q+31
-//                    (thread = row) into the pipeline's 64 columns
+//                    (thread = row) into the pipeline's 64 columns, as 64 x code so that a left shift and one AND do
 //   MMA warps      : one thread each issues the 8 tcgen05.mma (128 x 16 x 32, A from tensor memory) of a step
-//   epilogue warps : tcgen05.ld of the finished partial accumulators (double buffered), their sum minus the code
-//                    sum, two fp32 multiplies, stores coalesced along the weight rows
+//   epilogue warps : tcgen05.ld of the finished partial accumulators (double buffered), their sum / 64 minus the
+//                    code sum, two fp32 multiplies, stores coalesced along the weight rows
+// The work items and matmul descriptors of the CTA are copied to shared memory first.
 // Every wait is bounded; on a timeout the CTA raises the sticky status word and leaves.
 #include <algorithm>
 #include <vector>
