@@ -1,4 +1,5 @@
-// Batched decode: many independent BitLinear forwards (M <= 16 tokens each) in two launches.
+// Batched decode: many independent BitLinear forwards of ONE token each in two launches (sub-batches in which a
+// problem has 2 to 16 tokens run on the tensor cores instead, decode_mma.cu, which is faster from two tokens on).
 // (Paper Section 5.1: the decode cost is the packed weight bytes that must cross HBM; a single
 // decode matmul is smaller than the memory system's bandwidth-delay product, so the weights of a
 // whole batch of matmuls are streamed back to back by one persistent kernel.)
@@ -502,10 +503,11 @@ namespace bitlinear {
 size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const int* idx, int n);
 int prefill_group_forward(const bitlinear_problem* problems, const int* idx, int n, void* ws, bool skip_quant,
                           cudaStream_t st);
-// Sub-batches with a problem of more than kDp4aMaxTokens tokens run on the tensor cores (decode_mma.cu).
+// Sub-batches with a problem of more than kDp4aMaxTokens tokens run on the tensor cores (decode_mma.cu): measured on
+// the 210-matmul decode step, 145 us per step there at 2 to 5 tokens against 171 to 174 us for the kernel below.
 size_t decode_mma_workspace_bytes(const bitlinear_problem* problems, int count);
 int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes, void* stream);
-constexpr int kDp4aMaxTokens = 4;
+constexpr int kDp4aMaxTokens = 1;
 
 namespace {
 
@@ -640,9 +642,8 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     }
     // shared memory: chunk ring + descriptor table + activation arena; activations that do not fit the arena are read
     // through L1 instead, and only as many descriptors as fit a quarter of the space are cached
-    const int mt = max_m <= 1 ? 1 : 4;
-    const int chunk_tiles = mt == 1 ? 5 : 4;
-    const int groups = (max_m + mt - 1) / mt;  // 1 .. 4
+    const int chunk_tiles = 5;
+    const int groups = 1;  // one token per problem here: every warp runs its own pipeline
     const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles, groups) - 128;
     if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
     if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
@@ -693,8 +694,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.arena_bytes = (int)arena_max;
     const size_t smem = ring_bytes(chunk_tiles, groups) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
     cudaError_t e;
-    if (mt == 1) e = launch_stream<1, 5>(prm, grid, smem, st);
-    else e = launch_stream<4, 4>(prm, grid, smem, st);
+    e = launch_stream<1, 5>(prm, grid, smem, st);
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
