@@ -175,7 +175,9 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  * Problems of at most 16 tokens (the decode regime of Section 5.1, where the cost is the packed
  * weight bytes streamed from HBM) take two launches together: one fused RMSNorm+quantiser launch
  * over every token, then one persistent kernel that streams the packed weights of all of them
- * back to back.  Problems of more than 16 tokens (prefill; N must be a multiple of 128) take three
+ * back to back (dot-products-of-four when every such problem has one token; otherwise the tensor
+ * cores, with the codes unpacked in registers and handed over in tensor memory).  Problems of more
+ * than 16 tokens (prefill; N must be a multiple of 128) take three
  * launches together: the quantiser, the expansion of the packed weights into tensor-core tile
  * images, and one persistent tcgen05 kernel that runs every tile of every matmul; problems that
  * name the same x, gain, rms_eps, M and K (q/k/v or gate/up of a layer) share one quantised copy.
