@@ -186,6 +186,16 @@ __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeade
     quant_row_warp<3>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m, p.xsum_out + m, m & 7);
 }
 
+// 2 x 16 packed bytes (128 codes of one weight row) -> 32 tensor-memory columns of 64 x code.
+__device__ __forceinline__ void expand_codes(const uint4& qa, const uint4& qb, uint32_t (&v)[32]) {
+    const uint32_t w8[8] = {qa.x, qa.y, qa.z, qa.w, qb.x, qb.y, qb.z, qb.w};
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[4 * i + j] = (w8[i] * (64u >> (2 * j))) & 0xC0C0C0C0u;
+    }
+}
+
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     uint4 v;
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
@@ -311,27 +321,19 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
 #pragma unroll
                         for (int t = 0; t < 4; ++t) pw[t] = lds128(src + 16u * t);
                     }
-                    if (!mbar_wait(aempty + 8 * g, (n_own & 1u) ^ 1u, abort_flag)) { ok = false; break; }
-                    tc_fence_after();
                     // word i of piece t, bit plane j, byte b = column 64t + 16i + 4j + b: tensor-memory column 16t + 4i + j.
                     // The 2-bit codes are moved to the TOP of their bytes (value 64 * code, still an unsigned byte):
                     // that takes a left shift, which the multiplier pipe executes, and one AND, where a right shift
                     // and an AND would both go to the logic pipe; the epilogue divides by 64.
-#pragma unroll
-                    for (int half = 0; half < 2; ++half) {
-                        uint32_t v[32];
-#pragma unroll
-                        for (int tt = 0; tt < 2; ++tt) {
-                            const uint4 q4 = pw[2 * half + tt];
-                            const uint32_t w4[4] = {q4.x, q4.y, q4.z, q4.w};
-#pragma unroll
-                            for (int i = 0; i < 4; ++i) {
-#pragma unroll
-                                for (int j = 0; j < 4; ++j) v[16 * tt + 4 * i + j] = (w4[i] * (64u >> (2 * j))) & 0xC0C0C0C0u;
-                            }
-                        }
-                        tmem_st_32x32(a_dst + 32u * half, v);
-                    }
+                    // The first half is expanded BEFORE the wait for the tensor-memory stage (the MMAs of the
+                    // pipeline's previous step are still reading it), the second half after the first is stored.
+                    uint32_t v[32];
+                    expand_codes(pw[0], pw[1], v);
+                    if (!mbar_wait(aempty + 8 * g, (n_own & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    tmem_st_32x32(a_dst, v);
+                    expand_codes(pw[2], pw[3], v);
+                    tmem_st_32x32(a_dst + 32u, v);
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
