@@ -160,6 +160,38 @@ def test_batch_many_tokens_match_single_forward_bitwise(M):
         assert torch.equal(y, y1)
 
 
+@pytest.mark.parametrize("M", [1, 16])
+def test_batch_full_decode_step_sampled(M):
+    # the launch configuration the benchmark times, with its seeded weights: 30 layers x 7 matmuls in ONE call
+    # (210 problems, 521 MB of packed weights), checked on sampled outputs of every problem
+    rng = np.random.default_rng(1234 + M)
+    items, refs = [], []
+    for layer in range(wl.N_LAYERS):
+        for j, (name, n, k) in enumerate(wl.LAYER_SHAPES):
+            W = wl.latent_weights(n, k, wl.layer_seed(2, layer, name))
+            packed, s_w = bl.bitlinear_pack_weights(W.to(DEV), wl.WEIGHT_EPS)
+            wref = oracle.quantize_weights(W.numpy(), wl.WEIGHT_EPS)
+            assert np.array_equal(packed.cpu().numpy(), wref["packed"])
+            n_idx = np.concatenate([rng.integers(0, n, 44), [0, n - 1, 127 % n, 128 % n]]).astype(np.int32)
+            x = wl.activations_student_t(M, k, wl.seed_for(2, j, layer))
+            refs.append((x, n_idx, wref["wq"][n_idx].copy(), wref["s_w"]))
+            items.append((x.to(DEV), None, packed, s_w, torch.full((M, n), float("nan"), dtype=torch.float32, device=DEV)))
+    batch = bl.ProblemBatch(items, wl.RMS_EPS)
+    run(batch, reuse=True)
+    for i, ((x, n_idx, wq_rows, s_w), (_, _, _, _, y)) in enumerate(zip(refs, batch.tensors)):
+        qref = oracle.rmsnorm_quant(wl.bf16_bits(x), None, wl.RMS_EPS)
+        ok_rows = np.nonzero(qref["fragile"] == 0)[0]
+        y_host = y.cpu().numpy()
+        assert not np.isnan(y_host).any()
+        if len(ok_rows) == 0:
+            continue
+        m_idx = rng.choice(ok_rows, len(n_idx)).astype(np.int32)
+        acc = oracle.matmul_i32_sampled(qref["q"], wq_rows, m_idx, np.arange(len(n_idx), dtype=np.int32))
+        want = (oracle.dequant(acc.reshape(1, -1), s_w, np.ones(1, np.float32))[0] * qref["d"][m_idx]).astype(np.float64)
+        got = y_host[m_idx, n_idx].astype(np.float64)
+        assert np.all(np.abs(got - want) <= 1e-6 * np.abs(want)), i
+
+
 # ---- problems of more than 16 tokens in the same entry point: grouped tensor-core path ----
 
 
