@@ -157,11 +157,7 @@ struct ChunkCursor {
 // MT = tokens per warp (1 or 4).  kChunkTiles = 16x256 tiles (1 KiB each) per bulk copy at most.
 // The quantised activations of the problems the CTA touches are staged in shared memory once, as far as the arena
 // reaches; those of the remaining problems are read through L1, which is slower.
-// FUSED (one token per problem, every problem of the CTA in the table and the arena): the kernel also runs the
-// RMSNorm + int8 quantiser of the tokens it needs, one warp per token, straight into the arena - no quantiser launch.
-// A token that several CTAs need is quantised by each of them (a few KB each, the same bits); the results also go to
-// the workspace, where a later call with BITLINEAR_BATCH_REUSE_ACT finds them.
-template <int MT, int kChunkTiles, bool FUSED>
+template <int MT, int kChunkTiles>
 __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const StreamParams prm) {
     extern __shared__ __align__(128) uint8_t smem[];
     // [ring: (16 / G) row-block lanes x kRing slots][full barriers][empty barriers][abort flag][descriptor table]
@@ -268,35 +264,12 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             e.s_w = *pr.s_w;
         }
         if (lane < kGemvMaxTokens) {
-            table[i].d[lane] = (!FUSED && lane < pr.M) ? pr.d[lane] : 0.0f;
-            table[i].xsum[lane] = (!FUSED && lane < pr.M) ? pr.xsum[lane] : 0;
+            table[i].d[lane] = lane < pr.M ? pr.d[lane] : 0.0f;
+            table[i].xsum[lane] = lane < pr.M ? pr.xsum[lane] : 0;
         }
     }
     __syncthreads();
-    if (FUSED) {
-        if (threadIdx.x == 0) {
-            int off = 0;
-            for (int i = 0; i < n_tab; ++i) {  // the host launched this variant because everything fits
-                table[i].x_off = off;
-                off += table[i].K;
-            }
-        }
-        __syncthreads();
-        for (int i = warp; i < n_tab; i += kStreamWarps) {
-            const DevProblem& pr = probs[p_lo + i];
-            if (pr.M != 1) continue;
-            int8_t* row_s = reinterpret_cast<int8_t*>(arena) + table[i].x_off;
-            quant_row_warp<1>(pr.x, pr.gain, pr.eps, pr.K, row_s, &table[i].d[0], &table[i].xsum[0]);
-            __syncwarp();
-            for (int o = lane * 16; o < pr.K; o += 32 * 16)
-                *reinterpret_cast<uint4*>(pr.xq + o) = *reinterpret_cast<const uint4*>(row_s + o);
-            if (lane == 0) {
-                pr.d[0] = table[i].d[0];
-                pr.xsum[0] = table[i].xsum[0];
-            }
-        }
-        __syncthreads();
-    } else {
+    {
         if (threadIdx.x == 0) {
             int off = 0;
             for (int i = 0; i < n_tab; ++i) {
@@ -478,9 +451,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (*abort_flag && threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
 }
 
-template <int MT, int kChunkTiles, bool FUSED>
+template <int MT, int kChunkTiles>
 cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<MT, kChunkTiles, FUSED>,
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<MT, kChunkTiles>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // programmatic dependent launch: the kernel may begin (barrier set-up, first weight copies) while the quantiser
@@ -495,7 +468,7 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<MT, kChunkTiles, FUSED>, prm);
+    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<MT, kChunkTiles>, prm);
 }
 
 struct PlanLayout {
@@ -672,19 +645,9 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     const int chunk_tiles = 5;
     const int groups = 1;  // one token per problem here: every warp runs its own pipeline
     const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles, groups) - 128;
-    bool all_fit = true;  // every CTA has all its problems in the table and all their activations in the arena
-    if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) {
-        table_cap = (int)(smem_limit / 4 / sizeof(SProb));
-        all_fit = false;
-    }
-    if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) {
-        arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
-        all_fit = false;
-    }
-    arena_max = (arena_max + 255) & ~(size_t)255;
-    if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max -= 256;
-    // One token per problem and everything fits: the stream kernel quantises the tokens itself (no quantiser launch).
-    const bool fused = all_fit && max_m == 1 && !(flags & BITLINEAR_BATCH_REUSE_ACT);
+    if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
+    if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
+    arena_max &= ~(size_t)255;
 
     PlanHeader hdr_host;
     hdr_host.magic = kPlanMagic;
@@ -705,7 +668,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     const DevProblem* probs_dev = reinterpret_cast<const DevProblem*>(base + L.probs_off);
 
     // ---- launch 1: quantise every token of every problem ----
-    if (!fused && !(flags & BITLINEAR_BATCH_REUSE_ACT)) {
+    if (!(flags & BITLINEAR_BATCH_REUSE_ACT)) {
         const int vpt = (max_k / 8 + kQuantThreads - 1) / kQuantThreads;
         const dim3 g((unsigned)rows), b(kQuantThreads);
         const PlanHeader* h = reinterpret_cast<const PlanHeader*>(base);
@@ -731,8 +694,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.arena_bytes = (int)arena_max;
     const size_t smem = ring_bytes(chunk_tiles, groups) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
     cudaError_t e;
-    if (fused) e = launch_stream<1, 5, true>(prm, grid, smem, st);
-    else e = launch_stream<1, 5, false>(prm, grid, smem, st);
+    e = launch_stream<1, 5>(prm, grid, smem, st);
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
