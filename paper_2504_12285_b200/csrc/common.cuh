@@ -62,6 +62,9 @@ constexpr int kMaxGroup = 32;
 struct GemmGroupHeader {
     int count, total_tiles;
     unsigned long long region_base;  // CTA-pair kernel: address its tensor map starts at (tile images are addressed as rows of 128 B)
+    // CTA-pair kernel, or nullptr: ready[i] counts the packed words of problem i whose codes have been written; the
+    // kernel runs beside the expansion launch and reads problem i only once ready[i] == N * K / 16
+    const int* ready;
 };
 // layout of the uploaded group table: GemmGroupHeader, then count x GemmProblem
 constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof(GemmProblem);
@@ -69,8 +72,13 @@ constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof
 // Grouped launch: fills m_tiles / tile_begin, uploads the table to table_dev (kGroupTableBytes) and runs every tile of
 // every problem in one persistent kernel.  a_tiled = activations given as tile images (any count), else one problem with
 // row-major activations.  Returns a bitlinear_status.
+// `before` (optional) is called after the table upload and before the GEMM kernel is launched: launches that produce
+// the operands go there, so that no copy sits between them and the GEMM kernel.  With `ready` set (see
+// GemmGroupHeader) the CTA-pair kernel is launched as a programmatic dependent of the last of those launches.
+typedef int (*GemmBeforeKernel)(void* ctx);
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev, cudaStream_t st,
-                const void* region_base = nullptr, size_t region_bytes = 0);
+                const void* region_base = nullptr, size_t region_bytes = 0, const int* ready = nullptr,
+                GemmBeforeKernel before = nullptr, void* before_ctx = nullptr);
 size_t gemm_codes_bytes(int N, int K);
 size_t gemm_a_tiles_bytes(int M, int K);
 

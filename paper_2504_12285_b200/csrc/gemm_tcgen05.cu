@@ -242,6 +242,12 @@ __device__ __forceinline__ void drain_accumulator(const GemmProblem& p, uint32_t
 
 // Tile -> (problem, token rows, weight rows).  Tiles of one problem are numbered with the token tile
 // fastest, so CTAs that run side by side share the weight tile; problems follow each other in table order.
+__device__ __forceinline__ int ld_acquire_gpu_s32(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 struct TileWalk {
     const GemmProblem* probs;
     int count, pi;
@@ -494,10 +500,26 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
+            int ready_pi = -1;  // last problem whose codes are known to be complete
             for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
                 const GemmProblem& p = walk.find(tile);
                 const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
                 const int k_blocks = p.K / BK;
+                if (hdr.ready != nullptr && walk.pi != ready_pi) {
+                    // the expansion launch may still be writing this problem's codes: wait for its word count (bounded)
+                    const int target = (int)((long long)p.N * p.K / 16);
+                    const unsigned long long t0 = globaltimer_ns();
+                    unsigned spins = 0;
+                    while (ld_acquire_gpu_s32(hdr.ready + walk.pi) < target) {
+                        if ((++spins & 63u) == 0u) {
+                            if (*abort_flag) { ok = false; break; }
+                            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; ok = false; break; }
+                        }
+                    }
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");  // the copies below read what generic stores wrote
+                    ready_pi = walk.pi;
+                }
                 // rows (of 128 bytes) of this CTA's operand images inside the mapped region
                 const int a_row = (int)((reinterpret_cast<unsigned long long>(p.a_tiles) - hdr.region_base) >> 7) +
                                   (2 * mt + (int)rank) * k_blocks * 128;
@@ -635,7 +657,8 @@ bool make_map_rows128(CUtensorMap* map, const void* base, size_t bytes) {
 }
 
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev,
-                cudaStream_t st, const void* region_base, size_t region_bytes) {
+                cudaStream_t st, const void* region_base, size_t region_bytes, const int* ready, GemmBeforeKernel before,
+                void* before_ctx) {
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     static int sm_count = 0;
@@ -670,9 +693,14 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     hdr->count = count;
     hdr->total_tiles = tiles;
     hdr->region_base = reinterpret_cast<unsigned long long>(region_base);
+    hdr->ready = pairs ? ready : nullptr;
     if (cudaMemcpyAsync(table_dev, host, kGroupTableBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
+    }
+    if (before != nullptr) {
+        const int rc = before(before_ctx);
+        if (rc != BITLINEAR_OK) return rc;
     }
     CUtensorMap map_a;
     memset(&map_a, 0, sizeof(map_a));
@@ -684,13 +712,16 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
         cfg.blockDim = dim3(THREADS);
         cfg.dynamicSmemBytes = P_SMEM_BYTES;
         cfg.stream = st;
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = 2;
         attr[0].val.clusterDim.y = 1;
         attr[0].val.clusterDim.z = 1;
+        // beside the expansion launch: the kernel waits per problem on the ready counters, not on the whole launch
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = 1;
+        cfg.numAttrs = ready != nullptr ? 2 : 1;
         const cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_i8_pair_kernel, map_a, (const uint8_t*)table_dev, device_status_word());
         if (e != cudaSuccess) cudaGetLastError();
         return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;

@@ -6,9 +6,12 @@
 //   launch 1  group_quant_warp_kernel : one warp per token - fused RMSNorm + absmax int8 quantiser; codes go into
 //                                   128 x 128 tile images (128-byte swizzle) of the activation operand.  Problems
 //                                   that read the same activations share one quantised copy.
-//   launch 2  group_unpack_kernel : packed 2-bit weights -> byte codes in 256 x 128 tile images.
+//   launch 2  group_unpack_kernel : packed 2-bit weights -> byte codes in 256 x 128 tile images, with a count of
+//                                   finished words per problem.
 //   launch 3  gemm_i8_pair_kernel : every tile of every matmul on CTA pairs (gemm_i8_kernel<true> when the SMs do not
-//                                   pair up), operands fetched as whole tile images.
+//                                   pair up), operands fetched as whole tile images.  The pair kernel starts
+//                                   beside launch 2 (programmatic dependent launch) and begins a problem when
+//                                   its word count is complete.
 // Problems are ordered by decreasing K so that the long tiles are scheduled first and the tail is made of short ones.
 #include <algorithm>
 #include <vector>
@@ -49,31 +52,42 @@ __global__ void __launch_bounds__(kQuantThreads) group_quant_warp_kernel(const P
                       m & 7);
 }
 
-// One thread expands one packed word (16 codes) into its 16-byte piece of a 256 x 128 tile image.
+// Expansion of the packed weights into tile images: one thread per packed word (16 codes -> its 16-byte piece of a
+// 256 x 128 image), persistent CTAs that walk the words of all problems in table order, 256 words at a time.  After
+// every 256 words the CTA adds them to the problem's ready counter: the GEMM kernel, which starts beside this launch,
+// reads a problem's images as soon as all its words are counted.  (N * K / 16 is a multiple of 2,048 for every valid
+// shape, so 256 consecutive words never straddle two problems.)
 __global__ void __launch_bounds__(256) group_unpack_kernel(const PrefillItem* __restrict__ items, int count,
-                                                           long long total_words) {
-    const long long word = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    if (word >= total_words) return;
+                                                           long long total_words, int* __restrict__ ready) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int i = 0;
-    while (i + 1 < count && word >= items[i + 1].word_begin) ++i;
-    const PrefillItem& p = items[i];
-    const size_t w = (size_t)(word - p.word_begin);
-    const int k_tiles = p.K / kTileCols;
-    // position of packed word w (see "Packed weight layout" in bitlinear.h)
-    const size_t tile = w >> 8;
-    const int wo = (int)(w & 255);
-    const int h = wo >> 7, g = (wo >> 4) & 7, t = (wo >> 2) & 3, q = wo & 3;
-    const int n = (int)(tile / k_tiles) * kTileRows + 8 * h + g;
-    const int k0 = (int)(tile % k_tiles) * kTileCols + 64 * t + 16 * q;
-    const uint32_t v = p.packed[w];
-    const int r = n & 255, piece = (k0 & 127) >> 4;
-    const size_t img = (size_t)(n >> 8) * (p.K / 128) + (k0 >> 7);
-    *reinterpret_cast<uint4*>(p.codes + img * 32768 + (size_t)r * 128 + ((piece ^ (r & 7)) << 4)) =
-        make_uint4(v & 0x03030303u, (v >> 2) & 0x03030303u, (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
+    for (long long chunk = (long long)blockIdx.x * 256; chunk < total_words; chunk += (long long)gridDim.x * 256) {
+        const long long word = chunk + threadIdx.x;
+        while (i + 1 < count && chunk >= items[i + 1].word_begin) ++i;
+        const PrefillItem& p = items[i];
+        const size_t w = (size_t)(word - p.word_begin);
+        const int k_tiles = p.K / kTileCols;
+        // position of packed word w (see "Packed weight layout" in bitlinear.h)
+        const size_t tile = w >> 8;
+        const int wo = (int)(w & 255);
+        const int h = wo >> 7, g = (wo >> 4) & 7, t = (wo >> 2) & 3, q = wo & 3;
+        const int n = (int)(tile / k_tiles) * kTileRows + 8 * h + g;
+        const int k0 = (int)(tile % k_tiles) * kTileCols + 64 * t + 16 * q;
+        const uint32_t v = p.packed[w];
+        const int r = n & 255, piece = (k0 & 127) >> 4;
+        const size_t img = (size_t)(n >> 8) * (p.K / 128) + (k0 >> 7);
+        *reinterpret_cast<uint4*>(p.codes + img * 32768 + (size_t)r * 128 + ((piece ^ (r & 7)) << 4)) =
+            make_uint4(v & 0x03030303u, (v >> 2) & 0x03030303u, (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
+        __syncthreads();  // every store of the chunk is ordered before the fence and the count below
+        if (threadIdx.x == 0) {
+            __threadfence();
+            atomicAdd(ready + i, 256);
+        }
+    }
 }
 
 struct GroupLayout {
-    size_t table_off, items_off, total;
+    size_t table_off, items_off, ready_off, total;
     std::vector<size_t> a_off, codes_off, d_off, xsum_off;
 };
 
@@ -84,6 +98,8 @@ GroupLayout group_layout(const bitlinear_problem* problems, const int* idx, int 
     off = align_up(off + kGroupTableBytes, 256);
     L.items_off = off;
     off = align_up(off + kItemTableBytes, 256);
+    L.ready_off = off;
+    off = align_up(off + kMaxGroup * sizeof(int), 256);
     for (int i = 0; i < n; ++i) {
         const bitlinear_problem& q = problems[idx[i]];
         L.a_off.push_back(off);
@@ -112,6 +128,12 @@ size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const in
 int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, int n_in, void* ws, bool skip_quant,
                           cudaStream_t st) {
     char* base_all = static_cast<char*>(ws);
+    int sm_count = 0, dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        sm_count <= 0) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
     for (int b = 0; b < n_in; b += kMaxGroup) {
         const int n = std::min(kMaxGroup, n_in - b);
         std::vector<int> idx(idx_in + b, idx_in + b + n);
@@ -156,18 +178,37 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             g.M = q.M; g.N = q.N; g.K = q.K; g.y_dtype = q.y_dtype;
         }
         PrefillItem* items_dev = reinterpret_cast<PrefillItem*>(base + L.items_off);
-        if (cudaMemcpyAsync(items_dev, items, sizeof(PrefillItem) * n, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        int* ready = reinterpret_cast<int*>(base + L.ready_off);
+        if (cudaMemsetAsync(ready, 0, kMaxGroup * sizeof(int), st) != cudaSuccess ||
+            cudaMemcpyAsync(items_dev, items, sizeof(PrefillItem) * n, cudaMemcpyHostToDevice, st) != cudaSuccess) {
             cudaGetLastError();
             return BITLINEAR_ERR_CUDA;
         }
-        if (!skip_quant) {
-            const unsigned blocks = (unsigned)((rows + kQuantWarps - 1) / kQuantWarps);
-            group_quant_warp_kernel<<<blocks, kQuantThreads, 0, st>>>(items_dev, n, rows);
-            if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
-        }
-        group_unpack_kernel<<<(unsigned)((words + 255) / 256), 256, 0, st>>>(items_dev, n, words);
-        if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
-        const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st, base, L.total);
+        // The quantiser and expansion launches go between the GEMM's table upload and the GEMM kernel, which starts
+        // as a programmatic dependent of the expansion launch and follows it problem by problem.
+        struct Launches {
+            const PrefillItem* items_dev;
+            int* ready;
+            int n, rows, sm_count;
+            long long words;
+            bool skip_quant;
+            cudaStream_t st;
+            static int run(void* ctx) {
+                const Launches& a = *static_cast<const Launches*>(ctx);
+                if (!a.skip_quant) {
+                    const unsigned blocks = (unsigned)((a.rows + kQuantWarps - 1) / kQuantWarps);
+                    group_quant_warp_kernel<<<blocks, kQuantThreads, 0, a.st>>>(a.items_dev, a.n, a.rows);
+                    if (cudaGetLastError() != cudaSuccess) return (int)BITLINEAR_ERR_CUDA;
+                }
+                // at most four CTAs per SM, so that the GEMM kernel's CTAs find room beside them
+                const long long chunks = (a.words + 255) / 256;
+                const unsigned grid = (unsigned)std::min<long long>(chunks, 4LL * a.sm_count);
+                group_unpack_kernel<<<grid, 256, 0, a.st>>>(a.items_dev, a.n, a.words, a.ready);
+                return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
+            }
+        } launches = {items_dev, ready, n, rows, sm_count, words, skip_quant, st};
+        const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st, base, L.total, ready,
+                                   &Launches::run, &launches);
         if (rc != BITLINEAR_OK) return rc;
     }
     return BITLINEAR_OK;
