@@ -57,13 +57,16 @@ struct GemmProblem {
     int M, N, K, y_dtype;
     int m_tiles;     // ceil(M / 128)
     int tile_begin;  // tiles of the problems before this one
+    int nt_begin;    // 256-row weight tiles of the problems before this one (index into the ready counters)
+    int pad;
 };
 constexpr int kMaxGroup = 32;
 struct GemmGroupHeader {
     int count, total_tiles;
     unsigned long long region_base;  // CTA-pair kernel: address its tensor map starts at (tile images are addressed as rows of 128 B)
-    // CTA-pair kernel, or nullptr: ready[i] counts the packed words of problem i whose codes have been written; the
-    // kernel runs beside the expansion launch and reads problem i only once ready[i] == N * K / 16
+    // CTA-pair kernel, or nullptr: ready[nt_begin + nt] counts the packed words of 256-row weight tile nt of a problem
+    // whose codes have been written; the kernel runs beside the expansion launch and reads that tile only once the
+    // count has reached rows_in_tile * K / 16
     const int* ready;
 };
 // layout of the uploaded group table: GemmGroupHeader, then count x GemmProblem

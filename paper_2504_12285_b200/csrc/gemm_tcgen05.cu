@@ -500,17 +500,17 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            int ready_pi = -1;  // last problem whose codes are known to be complete
+            int ready_idx = -1;  // last weight tile whose codes are known to be complete
             for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
                 const GemmProblem& p = walk.find(tile);
                 const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
                 const int k_blocks = p.K / BK;
-                if (hdr.ready != nullptr && walk.pi != ready_pi) {
-                    // the expansion launch may still be writing this problem's codes: wait for its word count (bounded)
-                    const int target = (int)((long long)p.N * p.K / 16);
+                if (hdr.ready != nullptr && p.nt_begin + nt != ready_idx) {
+                    // the expansion launch may still be writing this weight tile's codes: wait for its word count (bounded)
+                    const int target = min(BN, p.N - nt * BN) * (p.K / 16);
                     const unsigned long long t0 = globaltimer_ns();
                     unsigned spins = 0;
-                    while (ld_acquire_gpu_s32(hdr.ready + walk.pi) < target) {
+                    while (ld_acquire_gpu_s32(hdr.ready + p.nt_begin + nt) < target) {
                         if ((++spins & 63u) == 0u) {
                             if (*abort_flag) { ok = false; break; }
                             if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; ok = false; break; }
@@ -518,7 +518,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
                     }
                     if (!ok) break;
                     asm volatile("fence.proxy.async;" ::: "memory");  // the copies below read what generic stores wrote
-                    ready_pi = walk.pi;
+                    ready_idx = p.nt_begin + nt;
                 }
                 // rows (of 128 bytes) of this CTA's operand images inside the mapped region
                 const int a_row = (int)((reinterpret_cast<unsigned long long>(p.a_tiles) - hdr.region_base) >> 7) +
@@ -683,11 +683,13 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     // CTA pairs (256 x 256 tiles) when the operands are tile images inside one mapped region and the SMs pair up
     const bool pairs = a_tiled && region_base != nullptr && (sm_count % 2) == 0;
     const int tile_m = pairs ? 256 : BM;
-    int tiles = 0;
+    int tiles = 0, n_tiles = 0;
     for (int i = 0; i < count; ++i) {
         probs[i].m_tiles = (probs[i].M + tile_m - 1) / tile_m;
         probs[i].tile_begin = tiles;
+        probs[i].nt_begin = n_tiles;
         tiles += probs[i].m_tiles * ((probs[i].N + BN - 1) / BN);
+        n_tiles += (probs[i].N + BN - 1) / BN;
         tab[i] = probs[i];
     }
     hdr->count = count;

@@ -34,7 +34,7 @@ struct PrefillItem {
     float eps;
     int M, N, K;
     int row_begin;  // tokens of the problems before this one
-    int pad;
+    int nt_begin;   // 256-row weight tiles of the problems before this one
 };
 constexpr size_t kItemTableBytes = kMaxGroup * sizeof(PrefillItem);
 
@@ -53,41 +53,49 @@ __global__ void __launch_bounds__(kQuantThreads) group_quant_warp_kernel(const P
 }
 
 // Expansion of the packed weights into tile images: one thread per packed word (16 codes -> its 16-byte piece of a
-// 256 x 128 image), persistent CTAs that walk the words of all problems in table order, 256 words at a time.  After
-// every 256 words the CTA adds them to the problem's ready counter: the GEMM kernel, which starts beside this launch,
-// reads a problem's images as soon as all its words are counted.  (N * K / 16 is a multiple of 2,048 for every valid
-// shape, so 256 consecutive words never straddle two problems.)
+// 256 x 128 image), persistent CTAs that walk the words of all problems in table order, 2,048 words at a time.  After
+// every step the CTA adds its words to the ready counter of the 256-row weight tile they belong to: the GEMM kernel,
+// which starts beside this launch and consumes the tiles in the same order, reads a tile's images as soon as all its
+// words are counted.  (A weight tile has 16 * K words, the last one of a matrix 8 * K: multiples of 2,048 for every
+// valid shape - N a multiple of 128, K of 256 - so a step never straddles two tiles.)
+constexpr int kUnpackChunk = 2048;  // packed words per CTA step: 8 per thread, all loaded before anything is stored
 __global__ void __launch_bounds__(256) group_unpack_kernel(const PrefillItem* __restrict__ items, int count,
                                                            long long total_words, int* __restrict__ ready) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     int i = 0;
-    for (long long chunk = (long long)blockIdx.x * 256; chunk < total_words; chunk += (long long)gridDim.x * 256) {
-        const long long word = chunk + threadIdx.x;
+    for (long long chunk = (long long)blockIdx.x * kUnpackChunk; chunk < total_words; chunk += (long long)gridDim.x * kUnpackChunk) {
         while (i + 1 < count && chunk >= items[i + 1].word_begin) ++i;
         const PrefillItem& p = items[i];
-        const size_t w = (size_t)(word - p.word_begin);
         const int k_tiles = p.K / kTileCols;
-        // position of packed word w (see "Packed weight layout" in bitlinear.h)
-        const size_t tile = w >> 8;
-        const int wo = (int)(w & 255);
-        const int h = wo >> 7, g = (wo >> 4) & 7, t = (wo >> 2) & 3, q = wo & 3;
-        const int n = (int)(tile / k_tiles) * kTileRows + 8 * h + g;
-        const int k0 = (int)(tile % k_tiles) * kTileCols + 64 * t + 16 * q;
-        const uint32_t v = p.packed[w];
-        const int r = n & 255, piece = (k0 & 127) >> 4;
-        const size_t img = (size_t)(n >> 8) * (p.K / 128) + (k0 >> 7);
-        *reinterpret_cast<uint4*>(p.codes + img * 32768 + (size_t)r * 128 + ((piece ^ (r & 7)) << 4)) =
-            make_uint4(v & 0x03030303u, (v >> 2) & 0x03030303u, (v >> 4) & 0x03030303u, (v >> 6) & 0x03030303u);
+        const size_t w0 = (size_t)(chunk - p.word_begin) + threadIdx.x;
+        uint32_t v[kUnpackChunk / 256];
+#pragma unroll
+        for (int u = 0; u < kUnpackChunk / 256; ++u) v[u] = p.packed[w0 + (size_t)u * 256];
+#pragma unroll
+        for (int u = 0; u < kUnpackChunk / 256; ++u) {
+            const size_t w = w0 + (size_t)u * 256;
+            // position of packed word w (see "Packed weight layout" in bitlinear.h)
+            const size_t tile = w >> 8;
+            const int wo = (int)(w & 255);
+            const int h = wo >> 7, g = (wo >> 4) & 7, t = (wo >> 2) & 3, q = wo & 3;
+            const int n = (int)(tile / k_tiles) * kTileRows + 8 * h + g;
+            const int k0 = (int)(tile % k_tiles) * kTileCols + 64 * t + 16 * q;
+            const int r = n & 255, piece = (k0 & 127) >> 4;
+            const size_t img = (size_t)(n >> 8) * (p.K / 128) + (k0 >> 7);
+            *reinterpret_cast<uint4*>(p.codes + img * 32768 + (size_t)r * 128 + ((piece ^ (r & 7)) << 4)) =
+                make_uint4(v[u] & 0x03030303u, (v[u] >> 2) & 0x03030303u, (v[u] >> 4) & 0x03030303u, (v[u] >> 6) & 0x03030303u);
+        }
         __syncthreads();  // every store of the chunk is ordered before the fence and the count below
         if (threadIdx.x == 0) {
             __threadfence();
-            atomicAdd(ready + i, 256);
+            // the step lies inside one 256-row weight tile (16 * K words each)
+            atomicAdd(ready + p.nt_begin + (int)((chunk - p.word_begin) / (16 * (long long)p.K)), kUnpackChunk);
         }
     }
 }
 
 struct GroupLayout {
-    size_t table_off, items_off, ready_off, total;
+    size_t table_off, items_off, ready_off, ready_bytes, total;
     std::vector<size_t> a_off, codes_off, d_off, xsum_off;
 };
 
@@ -99,7 +107,10 @@ GroupLayout group_layout(const bitlinear_problem* problems, const int* idx, int 
     L.items_off = off;
     off = align_up(off + kItemTableBytes, 256);
     L.ready_off = off;
-    off = align_up(off + kMaxGroup * sizeof(int), 256);
+    size_t n_tiles = 0;
+    for (int i = 0; i < n; ++i) n_tiles += (size_t)(problems[idx[i]].N + 255) / 256;
+    L.ready_bytes = align_up(n_tiles * sizeof(int), 256);
+    off += L.ready_bytes;
     for (int i = 0; i < n; ++i) {
         const bitlinear_problem& q = problems[idx[i]];
         L.a_off.push_back(off);
@@ -145,7 +156,7 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
         PrefillItem items[kMaxGroup] = {};
         GemmProblem gp[kMaxGroup] = {};
         long long words = 0;
-        int rows = 0;
+        int rows = 0, nt_total = 0;
         for (int i = 0; i < n; ++i) {
             const bitlinear_problem& q = problems[idx[i]];
             PrefillItem& it = items[i];
@@ -160,6 +171,8 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             it.eps = q.rms_eps;
             it.M = q.M; it.N = q.N; it.K = q.K;
             it.row_begin = rows;
+            it.nt_begin = nt_total;
+            nt_total += (q.N + 255) / 256;
             words += (long long)q.N * q.K / 16;
             // problems that read the same activations (q/k/v, gate/up of a layer) share one quantised copy
             int same = -1;
@@ -179,7 +192,7 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
         }
         PrefillItem* items_dev = reinterpret_cast<PrefillItem*>(base + L.items_off);
         int* ready = reinterpret_cast<int*>(base + L.ready_off);
-        if (cudaMemsetAsync(ready, 0, kMaxGroup * sizeof(int), st) != cudaSuccess ||
+        if (cudaMemsetAsync(ready, 0, L.ready_bytes, st) != cudaSuccess ||
             cudaMemcpyAsync(items_dev, items, sizeof(PrefillItem) * n, cudaMemcpyHostToDevice, st) != cudaSuccess) {
             cudaGetLastError();
             return BITLINEAR_ERR_CUDA;
@@ -201,7 +214,7 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
                     if (cudaGetLastError() != cudaSuccess) return (int)BITLINEAR_ERR_CUDA;
                 }
                 // at most four CTAs per SM, so that the GEMM kernel's CTAs find room beside them
-                const long long chunks = (a.words + 255) / 256;
+                const long long chunks = (a.words + kUnpackChunk - 1) / kUnpackChunk;
                 const unsigned grid = (unsigned)std::min<long long>(chunks, 4LL * a.sm_count);
                 group_unpack_kernel<<<grid, 256, 0, a.st>>>(a.items_dev, a.n, a.words, a.ready);
                 return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
