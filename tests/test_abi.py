@@ -106,6 +106,8 @@ def test_batch_entry_point_host_checks():
     assert lib.bitlinear_forward_batch(None, 2, 0, addr, need, None) == 1
     assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 0, 0, None, 0, None) == 0       # empty batch
     assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 8, addr, need, None) == 5    # unknown flag
+    arr[1].M = 16                      # several tokens: every problem of the call gets 16-row token images of 16 * K bytes
+    assert lib.bitlinear_batch_workspace_bytes(ctypes.addressof(arr), 2) >= 16 * (256 + 512)
     arr[1].M = 17                                                                               # decode sizes only
     assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, addr, 1 << 20, None) == 2
     assert lib.bitlinear_batch_workspace_bytes(ctypes.addressof(arr), 2) == 0
