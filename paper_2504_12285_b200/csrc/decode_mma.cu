@@ -12,7 +12,7 @@
 // (decode_mma_kernel) starts under programmatic dependent launch and streams weights while launch 1 still runs.
 //   producer warps : three warps, three bulk copies each (a thread starts a copy only every few hundred cycles):
 //                    eight packed 16-row blocks x up to four 16x256 tiles (4 KiB each) and the matching slice of
-//                    the token images, into a 4-slot ring of 48 KiB
+//                    the token images, into a 3-slot ring of 48 KiB
 // Tile g of every ring slot belongs to pipeline g (kLanes = 4 pipelines), each with its own unpack group, its own 64
 // tensor-memory columns for the codes, its own MMA-issuing thread and its own partial accumulator (one thread can
 // start a tcgen05.mma only every ~55 cycles whatever its shape, several threads scale; the integer partial sums are
@@ -38,7 +38,7 @@ constexpr int kRows = 128;        // weight rows per work item = tensor-memory l
 constexpr int kItemRb = kRows / kTileRows;
 constexpr int kTok = 16;          // tokens per matmul, padded (UMMA N)
 constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1024 columns)
-constexpr int kSlots = 4;         // ring slots of packed weights + token images
+constexpr int kSlots = 3;         // ring slots of packed weights + token images (see kAStages for why not more)
 constexpr int kLanes = 4;         // pipelines: unpack group + tensor-memory stage + MMA issuer + partial accumulator
 constexpr int kUnpackWarps = 4 * kLanes;  // groups of four (one warp per tensor-memory lane quarter)
 constexpr int kProdWarps = 3, kCopiesPerWarp = 3;  // 8 packed row blocks + the token images
@@ -52,8 +52,14 @@ constexpr uint32_t kAColBase = 2 * kLanes * kTok;                    // after th
 constexpr uint32_t kTmemCols = 512;
 // Stages of unpacked codes in tensor memory, shared by the pipelines: step s of the CTA uses stage s % kAStages.  With
 // more stages than pipelines a pipeline's unpack group does not wait for the pipeline's own previous MMAs.
+// A stage's two barriers are waited on by parity, which is only unambiguous while no waiter is two uses ahead.  A slot
+// is refilled only when every MMA on it has retired, so whoever works on ring slot i knows the MMAs of slots <= i -
+// kSlots to be complete; a stage's uses are kAStages steps apart and a slot holds at most kStepTiles steps, so with
+// 2 * kAStages >= kSlots * kStepTiles the use before the previous one has always retired.  (The issuer also waits for
+// the previous use's MMAs before it waits for the codes, which makes "previous use complete" hold on both barriers.)
 constexpr int kAStages = (int)((kTmemCols - kAColBase) / kAStageCols);  // 6
 static_assert(kAStages >= kLanes, "tensor memory");
+static_assert(2 * kAStages >= kSlots * kStepTiles, "a waiter could be two uses of a stage ahead");
 constexpr int kItemCap = 192;     // work items and matmul descriptors of the CTA kept in shared memory; what does
 constexpr int kProbCap = 48;      // not fit is read from global memory where it is needed (slow, still correct)
 
@@ -372,7 +378,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     if (g < tiles) {
                         const uint32_t step = st_base + (uint32_t)g, stage = step % kAStages, sphase = (step / kAStages) & 1u;
                         const uint32_t a_tmem = tmem_base + kAColBase + stage * kAStageCols;
-                        if (!mbar_wait(afull + 8 * stage, sphase, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag) ||  // the stage's previous use has retired,
+                            !mbar_wait(afull + 8 * stage, sphase, abort_flag)) {        // so this parity means THIS step's codes
+                            ok = false;
+                            break;
+                        }
                         tc_fence_after();
                         const uint64_t b_desc = x_desc + (uint64_t)(slot * (kXSlot >> 4));
 #pragma unroll
