@@ -12,7 +12,7 @@
 // (decode_mma_kernel) starts under programmatic dependent launch and streams weights while launch 1 still runs.
 //   producer warps : three warps, three bulk copies each (a thread starts a copy only every few hundred cycles):
 //                    eight packed 16-row blocks x up to four 16x256 tiles (4 KiB each) and the matching slice of
-//                    the token images, into a 3-slot ring of 48 KiB
+//                    the token images, into a 4-slot ring of 48 KiB
 // Tile g of every ring slot belongs to pipeline g (kLanes = 4 pipelines), each with its own unpack group, its own 64
 // tensor-memory columns for the codes, its own MMA-issuing thread and its own partial accumulator (one thread can
 // start a tcgen05.mma only every ~55 cycles whatever its shape, several threads scale; the integer partial sums are
@@ -38,7 +38,7 @@ constexpr int kRows = 128;        // weight rows per work item = tensor-memory l
 constexpr int kItemRb = kRows / kTileRows;
 constexpr int kTok = 16;          // tokens per matmul, padded (UMMA N)
 constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1024 columns)
-constexpr int kSlots = 3;         // ring slots of packed weights + token images (see kAStages for why not more)
+constexpr int kSlots = 4;         // ring slots of packed weights + token images
 constexpr int kLanes = 4;         // pipelines: unpack group + tensor-memory stage + MMA issuer + partial accumulator
 constexpr int kUnpackWarps = 4 * kLanes;  // groups of four (one warp per tensor-memory lane quarter)
 constexpr int kProdWarps = 3, kCopiesPerWarp = 3;  // 8 packed row blocks + the token images
@@ -49,17 +49,8 @@ constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;  // 32 KiB o
 constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;             // 16 KiB: 8 k-blocks of 16 x 128 token images
 constexpr uint32_t kAStageCols = kTileCols / 4;                      // 64 columns: 256 codes per row, 4 per column
 constexpr uint32_t kAColBase = 2 * kLanes * kTok;                    // after the two buffers of partial accumulators
-constexpr uint32_t kTmemCols = 512;
-// Stages of unpacked codes in tensor memory, shared by the pipelines: step s of the CTA uses stage s % kAStages.  With
-// more stages than pipelines a pipeline's unpack group does not wait for the pipeline's own previous MMAs.
-// A stage's two barriers are waited on by parity, which is only unambiguous while no waiter is two uses ahead.  A slot
-// is refilled only when every MMA on it has retired, so whoever works on ring slot i knows the MMAs of slots <= i -
-// kSlots to be complete; a stage's uses are kAStages steps apart and a slot holds at most kStepTiles steps, so with
-// 2 * kAStages >= kSlots * kStepTiles the use before the previous one has always retired.  (The issuer also waits for
-// the previous use's MMAs before it waits for the codes, which makes "previous use complete" hold on both barriers.)
-constexpr int kAStages = (int)((kTmemCols - kAColBase) / kAStageCols);  // 6
-static_assert(kAStages >= kLanes, "tensor memory");
-static_assert(2 * kAStages >= kSlots * kStepTiles, "a waiter could be two uses of a stage ahead");
+constexpr uint32_t kTmemCols = 512;                                  // power of two >= kAColBase + kLanes * 64
+static_assert(kAColBase + kLanes * kAStageCols <= kTmemCols, "tensor memory");
 constexpr int kItemCap = 192;     // work items and matmul descriptors of the CTA kept in shared memory; what does
 constexpr int kProbCap = 48;      // not fit is read from global memory where it is needed (slow, still correct)
 
@@ -108,7 +99,7 @@ struct alignas(16) SProb {
     void* y;
     int M, N, K, y_dtype;
 };
-constexpr int kNumBars = 3 * kSlots + 2 * kAStages + 4;               // pfull, pempty, xempty; afull, aempty; tfull, tempty
+constexpr int kNumBars = 3 * kSlots + 2 * kLanes + 4;               // pfull, pempty, xempty; afull, aempty; tfull, tempty
 constexpr size_t kBarBytes = 256;                                    // barriers, tensor-memory base, abort flag
 static_assert(kNumBars * 8 + 8 <= kBarBytes, "barrier block");
 constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + kBarBytes + kItemCap * sizeof(int2) + kProbCap * sizeof(SProb);
@@ -218,8 +209,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t p_s = x_s + kSlots * kXSlot;     // [kSlots] packed weights
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSlots * (size_t)(kXSlot + kPackedSlot));
     const uint32_t pfull = smem_u32(bars), pempty = pfull + 8 * kSlots, xempty = pempty + 8 * kSlots;
-    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kAStages;
-    const uint32_t tfull = aempty + 8 * kAStages, tempty = tfull + 16;
+    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kLanes;
+    const uint32_t tfull = aempty + 8 * kLanes, tempty = tfull + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int2* items_s = reinterpret_cast<int2*>(reinterpret_cast<uint8_t*>(bars) + kBarBytes);
@@ -237,7 +228,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             mbar_init(pempty + 8 * b, kUnpackWarps);
             mbar_init(xempty + 8 * b, kLanes);
         }
-        for (int b = 0; b < kAStages; ++b) {
+        for (int b = 0; b < kLanes; ++b) {
             mbar_init(afull + 8 * b, 4);
             mbar_init(aempty + 8 * b, 1);
         }
@@ -310,8 +301,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         // the 256 codes of row r16 = 8h + g of a 16 x 256 tile are 64 consecutive packed bytes at 512h + 64g
         const uint32_t row_off = (uint32_t)rbl * (kStepTiles * kTileBytes) + (uint32_t)(r16 >> 3) * 512u + (uint32_t)(r16 & 7) * 64u +
                                  (uint32_t)g * kTileBytes;
-        const uint32_t a_lane = tmem_base + ((uint32_t)(quarter * 32) << 16) + kAColBase;
-        uint32_t sc_idx = 0, st_base = 0;  // st_base: 256-column steps of the CTA before this slot
+        const uint32_t a_dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + kAColBase + (uint32_t)g * kAStageCols;
+        uint32_t sc_idx = 0, n_own = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
             const int2 item = item_at(it);
@@ -323,10 +314,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 // every warp waits for every slot, also one in which it has no step: a warp can then never be a whole
                 // ring lap ahead of another and arrive twice on pempty in one phase
                 if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
-                const int tiles = min(kStepTiles, k_tiles - t0);
-                if (g < tiles) {
-                    const uint32_t step = st_base + (uint32_t)g, stage = step % kAStages, sphase = (step / kAStages) & 1u;
-                    const uint32_t a_dst = a_lane + stage * kAStageCols;
+                if (g < k_tiles - t0) {
                     uint4 pw[4] = {};
                     if (have_row) {
                         const uint32_t src = p_s + slot * kPackedSlot + row_off;
@@ -338,10 +326,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     // that takes a left shift, which the multiplier pipe executes, and one AND, where a right shift
                     // and an AND would both go to the logic pipe; the epilogue divides by 64.
                     // The first half is expanded BEFORE the wait for the tensor-memory stage (the MMAs of the
-                    // step that used it last may still be running), the second half after the first is stored.
+                    // pipeline's previous step are still reading it), the second half after the first is stored.
                     uint32_t v[32];
                     expand_codes(pw[0], pw[1], v);
-                    if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(aempty + 8 * g, (n_own & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     tmem_st_32x32(a_dst, v);
                     expand_codes(pw[2], pw[3], v);
@@ -349,9 +337,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(afull + 8 * stage);
+                    if (lane == 0) mbar_arrive(afull + 8 * g);
+                    ++n_own;
                 }
-                st_base += (uint32_t)tiles;
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pempty + 8 * slot);
             }
@@ -360,9 +348,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         // ------------------------------------------------------------------ MMA issuers: one pipeline each
         if (lane == 0) {
             const int g = warp - kFirstMmaWarp;
+            const uint32_t a_tmem = tmem_base + kAColBase + (uint32_t)g * kAStageCols;
             // token images of tile g of a slot: k-block kb at 2 KiB * (2g + kb), 32-byte slice k inside it
             const uint64_t x_desc = smem_desc_sw128(x_s) + (uint64_t)((g * 2 * kTok * 128) >> 4);
-            uint32_t sc_idx = 0, st_base = 0, it_idx = 0;
+            uint32_t sc_idx = 0, n_own = 0, it_idx = 0;
             bool ok = true;
             for (int it = item_lo; ok && it < item_hi; ++it, ++it_idx) {
                 const int k_tiles = prob_at(item_at(it).x).K / kTileCols;
@@ -374,24 +363,17 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     const uint32_t slot = sc_idx % kSlots, phase = (sc_idx / kSlots) & 1u;
                     // every issuer waits for every slot, also one in which it has no step (see the unpack warps)
                     if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
-                    const int tiles = min(kStepTiles, k_tiles - t0);
-                    if (g < tiles) {
-                        const uint32_t step = st_base + (uint32_t)g, stage = step % kAStages, sphase = (step / kAStages) & 1u;
-                        const uint32_t a_tmem = tmem_base + kAColBase + stage * kAStageCols;
-                        if (!mbar_wait(aempty + 8 * stage, sphase ^ 1u, abort_flag) ||  // the stage's previous use has retired,
-                            !mbar_wait(afull + 8 * stage, sphase, abort_flag)) {        // so this parity means THIS step's codes
-                            ok = false;
-                            break;
-                        }
+                    if (g < k_tiles - t0) {
+                        if (!mbar_wait(afull + 8 * g, n_own & 1u, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint64_t b_desc = x_desc + (uint64_t)(slot * (kXSlot >> 4));
 #pragma unroll
                         for (int s = 0; s < 8; ++s)
                             umma_i8_ts(d_tmem, a_tmem + 8u * s, b_desc + (uint64_t)((s >> 2) * ((kTok * 128) >> 4) + 2 * (s & 3)),
                                        kIdesc, (uint32_t)(t0 != 0 || s != 0));
-                        umma_commit(aempty + 8 * stage);  // the codes may be overwritten once these MMAs retire
+                        umma_commit(aempty + 8 * g);  // the codes may be overwritten once these MMAs retire
+                        ++n_own;
                     }
-                    st_base += (uint32_t)tiles;
                     umma_commit(xempty + 8 * slot);  // counts kLanes arrivals: every issuer is done with the slot
                 }
                 if (ok) umma_commit(tfull + 8 * buf);
