@@ -192,6 +192,27 @@ def test_batch_full_decode_step_sampled(M):
         assert np.all(np.abs(got - want) <= 1e-6 * np.abs(want)), i
 
 
+def test_batch_many_tiny_problems_overflow_the_descriptor_cache():
+    # 30,000 one-item problems of two tokens: about 203 per CTA, more than the 192 work items and the 48 descriptors
+    # a CTA of the tensor-core decode kernel keeps in shared memory, so the rest is read from global memory
+    N, K, M, count = 16, 256, 2, 30000
+    W = wl.latent_weights(N, K, 900)
+    packed, s_w = bl.bitlinear_pack_weights(W.to(DEV), wl.WEIGHT_EPS)
+    wref = oracle.quantize_weights(W.numpy(), wl.WEIGHT_EPS)
+    xs = wl.activations_normal(M * count, K, 901)
+    xs_dev = xs.to(DEV)
+    ys = torch.full((count, M, N), float("nan"), dtype=torch.float32, device=DEV)
+    items = [(xs_dev[M * i:M * (i + 1)], None, packed, s_w, ys[i]) for i in range(count)]
+    batch = bl.ProblemBatch(items, wl.RMS_EPS)
+    run(batch)
+    ref = oracle.bitlinear_forward(wl.bf16_bits(xs), None, wl.RMS_EPS, wref["wq"], wref["s_w"])  # rows are independent
+    ok = ref["fragile"] == 0
+    got = ys.reshape(M * count, N).cpu().numpy().astype(np.float64)[ok]
+    want = ref["y"].astype(np.float64)[ok]
+    assert ok.mean() > 0.9
+    assert np.all(np.abs(got - want) <= 1e-6 * np.abs(want))
+
+
 # ---- problems of more than 16 tokens in the same entry point: grouped tensor-core path ----
 
 
