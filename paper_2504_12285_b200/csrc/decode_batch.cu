@@ -248,10 +248,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             advance_ld(false);
         }
 
-    // the quantiser launch that precedes this kernel must be complete before its results are read
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-
-    // ---- fill the descriptor table (one warp per problem), then stage the activations ----
+    // ---- fill the descriptor table (one warp per problem) with what does not come from the quantiser launch ----
     for (int i = warp; i < n_tab; i += kStreamWarps) {
         const DevProblem& pr = probs[p_lo + i];
         if (lane == 0) {
@@ -263,25 +260,33 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             e.x_off = 0;
             e.s_w = *pr.s_w;
         }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int off = 0;
+        for (int i = 0; i < n_tab; ++i) {
+            const int bytes = table[i].M * table[i].K;  // a multiple of 256
+            if (off + bytes <= prm.arena_bytes) {
+                table[i].x_off = off;
+                off += bytes;
+            } else {
+                table[i].x_off = -1;  // does not fit: read through L1
+            }
+        }
+    }
+
+    // the quantiser launch that precedes this kernel must be complete before its results are read
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    // ---- scales and code sums of the tokens, then stage the activations ----
+    for (int i = warp; i < n_tab; i += kStreamWarps) {
+        const DevProblem& pr = probs[p_lo + i];
         if (lane < kGemvMaxTokens) {
             table[i].d[lane] = lane < pr.M ? pr.d[lane] : 0.0f;
             table[i].xsum[lane] = lane < pr.M ? pr.xsum[lane] : 0;
         }
     }
-    __syncthreads();
     {
-        if (threadIdx.x == 0) {
-            int off = 0;
-            for (int i = 0; i < n_tab; ++i) {
-                const int bytes = table[i].M * table[i].K;  // a multiple of 256
-                if (off + bytes <= prm.arena_bytes) {
-                    table[i].x_off = off;
-                    off += bytes;
-                } else {
-                    table[i].x_off = -1;  // does not fit: read through L1
-                }
-            }
-        }
         __syncthreads();
         const uint32_t arena_s = smem_u32(arena);
         for (int i = 0; i < n_tab; ++i) {
