@@ -194,9 +194,9 @@ def run_ours(args):
                 "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                 "frac": round(achieved / peaks["hbm_gbs"], 4), "algorithmic_bytes_per_launch": packed_bytes,
                 "avg_launch_us": round(stream_s * 1e6, 2),
-                # dram__bytes_read.sum + dram__bytes_write.sum of this kernel on 10 of the 30 layers (173.96 MB + 4.62 MB,
+                # dram__bytes_read.sum + dram__bytes_write.sum of this kernel on 10 of the 30 layers (173.95 MB + 4.08 MB,
                 # profiles/decode_stream_10layers_m1.md), times 3: it streams every packed byte once
-                "traffic": 3 * (173955072 + 4621056)}
+                "traffic": 3 * (173954816 + 4077312)}
 
     # ---- the same 210 forwards as separate bitlinear_forward calls (two launches each), for comparison ----
     ws_call = torch.empty(max(bl.bitlinear_workspace_bytes(M, n, k) for _, n, k in wl.LAYER_SHAPES), dtype=torch.uint8,
