@@ -9,14 +9,12 @@
 //             stream kernel reads, see quant_row).
 //   launch 2  decode_stream_kernel : one persistent CTA of 16 warps per SM.  The work list is every
 //             block of 16 weight rows of every problem; each CTA owns a contiguous, byte-balanced
-//             range of it.  A row block belongs to ONE group of G warps (G = 1 for up to four tokens;
-//             each warp of a group takes up to four tokens), so 16/G row blocks are in progress per
-//             CTA and no partial sum ever crosses a warp.  Each group runs its own pipeline: one
-//             thread issues a linear bulk copy (cp.async.bulk, a few contiguous 16x256 tiles) into one
-//             of the group's two shared-memory slots; its warps wait on that slot's mbarrier, multiply,
-//             and the slot is refilled once they have all read it - across row-block and matrix
-//             boundaries, so HBM requests are always in flight (with G = 1: 16 issuing threads, ~80 KiB
-//             in flight per SM, and nothing is handed from warp to warp).
+//             range of it.  A row block belongs to ONE warp, so 16 row blocks are in progress per CTA
+//             and no partial sum ever crosses a warp.  Each warp runs its own pipeline: its lane 0
+//             issues a linear bulk copy (cp.async.bulk, a few contiguous 16x256 tiles) into one of the
+//             warp's two shared-memory slots; the warp waits on that slot's mbarrier, multiplies, and
+//             refills the slot - across row-block and matrix boundaries, so HBM requests are always in
+//             flight (16 issuing threads, ~160 KiB in flight per SM, nothing is handed from warp to warp).
 //             Before the stream starts the CTA copies the descriptors of the few problems its range
 //             touches, and their quantised activations, into shared memory once.
 //             Unpack: word & (0x03030303 << 2j) is 4^j x the codes of four consecutive columns, fed
@@ -65,12 +63,10 @@ __device__ __forceinline__ bool plan_matches(const PlanHeader* h, int count, int
 
 constexpr int kStreamWarps = 16;
 constexpr int kStreamThreads = kStreamWarps * 32;
-constexpr int kRing = 2;  // chunk slots per group of warps that share a row block
+constexpr int kRing = 2;  // chunk slots per warp
 constexpr int kBatchMaxK = 8192;
 constexpr size_t kBarBytes = (size_t)kStreamWarps * kRing * 2 * 8 + 128;  // full + empty barriers, abort flag
-constexpr size_t ring_bytes(int chunk_tiles, int groups) {
-    return (size_t)(kStreamWarps / groups) * kRing * chunk_tiles * kTileBytes + kBarBytes;
-}
+constexpr size_t ring_bytes(int chunk_tiles) { return (size_t)kStreamWarps * kRing * chunk_tiles * kTileBytes + kBarBytes; }
 
 // ------------------------------------------------------------------------------------ launch 1
 
@@ -116,7 +112,6 @@ struct StreamParams {
     const int4* cta_range;  // [grid] {first row block, one past the last, first problem, last problem} of each CTA
     const PlanHeader* hdr;
     int count, total_rb, rows;
-    int groups;     // G: warps that share a row block, each taking MT tokens
     int table_cap;  // problems of a CTA whose descriptors are cached in shared memory
     int arena_bytes;  // shared memory available for staged activations
     int* status_word;
@@ -131,8 +126,8 @@ struct alignas(16) SProb {
     int x_off;  // byte offset of token 0's codes in the CTA's activation arena
     float s_w;
     int pad[3];
-    float d[kGemvMaxTokens];
-    int xsum[kGemvMaxTokens];
+    float d;   // the token's scale
+    int xsum;  // and code sum
 };
 
 // Position of a warp in its sequence of weight chunks: row blocks rb, rb + par, ... of the CTA's range,
@@ -154,17 +149,16 @@ struct ChunkCursor {
     }
 };
 
-// MT = tokens per warp (1 or 4).  kChunkTiles = 16x256 tiles (1 KiB each) per bulk copy at most.
+// One token per problem.  kChunkTiles = 16x256 tiles (1 KiB each) per bulk copy at most.
 // The quantised activations of the problems the CTA touches are staged in shared memory once, as far as the arena
 // reaches; those of the remaining problems are read through L1, which is slower.
-template <int MT, int kChunkTiles>
+template <int kChunkTiles>
 __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const StreamParams prm) {
     extern __shared__ __align__(128) uint8_t smem[];
-    // [ring: (16 / G) row-block lanes x kRing slots][full barriers][empty barriers][abort flag][descriptor table]
+    // [ring: 16 warps x kRing slots][full barriers][empty barriers][abort flag][descriptor table]
     // [activation arena]
     constexpr uint32_t kSlotBytes = kChunkTiles * kTileBytes;
-    const int G = prm.groups;
-    const int par = kStreamWarps / G;  // row blocks in progress at a time in this CTA
+    constexpr int par = kStreamWarps;  // row blocks in progress at a time in this CTA: one per warp
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)par * kRing * kSlotBytes);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStreamWarps * kRing);
     SProb* table = reinterpret_cast<SProb*>(reinterpret_cast<uint8_t*>(bars) + kBarBytes);
@@ -179,7 +173,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (lane == 0 && warp < par) {  // warp i sets up the barriers of row-block lane i
         for (int r = 0; r < kRing; ++r) {
             mbar_init(smem_u32(bars + warp * kRing + r), 1);                          // full: the copy landed
-            mbar_init(smem_u32(bars + kStreamWarps * kRing + warp * kRing + r), G);   // empty: all G warps have read it
+            mbar_init(smem_u32(bars + kStreamWarps * kRing + warp * kRing + r), 1);   // empty: the warp has read it
         }
         if (warp == 0) *abort_flag = 0;
         mbar_init_fence();
@@ -190,13 +184,13 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     const int n_local = rb_lo < rb_hi ? range.w - p_lo + 1 : 0;
     const int n_tab = n_local < prm.table_cap ? n_local : prm.table_cap;
     const DevProblem* probs = prm.probs;
-    const int rl = warp / G, tg = warp - rl * G;  // the row-block lane this warp works on, and its token group
+    const int rl = warp;  // the row-block lane this warp works on
     const bool mine = rl < par && rb_lo + rl < rb_hi;
     const int g = lane >> 2, t = lane & 3;
     const uint32_t ring_s = smem_u32(smem) + (uint32_t)rl * kRing * kSlotBytes;
     const uint32_t bar_s = smem_u32(bars + rl * kRing);                            // full barriers of this lane
     const uint32_t ebar_s = smem_u32(bars + kStreamWarps * kRing + rl * kRing);    // empty barriers
-    const bool issuer = tg == 0 && lane == 0;  // the one thread of the group that issues its copies
+    const bool issuer = lane == 0;  // the thread of the warp that issues its copies
 
     // descriptor of the next problem that holds row block c.rb: from the shared-memory table when it is there
     auto enter = [&](ChunkCursor& c) {
@@ -216,7 +210,6 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     };
 
     // ---- start the weight stream before anything else: the first chunks come from one problem ----
-    // The warps of a group share the lane's ring: one thread issues, every warp of the group reads.
     ChunkCursor ld;  // where the next copy comes from
     ld.rb = rb_lo + rl; ld.c = 0; ld.p = p_lo;
     ld.rb_begin = 0; ld.rb_end = 0; ld.k_tiles = 1; ld.nc = 1; ld.ct = 1; ld.base = nullptr;
@@ -281,9 +274,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     // ---- scales and code sums of the tokens, then stage the activations ----
     for (int i = warp; i < n_tab; i += kStreamWarps) {
         const DevProblem& pr = probs[p_lo + i];
-        if (lane < kGemvMaxTokens) {
-            table[i].d[lane] = lane < pr.M ? pr.d[lane] : 0.0f;
-            table[i].xsum[lane] = lane < pr.M ? pr.xsum[lane] : 0;
+        if (lane == 0) {
+            table[i].d = pr.d[0];
+            table[i].xsum = pr.xsum[0];
         }
     }
     {
@@ -312,47 +305,38 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             }
 
         // per-problem state of the arithmetic side
-        int M = 0, N = 0, y_dtype = 0, xs_lane = 0;
+        int y_dtype = 0, xs = 0;
         void* y = nullptr;
-        float s_w = 0.0f, d_lane = 0.0f;
-        bool active = false, x_staged = false;
-        const int8_t* xrow_g[MT];  // token rows in global memory
-        uint32_t xrow_s[MT];       // token rows in the shared-memory arena (when staged)
+        float s_w = 0.0f, d = 0.0f;
+        bool x_staged = false;
+        const int8_t* xrow_g = nullptr;  // the token's codes in global memory
+        uint32_t xrow_s = 0;             // and in the shared-memory arena (when staged)
         auto load_problem_state = [&]() {
             const int i = cp.p - p_lo;
-            const int my_tok = tg * MT + (MT == 1 ? 0 : t);  // lane t finishes token tg*MT + t
-            int K = 0, x_off = -1;
+            int x_off = -1;
             const int8_t* xq = nullptr;
             if (i < n_tab) {
                 const SProb& e = table[i];
-                M = e.M; N = e.N; y_dtype = e.y_dtype; y = e.y; s_w = e.s_w; K = e.K; x_off = e.x_off; xq = e.xq;
-                d_lane = my_tok < M ? e.d[my_tok] : 0.0f;
-                xs_lane = my_tok < M ? e.xsum[my_tok] : 0;
+                y_dtype = e.y_dtype; y = e.y; s_w = e.s_w; x_off = e.x_off; xq = e.xq;
+                d = e.d;
+                xs = e.xsum;
             } else {
                 const DevProblem& pr = probs[cp.p];
-                M = pr.M; N = pr.N; y_dtype = pr.y_dtype; y = pr.y; s_w = *pr.s_w; K = pr.K; xq = pr.xq;
-                d_lane = my_tok < M ? pr.d[my_tok] : 0.0f;
-                xs_lane = my_tok < M ? pr.xsum[my_tok] : 0;
+                y_dtype = pr.y_dtype; y = pr.y; s_w = *pr.s_w; xq = pr.xq;
+                d = pr.d[0];
+                xs = pr.xsum[0];
             }
-            active = tg * MT < M;  // warp-uniform: this token group holds real tokens
             x_staged = x_off >= 0;
-#pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                int tok = tg * MT + m;
-                if (tok > M - 1) tok = M - 1;  // padding tokens re-read a real row; their sums are dropped
-                xrow_g[m] = xq + (size_t)tok * K + t * 16;
-                xrow_s[m] = smem_u32(arena) + (uint32_t)((x_staged ? x_off : 0) + tok * K + t * 16);
-            }
+            xrow_g = xq + t * 16;
+            xrow_s = smem_u32(arena) + (uint32_t)((x_staged ? x_off : 0) + t * 16);
         };
         load_problem_state();
 
-        int acc[2][4][MT];
+        int acc[2][4];
 #pragma unroll
         for (int h = 0; h < 2; ++h)
 #pragma unroll
-            for (int j = 0; j < 4; ++j)
-#pragma unroll
-                for (int m = 0; m < MT; ++m) acc[h][j][m] = 0;
+            for (int j = 0; j < 4; ++j) acc[h][j] = 0;
 
         uint32_t n_chunk = 0;  // chunks consumed: slot = n_chunk % kRing, phase = (n_chunk / kRing) & 1
         bool ok = true;
@@ -369,39 +353,29 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                     const uint4 w0v = lds128(wa), w1v = lds128(wa + 512);
                     const uint32_t w0[4] = {w0v.x, w0v.y, w0v.z, w0v.w};
                     const uint32_t w1[4] = {w1v.x, w1v.y, w1v.z, w1v.w};
-                    // the token rows are stored with the four 16-byte pieces of each lane's 64 columns interleaved
+                    // the token's codes are stored with the four 16-byte pieces of each lane's 64 columns interleaved
                     // (piece q of lane t at 64q + 16t inside the tile), so the four t lanes read 64 contiguous bytes
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        uint32_t xw[MT][4];
-#pragma unroll
-                        for (int m = 0; m < MT; ++m) {
-                            uint4 v;
-                            if (XS) v = lds128(xrow_s[m] + xo + 64u * q);
-                            else v = *reinterpret_cast<const uint4*>(xrow_g[m] + xo + 64 * q);
-                            xw[m][0] = v.x; xw[m][1] = v.y; xw[m][2] = v.z; xw[m][3] = v.w;
-                        }
+                        uint4 v;
+                        if (XS) v = lds128(xrow_s + xo + 64u * q);
+                        else v = *reinterpret_cast<const uint4*>(xrow_g + xo + 64 * q);
+                        const uint32_t xw[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
                         for (int j = 0; j < 4; ++j) {
                             const uint32_t mask = 0x03030303u << (2 * j);
-                            const uint32_t a0 = w0[q] & mask, a1 = w1[q] & mask;
-#pragma unroll
-                            for (int m = 0; m < MT; ++m) {
-                                acc[0][j][m] = dp4a_u8_s8(a0, xw[m][j], acc[0][j][m]);
-                                acc[1][j][m] = dp4a_u8_s8(a1, xw[m][j], acc[1][j][m]);
-                            }
+                            acc[0][j] = dp4a_u8_s8(w0[q] & mask, xw[j], acc[0][j]);
+                            acc[1][j] = dp4a_u8_s8(w1[q] & mask, xw[j], acc[1][j]);
                         }
                     }
                 }
             };
-            if (active) {
-                if (x_staged) run_tiles(std::true_type{});
-                else run_tiles(std::false_type{});
-            }
+            if (x_staged) run_tiles(std::true_type{});
+            else run_tiles(std::false_type{});
             __syncwarp();  // every lane of this warp has read the slot
             if (lane == 0) mbar_arrive(ebar_s + 8u * slot);
             if (ld_valid) {
-                // refill once all G warps of the group have read it
+                // refill the slot that has just been read
                 if (issuer && mbar_wait(ebar_s + 8u * slot, phase, abort_flag)) issue((int)slot);
                 advance_ld(true);
             }
@@ -409,36 +383,27 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             if (++cp.c == cp.nc) {
                 // ---- end of a row block: fold the four scales (accumulator j holds 4^j x its share), the four
                 //      column lanes, subtract the code offset, dequantise, store ----
-                if (active) {
-                    int v[2][MT];
+                int v[2];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                for (int h = 0; h < 2; ++h) {
+                    // 64 x the sum: ((a0*4 + a1)*4 + a2)*4 + a3; |sum| <= 254*K/4 per lane: no overflow for K <= 8192
+                    int sum = acc[h][0] * 4 + acc[h][1];
+                    sum = sum * 4 + acc[h][2];
+                    sum = sum * 4 + acc[h][3];
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                    sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                    v[h] = sum >> 6;  // exact: a multiple of 64
 #pragma unroll
-                        for (int m = 0; m < MT; ++m) {
-                            // 64 x the sum: ((a0*4 + a1)*4 + a2)*4 + a3; |sum| <= 254*K/4 per lane: no overflow for K <= 8192
-                            int sum = acc[h][0][m] * 4 + acc[h][1][m];
-                            sum = sum * 4 + acc[h][2][m];
-                            sum = sum * 4 + acc[h][3][m];
-                            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-                            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-                            v[h][m] = sum >> 6;  // exact: a multiple of 64
-#pragma unroll
-                            for (int j = 0; j < 4; ++j) acc[h][j][m] = 0;
-                        }
+                    for (int j = 0; j < 4; ++j) acc[h][j] = 0;
+                }
+                if (t == 0) {
                     const int n0 = (cp.rb - cp.rb_begin) * kTileRows + g;
-                    const int tok = tg * MT + (MT == 1 ? 0 : t);
-                    if (tok < M && (MT > 1 || t == 0)) {
 #pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            int sel = v[h][0];
-#pragma unroll
-                            for (int m = 1; m < MT; ++m) sel = (t == m) ? v[h][m] : sel;
-                            const int total = sel - xs_lane;
-                            const float val = __fmul_rn(__fmul_rn((float)total, s_w), d_lane);
-                            const size_t idx = (size_t)tok * N + n0 + 8 * h;
-                            if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
-                            else reinterpret_cast<float*>(y)[idx] = val;
-                        }
+                    for (int h = 0; h < 2; ++h) {
+                        const float val = __fmul_rn(__fmul_rn((float)(v[h] - xs), s_w), d);
+                        const size_t idx = (size_t)(n0 + 8 * h);
+                        if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
+                        else reinterpret_cast<float*>(y)[idx] = val;
                     }
                 }
                 cp.c = 0;
@@ -456,9 +421,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (*abort_flag && threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
 }
 
-template <int MT, int kChunkTiles>
+template <int kChunkTiles>
 cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<MT, kChunkTiles>,
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<kChunkTiles>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // programmatic dependent launch: the kernel may begin (barrier set-up, first weight copies) while the quantiser
@@ -473,7 +438,7 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<MT, kChunkTiles>, prm);
+    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<kChunkTiles>, prm);
 }
 
 struct PlanLayout {
@@ -647,9 +612,8 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     }
     // shared memory: chunk ring + descriptor table + activation arena; activations that do not fit the arena are read
     // through L1 instead, and only as many descriptors as fit a quarter of the space are cached
-    const int chunk_tiles = 5;
-    const int groups = 1;  // one token per problem here: every warp runs its own pipeline
-    const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles, groups) - 128;
+    constexpr int chunk_tiles = 5;
+    const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles) - 128;
     if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
     if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
     arena_max &= ~(size_t)255;
@@ -694,12 +658,10 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.total_rb = total_rb;
     prm.rows = (int)rows;
     prm.status_word = device_status_word();
-    prm.groups = groups;
     prm.table_cap = table_cap;
     prm.arena_bytes = (int)arena_max;
-    const size_t smem = ring_bytes(chunk_tiles, groups) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
-    cudaError_t e;
-    e = launch_stream<1, 5>(prm, grid, smem, st);
+    const size_t smem = ring_bytes(chunk_tiles) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
+    const cudaError_t e = launch_stream<chunk_tiles>(prm, grid, smem, st);
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
