@@ -68,6 +68,10 @@ struct GemmGroupHeader {
     // whose codes have been written; the kernel runs beside the expansion launch and reads that tile only once the
     // count has reached rows_in_tile * K / 16
     const int* ready;
+    // CTA-pair kernel: 1 if the launch right before it is the quantiser, whose results (token images, scales, code
+    // sums) it must wait for with griddepcontrol.wait; 0 if it is the expansion launch, which `ready` covers
+    int wait_primary;
+    int pad;
 };
 // layout of the uploaded group table: GemmGroupHeader, then count x GemmProblem
 constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof(GemmProblem);
@@ -81,7 +85,7 @@ constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof
 typedef int (*GemmBeforeKernel)(void* ctx);
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev, cudaStream_t st,
                 const void* region_base = nullptr, size_t region_bytes = 0, const int* ready = nullptr,
-                GemmBeforeKernel before = nullptr, void* before_ctx = nullptr);
+                GemmBeforeKernel before = nullptr, void* before_ctx = nullptr, bool wait_primary = false);
 size_t gemm_codes_bytes(int N, int K);
 size_t gemm_a_tiles_bytes(int M, int K);
 

@@ -501,6 +501,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
             uint32_t stage = 0, phase = 0;
             bool ok = true;
             int ready_idx = -1;  // last weight tile whose codes are known to be complete
+            if (hdr.wait_primary) asm volatile("griddepcontrol.wait;" ::: "memory");  // token images: quantiser launch
             for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
                 const GemmProblem& p = walk.find(tile);
                 const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
@@ -573,6 +574,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
         const uint32_t stage_s = smem_u32(smem + (size_t)P_STAGES * P_STAGE_BYTES + 256) + (uint32_t)quad * STAGE_OUT_BYTES;
         bool ok = true;
         int iter = 0;
+        if (hdr.wait_primary) asm volatile("griddepcontrol.wait;" ::: "memory");  // scales, code sums: quantiser launch
         for (int tile = pair; ok && tile < total_tiles; tile += n_pairs, ++iter) {
             const GemmProblem& p = walk.find(tile);
             const int lt = tile - p.tile_begin, mt = lt % p.m_tiles, nt = lt / p.m_tiles;
@@ -658,7 +660,7 @@ bool make_map_rows128(CUtensorMap* map, const void* base, size_t bytes) {
 
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev,
                 cudaStream_t st, const void* region_base, size_t region_bytes, const int* ready, GemmBeforeKernel before,
-                void* before_ctx) {
+                void* before_ctx, bool wait_primary) {
     static std::once_flag attr_once;
     static cudaError_t attr_err = cudaSuccess;
     static int sm_count = 0;
@@ -696,6 +698,7 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     hdr->total_tiles = tiles;
     hdr->region_base = reinterpret_cast<unsigned long long>(region_base);
     hdr->ready = pairs ? ready : nullptr;
+    hdr->wait_primary = (pairs && ready != nullptr && wait_primary) ? 1 : 0;
     if (cudaMemcpyAsync(table_dev, host, kGroupTableBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;

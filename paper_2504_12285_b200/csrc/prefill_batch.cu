@@ -3,15 +3,16 @@
 // the 8-bit activations; here the expansion and the activation quantiser write directly the shared-memory images of
 // the tensor-core kernel's tiles, and one persistent kernel runs the tiles of every matmul of the group.)
 //
-//   launch 1  group_quant_warp_kernel : one warp per token - fused RMSNorm + absmax int8 quantiser; codes go into
+//   launch 1  group_unpack_kernel : packed 2-bit weights -> byte codes in 256 x 128 tile images, with a count of
+//                                   finished words per 256-row weight tile.
+//   launch 2  group_quant_warp_kernel : one warp per token - fused RMSNorm + absmax int8 quantiser; codes go into
 //                                   128 x 128 tile images (128-byte swizzle) of the activation operand.  Problems
-//                                   that read the same activations share one quantised copy.
-//   launch 2  group_unpack_kernel : packed 2-bit weights -> byte codes in 256 x 128 tile images, with a count of
-//                                   finished words per problem.
+//                                   that read the same activations share one quantised copy.  Starts as a
+//                                   programmatic dependent of launch 1 and runs beside it (no shared data).
 //   launch 3  gemm_i8_pair_kernel : every tile of every matmul on CTA pairs (gemm_i8_kernel<true> when the SMs do not
-//                                   pair up), operands fetched as whole tile images.  The pair kernel starts
-//                                   beside launch 2 (programmatic dependent launch) and begins a problem when
-//                                   its word count is complete.
+//                                   pair up), operands fetched as whole tile images.  The pair kernel is a
+//                                   programmatic dependent too: it waits for launch 2 as a whole
+//                                   (griddepcontrol.wait) and for launch 1 tile by tile (the word counts).
 // Problems are ordered by decreasing K so that the long tiles are scheduled first and the tail is made of short ones.
 #include <algorithm>
 #include <vector>
@@ -41,6 +42,9 @@ constexpr size_t kItemTableBytes = kMaxGroup * sizeof(PrefillItem);
 // One warp per token, eight tokens per CTA.
 __global__ void __launch_bounds__(kQuantThreads) group_quant_warp_kernel(const PrefillItem* __restrict__ items, int count,
                                                                          int rows) {
+    // This launch runs beside the expansion launch before it (it reads nothing of it), and the GEMM launch after it
+    // may start: it waits for this grid with griddepcontrol.wait before it reads anything written here.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int row = blockIdx.x * kQuantWarps + (threadIdx.x >> 5);
     if (row >= rows) return;
     int i = 0;
@@ -208,20 +212,31 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             cudaStream_t st;
             static int run(void* ctx) {
                 const Launches& a = *static_cast<const Launches*>(ctx);
-                if (!a.skip_quant) {
-                    const unsigned blocks = (unsigned)((a.rows + kQuantWarps - 1) / kQuantWarps);
-                    group_quant_warp_kernel<<<blocks, kQuantThreads, 0, a.st>>>(a.items_dev, a.n, a.rows);
-                    if (cudaGetLastError() != cudaSuccess) return (int)BITLINEAR_ERR_CUDA;
-                }
-                // at most four CTAs per SM, so that the GEMM kernel's CTAs find room beside them
+                // the expansion first (at most four CTAs per SM, so that the other kernels find room beside them) ...
                 const long long chunks = (a.words + kUnpackChunk - 1) / kUnpackChunk;
                 const unsigned grid = (unsigned)std::min<long long>(chunks, 4LL * a.sm_count);
                 group_unpack_kernel<<<grid, 256, 0, a.st>>>(a.items_dev, a.n, a.words, a.ready);
-                return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
+                if (cudaGetLastError() != cudaSuccess) return (int)BITLINEAR_ERR_CUDA;
+                if (a.skip_quant) return (int)BITLINEAR_OK;
+                // ... then the quantiser as its programmatic dependent: the two share no data and run side by side
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3((unsigned)((a.rows + kQuantWarps - 1) / kQuantWarps));
+                cfg.blockDim = dim3(kQuantThreads);
+                cfg.stream = a.st;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                attr[0].val.programmaticStreamSerializationAllowed = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                if (cudaLaunchKernelEx(&cfg, group_quant_warp_kernel, a.items_dev, a.n, a.rows) != cudaSuccess) {
+                    cudaGetLastError();
+                    return (int)BITLINEAR_ERR_CUDA;
+                }
+                return (int)BITLINEAR_OK;
             }
         } launches = {items_dev, ready, n, rows, sm_count, words, skip_quant, st};
         const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st, base, L.total, ready,
-                                   &Launches::run, &launches);
+                                   &Launches::run, &launches, /*wait_primary=*/!skip_quant);
         if (rc != BITLINEAR_OK) return rc;
     }
     return BITLINEAR_OK;
