@@ -391,7 +391,7 @@ def run_prefill(bl, dev, pool, gains, peaks, reps):
         t_fwd_total += fw_s
         ops_total += ops
         del xs, ys, quant
-    # ---- the 7 matmuls of a layer as ONE grouped call (3 launches: quantise, unpack, every tile of every matmul) ----
+    # ---- the 7 matmuls of a layer as ONE grouped call (3 launches: unpack, quantise beside it, every tile of every matmul) ----
     group_sets = []
     shared_input = {"k": "q", "v": "q", "up": "gate"}  # as in the layer: q/k/v read one tensor, gate/up another
     for j in range(3):
@@ -412,7 +412,7 @@ def run_prefill(bl, dev, pool, gains, peaks, reps):
                            for j in range(n_calls)], flush.zero_)[3:]
     gm_s = statistics.median(t_gm) / 1e3  # activations of the last full call stay quantised: unpack + GEMM only
     grouped = {"api": "bitlinear_forward_batch on the 7 shapes of a layer at M=2048, q/k/v and gate/up sharing their input "
-                      "(3 launches: quantiser, unpack, every tile of every matmul)",
+                      "(3 launches: unpack, quantiser beside it, every tile of every matmul following the unpack tile by tile)",
                "forward_us_per_layer": round(g_s * 1e6, 2), "forward_tops": round(ops_total / g_s / 1e12, 1),
                "forward_frac": round(ops_total / g_s / 1e12 / int8_peak, 4),
                "matmul_us_per_layer": round(gm_s * 1e6, 2), "matmul_tops": round(ops_total / gm_s / 1e12, 1),
