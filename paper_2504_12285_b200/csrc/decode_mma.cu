@@ -1,4 +1,4 @@
-// Batched decode for 5 to 16 tokens per matmul on the tensor cores.
+// Batched decode for 2 to 16 tokens per matmul on the tensor cores.
 // (Paper Section 5.1: packed weights are loaded from HBM into shared memory and unpacked right before the product
 // with the 8-bit activations.  With more than a few tokens the dot-product-of-four kernel is bound by its arithmetic
 // - one instruction per token per four weights - so here the product runs on tcgen05:
@@ -9,7 +9,8 @@
 //
 // One persistent CTA per SM owns a contiguous, byte-balanced range of work items (128 weight rows of one matmul).
 // Launch 1 (mma_quant_kernel, one warp per token) writes the quantised tokens as 16-row tile images; launch 2
-// (decode_mma_kernel) starts under programmatic dependent launch and streams weights while launch 1 still runs.
+// (decode_mma_kernel) is its programmatic dependent: only the threads that read launch 1's results wait for it, so
+// where an SM has room for a CTA of launch 2 beside launch 1 (it needs almost all registers) the weights already flow.
 //   producer warps : three warps, three bulk copies each (a thread starts a copy only every few hundred cycles):
 //                    eight packed 16-row blocks x up to four 16x256 tiles (4 KiB each) and the matching slice of
 //                    the token images, into a 4-slot ring of 48 KiB
