@@ -167,12 +167,16 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 // D = s32, A = u8 (64 x weight code, tensor memory), B = s8 (activations, K-major shared memory), M = 128, N = 16.
 constexpr uint32_t kIdesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
 
-// One warp per token, eight tokens per CTA: few enough CTAs that all are resident at once, so the launch_dependents
-// below releases the weight-streaming kernel right away and the two overlap.
+// kQuantGroupWarps warps per token: there are at most a few thousand tokens here, and with one warp per token a
+// 6,912-element token is a serial chain of thousands of instructions for its warp while most of the GPU idles.
+// (Four warps per token while that still fits one wave of CTAs, two beyond.)
+template <int kQuantGroupWarps>
 __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeader* __restrict__ hdr,
                                                                   const MmaProblem* __restrict__ probs,
                                                                   const int* __restrict__ row_prob, int count, int total_items,
                                                                   int grid, int rows, int* status_word) {
+    constexpr int kQuantGroups = kQuantWarps / kQuantGroupWarps;  // tokens per CTA
+    __shared__ GroupReduceSmem sm[kQuantGroups];
     // the kernel that follows may start now: it fetches weights first and waits for this grid before it reads
     // anything written here (programmatic dependent launch)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -180,11 +184,13 @@ __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeade
         if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
         return;
     }
-    const int row = blockIdx.x * kQuantWarps + (threadIdx.x >> 5);
-    if (row >= rows) return;
+    const int group = threadIdx.x / (32 * kQuantGroupWarps);
+    const int row = blockIdx.x * kQuantGroups + group;
+    if (row >= rows) return;  // the whole group leaves: nobody is left waiting at its barrier
     const MmaProblem& p = probs[row_prob[row]];
     const int m = row - p.row_begin;
-    quant_row_warp<3>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m, p.xsum_out + m, m & 7);
+    quant_row_group<3, kQuantGroupWarps>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m,
+                                         p.xsum_out + m, sm[group], 1 + group, m & 7);
 }
 
 // 2 x 16 packed bytes (128 codes of one weight row) -> 32 tensor-memory columns of 64 x code.
@@ -588,8 +594,10 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
     // ---- launch 1: quantise every token into the 16-row tile images ----
     if (!(flags & BITLINEAR_BATCH_REUSE_ACT)) {
         const int* rp = reinterpret_cast<const int*>(base + L.row_prob_off);
-        mma_quant_kernel<<<(unsigned)((rows + kQuantWarps - 1) / kQuantWarps), kQuantThreads, 0, st>>>(hdr, probs_dev, rp, n_prob,
-                                                                                                   total_items, grid, rows, sw);
+        if (rows <= 2 * 8 * sm_count)  // two tokens per CTA, eight CTAs per SM
+            mma_quant_kernel<4><<<(unsigned)((rows + 1) / 2), kQuantThreads, 0, st>>>(hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
+        else
+            mma_quant_kernel<2><<<(unsigned)((rows + 3) / 4), kQuantThreads, 0, st>>>(hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
 

@@ -254,4 +254,109 @@ __device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__
     }
 }
 
+// WARPS warps per row (WARPS = 2 or 4; the group's threads are 32 * WARPS consecutive threads of the CTA): for calls
+// with few rows, where one warp per row leaves the GPU mostly idle and a long row is a long serial chain for its warp.
+// Same arithmetic and the same three passes as quant_row_warp; the partial results of the warps meet in shared memory
+// behind a named barrier of the group (bar_id, 1 .. 15, one per group of the CTA).
+struct GroupReduceSmem {
+    double sq[4];
+    float mx[4];
+    int sum[4];
+    float r;
+};
+
+template <int LAYOUT, int WARPS>
+__device__ __forceinline__ void quant_row_group(const __nv_bfloat16* __restrict__ x_row,
+                                                const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                                int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                                int32_t* __restrict__ xsum_out, GroupReduceSmem& sm, int bar_id, int swz = 0) {
+    constexpr int T = 32 * WARPS;
+    const int n_vec = K >> 3;
+    const int gt = threadIdx.x % T, w = gt >> 5, lane = gt & 31;
+    const uint4* xrow = reinterpret_cast<const uint4*>(x_row);
+    const uint4* grow = reinterpret_cast<const uint4*>(gain);
+    auto group_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(T) : "memory"); };
+    double sq = 0.0;
+#pragma unroll 4
+    for (int v = gt; v < n_vec; v += T) {
+        float f[8];
+        unpack_bf16x8(xrow[v], f);
+        sq += sum_squares8(f);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if (lane == 0) sm.sq[w] = sq;
+    group_sync();
+    if (gt == 0) {
+        double S = 0.0;
+#pragma unroll
+        for (int i = 0; i < WARPS; ++i) S += sm.sq[i];
+        sm.r = (float)(1.0 / sqrt(S / (double)K + (double)eps));  // one thread does the fp64 divide and root
+    }
+    group_sync();
+    const float r = sm.r;
+
+    float amax = 0.0f;
+#pragma unroll 2
+    for (int v = gt; v < n_vec; v += T) {
+        float f[8], g[8];
+        unpack_bf16x8(xrow[v], f);
+        if (gain != nullptr) {
+            unpack_bf16x8(grow[v], g);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = 1.0f;
+        }
+#pragma unroll
+        for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(__fmul_rn(__fmul_rn(f[e], r), g[e])));
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if (lane == 0) sm.mx[w] = amax;
+    group_sync();
+    float a = 1e-5f;
+#pragma unroll
+    for (int i = 0; i < WARPS; ++i) a = fmaxf(a, sm.mx[i]);
+    const float s = __fdiv_rn(127.0f, a);
+
+    int csum = 0;
+    uint2* qrow = reinterpret_cast<uint2*>(xq_row);
+#pragma unroll 2
+    for (int v = gt; v < n_vec; v += T) {
+        float f[8], g[8];
+        unpack_bf16x8(xrow[v], f);
+        if (gain != nullptr) {
+            unpack_bf16x8(grow[v], g);
+        } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) g[e] = 1.0f;
+        }
+        uint32_t c[8], packed[2];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) c[e] = round_code(__fmul_rn(__fmul_rn(__fmul_rn(f[e], r), g[e]), s));
+        packed[0] = pack_codes4(c[0], c[1], c[2], c[3], csum);
+        packed[1] = pack_codes4(c[4], c[5], c[6], c[7], csum);
+        int dst = v;  // in units of 8 codes
+        if (LAYOUT == 1) {
+            const int piece = (v >> 1) & 15;
+            dst = (v & ~31) | ((((piece & 3) << 2) | (piece >> 2)) << 1) | (v & 1);
+        } else if (LAYOUT == 2 || LAYOUT == 3) {
+            const int kb = v >> 4, piece = (v >> 1) & 7;
+            dst = kb * ((LAYOUT == 2 ? 128 : 16) * 128 / 8) + (((piece ^ swz) << 1) | (v & 1));
+        }
+        qrow[dst] = make_uint2(packed[0], packed[1]);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xffffffffu, csum, o);
+    if (lane == 0) sm.sum[w] = csum;
+    group_sync();
+    if (gt == 0) {
+        int total = 0;
+#pragma unroll
+        for (int i = 0; i < WARPS; ++i) total += sm.sum[i];
+        *d_out = __fdiv_rn(a, 127.0f);
+        if (xsum_out != nullptr) *xsum_out = total;
+    }
+}
+
 }  // namespace bitlinear
