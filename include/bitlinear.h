@@ -252,7 +252,8 @@ int bitlinear_glue_attn_standin(const float* q, const float* v, void* o_in_bf16,
  *   layers   : HOST array of n_layers descriptors; pointers inside are DEVICE pointers: packed / s_w of the seven
  *              matrices in the order q,k,v,o,gate,up,down, and the bf16 RMSNorm gains of the four BitLinear inputs
  *              (of {q,k,v}, o, {gate,up}, down; NULL = ones).
- *   dims     : hidden = n_q_heads * head_dim; hidden and ffn multiples of 256, at most 8192; one token.
+ *   dims     : hidden = n_q_heads * head_dim; head_dim a multiple of 4; hidden and ffn multiples of 256, at most
+ *              8192; one token.
  *   h_bf16   : [hidden] bf16, in and out.      k_out : nullable, [n_kv_heads*head_dim] fp32, the last layer's k.
  *   flags    : 0 or BITLINEAR_BATCH_REUSE_PLAN (the layer table uploaded by the previous call on ws is still valid).
  *   ws       : at least bitlinear_decode_chain_workspace_bytes(...); calls on one workspace must not overlap.

@@ -74,7 +74,9 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-__device__ __forceinline__ float ldcg_f32(const float* p) { return __ldcg(p); }  // bypass L1: written by other CTAs
+// bypass L1: written by other CTAs
+__device__ __forceinline__ float ldcg_f32(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ float4 ldcg_f32x4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
 struct BlockScratch {
     double sq[kChainWarps];
@@ -223,36 +225,44 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         for (int i = tid; i < n_rb * 16; i += kChainThreads) acc_s[i] = 0;
         const __nv_bfloat16* gain = desc_s[layer & 1].gain[level];
         float xv[kMaxEpt], gv[kMaxEpt];
-        // every load of the stage is issued before anything is computed, so the L2 round trips overlap
+        // Element e of this thread is column 4 * (tid + (e / 4) * kChainThreads) + e % 4: four consecutive columns per
+        // 16-byte load.  Every load of the stage is issued before anything is computed, so the L2 round trips overlap.
         float ra[kMaxEpt], rb[kMaxEpt];
 #pragma unroll
-        for (int e = 0; e < kMaxEpt; ++e) {
-            const int i = tid + e * kChainThreads;
-            const bool in = i < K;
-            ra[e] = 0.0f;
-            rb[e] = 0.0f;
-            if (level == 0) {
-                if (in && layer > 0) ra[e] = ldcg_f32(p.dn + i);
-            } else if (level == 1) {
-                if (in) {
-                    const int head = i / p.head_dim, j = i - head * p.head_dim;
-                    ra[e] = ldcg_f32(p.q + i);
-                    rb[e] = ldcg_f32(p.v + (head / group) * p.head_dim + j);
-                }
-            } else if (level == 2) {
-                if (in) ra[e] = ldcg_f32(p.o + i);
-            } else {
-                if (in) {
-                    ra[e] = ldcg_f32(p.g + i);
-                    rb[e] = ldcg_f32(p.u + i);
+        for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
+            const int i0 = 4 * (tid + q4 * kChainThreads);
+            const bool in = i0 < K;  // K is a multiple of 4: a group of four is inside or outside as a whole
+            float4 va = make_float4(0.0f, 0.0f, 0.0f, 0.0f), vb = va;
+            if (in) {
+                if (level == 0) {
+                    if (layer > 0) va = ldcg_f32x4(p.dn + i0);
+                } else if (level == 1) {
+                    const int head = i0 / p.head_dim, j = i0 - head * p.head_dim;  // head_dim is a multiple of 4
+                    va = ldcg_f32x4(p.q + i0);
+                    vb = ldcg_f32x4(p.v + (head / group) * p.head_dim + j);
+                } else if (level == 2) {
+                    va = ldcg_f32x4(p.o + i0);
+                } else {
+                    va = ldcg_f32x4(p.g + i0);
+                    vb = ldcg_f32x4(p.u + i0);
                 }
             }
-            gv[e] = (gain != nullptr && in) ? __bfloat162float(gain[i]) : 1.0f;
+            ra[4 * q4] = va.x; ra[4 * q4 + 1] = va.y; ra[4 * q4 + 2] = va.z; ra[4 * q4 + 3] = va.w;
+            rb[4 * q4] = vb.x; rb[4 * q4 + 1] = vb.y; rb[4 * q4 + 2] = vb.z; rb[4 * q4 + 3] = vb.w;
+            if (gain != nullptr && in) {
+                const uint2 gw = *reinterpret_cast<const uint2*>(gain + i0);
+                gv[4 * q4] = __uint_as_float(gw.x << 16);
+                gv[4 * q4 + 1] = __uint_as_float(gw.x & 0xffff0000u);
+                gv[4 * q4 + 2] = __uint_as_float(gw.y << 16);
+                gv[4 * q4 + 3] = __uint_as_float(gw.y & 0xffff0000u);
+            } else {
+                gv[4 * q4] = gv[4 * q4 + 1] = gv[4 * q4 + 2] = gv[4 * q4 + 3] = 1.0f;
+            }
         }
         double sq = 0.0;
 #pragma unroll
         for (int e = 0; e < kMaxEpt; ++e) {
-            const int i = tid + e * kChainThreads;
+            const int i = 4 * (tid + (e >> 2) * kChainThreads) + (e & 3);
             float x = 0.0f;
             if (i < K) {
                 if (level == 0) {
@@ -309,7 +319,7 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         int csum = 0;
 #pragma unroll
         for (int e = 0; e < kMaxEpt; ++e) {
-            const int i = tid + e * kChainThreads;
+            const int i = 4 * (tid + (e >> 2) * kChainThreads) + (e & 3);
             if (i < K) {
                 const uint32_t c = chain_round_code(__fmul_rn(xv[e], sc_q));
                 csum += (int)(int8_t)(c & 0xffu);
@@ -433,7 +443,7 @@ ChainLayout chain_layout(int n_layers, int hidden, int ffn, int kv) {
 
 bool chain_dims_ok(int n_layers, int hidden, int ffn, int n_q, int n_kv, int hd) {
     if (n_layers <= 0 || n_q <= 0 || n_kv <= 0 || hd <= 0 || n_q % n_kv) return false;
-    if (hidden != n_q * hd || (n_kv * hd) % kTileRows) return false;
+    if (hidden != n_q * hd || (n_kv * hd) % kTileRows || hd % 4) return false;  // 16-byte loads never straddle a head
     return shape_ok(hidden, hidden) && shape_ok(ffn, hidden) && shape_ok(hidden, ffn) && hidden <= kMaxEpt * kChainThreads &&
            ffn <= kMaxEpt * kChainThreads;
 }
