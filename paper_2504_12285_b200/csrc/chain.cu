@@ -318,14 +318,15 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         const float sc_q = __fdiv_rn(127.0f, a), d = __fdiv_rn(a, 127.0f);
         int csum = 0;
 #pragma unroll
-        for (int e = 0; e < kMaxEpt; ++e) {
-            const int i = 4 * (tid + (e >> 2) * kChainThreads) + (e & 3);
-            if (i < K) {
-                const uint32_t c = chain_round_code(__fmul_rn(xv[e], sc_q));
-                csum += (int)(int8_t)(c & 0xffu);
-                // lane-interleaved order inside each block of 256 columns: piece 4t+q -> byte 64q + 16t
-                const int blk = i & ~255, rr = i & 255;
-                xq_s[blk + 64 * ((rr >> 4) & 3) + 16 * (rr >> 6) + (rr & 15)] = (uint8_t)(c & 0xffu);
+        for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
+            const int i0 = 4 * (tid + q4 * kChainThreads);
+            if (i0 < K) {
+                const uint32_t word = pack_codes4(chain_round_code(__fmul_rn(xv[4 * q4], sc_q)), chain_round_code(__fmul_rn(xv[4 * q4 + 1], sc_q)),
+                                                  chain_round_code(__fmul_rn(xv[4 * q4 + 2], sc_q)), chain_round_code(__fmul_rn(xv[4 * q4 + 3], sc_q)), csum);
+                // lane-interleaved order inside each block of 256 columns: piece 4t+q -> byte 64q + 16t; four consecutive
+                // columns stay together inside their 16-byte piece
+                const int blk = i0 & ~255, rr = i0 & 255;
+                *reinterpret_cast<uint32_t*>(xq_s + blk + 64 * ((rr >> 4) & 3) + 16 * (rr >> 6) + (rr & 15)) = word;
             }
         }
 #pragma unroll
