@@ -391,10 +391,9 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             y[row] = __fmul_rn(__fmul_rn((float)(acc_s[o] - xsum), s_w), d);
         }
         CSYNC();
-        if (tid == 0) {
-            __threadfence();
-            atomicAdd(p.barrier, 1u);
-        }
+        // release at GPU scope: the stores of every thread of the CTA (ordered before this by the barrier above) are
+        // visible to whoever acquires the new count
+        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
     }
 
     // ---- after the last level: the final residual, written by CTA 0 ----
