@@ -86,6 +86,7 @@ struct BlockScratch {
     int xsum;
     int ok;
     int desc_ready;  // highest layer whose descriptor is in shared memory
+    int rb_lo[4], rb_hi[4];  // this CTA's share of the row blocks of each of the four levels of a layer
 };
 
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
@@ -126,6 +127,12 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         sc->desc_ready = 0;
         mbar_init_fence();
     }
+    if (tid < 4) {  // the shares do not change from layer to layer: two 64-bit divisions per level, once
+        const LevelShape s = level_shape(tid, p);
+        const int total_rb = (s.rows[0] + s.rows[1] + s.rows[2]) / kTileRows;
+        sc->rb_lo[tid] = (int)((long long)total_rb * cta / grid);
+        sc->rb_hi[tid] = (int)((long long)total_rb * (cta + 1) / grid);
+    }
     {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(p.layers);
         uint32_t* dst = reinterpret_cast<uint32_t*>(desc_s);
@@ -142,7 +149,7 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         const LevelShape s = level_shape(level, p);
         const ChainLayerDev& dsc = desc_s[layer & 1];
         const int total_rb = (s.rows[0] + s.rows[1] + s.rows[2]) / kTileRows;
-        const int lo = (int)((long long)total_rb * cta / grid), hi = (int)((long long)total_rb * (cta + 1) / grid);
+        const int lo = sc->rb_lo[level], hi = sc->rb_hi[level];
         const uint32_t rb_bytes = (uint32_t)(s.K / kTileCols) * kTileBytes;
         const uint32_t bar = smem_u32(bars + (L & 1));
         if (lane == 0) mbar_expect_tx(bar, (uint32_t)(hi - lo) * rb_bytes);
@@ -175,7 +182,7 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         const LevelShape s = level_shape(level, p);
         const int K = s.K, k_tiles = K / kTileCols;
         const int total_rb = (s.rows[0] + s.rows[1] + s.rows[2]) / kTileRows;
-        const int rb_lo = (int)((long long)total_rb * cta / grid), rb_hi = (int)((long long)total_rb * (cta + 1) / grid);
+        const int rb_lo = sc->rb_lo[level], rb_hi = sc->rb_hi[level];
         const int n_rb = rb_hi - rb_lo;
 
         // ---- descriptor / scale prefetch for the next layer, weight prefetch for the next level ----
