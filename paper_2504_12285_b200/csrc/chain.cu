@@ -156,7 +156,11 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         __syncwarp();
         for (int i = lane; i < hi - lo; i += 32) {
             int row = (lo + i) * kTileRows, m = 0;
-            while (row >= s.rows[m]) { row -= s.rows[m]; ++m; }
+            if (row >= s.rows[0]) {  // which of the level's stacked matrices (no indexed array: it would live in local memory)
+                row -= s.rows[0];
+                m = 1;
+                if (row >= s.rows[1]) { row -= s.rows[1]; m = 2; }
+            }
             bulk_load(smem_u32(wbuf + (size_t)(L & 1) * p.buf_bytes) + (uint32_t)i * rb_bytes,
                       dsc.packed[s.first + m] + (size_t)(row / kTileRows) * rb_bytes, rb_bytes, bar);
         }
@@ -388,7 +392,11 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         // ---- dequantising epilogue: this CTA's rows of the level's output ----
         for (int o = tid; o < n_rb * 16; o += kChainThreads) {
             int row = (rb_lo + (o >> 4)) * kTileRows + (o & 15), m = 0;
-            while (row >= s.rows[m]) { row -= s.rows[m]; ++m; }
+            if (row >= s.rows[0]) {  // which of the level's stacked matrices (no indexed array: it would live in local memory)
+                row -= s.rows[0];
+                m = 1;
+                if (row >= s.rows[1]) { row -= s.rows[1]; m = 2; }
+            }
             float* y;
             if (level == 0) y = m == 0 ? p.q : (m == 1 ? p.k : p.v);
             else if (level == 1) y = p.o;
