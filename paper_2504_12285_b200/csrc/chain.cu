@@ -41,12 +41,8 @@ struct ChainParams {
     int n_layers, hidden, ffn, n_q, n_kv, head_dim;
     float eps;
     __nv_bfloat16* h;                 // [hidden] in / out
-    // Level outputs.  Every element is a pair {fp32 bits, tag} written by ONE 8-byte store; the tag names the call and
-    // the level that produced it, so a reader needs no barrier and no fence: it loads the pair until the tag is the one
-    // it expects.  (A buffer is rewritten four levels later; by then every CTA has produced three more levels, each of
-    // which needed everyone's previous level, so nobody can still be reading the old values.)
-    uint2 *q, *k, *v, *o, *g, *u, *dn;
-    unsigned* epoch;                  // call counter of this workspace (bumped by CTA 0 at the end of every call)
+    float *q, *k, *v, *o, *g, *u, *dn;  // level outputs (fp32)
+    unsigned* barrier;                // grid barrier counter, zero at launch
     int* abort_word;                  // zero at launch
     int* status_word;
     int buf_bytes;                    // one weight buffer (the largest per-CTA share of a level)
@@ -78,15 +74,9 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-// Two tagged elements {value, tag, value, tag} by one volatile 16-byte load (never from L1: other CTAs write them).
-__device__ __forceinline__ uint4 ld_pairs2(const uint2* p) {
-    uint4 v;
-    asm volatile("ld.volatile.global.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_pair(uint2* p, float value, unsigned tag) {
-    asm volatile("st.volatile.global.v2.u32 [%0], {%1,%2};" ::"l"(p), "r"(__float_as_uint(value)), "r"(tag) : "memory");
-}
+// bypass L1: written by other CTAs
+__device__ __forceinline__ float ldcg_f32(const float* p) { return __ldcg(p); }
+__device__ __forceinline__ float4 ldcg_f32x4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 
 struct BlockScratch {
     double sq[kChainWarps];
@@ -103,6 +93,12 @@ __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(_
 
 // Same rounding as the stand-alone quantisers (see round_code in quant_row.cuh): low byte = int8 code.
 __device__ __forceinline__ uint32_t chain_round_code(float v) { return __float_as_uint(__fadd_rn(v, 12582912.0f)); }
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(const ChainParams p) {
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -122,8 +118,6 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
     const int g = lane >> 2, t = lane & 3;
     const int grid = (int)gridDim.x, cta = (int)blockIdx.x;
     const int total_levels = 4 * p.n_layers;
-    const unsigned epoch = *reinterpret_cast<const volatile unsigned*>(p.epoch);
-    const unsigned tag_base = epoch << 12;  // tag of level L (0-based) of this call: tag_base + L + 1
     const int group = p.n_q / p.n_kv;
 
     // ---- prologue: barriers, first descriptor, its scales, the hidden state ----
@@ -217,98 +211,64 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
 
-        // ---- build this level's input vector (glue), RMSNorm, absmax int8 quantiser ----
-        for (int i = tid; i < n_rb * 16; i += kChainThreads) acc_s[i] = 0;
-        const __nv_bfloat16* gain = desc_s[layer & 1].gain[level];
-        float xv[kMaxEpt], gv[kMaxEpt];
-        // Element e of this thread is column 4 * (tid + (e / 4) * kChainThreads) + e % 4: four consecutive columns = two
-        // 16-byte loads of tagged pairs per source.  A thread first polls its first group until the previous level's tag
-        // shows (the level's outputs appear at about the same time everywhere), then issues every load of the stage
-        // before anything is computed, so the L2 round trips overlap; a pair that is still old is loaded again.
-        float ra[kMaxEpt], rb[kMaxEpt];
-        {
-            const uint2* src_a = nullptr;
-            const uint2* src_b = nullptr;
-            if (level == 0) src_a = layer > 0 ? p.dn : nullptr;
-            else if (level == 1) { src_a = p.q; src_b = p.v; }
-            else if (level == 2) src_a = p.o;
-            else { src_a = p.g; src_b = p.u; }
-            const unsigned want = tag_base + (unsigned)L;  // tag of level L - 1 (levels are tagged from 1)
-            uint4 wa[kMaxEpt / 4][2], wb[kMaxEpt / 4][2];
-            int ib[kMaxEpt / 4];  // where the second source of a group starts
-#pragma unroll
-            for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
-                const int i0 = 4 * (tid + q4 * kChainThreads);
-                ib[q4] = i0;
-                if (level == 1 && i0 < K) {
-                    const int head = i0 / p.head_dim, j = i0 - head * p.head_dim;  // head_dim is a multiple of 4
-                    ib[q4] = (head / group) * p.head_dim + j;
-                }
-            }
-            bool good = true;
-            if (src_a != nullptr && 4 * tid < K) {  // poll the first group
+        // ---- wait for the outputs of the previous level (grid barrier, bounded) ----
+        if (L > 0) {
+            if (tid == 0) {
+                const unsigned target = (unsigned)grid * (unsigned)L;
                 const unsigned long long t0 = globaltimer_ns();
                 unsigned spins = 0;
-                for (;;) {
-                    const uint4 w = ld_pairs2(src_a + 4 * tid);
-                    if (w.y == want && w.w == want) break;
+                while (ld_acquire_u32(p.barrier) < target) {
                     if ((++spins & 255u) == 0u) {
-                        if (*reinterpret_cast<volatile int*>(p.abort_word) != 0) { good = false; break; }
+                        if (*reinterpret_cast<volatile int*>(p.abort_word) != 0) { sc->ok = 1; break; }
                         if (globaltimer_ns() - t0 > kWaitLimitNs) {
                             atomicExch(p.abort_word, 1);
-                            good = false;
+                            sc->ok = 1;
                             break;
                         }
                     }
                 }
             }
+            CSYNC();
+            if (sc->ok) { ok = false; break; }
+        }
+
+        // ---- build this level's input vector (glue), RMSNorm, absmax int8 quantiser ----
+        for (int i = tid; i < n_rb * 16; i += kChainThreads) acc_s[i] = 0;
+        const __nv_bfloat16* gain = desc_s[layer & 1].gain[level];
+        float xv[kMaxEpt], gv[kMaxEpt];
+        // Element e of this thread is column 4 * (tid + (e / 4) * kChainThreads) + e % 4: four consecutive columns per
+        // 16-byte load.  Every load of the stage is issued before anything is computed, so the L2 round trips overlap.
+        float ra[kMaxEpt], rb[kMaxEpt];
 #pragma unroll
-            for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
-                const int i0 = 4 * (tid + q4 * kChainThreads);
-                wa[q4][0] = wa[q4][1] = wb[q4][0] = wb[q4][1] = make_uint4(0u, want, 0u, want);
-                if (good && i0 < K) {
-                    if (src_a != nullptr) { wa[q4][0] = ld_pairs2(src_a + i0); wa[q4][1] = ld_pairs2(src_a + i0 + 2); }
-                    if (src_b != nullptr) { wb[q4][0] = ld_pairs2(src_b + ib[q4]); wb[q4][1] = ld_pairs2(src_b + ib[q4] + 2); }
-                }
-            }
-#pragma unroll
-            for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
-                const int i0 = 4 * (tid + q4 * kChainThreads);
-#pragma unroll
-                for (int hh = 0; hh < 2; ++hh) {
-                    unsigned spins = 0;
-                    const unsigned long long t0 = globaltimer_ns();
-                    while (good && (wa[q4][hh].y != want || wa[q4][hh].w != want)) {
-                        wa[q4][hh] = ld_pairs2(src_a + i0 + 2 * hh);
-                        if ((++spins & 255u) == 0u && (*reinterpret_cast<volatile int*>(p.abort_word) != 0 || globaltimer_ns() - t0 > kWaitLimitNs)) {
-                            atomicExch(p.abort_word, 1);
-                            good = false;
-                        }
-                    }
-                    while (good && (wb[q4][hh].y != want || wb[q4][hh].w != want)) {
-                        wb[q4][hh] = ld_pairs2(src_b + ib[q4] + 2 * hh);
-                        if ((++spins & 255u) == 0u && (*reinterpret_cast<volatile int*>(p.abort_word) != 0 || globaltimer_ns() - t0 > kWaitLimitNs)) {
-                            atomicExch(p.abort_word, 1);
-                            good = false;
-                        }
-                    }
-                }
-                ra[4 * q4] = __uint_as_float(wa[q4][0].x); ra[4 * q4 + 1] = __uint_as_float(wa[q4][0].z);
-                ra[4 * q4 + 2] = __uint_as_float(wa[q4][1].x); ra[4 * q4 + 3] = __uint_as_float(wa[q4][1].z);
-                rb[4 * q4] = __uint_as_float(wb[q4][0].x); rb[4 * q4 + 1] = __uint_as_float(wb[q4][0].z);
-                rb[4 * q4 + 2] = __uint_as_float(wb[q4][1].x); rb[4 * q4 + 3] = __uint_as_float(wb[q4][1].z);
-                const bool in = i0 < K;
-                if (gain != nullptr && in) {
-                    const uint2 gw = *reinterpret_cast<const uint2*>(gain + i0);
-                    gv[4 * q4] = __uint_as_float(gw.x << 16);
-                    gv[4 * q4 + 1] = __uint_as_float(gw.x & 0xffff0000u);
-                    gv[4 * q4 + 2] = __uint_as_float(gw.y << 16);
-                    gv[4 * q4 + 3] = __uint_as_float(gw.y & 0xffff0000u);
+        for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
+            const int i0 = 4 * (tid + q4 * kChainThreads);
+            const bool in = i0 < K;  // K is a multiple of 4: a group of four is inside or outside as a whole
+            float4 va = make_float4(0.0f, 0.0f, 0.0f, 0.0f), vb = va;
+            if (in) {
+                if (level == 0) {
+                    if (layer > 0) va = ldcg_f32x4(p.dn + i0);
+                } else if (level == 1) {
+                    const int head = i0 / p.head_dim, j = i0 - head * p.head_dim;  // head_dim is a multiple of 4
+                    va = ldcg_f32x4(p.q + i0);
+                    vb = ldcg_f32x4(p.v + (head / group) * p.head_dim + j);
+                } else if (level == 2) {
+                    va = ldcg_f32x4(p.o + i0);
                 } else {
-                    gv[4 * q4] = gv[4 * q4 + 1] = gv[4 * q4 + 2] = gv[4 * q4 + 3] = 1.0f;
+                    va = ldcg_f32x4(p.g + i0);
+                    vb = ldcg_f32x4(p.u + i0);
                 }
             }
-            if (!good) sc->ok = 1;  // seen by everybody after the next barrier of the compute threads
+            ra[4 * q4] = va.x; ra[4 * q4 + 1] = va.y; ra[4 * q4 + 2] = va.z; ra[4 * q4 + 3] = va.w;
+            rb[4 * q4] = vb.x; rb[4 * q4 + 1] = vb.y; rb[4 * q4 + 2] = vb.z; rb[4 * q4 + 3] = vb.w;
+            if (gain != nullptr && in) {
+                const uint2 gw = *reinterpret_cast<const uint2*>(gain + i0);
+                gv[4 * q4] = __uint_as_float(gw.x << 16);
+                gv[4 * q4 + 1] = __uint_as_float(gw.x & 0xffff0000u);
+                gv[4 * q4 + 2] = __uint_as_float(gw.y << 16);
+                gv[4 * q4 + 3] = __uint_as_float(gw.y & 0xffff0000u);
+            } else {
+                gv[4 * q4] = gv[4 * q4 + 1] = gv[4 * q4 + 2] = gv[4 * q4 + 3] = 1.0f;
+            }
         }
         double sq = 0.0;
 #pragma unroll
@@ -345,7 +305,6 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
         if (lane == 0) sc->sq[warp] = sq;
         CSYNC();
-        if (sc->ok) { ok = false; break; }  // a wait for the previous level's outputs ran out (or another CTA gave up)
         if (tid == 0) {
             double S = 0.0;
 #pragma unroll
@@ -438,38 +397,40 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
                 m = 1;
                 if (row >= s.rows[1]) { row -= s.rows[1]; m = 2; }
             }
-            uint2* y;
+            float* y;
             if (level == 0) y = m == 0 ? p.q : (m == 1 ? p.k : p.v);
             else if (level == 1) y = p.o;
             else if (level == 2) y = m == 0 ? p.g : p.u;
             else y = p.dn;
             const float s_w = sw_s[8 * (layer & 1) + s.first + m];
-            st_pair(y + row, __fmul_rn(__fmul_rn((float)(acc_s[o] - xsum), s_w), d), tag_base + (unsigned)L + 1u);
+            y[row] = __fmul_rn(__fmul_rn((float)(acc_s[o] - xsum), s_w), d);
         }
-        CSYNC();  // acc_s is cleared again at the top of the next level
+        CSYNC();
+        // release at GPU scope: the stores of every thread of the CTA (ordered before this by the barrier above) are
+        // visible to whoever acquires the new count
+        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
     }
 
-    // ---- after the last level: the final residual, written by CTA 0, which also closes the call's epoch ----
+    // ---- after the last level: the final residual, written by CTA 0 ----
     if (warp < kChainWarps && ok && cta == 0) {
-        const unsigned want = tag_base + (unsigned)total_levels;
-        bool good = true;
-        for (int i = tid; i < p.hidden; i += kChainThreads) {
-            unsigned spins = 0;
+        if (tid == 0) {
+            const unsigned target = (unsigned)grid * (unsigned)total_levels;
             const unsigned long long t0 = globaltimer_ns();
-            uint4 w = ld_pairs2(p.dn + (i & ~1));
-            while (good && (w.y != want || w.w != want)) {
-                w = ld_pairs2(p.dn + (i & ~1));
-                if ((++spins & 255u) == 0u && (*reinterpret_cast<volatile int*>(p.abort_word) != 0 || globaltimer_ns() - t0 > kWaitLimitNs)) {
+            unsigned spins = 0;
+            while (ld_acquire_u32(p.barrier) < target) {
+                if ((++spins & 255u) == 0u && (globaltimer_ns() - t0 > kWaitLimitNs || *reinterpret_cast<volatile int*>(p.abort_word))) {
                     atomicExch(p.abort_word, 1);
-                    good = false;
+                    sc->ok = 1;
+                    break;
                 }
             }
-            if (good) p.h[i] = __float2bfloat16_rn(__fadd_rn(__bfloat162float(h_s[i]), __uint_as_float((i & 1) ? w.z : w.x)));
         }
-        if (!good) sc->ok = 1;
+        CSYNC();
+        if (!sc->ok)
+            for (int i = tid; i < p.hidden; i += kChainThreads)
+                p.h[i] = __float2bfloat16_rn(__fadd_rn(__bfloat162float(h_s[i]), ldcg_f32(p.dn + i)));
     }
     __syncthreads();
-    if (tid == 0 && cta == 0) *p.epoch = epoch + 1u;  // the next call on this workspace uses other tags (also after an abort)
     if (!ok || sc->ok) abort_drain();  // bulk copies of this CTA may still be in flight
     if (tid == 0 && cta == 0 && *reinterpret_cast<volatile int*>(p.abort_word) != 0 && p.status_word != nullptr)
         atomicExch(p.status_word, BITLINEAR_ERR_TIMEOUT);
@@ -487,7 +448,7 @@ ChainLayout chain_layout(int n_layers, int hidden, int ffn, int kv) {
     const int widths[7] = {hidden, kv, kv, hidden, ffn, ffn, hidden};  // q k v o g u dn
     for (int i = 0; i < 7; ++i) {
         L.out_off[i] = off;
-        off = align_up(off + (size_t)widths[i] * sizeof(uint2), 256);  // {value, tag} pairs
+        off = align_up(off + (size_t)widths[i] * sizeof(float), 256);
     }
     L.sync_off = off;
     off += 256;
@@ -496,7 +457,7 @@ ChainLayout chain_layout(int n_layers, int hidden, int ffn, int kv) {
 }
 
 bool chain_dims_ok(int n_layers, int hidden, int ffn, int n_q, int n_kv, int hd) {
-    if (n_layers <= 0 || n_layers > 1000 || n_q <= 0 || n_kv <= 0 || hd <= 0 || n_q % n_kv) return false;  // level tags: 12 bits
+    if (n_layers <= 0 || n_q <= 0 || n_kv <= 0 || hd <= 0 || n_q % n_kv) return false;
     if (hidden != n_q * hd || (n_kv * hd) % kTileRows || hd % 4) return false;  // 16-byte loads never straddle a head
     return shape_ok(hidden, hidden) && shape_ok(ffn, hidden) && shape_ok(hidden, ffn) && hidden <= kMaxEpt * kChainThreads &&
            ffn <= kMaxEpt * kChainThreads;
@@ -554,11 +515,7 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
-    // abort word cleared every call; on a first call (descriptors uploaded) also the call counter and the tagged
-    // outputs, so that nothing left in the workspace can look like a value of this call
-    if (cudaMemsetAsync(base + L.sync_off, 0, 128, st) != cudaSuccess ||
-        (!(flags & BITLINEAR_BATCH_REUSE_PLAN) &&
-         cudaMemsetAsync(base + L.out_off[0], 0, L.total - L.out_off[0], st) != cudaSuccess)) {
+    if (cudaMemsetAsync(base + L.sync_off, 0, 256, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
@@ -567,11 +524,11 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
     prm.n_layers = n_layers; prm.hidden = hidden; prm.ffn = ffn; prm.n_q = n_q_heads; prm.n_kv = n_kv_heads;
     prm.head_dim = head_dim; prm.eps = rms_eps;
     prm.h = static_cast<__nv_bfloat16*>(h_bf16);
-    uint2* outs[7];
-    for (int i = 0; i < 7; ++i) outs[i] = reinterpret_cast<uint2*>(base + L.out_off[i]);
+    float* outs[7];
+    for (int i = 0; i < 7; ++i) outs[i] = reinterpret_cast<float*>(base + L.out_off[i]);
     prm.q = outs[0]; prm.k = outs[1]; prm.v = outs[2]; prm.o = outs[3]; prm.g = outs[4]; prm.u = outs[5]; prm.dn = outs[6];
+    prm.barrier = reinterpret_cast<unsigned*>(base + L.sync_off);
     prm.abort_word = reinterpret_cast<int*>(base + L.sync_off + 64);
-    prm.epoch = reinterpret_cast<unsigned*>(base + L.sync_off + 128);
     prm.status_word = device_status_word();
     // the largest per-CTA share of a level, in bytes of packed weights
     const int grid = sm_count;
@@ -596,9 +553,7 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
-    // the values of the last layer's k, without their tags
-    if (k_out && cudaMemcpy2DAsync(k_out, sizeof(float), prm.k, sizeof(uint2), sizeof(float), (size_t)kv, cudaMemcpyDeviceToDevice,
-                                   st) != cudaSuccess) {
+    if (k_out && cudaMemcpyAsync(k_out, prm.k, (size_t)kv * sizeof(float), cudaMemcpyDeviceToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
