@@ -36,7 +36,7 @@ def check(batch, refs):
         if ref is None:
             continue
         ok = ref["fragile"] == 0
-        assert ok.mean() > 0.9
+        assert ok.size - ok.sum() <= ok.size // 1000  # flagged rows: none at all in cases of fewer than 1000 rows
         if y.dtype == torch.float32:
             got = y.cpu().numpy().astype(np.float64)[ok]
             want = ref["y"].astype(np.float64)[ok]
@@ -209,7 +209,7 @@ def test_batch_many_tiny_problems_overflow_the_descriptor_cache():
     ok = ref["fragile"] == 0
     got = ys.reshape(M * count, N).cpu().numpy().astype(np.float64)[ok]
     want = ref["y"].astype(np.float64)[ok]
-    assert ok.mean() > 0.9
+    assert ok.size - ok.sum() <= ok.size // 1000
     assert np.all(np.abs(got - want) <= 1e-6 * np.abs(want))
 
 

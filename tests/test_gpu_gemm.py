@@ -27,7 +27,10 @@ def stable_rows(fragile):
     On the (about one in 1e5) rows the oracle flags, two equally valid fp64 summation orders may
     round the scale to neighbouring fp32 values, so bit-exactness is only required elsewhere."""
     ok = np.asarray(fragile) == 0
-    assert ok.mean() >= 0.995
+    flagged = int(ok.size - ok.sum())
+    if flagged:
+        print(f"rows flagged as fragile: {flagged} of {ok.size}")
+    assert flagged <= ok.size // 1000  # none at all in cases of fewer than 1000 rows
     return ok
 
 

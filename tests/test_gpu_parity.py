@@ -32,7 +32,10 @@ def stable_rows(fragile):
     """Rows whose RMSNorm scale does not sit on an fp32 rounding boundary of the sum of squares
     (the oracle flags about one row in 1e5 where two valid fp64 summation orders may differ)."""
     ok = np.asarray(fragile) == 0
-    assert ok.mean() >= 0.9
+    flagged = int(ok.size - ok.sum())
+    if flagged:
+        print(f"rows flagged as fragile: {flagged} of {ok.size}")
+    assert flagged <= ok.size // 1000  # none at all in cases of fewer than 1000 rows
     return ok
 
 
