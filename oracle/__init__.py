@@ -40,6 +40,9 @@ def _load():
         lib = ctypes.CDLL(str(_LIB))
         lib.oracle_pack.restype = ctypes.c_int
         lib.oracle_unpack.restype = ctypes.c_int
+        lib.oracle_pack5.restype = ctypes.c_int
+        lib.oracle_unpack5.restype = ctypes.c_int
+        lib.oracle_packed5_bytes.restype = ctypes.c_long
         lib.oracle_num_threads.restype = ctypes.c_int
         _lib = lib
     return _lib
@@ -143,6 +146,35 @@ def unpack(packed: np.ndarray, N: int, K: int) -> np.ndarray:
     rc = _load().oracle_unpack(_p(packed), N, K, _p(wq))
     if rc != 0:
         raise ValueError(f"oracle_unpack failed with {rc}")
+    return wq
+
+
+def packed5_bytes(N: int, K: int) -> int:
+    """Bytes of the five-per-byte form of an [N, K] ternary matrix (K padded to a multiple of 320 columns)."""
+    return int(_load().oracle_packed5_bytes(N, K))
+
+
+def pack5(wq: np.ndarray) -> np.ndarray:
+    """Step 7b -> uint8 [N * Kp / 5] in the tiled five-per-byte layout."""
+    wq = _c(wq, np.int8)
+    N, K = wq.shape
+    nbytes = packed5_bytes(N, K)
+    if nbytes == 0:
+        raise ValueError("oracle_pack5: unsupported shape")
+    out = np.empty(nbytes, np.uint8)
+    rc = _load().oracle_pack5(_p(wq), N, K, _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle_pack5 failed with {rc}")
+    return out
+
+
+def unpack5(packed: np.ndarray, N: int, K: int) -> np.ndarray:
+    packed = _c(packed, np.uint8)
+    assert packed.size == packed5_bytes(N, K)
+    wq = np.empty((N, K), np.int8)
+    rc = _load().oracle_unpack5(_p(packed), N, K, _p(wq))
+    if rc != 0:
+        raise ValueError(f"oracle_unpack5 failed with {rc}")
     return wq
 
 

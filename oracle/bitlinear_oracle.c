@@ -23,18 +23,21 @@
  *   5. Weight scale: beta = fl32( mean |W| ) over the whole matrix; s_w = fl32(beta + eps_w).
  *   6. Weight quantiser: W_q = clip( Round( fl32(W / s_w) ), -1, 1 ).
  *   7. Packing: four ternary codes per byte in the tiled order documented at
- *      oracle_pack_index() below.
+ *      oracle_pack_index() below; or (7b) five per byte, see oracle_pack5_index().
  *   8. Contraction: acc[m][n] = sum_k q[m][k] * W_q[n][k] in int32.
  *   9. Dequantising epilogue: y[m][n] = fl32( fl32( (float)acc * s_w ) * d[m] ).
  *
  * Parity pins (see tests/test_oracle_pins.py): hand-computed rounding, tie and
  * clip cases; range invariants; the Gaussian closed form for the share of zero
  * weights; textbook RMSNorm in fp64; int64 library matmul; identity / one-hot /
- * all-ones weight patterns; fp64 brute force of the dequantised operands.
+ * all-ones weight patterns; fp64 brute force of the dequantised operands; for the
+ * five-per-byte layout all 243 byte patterns against exact rational arithmetic,
+ * hand-derived positions and byte values, sizes, round trips, identity weights.
  * Parity on the released model weights is unpinned: they are not available here.
  */
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 /* ---- bf16 <-> fp32 ------------------------------------------------------- */
@@ -246,6 +249,90 @@ int oracle_unpack(const uint8_t *packed, int N, int K, int8_t *wq) {
             wq[(long)n * K + k] = (int8_t)(c - 1);
         }
     return bad ? -2 : 0;
+}
+
+/* ---- step 7b: the dense packed layout, five ternary values per byte -------- */
+
+/*
+ * 1.6 bits per weight: Table 1 of the paper counts the non-embedding memory of the 2B
+ * model at about 1.58 bits per weight, and Section 5.1 packs weights to cut the bytes
+ * that cross HBM; 3^5 = 243 <= 256, so five ternary values fit one byte.  The paper
+ * gives no layout for this; the one below is this library's.
+ *
+ * Byte value.  With the codes c_e = W_q + 1 (0, 1 or 2) of five weights, digit 0 the
+ * most significant, v = c_0*81 + c_1*27 + c_2*9 + c_3*3 + c_4 lies in [0, 242] and the
+ * stored byte is B = ceil(256 * v / 243): the base-3 fraction 0.c_0 c_1 c_2 c_3 c_4
+ * scaled to 8 bits and rounded up.  v is recovered as floor(243 * B / 256).  Thirteen
+ * of the 256 byte values are never produced.
+ *
+ * Position.  K is padded with zero weights to Kp = 320 * ceil(K / 320).  The matrix is
+ * cut into tiles of 16 rows x 320 columns, 1024 bytes each, stored row-block major:
+ * tile = (n / 16) * (Kp / 320) + (k / 320).  Inside a tile, for row r = 8*h + g and
+ * column c = 80*t + 20*i + 4*e + b  (t, i, b in 0..3, e in 0..4):
+ *     byte offset in the tile = 512*h + 64*g + 16*t + 4*i + b,   base-3 digit e.
+ * So a 16-byte chunk is 80 consecutive columns of one row, a 4-byte word is 20
+ * consecutive columns, and digit e of the four bytes of a word is four consecutive
+ * columns.  N must be a multiple of 16 and K of 256.
+ */
+long oracle_packed5_bytes(int N, int K) {
+    if (N <= 0 || K <= 0 || N % 16 || K % 256) return 0;
+    long kp = ((long)K + 319) / 320 * 320;
+    return (long)N * kp / 5;
+}
+
+static void oracle_pack5_index(int n, int k, int K, long *byte_index, int *digit) {
+    long tiles_per_block = ((long)K + 319) / 320;
+    long tile = (long)(n / 16) * tiles_per_block + (k / 320);
+    int r = n % 16, h = r / 8, g = r % 8;
+    int c = k % 320, t = c / 80, i = (c % 80) / 20, e = (c % 20) / 4, b = c % 4;
+    *byte_index = tile * 1024 + 512 * h + 64 * g + 16 * t + 4 * i + b;
+    *digit = e;
+}
+
+static const int kPow3[5] = {81, 27, 9, 3, 1}; /* weight of digit e */
+
+/* Returns 0 on success, -1 on an unsupported shape, -2 if a value is not in {-1,0,1}. */
+int oracle_pack5(const int8_t *wq, int N, int K, uint8_t *packed) {
+    long bytes = oracle_packed5_bytes(N, K);
+    if (bytes == 0) return -1;
+    /* v of every byte, starting from five zero weights (code 1 in every digit: 121) */
+    int16_t *v = (int16_t *)malloc((size_t)bytes * sizeof(int16_t));
+    if (!v) return -1;
+    for (long i = 0; i < bytes; ++i) v[i] = 121;
+    int rc = 0;
+    for (int n = 0; n < N && rc == 0; ++n)
+        for (int k = 0; k < K; ++k) {
+            int w = wq[(long)n * K + k];
+            if (w < -1 || w > 1) { rc = -2; break; }
+            long bi;
+            int e;
+            oracle_pack5_index(n, k, K, &bi, &e);
+            v[bi] = (int16_t)(v[bi] + w * kPow3[e]);
+        }
+    if (rc == 0)
+        for (long i = 0; i < bytes; ++i) packed[i] = (uint8_t)((256 * (int)v[i] + 242) / 243);
+    free(v);
+    return rc;
+}
+
+/* Returns 0 on success, -1 on an unsupported shape, -2 if a byte value that no five codes produce is met.
+ * Padding columns (k >= K) are not returned. */
+int oracle_unpack5(const uint8_t *packed, int N, int K, int8_t *wq) {
+    long bytes = oracle_packed5_bytes(N, K);
+    if (bytes == 0) return -1;
+    for (long i = 0; i < bytes; ++i) {
+        int v = (243 * (int)packed[i]) / 256;
+        if ((256 * v + 242) / 243 != (int)packed[i]) return -2;
+    }
+    for (int n = 0; n < N; ++n)
+        for (int k = 0; k < K; ++k) {
+            long bi;
+            int e;
+            oracle_pack5_index(n, k, K, &bi, &e);
+            int v = (243 * (int)packed[bi]) / 256;
+            wq[(long)n * K + k] = (int8_t)((v / kPow3[e]) % 3 - 1);
+        }
+    return 0;
 }
 
 /* ---- step 8: the contraction --------------------------------------------- */

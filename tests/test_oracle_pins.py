@@ -239,6 +239,114 @@ def test_pack_roundtrip_all_byte_patterns_and_random():
         oracle.pack(np.full((16, 256), 2, np.int8))
 
 
+# --------------------------------------------------------------------------- dense packing: five per byte
+
+
+def _golden_positions5():
+    rows = []
+    with open(os.path.join(GOLDEN, "pack5_layout_positions.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                rows.append(tuple(int(v) for v in line.split()))
+    return rows
+
+
+@pytest.mark.parametrize("n,k,byte,digit,plus,minus", _golden_positions5())
+def test_pack5_positions_match_hand_computed_layout(n, k, byte, digit, plus, minus):
+    N, K = 32, 512
+    for trit, value in ((1, plus), (-1, minus)):
+        wq = np.zeros((N, K), np.int8)
+        wq[n, k] = trit
+        packed = oracle.pack5(wq)
+        assert packed.size == 4096  # 32 rows x 640 padded columns / 5
+        expect = np.full(4096, 128, np.uint8)  # five zero weights: v = 121 -> byte 128
+        expect[byte] = value
+        assert np.array_equal(packed, expect)
+        assert np.array_equal(oracle.unpack5(packed, N, K), wq)
+
+
+def test_pack5_all_243_byte_patterns():
+    # Every combination of five neighbouring weights.  Column c = 4*e + b of a 20-column word is digit e of byte b,
+    # so the five weights of byte 0 of the first word of row 0 are columns 0, 4, 8, 12, 16.
+    from fractions import Fraction
+    combos = np.array(np.meshgrid(*[[-1, 0, 1]] * 5, indexing="ij")).reshape(5, -1).T  # 243 x 5, digit 0 slowest
+    seen = {}
+    for trits in combos:
+        wq = np.zeros((16, 256), np.int8)
+        wq[0, [0, 4, 8, 12, 16]] = trits
+        packed = oracle.pack5(wq)
+        assert packed.size == 16 * 320 // 5 and np.all(packed[1:] == 128)
+        B = int(packed[0])
+        # the byte is the base-3 fraction 0.c0 c1 c2 c3 c4 scaled by 256 and rounded up
+        frac = sum(Fraction(int(t) + 1, 3 ** (e + 1)) for e, t in enumerate(trits))
+        assert B == -((-256 * frac.numerator) // frac.denominator)
+        assert B not in seen
+        seen[B] = tuple(trits)
+        # peeling digits by repeated multiplication by 3 (what a decoder without division does) returns the codes
+        rem = B
+        for t in trits:
+            rem *= 3
+            assert rem >> 8 == int(t) + 1
+            rem &= 255
+        assert np.array_equal(oracle.unpack5(packed, 16, 256), wq)
+    assert len(seen) == 243 and min(seen) == 0 and max(seen) == 255
+    # byte values grow with the base-3 number, and the thirteen values no five codes produce are rejected
+    order = sorted(seen)
+    assert [seen[b] for b in order] == [tuple(c) for c in combos]
+    unused = sorted(set(range(256)) - set(seen))
+    assert len(unused) == 13
+    for b in unused:
+        bad = np.full(16 * 64, 128, np.uint8)
+        bad[5] = b
+        with pytest.raises(ValueError):
+            oracle.unpack5(bad, 16, 256)
+
+
+def test_pack5_size_roundtrip_and_locality():
+    # Table 1's budget: 5 weights per byte where K is a multiple of 320, at most one extra tile of padding otherwise
+    assert oracle.packed5_bytes(2560, 2560) == 2560 * 2560 // 5
+    assert oracle.packed5_bytes(640, 2560) == 640 * 2560 // 5
+    assert oracle.packed5_bytes(2560, 6912) == 2560 * 7040 // 5
+    layer = sum(oracle.packed5_bytes(n, k) for n, k in ((2560, 2560), (640, 2560), (640, 2560), (2560, 2560),
+                                                         (6912, 2560), (6912, 2560), (2560, 6912)))
+    assert layer == 13_959_168 and 30 * layer == 418_775_040  # against 521,011,200 at four per byte
+    assert oracle.packed5_bytes(8, 256) == 0 and oracle.packed5_bytes(16, 100) == 0
+    rng = np.random.default_rng(5)
+    for N, K in ((48, 768), (16, 256), (32, 6912), (640, 2560)):
+        wq = rng.integers(-1, 2, size=(N, K)).astype(np.int8)
+        packed = oracle.pack5(wq)
+        assert packed.size == oracle.packed5_bytes(N, K)
+        assert np.array_equal(oracle.unpack5(packed, N, K), wq)
+    # padding columns hold zero weights: the last tile of a 256-column matrix has 64 of them per row, i.e. whole
+    # words of value 128 wherever all 20 columns of the word are padding (columns 260..319 of the tile)
+    wq = rng.integers(-1, 2, size=(16, 256)).astype(np.int8)
+    tile = oracle.pack5(wq).reshape(2, 8, 4, 4, 4)  # h, g, t, i, b
+    assert np.all(tile[:, :, 3, 1:, :] == 128)  # t = 3 covers columns 240..319: words i = 1..3 are columns 260..319
+    # a 16-byte chunk is 80 consecutive columns of one row: flipping them touches only that chunk
+    wq = rng.integers(-1, 2, size=(48, 768)).astype(np.int8)
+    packed = oracle.pack5(wq)
+    wq2 = wq.copy()
+    wq2[17, 400:480] = -wq2[17, 400:480] + (wq2[17, 400:480] == 0)
+    diff = np.nonzero(oracle.pack5(wq2) != packed)[0]
+    assert diff.size > 0 and diff.min() // 16 == diff.max() // 16
+    with pytest.raises(ValueError):
+        oracle.pack5(np.full((16, 256), 2, np.int8))
+
+
+def test_pack5_identity_and_one_hot_weights_through_the_contraction():
+    # unpack5(pack5(W)) feeds the same contraction: the identity pattern returns the activations themselves, so any
+    # permutation of rows or columns inside the dense layout would show
+    rng = np.random.default_rng(6)
+    K = N = 512
+    q = rng.integers(-127, 128, size=(3, K)).astype(np.int8)
+    eye = np.eye(N, K, dtype=np.int8)
+    w = oracle.unpack5(oracle.pack5(eye), N, K)
+    assert np.array_equal(oracle.matmul_i32(q, w), q.astype(np.int32))
+    w = oracle.unpack5(oracle.pack5(-eye[::-1].copy()), N, K)
+    assert np.array_equal(oracle.matmul_i32(q, w), -q[:, ::-1].astype(np.int32))
+
+
 # --------------------------------------------------------------------------- contraction and epilogue
 
 
