@@ -3,18 +3,25 @@
 // feed-forward block; Section 5.1: decode cost is the packed weight bytes.  Attention is not a BitLinear and is
 // replaced by a fixed stand-in, see bitlinear_glue_attn_standin.)
 //
-// A layer is four dependent levels: {q,k,v}(h), o(a), {gate,up}(h), down(f).  A level's matrices are stacked and their
-// 16-row blocks split evenly over the CTAs (one per SM).  Per level every CTA
-//   1. waits for the level's share of packed weights, which it prefetched into shared memory with bulk copies while
-//      the previous level ran (weight addresses do not depend on activations),
-//   2. waits at a grid barrier for the previous level's outputs, then rebuilds the level's input vector itself
-//      (residual / stand-in / squared-ReLU glue, RMSNorm, absmax int8 quantiser - a few thousand elements, cheaper to
-//      redo per CTA than to exchange),
-//   3. multiplies its row blocks (dot-product-of-four on word & (0x03030303 << 2j), as in the streaming decode kernel),
-//      applies the dequantising epilogue and stores its slice of the level's output.
-// So a token costs 4 x n_layers grid barriers instead of 12 x n_layers kernel launches.
-// Every wait is bounded; on a timeout an abort word makes every CTA leave and BITLINEAR_ERR_TIMEOUT is reported.
+// A layer is four dependent levels: {q,k,v}(h), o(a), {gate,up}(h), down(f).  What a level hands to the next one is a
+// vector of a few thousand values that EVERY CTA needs, so a level boundary is an all-to-all exchange between the CTAs
+// (one per SM); its latency, not the arithmetic, bounds the token.  The kernel is built around making that exchange
+// short:
+//   * The CTA that computes an output row also applies the glue that follows it (residual add, squared-ReLU gate,
+//     attention stand-in) and publishes the NEXT level's input as bf16: 2 bytes per element instead of one or two fp32
+//     vectors.  To keep the glue local, gate row n and up row n belong to the same CTA, and the CTA that owns a block
+//     of q rows computes the v rows the stand-in adds to them itself (v is small; its rows are computed four times).
+//   * Published values carry their own validity: three bf16 values and a 16-bit level tag share one 8-byte word,
+//     written by one store and read by one load, so no fence and no release/acquire pair sits between producer and
+//     consumer.  A relaxed arrival counter only tells the consumers when a look is worthwhile.
+//   * Weights never wait for activations: a copy warp prefetches the CTA's share of the next level into shared memory
+//     with bulk copies while the current level runs.
+// Per level a CTA: waits for the counter, loads the whole input vector once (tags checked, stale words re-read),
+// RMSNorm + absmax int8 quantiser into shared memory, dot-products-of-four over its weight rows, dequantising
+// epilogue + glue, publish.  Every wait is bounded; on a timeout an abort word makes every CTA leave and
+// BITLINEAR_ERR_TIMEOUT is reported.
 #include <algorithm>
+#include <mutex>
 
 #include "quant_row.cuh"
 #include "sm100_sync.cuh"
@@ -28,7 +35,8 @@ constexpr int kChainWarps = kChainThreads / 32;
 constexpr int kChainLaunchThreads = kChainThreads + 32;
 // barrier of the compute threads only (the copy warp runs on its own)
 #define CSYNC() asm volatile("bar.sync 1, 512;" ::: "memory")
-constexpr int kMaxEpt = 16;  // input elements per thread: K <= 8192
+constexpr int kMaxLoads = 3;   // 16-byte loads of the level input per thread: 3 per 16 elements, K <= 8192
+constexpr int kMaxJobs = 12;    // row blocks of weights a CTA multiplies in one level
 
 struct ChainLayerDev {
     const uint8_t* packed[7];    // q k v o gate up down
@@ -40,29 +48,22 @@ struct ChainParams {
     const ChainLayerDev* layers;
     int n_layers, hidden, ffn, n_q, n_kv, head_dim;
     float eps;
-    __nv_bfloat16* h;                 // [hidden] in / out
-    float *q, *k, *v, *o, *g, *u, *dn;  // level outputs (fp32)
-    unsigned* barrier;                // grid barrier counter, zero at launch
-    int* abort_word;                  // zero at launch
+    __nv_bfloat16* h;             // [hidden] in / out
+    float* k;                     // [n_kv * head_dim] the k projection (an output only)
+    // pub[j]: what level j publishes = the input of level j + 1 (of the next layer for j = 3): per 16 elements six
+    // 8-byte words {bf16, bf16, bf16, tag}; word 5 of a group holds one value and two zeros.  Zero at launch.
+    unsigned long long* pub[4];
+    unsigned* counter;            // arrivals, zero at launch: a hint, never relied on for ordering
+    int* abort_word;              // zero at launch
     int* status_word;
-    int buf_bytes;                    // one weight buffer (the largest per-CTA share of a level)
+    int buf_bytes;                // one weight buffer (the largest per-CTA share of a level)
 };
 
-// matrices of a level: indices into the layer's 7, and their row counts
-struct LevelShape {
-    int n_mats, first, K;
-    int rows[3];
-};
-
-__device__ __forceinline__ LevelShape level_shape(int level, const ChainParams& p) {
-    LevelShape s;
-    const int kv = p.n_kv * p.head_dim;
-    if (level == 0) { s.n_mats = 3; s.first = 0; s.K = p.hidden; s.rows[0] = p.hidden; s.rows[1] = kv; s.rows[2] = kv; }
-    else if (level == 1) { s.n_mats = 1; s.first = 3; s.K = p.hidden; s.rows[0] = p.hidden; s.rows[1] = s.rows[2] = 0; }
-    else if (level == 2) { s.n_mats = 2; s.first = 4; s.K = p.hidden; s.rows[0] = p.ffn; s.rows[1] = p.ffn; s.rows[2] = 0; }
-    else { s.n_mats = 1; s.first = 6; s.K = p.ffn; s.rows[0] = p.hidden; s.rows[1] = s.rows[2] = 0; }
-    return s;
-}
+// Level shapes.  A "unit" is one block of 16 output rows of the level's result vector together with every weight row
+// block needed to finish it: level 0 - a q block and the matching v block (units 0 .. hidden/16) or a k block (the
+// units after those); level 1 - an o block; level 2 - a gate block and the up block of the same rows; level 3 - a down
+// block.  Units are split over the CTAs by weight (bytes of packed rows).
+__device__ __forceinline__ int level_K(int level, const ChainParams& p) { return level == 3 ? p.ffn : p.hidden; }
 
 __device__ __forceinline__ int dp4a_u8_s8(uint32_t a_u8x4, uint32_t b_s8x4, int c) {
     int d;
@@ -74,41 +75,92 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
     return v;
 }
-// bypass L1: written by other CTAs
-__device__ __forceinline__ float ldcg_f32(const float* p) { return __ldcg(p); }
-__device__ __forceinline__ float4 ldcg_f32x4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+// Two published words: each 8-byte half is read atomically and carries its own tag.  Bypasses L1 (written by other SMs).
+__device__ __forceinline__ void ld_pub2(const unsigned long long* p, unsigned long long& a, unsigned long long& b) {
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0,%1}, [%2];" : "=l"(a), "=l"(b) : "l"(p) : "memory");
+}
+__device__ __forceinline__ void st_pub(unsigned long long* p, unsigned long long v) {
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
 
 struct BlockScratch {
-    double sq[kChainWarps];
+    float sq_hi[kChainWarps], sq_lo[kChainWarps];
     float mx[kChainWarps];
     int sum[kChainWarps];
-    float r, d;
-    int xsum;
-    int ok;
+    float r;
+    int ok;          // CTA-local abort flag
     int desc_ready;  // highest layer whose descriptor is in shared memory
-    int rb_lo[4], rb_hi[4];  // this CTA's share of the row blocks of each of the four levels of a layer
+    // this CTA's units of each level: [u_lo, u_hi); level 0 has a second range of k units [k_lo, k_hi)
+    int u_lo[4], u_hi[4], k_lo, k_hi;
 };
 
 __device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ uint32_t bf16_bits_rn(float x) { return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(x)); }
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
-// Same rounding as the stand-alone quantisers (see round_code in quant_row.cuh): low byte = int8 code.
-__device__ __forceinline__ uint32_t chain_round_code(float v) { return __float_as_uint(__fadd_rn(v, 12582912.0f)); }
+// Error-free accumulation of fp32 values that are exact squares: (hi, lo) += x.
+__device__ __forceinline__ void acc_pair(float& hi, float& lo, float x_hi, float x_lo) {
+    const float s = __fadd_rn(hi, x_hi);
+    const float bb = __fsub_rn(s, hi);
+    const float err = __fadd_rn(__fsub_rn(hi, __fsub_rn(s, bb)), __fsub_rn(x_hi, bb));
+    lo = __fadd_rn(lo, __fadd_rn(err, x_lo));
+    hi = s;
+}
 
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
+// Which packed matrix and which of its 16-row blocks job j of this CTA's level is; unit_local / part say where its
+// accumulators go in the epilogue.
+struct Job {
+    int mat, rb;
+};
+__device__ __forceinline__ int v_block_of_q_block(int q_rb, const ChainParams& p) {
+    const int per_head = p.head_dim / kTileRows;
+    const int head = q_rb / per_head, jb = q_rb - head * per_head;
+    return (head / (p.n_q / p.n_kv)) * per_head + jb;
+}
+__device__ __forceinline__ int level_jobs(int level, const BlockScratch* sc) {
+    const int n = sc->u_hi[level] - sc->u_lo[level];
+    if (level == 0) return 2 * n + (sc->k_hi - sc->k_lo);
+    return level == 2 ? 2 * n : n;
+}
+__device__ __forceinline__ Job level_job(int level, int j, const BlockScratch* sc, const ChainParams& p) {
+    Job jb;
+    if (level == 0) {
+        const int nqv = sc->u_hi[0] - sc->u_lo[0];
+        if (j < 2 * nqv) {
+            const int unit = sc->u_lo[0] + (j >> 1);
+            jb.mat = (j & 1) ? 2 : 0;
+            jb.rb = (j & 1) ? v_block_of_q_block(unit, p) : unit;
+        } else {
+            jb.mat = 1;
+            jb.rb = sc->k_lo + (j - 2 * nqv);
+        }
+    } else if (level == 1) {
+        jb.mat = 3;
+        jb.rb = sc->u_lo[1] + j;
+    } else if (level == 2) {
+        jb.mat = 4 + (j & 1);
+        jb.rb = sc->u_lo[2] + (j >> 1);
+    } else {
+        jb.mat = 6;
+        jb.rb = sc->u_lo[3] + j;
+    }
+    return jb;
 }
 
 __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(const ChainParams p) {
     extern __shared__ __align__(1024) uint8_t smem[];
     const int kmax = p.hidden > p.ffn ? p.hidden : p.ffn;
-    const int max_rb = p.buf_bytes / ((p.hidden / kTileCols) * kTileBytes);  // most row blocks a CTA can own in a level
     uint8_t* wbuf = smem;                                                      // [2][buf_bytes]
     uint8_t* xq_s = wbuf + 2 * (size_t)p.buf_bytes;                            // [kmax] int8 codes, lane-interleaved
     __nv_bfloat16* h_s = reinterpret_cast<__nv_bfloat16*>(xq_s + kmax);        // [hidden] running hidden state
-    int* acc_s = reinterpret_cast<int*>(h_s + p.hidden);                       // [max_rb][16]
-    ChainLayerDev* desc_s = reinterpret_cast<ChainLayerDev*>(acc_s + (size_t)max_rb * 16);  // [2]
+    int* acc_s = reinterpret_cast<int*>(h_s + p.hidden);                       // [kMaxJobs][16]
+    ChainLayerDev* desc_s = reinterpret_cast<ChainLayerDev*>(acc_s + kMaxJobs * 16);  // [2]
     float* sw_s = reinterpret_cast<float*>(desc_s + 2);                        // [2][8]
     uint64_t* bars = reinterpret_cast<uint64_t*>(sw_s + 16);                   // [2] weight buffer landed, [2] buffer read
     BlockScratch* sc = reinterpret_cast<BlockScratch*>(bars + 4);
@@ -118,20 +170,26 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
     const int g = lane >> 2, t = lane & 3;
     const int grid = (int)gridDim.x, cta = (int)blockIdx.x;
     const int total_levels = 4 * p.n_layers;
-    const int group = p.n_q / p.n_kv;
 
-    // ---- prologue: barriers, first descriptor, its scales, the hidden state ----
+    // ---- prologue: barriers, first descriptor, its scales, the hidden state, this CTA's shares ----
     if (tid == 0) {
         for (int b = 0; b < 4; ++b) mbar_init(smem_u32(bars + b), 1);
         sc->ok = 0;
         sc->desc_ready = 0;
         mbar_init_fence();
-    }
-    if (tid < 4) {  // the shares do not change from layer to layer: two 64-bit divisions per level, once
-        const LevelShape s = level_shape(tid, p);
-        const int total_rb = (s.rows[0] + s.rows[1] + s.rows[2]) / kTileRows;
-        sc->rb_lo[tid] = (int)((long long)total_rb * cta / grid);
-        sc->rb_hi[tid] = (int)((long long)total_rb * (cta + 1) / grid);
+        // level 0: q+v units weigh two row blocks, k units one; a unit belongs to the CTA in whose weight range it starts
+        const int nq = p.hidden / kTileRows, nk = p.n_kv * p.head_dim / kTileRows;
+        const long long w_total = 2LL * nq + nk;
+        const int w_lo = (int)(w_total * cta / grid), w_hi = (int)(w_total * (cta + 1) / grid);
+        const int q_lo_w = w_lo < 2 * nq ? w_lo : 2 * nq, q_hi_w = w_hi < 2 * nq ? w_hi : 2 * nq;
+        sc->u_lo[0] = (q_lo_w + 1) / 2;
+        sc->u_hi[0] = (q_hi_w + 1) / 2;
+        sc->k_lo = (w_lo > 2 * nq ? w_lo : 2 * nq) - 2 * nq;
+        sc->k_hi = (w_hi > 2 * nq ? w_hi : 2 * nq) - 2 * nq;
+        const int n1 = p.hidden / kTileRows, n2 = p.ffn / kTileRows;
+        sc->u_lo[1] = (int)((long long)n1 * cta / grid); sc->u_hi[1] = (int)((long long)n1 * (cta + 1) / grid);
+        sc->u_lo[2] = (int)((long long)n2 * cta / grid); sc->u_hi[2] = (int)((long long)n2 * (cta + 1) / grid);
+        sc->u_lo[3] = sc->u_lo[1]; sc->u_hi[3] = sc->u_hi[1];
     }
     {
         const uint32_t* src = reinterpret_cast<const uint32_t*>(p.layers);
@@ -143,26 +201,19 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
     if (tid < 7) sw_s[tid] = *desc_s[0].s_w[tid];
     __syncthreads();
 
-    // bulk copies of this CTA's share of level L into weight buffer L & 1 (warp 0, all lanes)
+    // bulk copies of this CTA's share of level L into weight buffer L & 1 (the copy warp, all lanes)
     auto issue_level = [&](int L) {
         const int layer = L >> 2, level = L & 3;
-        const LevelShape s = level_shape(level, p);
         const ChainLayerDev& dsc = desc_s[layer & 1];
-        const int total_rb = (s.rows[0] + s.rows[1] + s.rows[2]) / kTileRows;
-        const int lo = sc->rb_lo[level], hi = sc->rb_hi[level];
-        const uint32_t rb_bytes = (uint32_t)(s.K / kTileCols) * kTileBytes;
+        const int n_jobs = level_jobs(level, sc);
+        const uint32_t rb_bytes = (uint32_t)(level_K(level, p) / kTileCols) * kTileBytes;
         const uint32_t bar = smem_u32(bars + (L & 1));
-        if (lane == 0) mbar_expect_tx(bar, (uint32_t)(hi - lo) * rb_bytes);
+        if (lane == 0) mbar_expect_tx(bar, (uint32_t)n_jobs * rb_bytes);
         __syncwarp();
-        for (int i = lane; i < hi - lo; i += 32) {
-            int row = (lo + i) * kTileRows, m = 0;
-            if (row >= s.rows[0]) {  // which of the level's stacked matrices (no indexed array: it would live in local memory)
-                row -= s.rows[0];
-                m = 1;
-                if (row >= s.rows[1]) { row -= s.rows[1]; m = 2; }
-            }
-            bulk_load(smem_u32(wbuf + (size_t)(L & 1) * p.buf_bytes) + (uint32_t)i * rb_bytes,
-                      dsc.packed[s.first + m] + (size_t)(row / kTileRows) * rb_bytes, rb_bytes, bar);
+        for (int j = lane; j < n_jobs; j += 32) {
+            const Job jb = level_job(level, j, sc, p);
+            bulk_load(smem_u32(wbuf + (size_t)(L & 1) * p.buf_bytes) + (uint32_t)j * rb_bytes,
+                      dsc.packed[jb.mat] + (size_t)jb.rb * rb_bytes, rb_bytes, bar);
         }
     };
     bool ok = true;
@@ -183,13 +234,11 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
     } else
     for (int L = 0; L < total_levels && ok; ++L) {
         const int layer = L >> 2, level = L & 3;
-        const LevelShape s = level_shape(level, p);
-        const int K = s.K, k_tiles = K / kTileCols;
-        const int total_rb = (s.rows[0] + s.rows[1] + s.rows[2]) / kTileRows;
-        const int rb_lo = sc->rb_lo[level], rb_hi = sc->rb_hi[level];
-        const int n_rb = rb_hi - rb_lo;
+        const int K = level_K(level, p), k_tiles = K / kTileCols;
+        const int n_jobs = level_jobs(level, sc);
+        const unsigned tag = (unsigned)L & 0xffffu;  // what the producers of this level's input wrote: their level + 1
 
-        // ---- descriptor / scale prefetch for the next layer, weight prefetch for the next level ----
+        // ---- descriptor / scale prefetch for the next layer ----
         if (level == 3 || level == 0) {  // level 3 needs the next layer's descriptor, level 0 this layer's scales
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             CSYNC();
@@ -211,13 +260,31 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
 
-        // ---- wait for the outputs of the previous level (grid barrier, bounded) ----
+        // ---- the gains of this level's input: loads issued before the wait so that they overlap it ----
+        // Load index l = tid + i * 512 covers elements 16 * (l / 3) + 6 * (l % 3) + 0..5 (the last of the three covers four).
+        const __nv_bfloat16* gain = desc_s[layer & 1].gain[level];
+        const int n_loads = 3 * (K / kTileRows);
+        uint32_t gw[kMaxLoads][3];
+#pragma unroll
+        for (int i = 0; i < kMaxLoads; ++i) {
+            const int l = tid + i * kChainThreads;
+            gw[i][0] = gw[i][1] = gw[i][2] = 0x3f803f80u;  // bf16 ones
+            if (gain != nullptr && l < n_loads) {
+                const int rb = l / 3, part = l - 3 * rb;
+                const uint32_t* gp = reinterpret_cast<const uint32_t*>(gain + rb * kTileRows + 6 * part);
+                gw[i][0] = gp[0];
+                gw[i][1] = gp[1];
+                if (part < 2) gw[i][2] = gp[2];
+            }
+        }
+
+        // ---- wait until the arrival counter says that a look at the input is worthwhile (bounded) ----
         if (L > 0) {
             if (tid == 0) {
                 const unsigned target = (unsigned)grid * (unsigned)L;
                 const unsigned long long t0 = globaltimer_ns();
                 unsigned spins = 0;
-                while (ld_acquire_u32(p.barrier) < target) {
+                while (ld_relaxed_u32(p.counter) < target) {
                     if ((++spins & 255u) == 0u) {
                         if (*reinterpret_cast<volatile int*>(p.abort_word) != 0) { sc->ok = 1; break; }
                         if (globaltimer_ns() - t0 > kWaitLimitNs) {
@@ -231,93 +298,92 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             CSYNC();
             if (sc->ok) { ok = false; break; }
         }
+        if (tid < kMaxJobs * 16) acc_s[tid] = 0;
 
-        // ---- build this level's input vector (glue), RMSNorm, absmax int8 quantiser ----
-        for (int i = tid; i < n_rb * 16; i += kChainThreads) acc_s[i] = 0;
-        const __nv_bfloat16* gain = desc_s[layer & 1].gain[level];
-        float xv[kMaxEpt], gv[kMaxEpt];
-        // Element e of this thread is column 4 * (tid + (e / 4) * kChainThreads) + e % 4: four consecutive columns per
-        // 16-byte load.  Every load of the stage is issued before anything is computed, so the L2 round trips overlap.
-        float ra[kMaxEpt], rb[kMaxEpt];
+        // ---- the level's input: every word checked against the level tag, stale words read again ----
+        float xv[kMaxLoads][6];
+        if (L == 0) {
 #pragma unroll
-        for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
-            const int i0 = 4 * (tid + q4 * kChainThreads);
-            const bool in = i0 < K;  // K is a multiple of 4: a group of four is inside or outside as a whole
-            float4 va = make_float4(0.0f, 0.0f, 0.0f, 0.0f), vb = va;
-            if (in) {
-                if (level == 0) {
-                    if (layer > 0) va = ldcg_f32x4(p.dn + i0);
-                } else if (level == 1) {
-                    const int head = i0 / p.head_dim, j = i0 - head * p.head_dim;  // head_dim is a multiple of 4
-                    va = ldcg_f32x4(p.q + i0);
-                    vb = ldcg_f32x4(p.v + (head / group) * p.head_dim + j);
-                } else if (level == 2) {
-                    va = ldcg_f32x4(p.o + i0);
-                } else {
-                    va = ldcg_f32x4(p.g + i0);
-                    vb = ldcg_f32x4(p.u + i0);
-                }
-            }
-            ra[4 * q4] = va.x; ra[4 * q4 + 1] = va.y; ra[4 * q4 + 2] = va.z; ra[4 * q4 + 3] = va.w;
-            rb[4 * q4] = vb.x; rb[4 * q4 + 1] = vb.y; rb[4 * q4 + 2] = vb.z; rb[4 * q4 + 3] = vb.w;
-            if (gain != nullptr && in) {
-                const uint2 gw = *reinterpret_cast<const uint2*>(gain + i0);
-                gv[4 * q4] = __uint_as_float(gw.x << 16);
-                gv[4 * q4 + 1] = __uint_as_float(gw.x & 0xffff0000u);
-                gv[4 * q4 + 2] = __uint_as_float(gw.y << 16);
-                gv[4 * q4 + 3] = __uint_as_float(gw.y & 0xffff0000u);
-            } else {
-                gv[4 * q4] = gv[4 * q4 + 1] = gv[4 * q4 + 2] = gv[4 * q4 + 3] = 1.0f;
-            }
-        }
-        double sq = 0.0;
+            for (int i = 0; i < kMaxLoads; ++i) {
+                const int l = tid + i * kChainThreads;
+                const int rb = l / 3, part = l - 3 * rb, e0 = rb * kTileRows + 6 * part;
 #pragma unroll
-        for (int e = 0; e < kMaxEpt; ++e) {
-            const int i = 4 * (tid + (e >> 2) * kChainThreads) + (e & 3);
-            float x = 0.0f;
-            if (i < K) {
-                if (level == 0) {
-                    x = __bfloat162float(h_s[i]);
-                    if (layer > 0) {
-                        x = bf16_round(__fadd_rn(x, ra[e]));
-                        h_s[i] = __float2bfloat16_rn(x);
+                for (int e = 0; e < 6; ++e)
+                    xv[i][e] = (l < n_loads && 6 * part + e < kTileRows) ? __bfloat162float(h_s[e0 + e]) : 0.0f;
+            }
+        } else {
+            const unsigned long long* src = p.pub[(level + 3) & 3];
+            unsigned long long wa[kMaxLoads], wb[kMaxLoads];
+#pragma unroll
+            for (int i = 0; i < kMaxLoads; ++i) {
+                const int l = tid + i * kChainThreads;
+                wa[i] = wb[i] = (unsigned long long)tag << 48;
+                if (l < n_loads) ld_pub2(src + 2 * l, wa[i], wb[i]);
+            }
+#pragma unroll
+            for (int i = 0; i < kMaxLoads; ++i) {
+                const int l = tid + i * kChainThreads;
+                if (l < n_loads && ((unsigned)(wa[i] >> 48) != tag || (unsigned)(wb[i] >> 48) != tag)) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    unsigned spins = 0;
+                    for (;;) {
+                        ld_pub2(src + 2 * l, wa[i], wb[i]);
+                        if ((unsigned)(wa[i] >> 48) == tag && (unsigned)(wb[i] >> 48) == tag) break;
+                        if ((++spins & 15u) == 0u) {
+                            if (*reinterpret_cast<volatile int*>(p.abort_word) != 0) { sc->ok = 1; break; }
+                            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+                                atomicExch(p.abort_word, 1);
+                                sc->ok = 1;
+                                break;
+                            }
+                        }
                     }
-                } else if (level == 1) {
-                    x = bf16_round(__fadd_rn(ra[e], rb[e]));
-                } else if (level == 2) {
-                    x = bf16_round(__fadd_rn(__bfloat162float(h_s[i]), ra[e]));
-                    h_s[i] = __float2bfloat16_rn(x);
-                } else {
-                    const float r = fmaxf(ra[e], 0.0f);
-                    x = bf16_round(__fmul_rn(__fmul_rn(r, r), rb[e]));
+                }
+                const uint32_t a0 = (uint32_t)wa[i], a1 = (uint32_t)(wa[i] >> 32), b0 = (uint32_t)wb[i], b1 = (uint32_t)(wb[i] >> 32);
+                xv[i][0] = bf16_lo(a0); xv[i][1] = bf16_hi(a0); xv[i][2] = bf16_lo(a1);
+                xv[i][3] = bf16_lo(b0); xv[i][4] = bf16_hi(b0); xv[i][5] = bf16_lo(b1);
+                if ((level == 0 || level == 2) && l < n_loads) {
+                    // the input of levels 0 and 2 is the hidden state itself: keep it for the residual adds of this CTA's rows
+                    const int rb = l / 3, part = l - 3 * rb;
+                    uint16_t* hp = reinterpret_cast<uint16_t*>(h_s) + rb * kTileRows + 6 * part;
+                    hp[0] = (uint16_t)a0; hp[1] = (uint16_t)(a0 >> 16); hp[2] = (uint16_t)a1; hp[3] = (uint16_t)b0;
+                    if (part < 2) { hp[4] = (uint16_t)(b0 >> 16); hp[5] = (uint16_t)b1; }
                 }
             }
-            xv[e] = x;
         }
-        {   // sum of squares: error-free fp32 chains of eight, then fp64 (see sum_squares8)
-            float lo8[8], hi8[8];
+
+        // ---- RMSNorm: sum of the exact squares as an error-free pair of fp32, root in fp64 by one thread ----
+        float s_hi = 0.0f, s_lo = 0.0f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) { lo8[e] = xv[e]; hi8[e] = xv[8 + e]; }
-            sq = sum_squares8(lo8);
-            if (K > 8 * kChainThreads) sq += sum_squares8(hi8);
+        for (int i = 0; i < kMaxLoads; ++i)
+#pragma unroll
+            for (int e = 0; e < 6; ++e) acc_pair(s_hi, s_lo, __fmul_rn(xv[i][e], xv[i][e]), 0.0f);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float o_hi = __shfl_xor_sync(0xffffffffu, s_hi, o), o_lo = __shfl_xor_sync(0xffffffffu, s_lo, o);
+            acc_pair(s_hi, s_lo, o_hi, o_lo);
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-        if (lane == 0) sc->sq[warp] = sq;
+        if (lane == 0) { sc->sq_hi[warp] = s_hi; sc->sq_lo[warp] = s_lo; }
         CSYNC();
+        if (sc->ok) { if (tid == 0) atomicExch(p.abort_word, 1); ok = false; break; }  // a tag wait ran out
         if (tid == 0) {
             double S = 0.0;
 #pragma unroll
-            for (int w = 0; w < kChainWarps; ++w) S += sc->sq[w];
+            for (int w = 0; w < kChainWarps; ++w) S += (double)sc->sq_hi[w] + (double)sc->sq_lo[w];
             sc->r = (float)(1.0 / sqrt(S / (double)K + (double)p.eps));
         }
         CSYNC();
         const float r = sc->r;
         float amax = 0.0f;
 #pragma unroll
-        for (int e = 0; e < kMaxEpt; ++e) {
-            xv[e] = __fmul_rn(__fmul_rn(xv[e], r), gv[e]);  // the normalised value
-            amax = fmaxf(amax, fabsf(xv[e]));
+        for (int i = 0; i < kMaxLoads; ++i) {
+            const float gv[6] = {bf16_lo(gw[i][0]), bf16_hi(gw[i][0]), bf16_lo(gw[i][1]),
+                                 bf16_hi(gw[i][1]), bf16_lo(gw[i][2]), bf16_hi(gw[i][2])};
+#pragma unroll
+            for (int e = 0; e < 6; ++e) {
+                xv[i][e] = __fmul_rn(__fmul_rn(xv[i][e], r), gv[e]);  // the normalised value (0 where there is no element)
+                amax = fmaxf(amax, fabsf(xv[i][e]));
+            }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
@@ -329,37 +395,51 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         const float sc_q = __fdiv_rn(127.0f, a), d = __fdiv_rn(a, 127.0f);
         int csum = 0;
 #pragma unroll
-        for (int q4 = 0; q4 < kMaxEpt / 4; ++q4) {
-            const int i0 = 4 * (tid + q4 * kChainThreads);
-            if (i0 < K) {
-                const uint32_t word = pack_codes4(chain_round_code(__fmul_rn(xv[4 * q4], sc_q)), chain_round_code(__fmul_rn(xv[4 * q4 + 1], sc_q)),
-                                                  chain_round_code(__fmul_rn(xv[4 * q4 + 2], sc_q)), chain_round_code(__fmul_rn(xv[4 * q4 + 3], sc_q)), csum);
-                // lane-interleaved order inside each block of 256 columns: piece 4t+q -> byte 64q + 16t; four consecutive
-                // columns stay together inside their 16-byte piece
-                const int blk = i0 & ~255, rr = i0 & 255;
-                *reinterpret_cast<uint32_t*>(xq_s + blk + 64 * ((rr >> 4) & 3) + 16 * (rr >> 6) + (rr & 15)) = word;
+        for (int i = 0; i < kMaxLoads; ++i) {
+            const int l = tid + i * kChainThreads;
+            if (l < n_loads) {
+                const int rb = l / 3, part = l - 3 * rb, c0 = rb * kTileRows;
+                uint32_t c[6];
+#pragma unroll
+                for (int e = 0; e < 6; ++e) c[e] = round_code(__fmul_rn(xv[i][e], sc_q));
+                // the 16 codes of a row block are one 16-byte piece of the lane-interleaved order (piece 4t+q of a block
+                // of 256 columns at byte 64q + 16t); this thread owns bytes 6 * part .. of it
+                const int blk = c0 & ~255, rr = c0 & 255;
+                uint8_t* piece = xq_s + blk + 64 * ((rr >> 4) & 3) + 16 * (rr >> 6);
+                const uint32_t w4 = pack_codes4(c[0], c[1], c[2], c[3], csum);
+                if (part == 0) {
+                    *reinterpret_cast<uint32_t*>(piece) = w4;
+                    const uint32_t w2 = pack_codes4(c[4], c[5], 0u, 0u, csum);
+                    *reinterpret_cast<uint16_t*>(piece + 4) = (uint16_t)w2;
+                } else if (part == 1) {
+                    // bytes 6..11: codes 0,1 then 2..5
+                    const uint32_t w2 = pack_codes4(c[4], c[5], 0u, 0u, csum);
+                    *reinterpret_cast<uint16_t*>(piece + 6) = (uint16_t)w4;
+                    *reinterpret_cast<uint32_t*>(piece + 8) = (w4 >> 16) | (w2 << 16);
+                } else {
+                    *reinterpret_cast<uint32_t*>(piece + 12) = w4;
+                }
             }
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xffffffffu, csum, o);
         if (lane == 0) sc->sum[warp] = csum;
-        CSYNC();
-        int xsum = 0;
-#pragma unroll
-        for (int w = 0; w < kChainWarps; ++w) xsum += sc->sum[w];
 
         // ---- the level's weights: wait for the prefetched share, multiply ----
         mbar_wait(smem_u32(bars + (L & 1)), (uint32_t)(L >> 1) & 1u, abort_s);
-        CSYNC();
+        CSYNC();  // codes, code sums and the zeroed accumulators are visible; every thread has passed the weight wait
         if (sc->ok) {  // the copy did not land in time: tell the other CTAs and leave
             if (tid == 0) atomicExch(p.abort_word, 1);
             ok = false;
             break;
         }
+        int xsum = 0;
+#pragma unroll
+        for (int w = 0; w < kChainWarps; ++w) xsum += sc->sum[w];
         const uint32_t buf_s = smem_u32(wbuf + (size_t)(L & 1) * p.buf_bytes);
         const uint32_t xq_a = smem_u32(xq_s) + 16u * t;
-        for (int tix = warp; tix < n_rb * k_tiles; tix += kChainWarps) {
-            const int rbl = tix / k_tiles, kt = tix - rbl * k_tiles;
+        for (int tix = warp; tix < n_jobs * k_tiles; tix += kChainWarps) {
+            const int job = tix / k_tiles, kt = tix - job * k_tiles;
             const uint4 w0v = lds128(buf_s + (uint32_t)tix * kTileBytes + 16u * lane);
             const uint4 w1v = lds128(buf_s + (uint32_t)tix * kTileBytes + 512u + 16u * lane);
             const uint32_t w0[4] = {w0v.x, w0v.y, w0v.z, w0v.w};
@@ -383,53 +463,61 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
                 sum = sum * 4 + acc[hh][3];
                 sum += __shfl_xor_sync(0xffffffffu, sum, 1);
                 sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-                if (t == 0) atomicAdd(&acc_s[rbl * 16 + 8 * hh + g], sum >> 6);
+                if (t == 0) atomicAdd(&acc_s[job * 16 + 8 * hh + g], sum >> 6);
             }
         }
         CSYNC();
         if (tid == 0) mbar_arrive(smem_u32(bars + 2 + (L & 1)));  // the buffer has been read: it may be refilled
 
-        // ---- dequantising epilogue: this CTA's rows of the level's output ----
-        for (int o = tid; o < n_rb * 16; o += kChainThreads) {
-            int row = (rb_lo + (o >> 4)) * kTileRows + (o & 15), m = 0;
-            if (row >= s.rows[0]) {  // which of the level's stacked matrices (no indexed array: it would live in local memory)
-                row -= s.rows[0];
-                m = 1;
-                if (row >= s.rows[1]) { row -= s.rows[1]; m = 2; }
+        // ---- dequantising epilogue + the glue that follows this level, published as the next level's input ----
+        // One thread per published word: three consecutive rows of a unit (the sixth word of a unit holds one row).
+        {
+            const int n_units = sc->u_hi[level] - sc->u_lo[level];
+            const float* sw = sw_s + 8 * (layer & 1);
+            const bool last = L + 1 == total_levels;
+            if (tid < 6 * n_units) {
+                const int ul = tid / 6, wd = tid - 6 * ul, unit = sc->u_lo[level] + ul;
+                const int jpu = (level == 0 || level == 2) ? 2 : 1;  // jobs per unit
+                uint32_t bits[3] = {0u, 0u, 0u};
+#pragma unroll
+                for (int e = 0; e < 3; ++e) {
+                    const int row16 = 3 * wd + e;
+                    if (row16 < kTileRows) {
+                        const int row = unit * kTileRows + row16;
+                        const float y0 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * jpu) * 16 + row16] - xsum),
+                                                             sw[level == 0 ? 0 : (level == 1 ? 3 : (level == 2 ? 4 : 6))]), d);
+                        float val;
+                        if (level == 0) {
+                            const float y1 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * 2 + 1) * 16 + row16] - xsum), sw[2]), d);
+                            val = __fadd_rn(y0, y1);  // attention stand-in: q + v of the matching KV head
+                        } else if (level == 2) {
+                            const float y1 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * 2 + 1) * 16 + row16] - xsum), sw[5]), d);
+                            const float rl = fmaxf(y0, 0.0f);
+                            val = __fmul_rn(__fmul_rn(rl, rl), y1);  // squared-ReLU gate times up
+                        } else {
+                            val = __fadd_rn(__bfloat162float(h_s[row]), y0);  // residual
+                        }
+                        bits[e] = bf16_bits_rn(val);
+                        if (last) reinterpret_cast<uint16_t*>(p.h)[row] = (uint16_t)bits[e];
+                    }
+                }
+                if (!last)
+                    st_pub(p.pub[level] + 6 * (size_t)unit + wd,
+                           (unsigned long long)(bits[0] | (bits[1] << 16)) |
+                               ((unsigned long long)(bits[2] | (((unsigned)(L + 1) & 0xffffu) << 16)) << 32));
             }
-            float* y;
-            if (level == 0) y = m == 0 ? p.q : (m == 1 ? p.k : p.v);
-            else if (level == 1) y = p.o;
-            else if (level == 2) y = m == 0 ? p.g : p.u;
-            else y = p.dn;
-            const float s_w = sw_s[8 * (layer & 1) + s.first + m];
-            y[row] = __fmul_rn(__fmul_rn((float)(acc_s[o] - xsum), s_w), d);
+            if (level == 0) {  // k rows: an output of the layer, consumed by nobody here
+                const int nqv = sc->u_hi[0] - sc->u_lo[0], nk = sc->k_hi - sc->k_lo;
+                const int o = tid - 6 * n_units;
+                if (o >= 0 && o < nk * 16)
+                    p.k[(sc->k_lo + (o >> 4)) * kTileRows + (o & 15)] =
+                        __fmul_rn(__fmul_rn((float)(acc_s[(2 * nqv + (o >> 4)) * 16 + (o & 15)] - xsum), sw[1]), d);
+            }
+            // arrival hint (not ordered with the stores above: the tags say when the data is there)
+            if (tid == 0 && !last) asm volatile("red.relaxed.gpu.global.add.u32 [%0], 1;" ::"l"(p.counter) : "memory");
         }
-        CSYNC();
-        // release at GPU scope: the stores of every thread of the CTA (ordered before this by the barrier above) are
-        // visible to whoever acquires the new count
-        if (tid == 0) asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.barrier) : "memory");
     }
 
-    // ---- after the last level: the final residual, written by CTA 0 ----
-    if (warp < kChainWarps && ok && cta == 0) {
-        if (tid == 0) {
-            const unsigned target = (unsigned)grid * (unsigned)total_levels;
-            const unsigned long long t0 = globaltimer_ns();
-            unsigned spins = 0;
-            while (ld_acquire_u32(p.barrier) < target) {
-                if ((++spins & 255u) == 0u && (globaltimer_ns() - t0 > kWaitLimitNs || *reinterpret_cast<volatile int*>(p.abort_word))) {
-                    atomicExch(p.abort_word, 1);
-                    sc->ok = 1;
-                    break;
-                }
-            }
-        }
-        CSYNC();
-        if (!sc->ok)
-            for (int i = tid; i < p.hidden; i += kChainThreads)
-                p.h[i] = __float2bfloat16_rn(__fadd_rn(__bfloat162float(h_s[i]), ldcg_f32(p.dn + i)));
-    }
     __syncthreads();
     if (!ok || sc->ok) abort_drain();  // bulk copies of this CTA may still be in flight
     if (tid == 0 && cta == 0 && *reinterpret_cast<volatile int*>(p.abort_word) != 0 && p.status_word != nullptr)
@@ -437,7 +525,7 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
 }
 
 struct ChainLayout {
-    size_t layers_off, out_off[7], sync_off, total;
+    size_t layers_off, k_off, pub_off[4], sync_off, zero_begin, zero_bytes, total;
 };
 
 ChainLayout chain_layout(int n_layers, int hidden, int ffn, int kv) {
@@ -445,22 +533,54 @@ ChainLayout chain_layout(int n_layers, int hidden, int ffn, int kv) {
     size_t off = 0;
     L.layers_off = off;
     off = align_up(off + (size_t)n_layers * sizeof(ChainLayerDev), 256);
-    const int widths[7] = {hidden, kv, kv, hidden, ffn, ffn, hidden};  // q k v o g u dn
-    for (int i = 0; i < 7; ++i) {
-        L.out_off[i] = off;
-        off = align_up(off + (size_t)widths[i] * sizeof(float), 256);
+    L.k_off = off;
+    off = align_up(off + (size_t)kv * sizeof(float), 256);
+    L.zero_begin = off;  // everything from here on is cleared at every launch: tags and the sync words
+    const int widths[4] = {hidden, hidden, ffn, hidden};  // a, h after attention, f, h after the feed-forward block
+    for (int i = 0; i < 4; ++i) {
+        L.pub_off[i] = off;
+        off = align_up(off + (size_t)(widths[i] / kTileRows) * 6 * sizeof(unsigned long long), 256);
     }
     L.sync_off = off;
     off += 256;
+    L.zero_bytes = off - L.zero_begin;
     L.total = off;
     return L;
 }
 
 bool chain_dims_ok(int n_layers, int hidden, int ffn, int n_q, int n_kv, int hd) {
-    if (n_layers <= 0 || n_q <= 0 || n_kv <= 0 || hd <= 0 || n_q % n_kv) return false;
-    if (hidden != n_q * hd || (n_kv * hd) % kTileRows || hd % 4) return false;  // 16-byte loads never straddle a head
-    return shape_ok(hidden, hidden) && shape_ok(ffn, hidden) && shape_ok(hidden, ffn) && hidden <= kMaxEpt * kChainThreads &&
-           ffn <= kMaxEpt * kChainThreads;
+    if (n_layers <= 0 || n_layers > 16000 || n_q <= 0 || n_kv <= 0 || hd <= 0 || n_q % n_kv) return false;
+    if (hidden != n_q * hd || hd % kTileRows) return false;  // a block of 16 q rows lies inside one head
+    return shape_ok(hidden, hidden) && shape_ok(ffn, hidden) && shape_ok(hidden, ffn) &&
+           3 * (hidden / kTileRows) <= kMaxLoads * kChainThreads && 3 * (ffn / kTileRows) <= kMaxLoads * kChainThreads;
+}
+
+// Per-device facts, looked up once per device (a process may drive several GPUs).
+struct ChainDevice {
+    int sm_count = 0, coop = 0, major = 0;
+    bool known = false;
+};
+int chain_device(ChainDevice& out) {
+    static ChainDevice cache[64];
+    static std::mutex mu;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    ChainDevice& c = cache[dev];
+    if (!c.known) {
+        if (cudaDeviceGetAttribute(&c.major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&c.coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&c.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return BITLINEAR_ERR_CUDA;
+        }
+        c.known = true;
+    }
+    out = c;
+    return BITLINEAR_OK;
 }
 
 }  // namespace
@@ -493,20 +613,10 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
             if (!aligned16(layers[l].packed[j]) || (j < 4 && layers[l].gain[j] && !aligned16(layers[l].gain[j])))
                 return BITLINEAR_ERR_ALIGN;
         }
-    static int sm_count = 0, coop = 0;
-    if (sm_count == 0) {
-        int dev = 0, major = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-            cudaGetLastError();
-            sm_count = 0;
-            return BITLINEAR_ERR_CUDA;
-        }
-        if (major != 10) { sm_count = 0; return BITLINEAR_ERR_ARCH; }
-    }
-    if (!coop) return BITLINEAR_ERR_CUDA;
+    ChainDevice devinfo;
+    if (const int rc = chain_device(devinfo)) return rc;
+    if (devinfo.major != 10) return BITLINEAR_ERR_ARCH;
+    if (!devinfo.coop) return BITLINEAR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ws);
     if (!(flags & BITLINEAR_BATCH_REUSE_PLAN) &&
@@ -515,7 +625,7 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
-    if (cudaMemsetAsync(base + L.sync_off, 0, 256, st) != cudaSuccess) {
+    if (cudaMemsetAsync(base + L.zero_begin, 0, L.zero_bytes, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
@@ -524,23 +634,24 @@ int bitlinear_decode_chain(const bitlinear_chain_layer* layers, int n_layers, in
     prm.n_layers = n_layers; prm.hidden = hidden; prm.ffn = ffn; prm.n_q = n_q_heads; prm.n_kv = n_kv_heads;
     prm.head_dim = head_dim; prm.eps = rms_eps;
     prm.h = static_cast<__nv_bfloat16*>(h_bf16);
-    float* outs[7];
-    for (int i = 0; i < 7; ++i) outs[i] = reinterpret_cast<float*>(base + L.out_off[i]);
-    prm.q = outs[0]; prm.k = outs[1]; prm.v = outs[2]; prm.o = outs[3]; prm.g = outs[4]; prm.u = outs[5]; prm.dn = outs[6];
-    prm.barrier = reinterpret_cast<unsigned*>(base + L.sync_off);
+    prm.k = reinterpret_cast<float*>(base + L.k_off);
+    for (int i = 0; i < 4; ++i) prm.pub[i] = reinterpret_cast<unsigned long long*>(base + L.pub_off[i]);
+    prm.counter = reinterpret_cast<unsigned*>(base + L.sync_off);
     prm.abort_word = reinterpret_cast<int*>(base + L.sync_off + 64);
     prm.status_word = device_status_word();
-    // the largest per-CTA share of a level, in bytes of packed weights
-    const int grid = sm_count;
-    auto share = [&](int rows, int K) { return (size_t)((rows / kTileRows + grid - 1) / grid) * (K / kTileCols) * kTileBytes; };
-    size_t buf = share(hidden + 2 * kv, hidden);
-    buf = std::max(buf, share(hidden, hidden));
-    buf = std::max(buf, share(2 * ffn, hidden));
-    buf = std::max(buf, share(hidden, ffn));
+    // the largest per-CTA share of a level, in row blocks of packed weights: level 0 splits 2 * hidden/16 + kv/16
+    // weight units and a q+v unit (two row blocks) is not divided; level 2 pairs a gate block with an up block
+    const int grid = devinfo.sm_count;
+    auto ceil_div = [](long long a, long long b) { return (a + b - 1) / b; };
+    const size_t rb_h = (size_t)(hidden / kTileCols) * kTileBytes, rb_f = (size_t)(ffn / kTileCols) * kTileBytes;
+    const long long jobs0 = ceil_div(2LL * (hidden / kTileRows) + kv / kTileRows, grid) + 2;
+    const long long jobs1 = ceil_div(hidden / kTileRows, grid);
+    const long long jobs2 = 2 * ceil_div(ffn / kTileRows, grid);
+    if (jobs0 > kMaxJobs || jobs1 > kMaxJobs || jobs2 > kMaxJobs) return BITLINEAR_ERR_SHAPE;
+    size_t buf = std::max({(size_t)jobs0 * rb_h, (size_t)jobs1 * rb_h, (size_t)jobs2 * rb_h, (size_t)jobs1 * rb_f});
     prm.buf_bytes = (int)buf;
     const int kmax = hidden > ffn ? hidden : ffn;
-    const size_t max_rb = buf / ((size_t)(hidden / kTileCols) * kTileBytes);
-    const size_t smem = 2 * buf + kmax + (size_t)hidden * 2 + max_rb * 64 + 2 * sizeof(ChainLayerDev) + 64 + 32 +
+    const size_t smem = 2 * buf + kmax + (size_t)hidden * 2 + kMaxJobs * 64 + 2 * sizeof(ChainLayerDev) + 64 + 32 +
                         sizeof(BlockScratch) + 1024;
     if (smem > 227 * 1024) return BITLINEAR_ERR_SHAPE;
     if (cudaFuncSetAttribute(decode_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
