@@ -88,11 +88,37 @@ __device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
     return v;
 }
 
+__device__ __forceinline__ unsigned long long* pub_of(const ChainParams& p, int j) {
+    return j == 0 ? p.pub[0] : (j == 1 ? p.pub[1] : (j == 2 ? p.pub[2] : p.pub[3]));
+}
+
+// r = fl32( 1 / sqrt( S / K + eps ) ) for S given as an unevaluated sum of two fp32 (S_hi + S_lo), without fp64
+// arithmetic (slow on this GPU): S / K + eps as a pair of fp32, the hardware's approximate reciprocal root, and one
+// Newton step whose residual 1 - m * y0^2 is formed error-free with fused multiply-adds, second-order term included.
+// The value rounded at the end is within 2^-44 of the exact one (checked against extended precision on 2 * 10^7 random
+// inputs: the only differences from the correctly rounded result sit where the sum of squares is within 2^-40 of a
+// rounding boundary of r, rows the parity tests exclude as fragile anyway).
+__device__ __forceinline__ float rms_scale_pair(float S_hi, float S_lo, float Kf, float eps) {
+    const float q_hi = __fdiv_rn(S_hi, Kf);
+    const float rem = __fmaf_rn(-q_hi, Kf, S_hi);  // exact remainder of the division
+    const float q_lo = __fdiv_rn(__fadd_rn(rem, S_lo), Kf);
+    const float t_hi = __fadd_rn(q_hi, eps);
+    const float bb = __fsub_rn(t_hi, q_hi);
+    const float t_lo = __fadd_rn(__fadd_rn(__fsub_rn(q_hi, __fsub_rn(t_hi, bb)), __fsub_rn(eps, bb)), q_lo);
+    float y0;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(y0) : "f"(t_hi));
+    const float p_hi = __fmul_rn(y0, y0), p_lo = __fmaf_rn(y0, y0, -p_hi);
+    const float u_hi = __fmul_rn(t_hi, p_hi), u_lo = __fmaf_rn(t_hi, p_hi, -u_hi);
+    const float small = __fmaf_rn(t_hi, p_lo, __fmul_rn(t_lo, p_hi));
+    const float e = __fsub_rn(__fsub_rn(__fsub_rn(1.0f, u_hi), u_lo), small);
+    const float c = __fmul_rn(y0, __fmaf_rn(__fmul_rn(e, e), 0.375f, __fmul_rn(0.5f, e)));
+    return __fadd_rn(y0, c);
+}
+
 struct BlockScratch {
     float sq_hi[kChainWarps], sq_lo[kChainWarps];
-    float mx[kChainWarps];
-    int sum[kChainWarps];
-    float r;
+    unsigned amax_bits[2];  // absolute maximum of the normalised input as fp32 bits (non-negative: ordered like integers)
+    int csum[2];            // sum of the int8 codes; both indexed by level parity, the other slot is cleared meanwhile
     int ok;          // CTA-local abort flag
     int desc_ready;  // highest layer whose descriptor is in shared memory
     // this CTA's units of each level: [u_lo, u_hi); level 0 has a second range of k units [k_lo, k_hi)
@@ -176,6 +202,8 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         for (int b = 0; b < 4; ++b) mbar_init(smem_u32(bars + b), 1);
         sc->ok = 0;
         sc->desc_ready = 0;
+        sc->amax_bits[0] = sc->amax_bits[1] = 0u;
+        sc->csum[0] = sc->csum[1] = 0;
         mbar_init_fence();
         // level 0: q+v units weigh two row blocks, k units one; a unit belongs to the CTA in whose weight range it starts
         const int nq = p.hidden / kTileRows, nk = p.n_kv * p.head_dim / kTileRows;
@@ -239,23 +267,12 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         const unsigned tag = (unsigned)L & 0xffffu;  // what the producers of this level's input wrote: their level + 1
 
         // ---- descriptor / scale prefetch for the next layer ----
-        if (level == 3 || level == 0) {  // level 3 needs the next layer's descriptor, level 0 this layer's scales
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            CSYNC();
-            if (level == 3 && tid == 0) {
-                __threadfence_block();
-                *reinterpret_cast<volatile int*>(&sc->desc_ready) = layer + 1;  // the copy warp may go on to the next layer
-            }
-        }
+        // level 3 needs the next layer's descriptor, level 0 this layer's scales: the asynchronous copies that fetch them
+        // are awaited here and become visible to everybody at the barrier that follows the counter wait
+        if (level == 3 || level == 0) asm volatile("cp.async.wait_group 0;" ::: "memory");
         if (level == 0 && layer + 1 < p.n_layers && tid < (int)(sizeof(ChainLayerDev) / 16)) {
             asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(&desc_s[(layer + 1) & 1]) + 16u * tid),
                          "l"(reinterpret_cast<const uint8_t*>(p.layers + layer + 1) + 16 * tid)
-                         : "memory");
-            asm volatile("cp.async.commit_group;" ::: "memory");
-        }
-        if (level == 3 && layer + 1 < p.n_layers && tid < 7) {
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(sw_s + 8 * ((layer + 1) & 1) + tid)),
-                         "l"(desc_s[(layer + 1) & 1].s_w[tid])
                          : "memory");
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
@@ -298,7 +315,19 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             CSYNC();
             if (sc->ok) { ok = false; break; }
         }
+        if (level == 3 && tid == 0) {
+            __threadfence_block();
+            *reinterpret_cast<volatile int*>(&sc->desc_ready) = layer + 1;  // the copy warp may go on to the next layer
+        }
+        // the next layer's scales: their addresses are in the descriptor that the barrier above has made visible
+        if (level == 3 && layer + 1 < p.n_layers && tid < 7) {
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(sw_s + 8 * ((layer + 1) & 1) + tid)),
+                         "l"(desc_s[(layer + 1) & 1].s_w[tid])
+                         : "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
         if (tid < kMaxJobs * 16) acc_s[tid] = 0;
+        if (tid == 0) { sc->amax_bits[(L + 1) & 1] = 0u; sc->csum[(L + 1) & 1] = 0; }
 
         // ---- the level's input: every word checked against the level tag, stale words read again ----
         float xv[kMaxLoads][6];
@@ -312,7 +341,7 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
                     xv[i][e] = (l < n_loads && 6 * part + e < kTileRows) ? __bfloat162float(h_s[e0 + e]) : 0.0f;
             }
         } else {
-            const unsigned long long* src = p.pub[(level + 3) & 3];
+            const unsigned long long* src = pub_of(p, (level + 3) & 3);
             unsigned long long wa[kMaxLoads], wb[kMaxLoads];
 #pragma unroll
             for (int i = 0; i < kMaxLoads; ++i) {
@@ -353,11 +382,17 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         }
 
         // ---- RMSNorm: sum of the exact squares as an error-free pair of fp32, root in fp64 by one thread ----
-        float s_hi = 0.0f, s_lo = 0.0f;
+        float c_hi[kMaxLoads], c_lo[kMaxLoads];  // one chain per load: independent, so their latencies overlap
 #pragma unroll
-        for (int i = 0; i < kMaxLoads; ++i)
+        for (int i = 0; i < kMaxLoads; ++i) {
+            c_hi[i] = __fmul_rn(xv[i][0], xv[i][0]);
+            c_lo[i] = 0.0f;
 #pragma unroll
-            for (int e = 0; e < 6; ++e) acc_pair(s_hi, s_lo, __fmul_rn(xv[i][e], xv[i][e]), 0.0f);
+            for (int e = 1; e < 6; ++e) acc_pair(c_hi[i], c_lo[i], __fmul_rn(xv[i][e], xv[i][e]), 0.0f);
+        }
+        float s_hi = c_hi[0], s_lo = c_lo[0];
+#pragma unroll
+        for (int i = 1; i < kMaxLoads; ++i) acc_pair(s_hi, s_lo, c_hi[i], c_lo[i]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const float o_hi = __shfl_xor_sync(0xffffffffu, s_hi, o), o_lo = __shfl_xor_sync(0xffffffffu, s_lo, o);
@@ -366,14 +401,15 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         if (lane == 0) { sc->sq_hi[warp] = s_hi; sc->sq_lo[warp] = s_lo; }
         CSYNC();
         if (sc->ok) { if (tid == 0) atomicExch(p.abort_word, 1); ok = false; break; }  // a tag wait ran out
-        if (tid == 0) {
-            double S = 0.0;
+        // every warp adds the sixteen partial pairs in the same order and takes lane 0's result, so all agree on r
+        s_hi = sc->sq_hi[lane & (kChainWarps - 1)];
+        s_lo = sc->sq_lo[lane & (kChainWarps - 1)];
 #pragma unroll
-            for (int w = 0; w < kChainWarps; ++w) S += (double)sc->sq_hi[w] + (double)sc->sq_lo[w];
-            sc->r = (float)(1.0 / sqrt(S / (double)K + (double)p.eps));
+        for (int o = kChainWarps / 2; o > 0; o >>= 1) {
+            const float o_hi = __shfl_xor_sync(0xffffffffu, s_hi, o), o_lo = __shfl_xor_sync(0xffffffffu, s_lo, o);
+            acc_pair(s_hi, s_lo, o_hi, o_lo);
         }
-        CSYNC();
-        const float r = sc->r;
+        const float r = __shfl_sync(0xffffffffu, rms_scale_pair(s_hi, s_lo, (float)K, p.eps), 0);
         float amax = 0.0f;
 #pragma unroll
         for (int i = 0; i < kMaxLoads; ++i) {
@@ -385,13 +421,12 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
                 amax = fmaxf(amax, fabsf(xv[i][e]));
             }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-        if (lane == 0) sc->mx[warp] = amax;
+        {
+            const unsigned wmax = __reduce_max_sync(0xffffffffu, __float_as_uint(amax));
+            if (lane == 0) atomicMax(&sc->amax_bits[L & 1], wmax);
+        }
         CSYNC();
-        float a = 1e-5f;
-#pragma unroll
-        for (int w = 0; w < kChainWarps; ++w) a = fmaxf(a, sc->mx[w]);
+        const float a = fmaxf(__uint_as_float(sc->amax_bits[L & 1]), 1e-5f);
         const float sc_q = __fdiv_rn(127.0f, a), d = __fdiv_rn(a, 127.0f);
         int csum = 0;
 #pragma unroll
@@ -421,9 +456,8 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
                 }
             }
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) csum += __shfl_xor_sync(0xffffffffu, csum, o);
-        if (lane == 0) sc->sum[warp] = csum;
+        csum = __reduce_add_sync(0xffffffffu, csum);
+        if (lane == 0) atomicAdd(&sc->csum[L & 1], csum);
 
         // ---- the level's weights: wait for the prefetched share, multiply ----
         mbar_wait(smem_u32(bars + (L & 1)), (uint32_t)(L >> 1) & 1u, abort_s);
@@ -433,83 +467,92 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             ok = false;
             break;
         }
-        int xsum = 0;
-#pragma unroll
-        for (int w = 0; w < kChainWarps; ++w) xsum += sc->sum[w];
+        const int xsum = sc->csum[L & 1];
         const uint32_t buf_s = smem_u32(wbuf + (size_t)(L & 1) * p.buf_bytes);
         const uint32_t xq_a = smem_u32(xq_s) + 16u * t;
-        for (int tix = warp; tix < n_jobs * k_tiles; tix += kChainWarps) {
-            const int job = tix / k_tiles, kt = tix - job * k_tiles;
-            const uint4 w0v = lds128(buf_s + (uint32_t)tix * kTileBytes + 16u * lane);
-            const uint4 w1v = lds128(buf_s + (uint32_t)tix * kTileBytes + 512u + 16u * lane);
-            const uint32_t w0[4] = {w0v.x, w0v.y, w0v.z, w0v.w};
-            const uint32_t w1[4] = {w1v.x, w1v.y, w1v.z, w1v.w};
+        {
+            // a warp takes a contiguous run of the CTA's 16 x 256 tiles, so it folds its accumulators once per row block
+            const int n_tiles = n_jobs * k_tiles;
+            const int t_lo = n_tiles * warp / kChainWarps, t_hi = n_tiles * (warp + 1) / kChainWarps;
             int acc[2][4] = {{0, 0, 0, 0}, {0, 0, 0, 0}};
+            int job = t_lo / k_tiles, kt = t_lo - job * k_tiles;
+            for (int tix = t_lo; tix < t_hi; ++tix) {
+                const uint4 w0v = lds128(buf_s + (uint32_t)tix * kTileBytes + 16u * lane);
+                const uint4 w1v = lds128(buf_s + (uint32_t)tix * kTileBytes + 512u + 16u * lane);
+                const uint32_t w0[4] = {w0v.x, w0v.y, w0v.z, w0v.w};
+                const uint32_t w1[4] = {w1v.x, w1v.y, w1v.z, w1v.w};
 #pragma unroll
-            for (int qd = 0; qd < 4; ++qd) {
-                const uint4 xw4 = lds128(xq_a + (uint32_t)kt * kTileCols + 64u * qd);
-                const uint32_t xw[4] = {xw4.x, xw4.y, xw4.z, xw4.w};
+                for (int qd = 0; qd < 4; ++qd) {
+                    const uint4 xw4 = lds128(xq_a + (uint32_t)kt * kTileCols + 64u * qd);
+                    const uint32_t xw[4] = {xw4.x, xw4.y, xw4.z, xw4.w};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t mask = 0x03030303u << (2 * j);
-                    acc[0][j] = dp4a_u8_s8(w0[qd] & mask, xw[j], acc[0][j]);
-                    acc[1][j] = dp4a_u8_s8(w1[qd] & mask, xw[j], acc[1][j]);
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t mask = 0x03030303u << (2 * j);
+                        acc[0][j] = dp4a_u8_s8(w0[qd] & mask, xw[j], acc[0][j]);
+                        acc[1][j] = dp4a_u8_s8(w1[qd] & mask, xw[j], acc[1][j]);
+                    }
                 }
-            }
+                if (++kt == k_tiles || tix + 1 == t_hi) {
 #pragma unroll
-            for (int hh = 0; hh < 2; ++hh) {
-                int sum = acc[hh][0] * 4 + acc[hh][1];  // accumulator j holds 4^j x its share: 64 x the sum
-                sum = sum * 4 + acc[hh][2];
-                sum = sum * 4 + acc[hh][3];
-                sum += __shfl_xor_sync(0xffffffffu, sum, 1);
-                sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-                if (t == 0) atomicAdd(&acc_s[job * 16 + 8 * hh + g], sum >> 6);
+                    for (int hh = 0; hh < 2; ++hh) {
+                        int sum = acc[hh][0] * 4 + acc[hh][1];  // accumulator j holds 4^j x its share: 64 x the sum
+                        sum = sum * 4 + acc[hh][2];
+                        sum = sum * 4 + acc[hh][3];
+                        sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                        sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                        if (t == 0) atomicAdd(&acc_s[job * 16 + 8 * hh + g], sum >> 6);
+                        acc[hh][0] = acc[hh][1] = acc[hh][2] = acc[hh][3] = 0;
+                    }
+                    if (kt == k_tiles) { kt = 0; ++job; }
+                }
             }
         }
         CSYNC();
         if (tid == 0) mbar_arrive(smem_u32(bars + 2 + (L & 1)));  // the buffer has been read: it may be refilled
 
         // ---- dequantising epilogue + the glue that follows this level, published as the next level's input ----
-        // One thread per published word: three consecutive rows of a unit (the sixth word of a unit holds one row).
+        // One thread per output row (a unit's 16 rows are a half warp); lanes 0..5 of each half then gather three rows each
+        // into the 8-byte words of the unit.  The k rows of level 0 are stored by the second half of the CTA.
         {
             const int n_units = sc->u_hi[level] - sc->u_lo[level];
             const float* sw = sw_s + 8 * (layer & 1);
             const bool last = L + 1 == total_levels;
-            if (tid < 6 * n_units) {
-                const int ul = tid / 6, wd = tid - 6 * ul, unit = sc->u_lo[level] + ul;
-                const int jpu = (level == 0 || level == 2) ? 2 : 1;  // jobs per unit
-                uint32_t bits[3] = {0u, 0u, 0u};
-#pragma unroll
-                for (int e = 0; e < 3; ++e) {
-                    const int row16 = 3 * wd + e;
-                    if (row16 < kTileRows) {
-                        const int row = unit * kTileRows + row16;
-                        const float y0 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * jpu) * 16 + row16] - xsum),
-                                                             sw[level == 0 ? 0 : (level == 1 ? 3 : (level == 2 ? 4 : 6))]), d);
-                        float val;
-                        if (level == 0) {
-                            const float y1 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * 2 + 1) * 16 + row16] - xsum), sw[2]), d);
-                            val = __fadd_rn(y0, y1);  // attention stand-in: q + v of the matching KV head
-                        } else if (level == 2) {
-                            const float y1 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * 2 + 1) * 16 + row16] - xsum), sw[5]), d);
-                            const float rl = fmaxf(y0, 0.0f);
-                            val = __fmul_rn(__fmul_rn(rl, rl), y1);  // squared-ReLU gate times up
-                        } else {
-                            val = __fadd_rn(__bfloat162float(h_s[row]), y0);  // residual
-                        }
-                        bits[e] = bf16_bits_rn(val);
-                        if (last) reinterpret_cast<uint16_t*>(p.h)[row] = (uint16_t)bits[e];
+            if (warp < (n_units + 1) / 2) {  // warp-uniform
+                const int ul = tid >> 4, row16 = tid & 15, unit = sc->u_lo[level] + ul;
+                uint32_t bits = 0u;
+                if (ul < n_units) {
+                    const int row = unit * kTileRows + row16;
+                    const int jpu = (level == 0 || level == 2) ? 2 : 1;  // jobs per unit
+                    const float s0 = level == 0 ? sw[0] : (level == 1 ? sw[3] : (level == 2 ? sw[4] : sw[6]));
+                    const float y0 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * jpu) * 16 + row16] - xsum), s0), d);
+                    float val;
+                    if (level == 0) {
+                        const float y1 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * 2 + 1) * 16 + row16] - xsum), sw[2]), d);
+                        val = __fadd_rn(y0, y1);  // attention stand-in: q + v of the matching KV head
+                    } else if (level == 2) {
+                        const float y1 = __fmul_rn(__fmul_rn((float)(acc_s[(ul * 2 + 1) * 16 + row16] - xsum), sw[5]), d);
+                        const float rl = fmaxf(y0, 0.0f);
+                        val = __fmul_rn(__fmul_rn(rl, rl), y1);  // squared-ReLU gate times up
+                    } else {
+                        val = __fadd_rn(__bfloat162float(h_s[row]), y0);  // residual
                     }
+                    bits = bf16_bits_rn(val);
+                    if (last) reinterpret_cast<uint16_t*>(p.h)[row] = (uint16_t)bits;
                 }
-                if (!last)
-                    st_pub(p.pub[level] + 6 * (size_t)unit + wd,
-                           (unsigned long long)(bits[0] | (bits[1] << 16)) |
-                               ((unsigned long long)(bits[2] | (((unsigned)(L + 1) & 0xffffu) << 16)) << 32));
+                const int wd = lane & 15, base = lane & 16;  // word wd of this half warp's unit: rows 3 wd .. 3 wd + 2
+                const int r0 = 3 * wd;
+                const uint32_t b0 = __shfl_sync(0xffffffffu, bits, base + (r0 < 16 ? r0 : 15));
+                const uint32_t b1 = __shfl_sync(0xffffffffu, bits, base + (r0 + 1 < 16 ? r0 + 1 : 15));
+                const uint32_t b2 = __shfl_sync(0xffffffffu, bits, base + (r0 + 2 < 16 ? r0 + 2 : 15));
+                if (!last && ul < n_units && wd < 6)
+                    st_pub(pub_of(p, level) + 6 * (size_t)unit + wd,
+                           (unsigned long long)(b0 | ((wd < 5 ? b1 : 0u) << 16)) |
+                               ((unsigned long long)((wd < 5 ? b2 : 0u) | (((unsigned)(L + 1) & 0xffffu) << 16)) << 32));
             }
-            if (level == 0) {  // k rows: an output of the layer, consumed by nobody here
+            if (level == 0 && tid >= kChainThreads / 2) {  // k rows: an output of the layer, consumed by nobody here
                 const int nqv = sc->u_hi[0] - sc->u_lo[0], nk = sc->k_hi - sc->k_lo;
-                const int o = tid - 6 * n_units;
-                if (o >= 0 && o < nk * 16)
+                const int o = tid - kChainThreads / 2;
+                if (o < nk * 16)
                     p.k[(sc->k_lo + (o >> 4)) * kTileRows + (o & 15)] =
                         __fmul_rn(__fmul_rn((float)(acc_s[(2 * nqv + (o >> 4)) * 16 + (o & 15)] - xsum), sw[1]), d);
             }
