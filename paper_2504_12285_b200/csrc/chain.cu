@@ -93,15 +93,15 @@ __device__ __forceinline__ unsigned long long* pub_of(const ChainParams& p, int 
 }
 
 // r = fl32( 1 / sqrt( S / K + eps ) ) for S given as an unevaluated sum of two fp32 (S_hi + S_lo), without fp64
-// arithmetic (slow on this GPU): S / K + eps as a pair of fp32, the hardware's approximate reciprocal root, and one
+// arithmetic (slow on this GPU) and without a division: S / K + eps as a pair of fp32, the hardware's approximate reciprocal root, and one
 // Newton step whose residual 1 - m * y0^2 is formed error-free with fused multiply-adds, second-order term included.
 // The value rounded at the end is within 2^-44 of the exact one (checked against extended precision on 2 * 10^7 random
 // inputs: the only differences from the correctly rounded result sit where the sum of squares is within 2^-40 of a
 // rounding boundary of r, rows the parity tests exclude as fragile anyway).
-__device__ __forceinline__ float rms_scale_pair(float S_hi, float S_lo, float Kf, float eps) {
-    const float q_hi = __fdiv_rn(S_hi, Kf);
-    const float rem = __fmaf_rn(-q_hi, Kf, S_hi);  // exact remainder of the division
-    const float q_lo = __fdiv_rn(__fadd_rn(rem, S_lo), Kf);
+__device__ __forceinline__ float rms_scale_pair(float S_hi, float S_lo, float ik_hi, float ik_lo, float eps) {
+    // S / K as S * (1 / K), the reciprocal given as a pair ik_hi + ik_lo (accurate to 2^-48)
+    const float q_hi = __fmul_rn(S_hi, ik_hi);
+    const float q_lo = __fadd_rn(__fmaf_rn(S_hi, ik_hi, -q_hi), __fmaf_rn(S_hi, ik_lo, __fmul_rn(S_lo, ik_hi)));
     const float t_hi = __fadd_rn(q_hi, eps);
     const float bb = __fsub_rn(t_hi, q_hi);
     const float t_lo = __fadd_rn(__fadd_rn(__fsub_rn(q_hi, __fsub_rn(t_hi, bb)), __fsub_rn(eps, bb)), q_lo);
@@ -245,6 +245,22 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         }
     };
     bool ok = true;
+    // Load index l = tid + i * 512 of a level input covers elements 16 * (l / 3) + 6 * (l % 3) + 0..5 (the last of the
+    // three loads of a 16-element group covers four).  None of this depends on the level.
+    int ld_part[kMaxLoads], ld_elem[kMaxLoads], ld_piece[kMaxLoads];
+#pragma unroll
+    for (int i = 0; i < kMaxLoads; ++i) {
+        const int l = tid + i * kChainThreads, rb = l / 3;
+        ld_part[i] = l - 3 * rb;
+        ld_elem[i] = rb * kTileRows + 6 * ld_part[i];
+        // the 16 codes of a group are one 16-byte piece of the lane-interleaved order (piece 4t+q of a block of 256
+        // columns at byte 64q + 16t); this thread owns bytes 6 * part .. of it
+        const int c0 = rb * kTileRows, rr = c0 & 255;
+        ld_piece[i] = (c0 & ~255) + 64 * ((rr >> 4) & 3) + 16 * (rr >> 6);
+    }
+    // 1 / K as a pair of fp32 for the two input widths
+    const float ikh_hi = __fdiv_rn(1.0f, (float)p.hidden), ikh_lo = __fdiv_rn(__fmaf_rn(-ikh_hi, (float)p.hidden, 1.0f), (float)p.hidden);
+    const float ikf_hi = __fdiv_rn(1.0f, (float)p.ffn), ikf_lo = __fdiv_rn(__fmaf_rn(-ikf_hi, (float)p.ffn, 1.0f), (float)p.ffn);
     if (warp == kChainWarps) {
         // ---- copy warp: one level ahead of the arithmetic, as soon as the buffer has been read and the layer's
         //      descriptor is in shared memory ----
@@ -278,20 +294,20 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         }
 
         // ---- the gains of this level's input: loads issued before the wait so that they overlap it ----
-        // Load index l = tid + i * 512 covers elements 16 * (l / 3) + 6 * (l % 3) + 0..5 (the last of the three covers four).
         const __nv_bfloat16* gain = desc_s[layer & 1].gain[level];
         const int n_loads = 3 * (K / kTileRows);
+        // whether load i concerns this WARP at all (warp-uniform): whole iterations are skipped where it does not
+        const bool act[kMaxLoads] = {(warp << 5) < n_loads, (warp << 5) + kChainThreads < n_loads,
+                                     (warp << 5) + 2 * kChainThreads < n_loads};
         uint32_t gw[kMaxLoads][3];
 #pragma unroll
         for (int i = 0; i < kMaxLoads; ++i) {
-            const int l = tid + i * kChainThreads;
             gw[i][0] = gw[i][1] = gw[i][2] = 0x3f803f80u;  // bf16 ones
-            if (gain != nullptr && l < n_loads) {
-                const int rb = l / 3, part = l - 3 * rb;
-                const uint32_t* gp = reinterpret_cast<const uint32_t*>(gain + rb * kTileRows + 6 * part);
+            if (act[i] && gain != nullptr && tid + i * kChainThreads < n_loads) {
+                const uint32_t* gp = reinterpret_cast<const uint32_t*>(gain + ld_elem[i]);
                 gw[i][0] = gp[0];
                 gw[i][1] = gp[1];
-                if (part < 2) gw[i][2] = gp[2];
+                if (ld_part[i] < 2) gw[i][2] = gp[2];
             }
         }
 
@@ -335,10 +351,9 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
 #pragma unroll
             for (int i = 0; i < kMaxLoads; ++i) {
                 const int l = tid + i * kChainThreads;
-                const int rb = l / 3, part = l - 3 * rb, e0 = rb * kTileRows + 6 * part;
 #pragma unroll
                 for (int e = 0; e < 6; ++e)
-                    xv[i][e] = (l < n_loads && 6 * part + e < kTileRows) ? __bfloat162float(h_s[e0 + e]) : 0.0f;
+                    xv[i][e] = (l < n_loads && 6 * ld_part[i] + e < kTileRows) ? __bfloat162float(h_s[ld_elem[i] + e]) : 0.0f;
             }
         } else {
             const unsigned long long* src = pub_of(p, (level + 3) & 3);
@@ -347,11 +362,12 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             for (int i = 0; i < kMaxLoads; ++i) {
                 const int l = tid + i * kChainThreads;
                 wa[i] = wb[i] = (unsigned long long)tag << 48;
-                if (l < n_loads) ld_pub2(src + 2 * l, wa[i], wb[i]);
+                if (act[i] && l < n_loads) ld_pub2(src + 2 * l, wa[i], wb[i]);
             }
 #pragma unroll
             for (int i = 0; i < kMaxLoads; ++i) {
                 const int l = tid + i * kChainThreads;
+                if (!act[i]) continue;
                 if (l < n_loads && ((unsigned)(wa[i] >> 48) != tag || (unsigned)(wb[i] >> 48) != tag)) {
                     const unsigned long long t0 = globaltimer_ns();
                     unsigned spins = 0;
@@ -373,26 +389,27 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
                 xv[i][3] = bf16_lo(b0); xv[i][4] = bf16_hi(b0); xv[i][5] = bf16_lo(b1);
                 if ((level == 0 || level == 2) && l < n_loads) {
                     // the input of levels 0 and 2 is the hidden state itself: keep it for the residual adds of this CTA's rows
-                    const int rb = l / 3, part = l - 3 * rb;
-                    uint16_t* hp = reinterpret_cast<uint16_t*>(h_s) + rb * kTileRows + 6 * part;
-                    hp[0] = (uint16_t)a0; hp[1] = (uint16_t)(a0 >> 16); hp[2] = (uint16_t)a1; hp[3] = (uint16_t)b0;
-                    if (part < 2) { hp[4] = (uint16_t)(b0 >> 16); hp[5] = (uint16_t)b1; }
+                    // (ld_elem is even: two values per 32-bit store)
+                    uint32_t* hp = reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(h_s) + ld_elem[i]);
+                    hp[0] = a0;
+                    hp[1] = (a1 & 0xffffu) | (b0 << 16);
+                    if (ld_part[i] < 2) hp[2] = (b0 >> 16) | (b1 << 16);
                 }
             }
         }
 
         // ---- RMSNorm: sum of the exact squares as an error-free pair of fp32, root in fp64 by one thread ----
-        float c_hi[kMaxLoads], c_lo[kMaxLoads];  // one chain per load: independent, so their latencies overlap
+        float s_hi = 0.0f, s_lo = 0.0f;
 #pragma unroll
         for (int i = 0; i < kMaxLoads; ++i) {
-            c_hi[i] = __fmul_rn(xv[i][0], xv[i][0]);
-            c_lo[i] = 0.0f;
+            if (!act[i]) continue;
+            // one chain per load: independent of the others, so their latencies overlap
+            float c_hi = __fmul_rn(xv[i][0], xv[i][0]), c_lo = 0.0f;
 #pragma unroll
-            for (int e = 1; e < 6; ++e) acc_pair(c_hi[i], c_lo[i], __fmul_rn(xv[i][e], xv[i][e]), 0.0f);
+            for (int e = 1; e < 6; ++e) acc_pair(c_hi, c_lo, __fmul_rn(xv[i][e], xv[i][e]), 0.0f);
+            if (i == 0) { s_hi = c_hi; s_lo = c_lo; }
+            else acc_pair(s_hi, s_lo, c_hi, c_lo);
         }
-        float s_hi = c_hi[0], s_lo = c_lo[0];
-#pragma unroll
-        for (int i = 1; i < kMaxLoads; ++i) acc_pair(s_hi, s_lo, c_hi[i], c_lo[i]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) {
             const float o_hi = __shfl_xor_sync(0xffffffffu, s_hi, o), o_lo = __shfl_xor_sync(0xffffffffu, s_lo, o);
@@ -409,10 +426,11 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
             const float o_hi = __shfl_xor_sync(0xffffffffu, s_hi, o), o_lo = __shfl_xor_sync(0xffffffffu, s_lo, o);
             acc_pair(s_hi, s_lo, o_hi, o_lo);
         }
-        const float r = __shfl_sync(0xffffffffu, rms_scale_pair(s_hi, s_lo, (float)K, p.eps), 0);
+        const float r = __shfl_sync(0xffffffffu, rms_scale_pair(s_hi, s_lo, level == 3 ? ikf_hi : ikh_hi, level == 3 ? ikf_lo : ikh_lo, p.eps), 0);
         float amax = 0.0f;
 #pragma unroll
         for (int i = 0; i < kMaxLoads; ++i) {
+            if (!act[i]) continue;
             const float gv[6] = {bf16_lo(gw[i][0]), bf16_hi(gw[i][0]), bf16_lo(gw[i][1]),
                                  bf16_hi(gw[i][1]), bf16_lo(gw[i][2]), bf16_hi(gw[i][2])};
 #pragma unroll
@@ -431,16 +449,12 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         int csum = 0;
 #pragma unroll
         for (int i = 0; i < kMaxLoads; ++i) {
-            const int l = tid + i * kChainThreads;
-            if (l < n_loads) {
-                const int rb = l / 3, part = l - 3 * rb, c0 = rb * kTileRows;
+            if (act[i] && tid + i * kChainThreads < n_loads) {
+                const int part = ld_part[i];
                 uint32_t c[6];
 #pragma unroll
                 for (int e = 0; e < 6; ++e) c[e] = round_code(__fmul_rn(xv[i][e], sc_q));
-                // the 16 codes of a row block are one 16-byte piece of the lane-interleaved order (piece 4t+q of a block
-                // of 256 columns at byte 64q + 16t); this thread owns bytes 6 * part .. of it
-                const int blk = c0 & ~255, rr = c0 & 255;
-                uint8_t* piece = xq_s + blk + 64 * ((rr >> 4) & 3) + 16 * (rr >> 6);
+                uint8_t* piece = xq_s + ld_piece[i];
                 const uint32_t w4 = pack_codes4(c[0], c[1], c[2], c[3], csum);
                 if (part == 0) {
                     *reinterpret_cast<uint32_t*>(piece) = w4;
