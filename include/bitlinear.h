@@ -46,6 +46,23 @@
  *   per byte - directly a dot-product-of-four or tensor-core operand.
  *   Kernels accumulate sum_k c*xq and subtract sum_k xq (produced by the
  *   activation quantiser) to recover sum_k Wq*xq.
+ *
+ * Dense packed weight layout (five ternary values per byte, 1.6 bits per weight; Table 1 of the
+ * paper counts the model's memory at about 1.58 bits per weight, and Section 5.1 packs weights
+ * to cut the bytes moved per token - the layout itself is this library's)
+ *   Byte value: with the codes c_e = Wq + 1 of five weights, digit 0 the most significant,
+ *   v = 81*c_0 + 27*c_1 + 9*c_2 + 3*c_3 + c_4 (0..242) and the stored byte is ceil(256 * v / 243),
+ *   i.e. the base-3 fraction 0.c_0c_1c_2c_3c_4 scaled to eight bits and rounded up: multiplying the
+ *   byte by 3 leaves digit c_0 in bits 8-9 and the fraction of the remaining digits in bits 0-7,
+ *   so a decoder peels the digits off with multiplications, no division.  v = floor(243 * B / 256).
+ *   Position: K is padded with zero weights to Kp = 320 * ceil(K / 320).  Tiles of 16 rows x 320
+ *   columns, 1024 bytes each, row-block major: tile index = (n / 16) * (Kp / 320) + (k / 320).
+ *   Inside a tile, row r = 8*h + g and column c = 80*t + 20*i + 4*e + b (t, i, b in 0..3,
+ *   e in 0..4) live at byte 512*h + 64*g + 16*t + 4*i + b, base-3 digit e.  Hence a 16-byte chunk
+ *   holds 80 consecutive columns of one row, a 32-bit word 20 consecutive columns, and digit e
+ *   of the four bytes of a word belongs to four consecutive columns - one dot-product-of-four.
+ *   Size: N * Kp / 5 bytes: 418.8 MB for the 210 matrices of the 2B model against 521.0 MB at
+ *   four per byte.
  */
 #ifndef BITLINEAR_H_
 #define BITLINEAR_H_
@@ -72,6 +89,10 @@ typedef enum {
 /* dtype codes */
 #define BITLINEAR_F32 0
 #define BITLINEAR_BF16 1
+
+/* Layout of a packed weight matrix (field w_format of bitlinear_problem). */
+#define BITLINEAR_WEIGHTS_2BIT 0   /* four values per byte, from bitlinear_pack_weights */
+#define BITLINEAR_WEIGHTS_DENSE5 1 /* five values per byte, from bitlinear_pack_weights5 */
 
 /* Which contraction kernel bitlinear_matmul_q / bitlinear_forward use. */
 #define BITLINEAR_PATH_AUTO 0  /* decode kernel for M <= 16, tensor-core kernel above */
@@ -118,6 +139,21 @@ int bitlinear_pack_weights(const void* W, int w_dtype, int N, int K, float eps_w
 
 /* Test hook: expand a packed matrix back to int8 values in {-1,0,1}, [N][K] row-major. */
 int bitlinear_unpack_weights(const void* packed, int N, int K, int8_t* wq_out, void* stream);
+
+/*
+ * The same quantiser writing the dense layout, five ternary values per byte (Table 1: about 1.58
+ * bits per weight; Section 5.1: packing exists to move fewer bytes).  Arguments as
+ * bitlinear_pack_weights; packed5_out holds bitlinear_packed5_bytes(N,K) = N * Kp / 5 bytes,
+ * Kp = K rounded up to a multiple of 320 (0 for an unsupported shape).  The scale and the ternary
+ * values are identical to those of bitlinear_pack_weights; only the storage differs.  Dense
+ * matrices are consumed by bitlinear_forward_batch (w_format = BITLINEAR_WEIGHTS_DENSE5) for
+ * problems of at most 16 tokens.
+ */
+size_t bitlinear_packed5_bytes(int N, int K);
+int bitlinear_pack_weights5(const void* W, int w_dtype, int N, int K, float eps_w, void* packed5_out,
+                            float* s_w_out, void* ws, size_t ws_bytes, void* stream);
+/* Test hook: expand a dense matrix back to int8 values in {-1,0,1}, [N][K] row-major (padding dropped). */
+int bitlinear_unpack_weights5(const void* packed5, int N, int K, int8_t* wq_out, void* stream);
 
 /*
  * Fused RMSNorm + per-token absmax int8 quantiser (Section 2, "Activation Quantization" and
@@ -182,6 +218,10 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  * images, and one persistent tcgen05 kernel that runs every tile of every matmul; problems that
  * name the same x, gain, rms_eps, M and K (q/k/v or gate/up of a layer) share one quantised copy.
  * Both kinds may be mixed in one call.
+ * Weights in the dense layout (w_format = BITLINEAR_WEIGHTS_DENSE5, Table 1 / Section 5.1) are accepted for
+ * problems of at most 16 tokens; all such problems of a call must use the same layout.  Their kernel is the
+ * one-token streaming kernel with the base-3 digits peeled off in registers; a problem of M tokens streams its
+ * weights M times, so this layout trades speed at M > 1 for 20 % less memory.
  *   problems : HOST array of `count` descriptors; the pointers inside are DEVICE pointers with the
  *              meaning, layout and alignment of the bitlinear_forward arguments.  K <= 8192 for
  *              problems of at most 16 tokens.  Problems with M == 0 are skipped.  Outputs must not
@@ -204,7 +244,7 @@ typedef struct bitlinear_problem {
     int M, N, K;
     int y_dtype;        /* BITLINEAR_F32 or BITLINEAR_BF16 */
     float rms_eps;
-    int reserved;       /* set to 0 */
+    int w_format;       /* layout of `packed`: BITLINEAR_WEIGHTS_2BIT (0) or BITLINEAR_WEIGHTS_DENSE5 (1) */
 } bitlinear_problem;
 
 #define BITLINEAR_BATCH_REUSE_PLAN 1 /* descriptors unchanged since the previous call on this workspace */
@@ -213,6 +253,16 @@ typedef struct bitlinear_problem {
 size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count);
 int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
                             void* stream);
+
+/*
+ * Parity hook: bitlinear_forward_batch that also stores the raw int32 accumulators sum_k xq*Wq of the contraction
+ * (Section 5.1: the integer product of unpacked ternary weights and 8-bit activations).
+ *   acc_out : HOST array of `count` DEVICE pointers, entry i nullable or [M][N] int32 for problem i.
+ * Available where the persistent streaming kernels run the problem: one-token problems in the 2-bit layout and
+ * problems of up to 16 tokens in the dense layout; BITLINEAR_ERR_SHAPE for a non-NULL entry anywhere else.
+ */
+int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, int flags, int32_t* const* acc_out,
+                                void* ws, size_t ws_bytes, void* stream);
 
 /*
  * bitlinear_forward_batch for callers whose activations live in HOST memory.  The x pointers of the

@@ -32,6 +32,11 @@ _SIGNATURES = {
     "bitlinear_pack_weights": (_c_int, [_c_void_p, _c_int, _c_int, _c_int, _c_float, _c_void_p, _c_void_p,
                                         _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_unpack_weights": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_void_p]),
+    "bitlinear_packed5_bytes": (_c_size_t, [_c_int, _c_int]),
+    "bitlinear_pack_weights5": (_c_int, [_c_void_p, _c_int, _c_int, _c_int, _c_float, _c_void_p, _c_void_p,
+                                         _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_unpack_weights5": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_void_p]),
+    "bitlinear_forward_batch_acc": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_quant_act": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_int, _c_int, _c_void_p, _c_void_p,
                                      _c_void_p, _c_void_p]),
     "bitlinear_matmul_q": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
@@ -56,6 +61,7 @@ _SIGNATURES = {
                                               _c_void_p, _c_size_t, _c_void_p, _c_size_t, _c_void_p]),
 }
 
+WEIGHTS_2BIT, WEIGHTS_DENSE5 = 0, 1
 BATCH_REUSE_PLAN = 1
 BATCH_REUSE_ACT = 2
 
@@ -64,7 +70,7 @@ class Problem(ctypes.Structure):
     """Mirror of the C struct bitlinear_problem."""
     _fields_ = [("x", _c_void_p), ("gain", _c_void_p), ("packed", _c_void_p), ("s_w", _c_void_p), ("y", _c_void_p),
                 ("M", _c_int), ("N", _c_int), ("K", _c_int), ("y_dtype", _c_int), ("rms_eps", _c_float),
-                ("reserved", _c_int)]
+                ("w_format", _c_int)]
 
 
 class BitLinearError(RuntimeError):
@@ -162,6 +168,35 @@ def bitlinear_pack_weights(W: torch.Tensor, eps_w: float = 1e-5):
                                       _ptr(s_w), _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_pack_weights")
     return packed, s_w
+
+
+def bitlinear_packed5_bytes(N: int, K: int) -> int:
+    return int(lib().bitlinear_packed5_bytes(N, K))
+
+
+def bitlinear_pack_weights5(W: torch.Tensor, eps_w: float = 1e-5):
+    """W [N, K] fp32 or bf16 on the GPU -> (dense packed uint8, five values per byte, s_w fp32 [1])."""
+    if W.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("W must be float32 or bfloat16")
+    _dev(W, W.dtype, "W")
+    N, K = W.shape
+    nbytes = bitlinear_packed5_bytes(N, K)
+    if nbytes == 0:
+        raise BitLinearError(2, "bitlinear_pack_weights5")
+    packed = torch.empty(nbytes, dtype=torch.uint8, device=W.device)
+    s_w = torch.empty(1, dtype=torch.float32, device=W.device)
+    ws = _workspace(bitlinear_pack_workspace_bytes(N, K), W.device)
+    rc = lib().bitlinear_pack_weights5(_ptr(W), F32 if W.dtype == torch.float32 else BF16, N, K, eps_w, _ptr(packed),
+                                       _ptr(s_w), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_pack_weights5")
+    return packed, s_w
+
+
+def bitlinear_unpack_weights5(packed: torch.Tensor, N: int, K: int) -> torch.Tensor:
+    _dev(packed, torch.uint8, "packed")
+    wq = torch.empty(N, K, dtype=torch.int8, device=packed.device)
+    _check(lib().bitlinear_unpack_weights5(_ptr(packed), N, K, _ptr(wq), _stream()), "bitlinear_unpack_weights5")
+    return wq
 
 
 def bitlinear_unpack_weights(packed: torch.Tensor, N: int, K: int) -> torch.Tensor:
@@ -336,8 +371,9 @@ def bitlinear_forward_static(x, gain, packed, s_w, N: int, rms_eps: float = 1e-5
 class ProblemBatch:
     """A host array of bitlinear_problem descriptors plus the tensors they point to (kept alive)."""
 
-    def __init__(self, items, rms_eps: float = 1e-5):
-        """items: iterable of (x [M,K] bf16, gain [K] bf16 or None, packed uint8, s_w fp32 [1], y [M,N])."""
+    def __init__(self, items, rms_eps: float = 1e-5, w_format: int = WEIGHTS_2BIT):
+        """items: iterable of (x [M,K] bf16, gain [K] bf16 or None, packed uint8, s_w fp32 [1], y [M,N]);
+        w_format: the layout of every packed matrix of the batch (WEIGHTS_2BIT or WEIGHTS_DENSE5)."""
         self.tensors = [tuple(it) for it in items]
         self.array = (Problem * max(len(self.tensors), 1))()
         for i, (x, gain, packed, s_w, y) in enumerate(self.tensors):
@@ -352,7 +388,7 @@ class ProblemBatch:
             if y.shape[0] != M:
                 raise ValueError("x and y disagree on M")
             self.array[i] = Problem(_ptr(x), _ptr(gain), _ptr(packed), _ptr(s_w), _ptr(y), M, y.shape[1], K,
-                                    _ydt(y.dtype), rms_eps, 0)
+                                    _ydt(y.dtype), rms_eps, w_format)
         self.count = len(self.tensors)
 
     def workspace_bytes(self) -> int:
@@ -371,6 +407,19 @@ def bitlinear_forward_batch(batch: ProblemBatch, ws: torch.Tensor, reuse_plan: b
     rc = lib().bitlinear_forward_batch(ctypes.addressof(batch.array), batch.count, flags, _ptr(ws), ws.numel(),
                                        _stream())
     _check(rc, "bitlinear_forward_batch")
+
+
+def bitlinear_forward_batch_acc(batch: ProblemBatch, accs, ws: torch.Tensor, reuse_plan: bool = False) -> None:
+    """bitlinear_forward_batch that also stores the int32 accumulators: accs[i] is None or an int32 [M, N] CUDA tensor."""
+    _dev(ws, torch.uint8, "ws")
+    arr = (_c_void_p * max(batch.count, 1))()
+    for i, a in enumerate(accs):
+        if a is not None:
+            _dev(a, torch.int32, "acc")
+            arr[i] = a.data_ptr()
+    rc = lib().bitlinear_forward_batch_acc(ctypes.addressof(batch.array), batch.count, BATCH_REUSE_PLAN if reuse_plan else 0,
+                                           ctypes.addressof(arr), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_forward_batch_acc")
 
 
 def bitlinear_forward_batch_host(batch: ProblemBatch, x_host: torch.Tensor, x_dev: torch.Tensor, y_dev: torch.Tensor,

@@ -126,6 +126,34 @@ int bitlinear_pack_weights(const void* W, int w_dtype, int N, int K, float eps_w
     return cuda_status(launch_quant_pack(W, w_dtype, N, K, s_w_out, static_cast<uint32_t*>(packed_out), st));
 }
 
+size_t bitlinear_packed5_bytes(int N, int K) {
+    return shape_ok(N, K) ? (size_t)(N / kTileRows) * dense_k_tiles(K) * kTileBytes : 0;
+}
+
+int bitlinear_pack_weights5(const void* W, int w_dtype, int N, int K, float eps_w, void* packed5_out, float* s_w_out,
+                            void* ws, size_t ws_bytes, void* stream) {
+    if (!W || !packed5_out || !s_w_out) return BITLINEAR_ERR_NULL;
+    if (w_dtype != BITLINEAR_F32 && w_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
+    if (!shape_ok(N, K)) return BITLINEAR_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(packed5_out) || (reinterpret_cast<uintptr_t>(s_w_out) & 3u)) return BITLINEAR_ERR_ALIGN;
+    if (!ws || ws_bytes < bitlinear_pack_workspace_bytes(N, K) || !aligned16(ws)) return BITLINEAR_ERR_WORKSPACE;
+    if (int rc = check_arch()) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t count = (size_t)N * K;
+    cudaError_t e = launch_absmean(W, w_dtype, count, eps_w, static_cast<double*>(ws), absmean_num_partials(count),
+                                   s_w_out, st);
+    if (e != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    return cuda_status(launch_quant_pack5(W, w_dtype, N, K, s_w_out, static_cast<uint32_t*>(packed5_out), st));
+}
+
+int bitlinear_unpack_weights5(const void* packed5, int N, int K, int8_t* wq_out, void* stream) {
+    if (!packed5 || !wq_out) return BITLINEAR_ERR_NULL;
+    if (!shape_ok(N, K)) return BITLINEAR_ERR_SHAPE;
+    if (!aligned16(packed5) || !aligned16(wq_out)) return BITLINEAR_ERR_ALIGN;
+    if (int rc = check_arch()) return rc;
+    return cuda_status(launch_unpack5_i8(static_cast<const uint8_t*>(packed5), N, K, wq_out, static_cast<cudaStream_t>(stream)));
+}
+
 int bitlinear_unpack_weights(const void* packed, int N, int K, int8_t* wq_out, void* stream) {
     if (!packed || !wq_out) return BITLINEAR_ERR_NULL;
     if (!shape_ok(N, K)) return BITLINEAR_ERR_SHAPE;

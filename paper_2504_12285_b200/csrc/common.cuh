@@ -14,6 +14,10 @@ constexpr int kTileRows = 16;
 constexpr int kTileCols = 256;
 constexpr int kTileBytes = 1024;
 constexpr int kMaxK = 16384;
+// Dense layout (five ternary values per byte): tiles of 16 rows x 320 columns, also 1024 bytes; K is padded with zero
+// weights to a whole number of tiles.
+constexpr int kDenseTileCols = 320;
+__host__ __device__ inline int dense_k_tiles(int K) { return (K + kDenseTileCols - 1) / kDenseTileCols; }
 constexpr int kGemvMaxTokens = 16;
 
 __host__ __device__ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
@@ -37,6 +41,8 @@ cudaError_t launch_quant_pack(const void* W, int w_dtype, int N, int K, const fl
 cudaError_t launch_unpack_i8(const uint32_t* packed, int N, int K, int8_t* wq, cudaStream_t st);
 cudaError_t launch_unpack_codes_u8(const uint32_t* packed, int N, int K, uint8_t* codes, cudaStream_t st);
 int absmean_num_partials(size_t count);
+cudaError_t launch_quant_pack5(const void* W, int w_dtype, int N, int K, const float* s_w, uint32_t* packed, cudaStream_t st);
+cudaError_t launch_unpack5_i8(const uint8_t* packed, int N, int K, int8_t* wq, cudaStream_t st);
 
 cudaError_t launch_quant_act(const __nv_bfloat16* x, const __nv_bfloat16* gain, float eps, int M, int K,
                              int8_t* xq, float* d, int32_t* xsum, cudaStream_t st);

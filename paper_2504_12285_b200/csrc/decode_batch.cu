@@ -37,9 +37,11 @@ struct DevProblem {
     int8_t* xq;
     float* d;
     int32_t* xsum;
+    int32_t* acc_out;  // nullable: raw accumulators sum_k xq * Wq of this problem, [M][N] (parity hook)
     int M, N, K, y_dtype;
     float eps;
-    int k_tiles;
+    int k_tiles;    // 1024-byte tiles per block of 16 weight rows: K / 256, or ceil(K / 320) in the dense layout
+    int x_stride;   // bytes between the quantised rows of two tokens: K, or 320 * k_tiles in the dense layout (zero padded)
     int rb_begin;   // index of this problem's first row block in the global row-block list
     int rb_end;     // one past its last
     int row_begin;  // index of its first token in the global token list
@@ -70,7 +72,9 @@ constexpr size_t ring_bytes(int chunk_tiles) { return (size_t)kStreamWarps * kRi
 
 // ------------------------------------------------------------------------------------ launch 1
 
-template <int VPT>
+// LAYOUT 1: codes in the lane-interleaved order of the 2-bit stream kernel; LAYOUT 0: plain column order with the row
+// padded with zeros up to x_stride (the dense-layout kernel reads whole tiles of 320 columns).
+template <int VPT, int LAYOUT>
 __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHeader* __restrict__ hdr,
                                                                     const DevProblem* __restrict__ probs,
                                                                     const int* __restrict__ row_prob, int count,
@@ -86,7 +90,10 @@ __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHe
     const int row = blockIdx.x;
     const DevProblem& p = probs[row_prob[row]];
     const int m = row - p.row_begin;
-    quant_row<VPT, 1>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq + (size_t)m * p.K, p.d + m, p.xsum + m, sm);
+    int8_t* xq_row = p.xq + (size_t)m * p.x_stride;
+    quant_row<VPT, LAYOUT>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, xq_row, p.d + m, p.xsum + m, sm);
+    if (LAYOUT == 0)
+        for (int k = p.K + 4 * threadIdx.x; k < p.x_stride; k += 4 * kQuantThreads) *reinterpret_cast<uint32_t*>(xq_row + k) = 0u;
 }
 
 // ------------------------------------------------------------------------------------ launch 2
@@ -122,10 +129,11 @@ struct alignas(16) SProb {
     const uint8_t* packed;
     void* y;
     const int8_t* xq;
-    int rb_begin, rb_end, k_tiles, M, N, K, y_dtype;
+    int32_t* acc_out;
+    int rb_begin, rb_end, k_tiles, M, N, x_stride, y_dtype;
     int x_off;  // byte offset of token 0's codes in the CTA's activation arena
     float s_w;
-    int pad[3];
+    int pad;
     float d;   // the token's scale
     int xsum;  // and code sum
 };
@@ -152,8 +160,15 @@ struct ChunkCursor {
 // One token per problem.  kChunkTiles = 16x256 tiles (1 KiB each) per bulk copy at most.
 // The quantised activations of the problems the CTA touches are staged in shared memory once, as far as the arena
 // reaches; those of the remaining problems are read through L1, which is slower.
-template <int kChunkTiles>
+// FMT 0: the 2-bit layout (tiles of 16 rows x 256 columns).  FMT 1: the dense layout, five values per byte (tiles of 16
+// rows x 320 columns): a lane's 16 bytes are 80 columns of one row; the base-3 digits of the four bytes of a word are
+// peeled off by repeated multiplication by 3 in two 16-bit fields per register (a byte times 3 leaves its digit in the
+// byte above and the remainder in place), gathered into one operand of four codes per digit with a byte permute, and
+// fed to the same dot-product-of-four against four consecutive activations.
+template <int kChunkTiles, int FMT>
 __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const StreamParams prm) {
+    constexpr int kCols = FMT ? kDenseTileCols : kTileCols;   // columns of a tile
+    constexpr int kLaneBytes = FMT ? 80 : 16;                 // activation bytes of a column lane t inside a tile
     extern __shared__ __align__(128) uint8_t smem[];
     // [ring: 16 warps x kRing slots][full barriers][empty barriers][abort flag][descriptor table]
     // [activation arena]
@@ -248,8 +263,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             SProb& e = table[i];
             e.packed = pr.packed;
             e.y = pr.y; e.xq = pr.xq;
+            e.acc_out = pr.acc_out;
             e.rb_begin = pr.rb_begin; e.rb_end = pr.rb_end; e.k_tiles = pr.k_tiles;
-            e.M = pr.M; e.N = pr.N; e.K = pr.K; e.y_dtype = pr.y_dtype;
+            e.M = pr.M; e.N = pr.N; e.x_stride = pr.x_stride; e.y_dtype = pr.y_dtype;
             e.x_off = 0;
             e.s_w = *pr.s_w;
         }
@@ -258,7 +274,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (threadIdx.x == 0) {
         int off = 0;
         for (int i = 0; i < n_tab; ++i) {
-            const int bytes = table[i].M * table[i].K;  // a multiple of 256
+            const int bytes = table[i].M * table[i].x_stride;  // a multiple of 64
             if (off + bytes <= prm.arena_bytes) {
                 table[i].x_off = off;
                 off += bytes;
@@ -284,7 +300,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         const uint32_t arena_s = smem_u32(arena);
         for (int i = 0; i < n_tab; ++i) {
             if (table[i].x_off < 0) continue;
-            const int bytes = table[i].M * table[i].K;
+            const int bytes = table[i].M * table[i].x_stride;
             const int8_t* src = table[i].xq;
             const uint32_t dst = arena_s + (uint32_t)table[i].x_off;
             for (int o = threadIdx.x * 16; o < bytes; o += kStreamThreads * 16) cp_async16(dst + o, src + o);
@@ -307,6 +323,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         // per-problem state of the arithmetic side
         int y_dtype = 0, xs = 0;
         void* y = nullptr;
+        int32_t* acc_out = nullptr;
         float s_w = 0.0f, d = 0.0f;
         bool x_staged = false;
         const int8_t* xrow_g = nullptr;  // the token's codes in global memory
@@ -317,18 +334,18 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             const int8_t* xq = nullptr;
             if (i < n_tab) {
                 const SProb& e = table[i];
-                y_dtype = e.y_dtype; y = e.y; s_w = e.s_w; x_off = e.x_off; xq = e.xq;
+                y_dtype = e.y_dtype; y = e.y; s_w = e.s_w; x_off = e.x_off; xq = e.xq; acc_out = e.acc_out;
                 d = e.d;
                 xs = e.xsum;
             } else {
                 const DevProblem& pr = probs[cp.p];
-                y_dtype = pr.y_dtype; y = pr.y; s_w = *pr.s_w; xq = pr.xq;
+                y_dtype = pr.y_dtype; y = pr.y; s_w = *pr.s_w; xq = pr.xq; acc_out = pr.acc_out;
                 d = pr.d[0];
                 xs = pr.xsum[0];
             }
             x_staged = x_off >= 0;
-            xrow_g = xq + t * 16;
-            xrow_s = smem_u32(arena) + (uint32_t)((x_staged ? x_off : 0) + t * 16);
+            xrow_g = xq + t * kLaneBytes;
+            xrow_s = smem_u32(arena) + (uint32_t)((x_staged ? x_off : 0) + t * kLaneBytes);
         };
         load_problem_state();
 
@@ -347,12 +364,39 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
             auto run_tiles = [&](auto staged) {
                 constexpr bool XS = decltype(staged)::value;  // activations of this problem are in the arena
                 uint32_t wa = ring_s + slot * kSlotBytes + (uint32_t)lane * 16u;
-                uint32_t xo = (uint32_t)(cp.c * cp.ct) * kTileCols;
+                uint32_t xo = (uint32_t)(cp.c * cp.ct) * kCols;
 #pragma unroll 2
-                for (int tile = 0; tile < tiles; ++tile, wa += kTileBytes, xo += kTileCols) {
+                for (int tile = 0; tile < tiles; ++tile, wa += kTileBytes, xo += kCols) {
                     const uint4 w0v = lds128(wa), w1v = lds128(wa + 512);
                     const uint32_t w0[4] = {w0v.x, w0v.y, w0v.z, w0v.w};
                     const uint32_t w1[4] = {w1v.x, w1v.y, w1v.z, w1v.w};
+                    if constexpr (FMT == 1) {
+                        // the lane's 80 activations: word 5 * i + e multiplies digit e of packed word i
+                        uint32_t xw[20];
+#pragma unroll
+                        for (int q = 0; q < 5; ++q) {
+                            uint4 v;
+                            if (XS) v = lds128(xrow_s + xo + 16u * q);
+                            else v = *reinterpret_cast<const uint4*>(xrow_g + xo + 16 * q);
+                            xw[4 * q] = v.x; xw[4 * q + 1] = v.y; xw[4 * q + 2] = v.z; xw[4 * q + 3] = v.w;
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            uint32_t ev[2] = {w0[i] & 0x00ff00ffu, w1[i] & 0x00ff00ffu};                // bytes 0 and 2
+                            uint32_t od[2] = {(w0[i] >> 8) & 0x00ff00ffu, (w1[i] >> 8) & 0x00ff00ffu};  // bytes 1 and 3
+#pragma unroll
+                            for (int e = 0; e < 5; ++e) {
+#pragma unroll
+                                for (int h = 0; h < 2; ++h) {
+                                    const uint32_t me = ev[h] * 3u, mo = od[h] * 3u;  // digit in bits 8-9 of each half
+                                    acc[h][0] = dp4a_u8_s8(__byte_perm(me, mo, 0x7351), xw[5 * i + e], acc[h][0]);
+                                    ev[h] = me & 0x00ff00ffu;
+                                    od[h] = mo & 0x00ff00ffu;
+                                }
+                            }
+                        }
+                        continue;
+                    }
                     // the token's codes are stored with the four 16-byte pieces of each lane's 64 columns interleaved
                     // (piece q of lane t at 64q + 16t inside the tile), so the four t lanes read 64 contiguous bytes
 #pragma unroll
@@ -387,12 +431,15 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
                     // 64 x the sum: ((a0*4 + a1)*4 + a2)*4 + a3; |sum| <= 254*K/4 per lane: no overflow for K <= 8192
-                    int sum = acc[h][0] * 4 + acc[h][1];
-                    sum = sum * 4 + acc[h][2];
-                    sum = sum * 4 + acc[h][3];
+                    int sum = acc[h][0];
+                    if constexpr (FMT == 0) {
+                        sum = sum * 4 + acc[h][1];
+                        sum = sum * 4 + acc[h][2];
+                        sum = sum * 4 + acc[h][3];
+                    }
                     sum += __shfl_xor_sync(0xffffffffu, sum, 1);
                     sum += __shfl_xor_sync(0xffffffffu, sum, 2);
-                    v[h] = sum >> 6;  // exact: a multiple of 64
+                    v[h] = FMT == 0 ? sum >> 6 : sum;  // 2-bit layout: exact, a multiple of 64
 #pragma unroll
                     for (int j = 0; j < 4; ++j) acc[h][j] = 0;
                 }
@@ -402,6 +449,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                     for (int h = 0; h < 2; ++h) {
                         const float val = __fmul_rn(__fmul_rn((float)(v[h] - xs), s_w), d);
                         const size_t idx = (size_t)(n0 + 8 * h);
+                        if (acc_out != nullptr) acc_out[idx] = v[h] - xs;
                         if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
                         else reinterpret_cast<float*>(y)[idx] = val;
                     }
@@ -421,9 +469,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (*abort_flag && threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
 }
 
-template <int kChunkTiles>
+template <int kChunkTiles, int FMT>
 cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<kChunkTiles>,
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<kChunkTiles, FMT>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // programmatic dependent launch: the kernel may begin (barrier set-up, first weight copies) while the quantiser
@@ -438,7 +486,7 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<kChunkTiles>, prm);
+    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<kChunkTiles, FMT>, prm);
 }
 
 struct PlanLayout {
@@ -481,41 +529,60 @@ constexpr int kDp4aMaxTokens = 1;
 
 namespace {
 
+// Bytes between the quantised rows of two tokens of a problem: K, or K padded to whole 320-column tiles (dense layout).
+inline int x_stride_of(const bitlinear_problem& q) {
+    return q.w_format == BITLINEAR_WEIGHTS_DENSE5 ? dense_k_tiles(q.K) * kDenseTileCols : q.K;
+}
+
 size_t decode_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
     if (!problems || count <= 0) return 0;
     size_t xq = 0, rows = 0;
     int max_m = 0;
+    const int fmt = problems[0].w_format;
     for (int i = 0; i < count; ++i) {
         const bitlinear_problem& q = problems[i];
-        if (q.M < 0 || q.M > kGemvMaxTokens || !shape_ok(q.N, q.K) || q.K > kBatchMaxK) return 0;
-        xq += align_up((size_t)q.M * q.K, 16);
+        if (q.M < 0 || q.M > kGemvMaxTokens || !shape_ok(q.N, q.K) || q.K > kBatchMaxK || q.w_format != fmt) return 0;
+        xq += align_up((size_t)q.M * x_stride_of(q), 16);
         rows += (size_t)q.M;
         if (q.M > max_m) max_m = q.M;
     }
-    if (max_m > kDp4aMaxTokens) return decode_mma_workspace_bytes(problems, count);
-    return plan_layout(count, kPlanGrid, xq, rows).total;
+    if (fmt == BITLINEAR_WEIGHTS_2BIT && max_m > kDp4aMaxTokens) return decode_mma_workspace_bytes(problems, count);
+    // the dense-layout kernel takes one token per problem: a problem of M tokens is planned as M problems
+    return plan_layout(fmt == BITLINEAR_WEIGHTS_DENSE5 ? (int)rows : count, kPlanGrid, xq, rows).total;
 }
 
-int decode_batch_forward(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
-                         void* stream) {
+// acc_outs: nullptr, or one (nullable) device pointer per problem for the raw accumulators.
+int decode_batch_forward(const bitlinear_problem* problems, int count, int flags, int32_t* const* acc_outs, void* ws,
+                         size_t ws_bytes, void* stream) {
     size_t xq_bytes = 0, rows = 0;
     int max_m = 0, max_k = 0;
+    const int fmt = problems[0].w_format;
+    const bool dense = fmt == BITLINEAR_WEIGHTS_DENSE5;
+    bool want_acc = false;
     for (int i = 0; i < count; ++i) {
         const bitlinear_problem& q = problems[i];
         if (q.y_dtype != BITLINEAR_F32 && q.y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
+        if (q.w_format != fmt) return BITLINEAR_ERR_DTYPE;  // one weight layout per call
         if (q.M < 0 || q.M > kGemvMaxTokens || !shape_ok(q.N, q.K) || q.K > kBatchMaxK) return BITLINEAR_ERR_SHAPE;
+        if (acc_outs && acc_outs[i]) {
+            if (reinterpret_cast<uintptr_t>(acc_outs[i]) & 3u) return BITLINEAR_ERR_ALIGN;
+            want_acc = true;
+        }
         if (q.M == 0) continue;
         if (!q.x || !q.packed || !q.s_w || !q.y) return BITLINEAR_ERR_NULL;
         if (!aligned16(q.x) || !aligned16(q.packed) || !aligned16(q.y) || (q.gain && !aligned16(q.gain)) ||
             (reinterpret_cast<uintptr_t>(q.s_w) & 3u))
             return BITLINEAR_ERR_ALIGN;
-        xq_bytes += align_up((size_t)q.M * q.K, 16);
+        xq_bytes += align_up((size_t)q.M * x_stride_of(q), 16);
         rows += (size_t)q.M;
         if (q.M > max_m) max_m = q.M;
         if (q.K > max_k) max_k = q.K;
     }
-    if (max_m > kDp4aMaxTokens) return decode_mma_forward(problems, count, flags, ws, ws_bytes, stream);
-    const PlanLayout L = plan_layout(count, kPlanGrid, xq_bytes, rows);
+    if (!dense && max_m > kDp4aMaxTokens) {
+        if (want_acc) return BITLINEAR_ERR_SHAPE;  // the tensor-core decode kernel has no accumulator output
+        return decode_mma_forward(problems, count, flags, ws, ws_bytes, stream);
+    }
+    const PlanLayout L = plan_layout(dense ? (int)rows : count, kPlanGrid, xq_bytes, rows);
     if (!ws || !aligned16(ws) || ws_bytes < L.total) return BITLINEAR_ERR_WORKSPACE;
     if (rows == 0) return BITLINEAR_OK;
 
@@ -548,26 +615,35 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         for (int i = 0; i < count; ++i) {
             const bitlinear_problem& q = problems[i];
             if (q.M == 0) continue;
-            DevProblem v;
-            v.packed = static_cast<const uint8_t*>(q.packed);
-            v.s_w = q.s_w;
-            v.y = q.y;
-            v.x = static_cast<const __nv_bfloat16*>(q.x);
-            v.gain = static_cast<const __nv_bfloat16*>(q.gain);
-            v.xq = reinterpret_cast<int8_t*>(xq_ptr);
-            v.d = d_ptr + row;
-            v.xsum = xs_ptr + row;
-            v.M = q.M; v.N = q.N; v.K = q.K; v.y_dtype = q.y_dtype;
-            v.eps = q.rms_eps;
-            v.k_tiles = q.K / kTileCols;
-            v.rb_begin = total_rb;
-            v.rb_end = total_rb + q.N / kTileRows;
-            v.row_begin = row;
-            for (int m = 0; m < q.M; ++m) row_prob.push_back((int)dp.size());
-            dp.push_back(v);
-            total_rb = v.rb_end;
-            row += q.M;
-            xq_ptr += align_up((size_t)q.M * q.K, 16);
+            const int stride = x_stride_of(q);
+            const size_t y_row = (size_t)q.N * (q.y_dtype == BITLINEAR_BF16 ? 2 : 4);
+            // the dense-layout kernel multiplies one token per problem: every token becomes a problem of its own
+            // (its weights are then streamed once per token)
+            const int parts = dense ? q.M : 1, m_each = dense ? 1 : q.M;
+            for (int part = 0; part < parts; ++part) {
+                DevProblem v;
+                v.packed = static_cast<const uint8_t*>(q.packed);
+                v.s_w = q.s_w;
+                v.y = static_cast<char*>(q.y) + (size_t)part * y_row;
+                v.x = static_cast<const __nv_bfloat16*>(q.x) + (size_t)part * q.K;
+                v.gain = static_cast<const __nv_bfloat16*>(q.gain);
+                v.xq = reinterpret_cast<int8_t*>(xq_ptr) + (size_t)part * stride;
+                v.d = d_ptr + row;
+                v.xsum = xs_ptr + row;
+                v.acc_out = (acc_outs && acc_outs[i]) ? acc_outs[i] + (size_t)part * q.N : nullptr;
+                v.M = m_each; v.N = q.N; v.K = q.K; v.y_dtype = q.y_dtype;
+                v.eps = q.rms_eps;
+                v.k_tiles = dense ? dense_k_tiles(q.K) : q.K / kTileCols;
+                v.x_stride = stride;
+                v.rb_begin = total_rb;
+                v.rb_end = total_rb + q.N / kTileRows;
+                v.row_begin = row;
+                for (int m = 0; m < m_each; ++m) row_prob.push_back((int)dp.size());
+                dp.push_back(v);
+                total_rb = v.rb_end;
+                row += m_each;
+            }
+            xq_ptr += align_up((size_t)q.M * stride, 16);
         }
         row_prob.push_back(0);
     }
@@ -605,7 +681,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
             if (lo < hi) {
                 if (pl - pf + 1 > table_cap) table_cap = pl - pf + 1;
                 size_t a = 0;
-                for (int i = pf; i <= pl; ++i) a += (size_t)dp[i].M * dp[i].K;
+                for (int i = pf; i <= pl; ++i) a += (size_t)dp[i].M * dp[i].x_stride;
                 if (a > arena_max) arena_max = a;
             }
         }
@@ -643,9 +719,15 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         const PlanHeader* h = reinterpret_cast<const PlanHeader*>(base);
         const int* rp = reinterpret_cast<const int*>(base + L.row_prob_off);
         int* sw = device_status_word();
-        if (vpt <= 1) batch_quant_kernel<1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
-        else if (vpt <= 2) batch_quant_kernel<2><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
-        else batch_quant_kernel<4><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+        if (dense) {
+            if (vpt <= 1) batch_quant_kernel<1, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+            else if (vpt <= 2) batch_quant_kernel<2, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+            else batch_quant_kernel<4, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+        } else {
+            if (vpt <= 1) batch_quant_kernel<1, 1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+            else if (vpt <= 2) batch_quant_kernel<2, 1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+            else batch_quant_kernel<4, 1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+        }
         if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
 
@@ -661,7 +743,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.table_cap = table_cap;
     prm.arena_bytes = (int)arena_max;
     const size_t smem = ring_bytes(chunk_tiles) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
-    const cudaError_t e = launch_stream<chunk_tiles>(prm, grid, smem, st);
+    const cudaError_t e = dense ? launch_stream<chunk_tiles, 1>(prm, grid, smem, st) : launch_stream<chunk_tiles, 0>(prm, grid, smem, st);
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
@@ -680,11 +762,12 @@ size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int co
     for (int i = 0; i < count; ++i) {
         const bitlinear_problem& q = problems[i];
         if (q.M < 0 || !shape_ok(q.N, q.K)) return 0;
+        if (q.w_format != BITLINEAR_WEIGHTS_2BIT && q.w_format != BITLINEAR_WEIGHTS_DENSE5) return 0;
         if (q.M <= kGemvMaxTokens) {
             if (q.K > kBatchMaxK) return 0;
             dec.push_back(q);
         } else {
-            if (q.N % 128) return 0;
+            if (q.N % 128 || q.w_format != BITLINEAR_WEIGHTS_2BIT) return 0;
             pre.push_back(i);
         }
     }
@@ -696,22 +779,31 @@ size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int co
 
 int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
                             void* stream) {
+    return bitlinear_forward_batch_acc(problems, count, flags, nullptr, ws, ws_bytes, stream);
+}
+
+int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, int flags, int32_t* const* acc_out,
+                                void* ws, size_t ws_bytes, void* stream) {
     if (count < 0) return BITLINEAR_ERR_SHAPE;
     if (count == 0) return BITLINEAR_OK;
     if (!problems) return BITLINEAR_ERR_NULL;
     if (flags & ~(BITLINEAR_BATCH_REUSE_PLAN | BITLINEAR_BATCH_REUSE_ACT)) return BITLINEAR_ERR_DTYPE;
     std::vector<bitlinear_problem> dec;
+    std::vector<int32_t*> dec_acc;
     std::vector<int> pre;
     for (int i = 0; i < count; ++i) {
         const bitlinear_problem& q = problems[i];
         if (q.y_dtype != BITLINEAR_F32 && q.y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
+        if (q.w_format != BITLINEAR_WEIGHTS_2BIT && q.w_format != BITLINEAR_WEIGHTS_DENSE5) return BITLINEAR_ERR_DTYPE;
         if (q.M < 0 || !shape_ok(q.N, q.K)) return BITLINEAR_ERR_SHAPE;
         if (q.M <= kGemvMaxTokens) {
             if (q.K > kBatchMaxK) return BITLINEAR_ERR_SHAPE;
             dec.push_back(q);
+            dec_acc.push_back(acc_out ? acc_out[i] : nullptr);
             continue;
         }
-        if (q.N % 128) return BITLINEAR_ERR_SHAPE;
+        // more than 16 tokens: the tensor-core path, which reads the 2-bit layout and has no accumulator output
+        if (q.N % 128 || q.w_format != BITLINEAR_WEIGHTS_2BIT || (acc_out && acc_out[i])) return BITLINEAR_ERR_SHAPE;
         if (!q.x || !q.packed || !q.s_w || !q.y) return BITLINEAR_ERR_NULL;
         if (!aligned16(q.x) || !aligned16(q.packed) || !aligned16(q.y) || (q.gain && !aligned16(q.gain)) ||
             (reinterpret_cast<uintptr_t>(q.s_w) & 3u))
@@ -722,7 +814,7 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
     const size_t pre_bytes = pre.empty() ? 0 : prefill_group_workspace_bytes(problems, pre.data(), (int)pre.size());
     if (!ws || !aligned16(ws) || ws_bytes < dec_bytes + pre_bytes) return BITLINEAR_ERR_WORKSPACE;
     if (!dec.empty()) {
-        const int rc = decode_batch_forward(dec.data(), (int)dec.size(), flags, ws, dec_bytes, stream);
+        const int rc = decode_batch_forward(dec.data(), (int)dec.size(), flags, acc_out ? dec_acc.data() : nullptr, ws, dec_bytes, stream);
         if (rc != BITLINEAR_OK) return rc;
     }
     if (!pre.empty()) {

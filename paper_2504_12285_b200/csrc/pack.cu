@@ -152,7 +152,78 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint32_t* __restrict_
     *reinterpret_cast<uint4*>(out + (size_t)n * K + k0) = make_uint4(v[0], v[1], v[2], v[3]);
 }
 
+// ---- dense layout: five ternary values per byte (see "Dense packed weight layout" in bitlinear.h) ----
+
+// One thread quantises the 20 consecutive weights of one packed 32-bit word: column k0 + 4*e + b is base-3 digit e
+// (digit 0 most significant) of byte b; columns past K are padding and count as zero weights.
+template <typename T>
+__global__ void __launch_bounds__(256) quant_pack5_kernel(const T* __restrict__ W, int N, int K,
+                                                          const float* __restrict__ s_w_ptr,
+                                                          uint32_t* __restrict__ packed) {
+    const int k_tiles = dense_k_tiles(K);
+    const size_t n_words = (size_t)(N / kTileRows) * k_tiles * (kTileBytes / 4);
+    const size_t word = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (word >= n_words) return;
+    const float s_w = *s_w_ptr;
+    const size_t tile = word >> 8;
+    const int wo = (int)(word & 255);
+    const int h = wo >> 7, g = (wo >> 4) & 7, t = (wo >> 2) & 3, i = wo & 3;
+    const int n = (int)(tile / k_tiles) * kTileRows + 8 * h + g;
+    const int k0 = (int)(tile % k_tiles) * kDenseTileCols + 80 * t + 20 * i;
+    const T* src = W + (size_t)n * K;
+    uint32_t v[4] = {0u, 0u, 0u, 0u};  // the base-3 number of each byte, built digit by digit
+#pragma unroll
+    for (int e = 0; e < 5; ++e)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int k = k0 + 4 * e + b;
+            uint32_t c = 1u;
+            if (k < K) {
+                float w;
+                if constexpr (sizeof(T) == 2) w = __bfloat162float(src[k]);
+                else w = src[k];
+                c = ternary_code(w, s_w);
+            }
+            v[b] = v[b] * 3u + c;
+        }
+    uint32_t out = 0;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) out |= ((256u * v[b] + 242u) / 243u) << (8 * b);  // ceil(256 v / 243)
+    packed[word] = out;
+}
+
+// Test hook: one thread per weight; the byte's base-3 number is recovered as floor(243 B / 256) and the digit by division.
+__global__ void __launch_bounds__(256) unpack5_kernel(const uint8_t* __restrict__ packed, int N, int K, int8_t* __restrict__ out) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)N * K) return;
+    const int n = (int)(idx / K), k = (int)(idx - (size_t)n * K);
+    const int k_tiles = dense_k_tiles(K);
+    const size_t tile = (size_t)(n / kTileRows) * k_tiles + k / kDenseTileCols;
+    const int r = n % kTileRows, c = k % kDenseTileCols;
+    const int t = c / 80, i = (c % 80) / 20, e = (c % 20) / 4, b = c % 4;
+    const uint32_t B = packed[tile * kTileBytes + 512 * (r / 8) + 64 * (r % 8) + 16 * t + 4 * i + b];
+    uint32_t v = (243u * B) >> 8;
+    for (int s = e; s < 4; ++s) v /= 3u;
+    out[idx] = (int8_t)((int)(v % 3u) - 1);
+}
+
 }  // namespace
+
+cudaError_t launch_quant_pack5(const void* W, int w_dtype, int N, int K, const float* s_w, uint32_t* packed, cudaStream_t st) {
+    const size_t n_words = (size_t)(N / kTileRows) * dense_k_tiles(K) * (kTileBytes / 4);
+    const unsigned blocks = (unsigned)((n_words + 255) / 256);
+    if (w_dtype == BITLINEAR_BF16)
+        quant_pack5_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W), N, K, s_w, packed);
+    else
+        quant_pack5_kernel<float><<<blocks, 256, 0, st>>>(static_cast<const float*>(W), N, K, s_w, packed);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack5_i8(const uint8_t* packed, int N, int K, int8_t* wq, cudaStream_t st) {
+    const size_t n = (size_t)N * K;
+    unpack5_kernel<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(packed, N, K, wq);
+    return cudaGetLastError();
+}
 
 int absmean_num_partials(size_t count) {
     size_t want = (count + (size_t)kRedThreads * 64 - 1) / ((size_t)kRedThreads * 64);
