@@ -383,7 +383,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
                             uint32_t ev[2] = {w0[i] & 0x00ff00ffu, w1[i] & 0x00ff00ffu};                // bytes 0 and 2
-                            uint32_t od[2] = {(w0[i] >> 8) & 0x00ff00ffu, (w1[i] >> 8) & 0x00ff00ffu};  // bytes 1 and 3
+                            uint32_t od[2] = {__byte_perm(w0[i], 0u, 0x4341), __byte_perm(w1[i], 0u, 0x4341)};  // bytes 1 and 3
 #pragma unroll
                             for (int e = 0; e < 5; ++e) {
 #pragma unroll
