@@ -353,6 +353,15 @@ int bitlinear_forward_static(const void* x_bf16, const void* gain, float rms_eps
  * Synchronises `stream` first. */
 int bitlinear_poll_status(void* stream);
 
+/*
+ * Self-test of the bounded device-side waits (no counterpart in the paper: every kernel of this library waits on
+ * barriers - for copies, for other warps, for other CTAs - and every such wait has a time limit, 2 s in production).
+ * Launches one small CTA that waits, with a limit of limit_us microseconds (1 .. 100000), on a barrier nobody arrives
+ * on.  The kernel gives up by itself, the context stays usable, and the next bitlinear_poll_status reports
+ * BITLINEAR_ERR_TIMEOUT once.  Nothing else is touched.
+ */
+int bitlinear_selftest_wait_timeout(unsigned limit_us, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

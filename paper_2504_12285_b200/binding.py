@@ -46,6 +46,7 @@ _SIGNATURES = {
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
+    "bitlinear_selftest_wait_timeout": (_c_int, [ctypes.c_uint, _c_void_p]),
     "bitlinear_glue_relu2_mul": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
     "bitlinear_glue_residual_add": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
     "bitlinear_glue_attn_standin": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_void_p]),
@@ -434,6 +435,11 @@ def bitlinear_forward_batch_host(batch: ProblemBatch, x_host: torch.Tensor, x_de
                                             BATCH_REUSE_PLAN if reuse_plan else 0, _ptr(x_host), _ptr(x_dev), xb,
                                             _ptr(y_dev), _ptr(y_host), yb, _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_forward_batch_host")
+
+
+def bitlinear_selftest_wait_timeout(limit_us: int = 1000) -> None:
+    """Launch the bounded-wait self-test: a tiny kernel whose wait runs out after limit_us microseconds."""
+    _check(lib().bitlinear_selftest_wait_timeout(int(limit_us), _stream()), "bitlinear_selftest_wait_timeout")
 
 
 def bitlinear_poll_status() -> int:

@@ -2,12 +2,30 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "sm100_sync.cuh"
 
 namespace bitlinear {
 
 namespace {
 
 __device__ int g_status_word = 0;
+
+// One CTA waits on an mbarrier that nobody ever arrives on: the bounded wait must give up after limit_ns, raise the
+// CTA's abort flag and let the kernel end by itself with the sticky status word set - the path every production kernel
+// takes when one of its waits runs out.
+__global__ void __launch_bounds__(64) wait_timeout_selftest_kernel(unsigned long long limit_ns, int* status_word) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        abort_flag = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const bool ok = mbar_wait(smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!ok || abort_flag) && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
+}
 
 constexpr size_t kWsAlign = 256;
 
@@ -42,6 +60,28 @@ bool use_gemm(int M, int N, int path) {
 }
 
 }  // namespace
+
+int device_sm_count(int* sm_count) {
+    static std::mutex mu;
+    static int sm_of[64];
+    if (int rc = check_arch()) return rc;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (sm_of[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+            cudaGetLastError();
+            return BITLINEAR_ERR_CUDA;
+        }
+        sm_of[dev] = n;
+    }
+    *sm_count = sm_of[dev];
+    return BITLINEAR_OK;
+}
 
 int* device_status_word() {
     int* p = nullptr;
@@ -254,6 +294,15 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
         return BITLINEAR_ERR_CUDA;
     }
     return BITLINEAR_OK;
+}
+
+int bitlinear_selftest_wait_timeout(unsigned limit_us, void* stream) {
+    if (limit_us == 0 || limit_us > 100000u) return BITLINEAR_ERR_SHAPE;  // 100 ms at most
+    if (int rc = check_arch()) return rc;
+    int* word = device_status_word();
+    if (!word) return BITLINEAR_ERR_CUDA;
+    wait_timeout_selftest_kernel<<<1, 64, 0, static_cast<cudaStream_t>(stream)>>>((unsigned long long)limit_us * 1000ull, word);
+    return cuda_status(cudaGetLastError());
 }
 
 int bitlinear_poll_status(void* stream) {

@@ -100,6 +100,9 @@ int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const ui
                  int M, int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st);
 size_t gemm_scratch_bytes(int N, int K);
 
+// SM count of the current device (cached per device; BITLINEAR_ERR_ARCH unless it is compute capability 10.x).
+int device_sm_count(int* sm_count);
+
 // Sticky device-side status word (set by kernels whose bounded waits ran out).
 int* device_status_word();
 

@@ -586,18 +586,8 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     if (!ws || !aligned16(ws) || ws_bytes < L.total) return BITLINEAR_ERR_WORKSPACE;
     if (rows == 0) return BITLINEAR_OK;
 
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0, n = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) {
-            cudaGetLastError();
-            return BITLINEAR_ERR_CUDA;
-        }
-        int major = 0;
-        cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
-        if (major != 10) return BITLINEAR_ERR_ARCH;
-        sm_count = n;
-    }
+    int sm_count = 0;
+    if (const int rc = device_sm_count(&sm_count)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ws);
 

@@ -494,20 +494,12 @@ size_t decode_mma_workspace_bytes(const bitlinear_problem* problems, int count) 
 int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes, void* stream) {
     const MmaLayout L = mma_layout(problems, count);
     if (!ws || !aligned16(ws) || ws_bytes < L.total) return BITLINEAR_ERR_WORKSPACE;
-    static int sm_count = 0;
-    if (sm_count == 0) {
-        int dev = 0, n = 0, major = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
-            cudaGetLastError();
-            return BITLINEAR_ERR_CUDA;
-        }
-        if (major != 10) return BITLINEAR_ERR_ARCH;
-        if (cudaFuncSetAttribute(decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem) != cudaSuccess) {
-            cudaGetLastError();
-            return BITLINEAR_ERR_CUDA;
-        }
-        sm_count = n;
+    int sm_count = 0;
+    if (const int rc = device_sm_count(&sm_count)) return rc;
+    // the attribute is per device and cheap to set: done on every call, like the streaming kernel's launcher does
+    if (cudaFuncSetAttribute(decode_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kMmaSmem) != cudaSuccess) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ws);

@@ -19,6 +19,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "sm100_sync.cuh"
 
 namespace bitlinear {
 
@@ -35,66 +36,12 @@ constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr int THREADS = 192;
 constexpr uint32_t TMEM_COLS = 512;  // two accumulator buffers of 256 columns
 constexpr size_t SMEM_BYTES = 1024 /*alignment slack*/ + (size_t)STAGES * STAGE_BYTES + 256 /*barriers*/ + 4 * 32 * 144 /*epilogue staging*/ + 3072 /*group table*/;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
-
-// ---- thin PTX wrappers -------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return done;
-}
-
-// Bounded wait: false if the CTA is aborting or the time limit ran out (which raises the abort flag).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
-    for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = 1;
-                return false;
-            }
-        }
-    }
-}
-
+// ---- thin PTX wrappers (mbarrier, bulk copy and the bounded wait come from sm100_sync.cuh) --------------------
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar)
         : "memory");
-}
-
-// Linear bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
 }
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -384,9 +331,7 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
-        // give copies that may still be in flight time to land before shared memory is released
-        const unsigned long long t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+        abort_drain();  // copies that may still be in flight land before shared memory is released
         if (threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
         __syncthreads();
     }
@@ -514,7 +459,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
                     while (ld_acquire_gpu_s32(hdr.ready + p.nt_begin + nt) < target) {
                         if ((++spins & 63u) == 0u) {
                             if (*abort_flag) { ok = false; break; }
-                            if (globaltimer_ns() - t0 > WAIT_LIMIT_NS) { *abort_flag = 1; ok = false; break; }
+                            if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; ok = false; break; }
                         }
                     }
                     if (!ok) break;
@@ -592,8 +537,7 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
     tc_fence_before();
     __syncthreads();
     if (*abort_flag) {
-        const unsigned long long t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+        abort_drain();
         if (threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
         __syncthreads();
     }
@@ -661,22 +605,29 @@ bool make_map_rows128(CUtensorMap* map, const void* base, size_t bytes) {
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev,
                 cudaStream_t st, const void* region_base, size_t region_bytes, const int* ready, GemmBeforeKernel before,
                 void* before_ctx, bool wait_primary) {
-    static std::once_flag attr_once;
-    static cudaError_t attr_err = cudaSuccess;
-    static int sm_count = 0;
-    std::call_once(attr_once, [] {
-        attr_err = cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES);
-        if (attr_err == cudaSuccess)
-            attr_err = cudaFuncSetAttribute(gemm_i8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P_SMEM_BYTES);
+    // kernel attributes and the SM count are per device: set / looked up once for each device a process uses
+    int sm_count = 0;
+    {
+        static std::mutex mu;
+        static int sm_of[64];  // 0 = this device has not been set up yet
         int dev = 0;
-        if (attr_err == cudaSuccess) attr_err = cudaGetDevice(&dev);
-        if (attr_err == cudaSuccess) attr_err = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev);
-    });
-    if (attr_err != cudaSuccess || sm_count <= 0) {
-        cudaGetLastError();
-        return BITLINEAR_ERR_CUDA;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+            cudaGetLastError();
+            return BITLINEAR_ERR_CUDA;
+        }
+        std::lock_guard<std::mutex> lock(mu);
+        if (sm_of[dev] == 0) {
+            int n = 0;
+            if (cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess ||
+                cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess ||
+                cudaFuncSetAttribute(gemm_i8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P_SMEM_BYTES) != cudaSuccess ||
+                cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
+                cudaGetLastError();
+                return BITLINEAR_ERR_CUDA;
+            }
+            sm_of[dev] = n;
+        }
+        sm_count = sm_of[dev];
     }
     if (count < 1 || count > kMaxGroup || (!a_tiled && count != 1)) return BITLINEAR_ERR_SHAPE;
     alignas(16) uint8_t host[kGroupTableBytes] = {};
