@@ -226,3 +226,57 @@ def bitlinear_forward(x_bf16: np.ndarray, gain_bf16, rms_eps: float, wq: np.ndar
     acc = matmul_i32(a["q"], wq)
     y = dequant(acc, s_w, a["d"])
     return dict(q=a["q"], d=a["d"], xsum=a["xsum"], fragile=a["fragile"], acc=acc, y=y)
+
+
+# ---- glue between the BitLinear matmuls of a decoder layer (paper Section 2: squared ReLU in the feed-forward block,
+# ---- residual connections), each followed by the next BitLinear's own RMSNorm + quantiser.  One fp32 operation per
+# ---- arithmetic step, then one round-to-nearest-even cast to bf16: the next BitLinear reads bf16.
+
+
+def glue_relu2(gate: np.ndarray, up: np.ndarray) -> np.ndarray:
+    """f = bf16( fl32( fl32(r * r) * up ) ), r = max(gate, 0)  ->  bf16 bit patterns."""
+    gate, up = _c(gate, np.float32), _c(up, np.float32)
+    r = np.maximum(gate, np.float32(0.0))
+    return f32_to_bf16(((r * r).astype(np.float32) * up).astype(np.float32))
+
+
+def glue_residual(h_bits: np.ndarray, y: np.ndarray) -> np.ndarray:
+    """h' = bf16( fl32( float(h) + y ) )  ->  bf16 bit patterns."""
+    return f32_to_bf16((bf16_to_f32(h_bits) + _c(y, np.float32)).astype(np.float32))
+
+
+def glue_attn_standin(q: np.ndarray, v: np.ndarray, n_q_heads: int, n_kv_heads: int, head_dim: int) -> np.ndarray:
+    """Stand-in for attention (which is not a BitLinear): a[m, h*D + j] = bf16( fl32( q[m, h*D + j] + v[m, kv(h)*D + j] ) ),
+    kv(h) = h // (n_q_heads // n_kv_heads)."""
+    q, v = _c(q, np.float32), _c(v, np.float32)
+    group = n_q_heads // n_kv_heads
+    a = np.empty_like(q)
+    for head in range(n_q_heads):
+        kv = head // group
+        a[:, head * head_dim:(head + 1) * head_dim] = (q[:, head * head_dim:(head + 1) * head_dim] +
+                                                       v[:, kv * head_dim:(kv + 1) * head_dim]).astype(np.float32)
+    return f32_to_bf16(a)
+
+
+def relu2_rmsnorm_quant(gate, up, gain_bf16, eps: float):
+    """Squared-ReLU gate fused with the down projection's sub-LN + int8 quantiser: rmsnorm_quant(glue_relu2(gate, up)).
+    Returns the dict of rmsnorm_quant plus x = the bf16 bit patterns that were quantised."""
+    x = glue_relu2(gate, up)
+    out = rmsnorm_quant(x, gain_bf16, eps)
+    out["x"] = x
+    return out
+
+
+def residual_rmsnorm_quant(h_bits, y, gain_bf16, eps: float):
+    """Residual add fused with the next BitLinear's RMSNorm + quantiser; x = the new hidden state (bf16 bits)."""
+    x = glue_residual(h_bits, y)
+    out = rmsnorm_quant(x, gain_bf16, eps)
+    out["x"] = x
+    return out
+
+
+def attn_standin_rmsnorm_quant(q, v, n_q_heads: int, n_kv_heads: int, head_dim: int, gain_bf16, eps: float):
+    x = glue_attn_standin(q, v, n_q_heads, n_kv_heads, head_dim)
+    out = rmsnorm_quant(x, gain_bf16, eps)
+    out["x"] = x
+    return out

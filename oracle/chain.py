@@ -18,7 +18,7 @@ from __future__ import annotations
 
 import numpy as np
 
-from . import bf16_to_f32, bitlinear_forward, f32_to_bf16
+from . import bitlinear_forward, glue_attn_standin, glue_relu2, glue_residual
 
 
 def _bitlinear(x_bits, mat, rms_eps):
@@ -29,26 +29,15 @@ def decode_chain(h_bits: np.ndarray, layers, n_q_heads: int, n_kv_heads: int, he
     """h_bits: uint16 [M, H] bf16 bit patterns.  layers: list of dicts name -> dict(wq, s_w[, gain]) for the names
     q, k, v, o, gate, up, down.  Returns dict(h=final hidden bits, k=last layer's k projection fp32)."""
     h = np.array(h_bits, dtype=np.uint16, copy=True)
-    M = h.shape[0]
-    group = n_q_heads // n_kv_heads
     k_last = None
     for layer in layers:
         q = _bitlinear(h, layer["q"], rms_eps)
         k_last = _bitlinear(h, layer["k"], rms_eps)
         v = _bitlinear(h, layer["v"], rms_eps)
-        a = np.empty((M, n_q_heads * head_dim), np.float32)
-        for head in range(n_q_heads):
-            kv = head // group
-            a[:, head * head_dim:(head + 1) * head_dim] = (
-                q[:, head * head_dim:(head + 1) * head_dim] + v[:, kv * head_dim:(kv + 1) * head_dim]).astype(np.float32)
-        a_bits = f32_to_bf16(a)
-        o = _bitlinear(a_bits, layer["o"], rms_eps)
-        h = f32_to_bf16((bf16_to_f32(h) + o).astype(np.float32))
+        a_bits = glue_attn_standin(q, v, n_q_heads, n_kv_heads, head_dim)
+        h = glue_residual(h, _bitlinear(a_bits, layer["o"], rms_eps))
         g = _bitlinear(h, layer["gate"], rms_eps)
         u = _bitlinear(h, layer["up"], rms_eps)
-        r = np.maximum(g, np.float32(0.0))
-        f = ((r * r).astype(np.float32) * u).astype(np.float32)
-        f_bits = f32_to_bf16(f)
-        dn = _bitlinear(f_bits, layer["down"], rms_eps)
-        h = f32_to_bf16((bf16_to_f32(h) + dn).astype(np.float32))
+        f_bits = glue_relu2(g, u)
+        h = glue_residual(h, _bitlinear(f_bits, layer["down"], rms_eps))
     return dict(h=h, k=k_last)

@@ -483,3 +483,51 @@ def test_chain_attention_standin_and_relu2_by_hand():
     f_bits = bf(((r * r).astype(np.float32) * u).astype(np.float32))
     h2 = bf((oracle.bf16_to_f32(h1).astype(np.float64) + lin(f_bits, mats["down"])).astype(np.float32))
     assert np.array_equal(out["h"], h2)
+
+
+# --------------------------------------------------------------------------- glue fused into the quantiser
+
+
+def test_glue_functions_by_hand():
+    bf = lambda a: oracle.bf16_to_f32(a)  # noqa: E731
+    # squared ReLU gate: negative gates give 0 whatever `up` is; bf16 keeps 8 significant bits
+    f = bf(oracle.glue_relu2(np.array([[-1.0, 2.0, 0.5, 3.0, 1.5]], np.float32), np.array([[5.0, 0.25, -4.0, 1.0, 1.0078125]], np.float32)))
+    #  r*r = 0, 4, 0.25, 9, 2.25 ; times up = 0, 1, -1, 9, 2.267578125 -> bf16: 2.265625 (2.2676 lies between 2.265625 and 2.28125)
+    assert f.tolist() == [[0.0, 1.0, -1.0, 9.0, 2.265625]]
+    # residual: exact tie 1 + 2^-8 rounds to even (1.0); 1 + 3 * 2^-8 rounds up to 1 + 2^-6
+    h = oracle.f32_to_bf16(np.array([[1.0, 1.0, -2.0]], np.float32))
+    out = bf(oracle.glue_residual(h, np.array([[2.0 ** -8, 3 * 2.0 ** -8, 0.5]], np.float32)))
+    assert out.tolist() == [[1.0, 1.015625, -1.5]]
+    # stand-in: 4 query heads on 2 KV heads of width 2: heads 0,1 read KV head 0, heads 2,3 read KV head 1
+    q = np.arange(8, dtype=np.float32).reshape(1, 8)
+    v = np.array([[100.0, 200.0, 300.0, 400.0]], np.float32)
+    a = bf(oracle.glue_attn_standin(q, v, 4, 2, 2))
+    # 405 and 407 need nine significant bits: both are ties and round to the even neighbour (404, 408)
+    assert a.tolist() == [[100.0, 201.0, 102.0, 203.0, 304.0, 404.0, 306.0, 408.0]]
+
+
+def test_fused_glue_quantisers_are_glue_then_quantiser():
+    rng = np.random.default_rng(12)
+    M, F = 3, 512
+    gate = rng.standard_normal((M, F)).astype(np.float32)
+    up = rng.standard_normal((M, F)).astype(np.float32)
+    gain = oracle.f32_to_bf16((1 + 0.25 * rng.standard_normal(F)).astype(np.float32))
+    out = oracle.relu2_rmsnorm_quant(gate, up, gain, 1e-5)
+    # closed form of the quantiser on a row whose gates are all negative: x = 0, codes 0, scale floor 1e-5 / 127
+    z = oracle.relu2_rmsnorm_quant(-np.abs(gate), up, gain, 1e-5)
+    assert not z["q"].any() and np.all(z["d"] == np.float32(1e-5) / np.float32(127.0)) and not z["x"].any()
+    # about half of the gates are negative, so about half of the inputs of the quantiser are exactly zero
+    assert 0.4 < (out["x"] == 0).mean() < 0.6
+    # every non-zero row reaches +-127 and the norm is applied to the bf16-rounded product (textbook fp64 check)
+    assert np.all(np.abs(out["q"]).max(axis=1) == 127)
+    x = oracle.bf16_to_f32(out["x"]).astype(np.float64)
+    g64 = oracle.bf16_to_f32(gain).astype(np.float64)
+    yn = x / np.sqrt((x * x).mean(axis=1, keepdims=True) + 1e-5) * g64
+    a = np.abs(yn).max(axis=1, keepdims=True)
+    assert np.abs(out["q"] - yn * 127.0 / a).max() <= 0.5 + 1e-3
+    # residual and stand-in variants: x is the glue result, the rest the plain quantiser of that x
+    h = oracle.f32_to_bf16(rng.standard_normal((M, F)).astype(np.float32))
+    res = oracle.residual_rmsnorm_quant(h, up, None, 1e-5)
+    ref = oracle.rmsnorm_quant(oracle.glue_residual(h, up), None, 1e-5)
+    assert np.array_equal(res["q"], ref["q"]) and np.array_equal(res["d"], ref["d"])
+    assert np.array_equal(oracle.bf16_to_f32(res["x"]), oracle.bf16_to_f32(oracle.f32_to_bf16((oracle.bf16_to_f32(h) + up).astype(np.float32))))
