@@ -168,6 +168,17 @@ int bitlinear_quant_act(const void* x_bf16, const void* gain, float rms_eps, int
                         int8_t* xq_out, float* d_out, int32_t* xsum_out, void* stream);
 
 /*
+ * The same quantiser with the squared-ReLU gate of the feed-forward block in front (Section 2: ReLU^2 replaces SwiGLU;
+ * the down projection is a BitLinear, so its subln norm and its 8-bit quantiser follow the gate directly).  One launch
+ * computes f = bf16( fl32( fl32(r * r) * up ) ), r = max(gate, 0), and quantises f exactly as bitlinear_quant_act does.
+ *   gate, up   in : [M][F] fp32 (outputs of the gate and up projections).
+ *   x_out_bf16 out: nullable; [M][F] bf16, receives f.
+ *   gain, xq_out, d_out, xsum_out: as in bitlinear_quant_act, with K = F.
+ */
+int bitlinear_quant_act_relu2(const float* gate, const float* up, const void* gain, float rms_eps, int M, int F,
+                              void* x_out_bf16, int8_t* xq_out, float* d_out, int32_t* xsum_out, void* stream);
+
+/*
  * Ternary x int8 contraction over packed weights with the dequantising epilogue
  * (Section 5.1: packed weights are loaded from HBM, unpacked on chip and multiplied with the
  * 8-bit activations; Section 2 fixes the two scales the epilogue undoes).
@@ -236,7 +247,7 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  *              workspace.
  */
 typedef struct bitlinear_problem {
-    const void* x;      /* [M][K] bf16 */
+    const void* x;      /* [M][K] bf16 (another operand where x_op says so) */
     const void* gain;   /* [K] bf16 or NULL */
     const void* packed; /* packed weights of an [N][K] matrix */
     const float* s_w;   /* its scale */
@@ -245,7 +256,28 @@ typedef struct bitlinear_problem {
     int y_dtype;        /* BITLINEAR_F32 or BITLINEAR_BF16 */
     float rms_eps;
     int w_format;       /* layout of `packed`: BITLINEAR_WEIGHTS_2BIT (0) or BITLINEAR_WEIGHTS_DENSE5 (1) */
+    /* The element-wise step of a decoder layer that sits in front of this BitLinear, fused into its quantiser launch
+     * (Section 2: squared-ReLU feed-forward block, residual connections; the subln norm then applies to the result).
+     * Same arithmetic as the bitlinear_glue_* calls below: one fp32 operation per step, one bf16 rounding.
+     *   BITLINEAR_X_PLAIN (0)        x is the input, bf16 [M][K]; x2 and x_out are ignored.
+     *   BITLINEAR_X_RELU2 (1)        x = gate, x2 = up, both fp32 [M][K]:   input = bf16(max(gate,0)^2 * up)
+     *   BITLINEAR_X_RESIDUAL (2)     x = h bf16 [M][K], x2 = y fp32 [M][K]: input = bf16(h + y)
+     *   BITLINEAR_X_ATTN_STANDIN (3) x = q fp32 [M][K], x2 = v fp32 [M][K / x_arg1], x_arg0 = head_dim (a multiple
+     *                                of 8), x_arg1 = query heads per KV head: input = q + v of the matching KV head
+     *                                (a stand-in for attention, which is not a BitLinear)
+     * x_out: nullable bf16 [M][K] that receives the input so formed (the new hidden state after a residual); it must
+     * not alias x.  Problems of a call that name the same x, x2, x_op, gain, rms_eps, M and K share one quantised copy. */
+    int x_op;
+    int x_arg0, x_arg1;
+    int reserved;       /* set to 0 */
+    const void* x2;
+    void* x_out;
 } bitlinear_problem;
+
+#define BITLINEAR_X_PLAIN 0
+#define BITLINEAR_X_RELU2 1
+#define BITLINEAR_X_RESIDUAL 2
+#define BITLINEAR_X_ATTN_STANDIN 3
 
 #define BITLINEAR_BATCH_REUSE_PLAN 1 /* descriptors unchanged since the previous call on this workspace */
 #define BITLINEAR_BATCH_REUSE_ACT 2  /* inputs x unchanged too: skip the quantiser launch, reuse its results in ws */

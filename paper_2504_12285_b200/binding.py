@@ -39,6 +39,8 @@ _SIGNATURES = {
     "bitlinear_forward_batch_acc": (_c_int, [_c_void_p, _c_int, _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_quant_act": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_int, _c_int, _c_void_p, _c_void_p,
                                      _c_void_p, _c_void_p]),
+    "bitlinear_quant_act_relu2": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_float, _c_int, _c_int, _c_void_p, _c_void_p,
+                                           _c_void_p, _c_void_p, _c_void_p]),
     "bitlinear_matmul_q": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
                                     _c_void_p, _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_forward": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int, _c_int,
@@ -63,6 +65,7 @@ _SIGNATURES = {
 }
 
 WEIGHTS_2BIT, WEIGHTS_DENSE5 = 0, 1
+X_PLAIN, X_RELU2, X_RESIDUAL, X_ATTN_STANDIN = 0, 1, 2, 3
 BATCH_REUSE_PLAN = 1
 BATCH_REUSE_ACT = 2
 
@@ -71,7 +74,8 @@ class Problem(ctypes.Structure):
     """Mirror of the C struct bitlinear_problem."""
     _fields_ = [("x", _c_void_p), ("gain", _c_void_p), ("packed", _c_void_p), ("s_w", _c_void_p), ("y", _c_void_p),
                 ("M", _c_int), ("N", _c_int), ("K", _c_int), ("y_dtype", _c_int), ("rms_eps", _c_float),
-                ("w_format", _c_int)]
+                ("w_format", _c_int), ("x_op", _c_int), ("x_arg0", _c_int), ("x_arg1", _c_int), ("reserved", _c_int),
+                ("x2", _c_void_p), ("x_out", _c_void_p)]
 
 
 class BitLinearError(RuntimeError):
@@ -219,6 +223,24 @@ def bitlinear_quant_act(x: torch.Tensor, gain: torch.Tensor | None, rms_eps: flo
     rc = lib().bitlinear_quant_act(_ptr(x), _ptr(gain), rms_eps, M, K, _ptr(xq), _ptr(d), _ptr(xsum), _stream())
     _check(rc, "bitlinear_quant_act")
     return xq, d, xsum
+
+
+def bitlinear_quant_act_relu2(gate: torch.Tensor, up: torch.Tensor, gain: torch.Tensor | None, rms_eps: float = 1e-5,
+                              want_x: bool = False):
+    """gate, up [M, F] fp32 -> (xq int8 [M, F], d fp32 [M], xsum int32 [M][, f bf16 [M, F]]): squared-ReLU gate fused
+    with the down projection's RMSNorm + int8 quantiser."""
+    _dev(gate, torch.float32, "gate"), _dev(up, torch.float32, "up")
+    if gain is not None:
+        _dev(gain, torch.bfloat16, "gain")
+    M, F = gate.shape
+    xq = torch.empty(M, F, dtype=torch.int8, device=gate.device)
+    d = torch.empty(max(M, 1), dtype=torch.float32, device=gate.device)[:M]
+    xsum = torch.empty(max(M, 1), dtype=torch.int32, device=gate.device)[:M]
+    f = torch.empty(M, F, dtype=torch.bfloat16, device=gate.device) if want_x else None
+    rc = lib().bitlinear_quant_act_relu2(_ptr(gate), _ptr(up), _ptr(gain), rms_eps, M, F, _ptr(f), _ptr(xq), _ptr(d),
+                                         _ptr(xsum), _stream())
+    _check(rc, "bitlinear_quant_act_relu2")
+    return (xq, d, xsum, f) if want_x else (xq, d, xsum)
 
 
 def bitlinear_matmul_q(xq, d, xsum, packed, s_w, N: int, y_dtype=torch.float32, want_acc: bool = False,
@@ -373,12 +395,17 @@ class ProblemBatch:
     """A host array of bitlinear_problem descriptors plus the tensors they point to (kept alive)."""
 
     def __init__(self, items, rms_eps: float = 1e-5, w_format: int = WEIGHTS_2BIT):
-        """items: iterable of (x [M,K] bf16, gain [K] bf16 or None, packed uint8, s_w fp32 [1], y [M,N]);
+        """items: iterable of (x [M,K] bf16, gain [K] bf16 or None, packed uint8, s_w fp32 [1], y [M,N]) with an
+        optional sixth entry (x_op, x2, x_out, x_arg0, x_arg1): the element-wise step fused into the quantiser (X_RELU2:
+        x = gate fp32, x2 = up fp32; X_RESIDUAL: x = h bf16, x2 = y fp32; X_ATTN_STANDIN: x = q fp32, x2 = v fp32,
+        x_arg0 = head_dim, x_arg1 = query heads per KV head; x_out = bf16 [M,K] or None);
         w_format: the layout of every packed matrix of the batch (WEIGHTS_2BIT or WEIGHTS_DENSE5)."""
-        self.tensors = [tuple(it) for it in items]
+        self.tensors = [tuple(it[:5]) for it in items]
+        self.steps = [it[5] if len(it) > 5 else None for it in items]  # kept alive with the batch
         self.array = (Problem * max(len(self.tensors), 1))()
         for i, (x, gain, packed, s_w, y) in enumerate(self.tensors):
-            _dev(x, torch.bfloat16, "x")
+            step = self.steps[i]
+            _dev(x, torch.bfloat16 if step is None or step[0] == X_RESIDUAL else torch.float32, "x")
             if gain is not None:
                 _dev(gain, torch.bfloat16, "gain")
             _dev(packed, torch.uint8, "packed")
@@ -388,8 +415,13 @@ class ProblemBatch:
             M, K = x.shape
             if y.shape[0] != M:
                 raise ValueError("x and y disagree on M")
+            op, x2, x_out, arg0, arg1 = (X_PLAIN, None, None, 0, 0) if step is None else step
+            if x2 is not None:
+                _dev(x2, torch.float32, "x2")
+            if x_out is not None:
+                _dev(x_out, torch.bfloat16, "x_out")
             self.array[i] = Problem(_ptr(x), _ptr(gain), _ptr(packed), _ptr(s_w), _ptr(y), M, y.shape[1], K,
-                                    _ydt(y.dtype), rms_eps, w_format)
+                                    _ydt(y.dtype), rms_eps, w_format, op, arg0, arg1, 0, _ptr(x2), _ptr(x_out))
         self.count = len(self.tensors)
 
     def workspace_bytes(self) -> int:

@@ -1,8 +1,9 @@
 """Chained decode over a stack of decoder layers: argument marshalling for the benchmark's 30-layer configuration.
 
 Every step runs in the library's kernels: per layer four batched BitLinear calls (q/k/v, o, gate/up, down - the
-problems of a call share their input and are independent of each other) and four element-wise glue launches
-(attention stand-in, residual, squared-ReLU gate, residual).  This module only owns the buffers and the call order.
+problems of a call share their input and are independent of each other), each with the element-wise step in front of
+it (residual, attention stand-in, residual, squared-ReLU gate) fused into its quantiser launch.  This module only owns
+the buffers and the call order.
 """
 from __future__ import annotations
 
@@ -19,22 +20,33 @@ class DecodeChain:
         self.M, self.dims = M, (n_q_heads, n_kv_heads, head_dim)
         kv = n_kv_heads * head_dim
         f32 = dict(dtype=torch.float32, device=dev)
-        self.h = torch.zeros(M, hidden, dtype=torch.bfloat16, device=dev)
+        bf = dict(dtype=torch.bfloat16, device=dev)
+        # the hidden state alternates between two buffers: a fused residual step reads one and writes the other
+        self.h_in, self.h_mid = torch.zeros(M, hidden, **bf), torch.zeros(M, hidden, **bf)
         self.q, self.k, self.v = torch.empty(M, hidden, **f32), torch.empty(M, kv, **f32), torch.empty(M, kv, **f32)
-        self.a = torch.empty(M, hidden, dtype=torch.bfloat16, device=dev)
         self.o = torch.empty(M, hidden, **f32)
         self.g, self.u = torch.empty(M, ffn, **f32), torch.empty(M, ffn, **f32)
-        self.f = torch.empty(M, ffn, dtype=torch.bfloat16, device=dev)
         self.dn = torch.empty(M, hidden, **f32)
+        group = n_q_heads // n_kv_heads
         self.calls = []  # per layer: four (ProblemBatch, workspace)
-        for layer in layers:
-            def item(name, x, y):
+        for li, layer in enumerate(layers):
+            def item(name, x, y, step=None):
                 packed, s_w, gain = layer[name]
-                return (x, gain, packed, s_w, y)
-            groups = [[item("q", self.h, self.q), item("k", self.h, self.k), item("v", self.h, self.v)],
-                      [item("o", self.a, self.o)],
-                      [item("gate", self.h, self.g), item("up", self.h, self.u)],
-                      [item("down", self.f, self.dn)]]
+                return (x, gain, packed, s_w, y) if step is None else (x, gain, packed, s_w, y, step)
+            # the element-wise step in front of each level is fused into that level's quantiser launch:
+            #   q,k,v : h = h_mid(previous layer) + down output  (plain input in the first layer)
+            #   o     : attention stand-in on q and v
+            #   gate,up: h_mid = h + o output
+            #   down  : squared-ReLU gate
+            res_in = None if li == 0 else (bl.X_RESIDUAL, self.dn, self.h_in, 0, 0)
+            x_qkv = self.h_in if li == 0 else self.h_mid
+            standin = (bl.X_ATTN_STANDIN, self.v, None, head_dim, group)
+            res_mid = (bl.X_RESIDUAL, self.o, self.h_mid, 0, 0)
+            relu2 = (bl.X_RELU2, self.u, None, 0, 0)
+            groups = [[item("q", x_qkv, self.q, res_in), item("k", x_qkv, self.k, res_in), item("v", x_qkv, self.v, res_in)],
+                      [item("o", self.q, self.o, standin)],
+                      [item("gate", self.h_in, self.g, res_mid), item("up", self.h_in, self.u, res_mid)],
+                      [item("down", self.g, self.dn, relu2)]]
             per_layer = []
             for grp in groups:
                 batch = bl.ProblemBatch(grp, rms_eps)
@@ -42,25 +54,19 @@ class DecodeChain:
                 bl.bitlinear_forward_batch(batch, ws)  # uploads the plan; results are overwritten by step()
                 per_layer.append((batch, ws))
             self.calls.append(per_layer)
+        self.h = self.h_mid  # where the hidden state is after step()
         torch.cuda.synchronize(dev)
 
-    launches_per_layer = 12  # 4 x (quantiser + weight stream) + 4 glue kernels
+    launches_per_layer = 8  # 4 x (quantiser with its fused element-wise step + weight stream)
 
     def step(self, h0: torch.Tensor | None = None) -> torch.Tensor:
         """One pass over all layers, starting from h0 (bf16 [M, hidden]) or from the current hidden state."""
-        if h0 is not None:
-            self.h.copy_(h0)
-        nq, nkv, hd = self.dims
+        self.h_in.copy_(self.h_mid if h0 is None else h0)
         for qkv, o, gu, down in self.calls:
-            bl.bitlinear_forward_batch(qkv[0], qkv[1], reuse_plan=True)
-            bl.bitlinear_glue_attn_standin(self.q, self.v, self.a, nq, nkv, hd)
-            bl.bitlinear_forward_batch(o[0], o[1], reuse_plan=True)
-            bl.bitlinear_glue_residual_add(self.h, self.o)
-            bl.bitlinear_forward_batch(gu[0], gu[1], reuse_plan=True)
-            bl.bitlinear_glue_relu2_mul(self.g, self.u, self.f)
-            bl.bitlinear_forward_batch(down[0], down[1], reuse_plan=True)
-            bl.bitlinear_glue_residual_add(self.h, self.dn)
-        return self.h
+            for batch, ws in (qkv, o, gu, down):
+                bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
+        bl.bitlinear_glue_residual_add(self.h_mid, self.dn)  # the last layer's residual
+        return self.h_mid
 
 
 class PersistentChain:

@@ -217,6 +217,20 @@ int bitlinear_quant_act(const void* x_bf16, const void* gain, float rms_eps, int
                                         xsum_out, static_cast<cudaStream_t>(stream)));
 }
 
+int bitlinear_quant_act_relu2(const float* gate, const float* up, const void* gain, float rms_eps, int M, int F,
+                              void* x_out_bf16, int8_t* xq_out, float* d_out, int32_t* xsum_out, void* stream) {
+    if (M < 0 || !shape_ok(kTileRows, F)) return BITLINEAR_ERR_SHAPE;
+    if (M == 0) return BITLINEAR_OK;
+    if (!gate || !up || !xq_out || !d_out) return BITLINEAR_ERR_NULL;
+    if (!aligned16(gate) || !aligned16(up) || !aligned16(xq_out) || (gain && !aligned16(gain)) ||
+        (x_out_bf16 && !aligned16(x_out_bf16)) || (reinterpret_cast<uintptr_t>(d_out) & 3u) ||
+        (reinterpret_cast<uintptr_t>(xsum_out) & 3u))
+        return BITLINEAR_ERR_ALIGN;
+    if (int rc = check_arch()) return rc;
+    return cuda_status(launch_quant_act_step(BITLINEAR_X_RELU2, gate, up, x_out_bf16, 0, 0, static_cast<const __nv_bfloat16*>(gain),
+                                             rms_eps, M, F, xq_out, d_out, xsum_out, static_cast<cudaStream_t>(stream)));
+}
+
 int bitlinear_matmul_q(const int8_t* xq, const float* d, const int32_t* xsum, const void* packed, const float* s_w,
                        int M, int N, int K, void* y_out, int y_dtype, int32_t* acc_out, int path, void* ws,
                        size_t ws_bytes, void* stream) {

@@ -47,6 +47,11 @@ cudaError_t launch_unpack5_i8(const uint8_t* packed, int N, int K, int8_t* wq, c
 cudaError_t launch_quant_act(const __nv_bfloat16* x, const __nv_bfloat16* gain, float eps, int M, int K,
                              int8_t* xq, float* d, int32_t* xsum, cudaStream_t st);
 
+// The same with an element-wise step in front (x_op = BITLINEAR_X_*, operands as in bitlinear_problem).
+cudaError_t launch_quant_act_step(int x_op, const void* x, const void* x2, void* x_out, int arg0, int arg1,
+                                  const __nv_bfloat16* gain, float eps, int M, int K, int8_t* xq, float* d, int32_t* xsum,
+                                  cudaStream_t st);
+
 cudaError_t launch_gemv(const int8_t* xq, const float* d, const int32_t* xsum, const uint32_t* packed,
                         const float* s_w, int M, int N, int K, void* y, int y_dtype, int32_t* acc_out,
                         cudaStream_t st);

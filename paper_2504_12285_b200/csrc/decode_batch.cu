@@ -20,6 +20,8 @@
 //             Unpack: word & (0x03030303 << 2j) is 4^j x the codes of four consecutive columns, fed
 //             to a dot-product-of-four with the int8 activations; one accumulator per j keeps the
 //             scale uniform and the four are folded once per row block.
+#include <map>
+#include <tuple>
 #include <type_traits>
 #include <vector>
 
@@ -32,8 +34,11 @@ struct DevProblem {
     const uint8_t* packed;
     const float* s_w;
     void* y;
-    const __nv_bfloat16* x;
+    const void* x;     // first operand of the problem's input step, all M rows of the ORIGINAL problem (see RowOp)
     const __nv_bfloat16* gain;
+    RowOp op;          // the element-wise step in front of the quantiser
+    int x_row0;        // row of x (and of the step's other operands) that token 0 of this entry is
+    int pad0;
     int8_t* xq;
     float* d;
     int32_t* xsum;
@@ -91,7 +96,9 @@ __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHe
     const DevProblem& p = probs[row_prob[row]];
     const int m = row - p.row_begin;
     int8_t* xq_row = p.xq + (size_t)m * p.x_stride;
-    quant_row<VPT, LAYOUT>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, xq_row, p.d + m, p.xsum + m, sm);
+    with_row_source(p.op, p.x, p.x_row0 + m, p.K, [&](auto src) {
+        quant_row_src<VPT, LAYOUT>(src, p.gain, p.eps, p.K, xq_row, p.d + m, p.xsum + m, sm);
+    });
     if (LAYOUT == 0)
         for (int k = p.K + 4 * threadIdx.x; k < p.x_stride; k += 4 * kQuantThreads) *reinterpret_cast<uint32_t*>(xq_row + k) = 0u;
 }
@@ -529,6 +536,17 @@ constexpr int kDp4aMaxTokens = 1;
 
 namespace {
 
+// What identifies the quantised input of a plan entry: entries with equal keys share one quantised copy.
+struct QuantKey {
+    const void *x, *x2, *gain, *x_out;
+    int M, K, op, arg0, arg1, row0;
+    float eps;
+    bool operator<(const QuantKey& o) const {
+        return std::tie(x, x2, gain, x_out, M, K, op, arg0, arg1, row0, eps) <
+               std::tie(o.x, o.x2, o.gain, o.x_out, o.M, o.K, o.op, o.arg0, o.arg1, o.row0, o.eps);
+    }
+};
+
 // Bytes between the quantised rows of two tokens of a problem: K, or K padded to whole 320-column tiles (dense layout).
 inline int x_stride_of(const bitlinear_problem& q) {
     return q.w_format == BITLINEAR_WEIGHTS_DENSE5 ? dense_k_tiles(q.K) * kDenseTileCols : q.K;
@@ -594,6 +612,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     // ---- host plan: device descriptors, token -> problem table, byte-balanced CTA ranges ----
     std::vector<DevProblem> dp;
     std::vector<int> row_prob;
+    std::map<QuantKey, int> quantised;  // first entry of dp that quantises a given input
     dp.reserve(count);
     row_prob.reserve(rows + 1);
     int total_rb = 0;
@@ -615,8 +634,30 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
                 v.packed = static_cast<const uint8_t*>(q.packed);
                 v.s_w = q.s_w;
                 v.y = static_cast<char*>(q.y) + (size_t)part * y_row;
-                v.x = static_cast<const __nv_bfloat16*>(q.x) + (size_t)part * q.K;
+                v.x = q.x;
+                v.x_row0 = part;
+                v.pad0 = 0;
+                v.op.x2 = q.x2; v.op.x_out = q.x_out; v.op.op = q.x_op; v.op.arg0 = q.x_arg0; v.op.arg1 = q.x_arg1; v.op.pad = 0;
                 v.gain = static_cast<const __nv_bfloat16*>(q.gain);
+                // entries that read the same rows through the same step with the same norm share one quantised copy
+                const QuantKey key{q.x, q.x2, q.gain, q.x_out, q.M, q.K, q.x_op, q.x_arg0, q.x_arg1, part, q.rms_eps};
+                const auto seen = quantised.find(key);
+                if (seen != quantised.end()) {
+                    const DevProblem& first = dp[seen->second];
+                    v.xq = first.xq; v.d = first.d; v.xsum = first.xsum;
+                    v.acc_out = (acc_outs && acc_outs[i]) ? acc_outs[i] + (size_t)part * q.N : nullptr;
+                    v.M = m_each; v.N = q.N; v.K = q.K; v.y_dtype = q.y_dtype;
+                    v.eps = q.rms_eps;
+                    v.k_tiles = dense ? dense_k_tiles(q.K) : q.K / kTileCols;
+                    v.x_stride = stride;
+                    v.rb_begin = total_rb;
+                    v.rb_end = total_rb + q.N / kTileRows;
+                    v.row_begin = first.row_begin;
+                    dp.push_back(v);
+                    total_rb = v.rb_end;
+                    continue;
+                }
+                quantised.emplace(key, (int)dp.size());
                 v.xq = reinterpret_cast<int8_t*>(xq_ptr) + (size_t)part * stride;
                 v.d = d_ptr + row;
                 v.xsum = xs_ptr + row;
@@ -635,6 +676,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
             }
             xq_ptr += align_up((size_t)q.M * stride, 16);
         }
+        rows = (size_t)row;  // tokens actually quantised (shared copies counted once)
         row_prob.push_back(0);
     }
     const int n_prob = (int)dp.size();
@@ -743,6 +785,24 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
 
 using namespace bitlinear;
 
+namespace {
+
+// The element-wise step in front of a problem's quantiser (x_op and its operands), checked on the host.
+int check_input_step(const bitlinear_problem& q) {
+    if (q.x_op < BITLINEAR_X_PLAIN || q.x_op > BITLINEAR_X_ATTN_STANDIN) return BITLINEAR_ERR_DTYPE;
+    if (q.x_op == BITLINEAR_X_PLAIN || q.M == 0) return BITLINEAR_OK;
+    if (!q.x2) return BITLINEAR_ERR_NULL;
+    if (!aligned16(q.x2) || (q.x_out && !aligned16(q.x_out))) return BITLINEAR_ERR_ALIGN;
+    if (q.x_out == q.x) return BITLINEAR_ERR_SHAPE;  // rows are read more than once: the result cannot replace them
+    if (q.x_op == BITLINEAR_X_ATTN_STANDIN) {
+        if (q.x_arg0 <= 0 || q.x_arg0 % 8 || q.x_arg1 <= 0 || q.K % q.x_arg0 || (q.K / q.x_arg0) % q.x_arg1) return BITLINEAR_ERR_SHAPE;
+        if (((size_t)(q.K / q.x_arg1) * sizeof(float)) % 16) return BITLINEAR_ERR_ALIGN;  // rows of v stay 16-byte aligned
+    }
+    return BITLINEAR_OK;
+}
+
+}  // namespace
+
 extern "C" {
 
 size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
@@ -786,6 +846,7 @@ int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, in
         if (q.y_dtype != BITLINEAR_F32 && q.y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
         if (q.w_format != BITLINEAR_WEIGHTS_2BIT && q.w_format != BITLINEAR_WEIGHTS_DENSE5) return BITLINEAR_ERR_DTYPE;
         if (q.M < 0 || !shape_ok(q.N, q.K)) return BITLINEAR_ERR_SHAPE;
+        if (const int rc = check_input_step(q)) return rc;
         if (q.M <= kGemvMaxTokens) {
             if (q.K > kBatchMaxK) return BITLINEAR_ERR_SHAPE;
             dec.push_back(q);

@@ -62,8 +62,9 @@ struct MmaProblem {
     const float* d;
     const int32_t* xsum;
     void* y;
-    const __nv_bfloat16* x;
+    const void* x;   // first operand of the input step (see RowOp)
     const __nv_bfloat16* gain;
+    RowOp op;        // the element-wise step in front of the quantiser
     int8_t* xq_out;  // = x_img, for the quantiser launch
     float* d_out;
     int32_t* xsum_out;
@@ -189,8 +190,10 @@ __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeade
     if (row >= rows) return;  // the whole group leaves: nobody is left waiting at its barrier
     const MmaProblem& p = probs[row_prob[row]];
     const int m = row - p.row_begin;
-    quant_row_group<3, kQuantGroupWarps>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m,
-                                         p.xsum_out + m, sm[group], 1 + group, m & 7);
+    with_row_source(p.op, p.x, m, p.K, [&](auto src) {
+        quant_row_group_src<3, kQuantGroupWarps>(src, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m,
+                                                 p.xsum_out + m, sm[group], 1 + group, m & 7);
+    });
 }
 
 // 2 x 16 packed bytes (128 codes of one weight row) -> 32 tensor-memory columns of 64 x code.
@@ -524,7 +527,8 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
             v.d = d_ptr + row;
             v.xsum = xs_ptr + row;
             v.y = q.y;
-            v.x = static_cast<const __nv_bfloat16*>(q.x);
+            v.x = q.x;
+            v.op.x2 = q.x2; v.op.x_out = q.x_out; v.op.op = q.x_op; v.op.arg0 = q.x_arg0; v.op.arg1 = q.x_arg1; v.op.pad = 0;
             v.gain = static_cast<const __nv_bfloat16*>(q.gain);
             v.xq_out = reinterpret_cast<int8_t*>(x_ptr);
             v.d_out = d_ptr + row;

@@ -24,7 +24,8 @@ namespace bitlinear {
 namespace {
 
 struct PrefillItem {
-    const __nv_bfloat16* x;
+    const void* x;  // first operand of the input step (see RowOp)
+    RowOp op;       // the element-wise step in front of the quantiser
     const __nv_bfloat16* gain;
     const uint32_t* packed;
     uint8_t* a_tiles;
@@ -52,8 +53,9 @@ __global__ void __launch_bounds__(kQuantThreads) group_quant_warp_kernel(const P
     const PrefillItem& p = items[i];
     const int m = row - p.row_begin;
     uint8_t* dst = p.a_tiles + (size_t)(m >> 7) * (p.K >> 7) * (128 * 128) + (size_t)(m & 127) * 128;
-    quant_row_warp<2>(p.x + (size_t)m * p.K, p.gain, p.eps, p.K, reinterpret_cast<int8_t*>(dst), p.d + m, p.xsum + m,
-                      m & 7);
+    with_row_source(p.op, p.x, m, p.K, [&](auto src) {
+        quant_row_warp_src<2>(src, p.gain, p.eps, p.K, reinterpret_cast<int8_t*>(dst), p.d + m, p.xsum + m, m & 7);
+    });
 }
 
 // Expansion of the packed weights into tile images: one thread per packed word (16 codes -> its 16-byte piece of a
@@ -164,7 +166,8 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
         for (int i = 0; i < n; ++i) {
             const bitlinear_problem& q = problems[idx[i]];
             PrefillItem& it = items[i];
-            it.x = static_cast<const __nv_bfloat16*>(q.x);
+            it.x = q.x;
+            it.op.x2 = q.x2; it.op.x_out = q.x_out; it.op.op = q.x_op; it.op.arg0 = q.x_arg0; it.op.arg1 = q.x_arg1; it.op.pad = 0;
             it.gain = static_cast<const __nv_bfloat16*>(q.gain);
             it.packed = static_cast<const uint32_t*>(q.packed);
             it.a_tiles = reinterpret_cast<uint8_t*>(base + L.a_off[i]);
@@ -182,7 +185,9 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             int same = -1;
             for (int j = 0; j < i && same < 0; ++j) {
                 const bitlinear_problem& o = problems[idx[j]];
-                if (o.x == q.x && o.gain == q.gain && o.rms_eps == q.rms_eps && o.M == q.M && o.K == q.K) same = j;
+                if (o.x == q.x && o.x2 == q.x2 && o.x_op == q.x_op && o.x_out == q.x_out && o.x_arg0 == q.x_arg0 &&
+                    o.x_arg1 == q.x_arg1 && o.gain == q.gain && o.rms_eps == q.rms_eps && o.M == q.M && o.K == q.K)
+                    same = j;
             }
             if (same >= 0) {
                 it.a_tiles = items[same].a_tiles; it.d = items[same].d; it.xsum = items[same].xsum;

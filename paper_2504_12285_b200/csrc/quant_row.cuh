@@ -60,6 +60,118 @@ __device__ __forceinline__ double sum_squares8(const float (&f)[8]) {
     return (double)hi + (double)lo;
 }
 
+// ---- where a row comes from -------------------------------------------------------------------------------------
+// The quantisers read their input through a source object: load(v) returns 16-byte vector v of the row as eight bf16
+// bit patterns, store(v, bits) is called once per vector for sources that also have to write the row they produce.
+// Besides a plain bf16 row, a source can apply the element-wise step that sits in front of a BitLinear in a decoder
+// layer (paper Section 2: squared-ReLU feed-forward block, residual connections), so that the step costs no launch of
+// its own: one fp32 operation per arithmetic step, then one round-to-nearest-even cast to bf16, exactly as the
+// stand-alone glue kernels do.
+__device__ __forceinline__ uint32_t bf16x2_rn(float lo, float hi) {
+    const __nv_bfloat162 pk = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&pk);
+}
+
+struct RowBf16 {
+    const uint4* x;
+    __device__ __forceinline__ uint4 load(int v) const { return x[v]; }
+    __device__ __forceinline__ void store(int, const uint4&) const {}
+};
+
+// x = bf16( fl32( fl32(r * r) * up ) ), r = max(gate, 0)
+struct RowRelu2 {
+    const float4* gate;
+    const float4* up;
+    uint4* out;  // nullable
+    __device__ __forceinline__ uint4 load(int v) const {
+        const float4 g0 = gate[2 * v], g1 = gate[2 * v + 1], u0 = up[2 * v], u1 = up[2 * v + 1];
+        const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+        const float u[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+        float f[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float r = fmaxf(g[e], 0.0f);
+            f[e] = __fmul_rn(__fmul_rn(r, r), u[e]);
+        }
+        return make_uint4(bf16x2_rn(f[0], f[1]), bf16x2_rn(f[2], f[3]), bf16x2_rn(f[4], f[5]), bf16x2_rn(f[6], f[7]));
+    }
+    __device__ __forceinline__ void store(int v, const uint4& b) const {
+        if (out != nullptr) out[v] = b;
+    }
+};
+
+// x = bf16( fl32( float(h) + y ) ); the new hidden state goes to `out` (which must not be `h`: some quantisers read a
+// row three times)
+struct RowResidual {
+    const uint4* h;
+    const float4* y;
+    uint4* out;
+    __device__ __forceinline__ uint4 load(int v) const {
+        const uint4 hb = h[v];
+        const float4 y0 = y[2 * v], y1 = y[2 * v + 1];
+        const uint32_t w[4] = {hb.x, hb.y, hb.z, hb.w};
+        const float yy[8] = {y0.x, y0.y, y0.z, y0.w, y1.x, y1.y, y1.z, y1.w};
+        uint32_t r[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            r[e] = bf16x2_rn(__fadd_rn(__uint_as_float(w[e] << 16), yy[2 * e]),
+                             __fadd_rn(__uint_as_float(w[e] & 0xffff0000u), yy[2 * e + 1]));
+        return make_uint4(r[0], r[1], r[2], r[3]);
+    }
+    __device__ __forceinline__ void store(int v, const uint4& b) const {
+        if (out != nullptr) out[v] = b;
+    }
+};
+
+// Stand-in for attention (not a BitLinear): x[h * D + j] = bf16( fl32( q[h * D + j] + v[(h / group) * D + j] ) );
+// D a multiple of 8, so the eight elements of a vector lie inside one head.
+struct RowStandin {
+    const float* q;
+    const float* v;
+    uint4* out;  // nullable
+    int head_dim, group;
+    __device__ __forceinline__ uint4 load(int vec) const {
+        const int c = 8 * vec, head = c / head_dim, j = c - head * head_dim;
+        const float4* qp = reinterpret_cast<const float4*>(q + c);
+        const float4* vp = reinterpret_cast<const float4*>(v + (head / group) * head_dim + j);
+        const float4 q0 = qp[0], q1 = qp[1], v0 = vp[0], v1 = vp[1];
+        return make_uint4(bf16x2_rn(__fadd_rn(q0.x, v0.x), __fadd_rn(q0.y, v0.y)), bf16x2_rn(__fadd_rn(q0.z, v0.z), __fadd_rn(q0.w, v0.w)),
+                          bf16x2_rn(__fadd_rn(q1.x, v1.x), __fadd_rn(q1.y, v1.y)), bf16x2_rn(__fadd_rn(q1.z, v1.z), __fadd_rn(q1.w, v1.w)));
+    }
+    __device__ __forceinline__ void store(int vec, const uint4& b) const {
+        if (out != nullptr) out[vec] = b;
+    }
+};
+
+// The element-wise step in front of a problem's quantiser, as the batch descriptors carry it.
+struct RowOp {
+    const void* x2;  // second operand (up / y / v), fp32
+    void* x_out;     // bf16 [M][K] result of the step, nullable except for the residual step
+    int op;          // BITLINEAR_X_*
+    int arg0, arg1;  // attention stand-in: head_dim, query heads per KV head
+    int pad;
+};
+
+// Calls f(source) with the source of row m of a problem whose first operand is x ([M][K]; bf16 or fp32 as the step says).
+template <class F>
+__device__ __forceinline__ void with_row_source(const RowOp& o, const void* x, int m, int K, F&& f) {
+    const size_t off = (size_t)m * K;
+    if (o.op == BITLINEAR_X_RELU2) {
+        f(RowRelu2{reinterpret_cast<const float4*>(static_cast<const float*>(x) + off),
+                   reinterpret_cast<const float4*>(static_cast<const float*>(o.x2) + off),
+                   o.x_out ? reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(o.x_out) + off) : nullptr});
+    } else if (o.op == BITLINEAR_X_RESIDUAL) {
+        f(RowResidual{reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(x) + off),
+                      reinterpret_cast<const float4*>(static_cast<const float*>(o.x2) + off),
+                      o.x_out ? reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(o.x_out) + off) : nullptr});
+    } else if (o.op == BITLINEAR_X_ATTN_STANDIN) {
+        f(RowStandin{static_cast<const float*>(x) + off, static_cast<const float*>(o.x2) + (size_t)m * (K / o.arg1),
+                     o.x_out ? reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(o.x_out) + off) : nullptr, o.arg0, o.arg1});
+    } else {
+        f(RowBf16{reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(x) + off)});
+    }
+}
+
 // Quantises one row with the kQuantThreads threads of the calling CTA (all must call it).
 // LAYOUT 0: codes are stored in column order.
 // LAYOUT 1: inside every block of 256 columns the sixteen 16-byte pieces are stored transposed (piece 4t+q,
@@ -70,21 +182,23 @@ __device__ __forceinline__ double sum_squares8(const float (&f)[8]) {
 //           swz = row & 7 - the 128-byte shared-memory swizzle.
 // LAYOUT 3: the same with tiles of 16 rows x 128 columns (2 KiB): the token-side operand of the decode kernel that
 //           runs on the tensor cores with the tokens as the narrow dimension.
-template <int VPT, int LAYOUT = 0>  // VPT = 16-byte vectors (8 bf16) per thread
-__device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_row,
-                                          const __nv_bfloat16* __restrict__ gain, float eps, int K,
-                                          int8_t* __restrict__ xq_row, float* __restrict__ d_out,
-                                          int32_t* __restrict__ xsum_out, RowReduceSmem& sm, int swz = 0) {
+template <int VPT, int LAYOUT = 0, class Src = RowBf16>  // VPT = 16-byte vectors (8 bf16) per thread
+__device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                              int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                              int32_t* __restrict__ xsum_out, RowReduceSmem& sm, int swz = 0) {
     const int n_vec = K >> 3;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const uint4* xrow = reinterpret_cast<const uint4*>(x_row);
     const uint4* grow = reinterpret_cast<const uint4*>(gain);
 
     uint4 xv[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
         const int v = tid + i * kQuantThreads;
-        xv[i] = (v < n_vec) ? xrow[v] : make_uint4(0, 0, 0, 0);
+        xv[i] = make_uint4(0, 0, 0, 0);
+        if (v < n_vec) {
+            xv[i] = src.load(v);
+            src.store(v, xv[i]);
+        }
     }
 
     // ---- sum of squares in fp64 (each square of a bf16 value is exact) ----
@@ -173,23 +287,30 @@ __device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_ro
 }
 
 
+template <int VPT, int LAYOUT = 0>
+__device__ __forceinline__ void quant_row(const __nv_bfloat16* __restrict__ x_row,
+                                          const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                          int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                          int32_t* __restrict__ xsum_out, RowReduceSmem& sm, int swz = 0) {
+    quant_row_src<VPT, LAYOUT>(RowBf16{reinterpret_cast<const uint4*>(x_row)}, gain, eps, K, xq_row, d_out, xsum_out, sm, swz);
+}
+
 // Warp-per-row variant for many-token calls: the same arithmetic with one warp owning a whole row (16-byte
 // vector v of the row belongs to lane v % 32), so a CTA of kQuantThreads threads quantises eight rows with no
 // block-wide barrier.  The row is read from HBM once; the second and third pass read it again (it is still in
 // L1 / L2), which keeps the register count low and no shared memory is needed, so many rows are in flight per SM.
-template <int LAYOUT = 0>
-__device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__ x_row,
-                                               const __nv_bfloat16* __restrict__ gain, float eps, int K,
-                                               int8_t* __restrict__ xq_row, float* __restrict__ d_out,
-                                               int32_t* __restrict__ xsum_out, int swz = 0) {
+template <int LAYOUT = 0, class Src = RowBf16>
+__device__ __forceinline__ void quant_row_warp_src(const Src src, const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                                   int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                                   int32_t* __restrict__ xsum_out, int swz = 0) {
     const int n_vec = K >> 3;
     const int lane = threadIdx.x & 31;
-    const uint4* xrow = reinterpret_cast<const uint4*>(x_row);
     const uint4* grow = reinterpret_cast<const uint4*>(gain);
     double sq = 0.0;
 #pragma unroll 4
     for (int v = lane; v < n_vec; v += 32) {
-        const uint4 u = xrow[v];
+        const uint4 u = src.load(v);
+        src.store(v, u);
         float f[8];
         unpack_bf16x8(u, f);
         sq += sum_squares8(f);
@@ -204,7 +325,7 @@ __device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__
 #pragma unroll 2
     for (int v = lane; v < n_vec; v += 32) {
         float f[8], g[8];
-        unpack_bf16x8(xrow[v], f);
+        unpack_bf16x8(src.load(v), f);
         if (gain != nullptr) {
             unpack_bf16x8(grow[v], g);
         } else {
@@ -224,7 +345,7 @@ __device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__
 #pragma unroll 2
     for (int v = lane; v < n_vec; v += 32) {
         float f[8], g[8];
-        unpack_bf16x8(xrow[v], f);
+        unpack_bf16x8(src.load(v), f);
         if (gain != nullptr) {
             unpack_bf16x8(grow[v], g);
         } else {
@@ -254,6 +375,14 @@ __device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__
     }
 }
 
+template <int LAYOUT = 0>
+__device__ __forceinline__ void quant_row_warp(const __nv_bfloat16* __restrict__ x_row,
+                                               const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                               int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                               int32_t* __restrict__ xsum_out, int swz = 0) {
+    quant_row_warp_src<LAYOUT>(RowBf16{reinterpret_cast<const uint4*>(x_row)}, gain, eps, K, xq_row, d_out, xsum_out, swz);
+}
+
 // WARPS warps per row (WARPS = 2 or 4; the group's threads are 32 * WARPS consecutive threads of the CTA): for calls
 // with few rows, where one warp per row leaves the GPU mostly idle and a long row is a long serial chain for its warp.
 // Same arithmetic and the same three passes as quant_row_warp; the partial results of the warps meet in shared memory
@@ -265,22 +394,22 @@ struct GroupReduceSmem {
     float r;
 };
 
-template <int LAYOUT, int WARPS>
-__device__ __forceinline__ void quant_row_group(const __nv_bfloat16* __restrict__ x_row,
-                                                const __nv_bfloat16* __restrict__ gain, float eps, int K,
-                                                int8_t* __restrict__ xq_row, float* __restrict__ d_out,
-                                                int32_t* __restrict__ xsum_out, GroupReduceSmem& sm, int bar_id, int swz = 0) {
+template <int LAYOUT, int WARPS, class Src = RowBf16>
+__device__ __forceinline__ void quant_row_group_src(const Src src, const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                                    int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                                    int32_t* __restrict__ xsum_out, GroupReduceSmem& sm, int bar_id, int swz = 0) {
     constexpr int T = 32 * WARPS;
     const int n_vec = K >> 3;
     const int gt = threadIdx.x % T, w = gt >> 5, lane = gt & 31;
-    const uint4* xrow = reinterpret_cast<const uint4*>(x_row);
     const uint4* grow = reinterpret_cast<const uint4*>(gain);
     auto group_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "r"(T) : "memory"); };
     double sq = 0.0;
 #pragma unroll 4
     for (int v = gt; v < n_vec; v += T) {
         float f[8];
-        unpack_bf16x8(xrow[v], f);
+        const uint4 u = src.load(v);
+        src.store(v, u);
+        unpack_bf16x8(u, f);
         sq += sum_squares8(f);
     }
 #pragma unroll
@@ -300,7 +429,7 @@ __device__ __forceinline__ void quant_row_group(const __nv_bfloat16* __restrict_
 #pragma unroll 2
     for (int v = gt; v < n_vec; v += T) {
         float f[8], g[8];
-        unpack_bf16x8(xrow[v], f);
+        unpack_bf16x8(src.load(v), f);
         if (gain != nullptr) {
             unpack_bf16x8(grow[v], g);
         } else {
@@ -324,7 +453,7 @@ __device__ __forceinline__ void quant_row_group(const __nv_bfloat16* __restrict_
 #pragma unroll 2
     for (int v = gt; v < n_vec; v += T) {
         float f[8], g[8];
-        unpack_bf16x8(xrow[v], f);
+        unpack_bf16x8(src.load(v), f);
         if (gain != nullptr) {
             unpack_bf16x8(grow[v], g);
         } else {
@@ -357,6 +486,15 @@ __device__ __forceinline__ void quant_row_group(const __nv_bfloat16* __restrict_
         *d_out = __fdiv_rn(a, 127.0f);
         if (xsum_out != nullptr) *xsum_out = total;
     }
+}
+
+template <int LAYOUT, int WARPS>
+__device__ __forceinline__ void quant_row_group(const __nv_bfloat16* __restrict__ x_row,
+                                                const __nv_bfloat16* __restrict__ gain, float eps, int K,
+                                                int8_t* __restrict__ xq_row, float* __restrict__ d_out,
+                                                int32_t* __restrict__ xsum_out, GroupReduceSmem& sm, int bar_id, int swz = 0) {
+    quant_row_group_src<LAYOUT, WARPS>(RowBf16{reinterpret_cast<const uint4*>(x_row)}, gain, eps, K, xq_row, d_out, xsum_out, sm,
+                                       bar_id, swz);
 }
 
 }  // namespace bitlinear
