@@ -394,6 +394,16 @@ int bitlinear_poll_status(void* stream);
  */
 int bitlinear_selftest_wait_timeout(unsigned limit_us, void* stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): the rate at which this GPU executes the int8 tensor-core
+ * instruction the prefill contraction is made of.  Launches, on every SM, n_mma_per_sm (1 .. 4,000,000)
+ * tcgen05.mma kind::i8 operations of 128 x 256 x 32 on operands that stay in shared memory - no global traffic, no
+ * epilogue - and returns at once; *ops_out (HOST pointer, nullable) receives the integer operations of the launch,
+ * 2 per multiply-accumulate.  Time the launch with events on `stream`: operations / time is the int8 peak the
+ * benchmark reports prefill fractions against.
+ */
+int bitlinear_probe_int8_mma_rate(int n_mma_per_sm, double* ops_out, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

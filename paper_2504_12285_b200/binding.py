@@ -48,6 +48,7 @@ _SIGNATURES = {
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
+    "bitlinear_probe_int8_mma_rate": (_c_int, [_c_int, ctypes.POINTER(ctypes.c_double), _c_void_p]),
     "bitlinear_selftest_wait_timeout": (_c_int, [ctypes.c_uint, _c_void_p]),
     "bitlinear_glue_relu2_mul": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
     "bitlinear_glue_residual_add": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
@@ -472,6 +473,13 @@ def bitlinear_forward_batch_host(batch: ProblemBatch, x_host: torch.Tensor, x_de
 def bitlinear_selftest_wait_timeout(limit_us: int = 1000) -> None:
     """Launch the bounded-wait self-test: a tiny kernel whose wait runs out after limit_us microseconds."""
     _check(lib().bitlinear_selftest_wait_timeout(int(limit_us), _stream()), "bitlinear_selftest_wait_timeout")
+
+
+def bitlinear_probe_int8_mma_rate(n_mma_per_sm: int) -> float:
+    """Launch the int8 tensor-core rate probe on the current stream; returns the integer operations of the launch."""
+    ops = ctypes.c_double(0.0)
+    _check(lib().bitlinear_probe_int8_mma_rate(int(n_mma_per_sm), ctypes.byref(ops), _stream()), "bitlinear_probe_int8_mma_rate")
+    return ops.value
 
 
 def bitlinear_poll_status() -> int:

@@ -319,6 +319,12 @@ int bitlinear_selftest_wait_timeout(unsigned limit_us, void* stream) {
     return cuda_status(cudaGetLastError());
 }
 
+int bitlinear_probe_int8_mma_rate(int n_mma_per_sm, double* ops_out, void* stream) {
+    if (n_mma_per_sm < 1 || n_mma_per_sm > 4000000) return BITLINEAR_ERR_SHAPE;  // a few milliseconds at most
+    if (int rc = check_arch()) return rc;
+    return int8_mma_rate_probe(n_mma_per_sm, ops_out, static_cast<cudaStream_t>(stream));
+}
+
 int bitlinear_poll_status(void* stream) {
     if (int rc = check_arch()) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

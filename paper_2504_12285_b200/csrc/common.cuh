@@ -104,6 +104,7 @@ size_t gemm_a_tiles_bytes(int M, int K);
 int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* codes, const float* s_w,
                  int M, int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st);
 size_t gemm_scratch_bytes(int N, int K);
+int int8_mma_rate_probe(int n_mma, double* ops_out, cudaStream_t st);
 
 // SM count of the current device (cached per device; BITLINEAR_ERR_ARCH unless it is compute capability 10.x).
 int device_sm_count(int* sm_count);

@@ -548,6 +548,54 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
     }
 }
 
+// ================================================================================================
+// Rate probe: how fast this GPU issues and retires tcgen05.mma kind::i8 when nothing else limits it.  Every CTA
+// (one per SM) fills one 128 x 128-byte A image and one 256 x 128-byte B image in shared memory once, then one thread
+// issues n_mma MMAs of 128 x 256 x 32 on them, alternating between the two accumulator halves of tensor memory; no
+// global memory traffic, no epilogue.  The benchmark divides the operations by the launch's device time and uses the
+// result as the denominator of the prefill numbers (a measured int8 peak instead of a datasheet figure).
+// ================================================================================================
+__global__ void __launch_bounds__(128, 1) int8_mma_rate_kernel(int n_mma, int* status_word) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    __shared__ uint64_t done_bar;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+    for (uint32_t o = threadIdx.x * 16; o < STAGE_BYTES; o += blockDim.x * 16)
+        *reinterpret_cast<uint4*>(smem + o) = make_uint4(0x01010101u, 0x01010101u, 0x01010101u, 0x01010101u);
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&done_bar), 1);
+        abort_flag = 0;
+        mbar_init_fence();
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read what generic stores wrote
+    if (threadIdx.x < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(TMEM_COLS)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_slot;
+    if (threadIdx.x == 0) {
+        constexpr uint32_t idesc = make_idesc(BM, BN);
+        const uint64_t a_desc = make_smem_desc(smem_u32(smem)), b_desc = make_smem_desc(smem_u32(smem) + A_BYTES);
+        for (int i = 0; i < n_mma; ++i)
+            umma_i8(tmem_base + (uint32_t)(i & 1) * BN, a_desc + (uint64_t)((i & 3) * UMMA_K / 16),
+                    b_desc + (uint64_t)((i & 3) * UMMA_K / 16), idesc, (uint32_t)(i > 1));
+        umma_commit(smem_u32(&done_bar));  // arrives once every MMA above has retired
+        mbar_wait(smem_u32(&done_bar), 0u, &abort_flag);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
+    if (threadIdx.x < 32) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
 // ---- host side -----------------------------------------------------------------------------------
 
 using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -687,6 +735,21 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     if (a_tiled) gemm_i8_kernel<true><<<grid, THREADS, SMEM_BYTES, st>>>(map_a, table_dev, device_status_word());
     else gemm_i8_kernel<false><<<grid, THREADS, SMEM_BYTES, st>>>(map_a, table_dev, device_status_word());
     return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+
+// Launches the rate probe on every SM; ops_out (host) receives the integer operations of the launch (2 per MAC).
+int int8_mma_rate_probe(int n_mma, double* ops_out, cudaStream_t st) {
+    int sm_count = 0;
+    if (const int rc = device_sm_count(&sm_count)) return rc;
+    const size_t smem = STAGE_BYTES + 1024;
+    if (cudaFuncSetAttribute(int8_mma_rate_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
+    int8_mma_rate_kernel<<<sm_count, 128, smem, st>>>(n_mma, device_status_word());
+    if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    if (ops_out) *ops_out = 2.0 * BM * BN * UMMA_K * (double)n_mma * sm_count;
+    return BITLINEAR_OK;
 }
 
 // One matmul on row-major int8 activations; `scratch` holds the code tiles followed by the group table.
