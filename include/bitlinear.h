@@ -223,12 +223,14 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  * weight bytes streamed from HBM) take two launches together: one fused RMSNorm+quantiser launch
  * over every token, then one persistent kernel that streams the packed weights of all of them
  * back to back (dot-products-of-four when every such problem has one token; otherwise the tensor
- * cores, with the codes unpacked in registers and handed over in tensor memory).  Problems of more
- * than 16 tokens (prefill; N must be a multiple of 128) take three
+ * cores, with the codes unpacked in registers and handed over in tensor memory).  Problems of 17 to
+ * 96 tokens (K <= 8192) are cut into 16-token problems for that same decode kernel: streaming the
+ * packed weights once per 16 tokens is measured faster there than a tensor-core tile that is mostly
+ * padding.  Longer problems (prefill; N must be a multiple of 128) take three
  * launches together: the quantiser, the expansion of the packed weights into tensor-core tile
  * images, and one persistent tcgen05 kernel that runs every tile of every matmul; problems that
  * name the same x, gain, rms_eps, M and K (q/k/v or gate/up of a layer) share one quantised copy.
- * Both kinds may be mixed in one call.
+ * All kinds may be mixed in one call.
  * Weights in the dense layout (w_format = BITLINEAR_WEIGHTS_DENSE5, Table 1 / Section 5.1) are accepted for
  * problems of at most 16 tokens; all such problems of a call must use the same layout.  Their kernel is the
  * one-token streaming kernel with the base-3 digits peeled off in registers; a problem of M tokens streams its

@@ -20,6 +20,7 @@
 //             Unpack: word & (0x03030303 << 2j) is 4^j x the codes of four consecutive columns, fed
 //             to a dot-product-of-four with the int8 activations; one accumulator per j keeps the
 //             scale uniform and the four are folded once per row block.
+#include <algorithm>
 #include <map>
 #include <tuple>
 #include <type_traits>
@@ -801,6 +802,64 @@ int check_input_step(const bitlinear_problem& q) {
     return BITLINEAR_OK;
 }
 
+// Up to this many tokens a problem of the 2-bit layout is cut into problems of 16 tokens for the tensor-core decode
+// kernel, which streams the packed weights once per 16 tokens; above it the weights are expanded to byte codes and
+// multiplied by the tcgen05 GEMM on 256-token tiles.  Measured on the FFN down projection (2560 x 6912) in a batch of 32
+// such matmuls: 2.2 us per matmul at 32 tokens and 4.0 us at 64 through the decode kernel, 7.7 us through the GEMM at
+// either (a 256 x 256 tile is mostly padding below 128 tokens); at 256 tokens the GEMM takes 7.8 us.
+constexpr int kDecodeChunkMaxTokens = 96;
+
+// Row m0 onwards of a problem as a problem of its own (m rows): every operand advanced by its own row size.
+bitlinear_problem rows_of(const bitlinear_problem& q, int m0, int m) {
+    bitlinear_problem c = q;
+    const size_t K = (size_t)q.K;
+    auto adv = [&](const void* p, size_t row_bytes) {
+        return p ? static_cast<const void*>(static_cast<const char*>(p) + (size_t)m0 * row_bytes) : nullptr;
+    };
+    const bool x_is_f32 = q.x_op == BITLINEAR_X_RELU2 || q.x_op == BITLINEAR_X_ATTN_STANDIN;
+    c.x = adv(q.x, K * (x_is_f32 ? 4 : 2));
+    c.x2 = adv(q.x2, (q.x_op == BITLINEAR_X_ATTN_STANDIN ? K / q.x_arg1 : K) * 4);
+    c.x_out = const_cast<void*>(adv(q.x_out, K * 2));
+    c.y = const_cast<void*>(adv(q.y, (size_t)q.N * (q.y_dtype == BITLINEAR_BF16 ? 2 : 4)));
+    c.M = m;
+    return c;
+}
+
+// Splits the problems of a call into those of the decode kernels (at most 16 tokens each, longer ones cut into chunks
+// where that is the faster path) and those of the grouped GEMM (indices).  Returns a status.
+int partition_problems(const bitlinear_problem* problems, int count, int32_t* const* acc_out, std::vector<bitlinear_problem>& dec,
+                       std::vector<int32_t*>& dec_acc, std::vector<int>& pre) {
+    for (int i = 0; i < count; ++i) {
+        const bitlinear_problem& q = problems[i];
+        if (q.y_dtype != BITLINEAR_F32 && q.y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
+        if (q.w_format != BITLINEAR_WEIGHTS_2BIT && q.w_format != BITLINEAR_WEIGHTS_DENSE5) return BITLINEAR_ERR_DTYPE;
+        if (q.M < 0 || !shape_ok(q.N, q.K)) return BITLINEAR_ERR_SHAPE;
+        if (const int rc = check_input_step(q)) return rc;
+        int32_t* acc = acc_out ? acc_out[i] : nullptr;
+        if (q.M <= kGemvMaxTokens) {
+            if (q.K > kBatchMaxK) return BITLINEAR_ERR_SHAPE;
+            dec.push_back(q);
+            dec_acc.push_back(acc);
+            continue;
+        }
+        if (q.w_format != BITLINEAR_WEIGHTS_2BIT || acc) return BITLINEAR_ERR_SHAPE;  // dense layout / accumulators: decode sizes only
+        if (q.M <= kDecodeChunkMaxTokens && q.K <= kBatchMaxK) {
+            for (int m0 = 0; m0 < q.M; m0 += kGemvMaxTokens) {
+                dec.push_back(rows_of(q, m0, std::min(kGemvMaxTokens, q.M - m0)));
+                dec_acc.push_back(nullptr);
+            }
+            continue;
+        }
+        if (q.N % 128) return BITLINEAR_ERR_SHAPE;
+        if (!q.x || !q.packed || !q.s_w || !q.y) return BITLINEAR_ERR_NULL;
+        if (!aligned16(q.x) || !aligned16(q.packed) || !aligned16(q.y) || (q.gain && !aligned16(q.gain)) ||
+            (reinterpret_cast<uintptr_t>(q.s_w) & 3u))
+            return BITLINEAR_ERR_ALIGN;
+        pre.push_back(i);
+    }
+    return BITLINEAR_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -808,19 +867,9 @@ extern "C" {
 size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
     if (!problems || count <= 0) return 0;
     std::vector<bitlinear_problem> dec;
+    std::vector<int32_t*> dec_acc;
     std::vector<int> pre;
-    for (int i = 0; i < count; ++i) {
-        const bitlinear_problem& q = problems[i];
-        if (q.M < 0 || !shape_ok(q.N, q.K)) return 0;
-        if (q.w_format != BITLINEAR_WEIGHTS_2BIT && q.w_format != BITLINEAR_WEIGHTS_DENSE5) return 0;
-        if (q.M <= kGemvMaxTokens) {
-            if (q.K > kBatchMaxK) return 0;
-            dec.push_back(q);
-        } else {
-            if (q.N % 128 || q.w_format != BITLINEAR_WEIGHTS_2BIT) return 0;
-            pre.push_back(i);
-        }
-    }
+    if (partition_problems(problems, count, nullptr, dec, dec_acc, pre) != BITLINEAR_OK) return 0;
     size_t total = 0;
     if (!dec.empty()) total += align_up(decode_batch_workspace_bytes(dec.data(), (int)dec.size()), 1024);
     if (!pre.empty()) total += prefill_group_workspace_bytes(problems, pre.data(), (int)pre.size());
@@ -841,26 +890,7 @@ int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, in
     std::vector<bitlinear_problem> dec;
     std::vector<int32_t*> dec_acc;
     std::vector<int> pre;
-    for (int i = 0; i < count; ++i) {
-        const bitlinear_problem& q = problems[i];
-        if (q.y_dtype != BITLINEAR_F32 && q.y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
-        if (q.w_format != BITLINEAR_WEIGHTS_2BIT && q.w_format != BITLINEAR_WEIGHTS_DENSE5) return BITLINEAR_ERR_DTYPE;
-        if (q.M < 0 || !shape_ok(q.N, q.K)) return BITLINEAR_ERR_SHAPE;
-        if (const int rc = check_input_step(q)) return rc;
-        if (q.M <= kGemvMaxTokens) {
-            if (q.K > kBatchMaxK) return BITLINEAR_ERR_SHAPE;
-            dec.push_back(q);
-            dec_acc.push_back(acc_out ? acc_out[i] : nullptr);
-            continue;
-        }
-        // more than 16 tokens: the tensor-core path, which reads the 2-bit layout and has no accumulator output
-        if (q.N % 128 || q.w_format != BITLINEAR_WEIGHTS_2BIT || (acc_out && acc_out[i])) return BITLINEAR_ERR_SHAPE;
-        if (!q.x || !q.packed || !q.s_w || !q.y) return BITLINEAR_ERR_NULL;
-        if (!aligned16(q.x) || !aligned16(q.packed) || !aligned16(q.y) || (q.gain && !aligned16(q.gain)) ||
-            (reinterpret_cast<uintptr_t>(q.s_w) & 3u))
-            return BITLINEAR_ERR_ALIGN;
-        pre.push_back(i);
-    }
+    if (const int rc = partition_problems(problems, count, acc_out, dec, dec_acc, pre)) return rc;
     const size_t dec_bytes = dec.empty() ? 0 : align_up(decode_batch_workspace_bytes(dec.data(), (int)dec.size()), 1024);
     const size_t pre_bytes = pre.empty() ? 0 : prefill_group_workspace_bytes(problems, pre.data(), (int)pre.size());
     if (!ws || !aligned16(ws) || ws_bytes < dec_bytes + pre_bytes) return BITLINEAR_ERR_WORKSPACE;

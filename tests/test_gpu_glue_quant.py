@@ -53,7 +53,7 @@ def check_y(y, ref):
     assert np.all(got[ref["acc"][ok] == 0] == 0.0)
 
 
-@pytest.mark.parametrize("M", [1, 4, 40])
+@pytest.mark.parametrize("M", [1, 4, 40, 130])  # one token, tensor-core decode, 16-token chunks, grouped GEMM
 def test_batch_with_fused_steps(M):
     # a layer's dependence pattern in one call each: {q,k,v}(residual), o(stand-in), {gate,up}(residual), down(relu2)
     H, F, n_q, n_kv, hd = 512, 768, 4, 2, 128
