@@ -724,6 +724,25 @@ def run_case_batch(args, bl, dev):
                       "hbm_peak": load_peaks()["hbm_gbs"]}))
 
 
+def run_case_chain(args, bl, dev):
+    """The dependent chain of --layers layers at one token through the persistent kernel (a smaller copy of configs[2])."""
+    from paper_2504_12285_b200 import chain as gpu_chain
+
+    pool = build_decode_pool(bl, dev, args.layers)
+    packed_bytes = sum(p["packed"].numel() for p in pool)
+    gains = {k: wl.gain_ones(k).to(dev) for k in (wl.HIDDEN, wl.FFN)}
+    pl = [dict({m["name"]: (m["packed"], m["s_w"]) for m in pool[layer * 7:(layer + 1) * 7]},
+               gains=[gains[wl.HIDDEN], gains[wl.HIDDEN], gains[wl.HIDDEN], gains[wl.FFN]]) for layer in range(args.layers)]
+    pc = gpu_chain.PersistentChain(pl, wl.HIDDEN, wl.FFN, wl.N_Q_HEADS, wl.N_KV_HEADS, wl.HEAD_DIM, wl.RMS_EPS, dev)
+    h0 = wl.activations_normal(1, wl.HIDDEN, wl.seed_for(3)).to(dev)
+    for _ in range(args.warmup):
+        pc.step(h0)
+    ms = cuda_time_ms(lambda: [pc.step(h0) for _ in range(args.steps)]) / args.steps
+    assert bl.bitlinear_poll_status() == 0
+    print(json.dumps({"case": "chain", "layers": args.layers, "packed_bytes": packed_bytes, "us_per_token": round(ms * 1e3, 1),
+                      "us_per_level": round(ms * 1e3 / (4 * args.layers), 3), "packed_GBps": round(packed_bytes / ms / 1e6, 1)}))
+
+
 def run_case_group(args, bl, dev):
     """The 7 shapes of a layer at --m tokens as one grouped call (quantiser + unpack + grouped GEMM)."""
     M = args.m
@@ -758,6 +777,8 @@ def run_case(args):
         return run_case_batch(args, bl, dev)
     if args.case == "group":
         return run_case_group(args, bl, dev)
+    if args.case == "chain":
+        return run_case_chain(args, bl, dev)
     n, k = wl.SHAPE_NK[args.shape]
     M = args.m
     peaks = load_peaks()
@@ -806,7 +827,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", choices=["gemv", "gemm", "quant", "pack", "batch", "group"], default=None)
+    ap.add_argument("--case", choices=["gemv", "gemm", "quant", "pack", "batch", "group", "chain"], default=None)
     ap.add_argument("--layers", type=int, default=10)
     ap.add_argument("--shape", choices=list(wl.SHAPE_NK), default="q")
     ap.add_argument("--m", type=int, default=1)
