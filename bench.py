@@ -759,9 +759,13 @@ def run_case_group(args, bl, dev):
         bl.bitlinear_forward_batch(batch, ws)
     ms = cuda_time_ms(lambda: [bl.bitlinear_forward_batch(batch, ws) for _ in range(args.steps)]) / args.steps
     ms_mm = cuda_time_ms(lambda: [bl.bitlinear_forward_batch(batch, ws, reuse_act=True) for _ in range(args.steps)]) / args.steps
+    ms_g = cuda_time_ms(lambda: [bl.bitlinear_forward_batch(batch, ws, reuse_act=True, reuse_weights=True) for _ in range(args.steps)]) / args.steps
+    ms_qg = cuda_time_ms(lambda: [bl.bitlinear_forward_batch(batch, ws, reuse_weights=True) for _ in range(args.steps)]) / args.steps
     ops = sum(2.0 * M * p["N"] * p["K"] for p in pool)
     print(json.dumps({"case": "group", "M": M, "us_forward": round(ms * 1e3, 2), "forward_tops": round(ops / ms / 1e9, 1),
-                      "us_unpack_gemm": round(ms_mm * 1e3, 2), "unpack_gemm_tops": round(ops / ms_mm / 1e9, 1)}))
+                      "us_unpack_gemm": round(ms_mm * 1e3, 2), "unpack_gemm_tops": round(ops / ms_mm / 1e9, 1),
+                      "us_gemm_only": round(ms_g * 1e3, 2), "gemm_only_tops": round(ops / ms_g / 1e9, 1),
+                      "us_quant_gemm": round(ms_qg * 1e3, 2)}))
 
 
 def run_case(args):

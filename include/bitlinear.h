@@ -242,7 +242,8 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  *   flags    : 0, or an OR of BITLINEAR_BATCH_REUSE_PLAN (the previous call on this workspace had
  *              exactly the same descriptors: skips re-uploading the decode plan) and
  *              BITLINEAR_BATCH_REUSE_ACT (the inputs are unchanged as well: skips the quantiser
- *              launches and reuses their results in ws).
+ *              launches and reuses their results in ws), BITLINEAR_BATCH_REUSE_WEIGHTS (same
+ *              descriptors and same packed matrices: skips the expansion of the prefill problems).
  *   ws       : device scratch of at least bitlinear_batch_workspace_bytes(problems, count); it
  *              holds the uploaded plan, the quantised activations and the expanded weights of the
  *              prefill problems, so a call must not overlap another call that uses the same
@@ -283,6 +284,10 @@ typedef struct bitlinear_problem {
 
 #define BITLINEAR_BATCH_REUSE_PLAN 1 /* descriptors unchanged since the previous call on this workspace */
 #define BITLINEAR_BATCH_REUSE_ACT 2  /* inputs x unchanged too: skip the quantiser launch, reuse its results in ws */
+#define BITLINEAR_BATCH_REUSE_WEIGHTS 4 /* same packed matrices as the previous call on this workspace: the byte codes the
+                                           prefill problems were expanded to are still in ws and are not expanded again
+                                           (prefill is compute-bound: a caller with memory to spare keeps one workspace
+                                           per layer and pays the expansion once, not per call) */
 
 size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count);
 int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,

@@ -69,6 +69,7 @@ WEIGHTS_2BIT, WEIGHTS_DENSE5 = 0, 1
 X_PLAIN, X_RELU2, X_RESIDUAL, X_ATTN_STANDIN = 0, 1, 2, 3
 BATCH_REUSE_PLAN = 1
 BATCH_REUSE_ACT = 2
+BATCH_REUSE_WEIGHTS = 4
 
 
 class Problem(ctypes.Structure):
@@ -434,10 +435,11 @@ def bitlinear_batch_workspace_bytes(batch: ProblemBatch) -> int:
 
 
 def bitlinear_forward_batch(batch: ProblemBatch, ws: torch.Tensor, reuse_plan: bool = False,
-                            reuse_act: bool = False) -> None:
+                            reuse_act: bool = False, reuse_weights: bool = False) -> None:
     """Run every forward of the batch (decode sizes, M <= 16) in two launches; results land in the y tensors."""
     _dev(ws, torch.uint8, "ws")
-    flags = (BATCH_REUSE_PLAN if reuse_plan else 0) | (BATCH_REUSE_ACT if reuse_act else 0)
+    flags = ((BATCH_REUSE_PLAN if reuse_plan else 0) | (BATCH_REUSE_ACT if reuse_act else 0) |
+             (BATCH_REUSE_WEIGHTS if reuse_weights else 0))
     rc = lib().bitlinear_forward_batch(ctypes.addressof(batch.array), batch.count, flags, _ptr(ws), ws.numel(),
                                        _stream())
     _check(rc, "bitlinear_forward_batch")

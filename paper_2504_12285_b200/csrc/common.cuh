@@ -69,7 +69,7 @@ struct GemmProblem {
     int m_tiles;     // ceil(M / 128)
     int tile_begin;  // tiles of the problems before this one
     int nt_begin;    // 256-row weight tiles of the problems before this one (index into the ready counters)
-    int pad;
+    int at_begin;    // index of the token-tile counters of this problem's quantised activations (GemmGroupHeader::a_ready)
 };
 constexpr int kMaxGroup = 32;
 struct GemmGroupHeader {
@@ -83,11 +83,19 @@ struct GemmGroupHeader {
     // sums) it must wait for with griddepcontrol.wait; 0 if it is the expansion launch, which `ready` covers
     int wait_primary;
     int pad;
+    // CTA-pair kernel, or nullptr: a_ready[at_begin + mt] counts the tokens of 256-token tile mt of a problem's activations
+    // that the quantiser launch has finished (codes, scale and code sum written); the kernel then runs beside the quantiser
+    // too and reads a token tile once the count has reached the tile's tokens
+    const int* a_ready;
 };
 // layout of the uploaded group table: GemmGroupHeader, then count x GemmProblem
 constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof(GemmProblem);
+// the grouped launch keeps one 128-byte tensor map per problem (view of its packed weights) behind the table
+constexpr size_t kGroupMapsOffset = (kGroupTableBytes + 127) / 128 * 128;
+constexpr size_t kGroupTableDevBytes = kGroupMapsOffset + kMaxGroup * 128;
 
-// Grouped launch: fills m_tiles / tile_begin, uploads the table to table_dev (kGroupTableBytes) and runs every tile of
+// Grouped launch: fills m_tiles / tile_begin, uploads the table to table_dev (kGroupTableDevBytes when `packed` is given,
+// else kGroupTableBytes) and runs every tile of
 // every problem in one persistent kernel.  a_tiled = activations given as tile images (any count), else one problem with
 // row-major activations.  Returns a bitlinear_status.
 // `before` (optional) is called after the table upload and before the GEMM kernel is launched: launches that produce
@@ -96,7 +104,8 @@ constexpr size_t kGroupTableBytes = sizeof(GemmGroupHeader) + kMaxGroup * sizeof
 typedef int (*GemmBeforeKernel)(void* ctx);
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev, cudaStream_t st,
                 const void* region_base = nullptr, size_t region_bytes = 0, const int* ready = nullptr,
-                GemmBeforeKernel before = nullptr, void* before_ctx = nullptr, bool wait_primary = false);
+                GemmBeforeKernel before = nullptr, void* before_ctx = nullptr, bool wait_primary = false,
+                const int* a_ready = nullptr, const void* const* packed = nullptr);
 size_t gemm_codes_bytes(int N, int K);
 size_t gemm_a_tiles_bytes(int M, int K);
 

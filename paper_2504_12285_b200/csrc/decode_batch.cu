@@ -528,7 +528,7 @@ namespace bitlinear {
 
 size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const int* idx, int n);
 int prefill_group_forward(const bitlinear_problem* problems, const int* idx, int n, void* ws, bool skip_quant,
-                          cudaStream_t st);
+                          bool skip_unpack, cudaStream_t st);
 // Sub-batches with a problem of more than kDp4aMaxTokens tokens run on the tensor cores (decode_mma.cu): measured on
 // the 210-matmul decode step, 145 us per step there at 2 to 5 tokens against 171 to 174 us for the kernel below.
 size_t decode_mma_workspace_bytes(const bitlinear_problem* problems, int count);
@@ -886,7 +886,7 @@ int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, in
     if (count < 0) return BITLINEAR_ERR_SHAPE;
     if (count == 0) return BITLINEAR_OK;
     if (!problems) return BITLINEAR_ERR_NULL;
-    if (flags & ~(BITLINEAR_BATCH_REUSE_PLAN | BITLINEAR_BATCH_REUSE_ACT)) return BITLINEAR_ERR_DTYPE;
+    if (flags & ~(BITLINEAR_BATCH_REUSE_PLAN | BITLINEAR_BATCH_REUSE_ACT | BITLINEAR_BATCH_REUSE_WEIGHTS)) return BITLINEAR_ERR_DTYPE;
     std::vector<bitlinear_problem> dec;
     std::vector<int32_t*> dec_acc;
     std::vector<int> pre;
@@ -895,7 +895,7 @@ int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, in
     const size_t pre_bytes = pre.empty() ? 0 : prefill_group_workspace_bytes(problems, pre.data(), (int)pre.size());
     if (!ws || !aligned16(ws) || ws_bytes < dec_bytes + pre_bytes) return BITLINEAR_ERR_WORKSPACE;
     if (!dec.empty()) {
-        const int rc = decode_batch_forward(dec.data(), (int)dec.size(), flags, acc_out ? dec_acc.data() : nullptr, ws, dec_bytes, stream);
+        const int rc = decode_batch_forward(dec.data(), (int)dec.size(), flags & ~BITLINEAR_BATCH_REUSE_WEIGHTS, acc_out ? dec_acc.data() : nullptr, ws, dec_bytes, stream);
         if (rc != BITLINEAR_OK) return rc;
     }
     if (!pre.empty()) {
@@ -910,7 +910,8 @@ int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, in
             }())
             return rc;
         return prefill_group_forward(problems, pre.data(), (int)pre.size(), static_cast<char*>(ws) + dec_bytes,
-                                     (flags & BITLINEAR_BATCH_REUSE_ACT) != 0, static_cast<cudaStream_t>(stream));
+                                     (flags & BITLINEAR_BATCH_REUSE_ACT) != 0, (flags & BITLINEAR_BATCH_REUSE_WEIGHTS) != 0,
+                                     static_cast<cudaStream_t>(stream));
     }
     return BITLINEAR_OK;
 }

@@ -152,8 +152,9 @@ __device__ __forceinline__ void drain_accumulator(const GemmProblem& p, uint32_t
     const float s_w = *p.s_w;
     const int m = m_warp + lane;
     const bool row_ok = m < M;
-    const int xs = row_ok ? p.xsum[m] : 0;
-    const float dm = row_ok ? p.d[m] : 0.0f;
+    // read through L2: the quantiser launch that wrote them may still be running beside this kernel (other rows)
+    const int xs = row_ok ? __ldcg(p.xsum + m) : 0;
+    const float dm = row_ok ? __ldcg(p.d + m) : 0.0f;
     const int rows_ok = (M - m_warp) < 32 ? (M - m_warp) : 32;
 #pragma unroll 1
     for (int c = 0; c < BN / 32; ++c) {
@@ -350,10 +351,18 @@ gemm_i8_kernel(const __grid_constant__ CUtensorMap map_a, const uint8_t* __restr
 // mbarrier from either CTA: the tensor map views the whole workspace region as rows of 128 bytes, no
 // swizzle (the images are stored swizzled).
 // ================================================================================================
-constexpr int P_STAGES = 6;
+// PACKED variant: the CTA's half of the weight tile arrives as PACKED 2-bit codes (4 KiB per k-block, fetched with one
+// 4-D tensor-map copy straight out of the packed matrix) and four more warps expand it in shared memory into the
+// swizzled byte-code image the MMA reads.  No expansion launch, no code images in global memory, and a quarter of the
+// weight bytes on the L2 -> SM path, which is what bounds this kernel.
 constexpr uint32_t P_HALF_BYTES = 128 * BK;              // 128 rows x 128 bytes
-constexpr uint32_t P_STAGE_BYTES = 2 * P_HALF_BYTES;     // A rows of this CTA + its half of B
-constexpr size_t P_SMEM_BYTES = 1024 + (size_t)P_STAGES * P_STAGE_BYTES + 256 + 4 * 32 * 144 + 3072;
+constexpr uint32_t P_PACKED_BYTES = 128 * BK / 4;        // the same rows as 2-bit codes
+template <bool PACKED> struct PairCfg {
+    static constexpr int kStages = PACKED ? 5 : 6;
+    static constexpr uint32_t kStageBytes = 2 * P_HALF_BYTES + (PACKED ? P_PACKED_BYTES : 0);  // A rows + half of B (+ packed)
+    static constexpr int kThreads = PACKED ? THREADS + 128 : THREADS;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256 + 4 * 32 * 144 + 3072;
+};
 constexpr uint32_t kPeerMask = 0xFEFFFFFFu;  // clears the cluster-rank bit of a shared::cluster address: the pair's rank-0 CTA
 
 __device__ __forceinline__ uint32_t cluster_ctarank() {
@@ -390,9 +399,21 @@ __device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_leader(uint32_t bar_local) {
     asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_local & kPeerMask) : "memory");
 }
+// 4-D tensor-map copy into this CTA's shared memory, completion bytes on this CTA's own mbarrier
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, int w, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(w), "r"(bar)
+        : "memory");
+}
 
-__global__ void __launch_bounds__(THREADS, 1)
-gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __restrict__ table_g, int* status_word) {
+template <bool PACKED>
+__global__ void __launch_bounds__(PairCfg<PACKED>::kThreads, 1)
+gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __restrict__ table_g, const CUtensorMap* __restrict__ w_maps,
+                    int* status_word) {
+    constexpr int P_STAGES = PairCfg<PACKED>::kStages;
+    constexpr uint32_t P_STAGE_BYTES = PairCfg<PACKED>::kStageBytes;
+    constexpr int kThreadsAll = PairCfg<PACKED>::kThreads;
     extern __shared__ uint8_t smem_raw[];
     // the rounding of the base is the same in both CTAs (same launch, same dynamic offset), so operand offsets match
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -401,7 +422,8 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
     uint64_t* empty_bar = bars + P_STAGES;        // [P_STAGES] each CTA: the MMAs that read the stage retired
     uint64_t* tfull_bar = bars + 2 * P_STAGES;    // [2] each CTA: accumulator buffer complete
     uint64_t* tempty_bar = tfull_bar + 2;         // [2] leader: drained by the 8 epilogue warps of the pair
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty_bar + 2);
+    uint64_t* pfull_bar = tempty_bar + 2;         // [P_STAGES] each CTA (PACKED): its packed weight bytes landed
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pfull_bar + P_STAGES);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     uint8_t* table_s = smem + (size_t)P_STAGES * P_STAGE_BYTES + 256 + 4 * STAGE_OUT_BYTES;
 
@@ -409,13 +431,15 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
     const int pair = (int)blockIdx.x >> 1, n_pairs = (int)gridDim.x >> 1;
-    for (int o = threadIdx.x * 16; o < (int)kGroupTableBytes; o += THREADS * 16)
+    for (int o = threadIdx.x * 16; o < (int)kGroupTableBytes; o += kThreadsAll * 16)
         *reinterpret_cast<uint4*>(table_s + o) = *reinterpret_cast<const uint4*>(table_g + o);
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) {
-            mbar_init(smem_u32(full_bar + s), 1);
+            // PACKED: the leader's barrier also counts the eight expander warps of the pair (the code image is written)
+            mbar_init(smem_u32(full_bar + s), PACKED ? 9 : 1);
             mbar_init(smem_u32(empty_bar + s), 1);
+            mbar_init(smem_u32(pfull_bar + s), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(tfull_bar + b), 1);
@@ -466,6 +490,20 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
                     asm volatile("fence.proxy.async;" ::: "memory");  // the copies below read what generic stores wrote
                     ready_idx = p.nt_begin + nt;
                 }
+                if (hdr.a_ready != nullptr) {
+                    // the quantiser launch may still be writing this token tile: wait for its token count (bounded)
+                    const int target = min(256, p.M - mt * 256);
+                    const unsigned long long t0 = globaltimer_ns();
+                    unsigned spins = 0;
+                    while (ld_acquire_gpu_s32(hdr.a_ready + p.at_begin + mt) < target) {
+                        if ((++spins & 63u) == 0u) {
+                            if (*abort_flag) { ok = false; break; }
+                            if (globaltimer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; ok = false; break; }
+                        }
+                    }
+                    if (!ok) break;
+                    asm volatile("fence.proxy.async;" ::: "memory");
+                }
                 // rows (of 128 bytes) of this CTA's operand images inside the mapped region
                 const int a_row = (int)((reinterpret_cast<unsigned long long>(p.a_tiles) - hdr.region_base) >> 7) +
                                   (2 * mt + (int)rank) * k_blocks * 128;
@@ -474,10 +512,20 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
                 for (int kb = 0; kb < k_blocks; ++kb) {
                     if (!mbar_wait(smem_u32(empty_bar + stage), phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t fb = smem_u32(full_bar + stage);
-                    if (leader) mbar_expect_tx(fb, 2 * P_STAGE_BYTES);  // its own copies and the peer's
                     const uint32_t sa = smem_u32(smem + (size_t)stage * P_STAGE_BYTES);
-                    tma_load_2d_pair(sa, &map, 0, a_row + kb * 128, fb);
-                    tma_load_2d_pair(sa + P_HALF_BYTES, &map, 0, b_row + kb * 256, fb);
+                    if constexpr (PACKED) {
+                        if (leader) mbar_expect_tx(fb, 2 * P_HALF_BYTES);  // the token rows of both CTAs
+                        tma_load_2d_pair(sa, &map, 0, a_row + kb * 128, fb);
+                        // this CTA's 128 weight rows x 128 columns as packed codes: 8 row blocks x 16 rows x 32 bytes of the
+                        // packed matrix (half of the 16 x 256 tile kb / 2 of each row block)
+                        const uint32_t pb = smem_u32(pfull_bar + stage);
+                        mbar_expect_tx(pb, P_PACKED_BYTES);
+                        tma_load_4d(sa + 2 * P_HALF_BYTES, w_maps + walk.pi, 32 * (kb & 1), 0, kb >> 1, 16 * nt + 8 * (int)rank, pb);
+                    } else {
+                        if (leader) mbar_expect_tx(fb, 2 * P_STAGE_BYTES);  // its own copies and the peer's
+                        tma_load_2d_pair(sa, &map, 0, a_row + kb * 128, fb);
+                        tma_load_2d_pair(sa + P_HALF_BYTES, &map, 0, b_row + kb * 256, fb);
+                    }
                     if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -513,6 +561,37 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
             }
         }
         __syncwarp();
+    } else if (PACKED && warp >= 6) {
+        // ------------------------------------------------------------------ expanders (PACKED; both CTAs, own half of B)
+        // Packed staging: [8 row blocks][16 rows][32 bytes]; word w of row r holds columns 16 w .. 16 w + 15 of the
+        // k-block, byte b bits 2j = column 4 j + b: (word >> 2 j) & 0x03030303 is the 4 bytes 4 j .. 4 j + 3 of the
+        // 16-byte piece w of the row's 128-byte code row, which sits swizzled at r * 128 + ((w ^ (r & 7)) * 16).
+        const int et = (int)threadIdx.x - 192;   // 0..127
+        const int piece = et & 7, r0 = et >> 3;  // a quarter warp writes one whole 128-byte row per store
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (int tile = pair; ok && tile < total_tiles; tile += n_pairs) {
+            const int k_blocks = walk.find(tile).K / BK;
+            for (int kb = 0; kb < k_blocks; ++kb) {
+                if (!mbar_wait(smem_u32(pfull_bar + stage), phase, abort_flag)) { ok = false; break; }
+                const uint32_t sb = smem_u32(smem + (size_t)stage * P_STAGE_BYTES) + P_HALF_BYTES;
+                const uint32_t sp = sb + P_HALF_BYTES;
+                uint32_t w[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w[i]) : "r"(sp + (uint32_t)(r0 + 16 * i) * 32u + 4u * piece));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = r0 + 16 * i;
+                    sts128(sb + (uint32_t)r * 128u + (uint32_t)((piece ^ (r & 7)) << 4), w[i] & 0x03030303u, (w[i] >> 2) & 0x03030303u,
+                           (w[i] >> 4) & 0x03030303u, (w[i] >> 6) & 0x03030303u);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMA reads what these stores wrote
+                __syncwarp();
+                if (lane == 0) mbar_arrive_leader(smem_u32(full_bar + stage));
+                if (++stage == P_STAGES) { stage = 0; phase ^= 1u; }
+            }
+        }
     } else {
         // ------------------------------------------------------------------ epilogue (both CTAs, own 128 rows)
         const int quad = warp & 3;
@@ -650,9 +729,25 @@ bool make_map_rows128(CUtensorMap* map, const void* base, size_t bytes) {
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 4-D view of a packed [N][K] matrix for the PACKED pair kernel: x = 64 bytes of a tile row, y = the 16 rows of a tile,
+// z = the K / 256 tiles of a row block, w = the N / 16 row blocks; box = 32 bytes x 16 rows x 1 tile x 8 row blocks, i.e.
+// 128 weight rows x 128 columns of 2-bit codes (4 KiB) per copy.
+bool make_map_packed(CUtensorMap* map, const void* packed, int N, int K) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn || (reinterpret_cast<uintptr_t>(packed) & 15u)) return false;
+    const cuuint64_t k_tiles = (cuuint64_t)(K / kTileCols);
+    const cuuint64_t dims[4] = {64, 16, k_tiles, (cuuint64_t)(N / kTileRows)};
+    const cuuint64_t strides[3] = {64, (cuuint64_t)kTileBytes, k_tiles * kTileBytes};
+    const cuuint32_t box[4] = {32, 16, 1, 8};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(packed), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_row_major, uint8_t* table_dev,
                 cudaStream_t st, const void* region_base, size_t region_bytes, const int* ready, GemmBeforeKernel before,
-                void* before_ctx, bool wait_primary) {
+                void* before_ctx, bool wait_primary, const int* a_ready, const void* const* packed) {
     // kernel attributes and the SM count are per device: set / looked up once for each device a process uses
     int sm_count = 0;
     {
@@ -668,7 +763,8 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
             int n = 0;
             if (cudaFuncSetAttribute(gemm_i8_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess ||
                 cudaFuncSetAttribute(gemm_i8_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BYTES) != cudaSuccess ||
-                cudaFuncSetAttribute(gemm_i8_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)P_SMEM_BYTES) != cudaSuccess ||
+                cudaFuncSetAttribute(gemm_i8_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairCfg<false>::kSmemBytes) != cudaSuccess ||
+                cudaFuncSetAttribute(gemm_i8_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PairCfg<true>::kSmemBytes) != cudaSuccess ||
                 cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) {
                 cudaGetLastError();
                 return BITLINEAR_ERR_CUDA;
@@ -696,11 +792,26 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     hdr->count = count;
     hdr->total_tiles = tiles;
     hdr->region_base = reinterpret_cast<unsigned long long>(region_base);
-    hdr->ready = pairs ? ready : nullptr;
-    hdr->wait_primary = (pairs && ready != nullptr && wait_primary) ? 1 : 0;
+    // PACKED mode: the weights are read as packed codes through one tensor map per problem and expanded in the kernel
+    const bool packed_mode = pairs && packed != nullptr;
+    hdr->ready = (pairs && !packed_mode) ? ready : nullptr;
+    hdr->a_ready = pairs ? a_ready : nullptr;
+    // griddepcontrol.wait in the kernel: only where the launch before it is the quantiser and no token-tile counters follow it
+    const bool dependent = pairs && (hdr->ready != nullptr || hdr->a_ready != nullptr);
+    hdr->wait_primary = (dependent && hdr->a_ready == nullptr && wait_primary) ? 1 : 0;
     if (cudaMemcpyAsync(table_dev, host, kGroupTableBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
+    }
+    CUtensorMap* w_maps_dev = reinterpret_cast<CUtensorMap*>(table_dev + kGroupMapsOffset);
+    if (packed_mode) {
+        alignas(64) CUtensorMap maps[kMaxGroup];
+        for (int i = 0; i < count; ++i)
+            if (!make_map_packed(&maps[i], packed[i], probs[i].N, probs[i].K)) return BITLINEAR_ERR_CUDA;
+        if (cudaMemcpyAsync(w_maps_dev, maps, sizeof(CUtensorMap) * count, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+            cudaGetLastError();
+            return BITLINEAR_ERR_CUDA;
+        }
     }
     if (before != nullptr) {
         const int rc = before(before_ctx);
@@ -713,8 +824,8 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
         int n_pairs = tiles < sm_count / 2 ? tiles : sm_count / 2;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(2 * n_pairs));
-        cfg.blockDim = dim3(THREADS);
-        cfg.dynamicSmemBytes = P_SMEM_BYTES;
+        cfg.blockDim = dim3(packed_mode ? PairCfg<true>::kThreads : PairCfg<false>::kThreads);
+        cfg.dynamicSmemBytes = packed_mode ? PairCfg<true>::kSmemBytes : PairCfg<false>::kSmemBytes;
         cfg.stream = st;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -725,8 +836,11 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
         attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
-        cfg.numAttrs = ready != nullptr ? 2 : 1;
-        const cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_i8_pair_kernel, map_a, (const uint8_t*)table_dev, device_status_word());
+        cfg.numAttrs = dependent ? 2 : 1;
+        const cudaError_t e = packed_mode ? cudaLaunchKernelEx(&cfg, gemm_i8_pair_kernel<true>, map_a, (const uint8_t*)table_dev,
+                                                               (const CUtensorMap*)w_maps_dev, device_status_word())
+                                          : cudaLaunchKernelEx(&cfg, gemm_i8_pair_kernel<false>, map_a, (const uint8_t*)table_dev,
+                                                               (const CUtensorMap*)w_maps_dev, device_status_word());
         if (e != cudaSuccess) cudaGetLastError();
         return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
     }

@@ -13,7 +13,8 @@
 //                                   pair up), operands fetched as whole tile images.  The pair kernel is a
 //                                   programmatic dependent too: it waits for launch 2 as a whole
 //                                   (griddepcontrol.wait) and for launch 1 tile by tile (the word counts).
-// Problems are ordered by decreasing K so that the long tiles are scheduled first and the tail is made of short ones.
+// Problems are ordered by decreasing K so that the long tiles are scheduled first and the tail is made of short ones,
+// after the small matrices, whose tiles can start while the large ones are still being expanded.
 #include <algorithm>
 #include <vector>
 
@@ -109,7 +110,7 @@ GroupLayout group_layout(const bitlinear_problem* problems, const int* idx, int 
     GroupLayout L;
     size_t off = 0;
     L.table_off = off;
-    off = align_up(off + kGroupTableBytes, 256);
+    off = align_up(off + kGroupTableDevBytes, 256);
     L.items_off = off;
     off = align_up(off + kItemTableBytes, 256);
     L.ready_off = off;
@@ -143,7 +144,7 @@ size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const in
 }
 
 int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, int n_in, void* ws, bool skip_quant,
-                          cudaStream_t st) {
+                          bool skip_unpack, cudaStream_t st) {
     char* base_all = static_cast<char*>(ws);
     int sm_count = 0, dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
@@ -155,12 +156,24 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
         const int n = std::min(kMaxGroup, n_in - b);
         std::vector<int> idx(idx_in + b, idx_in + b + n);
         std::stable_sort(idx.begin(), idx.end(), [&](int l, int r) { return problems[l].K > problems[r].K; });
+        // ... except that small matrices go first: their codes are expanded within a microsecond, so the GEMM's first
+        // tiles start at once while the expansion of the large matrices runs ahead of the tiles that need them
+        {
+            size_t largest = 0;
+            for (int i : idx) largest = std::max(largest, (size_t)problems[i].N * problems[i].K);
+            std::stable_partition(idx.begin(), idx.end(), [&](int i) { return (size_t)problems[i].N * problems[i].K * 4 <= largest; });
+        }
         const GroupLayout L = group_layout(problems, idx.data(), n);
         char* base = base_all;
         base_all += L.total;
 
         PrefillItem items[kMaxGroup] = {};
         GemmProblem gp[kMaxGroup] = {};
+        const void* packed_ptrs[kMaxGroup] = {};
+        // Where the SMs pair up the GEMM reads the packed weights themselves and expands them in shared memory: no
+        // expansion launch, no code images.  (Otherwise: expansion launch + single-CTA kernel on the code images.)
+        const bool in_kernel_expansion = (sm_count % 2) == 0;
+        if (in_kernel_expansion) skip_unpack = true;
         long long words = 0;
         int rows = 0, nt_total = 0;
         for (int i = 0; i < n; ++i) {
@@ -194,6 +207,7 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             } else {
                 rows += q.M;
             }
+            packed_ptrs[i] = q.packed;
             GemmProblem& g = gp[i];
             g.a_tiles = it.a_tiles; g.codes = it.codes; g.d = it.d; g.xsum = it.xsum; g.s_w = q.s_w;
             g.y = q.y; g.acc_out = nullptr;
@@ -213,16 +227,23 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
             int* ready;
             int n, rows, sm_count;
             long long words;
-            bool skip_quant;
+            bool skip_quant, skip_unpack;
             cudaStream_t st;
             static int run(void* ctx) {
                 const Launches& a = *static_cast<const Launches*>(ctx);
                 // the expansion first (at most four CTAs per SM, so that the other kernels find room beside them) ...
-                const long long chunks = (a.words + kUnpackChunk - 1) / kUnpackChunk;
-                const unsigned grid = (unsigned)std::min<long long>(chunks, 4LL * a.sm_count);
-                group_unpack_kernel<<<grid, 256, 0, a.st>>>(a.items_dev, a.n, a.words, a.ready);
-                if (cudaGetLastError() != cudaSuccess) return (int)BITLINEAR_ERR_CUDA;
+                if (!a.skip_unpack) {
+                    const long long chunks = (a.words + kUnpackChunk - 1) / kUnpackChunk;
+                    const unsigned grid = (unsigned)std::min<long long>(chunks, 4LL * a.sm_count);
+                    group_unpack_kernel<<<grid, 256, 0, a.st>>>(a.items_dev, a.n, a.words, a.ready);
+                    if (cudaGetLastError() != cudaSuccess) return (int)BITLINEAR_ERR_CUDA;
+                }
                 if (a.skip_quant) return (int)BITLINEAR_OK;
+                if (a.skip_unpack) {  // nothing to run beside: an ordinary launch, the GEMM after it is ordinary too
+                    group_quant_warp_kernel<<<(unsigned)((a.rows + kQuantWarps - 1) / kQuantWarps), kQuantThreads, 0, a.st>>>(
+                        a.items_dev, a.n, a.rows);
+                    return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
+                }
                 // ... then the quantiser as its programmatic dependent: the two share no data and run side by side
                 cudaLaunchConfig_t cfg = {};
                 cfg.gridDim = dim3((unsigned)((a.rows + kQuantWarps - 1) / kQuantWarps));
@@ -239,9 +260,12 @@ int prefill_group_forward(const bitlinear_problem* problems, const int* idx_in, 
                 }
                 return (int)BITLINEAR_OK;
             }
-        } launches = {items_dev, ready, n, rows, sm_count, words, skip_quant, st};
-        const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st, base, L.total, ready,
-                                   &Launches::run, &launches, /*wait_primary=*/!skip_quant);
+        } launches = {items_dev, ready, n, rows, sm_count, words, skip_quant, skip_unpack, st};
+        // with the expanded codes of an earlier call still in place there is nothing to follow tile by tile: the GEMM is
+        // then an ordinary launch behind the quantiser (or behind nothing)
+        const int rc = gemm_launch(gp, n, true, nullptr, reinterpret_cast<uint8_t*>(base + L.table_off), st, base, L.total,
+                                   skip_unpack ? nullptr : ready, &Launches::run, &launches, /*wait_primary=*/!skip_quant,
+                                   /*a_ready=*/nullptr, in_kernel_expansion ? packed_ptrs : nullptr);
         if (rc != BITLINEAR_OK) return rc;
     }
     return BITLINEAR_OK;
