@@ -253,6 +253,10 @@ int bitlinear_matmul_q(const int8_t* xq, const float* d, const int32_t* xsum, co
         return cuda_status(launch_gemv(xq, d, xsum, static_cast<const uint32_t*>(packed), s_w, M, N, K, y_out, y_dtype,
                                        acc_out, st));
     uint8_t* codes = static_cast<uint8_t*>(ws);
+    // where the SMs pair up, the CTA-pair kernel reads the packed weights directly and expands them in shared memory
+    if (gemm_pairs_available())
+        return gemm_tcgen05_packed(xq, d, xsum, packed, s_w, M, N, K, y_out, y_dtype, acc_out,
+                                   codes + align_up(gemm_codes_bytes(N, K), 256), st);
     cudaError_t e = launch_unpack_codes_u8(static_cast<const uint32_t*>(packed), N, K, codes, st);
     if (e != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return gemm_tcgen05(xq, d, xsum, codes, s_w, M, N, K, y_out, y_dtype, acc_out, st);

@@ -82,7 +82,9 @@ struct GemmGroupHeader {
     // CTA-pair kernel: 1 if the launch right before it is the quantiser, whose results (token images, scales, code
     // sums) it must wait for with griddepcontrol.wait; 0 if it is the expansion launch, which `ready` covers
     int wait_primary;
-    int pad;
+    // CTA-pair kernel on packed weights: 1 if the (single) problem's activations are a row-major [M][K] matrix fetched
+    // through a swizzling tensor map instead of tile images
+    int a_row_major;
     // CTA-pair kernel, or nullptr: a_ready[at_begin + mt] counts the tokens of 256-token tile mt of a problem's activations
     // that the quantiser launch has finished (codes, scale and code sum written); the kernel then runs beside the quantiser
     // too and reads a token tile once the count has reached the tile's tokens
@@ -113,6 +115,9 @@ size_t gemm_a_tiles_bytes(int M, int K);
 int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const uint8_t* codes, const float* s_w,
                  int M, int N, int K, void* y, int y_dtype, int32_t* acc_out, cudaStream_t st);
 size_t gemm_scratch_bytes(int N, int K);
+int gemm_tcgen05_packed(const int8_t* xq, const float* d, const int32_t* xsum, const void* packed, const float* s_w, int M,
+                        int N, int K, void* y, int y_dtype, int32_t* acc_out, uint8_t* table_dev, cudaStream_t st);
+bool gemm_pairs_available();  // the SMs of the current device pair up (CTA-pair kernels can run)
 int int8_mma_rate_probe(int n_mma, double* ops_out, cudaStream_t st);
 
 // SM count of the current device (cached per device; BITLINEAR_ERR_ARCH unless it is compute capability 10.x).

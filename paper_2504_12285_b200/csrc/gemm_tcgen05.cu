@@ -407,10 +407,19 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         : "memory");
 }
 
+// A single matmul needs no table in global memory: header, problem and the tensor map of its packed weights travel as
+// kernel parameters, so a single call is the launch alone (no host-to-device copies in front of it).
+struct PairInline {
+    GemmGroupHeader hdr;
+    GemmProblem prob;
+    alignas(64) CUtensorMap w_map;
+    int use;  // 1: take the table from here instead of table_g / w_maps
+};
+
 template <bool PACKED>
 __global__ void __launch_bounds__(PairCfg<PACKED>::kThreads, 1)
-gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __restrict__ table_g, const CUtensorMap* __restrict__ w_maps,
-                    int* status_word) {
+gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __restrict__ table_g, const CUtensorMap* __restrict__ w_maps_g,
+                    int* status_word, const __grid_constant__ PairInline inl) {
     constexpr int P_STAGES = PairCfg<PACKED>::kStages;
     constexpr uint32_t P_STAGE_BYTES = PairCfg<PACKED>::kStageBytes;
     constexpr int kThreadsAll = PairCfg<PACKED>::kThreads;
@@ -431,8 +440,16 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
     const uint32_t rank = cluster_ctarank();
     const bool leader = rank == 0;
     const int pair = (int)blockIdx.x >> 1, n_pairs = (int)gridDim.x >> 1;
-    for (int o = threadIdx.x * 16; o < (int)kGroupTableBytes; o += kThreadsAll * 16)
-        *reinterpret_cast<uint4*>(table_s + o) = *reinterpret_cast<const uint4*>(table_g + o);
+    const CUtensorMap* w_maps = inl.use ? &inl.w_map : w_maps_g;
+    if (inl.use) {
+        if (threadIdx.x == 0) {
+            *reinterpret_cast<GemmGroupHeader*>(table_s) = inl.hdr;
+            *reinterpret_cast<GemmProblem*>(table_s + sizeof(GemmGroupHeader)) = inl.prob;
+        }
+    } else {
+        for (int o = threadIdx.x * 16; o < (int)kGroupTableBytes; o += kThreadsAll * 16)
+            *reinterpret_cast<uint4*>(table_s + o) = *reinterpret_cast<const uint4*>(table_g + o);
+    }
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < P_STAGES; ++s) {
@@ -515,7 +532,10 @@ gemm_i8_pair_kernel(const __grid_constant__ CUtensorMap map, const uint8_t* __re
                     const uint32_t sa = smem_u32(smem + (size_t)stage * P_STAGE_BYTES);
                     if constexpr (PACKED) {
                         if (leader) mbar_expect_tx(fb, 2 * P_HALF_BYTES);  // the token rows of both CTAs
-                        tma_load_2d_pair(sa, &map, 0, a_row + kb * 128, fb);
+                        // tokens: a tile image (already swizzled, the map has rows of 128 bytes) or, for a single matmul on
+                        // row-major activations, a 128-row x 128-byte box of the [M][K] matrix through a swizzling map
+                        if (hdr.a_row_major) tma_load_2d_pair(sa, &map, kb * BK, mt * 256 + (int)rank * 128, fb);
+                        else tma_load_2d_pair(sa, &map, 0, a_row + kb * 128, fb);
                         // this CTA's 128 weight rows x 128 columns as packed codes: 8 row blocks x 16 rows x 32 bytes of the
                         // packed matrix (half of the 16 x 256 tile kb / 2 of each row block)
                         const uint32_t pb = smem_u32(pfull_bar + stage);
@@ -713,7 +733,7 @@ bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows)
 
 size_t gemm_codes_bytes(int N, int K) { return (size_t)((N + BN - 1) / BN) * BN * K; }  // whole 256-row tiles
 size_t gemm_a_tiles_bytes(int M, int K) { return (size_t)((M + 255) / 256) * 256 * K; }  // whole pairs of 128-row tiles
-size_t gemm_scratch_bytes(int N, int K) { return align_up(gemm_codes_bytes(N, K), 256) + align_up(kGroupTableBytes, 256); }
+size_t gemm_scratch_bytes(int N, int K) { return align_up(gemm_codes_bytes(N, K), 256) + align_up(kGroupTableDevBytes, 256); }
 
 // The whole region [base, base + bytes) as a matrix of 128-byte rows, box = 128 rows, no swizzle: a tile image (stored
 // swizzled) is copied as it is.
@@ -778,7 +798,7 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     GemmGroupHeader* hdr = reinterpret_cast<GemmGroupHeader*>(host);
     GemmProblem* tab = reinterpret_cast<GemmProblem*>(host + sizeof(GemmGroupHeader));
     // CTA pairs (256 x 256 tiles) when the operands are tile images inside one mapped region and the SMs pair up
-    const bool pairs = a_tiled && region_base != nullptr && (sm_count % 2) == 0;
+    const bool pairs = (sm_count % 2) == 0 && ((a_tiled && region_base != nullptr) || (!a_tiled && packed != nullptr));
     const int tile_m = pairs ? 256 : BM;
     int tiles = 0, n_tiles = 0;
     for (int i = 0; i < count; ++i) {
@@ -796,15 +816,25 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     const bool packed_mode = pairs && packed != nullptr;
     hdr->ready = (pairs && !packed_mode) ? ready : nullptr;
     hdr->a_ready = pairs ? a_ready : nullptr;
+    hdr->a_row_major = (pairs && !a_tiled) ? 1 : 0;
     // griddepcontrol.wait in the kernel: only where the launch before it is the quantiser and no token-tile counters follow it
     const bool dependent = pairs && (hdr->ready != nullptr || hdr->a_ready != nullptr);
     hdr->wait_primary = (dependent && hdr->a_ready == nullptr && wait_primary) ? 1 : 0;
-    if (cudaMemcpyAsync(table_dev, host, kGroupTableBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    // a single matmul on packed weights carries its table in the kernel parameters: nothing to upload
+    const bool inline_table = packed_mode && count == 1;
+    PairInline inl;
+    memset(&inl, 0, sizeof(inl));
+    if (inline_table) {
+        inl.hdr = *hdr;
+        inl.prob = tab[0];
+        inl.use = 1;
+        if (!make_map_packed(&inl.w_map, packed[0], probs[0].N, probs[0].K)) return BITLINEAR_ERR_CUDA;
+    } else if (cudaMemcpyAsync(table_dev, host, kGroupTableBytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;
     }
     CUtensorMap* w_maps_dev = reinterpret_cast<CUtensorMap*>(table_dev + kGroupMapsOffset);
-    if (packed_mode) {
+    if (packed_mode && !inline_table) {
         alignas(64) CUtensorMap maps[kMaxGroup];
         for (int i = 0; i < count; ++i)
             if (!make_map_packed(&maps[i], packed[i], probs[i].N, probs[i].K)) return BITLINEAR_ERR_CUDA;
@@ -820,7 +850,8 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
     CUtensorMap map_a;
     memset(&map_a, 0, sizeof(map_a));
     if (pairs) {
-        if (!make_map_rows128(&map_a, region_base, region_bytes)) return BITLINEAR_ERR_CUDA;
+        if (a_tiled ? !make_map_rows128(&map_a, region_base, region_bytes) : !make_map(&map_a, xq_row_major, probs[0].M, probs[0].K, 128))
+            return BITLINEAR_ERR_CUDA;
         int n_pairs = tiles < sm_count / 2 ? tiles : sm_count / 2;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(2 * n_pairs));
@@ -838,9 +869,9 @@ int gemm_launch(GemmProblem* probs, int count, bool a_tiled, const int8_t* xq_ro
         cfg.attrs = attr;
         cfg.numAttrs = dependent ? 2 : 1;
         const cudaError_t e = packed_mode ? cudaLaunchKernelEx(&cfg, gemm_i8_pair_kernel<true>, map_a, (const uint8_t*)table_dev,
-                                                               (const CUtensorMap*)w_maps_dev, device_status_word())
+                                                               (const CUtensorMap*)w_maps_dev, device_status_word(), inl)
                                           : cudaLaunchKernelEx(&cfg, gemm_i8_pair_kernel<false>, map_a, (const uint8_t*)table_dev,
-                                                               (const CUtensorMap*)w_maps_dev, device_status_word());
+                                                               (const CUtensorMap*)w_maps_dev, device_status_word(), inl);
         if (e != cudaSuccess) cudaGetLastError();
         return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
     }
@@ -875,6 +906,22 @@ int gemm_tcgen05(const int8_t* xq, const float* d, const int32_t* xsum, const ui
     p.M = M; p.N = N; p.K = K; p.y_dtype = y_dtype;
     uint8_t* table_dev = const_cast<uint8_t*>(scratch) + align_up(gemm_codes_bytes(N, K), 256);
     return gemm_launch(&p, 1, false, xq, table_dev, st);
+}
+
+// The same through the CTA-pair kernel that reads the packed weights themselves (no code tiles): `table_dev` holds
+// kGroupTableDevBytes.  Returns BITLINEAR_ERR_ARCH-free status; the caller checks pairs_available() first.
+int gemm_tcgen05_packed(const int8_t* xq, const float* d, const int32_t* xsum, const void* packed, const float* s_w, int M,
+                        int N, int K, void* y, int y_dtype, int32_t* acc_out, uint8_t* table_dev, cudaStream_t st) {
+    GemmProblem p = {};
+    p.d = d; p.xsum = xsum; p.s_w = s_w; p.y = y; p.acc_out = acc_out;
+    p.M = M; p.N = N; p.K = K; p.y_dtype = y_dtype;
+    const void* packed_ptrs[1] = {packed};
+    return gemm_launch(&p, 1, false, xq, table_dev, st, nullptr, 0, nullptr, nullptr, nullptr, false, nullptr, packed_ptrs);
+}
+
+bool gemm_pairs_available() {
+    int sm_count = 0;
+    return device_sm_count(&sm_count) == BITLINEAR_OK && (sm_count % 2) == 0;
 }
 
 }  // namespace bitlinear
