@@ -38,9 +38,13 @@ namespace {
 constexpr int kRows = 128;        // weight rows per work item = tensor-memory lanes = UMMA M
 constexpr int kItemRb = kRows / kTileRows;
 constexpr int kTok = 16;          // tokens per matmul, padded (UMMA N)
-constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1024 columns)
-constexpr int kSlots = 4;         // ring slots of packed weights + token images
-constexpr int kLanes = 4;         // pipelines: unpack group + tensor-memory stage + MMA issuer + partial accumulator
+constexpr int kStepTiles = 4;     // 16x256 tiles per row block per ring slot (1024 columns): one per pipeline
+constexpr int kSlots = 4;         // ring slots of packed weights + token images (48 KiB each)
+constexpr int kLanes = 4;         // pipelines: unpack group + tensor-memory stage(s) + MMA issuer + partial accumulator
+// Code stages per pipeline.  Measured with three pipelines of two private stages each (the group expands step s + 1 while
+// the MMAs of step s run; 3 tiles per slot, 5 slots): 155.5 / 168.8 us per 521 MB step at 4 / 16 tokens, against
+// 140.8 / 156.2 us on the same GPU for four pipelines of one stage: the stage is not what the roles wait for.
+constexpr int kAStages = 1;
 constexpr int kUnpackWarps = 4 * kLanes;  // groups of four (one warp per tensor-memory lane quarter)
 constexpr int kProdWarps = 3, kCopiesPerWarp = 3;  // 8 packed row blocks + the token images
 constexpr int kFirstMmaWarp = kProdWarps + kUnpackWarps;
@@ -50,8 +54,8 @@ constexpr uint32_t kPackedSlot = kItemRb * kStepTiles * kTileBytes;  // 32 KiB o
 constexpr uint32_t kXSlot = kStepTiles * 2 * kTok * 128;             // 16 KiB: 8 k-blocks of 16 x 128 token images
 constexpr uint32_t kAStageCols = kTileCols / 4;                      // 64 columns: 256 codes per row, 4 per column
 constexpr uint32_t kAColBase = 2 * kLanes * kTok;                    // after the two buffers of partial accumulators
-constexpr uint32_t kTmemCols = 512;                                  // power of two >= kAColBase + kLanes * 64
-static_assert(kAColBase + kLanes * kAStageCols <= kTmemCols, "tensor memory");
+constexpr uint32_t kTmemCols = 512;                                  // power of two >= kAColBase + kLanes * kAStages * 64
+static_assert(kAColBase + kLanes * kAStages * kAStageCols <= kTmemCols, "tensor memory");
 constexpr int kItemCap = 192;     // work items and matmul descriptors of the CTA kept in shared memory; what does
 constexpr int kProbCap = 48;      // not fit is read from global memory where it is needed (slow, still correct)
 
@@ -101,7 +105,7 @@ struct alignas(16) SProb {
     void* y;
     int M, N, K, y_dtype;
 };
-constexpr int kNumBars = 3 * kSlots + 2 * kLanes + 4;               // pfull, pempty, xempty; afull, aempty; tfull, tempty
+constexpr int kNumBars = 3 * kSlots + 2 * kLanes * kAStages + 4;    // pfull, pempty, xempty; afull, aempty; tfull, tempty
 constexpr size_t kBarBytes = 256;                                    // barriers, tensor-memory base, abort flag
 static_assert(kNumBars * 8 + 8 <= kBarBytes, "barrier block");
 constexpr size_t kMmaSmem = 1024 + kSlots * (size_t)(kPackedSlot + kXSlot) + kBarBytes + kItemCap * sizeof(int2) + kProbCap * sizeof(SProb);
@@ -219,8 +223,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
     const uint32_t p_s = x_s + kSlots * kXSlot;     // [kSlots] packed weights
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + kSlots * (size_t)(kXSlot + kPackedSlot));
     const uint32_t pfull = smem_u32(bars), pempty = pfull + 8 * kSlots, xempty = pempty + 8 * kSlots;
-    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kLanes;
-    const uint32_t tfull = aempty + 8 * kLanes, tempty = tfull + 16;
+    const uint32_t afull = xempty + 8 * kSlots, aempty = afull + 8 * kLanes * kAStages;  // [pipeline][stage]
+    const uint32_t tfull = aempty + 8 * kLanes * kAStages, tempty = tfull + 16;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
     int2* items_s = reinterpret_cast<int2*>(reinterpret_cast<uint8_t*>(bars) + kBarBytes);
@@ -238,7 +242,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
             mbar_init(pempty + 8 * b, kUnpackWarps);
             mbar_init(xempty + 8 * b, kLanes);
         }
-        for (int b = 0; b < kLanes; ++b) {
+        for (int b = 0; b < kLanes * kAStages; ++b) {
             mbar_init(afull + 8 * b, 4);
             mbar_init(aempty + 8 * b, 1);
         }
@@ -311,7 +315,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         // the 256 codes of row r16 = 8h + g of a 16 x 256 tile are 64 consecutive packed bytes at 512h + 64g
         const uint32_t row_off = (uint32_t)rbl * (kStepTiles * kTileBytes) + (uint32_t)(r16 >> 3) * 512u + (uint32_t)(r16 & 7) * 64u +
                                  (uint32_t)g * kTileBytes;
-        const uint32_t a_dst = tmem_base + ((uint32_t)(quarter * 32) << 16) + kAColBase + (uint32_t)g * kAStageCols;
+        const uint32_t a_dst0 = tmem_base + ((uint32_t)(quarter * 32) << 16) + kAColBase + (uint32_t)g * kAStages * kAStageCols;
         uint32_t sc_idx = 0, n_own = 0;
         bool ok = true;
         for (int it = item_lo; ok && it < item_hi; ++it) {
@@ -339,7 +343,10 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     // pipeline's previous step are still reading it), the second half after the first is stored.
                     uint32_t v[32];
                     expand_codes(pw[0], pw[1], v);
-                    if (!mbar_wait(aempty + 8 * g, (n_own & 1u) ^ 1u, abort_flag)) { ok = false; break; }
+                    // the pipeline's steps alternate between its two code stages: stage st is free once the MMAs of the
+                    // step before last have retired
+                    const uint32_t st = n_own % kAStages, a_dst = a_dst0 + st * kAStageCols;
+                    if (!mbar_wait(aempty + 8 * (g * kAStages + st), ((n_own / kAStages) & 1u) ^ 1u, abort_flag)) { ok = false; break; }
                     tc_fence_after();
                     tmem_st_32x32(a_dst, v);
                     expand_codes(pw[2], pw[3], v);
@@ -347,7 +354,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     tmem_st_wait();
                     tc_fence_before();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(afull + 8 * g);
+                    if (lane == 0) mbar_arrive(afull + 8 * (g * kAStages + st));
                     ++n_own;
                 }
                 __syncwarp();
@@ -358,7 +365,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
         // ------------------------------------------------------------------ MMA issuers: one pipeline each
         if (lane == 0) {
             const int g = warp - kFirstMmaWarp;
-            const uint32_t a_tmem = tmem_base + kAColBase + (uint32_t)g * kAStageCols;
+            const uint32_t a_tmem0 = tmem_base + kAColBase + (uint32_t)g * kAStages * kAStageCols;
             // token images of tile g of a slot: k-block kb at 2 KiB * (2g + kb), 32-byte slice k inside it
             const uint64_t x_desc = smem_desc_sw128(x_s) + (uint64_t)((g * 2 * kTok * 128) >> 4);
             uint32_t sc_idx = 0, n_own = 0, it_idx = 0;
@@ -374,14 +381,15 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                     // every issuer waits for every slot, also one in which it has no step (see the unpack warps)
                     if (!mbar_wait(pfull + 8 * slot, phase, abort_flag)) { ok = false; break; }
                     if (g < k_tiles - t0) {
-                        if (!mbar_wait(afull + 8 * g, n_own & 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t st = n_own % kAStages, a_tmem = a_tmem0 + st * kAStageCols;
+                        if (!mbar_wait(afull + 8 * (g * kAStages + st), (n_own / kAStages) & 1u, abort_flag)) { ok = false; break; }
                         tc_fence_after();
                         const uint64_t b_desc = x_desc + (uint64_t)(slot * (kXSlot >> 4));
 #pragma unroll
                         for (int s = 0; s < 8; ++s)
                             umma_i8_ts(d_tmem, a_tmem + 8u * s, b_desc + (uint64_t)((s >> 2) * ((kTok * 128) >> 4) + 2 * (s & 3)),
                                        kIdesc, (uint32_t)(t0 != 0 || s != 0));
-                        umma_commit(aempty + 8 * g);  // the codes may be overwritten once these MMAs retire
+                        umma_commit(aempty + 8 * (g * kAStages + st));  // the stage may be overwritten once these MMAs retire
                         ++n_own;
                     }
                     umma_commit(xempty + 8 * slot);  // counts kLanes arrivals: every issuer is done with the slot
