@@ -386,6 +386,11 @@ def bitlinear_forward_static(x, gain, packed, s_w, N: int, rms_eps: float = 1e-5
     _dev(packed, torch.uint8, "packed")
     _dev(s_w, torch.float32, "s_w")
     M, K = x.shape
+    if out is not None:
+        if not out.is_cuda or not out.is_contiguous() or out.dtype not in (torch.float32, torch.bfloat16):
+            raise TypeError("out must be a contiguous CUDA tensor of float32 or bfloat16")
+        if tuple(out.shape) != (M, N):
+            raise ValueError(f"out must have shape ({M}, {N})")
     y = out if out is not None else torch.empty(M, N, dtype=y_dtype, device=x.device)
     rc = lib().bitlinear_forward_static(_ptr(x), _ptr(gain), rms_eps, _ptr(packed), _ptr(s_w), M, N, K, _ptr(y),
                                         _ydt(y.dtype), _stream())

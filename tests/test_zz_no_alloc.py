@@ -30,12 +30,18 @@ def test_static_forward_matches_workspace_forward_on_two_calls_in_a_row():
         gain = wl.gain_random(K, 7300 + i).to(DEV)
         want = bl.bitlinear_forward(x, gain, packed, s_w, N, wl.RMS_EPS, y_dtype=ydt)
         out = torch.full((M, N), float("nan"), dtype=ydt, device=DEV)  # the caller owns the output, as always
+        torch.cuda.synchronize()
+        held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         got = bl.bitlinear_forward_static(x, gain, packed, s_w, N, wl.RMS_EPS, out=out)
         torch.cuda.synchronize()
+        # the call took no device memory, neither from torch's pool nor from the driver
+        assert torch.cuda.memory_allocated() == held and torch.cuda.mem_get_info()[0] == free
+        assert got is out
         g, w = got.float().cpu().numpy().astype(np.float64), want.float().cpu().numpy().astype(np.float64)
         assert np.all(np.isfinite(g))
         tol = 1e-6 if ydt == torch.float32 else 2.0 ** -7  # fp32: the suite's relative bound; bf16: one ulp
         assert np.all(np.abs(g - w) <= tol * np.abs(w))
+        assert torch.equal(got, want)  # in fact the same kernels run: the results are identical
     assert bl.bitlinear_poll_status() == 0
 
 
@@ -50,3 +56,14 @@ def test_static_forward_refuses_sizes_beyond_its_array():
     assert lib.bitlinear_forward_static(fake, None, 1e-5, fake, fake, 1, 2560, 2560, fake, 7, None) == 5
     assert lib.bitlinear_forward_static(None, None, 1e-5, fake, fake, 1, 2560, 2560, fake, 0, None) == 1
     assert lib.bitlinear_forward_static(fake, None, 1e-5, fake, fake, 0, 2560, 2560, fake, 0, None) == 0
+
+
+@pytest.mark.gpu
+def test_static_forward_binding_checks_the_output_tensor():
+    N, K = 256, 512
+    packed, s_w = bl.bitlinear_pack_weights(wl.latent_weights(N, K, 1).to(DEV))
+    x = wl.activations_normal(2, K, 2).to(DEV)
+    for bad in (torch.empty(2, N + 16, device=DEV), torch.empty(3, N, device=DEV), torch.empty(2, N),
+                torch.empty(2, 2 * N, device=DEV)[:, ::2], torch.empty(2, N, dtype=torch.float16, device=DEV)):
+        with pytest.raises((TypeError, ValueError)):
+            bl.bitlinear_forward_static(x, None, packed, s_w, N, out=bad)
