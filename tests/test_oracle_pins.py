@@ -531,3 +531,77 @@ def test_fused_glue_quantisers_are_glue_then_quantiser():
     ref = oracle.rmsnorm_quant(oracle.glue_residual(h, up), None, 1e-5)
     assert np.array_equal(res["q"], ref["q"]) and np.array_equal(res["d"], ref["d"])
     assert np.array_equal(oracle.bf16_to_f32(res["x"]), oracle.bf16_to_f32(oracle.f32_to_bf16((oracle.bf16_to_f32(h) + up).astype(np.float32))))
+
+
+# --------------------------------------------------------------------------- the rest of a decode step
+
+
+def test_rope_pins():
+    from oracle import decode_step as ds
+    rng = np.random.default_rng(21)
+    hd, nh = 8, 3
+    x = rng.standard_normal((4, nh * hd))
+    pos = np.array([0, 1, 7, 1000])
+    y = ds.rope(x, pos, nh, hd, base=10000.0)
+    assert np.array_equal(y[0], x[0])  # position 0 is the identity
+    # a rotation: the norm of every pair (i, i + hd/2), hence of every head, is kept
+    assert np.allclose((y.reshape(4, nh, hd) ** 2).sum(-1), (x.reshape(4, nh, hd) ** 2).sum(-1), rtol=1e-12)
+    # hand case: head_dim 2 has one pair and angle = pos (frequency base^0 = 1): (1, 0) at pos = pi/2 -> (0, 1)
+    y2 = ds.rope(np.array([[1.0, 0.0]]), np.array([np.pi / 2]), 1, 2, base=10000.0)
+    assert np.allclose(y2, [[0.0, 1.0]], atol=1e-15)
+    # head_dim 4, base 100: frequencies 1 and 100^(-1/2) = 0.1; pairs (0,2) and (1,3)
+    y4 = ds.rope(np.array([[1.0, 1.0, 0.0, 0.0]]), np.array([2.0]), 1, 4, base=100.0)
+    assert np.allclose(y4, [[np.cos(2.0), np.cos(0.2), np.sin(2.0), np.sin(0.2)]], atol=1e-15)
+    # the reason for the scheme: the product of a rotated query and a rotated key depends on the distance only
+    q, k = rng.standard_normal((1, hd)), rng.standard_normal((1, hd))
+    d1 = ds.rope(q, [5], 1, hd) @ ds.rope(k, [3], 1, hd).T
+    d2 = ds.rope(q, [105], 1, hd) @ ds.rope(k, [103], 1, hd).T
+    assert np.allclose(d1, d2, rtol=1e-9)
+
+
+def test_attention_decode_pins():
+    from oracle import decode_step as ds
+    rng = np.random.default_rng(22)
+    n_q, n_kv, hd, T = 4, 2, 8, 6
+    f = lambda a: oracle.f32_to_bf16(np.asarray(a, np.float32))  # noqa: E731
+    k = rng.standard_normal((T, n_kv * hd)).astype(np.float32)
+    v = rng.standard_normal((T, n_kv * hd)).astype(np.float32)
+    vb = oracle.bf16_to_f32(f(v)).astype(np.float64).reshape(T, n_kv, hd)
+    # a zero query scores every position alike: the output is the mean of the first `length` values of the KV head
+    out = ds.attention_decode(f(np.zeros(n_q * hd)), f(k), f(v), 5, n_q, n_kv, hd).reshape(n_q, hd)
+    for h in range(n_q):
+        assert np.allclose(out[h], vb[:5, h // 2].mean(axis=0), rtol=1e-12)
+    # length 1: the output is the first value row, whatever the query
+    out = ds.attention_decode(f(rng.standard_normal(n_q * hd)), f(k), f(v), 1, n_q, n_kv, hd).reshape(n_q, hd)
+    assert np.allclose(out[3], vb[0, 1]) and np.allclose(out[0], vb[0, 0])
+    # a query 64 times a key direction makes that position win: keys are unit vectors e_t, query = 64 e_2 for head 0
+    kk = np.zeros((T, n_kv * hd), np.float32)
+    for t in range(T):
+        kk[t, t] = 1.0       # KV head 0
+        kk[t, hd + t] = 1.0  # KV head 1
+    q = np.zeros(n_q * hd, np.float32)
+    q[2] = 64.0              # query head 0 -> KV head 0, position 2
+    q[3 * hd + 4] = 64.0     # query head 3 -> KV head 1, position 4
+    out = ds.attention_decode(f(q), f(kk), f(v), T, n_q, n_kv, hd).reshape(n_q, hd)
+    w = np.exp(64.0 / np.sqrt(hd))  # weight of the winner against weight 1 of the five others
+    assert np.allclose(out[0], (w * vb[2, 0] + (vb[:, 0].sum(0) - vb[2, 0])) / (w + 5), rtol=1e-12)
+    assert np.allclose(out[3], (w * vb[4, 1] + (vb[:, 1].sum(0) - vb[4, 1])) / (w + 5), rtol=1e-12)
+    # heads 1 and 2 have a zero query: plain means
+    assert np.allclose(out[1], vb[:, 0].mean(0)) and np.allclose(out[2], vb[:, 1].mean(0))
+
+
+def test_lm_head_and_embedding_pins():
+    from oracle import decode_step as ds
+    rng = np.random.default_rng(23)
+    V, K = 40, 16
+    table = oracle.f32_to_bf16(rng.standard_normal((V, K)).astype(np.float32))
+    ids = np.array([3, 39, 0, 3])
+    rows = ds.embed(ids, table)
+    assert np.array_equal(rows, table[[3, 39, 0, 3]])
+    # logits of a one-hot input are a column of the table; of an embedding row, its products with every row
+    onehot = np.zeros((1, K), np.float32)
+    onehot[0, 5] = 2.0
+    logits = ds.lm_head(oracle.f32_to_bf16(onehot), table)
+    assert np.array_equal(logits[0], 2.0 * oracle.bf16_to_f32(table)[:, 5].astype(np.float64))
+    e = oracle.bf16_to_f32(table).astype(np.float64)
+    assert np.allclose(ds.lm_head(rows, table), e[[3, 39, 0, 3]] @ e.T, rtol=1e-14)
