@@ -226,10 +226,12 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  * cores, with the codes unpacked in registers and handed over in tensor memory).  Problems of 17 to
  * 96 tokens (K <= 8192) are cut into 16-token problems for that same decode kernel: streaming the
  * packed weights once per 16 tokens is measured faster there than a tensor-core tile that is mostly
- * padding.  Longer problems (prefill; N must be a multiple of 128) take three
- * launches together: the quantiser, the expansion of the packed weights into tensor-core tile
- * images, and one persistent tcgen05 kernel that runs every tile of every matmul; problems that
- * name the same x, gain, rms_eps, M and K (q/k/v or gate/up of a layer) share one quantised copy.
+ * padding.  Longer problems (prefill; N must be a multiple of 128) take two launches together: the
+ * quantiser and one persistent tcgen05 kernel that runs every tile of every matmul and expands the
+ * packed weights into tensor-core tile images in shared memory as it goes (on a device with an odd
+ * number of SMs, where CTA pairs cannot cover the chip, a separate expansion launch into ws comes
+ * first); problems that name the same x, gain, rms_eps, M and K (q/k/v or gate/up of a layer) share
+ * one quantised copy.
  * All kinds may be mixed in one call.
  * Weights in the dense layout (w_format = BITLINEAR_WEIGHTS_DENSE5, Table 1 / Section 5.1) are accepted for
  * problems of at most 16 tokens; all such problems of a call must use the same layout.  Their kernel is the
@@ -391,6 +393,40 @@ int bitlinear_forward_static(const void* x_bf16, const void* gain, float rms_eps
  * its workspace was no longer the one it had uploaded (the call then computed nothing).
  * Synchronises `stream` first. */
 int bitlinear_poll_status(void* stream);
+
+/*
+ * The rest of a decode step around the BitLinear layers.  The paper names these parts without formulas (Section 2:
+ * rotary position embeddings; a Transformer decoder; a tokenizer with 128,256 entries, hence an embedding table and an
+ * output head of that many rows); the definitions taken are the textbook ones, stated here.  None is a BitLinear: they
+ * exist so that a whole decoded token can be run and timed on the device.
+ *
+ * bitlinear_rope_kv: rotary embedding of the q and k projections and append of k, v to the cache.
+ *   q [M][n_q*D], k, v [M][n_kv*D] fp32 (BitLinear outputs); positions [M] int32 (device); seq_ids [M] int32 (device)
+ *   or NULL (one sequence).  Coordinate i of a head is paired with i + D/2, angle = position * rope_base^(-2i/D):
+ *   (x_i, x_j) -> (x_i cos - x_j sin, x_j cos + x_i sin); angles in fp64, rotation in fp32, results rounded to bf16.
+ *   q_out bf16 [M][n_q*D]; caches bf16 [n_seq][t_max][n_kv*D]: row positions[m] of sequence seq_ids[m] receives the
+ *   rotated k and the unrotated v (positions outside 0 .. t_max-1 are not stored).  D a multiple of 8.
+ * bitlinear_attention_decode: one query token per row against the first lengths[m] cache rows of its sequence.
+ *   Query head h reads key/value head h / (n_q / n_kv); scores q.k / sqrt(D), softmax over the rows, weighted sum of
+ *   the values, fp32 arithmetic, bf16 output [M][n_q*D] (the input of the o projection; zeros for a length <= 0,
+ *   lengths above t_max are taken as t_max).  D = 64 or 128, n_q / n_kv <= 8, t_max <= 2^22, all pointers 16-byte
+ *   aligned; ws (device, 16-byte aligned, contents need not survive the call) at least
+ *   bitlinear_attention_workspace_bytes(...) bytes (0 for unsupported sizes): one partial result per 64 cache rows.
+ *   A copy that does not land within the wait limit ends the call's kernels and sets BITLINEAR_ERR_TIMEOUT in the
+ *   status word (bitlinear_poll_status).
+ * bitlinear_lm_head: logits[m][v] = sum_k x[m][k] * table[v][k], x bf16 [M][K] (M <= 16), table bf16 [V][K], fp32
+ *   accumulation and output [M][V].  The table is streamed once per call.
+ * bitlinear_embed: out[m] = table[ids[m]] (bf16 rows; ids outside 0 .. V-1 are clamped).
+ */
+int bitlinear_rope_kv(const float* q, const float* k, const float* v, const int32_t* positions, const int32_t* seq_ids, int M,
+                      int n_q_heads, int n_kv_heads, int head_dim, float rope_base, void* q_out_bf16, void* k_cache_bf16,
+                      void* v_cache_bf16, int t_max, void* stream);
+size_t bitlinear_attention_workspace_bytes(int M, int n_q_heads, int n_kv_heads, int head_dim, int t_max);
+int bitlinear_attention_decode(const void* q_bf16, const void* k_cache_bf16, const void* v_cache_bf16, const int32_t* lengths,
+                               const int32_t* seq_ids, int M, int n_q_heads, int n_kv_heads, int head_dim, int t_max,
+                               void* out_bf16, void* ws, size_t ws_bytes, void* stream);
+int bitlinear_lm_head(const void* x_bf16, const void* table_bf16, int M, int V, int K, float* logits, void* stream);
+int bitlinear_embed(const int32_t* ids, const void* table_bf16, int M, int V, int K, void* out_bf16, void* stream);
 
 /*
  * Self-test of the bounded device-side waits (no counterpart in the paper: every kernel of this library waits on

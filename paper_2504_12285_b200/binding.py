@@ -47,6 +47,13 @@ _SIGNATURES = {
                                    _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_rope_kv": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_float,
+                                   _c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]),
+    "bitlinear_attention_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int, _c_int]),
+    "bitlinear_attention_decode": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int,
+                                            _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_lm_head": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_void_p]),
+    "bitlinear_embed": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
     "bitlinear_probe_int8_mma_rate": (_c_int, [_c_int, ctypes.POINTER(ctypes.c_double), _c_void_p]),
     "bitlinear_selftest_wait_timeout": (_c_int, [ctypes.c_uint, _c_void_p]),
@@ -475,6 +482,66 @@ def bitlinear_forward_batch_host(batch: ProblemBatch, x_host: torch.Tensor, x_de
                                             BATCH_REUSE_PLAN if reuse_plan else 0, _ptr(x_host), _ptr(x_dev), xb,
                                             _ptr(y_dev), _ptr(y_host), yb, _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_forward_batch_host")
+
+
+def bitlinear_rope_kv(q, k, v, positions, k_cache, v_cache, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                      rope_base: float = 500000.0, seq_ids=None, q_out=None):
+    """Rotate q, k (fp32 [M, heads * D]) at `positions` (int32 [M]); q -> bf16 (returned), k / v appended to the bf16
+    caches [n_seq, t_max, n_kv * D] at those positions."""
+    _dev(q, torch.float32, "q"), _dev(k, torch.float32, "k"), _dev(v, torch.float32, "v")
+    _dev(positions, torch.int32, "positions"), _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache")
+    if seq_ids is not None:
+        _dev(seq_ids, torch.int32, "seq_ids")
+    M = q.shape[0]
+    if q_out is None:
+        q_out = torch.empty(M, n_q_heads * head_dim, dtype=torch.bfloat16, device=q.device)
+    rc = lib().bitlinear_rope_kv(_ptr(q), _ptr(k), _ptr(v), _ptr(positions), _ptr(seq_ids), M, n_q_heads, n_kv_heads, head_dim,
+                                 rope_base, _ptr(q_out), _ptr(k_cache), _ptr(v_cache), k_cache.shape[-2], _stream())
+    _check(rc, "bitlinear_rope_kv")
+    return q_out
+
+
+def bitlinear_attention_workspace_bytes(M: int, n_q_heads: int, n_kv_heads: int, head_dim: int, t_max: int) -> int:
+    return int(lib().bitlinear_attention_workspace_bytes(M, n_q_heads, n_kv_heads, head_dim, t_max))
+
+
+def bitlinear_attention_decode(q, k_cache, v_cache, lengths, n_q_heads: int, n_kv_heads: int, head_dim: int, seq_ids=None,
+                               out=None, ws=None):
+    """q bf16 [M, n_q * D] against the first lengths[m] rows of its sequence's bf16 cache -> bf16 [M, n_q * D]."""
+    _dev(q, torch.bfloat16, "q"), _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache")
+    _dev(lengths, torch.int32, "lengths")
+    if seq_ids is not None:
+        _dev(seq_ids, torch.int32, "seq_ids")
+    M, t_max = q.shape[0], k_cache.shape[-2]
+    if out is None:
+        out = torch.empty(M, n_q_heads * head_dim, dtype=torch.bfloat16, device=q.device)
+    if ws is None:
+        ws = _workspace(bitlinear_attention_workspace_bytes(M, n_q_heads, n_kv_heads, head_dim, t_max), q.device)
+    rc = lib().bitlinear_attention_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(lengths), _ptr(seq_ids), M, n_q_heads,
+                                          n_kv_heads, head_dim, t_max, _ptr(out), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_attention_decode")
+    return out
+
+
+def bitlinear_lm_head(x, table, out=None):
+    """x bf16 [M, K] (M <= 16), table bf16 [V, K] -> logits fp32 [M, V]."""
+    _dev(x, torch.bfloat16, "x"), _dev(table, torch.bfloat16, "table")
+    M, K = x.shape
+    V = table.shape[0]
+    if out is None:
+        out = torch.empty(M, V, dtype=torch.float32, device=x.device)
+    _check(lib().bitlinear_lm_head(_ptr(x), _ptr(table), M, V, K, _ptr(out), _stream()), "bitlinear_lm_head")
+    return out
+
+
+def bitlinear_embed(ids, table, out=None):
+    """ids int32 [M], table bf16 [V, K] -> bf16 [M, K]."""
+    _dev(ids, torch.int32, "ids"), _dev(table, torch.bfloat16, "table")
+    M, (V, K) = ids.shape[0], table.shape
+    if out is None:
+        out = torch.empty(M, K, dtype=torch.bfloat16, device=table.device)
+    _check(lib().bitlinear_embed(_ptr(ids), _ptr(table), M, V, K, _ptr(out), _stream()), "bitlinear_embed")
+    return out
 
 
 def bitlinear_selftest_wait_timeout(limit_us: int = 1000) -> None:

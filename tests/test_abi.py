@@ -108,9 +108,12 @@ def test_batch_entry_point_host_checks():
     assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 8, addr, need, None) == 5    # unknown flag
     arr[1].M = 16                      # several tokens: every problem of the call gets 16-row token images of 16 * K bytes
     assert lib.bitlinear_batch_workspace_bytes(ctypes.addressof(arr), 2) >= 16 * (256 + 512)
-    arr[1].M = 17                                                                               # decode sizes only
+    arr[1].M = 17                      # 17 to 96 tokens are cut into 16-token problems: two 16-row images for this one
+    assert lib.bitlinear_batch_workspace_bytes(ctypes.addressof(arr), 2) >= 16 * 256 + 32 * 512
+    arr[1].w_format = 1                                                                         # dense layout: decode sizes only
     assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, addr, 1 << 20, None) == 2
     assert lib.bitlinear_batch_workspace_bytes(ctypes.addressof(arr), 2) == 0
+    arr[1].w_format = 0
     arr[1].M = 4
     arr[1].packed = None
     assert lib.bitlinear_forward_batch(ctypes.addressof(arr), 2, 0, addr, 1 << 20, None) == 1

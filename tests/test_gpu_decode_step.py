@@ -1,0 +1,143 @@
+"""The parts of a decode step that are not BitLinear (rotary embedding + cache append, grouped-query decode attention,
+output head, embedding) against the fp64 oracle.  These are floating-point kernels whose summation order differs from
+the oracle's, so the bounds are tolerances, derived below from the arithmetic."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import decode_step as ds
+from paper_2504_12285_b200 import binding as bl
+from paper_2504_12285_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def bits(t):
+    return wl.bf16_bits(t.cpu())
+
+
+def bf(a):
+    return oracle.bf16_to_f32(a).astype(np.float64)
+
+
+def randn(shape, seed, scale=1.0):
+    return (torch.randn(*shape, generator=torch.Generator().manual_seed(seed), dtype=torch.float32) * scale).contiguous()
+
+
+@pytest.mark.parametrize("M,n_q,n_kv,hd", [(1, 20, 5, 128), (7, 4, 2, 64), (16, 20, 5, 128)])
+def test_rope_and_cache_append(M, n_q, n_kv, hd):
+    t_max, n_seq = 4096, 3
+    q, k, v = randn((M, n_q * hd), 1), randn((M, n_kv * hd), 2), randn((M, n_kv * hd), 3)
+    rng = np.random.default_rng(M)
+    pos = rng.choice(t_max, M, replace=False).astype(np.int32)  # distinct rows, up to the end of the cache
+    pos[0] = 0
+    seq = rng.integers(0, n_seq, M).astype(np.int32)
+    kc = torch.zeros(n_seq, t_max, n_kv * hd, dtype=torch.bfloat16, device=DEV)
+    vc = torch.zeros_like(kc)
+    q_out = bl.bitlinear_rope_kv(q.to(DEV), k.to(DEV), v.to(DEV), torch.from_numpy(pos).to(DEV), kc, vc, n_q, n_kv, hd,
+                                 seq_ids=torch.from_numpy(seq).to(DEV))
+    torch.cuda.synchronize()
+    q_ref = ds.rope(q.numpy(), pos, n_q, hd)
+    k_ref = ds.rope(k.numpy(), pos, n_kv, hd)
+    # the kernel forms the angle in fp64 and rotates in fp32 (error below 2^-22 of the pair's norm), then rounds to bf16:
+    # one bf16 ulp of the result (2^-8 relative after rounding) plus that absolute slack
+    def close(got_bits, ref, norm):
+        got = bf(got_bits)
+        assert np.all(np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 2.0 ** -20 * norm)
+
+    def pair_norm(x, nh):  # the norm of the (i, i + hd/2) pair each coordinate belongs to
+        xs = x.astype(np.float64).reshape(-1, nh, 2, hd // 2)
+        return np.broadcast_to(np.sqrt((xs ** 2).sum(2, keepdims=True)), xs.shape).reshape(x.shape[0], -1)
+
+    close(bits(q_out), q_ref, pair_norm(q.numpy(), n_q))
+    assert np.array_equal(bits(q_out)[0], oracle.f32_to_bf16(q.numpy()[0]))  # position 0: the identity, bit for bit
+    kc_h, vc_h = bits(kc), bits(vc)
+    for m in range(M):
+        close(kc_h[seq[m], pos[m]][None], k_ref[m][None], pair_norm(k.numpy(), n_kv)[m][None])
+        assert np.array_equal(vc_h[seq[m], pos[m]], oracle.f32_to_bf16(v.numpy()[m]))  # values are stored unrotated
+    # nothing else was written
+    mask = np.ones((n_seq, t_max), bool)
+    mask[seq, pos] = False
+    assert not kc_h[mask].any() and not vc_h[mask].any()
+
+
+@pytest.mark.parametrize("n_q,n_kv,hd,lengths", [
+    (20, 5, 128, [4096]),                      # the 2B configuration at a full cache: 64 slices
+    (20, 5, 128, [1, 7, 8, 9, 300, 1000]),     # ragged lengths, several tokens
+    (4, 2, 64, [5, 64, 65, 513]),
+    (8, 1, 128, [33]),                         # eight query heads on one KV head
+])
+def test_attention_decode(n_q, n_kv, hd, lengths):
+    M = len(lengths)
+    t_max = max(max(lengths), 16)
+    n_seq = 2
+    kc = randn((n_seq, t_max, n_kv * hd), 10).to(torch.bfloat16)
+    vc = randn((n_seq, t_max, n_kv * hd), 11).to(torch.bfloat16)
+    q = randn((M, n_q * hd), 12, 2.0).to(torch.bfloat16)  # scores with a standard deviation of about 2: a peaked softmax
+    seq = (np.arange(M) % n_seq).astype(np.int32)
+    out = bl.bitlinear_attention_decode(q.to(DEV), kc.to(DEV), vc.to(DEV), torch.tensor(lengths, dtype=torch.int32, device=DEV),
+                                        n_q, n_kv, hd, seq_ids=torch.from_numpy(seq).to(DEV))
+    torch.cuda.synchronize()
+    got = bf(bits(out))
+    kb, vb, qb = bits(kc), bits(vc), bits(q)
+    for m in range(M):
+        ref = ds.attention_decode(qb[m], kb[seq[m]], vb[seq[m]], lengths[m], n_q, n_kv, hd)
+        # fp32 scores (error ~1e-6 relative to |q||k|), fp32 softmax and accumulation, one bf16 rounding at the end:
+        # 2^-8 relative for the rounding plus 1e-4 of the largest value magnitude for the fp32 arithmetic
+        vmax = np.abs(bf(vb[seq[m], :lengths[m]])).max()
+        assert np.all(np.abs(got[m] - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-4 * vmax), m
+
+
+def test_attention_hand_cases():
+    n_q, n_kv, hd, T = 4, 2, 64, 40
+    kc = randn((1, T, n_kv * hd), 20).to(torch.bfloat16)
+    vc = randn((1, T, n_kv * hd), 21).to(torch.bfloat16)
+    lengths = torch.tensor([1, 25], dtype=torch.int32, device=DEV)
+    q = torch.zeros(2, n_q * hd, dtype=torch.bfloat16)
+    q[0] = randn((n_q * hd,), 22).to(torch.bfloat16)
+    out = bf(bits(bl.bitlinear_attention_decode(q.to(DEV), kc.to(DEV), vc.to(DEV), lengths, n_q, n_kv, hd)))
+    v64 = bf(bits(vc))[0].reshape(T, n_kv, hd)
+    # length 1: the first value row, whatever the query (exact: the weight is 1)
+    assert np.array_equal(out[0].reshape(n_q, hd)[3], v64[0, 1])
+    # zero query: the mean of the first 25 value rows
+    want = v64[:25].mean(axis=0)
+    assert np.all(np.abs(out[1].reshape(n_q, hd)[0] - want[0]) <= 2.0 ** -8 * np.abs(want[0]) + 1e-5)
+
+
+@pytest.mark.parametrize("M,V,K", [(1, 1000, 256), (3, 5000, 2560), (16, 2048, 2560), (1, 128256, 2560)])
+def test_lm_head(M, V, K):
+    x = randn((M, K), 30).to(torch.bfloat16)
+    table = randn((V, K), 31, 0.05).to(torch.bfloat16)
+    logits = bl.bitlinear_lm_head(x.to(DEV), table.to(DEV)).cpu().numpy().astype(np.float64)
+    if V > 20000:  # the full vocabulary: sampled rows
+        rows = np.concatenate([np.random.default_rng(1).integers(0, V, 2000), [0, V - 1]])
+    else:
+        rows = np.arange(V)
+    ref = ds.lm_head(bits(x), bits(table)[rows])
+    # K products of bf16 values accumulated in fp32 in another order: error below K * 2^-24 * sum |x e|
+    bound = K * 2.0 ** -24 * (np.abs(bf(bits(x))) @ np.abs(bf(bits(table)[rows])).T)
+    assert np.all(np.abs(logits[:, rows] - ref) <= bound + 1e-30)
+    assert not np.isnan(logits).any()
+
+
+def test_embed():
+    V, K = 300, 512
+    table = randn((V, K), 40).to(torch.bfloat16)
+    ids = torch.tensor([0, 299, 17, 17, 5], dtype=torch.int32)
+    out = bl.bitlinear_embed(ids.to(DEV), table.to(DEV))
+    assert np.array_equal(bits(out), ds.embed(ids.numpy(), bits(table)))
+
+
+def test_argument_checks():
+    lib = bl.lib()
+    fake = 0x1000
+    assert lib.bitlinear_lm_head(fake, fake, 17, 100, 256, fake, None) == 2
+    assert lib.bitlinear_lm_head(fake, fake, 1, 100, 250, fake, None) == 2
+    assert lib.bitlinear_lm_head(None, fake, 1, 100, 256, fake, None) == 1
+    assert lib.bitlinear_attention_workspace_bytes(1, 20, 5, 96, 128) == 0  # head_dim 64 or 128
+    assert lib.bitlinear_attention_decode(fake, fake, fake, fake, None, 1, 20, 6, 128, 128, fake, fake, 1 << 20, None) == 2
+    assert lib.bitlinear_attention_decode(fake, fake, fake, fake, None, 1, 20, 5, 128, 128, fake, fake, 16, None) == 4
+    assert lib.bitlinear_rope_kv(fake, fake, fake, fake, None, 1, 20, 5, 100, 500000.0, fake, fake, fake, 16, None) == 2
+    assert lib.bitlinear_embed(fake, fake, 0, 10, 256, fake, None) == 0
