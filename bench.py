@@ -306,6 +306,11 @@ def run_ours(args):
     if rank == 0:
         chain = run_chain(bl, dev, pool, gains, peaks, packed_bytes, reps=max(5, args.steps))
 
+    # ---- a whole decoded token: the chain plus rotary embedding, attention over a 4096-token cache, output head ----
+    decode_step = None
+    if rank == 0:
+        decode_step = run_decode_step(bl, dev, pool, gains, peaks, packed_bytes, reps=max(5, args.steps))
+
     # ---- prefill: int8 tensor-core path at M = 2048 on the 7 shapes (rank 0 only) ----
     prefill = None
     if rank == 0:
@@ -329,7 +334,8 @@ def run_ours(args):
             "frac_of_hbm_peak": round(value / world / peaks["hbm_gbs"], 4),
             "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "sustained": sustained, "per_call": per_call, "config1": config1,
-            "decode_more_tokens": decode_m, "dense_layout": dense, "chain": chain, "prefill": prefill, "sweep": sweep,
+            "decode_more_tokens": decode_m, "dense_layout": dense, "chain": chain, "decode_step": decode_step,
+            "prefill": prefill, "sweep": sweep,
             "cpu_baseline": cpu,
         }
         print(json.dumps(out))
@@ -382,6 +388,79 @@ def run_chain(bl, dev, pool, gains, peaks, packed_bytes, reps):
                 "persistent_launches_per_token": 1,
                 "persistent_equals_per_level_calls": bool(torch.equal(h_ref, h_p))})
     return out
+
+
+def graph_time_ms(fn, reps):
+    """fn's launches captured once into a CUDA graph; mean device time of a replay.  None if the capture is refused."""
+    try:
+        graph = torch.cuda.CUDAGraph()
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            fn()
+            with torch.cuda.graph(graph, stream=side):
+                fn()
+        torch.cuda.current_stream().wait_stream(side)
+        graph.replay()
+        return cuda_time_ms(lambda: [graph.replay() for _ in range(reps)]) / reps
+    except Exception:
+        return None
+
+
+def run_decode_step(bl, dev, pool, gains, peaks, packed_bytes, reps, M=1, context=4096):
+    """One whole decoded token of the 2B configuration at M sequences with `context` - 1 tokens already in the cache:
+    embedding gather, 30 x {q/k/v, rotary embedding + cache append, grouped-query attention, o, gate/up, down}, output
+    head over the 128,256-row table.  The cache and the table are bf16; the parts that are not BitLinear are timed on
+    their own as well (the 30 attention calls read 30 different caches, 315 MB at M = 1: larger than L2)."""
+    from paper_2504_12285_b200 import chain as gpu_chain
+
+    vocab = 128256
+    layers = []
+    for layer in range(wl.N_LAYERS):
+        layers.append({m["name"]: (m["packed"], m["s_w"], gains[m["K"]]) for m in pool[layer * 7:(layer + 1) * 7]})
+    gen = torch.Generator(device=dev).manual_seed(wl.seed_for(5))
+    table = (torch.randn(vocab, wl.HIDDEN, generator=gen, device=dev) * 0.02).to(torch.bfloat16)
+    st = gpu_chain.DecodeStep(layers, table, M, context, wl.HIDDEN, wl.FFN, wl.N_Q_HEADS, wl.N_KV_HEADS, wl.HEAD_DIM, wl.RMS_EPS,
+                              device=dev)
+    for kc, vc in zip(st.k_cache, st.v_cache):
+        kc.copy_(torch.randn(kc.shape, generator=gen, device=dev))
+        vc.copy_(torch.randn(vc.shape, generator=gen, device=dev))
+    st.set_positions(torch.full((M,), context - 1, dtype=torch.int32, device=dev))
+    ids = torch.randint(0, vocab, (M,), generator=gen, device=dev, dtype=torch.int32)
+    n_q, n_kv, hd = st.dims
+    st.step(ids)
+    torch.cuda.synchronize()
+    assert bl.bitlinear_poll_status() == 0 and bool(torch.isfinite(st.logits).all())
+    eager_ms = cuda_time_ms(lambda: [st.step(ids) for _ in range(reps)]) / reps
+    graph_ms = graph_time_ms(lambda: st.step(ids), reps)
+
+    def attention_all():
+        for kc, vc in zip(st.k_cache, st.v_cache):
+            bl.bitlinear_attention_decode(st.q_rot, kc, vc, st.lengths, n_q, n_kv, hd, seq_ids=st.seq_ids, out=st.attn, ws=st.attn_ws)
+
+    def rope_all():
+        for kc, vc in zip(st.k_cache, st.v_cache):
+            bl.bitlinear_rope_kv(st.q, st.k, st.v, st.positions, kc, vc, n_q, n_kv, hd, seq_ids=st.seq_ids, q_out=st.q_rot)
+
+    attn_ms = graph_time_ms(attention_all, reps)
+    rope_ms = graph_time_ms(rope_all, reps)
+    # the table (657 MB) is larger than L2: back-to-back calls each stream it from HBM
+    head_ms = cuda_time_ms(lambda: [bl.bitlinear_lm_head(st.h_mid, table, out=st.logits) for _ in range(reps)]) / reps
+    cache_bytes = 2 * wl.N_LAYERS * M * context * n_kv * hd * 2
+    table_bytes = table.numel() * 2
+    us = lambda ms: None if ms is None else round(ms * 1e3, 1)  # noqa: E731
+    gbs = lambda b, ms: None if ms is None else round(b / ms / 1e6, 1)  # noqa: E731
+    total = graph_ms if graph_ms is not None else eager_ms
+    return {"workload": f"one decoded token, M={M}, {context - 1} tokens in a bf16 KV cache, 30 layers, bf16 output head of {vocab} rows",
+            "launches_per_token": wl.N_LAYERS * st.launches_per_layer + 3,
+            "eager_us_per_token": us(eager_ms), "graph_us_per_token": us(graph_ms),
+            "bytes_per_token": {"packed_weights": packed_bytes, "kv_cache": cache_bytes, "output_head": table_bytes},
+            "frac_of_hbm_peak": round((packed_bytes + cache_bytes + table_bytes) / total / 1e6 / peaks["hbm_gbs"], 4),
+            "attention_30_layers": {"us": us(attn_ms), "GBps": gbs(cache_bytes, attn_ms),
+                                    "frac_of_hbm_peak": None if attn_ms is None else round(cache_bytes / attn_ms / 1e6 / peaks["hbm_gbs"], 4)},
+            "rope_append_30_layers_us": us(rope_ms),
+            "output_head": {"us": us(head_ms), "GBps": gbs(table_bytes, head_ms),
+                            "frac_of_hbm_peak": round(table_bytes / head_ms / 1e6 / peaks["hbm_gbs"], 4)}}
 
 
 def timed_sequence(calls, blocker):
@@ -743,6 +822,15 @@ def run_case_chain(args, bl, dev):
                       "us_per_level": round(ms * 1e3 / (4 * args.layers), 3), "packed_GBps": round(packed_bytes / ms / 1e6, 1)}))
 
 
+def run_case_step(args, bl, dev):
+    """A whole decoded token at --m sequences with --context cache rows (see run_decode_step)."""
+    pool = build_decode_pool(bl, dev, wl.N_LAYERS)
+    gains = {k: wl.gain_ones(k).to(dev) for k in (wl.HIDDEN, wl.FFN)}
+    out = run_decode_step(bl, dev, pool, gains, load_peaks(), sum(p["packed"].numel() for p in pool), max(3, args.steps),
+                          M=args.m, context=args.context)
+    print(json.dumps(dict(out, case="step")))
+
+
 def run_case_group(args, bl, dev):
     """The 7 shapes of a layer at --m tokens as one grouped call (quantiser + unpack + grouped GEMM)."""
     M = args.m
@@ -781,6 +869,8 @@ def run_case(args):
         return run_case_batch(args, bl, dev)
     if args.case == "group":
         return run_case_group(args, bl, dev)
+    if args.case == "step":
+        return run_case_step(args, bl, dev)
     if args.case == "chain":
         return run_case_chain(args, bl, dev)
     n, k = wl.SHAPE_NK[args.shape]
@@ -831,11 +921,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--case", choices=["gemv", "gemm", "quant", "pack", "batch", "group", "chain"], default=None)
+    ap.add_argument("--case", choices=["gemv", "gemm", "quant", "pack", "batch", "group", "chain", "step"], default=None)
     ap.add_argument("--layers", type=int, default=10)
     ap.add_argument("--shape", choices=list(wl.SHAPE_NK), default="q")
     ap.add_argument("--m", type=int, default=1)
     ap.add_argument("--copies", type=int, default=1)
+    ap.add_argument("--context", type=int, default=4096)
     ap.add_argument("--ydtype", choices=["f32", "bf16"], default="f32")
     args = ap.parse_args()
     if args.case:

@@ -48,10 +48,10 @@ _SIGNATURES = {
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_rope_kv": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_float,
-                                   _c_void_p, _c_void_p, _c_void_p, _c_int, _c_void_p]),
+                                   _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
     "bitlinear_attention_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int, _c_int]),
     "bitlinear_attention_decode": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int,
-                                            _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p]),
+                                            _c_int, _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_lm_head": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_void_p]),
     "bitlinear_embed": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
@@ -484,19 +484,27 @@ def bitlinear_forward_batch_host(batch: ProblemBatch, x_host: torch.Tensor, x_de
     _check(rc, "bitlinear_forward_batch_host")
 
 
+def _cache_dims(k_cache, v_cache, width: int):
+    """(n_seq, t_max) of a key/value cache pair [n_seq, t_max, width] or [t_max, width]."""
+    if k_cache.shape != v_cache.shape or k_cache.dim() not in (2, 3) or k_cache.shape[-1] != width:
+        raise ValueError(f"caches must both be [n_seq, t_max, {width}] or [t_max, {width}]")
+    return (k_cache.shape[0] if k_cache.dim() == 3 else 1), k_cache.shape[-2]
+
+
 def bitlinear_rope_kv(q, k, v, positions, k_cache, v_cache, n_q_heads: int, n_kv_heads: int, head_dim: int,
                       rope_base: float = 500000.0, seq_ids=None, q_out=None):
     """Rotate q, k (fp32 [M, heads * D]) at `positions` (int32 [M]); q -> bf16 (returned), k / v appended to the bf16
-    caches [n_seq, t_max, n_kv * D] at those positions."""
+    caches [n_seq, t_max, n_kv * D] (contiguous) at those positions."""
     _dev(q, torch.float32, "q"), _dev(k, torch.float32, "k"), _dev(v, torch.float32, "v")
     _dev(positions, torch.int32, "positions"), _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache")
     if seq_ids is not None:
         _dev(seq_ids, torch.int32, "seq_ids")
     M = q.shape[0]
+    n_seq, t_max = _cache_dims(k_cache, v_cache, n_kv_heads * head_dim)
     if q_out is None:
         q_out = torch.empty(M, n_q_heads * head_dim, dtype=torch.bfloat16, device=q.device)
     rc = lib().bitlinear_rope_kv(_ptr(q), _ptr(k), _ptr(v), _ptr(positions), _ptr(seq_ids), M, n_q_heads, n_kv_heads, head_dim,
-                                 rope_base, _ptr(q_out), _ptr(k_cache), _ptr(v_cache), k_cache.shape[-2], _stream())
+                                 rope_base, _ptr(q_out), _ptr(k_cache), _ptr(v_cache), n_seq, t_max, _stream())
     _check(rc, "bitlinear_rope_kv")
     return q_out
 
@@ -512,13 +520,14 @@ def bitlinear_attention_decode(q, k_cache, v_cache, lengths, n_q_heads: int, n_k
     _dev(lengths, torch.int32, "lengths")
     if seq_ids is not None:
         _dev(seq_ids, torch.int32, "seq_ids")
-    M, t_max = q.shape[0], k_cache.shape[-2]
+    M = q.shape[0]
+    n_seq, t_max = _cache_dims(k_cache, v_cache, n_kv_heads * head_dim)
     if out is None:
         out = torch.empty(M, n_q_heads * head_dim, dtype=torch.bfloat16, device=q.device)
     if ws is None:
         ws = _workspace(bitlinear_attention_workspace_bytes(M, n_q_heads, n_kv_heads, head_dim, t_max), q.device)
     rc = lib().bitlinear_attention_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(lengths), _ptr(seq_ids), M, n_q_heads,
-                                          n_kv_heads, head_dim, t_max, _ptr(out), _ptr(ws), ws.numel(), _stream())
+                                          n_kv_heads, head_dim, n_seq, t_max, _ptr(out), _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_attention_decode")
     return out
 

@@ -69,6 +69,79 @@ class DecodeChain:
         return self.h_mid
 
 
+class DecodeStep:
+    """One whole decoded token for M sequences: embedding gather, per layer {q/k/v BitLinear, rotary embedding + cache
+    append, grouped-query attention over the cache, o BitLinear, gate/up BitLinear, down BitLinear} with the residual
+    adds and the squared-ReLU gate fused into the quantiser launches, then the output head.  Sequence m owns row m of
+    every layer's cache."""
+
+    def __init__(self, layers, embedding: torch.Tensor, M: int, t_max: int, hidden: int, ffn: int, n_q_heads: int,
+                 n_kv_heads: int, head_dim: int, rms_eps: float = 1e-5, rope_base: float = 500000.0, device="cuda:0"):
+        """layers: as for DecodeChain; embedding: bf16 [V, hidden], used for the gather and as the output head."""
+        dev = torch.device(device)
+        self.M, self.dims, self.rope_base, self.table = M, (n_q_heads, n_kv_heads, head_dim), rope_base, embedding
+        kv = n_kv_heads * head_dim
+        f32 = dict(dtype=torch.float32, device=dev)
+        bf = dict(dtype=torch.bfloat16, device=dev)
+        self.h_in, self.h_mid = torch.zeros(M, hidden, **bf), torch.zeros(M, hidden, **bf)
+        self.q, self.k, self.v = torch.empty(M, hidden, **f32), torch.empty(M, kv, **f32), torch.empty(M, kv, **f32)
+        self.q_rot, self.attn = torch.empty(M, hidden, **bf), torch.empty(M, hidden, **bf)
+        self.o = torch.empty(M, hidden, **f32)
+        self.g, self.u = torch.empty(M, ffn, **f32), torch.empty(M, ffn, **f32)
+        self.dn = torch.empty(M, hidden, **f32)
+        self.logits = torch.empty(M, embedding.shape[0], **f32)
+        self.k_cache = [torch.zeros(M, t_max, kv, **bf) for _ in layers]
+        self.v_cache = [torch.zeros(M, t_max, kv, **bf) for _ in layers]
+        self.seq_ids = torch.arange(M, dtype=torch.int32, device=dev)
+        self.positions = torch.zeros(M, dtype=torch.int32, device=dev)  # where this token goes in its sequence
+        self.lengths = torch.ones(M, dtype=torch.int32, device=dev)     # cache rows attended to: positions + 1
+        self.attn_ws = torch.empty(bl.bitlinear_attention_workspace_bytes(M, n_q_heads, n_kv_heads, head_dim, t_max),
+                                   dtype=torch.uint8, device=dev)
+        self.calls = []
+        for li, layer in enumerate(layers):
+            def item(name, x, y, step=None):
+                packed, s_w, gain = layer[name]
+                return (x, gain, packed, s_w, y) if step is None else (x, gain, packed, s_w, y, step)
+            res_in = None if li == 0 else (bl.X_RESIDUAL, self.dn, self.h_in, 0, 0)
+            x_qkv = self.h_in if li == 0 else self.h_mid
+            res_mid = (bl.X_RESIDUAL, self.o, self.h_mid, 0, 0)
+            relu2 = (bl.X_RELU2, self.u, None, 0, 0)
+            groups = [[item("q", x_qkv, self.q, res_in), item("k", x_qkv, self.k, res_in), item("v", x_qkv, self.v, res_in)],
+                      [item("o", self.attn, self.o)],
+                      [item("gate", self.h_in, self.g, res_mid), item("up", self.h_in, self.u, res_mid)],
+                      [item("down", self.g, self.dn, relu2)]]
+            per_layer = []
+            for grp in groups:
+                batch = bl.ProblemBatch(grp, rms_eps)
+                ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=dev)
+                bl.bitlinear_forward_batch(batch, ws)  # uploads the plan; results are overwritten by step()
+                per_layer.append((batch, ws))
+            self.calls.append(per_layer)
+        torch.cuda.synchronize(dev)
+
+    launches_per_layer = 11  # 4 x (quantiser + weight stream), rotary/append, attention slices, attention merge
+
+    def set_positions(self, positions: torch.Tensor) -> None:
+        """positions: int32 [M] (device): where the next token of each sequence goes; it attends to rows 0 .. position."""
+        self.positions.copy_(positions)
+        torch.add(self.positions, 1, out=self.lengths)
+
+    def step(self, ids: torch.Tensor) -> torch.Tensor:
+        """ids: int32 [M] (device) -> logits fp32 [M, V]; appends this token's keys and values to every layer's cache."""
+        n_q, n_kv, hd = self.dims
+        bl.bitlinear_embed(ids, self.table, out=self.h_in)
+        for li, (qkv, o, gu, down) in enumerate(self.calls):
+            bl.bitlinear_forward_batch(*qkv, reuse_plan=True)
+            bl.bitlinear_rope_kv(self.q, self.k, self.v, self.positions, self.k_cache[li], self.v_cache[li], n_q, n_kv, hd,
+                                 rope_base=self.rope_base, seq_ids=self.seq_ids, q_out=self.q_rot)
+            bl.bitlinear_attention_decode(self.q_rot, self.k_cache[li], self.v_cache[li], self.lengths, n_q, n_kv, hd,
+                                          seq_ids=self.seq_ids, out=self.attn, ws=self.attn_ws)
+            for batch, ws in (o, gu, down):
+                bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
+        bl.bitlinear_glue_residual_add(self.h_mid, self.dn)  # the last layer's residual
+        return bl.bitlinear_lm_head(self.h_mid, self.table, out=self.logits)
+
+
 class PersistentChain:
     """The same chain at one token through bitlinear_decode_chain: one cooperative kernel per token."""
 

@@ -6,16 +6,20 @@
 //   rope_kv_kernel            : rotates q and k (pairs i, i + head_dim/2; angle = position * base^(-2i/head_dim), formed
 //                               in fp64 because positions reach the thousands), writes q as bf16 and appends k, v to
 //                               the bf16 cache of the token's sequence.
-//   attn_decode_partial_kernel: one CTA per (token, KV head, slice of 64 cache positions), one warp per query head of the
-//                               group; the slice is bulk-copied into shared memory once and scored by all heads;
-//                               softmax in fp32; partial (max, sum, weighted values) per slice.
+//   attn_decode_partial_kernel: one CTA per (token, KV head, slice of the cache); 64-row tiles of keys and values arrive
+//                               by tensor-map copies, the query heads of the group are the rows of a tensor-core
+//                               operand (mma.sync, bf16 inputs, fp32 accumulation), softmax in fp32; partial
+//                               (max, sum, weighted values) per slice.
 //   attn_decode_combine_kernel: merges the slices of a (token, query head) and writes bf16.
 //   lm_head_kernel            : logits = x . E^T for up to 16 tokens, one warp per vocabulary row, the table streamed
 //                               once with 128-bit loads (HBM-bound: 657 MB for 128,256 x 2560).
 //   embed_kernel              : row gather.
 #include "common.cuh"
 #include "sm100_sync.cuh"
+#include "tensor_map.cuh"
 
+#include <algorithm>
+#include <mutex>
 #include <type_traits>
 
 namespace bitlinear {
@@ -29,7 +33,7 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 
 __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                                       const float* __restrict__ v, const int* __restrict__ positions,
-                                                      const int* __restrict__ seq_ids, int M, int n_q, int n_kv, int hd,
+                                                      const int* __restrict__ seq_ids, int M, int n_q, int n_kv, int hd, int n_seq,
                                                       double log2_base, __nv_bfloat16* __restrict__ q_out,
                                                       __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
                                                       int t_max) {
@@ -51,24 +55,28 @@ __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ 
         const float lo = src[i], hi = src[i + half];
         const float o_lo = __fsub_rn(__fmul_rn(lo, c), __fmul_rn(hi, s));
         const float o_hi = __fadd_rn(__fmul_rn(hi, c), __fmul_rn(lo, s));
-        if (!is_q && (pos < 0 || pos >= t_max)) return;  // a position outside the cache is not stored
+        const int seq = seq_ids ? seq_ids[m] : 0;
+        if (!is_q && (pos < 0 || pos >= t_max || seq < 0 || seq >= n_seq)) return;  // a row outside the cache is not stored
         __nv_bfloat16* dst;
         if (is_q) dst = q_out + (size_t)m * n_q * hd + (size_t)head * hd;
-        else dst = k_cache + ((size_t)(seq_ids ? seq_ids[m] : 0) * t_max + pos) * vals_per_tok + (size_t)(head - n_q) * hd;
+        else dst = k_cache + ((size_t)seq * t_max + pos) * vals_per_tok + (size_t)(head - n_q) * hd;
         dst[i] = __float2bfloat16_rn(o_lo);
         dst[i + half] = __float2bfloat16_rn(o_hi);
     } else if (idx < n_rot + (long long)M * vals_per_tok) {
         const long long j = idx - n_rot;
         const int m = (int)(j / vals_per_tok), e = (int)(j - (long long)m * vals_per_tok);
-        if (positions[m] < 0 || positions[m] >= t_max) return;
-        v_cache[((size_t)(seq_ids ? seq_ids[m] : 0) * t_max + positions[m]) * vals_per_tok + e] =
+        const int seq = seq_ids ? seq_ids[m] : 0;
+        if (positions[m] < 0 || positions[m] >= t_max || seq < 0 || seq >= n_seq) return;
+        v_cache[((size_t)seq * t_max + positions[m]) * vals_per_tok + e] =
             __float2bfloat16_rn(v[(size_t)m * vals_per_tok + e]);
     }
 }
 
 // ---------------------------------------------------------------------------------------------- decode attention
 
-constexpr int kAttnKeys = 64;  // cache positions per CTA
+constexpr int kAttnKeys = 64;       // cache rows per tile
+constexpr int kAttnStages = 3;      // tiles in flight per CTA
+constexpr int kAttnMaxSplits = 64;  // partial results per (token, query head)
 
 // partial result of one slice of the cache for one (token, query head): weighted values, running maximum, sum of weights
 template <int HD>
@@ -78,165 +86,292 @@ struct __align__(16) AttnPartial {
 };
 
 template <int HD>
-constexpr size_t attn_smem_bytes(int group) {
-    return (size_t)2 * kAttnKeys * HD * 2 + (size_t)group * (HD + kAttnKeys) * sizeof(float) + 16;
+constexpr size_t attn_smem_bytes() {
+    return 1024 /*alignment slack*/ + (size_t)kAttnStages * 2 * kAttnKeys * HD * 2 + 8 * kAttnStages + 8;
 }
 
-// One CTA per (slice of 64 cache positions, KV head, token); one warp per query head of the group.  The slice's key and
-// value rows of this KV head (HD bf16 each, contiguous) are brought into shared memory by one bulk copy per row, all in
-// flight at once, so that a CTA pays one round trip to HBM; then every warp scores the 64 keys against its query
-// (one key per lane, the 16-byte chunks of a row visited in a lane-rotated order so that the lanes of a quarter-warp
-// hit distinct banks), takes the softmax weights of the slice and accumulates the values (one lane per HD/32
-// coordinates).  Slices past the token's length return at once and are not read by the combine kernel.
+// How the 64-row tiles of a token's live cache rows are dealt to the slices: `per` tiles each, `live` slices in use.
+struct AttnSlices {
+    int per, live;
+};
+__host__ __device__ inline AttnSlices attn_slices(int len, int splits) {
+    const int tiles = (len + kAttnKeys - 1) / kAttnKeys;
+    const int per = tiles > 0 ? (tiles + splits - 1) / splits : 1;
+    return {per, (tiles + per - 1) / per};
+}
+
+__device__ __forceinline__ void tma_tile_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar)
+        : "memory");
+}
+// four 8 x 8 matrices of 16-bit elements, row addresses from lanes 8i .. 8i+7 for matrix i
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];" : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr));
+}
+// d += a * b, 16 x 8 x 16, bf16 operands, fp32 accumulation; rows 8 .. 15 of a are zero here (a1 = a3 = 0)
+__device__ __forceinline__ void mma_rows8(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+// One CTA of four warps per (slice of the cache, KV head, token).  A slice is a run of 64-row tiles; each tile's key and
+// value rows of this KV head (64 x HD bf16 each) arrive in shared memory by tensor-map copies of 64 rows x 128 bytes
+// (128-byte swizzle), up to three tiles in flight, so every query head of the group reads the cache from HBM once.
+// The group's query heads (at most 8) are the rows of a 16-row tensor-core operand: warp w takes keys 16w .. 16w+15 of
+// every tile, S = Q K^T by mma.sync (bf16 x bf16 products are exact, fp32 accumulation), a running softmax per head in
+// fp32, and O += P V with the weights split into two bf16 parts (P = P_hi + P_lo, relative error 2^-17) so that the
+// tensor core's bf16 operand costs no accuracy.  The four warps' results are merged in shared memory at the end.
+// Slices past the token's length return at once and are not read by the combine kernel.  Rows of a tile past the
+// token's length are copied (they are inside the cache, or zero-filled past its end); their scores are discarded by a
+// select and their value rows are overwritten with zeros before use, so whatever bits they hold never enter a result.
 template <int HD>
-__global__ void __launch_bounds__(256) attn_decode_partial_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_cache,
-                                                                  const __nv_bfloat16* __restrict__ v_cache, const int* __restrict__ lengths,
-                                                                  const int* __restrict__ seq_ids, int n_q, int n_kv, int t_max,
+__global__ void __launch_bounds__(128) attn_decode_partial_kernel(const __grid_constant__ CUtensorMap map_k,
+                                                                  const __grid_constant__ CUtensorMap map_v,
+                                                                  const __nv_bfloat16* __restrict__ q, const int* __restrict__ lengths,
+                                                                  const int* __restrict__ seq_ids, int n_q, int n_kv, int n_seq, int t_max,
                                                                   int splits, float scale, AttnPartial<HD>* __restrict__ part,
                                                                   int* __restrict__ status_word) {
-    constexpr int NCH = HD / 8;   // 16-byte chunks per row
-    constexpr int CPL = HD / 32;  // value coordinates per lane
-    extern __shared__ __align__(16) uint8_t attn_smem[];
+    constexpr int HALVES = HD / 64;                 // 128-byte column blocks of a row
+    constexpr uint32_t kHalfBytes = kAttnKeys * 128;  // one block of a tile: 64 rows x 128 bytes
+    constexpr uint32_t kTileBytes = HALVES * kHalfBytes;
+    constexpr int KS = HD / 16;  // k-steps of Q K^T
+    constexpr int NT = HD / 8;   // 8-column tiles of O
+    constexpr int OPAD = HD + 8; // row stride of the merge buffer (floats)
+    extern __shared__ uint8_t attn_smem_raw[];
     const int split = blockIdx.x, g = blockIdx.y, m = blockIdx.z;
     const int group = n_q / n_kv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int h = g * group + warp;  // this warp's query head
-    const int len = min(max(lengths[m], 0), t_max);
-    const int t0 = split * kAttnKeys;
-    if (t0 >= len) return;  // the whole CTA: nothing of this slice is live
-    const int n = min(kAttnKeys, len - t0);
+    const int r = lane >> 2, qd = lane & 3;  // this lane's row (query head of the group) and column pair in a fragment
+    const int seq = seq_ids ? seq_ids[m] : 0;
+    const int len = (seq >= 0 && seq < n_seq) ? min(max(lengths[m], 0), t_max) : 0;
+    const AttnSlices sl = attn_slices(len, splits);
+    if (split >= sl.live) return;  // the whole CTA: nothing of this slice is live
+    const int tile0 = split * sl.per;
+    const int n_tiles = min(sl.per, (len + kAttnKeys - 1) / kAttnKeys - tile0);
 
-    uint4* k_s = reinterpret_cast<uint4*>(attn_smem);                                  // [64][NCH]
-    uint4* v_s = k_s + kAttnKeys * NCH;                                                // [64][NCH]
-    float* q_s = reinterpret_cast<float*>(v_s + kAttnKeys * NCH) + warp * HD;          // two planes [NCH][4] per head
-    float* p_s = reinterpret_cast<float*>(v_s + kAttnKeys * NCH) + group * HD + warp * kAttnKeys;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(reinterpret_cast<float*>(v_s + kAttnKeys * NCH) + group * (HD + kAttnKeys));
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar + 1);
-    const uint32_t bar_s = smem_u32(bar);
+    uint8_t* smem = attn_smem_raw + ((1024u - (smem_u32(attn_smem_raw) & 1023u)) & 1023u);
+    const uint32_t ring_s = smem_u32(smem);  // [stage][K, V][block][64 rows][128 bytes, swizzled]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnStages * 2 * kTileBytes);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kAttnStages);
+    const uint32_t bar_s = smem_u32(bars);
 
+    const int row0 = seq * t_max + tile0 * kAttnKeys;
+    auto issue = [&](int i) {  // one thread: tile i of the slice into stage i % kAttnStages
+        const uint32_t st = (uint32_t)(i % kAttnStages), dst = ring_s + st * 2u * kTileBytes, bar = bar_s + 8u * st;
+        mbar_expect_tx(bar, 2u * kTileBytes);
+#pragma unroll
+        for (int hf = 0; hf < HALVES; ++hf) {
+            tma_tile_2d(dst + hf * kHalfBytes, &map_k, g * HD + hf * 64, row0 + i * kAttnKeys, bar);
+            tma_tile_2d(dst + kTileBytes + hf * kHalfBytes, &map_v, g * HD + hf * 64, row0 + i * kAttnKeys, bar);
+        }
+    };
     if (threadIdx.x == 0) {
         *abort_flag = 0;
-        mbar_init(bar_s, 1);
+        for (int st = 0; st < kAttnStages; ++st) mbar_init(bar_s + 8u * st, 1);
         mbar_init_fence();
+        for (int i = 0; i < min(kAttnStages, n_tiles); ++i) issue(i);
     }
-    __syncthreads();
-    if (warp == 0) {
-        if (lane == 0) mbar_expect_tx(bar_s, (uint32_t)n * HD * 2u * 2u);
-        __syncwarp();
-        const size_t row0 = ((size_t)(seq_ids ? seq_ids[m] : 0) * t_max + t0) * ((size_t)n_kv * HD) + (size_t)g * HD;
-        for (int r = lane; r < n; r += 32) {
-            const size_t off = row0 + (size_t)r * n_kv * HD;
-            bulk_load(smem_u32(k_s + r * NCH), k_cache + off, HD * 2, bar_s);
-            bulk_load(smem_u32(v_s + r * NCH), v_cache + off, HD * 2, bar_s);
+    // the group's queries as the A operand: row r = head g * group + r (zero rows past the group), two registers per k-step
+    uint32_t qa[KS][2];
+    {
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)m * n_q + (size_t)g * group + min(r, group - 1)) * HD);
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qa[ks][0] = r < group ? qrow[8 * ks + qd] : 0u;
+            qa[ks][1] = r < group ? qrow[8 * ks + 4 + qd] : 0u;
         }
     }
-    // the query as fp32 in two planes: plane 0 holds coordinates 8j .. 8j+3 of chunk j, plane 1 coordinates 8j+4 .. 8j+7,
-    // so that lanes reading eight different chunks with 16-byte loads cover all 32 banks once
-    {
-        const __nv_bfloat16* qh = q + ((size_t)m * n_q + h) * HD;
-        for (int c = lane; c < HD; c += 32) q_s[(c >> 2 & 1) * (HD / 2) + (c >> 3) * 4 + (c & 3)] = __bfloat162float(qh[c]);
+    __syncthreads();  // barriers initialised, abort flag cleared
+
+    float m_run = -INFINITY, l_run = 0.0f;  // of row r over this warp's keys (the four lanes of a quad agree)
+    float o[NT][4];
+#pragma unroll
+    for (int d = 0; d < NT; ++d) o[d][0] = o[d][1] = o[d][2] = o[d][3] = 0.0f;
+    const int kb = warp * 16;                // this warp's keys of a tile
+    const int mi = lane >> 3, mr = lane & 7; // the matrix and row this lane addresses for ldmatrix
+
+    for (int i = 0; i < n_tiles; ++i) {
+        const uint32_t st = (uint32_t)(i % kAttnStages);
+        const bool ok = mbar_wait(bar_s + 8u * st, (uint32_t)(i / kAttnStages) & 1u, abort_flag);
+        const int n = min(kAttnKeys, len - (tile0 + i) * kAttnKeys);  // live rows of the tile, >= 1
+        if (ok && kb < n) {
+            const uint32_t kbase = ring_s + st * 2u * kTileBytes, vbase = kbase + kTileBytes;
+            if (n < kb + 16) {  // the ragged end: zero this warp's dead value rows
+                for (int idx = lane; idx < (kb + 16 - n) * HALVES * 8; idx += 32) {
+                    const int row = n + idx / (HALVES * 8), c = idx % (HALVES * 8);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + (c >> 3) * kHalfBytes + row * 128 + (c & 7) * 16), "r"(0u)
+                                 : "memory");
+                }
+                __syncwarp();
+            }
+            // S = Q K^T for keys kb .. kb+15: two 8-key column tiles
+            float s[2][4];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.0f;
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                // matrices: (keys 0-7, chunk c), (keys 0-7, c+1), (keys 8-15, c), (keys 8-15, c+1)
+                const int key = kb + 8 * (mi >> 1) + mr, chunk = ((2 * ks) & 7) + (mi & 1);
+                uint32_t b[4];
+                ldsm_x4(kbase + (ks >> 2) * kHalfBytes + key * 128 + ((chunk ^ mr) << 4), b);
+                mma_rows8(s[0], qa[ks][0], qa[ks][1], b[0], b[1]);
+                mma_rows8(s[1], qa[ks][0], qa[ks][1], b[2], b[3]);
+            }
+            // running softmax of row r; this lane holds keys kb + 8j + 2qd + {0, 1}
+            float sv[4];
+#pragma unroll
+            for (int j = 0; j < 2; ++j)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) sv[2 * j + e] = (kb + 8 * j + 2 * qd + e < n) ? s[j][e] * scale : -INFINITY;
+            float mt = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
+            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
+            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
+            const float m_new = fmaxf(m_run, mt);    // finite: key kb is live
+            const float corr = expf(m_run - m_new);  // expf(-inf) = 0 the first time
+            float pv[4], lt = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                pv[e] = expf(sv[e] - m_new);  // 0 for a dead key
+                lt += pv[e];
+            }
+            lt += __shfl_xor_sync(0xffffffffu, lt, 1);
+            lt += __shfl_xor_sync(0xffffffffu, lt, 2);
+            l_run = fmaf(l_run, corr, lt);
+            m_run = m_new;
+            // P as the A operand of P V: its fragment layout is the accumulator layout of S
+            float ph[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) ph[e] = __bfloat162float(__float2bfloat16_rn(pv[e]));
+            const uint32_t a0h = pack_bf16(ph[0], ph[1]), a2h = pack_bf16(ph[2], ph[3]);
+            const uint32_t a0l = pack_bf16(pv[0] - ph[0], pv[1] - ph[1]), a2l = pack_bf16(pv[2] - ph[2], pv[3] - ph[3]);
+#pragma unroll
+            for (int d = 0; d < NT; ++d) {
+                o[d][0] *= corr;
+                o[d][1] *= corr;
+            }
+#pragma unroll
+            for (int d = 0; d < NT; d += 2) {
+                // matrices (transposed on load): (keys 0-7, chunk d), (keys 8-15, d), (keys 0-7, d+1), (keys 8-15, d+1)
+                const int key = kb + 8 * (mi & 1) + mr, chunk = (d & 7) + (mi >> 1);
+                uint32_t b[4];
+                ldsm_x4_t(vbase + (d >> 3) * kHalfBytes + key * 128 + ((chunk ^ mr) << 4), b);
+                mma_rows8(o[d], a0h, a2h, b[0], b[1]);
+                mma_rows8(o[d], a0l, a2l, b[0], b[1]);
+                mma_rows8(o[d + 1], a0h, a2h, b[2], b[3]);
+                mma_rows8(o[d + 1], a0l, a2l, b[2], b[3]);
+            }
+        }
+        if (!__syncthreads_and(ok)) break;  // every warp is done with the stage - or the CTA gives up together
+        if (threadIdx.x == 0 && i + kAttnStages < n_tiles) issue(i + kAttnStages);
     }
-    __syncwarp();
-    const bool ok = mbar_wait(bar_s, 0, abort_flag);
-    if (!ok) {
-        if (lane == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
+    if (*abort_flag) {
+        if (threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
         abort_drain();
         return;
     }
-
-    // scores of keys lane and lane + 32
-    float s[kAttnKeys / 32];
+    // merge the four warps (every copy has landed and been consumed: the ring is free)
+    float* om = reinterpret_cast<float*>(smem);  // [warp][row][OPAD]
+    float* mm = om + 4 * 8 * OPAD;               // [warp][row]
+    float* ll = mm + 32;
+    if (r < group) {
 #pragma unroll
-    for (int pass = 0; pass < kAttnKeys / 32; ++pass) {
-        const int t = pass * 32 + lane;
-        float dot = 0.0f;
-        if (t < n) {
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-                const int j = (c + lane) & (NCH - 1);
-                const uint4 u = k_s[t * NCH + j];
-                const float4 qa = *reinterpret_cast<const float4*>(q_s + j * 4);
-                const float4 qb = *reinterpret_cast<const float4*>(q_s + HD / 2 + j * 4);
-                dot = fmaf(qa.x, bf16_lo_f(u.x), dot);
-                dot = fmaf(qa.y, bf16_hi_f(u.x), dot);
-                dot = fmaf(qa.z, bf16_lo_f(u.y), dot);
-                dot = fmaf(qa.w, bf16_hi_f(u.y), dot);
-                dot = fmaf(qb.x, bf16_lo_f(u.z), dot);
-                dot = fmaf(qb.y, bf16_hi_f(u.z), dot);
-                dot = fmaf(qb.z, bf16_lo_f(u.w), dot);
-                dot = fmaf(qb.w, bf16_hi_f(u.w), dot);
-            }
+        for (int d = 0; d < NT; ++d) *reinterpret_cast<float2*>(om + (warp * 8 + r) * OPAD + 8 * d + 2 * qd) = make_float2(o[d][0], o[d][1]);
+        if (qd == 0) {
+            mm[warp * 8 + r] = m_run;
+            ll[warp * 8 + r] = l_run;
         }
-        s[pass] = t < n ? dot * scale : -INFINITY;
     }
-    float mx = s[0];
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < group * HD; idx += 128) {
+        const int row = idx / HD, d = idx - row * HD;
+        float m_all = mm[row];
 #pragma unroll
-    for (int pass = 1; pass < kAttnKeys / 32; ++pass) mx = fmaxf(mx, s[pass]);
+        for (int w = 1; w < 4; ++w) m_all = fmaxf(m_all, mm[w * 8 + row]);  // finite: warp 0 always has a live key
+        float l = 0.0f, acc = 0.0f;
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));  // finite: key t0 is live
-    float l = 0.0f;
-#pragma unroll
-    for (int pass = 0; pass < kAttnKeys / 32; ++pass) {
-        const float p = expf(s[pass] - mx);  // expf(-inf) = 0 for the keys past the end
-        p_s[pass * 32 + lane] = p;
-        l += p;
-    }
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
-    __syncwarp();
-
-    // weighted values: this lane's CPL coordinates over the n live keys, two independent chains
-    float o0[CPL], o1[CPL];
-#pragma unroll
-    for (int e = 0; e < CPL; ++e) o0[e] = o1[e] = 0.0f;
-    const uint16_t* v16 = reinterpret_cast<const uint16_t*>(v_s) + lane * CPL;
-    auto add_key = [&](int t, float (&o)[CPL]) {
-        const float p = p_s[t];
-        if constexpr (CPL == 4) {
-            const uint2 u = *reinterpret_cast<const uint2*>(v16 + t * HD);
-            o[0] = fmaf(p, bf16_lo_f(u.x), o[0]);
-            o[1] = fmaf(p, bf16_hi_f(u.x), o[1]);
-            o[2] = fmaf(p, bf16_lo_f(u.y), o[2]);
-            o[3] = fmaf(p, bf16_hi_f(u.y), o[3]);
-        } else {
-            const uint32_t u = *reinterpret_cast<const uint32_t*>(v16 + t * HD);
-            o[0] = fmaf(p, bf16_lo_f(u), o[0]);
-            o[1] = fmaf(p, bf16_hi_f(u), o[1]);
+        for (int w = 0; w < 4; ++w) {
+            const float f = expf(mm[w * 8 + row] - m_all);  // 0 for a warp that saw no key
+            l = fmaf(ll[w * 8 + row], f, l);
+            acc = fmaf(om[(w * 8 + row) * OPAD + d], f, acc);
         }
-    };
-    int t = 0;
-    for (; t + 2 <= n; t += 2) {
-        add_key(t, o0);
-        add_key(t + 1, o1);
+        AttnPartial<HD>& dst = part[((size_t)m * n_q + (size_t)g * group + row) * splits + split];
+        dst.o[d] = acc;
+        if (d == 0) { dst.m = m_all; dst.l = l; }
     }
-    if (t < n) add_key(t, o0);
-
-    AttnPartial<HD>& dst = part[((size_t)m * n_q + h) * splits + split];
-    if constexpr (CPL == 4) {
-        *reinterpret_cast<float4*>(dst.o + lane * 4) = make_float4(o0[0] + o1[0], o0[1] + o1[1], o0[2] + o1[2], o0[3] + o1[3]);
-    } else {
-        *reinterpret_cast<float2*>(dst.o + lane * 2) = make_float2(o0[0] + o1[0], o0[1] + o1[1]);
-    }
-    if (lane == 0) { dst.m = mx; dst.l = l; }
 }
 
-// Merges the live slices of a (token, query head) and writes bf16; a token of length 0 gets zeros.
+// Merges the live slices (at most 64) of a (token, query head) and writes bf16; a token of length 0 gets zeros.  Four
+// warps deal the slices among themselves, every load of a warp independent of the others, and meet in shared memory.
 template <int HD>
-__global__ void __launch_bounds__(HD) attn_decode_combine_kernel(const AttnPartial<HD>* __restrict__ part, const int* __restrict__ lengths,
-                                                                 int n_q, int t_max, int splits, __nv_bfloat16* __restrict__ out) {
+__global__ void __launch_bounds__(128) attn_decode_combine_kernel(const AttnPartial<HD>* __restrict__ part, const int* __restrict__ lengths,
+                                                                  const int* __restrict__ seq_ids, int n_q, int n_seq, int t_max, int splits,
+                                                                  __nv_bfloat16* __restrict__ out) {
+    constexpr int CPL = HD / 32;
+    __shared__ float red[4][HD];
     const size_t mh = blockIdx.x;  // token * n_q + head
-    const int len = min(max(lengths[mh / n_q], 0), t_max);
-    const int live = (len + kAttnKeys - 1) / kAttnKeys;
+    const int m = (int)(mh / n_q);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int seq = seq_ids ? seq_ids[m] : 0;
+    const int len = (seq >= 0 && seq < n_seq) ? min(max(lengths[m], 0), t_max) : 0;
+    const int live = attn_slices(len, splits).live;  // <= splits <= 64
     const AttnPartial<HD>* p = part + mh * splits;
-    float m_all = -INFINITY;
-    for (int s = 0; s < live; ++s) m_all = fmaxf(m_all, p[s].m);
-    float l = 0.0f, o = 0.0f;
-    for (int s = 0; s < live; ++s) {
-        const float f = expf(p[s].m - m_all);
-        l = fmaf(p[s].l, f, l);
-        o = fmaf(p[s].o[threadIdx.x], f, o);
+    const float m0 = lane < live ? p[lane].m : -INFINITY, m1 = lane + 32 < live ? p[lane + 32].m : -INFINITY;
+    const float l0 = lane < live ? p[lane].l : 0.0f, l1 = lane + 32 < live ? p[lane + 32].l : 0.0f;
+    float m_all = fmaxf(m0, m1);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, off));
+    const float f0 = lane < live ? expf(m0 - m_all) : 0.0f, f1 = lane + 32 < live ? expf(m1 - m_all) : 0.0f;
+    float l = fmaf(l0, f0, l1 * f1);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) l += __shfl_xor_sync(0xffffffffu, l, off);
+    float acc[CPL];
+#pragma unroll
+    for (int e = 0; e < CPL; ++e) acc[e] = 0.0f;
+    if (live == 0) {  // block-uniform
+        for (int d = threadIdx.x; d < HD; d += blockDim.x) out[mh * HD + d] = __float2bfloat16_rn(0.0f);
+        return;
     }
-    out[mh * HD + threadIdx.x] = __float2bfloat16_rn(l > 0.0f ? o / l : 0.0f);
+    // all sixteen loads of the warp first (a dead slot re-reads a live one and gets weight 0: no branch), then the sums
+    float v[kAttnMaxSplits / 4][CPL];
+#pragma unroll
+    for (int i = 0; i < kAttnMaxSplits / 4; ++i) {
+        const float* po = p[min(warp + 4 * i, live - 1)].o + lane * CPL;
+        if constexpr (CPL == 4) {
+            const float4 t = *reinterpret_cast<const float4*>(po);
+            v[i][0] = t.x, v[i][1] = t.y, v[i][2] = t.z, v[i][3] = t.w;
+        } else {
+            const float2 t = *reinterpret_cast<const float2*>(po);
+            v[i][0] = t.x, v[i][1] = t.y;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kAttnMaxSplits / 4; ++i) {
+        const int s = warp + 4 * i;  // warp-uniform
+        const float fs = __shfl_sync(0xffffffffu, s < 32 ? f0 : f1, s & 31);
+        const float f = s < live ? fs : 0.0f;
+#pragma unroll
+        for (int e = 0; e < CPL; ++e) acc[e] = fmaf(v[i][e], f, acc[e]);
+    }
+#pragma unroll
+    for (int e = 0; e < CPL; ++e) red[warp][lane * CPL + e] = acc[e];
+    __syncthreads();
+    for (int d = threadIdx.x; d < HD; d += blockDim.x) {
+        const float o = (red[0][d] + red[1][d]) + (red[2][d] + red[3][d]);
+        out[mh * HD + d] = __float2bfloat16_rn(l > 0.0f ? o / l : 0.0f);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------- output head, embedding
@@ -298,10 +433,52 @@ __global__ void __launch_bounds__(256) embed_kernel(const int* __restrict__ ids,
     reinterpret_cast<uint4*>(out)[i] = reinterpret_cast<const uint4*>(table)[(size_t)id * n_vec + c];
 }
 
-int attn_splits(int t_max) { return (t_max + kAttnKeys - 1) / kAttnKeys; }
+// partial results reserved per (token, query head): one per tile of the cache, 64 at most
+int attn_splits_max(int t_max) { return std::min(kAttnMaxSplits, (t_max + kAttnKeys - 1) / kAttnKeys); }
+
+// Slices per (token, KV head) for a launch: enough CTAs for four per SM, never more than the tiles of the cache.
+int attn_splits(int M, int n_kv, int t_max, int sm_count) {
+    const int want = (4 * sm_count + M * n_kv - 1) / (M * n_kv);
+    return std::max(1, std::min(attn_splits_max(t_max), want));
+}
+
+// rows = every cache row of every sequence, columns = n_kv * hd; box = 64 rows x 64 columns (128 bytes), 128-byte swizzle
+bool make_cache_map(CUtensorMap* map, const void* cache, int n_seq, int t_max, int n_kv, int hd) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)n_kv * hd, (cuuint64_t)n_seq * t_max};
+    const cuuint64_t strides[1] = {(cuuint64_t)n_kv * hd * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kAttnKeys};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// the attention kernels need more than the default dynamic shared memory: opted in once per device
+template <int HD>
+bool attn_opt_in() {
+    static std::mutex mu;
+    static bool done[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return false;
+    }
+    std::lock_guard<std::mutex> lock(mu);
+    if (!done[dev]) {
+        if (cudaFuncSetAttribute(attn_decode_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)attn_smem_bytes<HD>()) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        done[dev] = true;
+    }
+    return true;
+}
 
 bool attn_dims_ok(int M, int n_q, int n_kv, int hd, int t_max) {
-    return M >= 0 && n_q > 0 && n_kv > 0 && n_q % n_kv == 0 && n_q / n_kv <= 8 && (hd == 64 || hd == 128) && t_max > 0 && t_max <= (1 << 22);
+    return M >= 0 && M <= 65535 && n_q > 0 && n_kv > 0 && n_q % n_kv == 0 && n_q / n_kv <= 8 && (hd == 64 || hd == 128) && t_max > 0 && t_max <= (1 << 22);
 }
 
 }  // namespace
@@ -314,14 +491,14 @@ extern "C" {
 
 int bitlinear_rope_kv(const float* q, const float* k, const float* v, const int32_t* positions, const int32_t* seq_ids, int M,
                       int n_q_heads, int n_kv_heads, int head_dim, float rope_base, void* q_out_bf16, void* k_cache_bf16,
-                      void* v_cache_bf16, int t_max, void* stream) {
-    if (M < 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0 || head_dim % 8 || t_max <= 0 || !(rope_base > 1.0f))
+                      void* v_cache_bf16, int n_seq, int t_max, void* stream) {
+    if (M < 0 || n_q_heads <= 0 || n_kv_heads <= 0 || head_dim <= 0 || head_dim % 8 || n_seq <= 0 || t_max <= 0 || !(rope_base > 1.0f))
         return BITLINEAR_ERR_SHAPE;
     if (M == 0) return BITLINEAR_OK;
     if (!q || !k || !v || !positions || !q_out_bf16 || !k_cache_bf16 || !v_cache_bf16) return BITLINEAR_ERR_NULL;
     const long long work = (long long)M * ((n_q_heads + n_kv_heads) * (head_dim / 2) + n_kv_heads * head_dim);
     rope_kv_kernel<<<(unsigned)((work + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        q, k, v, positions, seq_ids, M, n_q_heads, n_kv_heads, head_dim, log2((double)rope_base),
+        q, k, v, positions, seq_ids, M, n_q_heads, n_kv_heads, head_dim, n_seq, log2((double)rope_base),
         static_cast<__nv_bfloat16*>(q_out_bf16), static_cast<__nv_bfloat16*>(k_cache_bf16), static_cast<__nv_bfloat16*>(v_cache_bf16),
         t_max);
     return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
@@ -329,36 +506,42 @@ int bitlinear_rope_kv(const float* q, const float* k, const float* v, const int3
 
 size_t bitlinear_attention_workspace_bytes(int M, int n_q_heads, int n_kv_heads, int head_dim, int t_max) {
     if (!attn_dims_ok(M, n_q_heads, n_kv_heads, head_dim, t_max)) return 0;
-    return (size_t)(M > 0 ? M : 1) * n_q_heads * attn_splits(t_max) * (sizeof(float) * (4 + head_dim));
+    return (size_t)(M > 0 ? M : 1) * n_q_heads * attn_splits_max(t_max) * (sizeof(float) * (4 + head_dim));
 }
 
 int bitlinear_attention_decode(const void* q_bf16, const void* k_cache_bf16, const void* v_cache_bf16, const int32_t* lengths,
-                               const int32_t* seq_ids, int M, int n_q_heads, int n_kv_heads, int head_dim, int t_max,
+                               const int32_t* seq_ids, int M, int n_q_heads, int n_kv_heads, int head_dim, int n_seq, int t_max,
                                void* out_bf16, void* ws, size_t ws_bytes, void* stream) {
-    if (!attn_dims_ok(M, n_q_heads, n_kv_heads, head_dim, t_max)) return BITLINEAR_ERR_SHAPE;
+    if (!attn_dims_ok(M, n_q_heads, n_kv_heads, head_dim, t_max) || n_seq <= 0 || (long long)n_seq * t_max > (1ll << 30))
+        return BITLINEAR_ERR_SHAPE;
     if (M == 0) return BITLINEAR_OK;
     if (!q_bf16 || !k_cache_bf16 || !v_cache_bf16 || !lengths || !out_bf16) return BITLINEAR_ERR_NULL;
     if (!aligned16(q_bf16) || !aligned16(k_cache_bf16) || !aligned16(v_cache_bf16) || !aligned16(out_bf16)) return BITLINEAR_ERR_ALIGN;
     if (!ws || !aligned16(ws) || ws_bytes < bitlinear_attention_workspace_bytes(M, n_q_heads, n_kv_heads, head_dim, t_max))
         return BITLINEAR_ERR_WORKSPACE;
+    int sm_count = 0;
+    if (const int rc = device_sm_count(&sm_count)) return rc;
+    CUtensorMap map_k, map_v;
+    if (!make_cache_map(&map_k, k_cache_bf16, n_seq, t_max, n_kv_heads, head_dim) ||
+        !make_cache_map(&map_v, v_cache_bf16, n_seq, t_max, n_kv_heads, head_dim))
+        return BITLINEAR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int splits = attn_splits(t_max), group = n_q_heads / n_kv_heads;
+    const int splits = attn_splits(M, n_kv_heads, t_max, sm_count);
     const float scale = 1.0f / sqrtf((float)head_dim);
     const dim3 grid((unsigned)splits, (unsigned)n_kv_heads, (unsigned)M);
-    const __nv_bfloat16 *qp = static_cast<const __nv_bfloat16*>(q_bf16), *kp = static_cast<const __nv_bfloat16*>(k_cache_bf16),
-                        *vp = static_cast<const __nv_bfloat16*>(v_cache_bf16);
+    const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q_bf16);
     int* status = device_status_word();
     auto launch = [&](auto hd_tag) {
         constexpr int HD = decltype(hd_tag)::value;
+        if (!attn_opt_in<HD>()) return (int)BITLINEAR_ERR_CUDA;
         auto* part = static_cast<AttnPartial<HD>*>(ws);
-        attn_decode_partial_kernel<HD><<<grid, 32 * group, attn_smem_bytes<HD>(group), st>>>(qp, kp, vp, lengths, seq_ids, n_q_heads, n_kv_heads,
-                                                                                          t_max, splits, scale, part, status);
-        attn_decode_combine_kernel<HD><<<(unsigned)(M * n_q_heads), HD, 0, st>>>(part, lengths, n_q_heads, t_max, splits,
-                                                                               static_cast<__nv_bfloat16*>(out_bf16));
+        attn_decode_partial_kernel<HD><<<grid, 128, attn_smem_bytes<HD>(), st>>>(map_k, map_v, qp, lengths, seq_ids, n_q_heads,
+                                                                                          n_kv_heads, n_seq, t_max, splits, scale, part, status);
+        attn_decode_combine_kernel<HD><<<(unsigned)(M * n_q_heads), 128, 0, st>>>(part, lengths, seq_ids, n_q_heads, n_seq, t_max, splits,
+                                                                                static_cast<__nv_bfloat16*>(out_bf16));
+        return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
     };
-    if (head_dim == 128) launch(std::integral_constant<int, 128>{});
-    else launch(std::integral_constant<int, 64>{});
-    return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+    return head_dim == 128 ? launch(std::integral_constant<int, 128>{}) : launch(std::integral_constant<int, 64>{});
 }
 
 int bitlinear_lm_head(const void* x_bf16, const void* table_bf16, int M, int V, int K, float* logits, void* stream) {

@@ -20,6 +20,7 @@
 
 #include "common.cuh"
 #include "sm100_sync.cuh"
+#include "tensor_map.cuh"
 
 namespace bitlinear {
 
@@ -696,25 +697,6 @@ __global__ void __launch_bounds__(128, 1) int8_mma_rate_kernel(int n_mma, int* s
 }
 
 // ---- host side -----------------------------------------------------------------------------------
-
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn() {
-    static std::once_flag once;
-    static EncodeTiledFn fn = nullptr;
-    std::call_once(once, [] {
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        else
-            cudaGetLastError();
-    });
-    return fn;
-}
 
 // 2-D map over a row-major [rows][K] byte matrix; box = box_rows x 128 bytes, 128-byte swizzle.
 bool make_map(CUtensorMap* map, const void* base, int rows, int K, int box_rows) {

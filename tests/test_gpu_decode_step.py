@@ -137,7 +137,71 @@ def test_argument_checks():
     assert lib.bitlinear_lm_head(fake, fake, 1, 100, 250, fake, None) == 2
     assert lib.bitlinear_lm_head(None, fake, 1, 100, 256, fake, None) == 1
     assert lib.bitlinear_attention_workspace_bytes(1, 20, 5, 96, 128) == 0  # head_dim 64 or 128
-    assert lib.bitlinear_attention_decode(fake, fake, fake, fake, None, 1, 20, 6, 128, 128, fake, fake, 1 << 20, None) == 2
-    assert lib.bitlinear_attention_decode(fake, fake, fake, fake, None, 1, 20, 5, 128, 128, fake, fake, 16, None) == 4
-    assert lib.bitlinear_rope_kv(fake, fake, fake, fake, None, 1, 20, 5, 100, 500000.0, fake, fake, fake, 16, None) == 2
+    assert lib.bitlinear_attention_decode(fake, fake, fake, fake, None, 1, 20, 6, 128, 1, 128, fake, fake, 1 << 20, None) == 2
+    assert lib.bitlinear_attention_decode(fake, fake, fake, fake, None, 1, 20, 5, 128, 0, 128, fake, fake, 1 << 20, None) == 2
+    assert lib.bitlinear_attention_decode(fake, fake, fake, fake, None, 1, 20, 5, 128, 1, 128, fake, fake, 16, None) == 4
+    assert lib.bitlinear_rope_kv(fake, fake, fake, fake, None, 1, 20, 5, 100, 500000.0, fake, fake, fake, 1, 16, None) == 2
     assert lib.bitlinear_embed(fake, fake, 0, 10, 256, fake, None) == 0
+
+
+def test_whole_decode_step_stage_by_stage():
+    """One decoder layer + embedding + output head through DecodeStep; every stage is checked against the oracle applied
+    to the values the GPU fed into that stage (a quantiser between two stages would turn a last-bit difference of an
+    earlier floating-point stage into a different code, so the stages are not chained on the oracle side)."""
+    from paper_2504_12285_b200 import chain as gpu_chain
+
+    H, F, n_q, n_kv, hd, V, M, t_max = 256, 512, 4, 2, 64, 500, 3, 80
+    kv = n_kv * hd
+    mats, layer = {}, {}
+    for i, (name, n, k) in enumerate((("q", H, H), ("k", kv, H), ("v", kv, H), ("o", H, H), ("gate", F, H), ("up", F, H),
+                                      ("down", H, F))):
+        W = wl.latent_weights(n, k, 8100 + i)
+        packed, s_w = bl.bitlinear_pack_weights(W.to(DEV), wl.WEIGHT_EPS)
+        gain = wl.gain_random(k, 8200 + i)
+        layer[name] = (packed, s_w, gain.to(DEV))
+        mats[name] = (oracle.quantize_weights(W.numpy(), wl.WEIGHT_EPS), wl.bf16_bits(gain))
+    table = randn((V, H), 50).to(torch.bfloat16)
+    st = gpu_chain.DecodeStep([layer], table.to(DEV), M, t_max, H, F, n_q, n_kv, hd, wl.RMS_EPS, device=DEV)
+    # a context in the caches: sequence m has positions[m] earlier tokens
+    pos = np.array([0, 37, 79], np.int32)
+    st.k_cache[0].copy_(randn((M, t_max, kv), 51).to(torch.bfloat16))
+    st.v_cache[0].copy_(randn((M, t_max, kv), 52).to(torch.bfloat16))
+    st.set_positions(torch.from_numpy(pos).to(DEV))
+    ids = torch.tensor([7, 499, 123], dtype=torch.int32)
+    logits = st.step(ids.to(DEV))
+    torch.cuda.synchronize()
+    assert bl.bitlinear_poll_status() == 0
+
+    def bitlinear(name, x_bits):
+        ref = oracle.bitlinear_forward(x_bits, mats[name][1], wl.RMS_EPS, mats[name][0]["wq"], mats[name][0]["s_w"])
+        assert not ref["fragile"].any()
+        return ref["y"].astype(np.float64)
+
+    def close_f32(got, want):
+        assert np.all(np.abs(got.cpu().numpy().astype(np.float64) - want) <= 1e-6 * np.abs(want))
+
+    h0 = ds.embed(ids.numpy(), bits(table))
+    assert np.array_equal(bits(st.h_in), h0)
+    for name, buf in (("q", st.q), ("k", st.k), ("v", st.v)):
+        close_f32(buf, bitlinear(name, h0))
+    qg, kg, vg = (t.cpu().numpy() for t in (st.q, st.k, st.v))
+    q_ref, k_ref = ds.rope(qg, pos, n_q, hd), ds.rope(kg, pos, n_kv, hd)
+    slack = 2.0 ** -20 * max(np.abs(qg).max(), np.abs(kg).max()) * 2
+    assert np.all(np.abs(bf(bits(st.q_rot)) - q_ref) <= 2.0 ** -8 * np.abs(q_ref) + slack)
+    kc, vc = bits(st.k_cache[0]), bits(st.v_cache[0])
+    for m in range(M):
+        assert np.all(np.abs(bf(kc[m, pos[m]]) - k_ref[m]) <= 2.0 ** -8 * np.abs(k_ref[m]) + slack)
+        assert np.array_equal(vc[m, pos[m]], oracle.f32_to_bf16(vg[m]))
+        a_ref = ds.attention_decode(bits(st.q_rot)[m], kc[m], vc[m], int(pos[m]) + 1, n_q, n_kv, hd)
+        vmax = np.abs(bf(vc[m, :pos[m] + 1])).max()
+        assert np.all(np.abs(bf(bits(st.attn))[m] - a_ref) <= 2.0 ** -8 * np.abs(a_ref) + 1e-4 * vmax)
+    close_f32(st.o, bitlinear("o", bits(st.attn)))
+    h_mid = oracle.glue_residual(h0, st.o.cpu().numpy())
+    close_f32(st.g, bitlinear("gate", h_mid))
+    close_f32(st.u, bitlinear("up", h_mid))
+    close_f32(st.dn, bitlinear("down", oracle.glue_relu2(st.g.cpu().numpy(), st.u.cpu().numpy())))
+    h_end = oracle.glue_residual(h_mid, st.dn.cpu().numpy())
+    assert np.array_equal(bits(st.h_mid), h_end)
+    ref = ds.lm_head(h_end, bits(table))
+    bound = H * 2.0 ** -24 * (np.abs(bf(h_end)) @ np.abs(bf(bits(table))).T)
+    assert np.all(np.abs(logits.cpu().numpy().astype(np.float64) - ref) <= bound)
