@@ -404,21 +404,24 @@ int bitlinear_poll_status(void* stream);
  *   q [M][n_q*D], k, v [M][n_kv*D] fp32 (BitLinear outputs); positions [M] int32 (device); seq_ids [M] int32 (device)
  *   or NULL (one sequence).  Coordinate i of a head is paired with i + D/2, angle = position * rope_base^(-2i/D):
  *   (x_i, x_j) -> (x_i cos - x_j sin, x_j cos + x_i sin); angles in fp64, rotation in fp32, results rounded to bf16.
- *   q_out bf16 [M][n_q*D]; caches bf16 [n_seq][t_max][n_kv*D]: row positions[m] of sequence seq_ids[m] receives the
- *   rotated k and the unrotated v (positions outside 0 .. t_max-1 and sequences outside 0 .. n_seq-1 are not
- *   stored).  D a multiple of 8.
+ *   q_out bf16 [M][n_q*D]; caches bf16 [n_seq][n_kv][t_max][D] (the rows of one KV head of one sequence are
+ *   contiguous, so that attention streams a head's keys as one run of memory): row positions[m] of every head of
+ *   sequence seq_ids[m] receives the rotated k and the unrotated v (positions outside 0 .. t_max-1 and sequences
+ *   outside 0 .. n_seq-1 are not stored).  D a multiple of 8.
  * bitlinear_attention_decode: one query token per row against the first lengths[m] cache rows of its sequence.
  *   Query head h reads key/value head h / (n_q / n_kv); scores q.k / sqrt(D), softmax over the rows, weighted sum of
  *   the values, fp32 arithmetic, bf16 output [M][n_q*D] (the input of the o projection; zeros for a length <= 0 or
  *   a sequence outside 0 .. n_seq-1, lengths above t_max are taken as t_max).  D = 64 or 128, n_q / n_kv <= 8,
- *   n_seq * t_max <= 2^30, M <= 65535, all pointers 16-byte aligned; the caches are read through tensor maps
+ *   n_seq * n_kv * t_max <= 2^30, M <= 65535, all pointers 16-byte aligned; the caches are read through tensor maps
  *   encoded per call from their addresses and n_seq, t_max.  ws (device, 16-byte aligned, contents need not
  *   survive the call) at least bitlinear_attention_workspace_bytes(...) bytes (0 for unsupported sizes): up to 64
  *   partial results per token and query head.
  *   A copy that does not land within the wait limit ends the call's kernels and sets BITLINEAR_ERR_TIMEOUT in the
  *   status word (bitlinear_poll_status).
  * bitlinear_lm_head: logits[m][v] = sum_k x[m][k] * table[v][k], x bf16 [M][K] (M <= 16), table bf16 [V][K], fp32
- *   accumulation and output [M][V].  The table is streamed once per call.
+ *   accumulation and output [M][V].  The table is streamed once per call (one token: fp32 FMAs; 2 to 16 tokens: bf16
+ *   tensor-core products, which are exact, accumulated in fp32).  K a multiple of 8; x is staged in shared memory, so
+ *   K <= 7168 for M > 1 (BITLINEAR_ERR_SHAPE beyond).
  * bitlinear_embed: out[m] = table[ids[m]] (bf16 rows; ids outside 0 .. V-1 are clamped).
  */
 int bitlinear_rope_kv(const float* q, const float* k, const float* v, const int32_t* positions, const int32_t* seq_ids, int M,

@@ -484,23 +484,23 @@ def bitlinear_forward_batch_host(batch: ProblemBatch, x_host: torch.Tensor, x_de
     _check(rc, "bitlinear_forward_batch_host")
 
 
-def _cache_dims(k_cache, v_cache, width: int):
-    """(n_seq, t_max) of a key/value cache pair [n_seq, t_max, width] or [t_max, width]."""
-    if k_cache.shape != v_cache.shape or k_cache.dim() not in (2, 3) or k_cache.shape[-1] != width:
-        raise ValueError(f"caches must both be [n_seq, t_max, {width}] or [t_max, {width}]")
-    return (k_cache.shape[0] if k_cache.dim() == 3 else 1), k_cache.shape[-2]
+def _cache_dims(k_cache, v_cache, n_kv_heads: int, head_dim: int):
+    """(n_seq, t_max) of a key/value cache pair [n_seq, n_kv, t_max, D] or [n_kv, t_max, D]."""
+    if k_cache.shape != v_cache.shape or k_cache.dim() not in (3, 4) or tuple(k_cache.shape[-3::2]) != (n_kv_heads, head_dim):
+        raise ValueError(f"caches must both be [n_seq, {n_kv_heads}, t_max, {head_dim}] or [{n_kv_heads}, t_max, {head_dim}]")
+    return (k_cache.shape[0] if k_cache.dim() == 4 else 1), k_cache.shape[-2]
 
 
 def bitlinear_rope_kv(q, k, v, positions, k_cache, v_cache, n_q_heads: int, n_kv_heads: int, head_dim: int,
                       rope_base: float = 500000.0, seq_ids=None, q_out=None):
     """Rotate q, k (fp32 [M, heads * D]) at `positions` (int32 [M]); q -> bf16 (returned), k / v appended to the bf16
-    caches [n_seq, t_max, n_kv * D] (contiguous) at those positions."""
+    caches [n_seq, n_kv, t_max, D] (contiguous) at those positions."""
     _dev(q, torch.float32, "q"), _dev(k, torch.float32, "k"), _dev(v, torch.float32, "v")
     _dev(positions, torch.int32, "positions"), _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache")
     if seq_ids is not None:
         _dev(seq_ids, torch.int32, "seq_ids")
     M = q.shape[0]
-    n_seq, t_max = _cache_dims(k_cache, v_cache, n_kv_heads * head_dim)
+    n_seq, t_max = _cache_dims(k_cache, v_cache, n_kv_heads, head_dim)
     if q_out is None:
         q_out = torch.empty(M, n_q_heads * head_dim, dtype=torch.bfloat16, device=q.device)
     rc = lib().bitlinear_rope_kv(_ptr(q), _ptr(k), _ptr(v), _ptr(positions), _ptr(seq_ids), M, n_q_heads, n_kv_heads, head_dim,
@@ -521,7 +521,7 @@ def bitlinear_attention_decode(q, k_cache, v_cache, lengths, n_q_heads: int, n_k
     if seq_ids is not None:
         _dev(seq_ids, torch.int32, "seq_ids")
     M = q.shape[0]
-    n_seq, t_max = _cache_dims(k_cache, v_cache, n_kv_heads * head_dim)
+    n_seq, t_max = _cache_dims(k_cache, v_cache, n_kv_heads, head_dim)
     if out is None:
         out = torch.empty(M, n_q_heads * head_dim, dtype=torch.bfloat16, device=q.device)
     if ws is None:

@@ -90,8 +90,8 @@ class DecodeStep:
         self.g, self.u = torch.empty(M, ffn, **f32), torch.empty(M, ffn, **f32)
         self.dn = torch.empty(M, hidden, **f32)
         self.logits = torch.empty(M, embedding.shape[0], **f32)
-        self.k_cache = [torch.zeros(M, t_max, kv, **bf) for _ in layers]
-        self.v_cache = [torch.zeros(M, t_max, kv, **bf) for _ in layers]
+        self.k_cache = [torch.zeros(M, n_kv_heads, t_max, head_dim, **bf) for _ in layers]
+        self.v_cache = [torch.zeros(M, n_kv_heads, t_max, head_dim, **bf) for _ in layers]
         self.seq_ids = torch.arange(M, dtype=torch.int32, device=dev)
         self.positions = torch.zeros(M, dtype=torch.int32, device=dev)  # where this token goes in its sequence
         self.lengths = torch.ones(M, dtype=torch.int32, device=dev)     # cache rows attended to: positions + 1

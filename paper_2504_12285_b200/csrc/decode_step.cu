@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ 
                                                       double log2_base, __nv_bfloat16* __restrict__ q_out,
                                                       __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
                                                       int t_max) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int half = hd / 2;
     const int pairs_per_tok = (n_q + n_kv) * half;
     const int vals_per_tok = n_kv * hd;
@@ -59,7 +60,7 @@ __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ 
         if (!is_q && (pos < 0 || pos >= t_max || seq < 0 || seq >= n_seq)) return;  // a row outside the cache is not stored
         __nv_bfloat16* dst;
         if (is_q) dst = q_out + (size_t)m * n_q * hd + (size_t)head * hd;
-        else dst = k_cache + ((size_t)seq * t_max + pos) * vals_per_tok + (size_t)(head - n_q) * hd;
+        else dst = k_cache + (((size_t)seq * n_kv + (size_t)(head - n_q)) * t_max + pos) * hd;
         dst[i] = __float2bfloat16_rn(o_lo);
         dst[i + half] = __float2bfloat16_rn(o_hi);
     } else if (idx < n_rot + (long long)M * vals_per_tok) {
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ 
         const int m = (int)(j / vals_per_tok), e = (int)(j - (long long)m * vals_per_tok);
         const int seq = seq_ids ? seq_ids[m] : 0;
         if (positions[m] < 0 || positions[m] >= t_max || seq < 0 || seq >= n_seq) return;
-        v_cache[((size_t)seq * t_max + positions[m]) * vals_per_tok + e] =
+        v_cache[(((size_t)seq * n_kv + (size_t)(e / hd)) * t_max + positions[m]) * hd + (e % hd)] =
             __float2bfloat16_rn(v[(size_t)m * vals_per_tok + e]);
     }
 }
@@ -75,7 +76,7 @@ __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ 
 // ---------------------------------------------------------------------------------------------- decode attention
 
 constexpr int kAttnKeys = 64;       // cache rows per tile
-constexpr int kAttnStages = 3;      // tiles in flight per CTA
+constexpr int kAttnMaxStages = 3;   // tiles in flight per CTA (1 when every slice is a single tile)
 constexpr int kAttnMaxSplits = 64;  // partial results per (token, query head)
 
 // partial result of one slice of the cache for one (token, query head): weighted values, running maximum, sum of weights
@@ -86,8 +87,8 @@ struct __align__(16) AttnPartial {
 };
 
 template <int HD>
-constexpr size_t attn_smem_bytes() {
-    return 1024 /*alignment slack*/ + (size_t)kAttnStages * 2 * kAttnKeys * HD * 2 + 8 * kAttnStages + 8;
+constexpr size_t attn_smem_bytes(int stages) {
+    return 1024 /*alignment slack*/ + (size_t)stages * 2 * kAttnKeys * HD * 2 + 16 * kAttnMaxStages + 8;
 }
 
 // How the 64-row tiles of a token's live cache rows are dealt to the slices: `per` tiles each, `live` slices in use.
@@ -115,187 +116,238 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                  : "r"(addr));
 }
-// d += a * b, 16 x 8 x 16, bf16 operands, fp32 accumulation; rows 8 .. 15 of a are zero here (a1 = a3 = 0)
-__device__ __forceinline__ void mma_rows8(float (&d)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+// d += a * b, 16 x 8 x 16, bf16 operands, fp32 accumulation
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
         "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1));
+        : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// transpose of an 8 x 8 matrix of 16-bit elements held one row pair per lane (the layout ldmatrix delivers)
+__device__ __forceinline__ uint32_t movmatrix_t(uint32_t a) {
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
-// One CTA of four warps per (slice of the cache, KV head, token).  A slice is a run of 64-row tiles; each tile's key and
-// value rows of this KV head (64 x HD bf16 each) arrive in shared memory by tensor-map copies of 64 rows x 128 bytes
-// (128-byte swizzle), up to three tiles in flight, so every query head of the group reads the cache from HBM once.
-// The group's query heads (at most 8) are the rows of a 16-row tensor-core operand: warp w takes keys 16w .. 16w+15 of
-// every tile, S = Q K^T by mma.sync (bf16 x bf16 products are exact, fp32 accumulation), a running softmax per head in
-// fp32, and O += P V with the weights split into two bf16 parts (P = P_hi + P_lo, relative error 2^-17) so that the
-// tensor core's bf16 operand costs no accuracy.  The four warps' results are merged in shared memory at the end.
-// Slices past the token's length return at once and are not read by the combine kernel.  Rows of a tile past the
-// token's length are copied (they are inside the cache, or zero-filled past its end); their scores are discarded by a
-// select and their value rows are overwritten with zeros before use, so whatever bits they hold never enter a result.
+// One CTA per (slice of the cache, KV head, token): four consumer warps and one producer warp.  A slice is a run of
+// 64-row tiles; each tile's key and value rows of this KV head (64 x HD bf16 each) arrive in shared memory by
+// tensor-map copies of 64 rows x 128 bytes (128-byte swizzle; a head's rows are contiguous in the cache, so a tile is
+// 64 * HD * 2 contiguous bytes of HBM) issued by the producer into a ring of `stages` tiles
+// (full / empty barriers per stage), so every query head of the group reads the cache from HBM once.
+// Consumer warp w takes keys 16w .. 16w+15 of every tile and works on the transposed problem, which wastes the least
+// of the 16 x 8 x 16 tensor-core shape on a group of at most 8 heads:
+//   S^T (16 keys x 8 heads) = K (16 x HD) Q^T   - K fragments by ldmatrix, Q^T from registers; bf16 products are exact,
+//                                                 accumulation in fp32;
+//   a running softmax per head in fp32 (the keys of a head sit in one accumulator column);
+//   O^T (HD x 8 heads) += V^T (HD x 16 keys) P  - V^T fragments by ldmatrix.trans; P is the exponentiated S^T,
+//                                                 split into two bf16 parts (P = P_hi + P_lo, relative error 2^-17)
+//                                                 so that the bf16 operand costs no accuracy, and transposed into
+//                                                 the B-operand layout by movmatrix.
+// The four warps' results are merged in shared memory at the end.  Slices past the token's length return at once and
+// are not read by the combine kernel.  Rows of a tile past the token's length are copied (they are inside the cache,
+// or zero-filled past its end); their scores are discarded by a select and their value rows are overwritten with zeros
+// before use, so whatever bits they hold never enter a result.
 template <int HD>
-__global__ void __launch_bounds__(128) attn_decode_partial_kernel(const __grid_constant__ CUtensorMap map_k,
+__global__ void __launch_bounds__(160) attn_decode_partial_kernel(const __grid_constant__ CUtensorMap map_k,
                                                                   const __grid_constant__ CUtensorMap map_v,
                                                                   const __nv_bfloat16* __restrict__ q, const int* __restrict__ lengths,
                                                                   const int* __restrict__ seq_ids, int n_q, int n_kv, int n_seq, int t_max,
-                                                                  int splits, float scale, AttnPartial<HD>* __restrict__ part,
-                                                                  int* __restrict__ status_word) {
-    constexpr int HALVES = HD / 64;                 // 128-byte column blocks of a row
+                                                                  int splits, int stages, float scale,
+                                                                  AttnPartial<HD>* __restrict__ part, int* __restrict__ status_word) {
+    constexpr int HALVES = HD / 64;                   // 128-byte column blocks of a row
     constexpr uint32_t kHalfBytes = kAttnKeys * 128;  // one block of a tile: 64 rows x 128 bytes
     constexpr uint32_t kTileBytes = HALVES * kHalfBytes;
-    constexpr int KS = HD / 16;  // k-steps of Q K^T
-    constexpr int NT = HD / 8;   // 8-column tiles of O
-    constexpr int OPAD = HD + 8; // row stride of the merge buffer (floats)
+    constexpr int KS = HD / 16;    // k-steps of K Q^T, and 16-row tiles of O^T
+    constexpr int OPAD = HD + 4;   // row stride of the merge buffer (floats)
     extern __shared__ uint8_t attn_smem_raw[];
-    const int split = blockIdx.x, g = blockIdx.y, m = blockIdx.z;
+    const int split = blockIdx.x, kvh = blockIdx.y, m = blockIdx.z;
     const int group = n_q / n_kv;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int r = lane >> 2, qd = lane & 3;  // this lane's row (query head of the group) and column pair in a fragment
+    const int g = lane >> 2, qd = lane & 3;  // fragment coordinates of this lane
+    uint8_t* smem = attn_smem_raw + ((1024u - (smem_u32(attn_smem_raw) & 1023u)) & 1023u);
+    const uint32_t ring_s = smem_u32(smem);  // [stage][K, V][block][64 rows][128 bytes, swizzled]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)stages * 2 * kTileBytes);  // full[3], empty[3]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kAttnMaxStages);
+    const uint32_t full_s = smem_u32(bars), empty_s = full_s + 8u * kAttnMaxStages;
+    // what needs no global data comes first: this launch is a programmatic dependent and may begin while the launch
+    // before it (rotary embedding + cache append, or whatever wrote the lengths) is still running
+    if (threadIdx.x == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_k) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_v) : "memory");
+        *abort_flag = 0;
+        for (int st = 0; st < stages; ++st) {
+            mbar_init(full_s + 8u * st, 1);
+            mbar_init(empty_s + 8u * st, 4);  // one arrival per consumer warp
+        }
+        mbar_init_fence();
+    }
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // nothing is read from global memory before this
     const int seq = seq_ids ? seq_ids[m] : 0;
     const int len = (seq >= 0 && seq < n_seq) ? min(max(lengths[m], 0), t_max) : 0;
     const AttnSlices sl = attn_slices(len, splits);
     if (split >= sl.live) return;  // the whole CTA: nothing of this slice is live
     const int tile0 = split * sl.per;
     const int n_tiles = min(sl.per, (len + kAttnKeys - 1) / kAttnKeys - tile0);
-
-    uint8_t* smem = attn_smem_raw + ((1024u - (smem_u32(attn_smem_raw) & 1023u)) & 1023u);
-    const uint32_t ring_s = smem_u32(smem);  // [stage][K, V][block][64 rows][128 bytes, swizzled]
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)kAttnStages * 2 * kTileBytes);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kAttnStages);
-    const uint32_t bar_s = smem_u32(bars);
-
-    const int row0 = seq * t_max + tile0 * kAttnKeys;
-    auto issue = [&](int i) {  // one thread: tile i of the slice into stage i % kAttnStages
-        const uint32_t st = (uint32_t)(i % kAttnStages), dst = ring_s + st * 2u * kTileBytes, bar = bar_s + 8u * st;
-        mbar_expect_tx(bar, 2u * kTileBytes);
-#pragma unroll
-        for (int hf = 0; hf < HALVES; ++hf) {
-            tma_tile_2d(dst + hf * kHalfBytes, &map_k, g * HD + hf * 64, row0 + i * kAttnKeys, bar);
-            tma_tile_2d(dst + kTileBytes + hf * kHalfBytes, &map_v, g * HD + hf * 64, row0 + i * kAttnKeys, bar);
-        }
-    };
-    if (threadIdx.x == 0) {
-        *abort_flag = 0;
-        for (int st = 0; st < kAttnStages; ++st) mbar_init(bar_s + 8u * st, 1);
-        mbar_init_fence();
-        for (int i = 0; i < min(kAttnStages, n_tiles); ++i) issue(i);
-    }
-    // the group's queries as the A operand: row r = head g * group + r (zero rows past the group), two registers per k-step
-    uint32_t qa[KS][2];
-    {
-        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)m * n_q + (size_t)g * group + min(r, group - 1)) * HD);
-#pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            qa[ks][0] = r < group ? qrow[8 * ks + qd] : 0u;
-            qa[ks][1] = r < group ? qrow[8 * ks + 4 + qd] : 0u;
-        }
-    }
+    // the merge kernel may be scheduled now; it waits for this whole grid before it reads a partial result
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     __syncthreads();  // barriers initialised, abort flag cleared
 
-    float m_run = -INFINITY, l_run = 0.0f;  // of row r over this warp's keys (the four lanes of a quad agree)
-    float o[NT][4];
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.0f, 0.0f};  // heads 2qd, 2qd+1 over this warp's keys
+    float o[KS][4];  // O^T: rows 16mt + g (+8), columns heads 2qd, 2qd+1
 #pragma unroll
-    for (int d = 0; d < NT; ++d) o[d][0] = o[d][1] = o[d][2] = o[d][3] = 0.0f;
-    const int kb = warp * 16;                // this warp's keys of a tile
-    const int mi = lane >> 3, mr = lane & 7; // the matrix and row this lane addresses for ldmatrix
+    for (int mt = 0; mt < KS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.0f;
 
-    for (int i = 0; i < n_tiles; ++i) {
-        const uint32_t st = (uint32_t)(i % kAttnStages);
-        const bool ok = mbar_wait(bar_s + 8u * st, (uint32_t)(i / kAttnStages) & 1u, abort_flag);
-        const int n = min(kAttnKeys, len - (tile0 + i) * kAttnKeys);  // live rows of the tile, >= 1
-        if (ok && kb < n) {
-            const uint32_t kbase = ring_s + st * 2u * kTileBytes, vbase = kbase + kTileBytes;
-            if (n < kb + 16) {  // the ragged end: zero this warp's dead value rows
-                for (int idx = lane; idx < (kb + 16 - n) * HALVES * 8; idx += 32) {
-                    const int row = n + idx / (HALVES * 8), c = idx % (HALVES * 8);
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + (c >> 3) * kHalfBytes + row * 128 + (c & 7) * 16), "r"(0u)
-                                 : "memory");
+    if (warp == 4) {
+        // ---- producer: one lane feeds the ring
+        if (lane == 0) {
+            const int row0 = (seq * n_kv + kvh) * t_max + tile0 * kAttnKeys;  // this head's rows are contiguous
+            for (int i = 0; i < n_tiles; ++i) {
+                const uint32_t st = (uint32_t)(i % stages), dst = ring_s + st * 2u * kTileBytes, bar = full_s + 8u * st;
+                if (i >= stages && !mbar_wait(empty_s + 8u * st, (uint32_t)(i / stages - 1) & 1u, abort_flag)) break;
+                mbar_expect_tx(bar, 2u * kTileBytes);
+#pragma unroll
+                for (int hf = 0; hf < HALVES; ++hf) {
+                    tma_tile_2d(dst + hf * kHalfBytes, &map_k, hf * 64, row0 + i * kAttnKeys, bar);
+                    tma_tile_2d(dst + kTileBytes + hf * kHalfBytes, &map_v, hf * 64, row0 + i * kAttnKeys, bar);
                 }
-                __syncwarp();
-            }
-            // S = Q K^T for keys kb .. kb+15: two 8-key column tiles
-            float s[2][4];
-#pragma unroll
-            for (int j = 0; j < 2; ++j) s[j][0] = s[j][1] = s[j][2] = s[j][3] = 0.0f;
-#pragma unroll
-            for (int ks = 0; ks < KS; ++ks) {
-                // matrices: (keys 0-7, chunk c), (keys 0-7, c+1), (keys 8-15, c), (keys 8-15, c+1)
-                const int key = kb + 8 * (mi >> 1) + mr, chunk = ((2 * ks) & 7) + (mi & 1);
-                uint32_t b[4];
-                ldsm_x4(kbase + (ks >> 2) * kHalfBytes + key * 128 + ((chunk ^ mr) << 4), b);
-                mma_rows8(s[0], qa[ks][0], qa[ks][1], b[0], b[1]);
-                mma_rows8(s[1], qa[ks][0], qa[ks][1], b[2], b[3]);
-            }
-            // running softmax of row r; this lane holds keys kb + 8j + 2qd + {0, 1}
-            float sv[4];
-#pragma unroll
-            for (int j = 0; j < 2; ++j)
-#pragma unroll
-                for (int e = 0; e < 2; ++e) sv[2 * j + e] = (kb + 8 * j + 2 * qd + e < n) ? s[j][e] * scale : -INFINITY;
-            float mt = fmaxf(fmaxf(sv[0], sv[1]), fmaxf(sv[2], sv[3]));
-            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 1));
-            mt = fmaxf(mt, __shfl_xor_sync(0xffffffffu, mt, 2));
-            const float m_new = fmaxf(m_run, mt);    // finite: key kb is live
-            const float corr = expf(m_run - m_new);  // expf(-inf) = 0 the first time
-            float pv[4], lt = 0.0f;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                pv[e] = expf(sv[e] - m_new);  // 0 for a dead key
-                lt += pv[e];
-            }
-            lt += __shfl_xor_sync(0xffffffffu, lt, 1);
-            lt += __shfl_xor_sync(0xffffffffu, lt, 2);
-            l_run = fmaf(l_run, corr, lt);
-            m_run = m_new;
-            // P as the A operand of P V: its fragment layout is the accumulator layout of S
-            float ph[4];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) ph[e] = __bfloat162float(__float2bfloat16_rn(pv[e]));
-            const uint32_t a0h = pack_bf16(ph[0], ph[1]), a2h = pack_bf16(ph[2], ph[3]);
-            const uint32_t a0l = pack_bf16(pv[0] - ph[0], pv[1] - ph[1]), a2l = pack_bf16(pv[2] - ph[2], pv[3] - ph[3]);
-#pragma unroll
-            for (int d = 0; d < NT; ++d) {
-                o[d][0] *= corr;
-                o[d][1] *= corr;
-            }
-#pragma unroll
-            for (int d = 0; d < NT; d += 2) {
-                // matrices (transposed on load): (keys 0-7, chunk d), (keys 8-15, d), (keys 0-7, d+1), (keys 8-15, d+1)
-                const int key = kb + 8 * (mi & 1) + mr, chunk = (d & 7) + (mi >> 1);
-                uint32_t b[4];
-                ldsm_x4_t(vbase + (d >> 3) * kHalfBytes + key * 128 + ((chunk ^ mr) << 4), b);
-                mma_rows8(o[d], a0h, a2h, b[0], b[1]);
-                mma_rows8(o[d], a0l, a2l, b[0], b[1]);
-                mma_rows8(o[d + 1], a0h, a2h, b[2], b[3]);
-                mma_rows8(o[d + 1], a0l, a2l, b[2], b[3]);
             }
         }
-        if (!__syncthreads_and(ok)) break;  // every warp is done with the stage - or the CTA gives up together
-        if (threadIdx.x == 0 && i + kAttnStages < n_tiles) issue(i + kAttnStages);
+    } else {
+        // ---- consumers
+        // Q^T as the B operand: column g = head kvh * group + g (zero columns past the group), two registers per k-step
+        uint32_t qb[KS][2];
+        {
+            const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)m * n_q + (size_t)kvh * group + min(g, group - 1)) * HD);
+#pragma unroll
+            for (int ks = 0; ks < KS; ++ks) {
+                qb[ks][0] = g < group ? qrow[8 * ks + qd] : 0u;
+                qb[ks][1] = g < group ? qrow[8 * ks + 4 + qd] : 0u;
+            }
+        }
+        const int kb = warp * 16;                 // this warp's keys of a tile
+        const int mi = lane >> 3, mr = lane & 7;  // the matrix and row this lane addresses for ldmatrix
+        for (int i = 0; i < n_tiles; ++i) {
+            const uint32_t st = (uint32_t)(i % stages);
+            if (!mbar_wait(full_s + 8u * st, (uint32_t)(i / stages) & 1u, abort_flag)) break;
+            const int n = min(kAttnKeys, len - (tile0 + i) * kAttnKeys);  // live rows of the tile, >= 1
+            if (kb < n) {
+                const uint32_t kbase = ring_s + st * 2u * kTileBytes, vbase = kbase + kTileBytes;
+                if (n < kb + 16) {  // the ragged end: zero this warp's dead value rows
+                    for (int idx = lane; idx < (kb + 16 - n) * HALVES * 8; idx += 32) {
+                        const int row = n + idx / (HALVES * 8), c = idx % (HALVES * 8);
+                        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(vbase + (c >> 3) * kHalfBytes + row * 128 + (c & 7) * 16),
+                                     "r"(0u)
+                                     : "memory");
+                    }
+                    __syncwarp();
+                }
+                // this lane's row of the four 8 x 8 blocks a ldmatrix.x4 fetches: keys kb + 8 (mi & 1) + mr, 16-byte chunk
+                // (mi >> 1) of the pair of chunks in turn - the same addressing for K (plain) and V (transposed)
+                const uint32_t row_off = (uint32_t)(kb + 8 * (mi & 1) + mr) * 128u;
+                // S^T = K Q^T, two accumulators to halve the dependent chain
+                float s0[4] = {0.0f, 0.0f, 0.0f, 0.0f}, s1[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int chunk = ((2 * ks) & 7) + (mi >> 1);
+                    uint32_t a[4];  // a0: keys 0-7, dims 0-7 of the step; a1: keys 8-15; a2, a3: dims 8-15
+                    ldsm_x4(kbase + (ks >> 2) * kHalfBytes + row_off + ((chunk ^ mr) << 4), a);
+                    if (ks & 1) mma_bf16(s1, a, qb[ks][0], qb[ks][1]);
+                    else mma_bf16(s0, a, qb[ks][0], qb[ks][1]);
+                }
+                // s[0], s[1]: key kb + g, heads 2qd, 2qd+1;  s[2], s[3]: key kb + g + 8
+                const bool live_lo = kb + g < n, live_hi = kb + g + 8 < n;
+                float sv[4];
+                sv[0] = live_lo ? (s0[0] + s1[0]) * scale : -INFINITY;  // a dead row may hold anything: selected away
+                sv[1] = live_lo ? (s0[1] + s1[1]) * scale : -INFINITY;
+                sv[2] = live_hi ? (s0[2] + s1[2]) * scale : -INFINITY;
+                sv[3] = live_hi ? (s0[3] + s1[3]) * scale : -INFINITY;
+                float mt0 = fmaxf(sv[0], sv[2]), mt1 = fmaxf(sv[1], sv[3]);
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    mt0 = fmaxf(mt0, __shfl_xor_sync(0xffffffffu, mt0, off));
+                    mt1 = fmaxf(mt1, __shfl_xor_sync(0xffffffffu, mt1, off));
+                }
+                const float mn0 = fmaxf(m_run[0], mt0), mn1 = fmaxf(m_run[1], mt1);  // finite: key kb is live
+                const float corr0 = expf(m_run[0] - mn0), corr1 = expf(m_run[1] - mn1);  // expf(-inf) = 0 the first time
+                float pv[4];
+                pv[0] = expf(sv[0] - mn0);  // 0 for a dead key
+                pv[1] = expf(sv[1] - mn1);
+                pv[2] = expf(sv[2] - mn0);
+                pv[3] = expf(sv[3] - mn1);
+                float lt0 = pv[0] + pv[2], lt1 = pv[1] + pv[3];
+#pragma unroll
+                for (int off = 4; off < 32; off <<= 1) {
+                    lt0 += __shfl_xor_sync(0xffffffffu, lt0, off);
+                    lt1 += __shfl_xor_sync(0xffffffffu, lt1, off);
+                }
+                l_run[0] = fmaf(l_run[0], corr0, lt0);
+                l_run[1] = fmaf(l_run[1], corr1, lt1);
+                m_run[0] = mn0;
+                m_run[1] = mn1;
+                // P (keys x heads) as the B operand: the accumulator holds it one row pair per lane, the operand wants
+                // it one column pair per lane - an 8 x 8 transpose per block of eight keys
+                float ph[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) ph[e] = __bfloat162float(__float2bfloat16_rn(pv[e]));
+                const uint32_t b0h = movmatrix_t(pack_bf16(ph[0], ph[1])), b1h = movmatrix_t(pack_bf16(ph[2], ph[3]));
+                const uint32_t b0l = movmatrix_t(pack_bf16(pv[0] - ph[0], pv[1] - ph[1]));
+                const uint32_t b1l = movmatrix_t(pack_bf16(pv[2] - ph[2], pv[3] - ph[3]));
+#pragma unroll
+                for (int mt = 0; mt < KS; ++mt) {
+                    o[mt][0] *= corr0;
+                    o[mt][1] *= corr1;
+                    o[mt][2] *= corr0;
+                    o[mt][3] *= corr1;
+                }
+#pragma unroll
+                for (int mt = 0; mt < KS; ++mt) {  // dims 16mt .. 16mt+15
+                    const int chunk = ((2 * mt) & 7) + (mi >> 1);
+                    uint32_t a[4];  // transposed on load: a0: dims 0-7 x keys 0-7; a1: dims 0-7 x keys 8-15; a2, a3: dims 8-15
+                    ldsm_x4_t(vbase + (mt >> 2) * kHalfBytes + row_off + ((chunk ^ mr) << 4), a);
+                    // the operand order is (dims 0-7, keys 0-7), (dims 8-15, keys 0-7), (dims 0-7, keys 8-15), (dims 8-15, keys 8-15)
+                    const uint32_t av[4] = {a[0], a[2], a[1], a[3]};
+                    mma_bf16(o[mt], av, b0h, b1h);
+                    mma_bf16(o[mt], av, b0l, b1l);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_s + 8u * st);  // this warp is done with the stage
+        }
     }
+    __syncthreads();  // every copy that was issued has landed and been consumed - or the CTA is giving up
     if (*abort_flag) {
         if (threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_TIMEOUT);
         abort_drain();
         return;
     }
-    // merge the four warps (every copy has landed and been consumed: the ring is free)
-    float* om = reinterpret_cast<float*>(smem);  // [warp][row][OPAD]
-    float* mm = om + 4 * 8 * OPAD;               // [warp][row]
+    // merge the four consumer warps (the ring is free)
+    float* om = reinterpret_cast<float*>(smem);  // [warp][head][OPAD]
+    float* mm = om + 4 * 8 * OPAD;               // [warp][head]
     float* ll = mm + 32;
-    if (r < group) {
+    if (warp < 4) {
 #pragma unroll
-        for (int d = 0; d < NT; ++d) *reinterpret_cast<float2*>(om + (warp * 8 + r) * OPAD + 8 * d + 2 * qd) = make_float2(o[d][0], o[d][1]);
-        if (qd == 0) {
-            mm[warp * 8 + r] = m_run;
-            ll[warp * 8 + r] = l_run;
+        for (int e = 0; e < 2; ++e) {
+            const int head = 2 * qd + e;
+            if (head < group) {
+#pragma unroll
+                for (int mt = 0; mt < KS; ++mt) {
+                    om[(warp * 8 + head) * OPAD + 16 * mt + g] = o[mt][e];
+                    om[(warp * 8 + head) * OPAD + 16 * mt + g + 8] = o[mt][2 + e];
+                }
+                if (g == 0) {
+                    mm[warp * 8 + head] = m_run[e];
+                    ll[warp * 8 + head] = l_run[e];
+                }
+            }
         }
     }
     __syncthreads();
-    for (int idx = threadIdx.x; idx < group * HD; idx += 128) {
+    for (int idx = threadIdx.x; idx < group * HD; idx += blockDim.x) {
         const int row = idx / HD, d = idx - row * HD;
         float m_all = mm[row];
 #pragma unroll
@@ -307,7 +359,7 @@ __global__ void __launch_bounds__(128) attn_decode_partial_kernel(const __grid_c
             l = fmaf(ll[w * 8 + row], f, l);
             acc = fmaf(om[(w * 8 + row) * OPAD + d], f, acc);
         }
-        AttnPartial<HD>& dst = part[((size_t)m * n_q + (size_t)g * group + row) * splits + split];
+        AttnPartial<HD>& dst = part[((size_t)m * n_q + (size_t)kvh * group + row) * splits + split];
         dst.o[d] = acc;
         if (d == 0) { dst.m = m_all; dst.l = l; }
     }
@@ -324,12 +376,34 @@ __global__ void __launch_bounds__(128) attn_decode_combine_kernel(const AttnPart
     const size_t mh = blockIdx.x;  // token * n_q + head
     const int m = (int)(mh / n_q);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // the partial results come from the launch before this one
+    const AttnPartial<HD>* p = part + mh * splits;
+    // every load of the kernel is issued before the first result is needed, the token's length included: sixteen
+    // slots per warp and the maxima and sums of all slots, live or not (a slot that no slice wrote holds whatever the
+    // workspace held; it is discarded by a select, never multiplied)
+    float v[kAttnMaxSplits / 4][CPL];
+#pragma unroll
+    for (int i = 0; i < kAttnMaxSplits / 4; ++i) {
+        const float* po = p[min(warp + 4 * i, splits - 1)].o + lane * CPL;
+        if constexpr (CPL == 4) {
+            const float4 t = *reinterpret_cast<const float4*>(po);
+            v[i][0] = t.x, v[i][1] = t.y, v[i][2] = t.z, v[i][3] = t.w;
+        } else {
+            const float2 t = *reinterpret_cast<const float2*>(po);
+            v[i][0] = t.x, v[i][1] = t.y;
+        }
+    }
+    const float2 ml0 = *reinterpret_cast<const float2*>(&p[min(lane, splits - 1)].m);
+    const float2 ml1 = *reinterpret_cast<const float2*>(&p[min(lane + 32, splits - 1)].m);
     const int seq = seq_ids ? seq_ids[m] : 0;
     const int len = (seq >= 0 && seq < n_seq) ? min(max(lengths[m], 0), t_max) : 0;
     const int live = attn_slices(len, splits).live;  // <= splits <= 64
-    const AttnPartial<HD>* p = part + mh * splits;
-    const float m0 = lane < live ? p[lane].m : -INFINITY, m1 = lane + 32 < live ? p[lane + 32].m : -INFINITY;
-    const float l0 = lane < live ? p[lane].l : 0.0f, l1 = lane + 32 < live ? p[lane + 32].l : 0.0f;
+    if (live == 0) {  // block-uniform
+        for (int d = threadIdx.x; d < HD; d += blockDim.x) out[mh * HD + d] = __float2bfloat16_rn(0.0f);
+        return;
+    }
+    const float m0 = lane < live ? ml0.x : -INFINITY, m1 = lane + 32 < live ? ml1.x : -INFINITY;
+    const float l0 = lane < live ? ml0.y : 0.0f, l1 = lane + 32 < live ? ml1.y : 0.0f;
     float m_all = fmaxf(m0, m1);
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) m_all = fmaxf(m_all, __shfl_xor_sync(0xffffffffu, m_all, off));
@@ -340,30 +414,12 @@ __global__ void __launch_bounds__(128) attn_decode_combine_kernel(const AttnPart
     float acc[CPL];
 #pragma unroll
     for (int e = 0; e < CPL; ++e) acc[e] = 0.0f;
-    if (live == 0) {  // block-uniform
-        for (int d = threadIdx.x; d < HD; d += blockDim.x) out[mh * HD + d] = __float2bfloat16_rn(0.0f);
-        return;
-    }
-    // all sixteen loads of the warp first (a dead slot re-reads a live one and gets weight 0: no branch), then the sums
-    float v[kAttnMaxSplits / 4][CPL];
-#pragma unroll
-    for (int i = 0; i < kAttnMaxSplits / 4; ++i) {
-        const float* po = p[min(warp + 4 * i, live - 1)].o + lane * CPL;
-        if constexpr (CPL == 4) {
-            const float4 t = *reinterpret_cast<const float4*>(po);
-            v[i][0] = t.x, v[i][1] = t.y, v[i][2] = t.z, v[i][3] = t.w;
-        } else {
-            const float2 t = *reinterpret_cast<const float2*>(po);
-            v[i][0] = t.x, v[i][1] = t.y;
-        }
-    }
 #pragma unroll
     for (int i = 0; i < kAttnMaxSplits / 4; ++i) {
         const int s = warp + 4 * i;  // warp-uniform
-        const float fs = __shfl_sync(0xffffffffu, s < 32 ? f0 : f1, s & 31);
-        const float f = s < live ? fs : 0.0f;
+        const float f = __shfl_sync(0xffffffffu, s < 32 ? f0 : f1, s & 31);
 #pragma unroll
-        for (int e = 0; e < CPL; ++e) acc[e] = fmaf(v[i][e], f, acc[e]);
+        for (int e = 0; e < CPL; ++e) acc[e] = s < live ? fmaf(v[i][e], f, acc[e]) : acc[e];
     }
 #pragma unroll
     for (int e = 0; e < CPL; ++e) red[warp][lane * CPL + e] = acc[e];
@@ -422,6 +478,67 @@ __global__ void __launch_bounds__(256) lm_head_kernel(const __nv_bfloat16* __res
     }
 }
 
+// The output head for 2 .. 16 tokens on the tensor cores: the tokens are the 16 rows of the A operand (zero rows past M),
+// eight vocabulary rows are the columns of B.  A lane loads 16 bytes (eight consecutive k) of its vocabulary row straight
+// from global memory and uses them as the B registers of two mma.sync steps; since a dot product does not care about
+// the order of k, the k-slots of a step are simply those eight values of the four lanes that share a column, and the
+// A operand (x, staged in shared memory) is read with the same assignment.  The table is streamed once.
+template <bool HI_ROWS>  // tokens 8 .. 15 present
+__global__ void __launch_bounds__(512) lm_head_mma_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ table,
+                                                          int M, int V, int K, int x_stride, float* __restrict__ logits) {
+    extern __shared__ __align__(16) uint8_t xs_raw[];  // [16][x_stride bytes]: rows 64 bytes apart modulo 128
+    const int n_vec = K / 8, pad_vec = (K + 31) / 32 * 4;  // 16-byte chunks of a row, and up to the next 32 columns
+    for (int i = threadIdx.x; i < 16 * pad_vec; i += blockDim.x) {
+        const int m = i / pad_vec, c = i - m * pad_vec;
+        *reinterpret_cast<uint4*>(xs_raw + (size_t)m * x_stride + c * 16) =
+            (m < M && c < n_vec) ? reinterpret_cast<const uint4*>(x)[(size_t)m * n_vec + c] : make_uint4(0, 0, 0, 0);
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, sq = lane & 3;
+    const int warps = gridDim.x * (blockDim.x >> 5);
+    const uint8_t* xa = xs_raw + (size_t)g * x_stride + sq * 16;
+    const uint8_t* xb = xa + (size_t)8 * x_stride;
+    const int k_blocks = K / 32;  // whole 32-k blocks; K % 32 is handled by the tail below
+    for (int v0 = 8 * (blockIdx.x * (blockDim.x >> 5) + warp); v0 < V; v0 += 8 * warps) {
+        const uint4* row = reinterpret_cast<const uint4*>(table + (size_t)min(v0 + g, V - 1) * K) + sq;
+        float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+        auto step = [&](const uint4& b, int kb) {
+            const uint4 a = *reinterpret_cast<const uint4*>(xa + kb * 64);
+            uint4 a8 = make_uint4(0, 0, 0, 0);
+            if constexpr (HI_ROWS) a8 = *reinterpret_cast<const uint4*>(xb + kb * 64);
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                         : "r"(a.x), "r"(a8.x), "r"(a.y), "r"(a8.y), "r"(b.x), "r"(b.y));
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                         : "r"(a.z), "r"(a8.z), "r"(a.w), "r"(a8.w), "r"(b.z), "r"(b.w));
+        };
+        int kb = 0;
+        for (; kb + 8 <= k_blocks; kb += 8) {  // eight loads in flight per lane
+            uint4 b[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) b[u] = __ldcs(row + (kb + u) * 4);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) step(b[u], kb + u);
+        }
+        for (; kb < k_blocks; ++kb) step(__ldcs(row + kb * 4), kb);
+        if (K % 32) {  // 8, 16 or 24 columns left: the lanes whose chunk lies past the end contribute zeros
+            const uint4 b = sq * 8 < K % 32 ? __ldcs(row + kb * 4) : make_uint4(0, 0, 0, 0);
+            step(b, kb);  // the staged x row is zero-padded up to the next 32 columns
+        }
+        const int v = v0 + 2 * sq;
+        if (g < M) {
+            if (v < V) logits[(size_t)g * V + v] = c[0];
+            if (v + 1 < V) logits[(size_t)g * V + v + 1] = c[1];
+        }
+        if (HI_ROWS && g + 8 < M) {
+            if (v < V) logits[(size_t)(g + 8) * V + v] = c[2];
+            if (v + 1 < V) logits[(size_t)(g + 8) * V + v + 1] = c[3];
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256) embed_kernel(const int* __restrict__ ids, const __nv_bfloat16* __restrict__ table, int M,
                                                     int V, int K, __nv_bfloat16* __restrict__ out) {
     const int n_vec = K / 8;
@@ -436,18 +553,38 @@ __global__ void __launch_bounds__(256) embed_kernel(const int* __restrict__ ids,
 // partial results reserved per (token, query head): one per tile of the cache, 64 at most
 int attn_splits_max(int t_max) { return std::min(kAttnMaxSplits, (t_max + kAttnKeys - 1) / kAttnKeys); }
 
-// Slices per (token, KV head) for a launch: enough CTAs for four per SM, never more than the tiles of the cache.
-int attn_splits(int M, int n_kv, int t_max, int sm_count) {
-    const int want = (4 * sm_count + M * n_kv - 1) / (M * n_kv);
-    return std::max(1, std::min(attn_splits_max(t_max), want));
+// Launch shape: slices per (token, KV head) and tiles in flight per CTA.  When one CTA per tile fits on the GPU at once
+// (a ring of one tile, six CTAs per SM) every tile gets its own CTA.  Otherwise CTAs carry a two-tile ring (three per
+// SM) and the slice count is the one that fills whole waves of resident CTAs best.
+struct AttnPlan {
+    int splits, stages;
+};
+AttnPlan attn_plan(int M, int n_kv, int t_max, int sm_count) {
+    const long long pairs = (long long)M * n_kv;
+    const int tiles = (t_max + kAttnKeys - 1) / kAttnKeys, cap = std::min(kAttnMaxSplits, tiles);
+    if (tiles <= kAttnMaxSplits && pairs * tiles <= 6ll * sm_count) return {tiles, 1};
+    // the fewest waves of resident CTAs that are at least 85 % full (long slices: a CTA's start-up and its merge are paid
+    // once per slice), else the fullest
+    const long long slots = 3ll * sm_count;
+    int best = 1;
+    double best_util = 0.0;
+    for (int w = 1; w <= 4; ++w) {
+        const int s = (int)std::min<long long>(cap, w * slots / pairs);
+        if (s < 1) continue;
+        const long long ctas = pairs * s, waves = (ctas + slots - 1) / slots;
+        const double util = (double)ctas / (double)(waves * slots);
+        if (util > best_util + 1e-9) best = s, best_util = util;
+        if (util >= 0.85) break;
+    }
+    return {best, std::min(2, (tiles + best - 1) / best)};
 }
 
-// rows = every cache row of every sequence, columns = n_kv * hd; box = 64 rows x 64 columns (128 bytes), 128-byte swizzle
+// rows = the cache rows of every (sequence, KV head), columns = hd; box = 64 rows x 64 columns (128 bytes), 128-byte swizzle
 bool make_cache_map(CUtensorMap* map, const void* cache, int n_seq, int t_max, int n_kv, int hd) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)n_kv * hd, (cuuint64_t)n_seq * t_max};
-    const cuuint64_t strides[1] = {(cuuint64_t)n_kv * hd * 2};
+    const cuuint64_t dims[2] = {(cuuint64_t)hd, (cuuint64_t)n_seq * n_kv * t_max};
+    const cuuint64_t strides[1] = {(cuuint64_t)hd * 2};
     const cuuint32_t box[2] = {64, (cuuint32_t)kAttnKeys};
     const cuuint32_t estr[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(cache), dims, strides, box, estr,
@@ -468,7 +605,7 @@ bool attn_opt_in() {
     std::lock_guard<std::mutex> lock(mu);
     if (!done[dev]) {
         if (cudaFuncSetAttribute(attn_decode_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                 (int)attn_smem_bytes<HD>()) != cudaSuccess) {
+                                 (int)attn_smem_bytes<HD>(kAttnMaxStages)) != cudaSuccess) {
             cudaGetLastError();
             return false;
         }
@@ -512,7 +649,7 @@ size_t bitlinear_attention_workspace_bytes(int M, int n_q_heads, int n_kv_heads,
 int bitlinear_attention_decode(const void* q_bf16, const void* k_cache_bf16, const void* v_cache_bf16, const int32_t* lengths,
                                const int32_t* seq_ids, int M, int n_q_heads, int n_kv_heads, int head_dim, int n_seq, int t_max,
                                void* out_bf16, void* ws, size_t ws_bytes, void* stream) {
-    if (!attn_dims_ok(M, n_q_heads, n_kv_heads, head_dim, t_max) || n_seq <= 0 || (long long)n_seq * t_max > (1ll << 30))
+    if (!attn_dims_ok(M, n_q_heads, n_kv_heads, head_dim, t_max) || n_seq <= 0 || (long long)n_seq * n_kv_heads * t_max > (1ll << 30))
         return BITLINEAR_ERR_SHAPE;
     if (M == 0) return BITLINEAR_OK;
     if (!q_bf16 || !k_cache_bf16 || !v_cache_bf16 || !lengths || !out_bf16) return BITLINEAR_ERR_NULL;
@@ -526,20 +663,40 @@ int bitlinear_attention_decode(const void* q_bf16, const void* k_cache_bf16, con
         !make_cache_map(&map_v, v_cache_bf16, n_seq, t_max, n_kv_heads, head_dim))
         return BITLINEAR_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int splits = attn_splits(M, n_kv_heads, t_max, sm_count);
+    const AttnPlan plan = attn_plan(M, n_kv_heads, t_max, sm_count);
     const float scale = 1.0f / sqrtf((float)head_dim);
-    const dim3 grid((unsigned)splits, (unsigned)n_kv_heads, (unsigned)M);
     const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q_bf16);
     int* status = device_status_word();
+    // both kernels are programmatic dependents of the launch before them: they may be scheduled while it drains, and
+    // call griddepcontrol.wait before reading anything
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
     auto launch = [&](auto hd_tag) {
         constexpr int HD = decltype(hd_tag)::value;
         if (!attn_opt_in<HD>()) return (int)BITLINEAR_ERR_CUDA;
         auto* part = static_cast<AttnPartial<HD>*>(ws);
-        attn_decode_partial_kernel<HD><<<grid, 128, attn_smem_bytes<HD>(), st>>>(map_k, map_v, qp, lengths, seq_ids, n_q_heads,
-                                                                                          n_kv_heads, n_seq, t_max, splits, scale, part, status);
-        attn_decode_combine_kernel<HD><<<(unsigned)(M * n_q_heads), 128, 0, st>>>(part, lengths, seq_ids, n_q_heads, n_seq, t_max, splits,
-                                                                                static_cast<__nv_bfloat16*>(out_bf16));
-        return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)plan.splits, (unsigned)n_kv_heads, (unsigned)M);
+        cfg.blockDim = dim3(160);
+        cfg.dynamicSmemBytes = attn_smem_bytes<HD>(plan.stages);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, attn_decode_partial_kernel<HD>, map_k, map_v, qp, lengths, seq_ids, n_q_heads, n_kv_heads, n_seq,
+                               t_max, plan.splits, plan.stages, scale, part, status) != cudaSuccess) {
+            cudaGetLastError();
+            return (int)BITLINEAR_ERR_CUDA;
+        }
+        cfg.gridDim = dim3((unsigned)(M * n_q_heads));
+        cfg.blockDim = dim3(128);
+        cfg.dynamicSmemBytes = 0;
+        if (cudaLaunchKernelEx(&cfg, attn_decode_combine_kernel<HD>, (const AttnPartial<HD>*)part, lengths, seq_ids, n_q_heads, n_seq,
+                               t_max, plan.splits, static_cast<__nv_bfloat16*>(out_bf16)) != cudaSuccess) {
+            cudaGetLastError();
+            return (int)BITLINEAR_ERR_CUDA;
+        }
+        return (int)BITLINEAR_OK;
     };
     return head_dim == 128 ? launch(std::integral_constant<int, 128>{}) : launch(std::integral_constant<int, 64>{});
 }
@@ -553,21 +710,22 @@ int bitlinear_lm_head(const void* x_bf16, const void* table_bf16, int M, int V, 
     if (const int rc = device_sm_count(&sm_count)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __nv_bfloat16 *xp = static_cast<const __nv_bfloat16*>(x_bf16), *tp = static_cast<const __nv_bfloat16*>(table_bf16);
-    const unsigned grid = (unsigned)(sm_count * 4);
-    auto launch = [&](auto kernel, int mt) {
-        const size_t smem = (size_t)mt * K * 2;
+    auto launch = [&](auto kernel, unsigned grid, unsigned threads, size_t smem, auto... args) {
         if (smem > 48 * 1024 && cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
             cudaGetLastError();
-            return (int)BITLINEAR_ERR_SHAPE;
+            return (int)BITLINEAR_ERR_SHAPE;  // K too large for the staged activations
         }
-        kernel<<<grid, 256, smem, st>>>(xp, tp, M, V, K, logits);
+        kernel<<<grid, threads, smem, st>>>(args...);
         return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
     };
-    if (M == 1) return launch(lm_head_kernel<1>, 1);
-    if (M <= 2) return launch(lm_head_kernel<2>, 2);
-    if (M <= 4) return launch(lm_head_kernel<4>, 4);
-    if (M <= 8) return launch(lm_head_kernel<8>, 8);
-    return launch(lm_head_kernel<16>, 16);
+    if (M == 1) return launch(lm_head_kernel<1>, (unsigned)(sm_count * 4), 256u, (size_t)K * 2, xp, tp, M, V, K, logits);
+    // rows of the staged x: K rounded up to 32 columns (zero-filled), 64 bytes apart modulo 128 so that the two rows a
+    // quarter-warp reads together fall into different halves of the banks
+    const int x_stride = ((K + 31) / 32 * 64 + 127) / 128 * 128 + 64;
+    const size_t smem = (size_t)16 * x_stride;
+    const unsigned grid = (unsigned)(sm_count * 2);
+    return M <= 8 ? launch(lm_head_mma_kernel<false>, grid, 512u, smem, xp, tp, M, V, K, x_stride, logits)
+                  : launch(lm_head_mma_kernel<true>, grid, 512u, smem, xp, tp, M, V, K, x_stride, logits);
 }
 
 int bitlinear_embed(const int32_t* ids, const void* table_bf16, int M, int V, int K, void* out_bf16, void* stream) {

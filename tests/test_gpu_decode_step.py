@@ -22,6 +22,18 @@ def bf(a):
     return oracle.bf16_to_f32(a).astype(np.float64)
 
 
+def cache_to_dev(t, n_kv, hd):
+    """[n_seq, t_max, n_kv * hd] (one row per position, as the oracle reads it) -> the library's [n_seq, n_kv, t_max, hd]."""
+    n_seq, t_max, _ = t.shape
+    return t.view(n_seq, t_max, n_kv, hd).permute(0, 2, 1, 3).contiguous().to(DEV)
+
+
+def cache_bits(c):
+    """The library's [n_seq, n_kv, t_max, hd] cache -> bf16 bit patterns [n_seq, t_max, n_kv * hd]."""
+    n_seq, n_kv, t_max, hd = c.shape
+    return bits(c.permute(0, 2, 1, 3).reshape(n_seq, t_max, n_kv * hd).contiguous())
+
+
 def randn(shape, seed, scale=1.0):
     return (torch.randn(*shape, generator=torch.Generator().manual_seed(seed), dtype=torch.float32) * scale).contiguous()
 
@@ -34,7 +46,7 @@ def test_rope_and_cache_append(M, n_q, n_kv, hd):
     pos = rng.choice(t_max, M, replace=False).astype(np.int32)  # distinct rows, up to the end of the cache
     pos[0] = 0
     seq = rng.integers(0, n_seq, M).astype(np.int32)
-    kc = torch.zeros(n_seq, t_max, n_kv * hd, dtype=torch.bfloat16, device=DEV)
+    kc = torch.zeros(n_seq, n_kv, t_max, hd, dtype=torch.bfloat16, device=DEV)
     vc = torch.zeros_like(kc)
     q_out = bl.bitlinear_rope_kv(q.to(DEV), k.to(DEV), v.to(DEV), torch.from_numpy(pos).to(DEV), kc, vc, n_q, n_kv, hd,
                                  seq_ids=torch.from_numpy(seq).to(DEV))
@@ -53,7 +65,7 @@ def test_rope_and_cache_append(M, n_q, n_kv, hd):
 
     close(bits(q_out), q_ref, pair_norm(q.numpy(), n_q))
     assert np.array_equal(bits(q_out)[0], oracle.f32_to_bf16(q.numpy()[0]))  # position 0: the identity, bit for bit
-    kc_h, vc_h = bits(kc), bits(vc)
+    kc_h, vc_h = cache_bits(kc), cache_bits(vc)
     for m in range(M):
         close(kc_h[seq[m], pos[m]][None], k_ref[m][None], pair_norm(k.numpy(), n_kv)[m][None])
         assert np.array_equal(vc_h[seq[m], pos[m]], oracle.f32_to_bf16(v.numpy()[m]))  # values are stored unrotated
@@ -77,7 +89,8 @@ def test_attention_decode(n_q, n_kv, hd, lengths):
     vc = randn((n_seq, t_max, n_kv * hd), 11).to(torch.bfloat16)
     q = randn((M, n_q * hd), 12, 2.0).to(torch.bfloat16)  # scores with a standard deviation of about 2: a peaked softmax
     seq = (np.arange(M) % n_seq).astype(np.int32)
-    out = bl.bitlinear_attention_decode(q.to(DEV), kc.to(DEV), vc.to(DEV), torch.tensor(lengths, dtype=torch.int32, device=DEV),
+    out = bl.bitlinear_attention_decode(q.to(DEV), cache_to_dev(kc, n_kv, hd), cache_to_dev(vc, n_kv, hd),
+                                        torch.tensor(lengths, dtype=torch.int32, device=DEV),
                                         n_q, n_kv, hd, seq_ids=torch.from_numpy(seq).to(DEV))
     torch.cuda.synchronize()
     got = bf(bits(out))
@@ -97,7 +110,8 @@ def test_attention_hand_cases():
     lengths = torch.tensor([1, 25], dtype=torch.int32, device=DEV)
     q = torch.zeros(2, n_q * hd, dtype=torch.bfloat16)
     q[0] = randn((n_q * hd,), 22).to(torch.bfloat16)
-    out = bf(bits(bl.bitlinear_attention_decode(q.to(DEV), kc.to(DEV), vc.to(DEV), lengths, n_q, n_kv, hd)))
+    out = bf(bits(bl.bitlinear_attention_decode(q.to(DEV), cache_to_dev(kc, n_kv, hd), cache_to_dev(vc, n_kv, hd), lengths,
+                                                n_q, n_kv, hd)))
     v64 = bf(bits(vc))[0].reshape(T, n_kv, hd)
     # length 1: the first value row, whatever the query (exact: the weight is 1)
     assert np.array_equal(out[0].reshape(n_q, hd)[3], v64[0, 1])
@@ -106,7 +120,8 @@ def test_attention_hand_cases():
     assert np.all(np.abs(out[1].reshape(n_q, hd)[0] - want[0]) <= 2.0 ** -8 * np.abs(want[0]) + 1e-5)
 
 
-@pytest.mark.parametrize("M,V,K", [(1, 1000, 256), (3, 5000, 2560), (16, 2048, 2560), (1, 128256, 2560)])
+@pytest.mark.parametrize("M,V,K", [(1, 1000, 256), (3, 5000, 2560), (5, 1003, 264), (8, 777, 2560), (16, 2048, 2560), (1, 128256, 2560),
+                                   (16, 128256, 2560)])
 def test_lm_head(M, V, K):
     x = randn((M, K), 30).to(torch.bfloat16)
     table = randn((V, K), 31, 0.05).to(torch.bfloat16)
@@ -164,8 +179,8 @@ def test_whole_decode_step_stage_by_stage():
     st = gpu_chain.DecodeStep([layer], table.to(DEV), M, t_max, H, F, n_q, n_kv, hd, wl.RMS_EPS, device=DEV)
     # a context in the caches: sequence m has positions[m] earlier tokens
     pos = np.array([0, 37, 79], np.int32)
-    st.k_cache[0].copy_(randn((M, t_max, kv), 51).to(torch.bfloat16))
-    st.v_cache[0].copy_(randn((M, t_max, kv), 52).to(torch.bfloat16))
+    st.k_cache[0].copy_(cache_to_dev(randn((M, t_max, kv), 51).to(torch.bfloat16), n_kv, hd))
+    st.v_cache[0].copy_(cache_to_dev(randn((M, t_max, kv), 52).to(torch.bfloat16), n_kv, hd))
     st.set_positions(torch.from_numpy(pos).to(DEV))
     ids = torch.tensor([7, 499, 123], dtype=torch.int32)
     logits = st.step(ids.to(DEV))
@@ -188,7 +203,7 @@ def test_whole_decode_step_stage_by_stage():
     q_ref, k_ref = ds.rope(qg, pos, n_q, hd), ds.rope(kg, pos, n_kv, hd)
     slack = 2.0 ** -20 * max(np.abs(qg).max(), np.abs(kg).max()) * 2
     assert np.all(np.abs(bf(bits(st.q_rot)) - q_ref) <= 2.0 ** -8 * np.abs(q_ref) + slack)
-    kc, vc = bits(st.k_cache[0]), bits(st.v_cache[0])
+    kc, vc = cache_bits(st.k_cache[0]), cache_bits(st.v_cache[0])
     for m in range(M):
         assert np.all(np.abs(bf(kc[m, pos[m]]) - k_ref[m]) <= 2.0 ** -8 * np.abs(k_ref[m]) + slack)
         assert np.array_equal(vc[m, pos[m]], oracle.f32_to_bf16(vg[m]))

@@ -7,6 +7,8 @@ the C ABI, that it returns what bitlinear_forward returns, on two calls in a row
 finds the first call's leftovers in the shared array), and that sizes beyond the array are refused.
 It is named so that pytest collects it after every other test file.
 """
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -30,6 +32,8 @@ def test_static_forward_matches_workspace_forward_on_two_calls_in_a_row():
         gain = wl.gain_random(K, 7300 + i).to(DEV)
         want = bl.bitlinear_forward(x, gain, packed, s_w, N, wl.RMS_EPS, y_dtype=ydt)
         out = torch.full((M, N), float("nan"), dtype=ydt, device=DEV)  # the caller owns the output, as always
+        got = None    # the previous case's output would otherwise be released inside the measured window
+        gc.collect()  # nor may tensors of earlier tests that are only waiting for the collector
         torch.cuda.synchronize()
         held, free = torch.cuda.memory_allocated(), torch.cuda.mem_get_info()[0]
         got = bl.bitlinear_forward_static(x, gain, packed, s_w, N, wl.RMS_EPS, out=out)
