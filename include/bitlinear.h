@@ -204,6 +204,25 @@ int bitlinear_forward(const void* x_bf16, const void* gain, float rms_eps, const
                       size_t ws_bytes, void* stream);
 
 /*
+ * The BitLinear forward as it runs in training (Section 2: the weights are quantised to 1.58 bits during the forward
+ * pass; Section 1: the released bf16 checkpoint is the master weight, used for training only): the absmean scale and
+ * the ternary codes are formed from the master weights on the fly, then the forward above runs on them.
+ *   W, w_dtype  in : master weights [N][K] row-major, BITLINEAR_F32 or BITLINEAR_BF16, device, 16-byte aligned.
+ *   eps_w       in : added to mean|W| to form the scale.
+ *   packed_out out : nullable; bitlinear_packed_bytes(N,K) bytes: the packed weights this call used (byte for byte what
+ *                    bitlinear_pack_weights writes - the inference artefact of the same step).
+ *   s_w_out    out : nullable; one fp32 on the device, the scale.
+ *   ws / ws_bytes  : device scratch of at least bitlinear_forward_master_workspace_bytes(M,N,K) (0 for an
+ *                    unsupported shape); holds the reduction partials, the packed weights and the forward's scratch.
+ * Three steps on `stream`: the absmean reduction (fixed order, deterministic), the quantise-and-pack pass, the forward.
+ * Everything else as bitlinear_forward.  The backward pass is not part of this library (the paper does not describe it).
+ */
+size_t bitlinear_forward_master_workspace_bytes(int M, int N, int K);
+int bitlinear_forward_master(const void* x_bf16, const void* gain, float rms_eps, const void* W, int w_dtype, float eps_w,
+                             int M, int N, int K, void* y_out, int y_dtype, void* packed_out, float* s_w_out, void* ws,
+                             size_t ws_bytes, void* stream);
+
+/*
  * bitlinear_forward for callers whose activations live in HOST memory: copies x (host, ideally
  * pinned) into the workspace, runs the forward, copies y back to the host buffer and
  * SYNCHRONISES the stream before returning.

@@ -47,6 +47,9 @@ _SIGNATURES = {
                                    _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_forward_host": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_void_p, _c_int, _c_int,
                                         _c_int, _c_void_p, _c_int, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_forward_master_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int]),
+    "bitlinear_forward_master": (_c_int, [_c_void_p, _c_void_p, _c_float, _c_void_p, _c_int, _c_float, _c_int, _c_int, _c_int,
+                                          _c_void_p, _c_int, _c_void_p, _c_void_p, _c_void_p, _c_size_t, _c_void_p]),
     "bitlinear_rope_kv": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int, _c_float,
                                    _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_void_p]),
     "bitlinear_attention_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int, _c_int]),
@@ -381,6 +384,34 @@ def bitlinear_decode_chain(layers: ChainLayers, hidden: int, ffn: int, n_q_heads
 
 def bitlinear_static_scratch_bytes() -> int:
     return int(lib().bitlinear_static_scratch_bytes())
+
+
+def bitlinear_forward_master_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().bitlinear_forward_master_workspace_bytes(M, N, K))
+
+
+def bitlinear_forward_master(x, gain, W, N: int | None = None, rms_eps: float = 1e-5, eps_w: float = 1e-5, y_dtype=torch.float32,
+                             want_packed: bool = False):
+    """The training-time forward: master weights W [N, K] (fp32 or bf16) are quantised on the fly.  Returns y, or
+    (y, packed, s_w) with want_packed."""
+    _dev(x, torch.bfloat16, "x")
+    if gain is not None:
+        _dev(gain, torch.bfloat16, "gain")
+    if W.dtype not in (torch.float32, torch.bfloat16):
+        raise TypeError("W must be float32 or bfloat16")
+    _dev(W, W.dtype, "W")
+    M, K = x.shape
+    if W.shape[1] != K or (N is not None and W.shape[0] != N):
+        raise ValueError("W must be [N, K]")
+    N = W.shape[0]
+    y = torch.empty(M, N, dtype=y_dtype, device=x.device)
+    ws = _workspace(bitlinear_forward_master_workspace_bytes(M, N, K), x.device)
+    packed = torch.empty(bitlinear_packed_bytes(N, K), dtype=torch.uint8, device=x.device) if want_packed else None
+    s_w = torch.empty(1, dtype=torch.float32, device=x.device) if want_packed else None
+    rc = lib().bitlinear_forward_master(_ptr(x), _ptr(gain), rms_eps, _ptr(W), BF16 if W.dtype == torch.bfloat16 else F32, eps_w,
+                                        M, N, K, _ptr(y), _ydt(y_dtype), _ptr(packed), _ptr(s_w), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_forward_master")
+    return (y, packed, s_w) if want_packed else y
 
 
 def bitlinear_forward_static(x, gain, packed, s_w, N: int, rms_eps: float = 1e-5, y_dtype=torch.float32,

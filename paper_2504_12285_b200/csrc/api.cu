@@ -281,6 +281,37 @@ int bitlinear_forward(const void* x_bf16, const void* gain, float rms_eps, const
                               mm_bytes ? base + w.mm_off : nullptr, mm_bytes, stream);
 }
 
+size_t bitlinear_forward_master_workspace_bytes(int M, int N, int K) {
+    if (!shape_ok(N, K) || M < 0) return 0;
+    return align_up(bitlinear_pack_workspace_bytes(N, K), 256) + align_up(bitlinear_packed_bytes(N, K), 256) + 256 /*scale*/ +
+           bitlinear_workspace_bytes(M, N, K);
+}
+
+int bitlinear_forward_master(const void* x_bf16, const void* gain, float rms_eps, const void* W, int w_dtype, float eps_w,
+                             int M, int N, int K, void* y_out, int y_dtype, void* packed_out, float* s_w_out, void* ws,
+                             size_t ws_bytes, void* stream) {
+    if (y_dtype != BITLINEAR_F32 && y_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
+    if (w_dtype != BITLINEAR_F32 && w_dtype != BITLINEAR_BF16) return BITLINEAR_ERR_DTYPE;
+    if (M < 0 || !shape_ok(N, K)) return BITLINEAR_ERR_SHAPE;
+    if (!W || (M > 0 && (!x_bf16 || !y_out))) return BITLINEAR_ERR_NULL;
+    if (!ws || !aligned16(ws) || ws_bytes < bitlinear_forward_master_workspace_bytes(M, N, K)) return BITLINEAR_ERR_WORKSPACE;
+    if (packed_out && !aligned16(packed_out)) return BITLINEAR_ERR_ALIGN;
+    char* base = static_cast<char*>(ws);
+    const size_t pack_ws = align_up(bitlinear_pack_workspace_bytes(N, K), 256), packed_bytes = bitlinear_packed_bytes(N, K);
+    void* packed = packed_out ? packed_out : static_cast<void*>(base + pack_ws);
+    float* s_w = reinterpret_cast<float*>(base + pack_ws + align_up(packed_bytes, 256));
+    if (const int rc = bitlinear_pack_weights(W, w_dtype, N, K, eps_w, packed, s_w, base, pack_ws, stream)) return rc;
+    if (s_w_out && cudaMemcpyAsync(s_w_out, s_w, sizeof(float), cudaMemcpyDeviceToDevice, static_cast<cudaStream_t>(stream)) !=
+                       cudaSuccess) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
+    if (M == 0) return BITLINEAR_OK;
+    char* fwd_ws = base + pack_ws + align_up(packed_bytes, 256) + 256;
+    return bitlinear_forward(x_bf16, gain, rms_eps, packed, s_w, M, N, K, y_out, y_dtype, fwd_ws,
+                             ws_bytes - (size_t)(fwd_ws - base), stream);
+}
+
 size_t bitlinear_host_staging_bytes(int M, int N, int K, int y_dtype) {
     if (!shape_ok(N, K) || M < 0) return 0;
     const size_t ysz = (y_dtype == BITLINEAR_BF16) ? 2 : 4;
