@@ -27,6 +27,7 @@
 #include <vector>
 
 #include "quant_row.cuh"
+#include "decode_level.cuh"
 #include "sm100_sync.cuh"
 
 namespace bitlinear {
@@ -130,6 +131,7 @@ struct StreamParams {
     int table_cap;  // problems of a CTA whose descriptors are cached in shared memory
     int arena_bytes;  // shared memory available for staged activations
     int* status_word;
+    int fuse_prob;    // FUSE kernels: the plan entry that owns the one quantised row of the call
 };
 
 // Shared-memory copy of what the stream kernel needs of one problem (filled once per CTA).
@@ -173,7 +175,11 @@ struct ChunkCursor {
 // peeled off by repeated multiplication by 3 in two 16-bit fields per register (a byte times 3 leaves its digit in the
 // byte above and the remainder in place), gathered into one operand of four codes per digit with a byte permute, and
 // fed to the same dot-product-of-four against four consecutive activations.
-template <int kChunkTiles, int FMT>
+// FUSE: the call has ONE input row (one token, every problem reads it through the same step with the same norm - q/k/v
+// or gate/up of a layer, or a single matmul): there is no quantiser launch; every CTA quantises the row itself, into
+// its arena, while its first weight chunks are in flight.  CTA 0 also writes the codes, the scale and the code sum
+// where the quantiser launch would have put them, so that a later call may reuse them.
+template <int kChunkTiles, int FMT, bool FUSE>
 __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const StreamParams prm) {
     constexpr int kCols = FMT ? kDenseTileCols : kTileCols;   // columns of a tile
     constexpr int kLaneBytes = FMT ? 80 : 16;                 // activation bytes of a column lane t inside a tile
@@ -283,7 +289,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         int off = 0;
         for (int i = 0; i < n_tab; ++i) {
             const int bytes = table[i].M * table[i].x_stride;  // a multiple of 64
-            if (off + bytes <= prm.arena_bytes) {
+            if (FUSE) {
+                table[i].x_off = 0;  // every problem reads the one row at the start of the arena
+            } else if (off + bytes <= prm.arena_bytes) {
                 table[i].x_off = off;
                 off += bytes;
             } else {
@@ -295,6 +303,36 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     // the quantiser launch that precedes this kernel must be complete before its results are read
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
+    if constexpr (FUSE) {
+        // ---- quantise the call's one input row into the arena (all threads), hand its scale and code sum to the table ----
+        __shared__ RowReduceSmemT<kStreamWarps> qsm;
+        __shared__ float d_s;
+        __shared__ int xsum_s;
+        const DevProblem& p0 = probs[prm.fuse_prob];
+        RowOp op = p0.op;
+        if (blockIdx.x != 0) op.x_out = nullptr;  // the step's own output (a new hidden state) is written once
+        __syncthreads();  // the table is complete before the arena (which follows it) is written
+        with_row_source(op, p0.x, p0.x_row0, p0.K, [&](auto src) {
+            quant_row_src<2, FMT ? 0 : 1, decltype(src), kStreamThreads>(src, p0.gain, p0.eps, p0.K, reinterpret_cast<int8_t*>(arena), &d_s,
+                                                                      &xsum_s, qsm);
+        });
+        if (FMT == 1)
+            for (int k = p0.K + 4 * (int)threadIdx.x; k < p0.x_stride; k += 4 * kStreamThreads) *reinterpret_cast<uint32_t*>(arena + k) = 0u;
+        __syncthreads();
+        for (int i = threadIdx.x; i < n_tab; i += kStreamThreads) {
+            table[i].d = d_s;
+            table[i].xsum = xsum_s;
+        }
+        if (blockIdx.x == 0) {
+            for (int o = threadIdx.x * 16; o < p0.x_stride; o += kStreamThreads * 16)
+                *reinterpret_cast<uint4*>(p0.xq + o) = *reinterpret_cast<const uint4*>(arena + o);
+            if (threadIdx.x == 0) {
+                p0.d[0] = d_s;
+                p0.xsum[0] = xsum_s;
+            }
+        }
+        __syncthreads();
+    } else {
     // ---- scales and code sums of the tokens, then stage the activations ----
     for (int i = warp; i < n_tab; i += kStreamWarps) {
         const DevProblem& pr = probs[p_lo + i];
@@ -316,6 +354,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         asm volatile("cp.async.commit_group;" ::: "memory");
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         __syncthreads();
+    }
     }
 
     if (mine) {
@@ -477,9 +516,9 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
     if (*abort_flag && threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
 }
 
-template <int kChunkTiles, int FMT>
+template <int kChunkTiles, int FMT, bool FUSE>
 cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
-    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<kChunkTiles, FMT>,
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<kChunkTiles, FMT, FUSE>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     // programmatic dependent launch: the kernel may begin (barrier set-up, first weight copies) while the quantiser
@@ -494,7 +533,7 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<kChunkTiles, FMT>, prm);
+    return cudaLaunchKernelEx(&cfg, decode_stream_kernel<kChunkTiles, FMT, FUSE>, prm);
 }
 
 struct PlanLayout {
@@ -723,6 +762,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     // through L1 instead, and only as many descriptors as fit a quarter of the space are cached
     constexpr int chunk_tiles = 5;
     const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles) - 128;
+    const int table_need = table_cap;  // with fewer cached descriptors some problems of a CTA are read from global memory
     if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
     if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
     arena_max &= ~(size_t)255;
@@ -745,8 +785,29 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     }
     const DevProblem* probs_dev = reinterpret_cast<const DevProblem*>(base + L.probs_off);
 
+    // One input row in the whole call (a single token, every problem reading it the same way - the usual shape of one level
+    // of a decoder layer at one token): no quantiser launch, the stream kernel quantises the row itself (FUSE).
+    const bool fuse = rows == 1 && !(flags & BITLINEAR_BATCH_REUSE_ACT) && table_cap == table_need && max_k <= 16 * kStreamThreads;
+    if (fuse) arena_max = std::max(arena_max, align_up((size_t)dp[0].x_stride, 256));
+
+    // ... and when the problems are few (a level of a decoder layer) the whole call is one launch that carries its
+    // descriptors in its arguments (decode_level.cu); the plan uploaded above stays valid for calls that reuse activations
+    if (fuse && !dense && decode_level_fits(n_prob, total_rb, max_k, sm_count)) {
+        LevelParams P = {};
+        P.count = n_prob;
+        for (int i = 0; i < n_prob; ++i) {
+            P.prob[i].packed = dp[i].packed; P.prob[i].s_w = dp[i].s_w; P.prob[i].y = dp[i].y; P.prob[i].acc_out = dp[i].acc_out;
+            P.prob[i].N = dp[i].N; P.prob[i].y_dtype = dp[i].y_dtype;
+        }
+        P.x = dp[0].x; P.op = dp[0].op; P.gain = dp[0].gain; P.eps = dp[0].eps; P.K = dp[0].K; P.x_row0 = dp[0].x_row0;
+        P.xq_out = dp[0].xq; P.d_out = dp[0].d; P.xsum_out = dp[0].xsum;
+        P.total_rb = total_rb;
+        P.status_word = device_status_word();
+        return decode_level_forward(P, sm_count, st);
+    }
+
     // ---- launch 1: quantise every token of every problem ----
-    if (!(flags & BITLINEAR_BATCH_REUSE_ACT)) {
+    if (!fuse && !(flags & BITLINEAR_BATCH_REUSE_ACT)) {
         const int vpt = (max_k / 8 + kQuantThreads - 1) / kQuantThreads;
         const dim3 g((unsigned)rows), b(kQuantThreads);
         const PlanHeader* h = reinterpret_cast<const PlanHeader*>(base);
@@ -776,7 +837,11 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.table_cap = table_cap;
     prm.arena_bytes = (int)arena_max;
     const size_t smem = ring_bytes(chunk_tiles) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
-    const cudaError_t e = dense ? launch_stream<chunk_tiles, 1>(prm, grid, smem, st) : launch_stream<chunk_tiles, 0>(prm, grid, smem, st);
+    prm.fuse_prob = 0;  // the first entry owns the quantised copy of the one row
+    const cudaError_t e = fuse ? (dense ? launch_stream<chunk_tiles, 1, true>(prm, grid, smem, st)
+                                        : launch_stream<chunk_tiles, 0, true>(prm, grid, smem, st))
+                               : (dense ? launch_stream<chunk_tiles, 1, false>(prm, grid, smem, st)
+                                        : launch_stream<chunk_tiles, 0, false>(prm, grid, smem, st));
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 

@@ -14,12 +14,14 @@ namespace bitlinear {
 constexpr int kQuantThreads = 256;
 constexpr int kQuantWarps = kQuantThreads / 32;
 
-struct RowReduceSmem {
-    double sq[kQuantWarps];
+template <int WARPS>
+struct RowReduceSmemT {
+    double sq[WARPS];
     float r;
-    float mx[kQuantWarps];
-    int sum[kQuantWarps];
+    float mx[WARPS];
+    int sum[WARPS];
 };
+using RowReduceSmem = RowReduceSmemT<kQuantWarps>;
 
 __device__ __forceinline__ void unpack_bf16x8(const uint4& u, float (&f)[8]) {
     const uint32_t w[4] = {u.x, u.y, u.z, u.w};
@@ -182,10 +184,11 @@ __device__ __forceinline__ void with_row_source(const RowOp& o, const void* x, i
 //           swz = row & 7 - the 128-byte shared-memory swizzle.
 // LAYOUT 3: the same with tiles of 16 rows x 128 columns (2 KiB): the token-side operand of the decode kernel that
 //           runs on the tensor cores with the tokens as the narrow dimension.
-template <int VPT, int LAYOUT = 0, class Src = RowBf16>  // VPT = 16-byte vectors (8 bf16) per thread
+// THREADS = threads of the CTA (all of them take part; the block-wide barriers are __syncthreads).
+template <int VPT, int LAYOUT = 0, class Src = RowBf16, int THREADS = kQuantThreads>  // VPT = 16-byte vectors (8 bf16) per thread
 __device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16* __restrict__ gain, float eps, int K,
                                               int8_t* __restrict__ xq_row, float* __restrict__ d_out,
-                                              int32_t* __restrict__ xsum_out, RowReduceSmem& sm, int swz = 0) {
+                                              int32_t* __restrict__ xsum_out, RowReduceSmemT<THREADS / 32>& sm, int swz = 0) {
     const int n_vec = K >> 3;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const uint4* grow = reinterpret_cast<const uint4*>(gain);
@@ -193,7 +196,7 @@ __device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16
     uint4 xv[VPT];
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-        const int v = tid + i * kQuantThreads;
+        const int v = tid + i * THREADS;
         xv[i] = make_uint4(0, 0, 0, 0);
         if (v < n_vec) {
             xv[i] = src.load(v);
@@ -216,7 +219,7 @@ __device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16
     if (tid == 0) {  // one thread does the fp64 divide and square root
         double S = 0.0;
 #pragma unroll
-        for (int w = 0; w < kQuantWarps; ++w) S += sm.sq[w];
+        for (int w = 0; w < THREADS / 32; ++w) S += sm.sq[w];
         sm.r = (float)(1.0 / sqrt(S / (double)K + (double)eps));
     }
     __syncthreads();
@@ -227,7 +230,7 @@ __device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16
     float amax = 0.0f;
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-        const int v = tid + i * kQuantThreads;
+        const int v = tid + i * THREADS;
         float f[8], g[8];
         unpack_bf16x8(xv[i], f);
         if (gain != nullptr && v < n_vec) {
@@ -248,7 +251,7 @@ __device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16
     __syncthreads();
     float a = 0.0f;
 #pragma unroll
-    for (int w = 0; w < kQuantWarps; ++w) a = fmaxf(a, sm.mx[w]);
+    for (int w = 0; w < THREADS / 32; ++w) a = fmaxf(a, sm.mx[w]);
     a = fmaxf(a, 1e-5f);
     const float s = __fdiv_rn(127.0f, a);
 
@@ -257,7 +260,7 @@ __device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16
     uint2* qrow = reinterpret_cast<uint2*>(xq_row);
 #pragma unroll
     for (int i = 0; i < VPT; ++i) {
-        const int v = tid + i * kQuantThreads;
+        const int v = tid + i * THREADS;
         uint32_t c[8], packed[2];
 #pragma unroll
         for (int e = 0; e < 8; ++e) c[e] = round_code(__fmul_rn(y[i][e], s));
@@ -280,7 +283,7 @@ __device__ __forceinline__ void quant_row_src(const Src src, const __nv_bfloat16
     if (tid == 0) {
         int total = 0;
 #pragma unroll
-        for (int w = 0; w < kQuantWarps; ++w) total += sm.sum[w];
+        for (int w = 0; w < THREADS / 32; ++w) total += sm.sum[w];
         *d_out = __fdiv_rn(a, 127.0f);
         if (xsum_out != nullptr) *xsum_out = total;
     }
