@@ -197,6 +197,8 @@ int bitlinear_matmul_q(const int8_t* xq, const float* d, const int32_t* xsum, co
 /*
  * The whole BitLinear forward: bitlinear_quant_act followed by bitlinear_matmul_q (path AUTO)
  * on the same stream (Section 2: norm -> activation quantiser -> W1.58A8 product -> rescale).
+ * At one token the two steps are one launch (every CTA quantises the row while its share of the
+ * packed weights is on its way from HBM); the result is the same, bit for bit.
  *   ws / ws_bytes : scratch of at least bitlinear_workspace_bytes(M,N,K).
  */
 int bitlinear_forward(const void* x_bf16, const void* gain, float rms_eps, const void* packed,

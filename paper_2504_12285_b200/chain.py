@@ -2,7 +2,8 @@
 
 Every step runs in the library's kernels: per layer four batched BitLinear calls (q/k/v, o, gate/up, down - the
 problems of a call share their input and are independent of each other), each with the element-wise step in front of
-it (residual, attention stand-in, residual, squared-ReLU gate) fused into its quantiser launch.  This module only owns
+it (residual, attention stand-in, residual, squared-ReLU gate) fused into its quantiser - which at one token is part
+of the same launch as the weight stream.  This module only owns
 the buffers and the call order.
 """
 from __future__ import annotations
@@ -57,7 +58,11 @@ class DecodeChain:
         self.h = self.h_mid  # where the hidden state is after step()
         torch.cuda.synchronize(dev)
 
-    launches_per_layer = 8  # 4 x (quantiser with its fused element-wise step + weight stream)
+    @property
+    def launches_per_layer(self) -> int:
+        """One token: each of the four levels is one launch (the kernel quantises its input row itself); more tokens:
+        4 x (quantiser with its fused element-wise step + weight stream)."""
+        return 4 if self.M == 1 else 8
 
     def step(self, h0: torch.Tensor | None = None) -> torch.Tensor:
         """One pass over all layers, starting from h0 (bf16 [M, hidden]) or from the current hidden state."""
@@ -119,7 +124,11 @@ class DecodeStep:
             self.calls.append(per_layer)
         torch.cuda.synchronize(dev)
 
-    launches_per_layer = 11  # 4 x (quantiser + weight stream), rotary/append, attention slices, attention merge
+    @property
+    def launches_per_layer(self) -> int:
+        """Four levels (one launch each at one token, quantiser + weight stream otherwise), rotary/append, attention
+        slices, attention merge."""
+        return (4 if self.M == 1 else 8) + 3
 
     def set_positions(self, positions: torch.Tensor) -> None:
         """positions: int32 [M] (device): where the next token of each sequence goes; it attends to rows 0 .. position."""

@@ -2,6 +2,7 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "decode_level.cuh"
 #include "sm100_sync.cuh"
 
 namespace bitlinear {
@@ -275,6 +276,22 @@ int bitlinear_forward(const void* x_bf16, const void* gain, float rms_eps, const
     int8_t* xq = reinterpret_cast<int8_t*>(base + w.xq_off);
     float* d = reinterpret_cast<float*>(base + w.d_off);
     int32_t* xsum = reinterpret_cast<int32_t*>(base + w.xsum_off);
+    // one token: a single launch that fetches its weights while it quantises the row (decode_level.cu); the same
+    // arithmetic as the two launches below, bit for bit
+    int sm_count = 0;
+    if (M == 1 && aligned16(x_bf16) && aligned16(packed) && aligned16(y_out) && (!gain || aligned16(gain)) &&
+        !(reinterpret_cast<uintptr_t>(s_w) & 3u) && check_arch() == BITLINEAR_OK && device_sm_count(&sm_count) == BITLINEAR_OK &&
+        decode_level_fits(1, N / kTileRows, K, sm_count)) {
+        LevelParams P = {};
+        P.count = 1;
+        P.prob[0].packed = static_cast<const uint8_t*>(packed); P.prob[0].s_w = s_w; P.prob[0].y = y_out;
+        P.prob[0].acc_out = nullptr; P.prob[0].N = N; P.prob[0].y_dtype = y_dtype;
+        P.x = x_bf16; P.op.op = BITLINEAR_X_PLAIN;
+        P.gain = static_cast<const __nv_bfloat16*>(gain); P.eps = rms_eps; P.K = K; P.x_row0 = 0;
+        P.total_rb = N / kTileRows;
+        P.status_word = device_status_word();
+        return decode_level_forward(P, sm_count, static_cast<cudaStream_t>(stream));
+    }
     int rc = bitlinear_quant_act(x_bf16, gain, rms_eps, M, K, xq, d, xsum, stream);
     if (rc != BITLINEAR_OK) return rc;
     return bitlinear_matmul_q(xq, d, xsum, packed, s_w, M, N, K, y_out, y_dtype, nullptr, BITLINEAR_PATH_AUTO,

@@ -13,8 +13,8 @@
 //   4. multiplies: a warp takes a slice of the 256-column tiles of one row block (dot-products-of-four on
 //      word & (0x03030303 << 2j), as in the streaming kernel), partial sums meet in shared memory (integers: exact);
 //   5. dequantises and stores.
-// CTA 0 also writes the codes, the scale and the code sum where a quantiser launch would have put them, so that a later
-// call on the same workspace may reuse them.
+// CTA 0 also writes the codes, the scale and the code sum where a quantiser launch would have put them (when the caller
+// names such a place), so that a later call on the same workspace may reuse them.
 #include "decode_level.cuh"
 #include "sm100_sync.cuh"
 
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(kLevelThreads) decode_level_kernel(const __gri
             quant_row_src<VPT, 1, decltype(src), kLevelThreads>(src, P.gain, P.eps, P.K, reinterpret_cast<int8_t*>(arena), &d_s, &xsum_s, qsm);
         });
         __syncthreads();
-        if (blockIdx.x == 0) {
+        if (blockIdx.x == 0 && P.xq_out != nullptr) {
             for (int o = threadIdx.x * 16; o < P.K; o += kLevelThreads * 16)
                 *reinterpret_cast<uint4*>(P.xq_out + o) = *reinterpret_cast<const uint4*>(arena + o);
             if (threadIdx.x == 0) {

@@ -23,7 +23,7 @@ struct LevelParams {
     const __nv_bfloat16* gain;
     float eps;
     int K, x_row0;
-    int8_t* xq_out;  // [K] codes in the layout of the quantiser launch (LAYOUT 1), scale, code sum
+    int8_t* xq_out;  // nullable, all three or none: [K] codes in the layout of the quantiser launch (LAYOUT 1), scale, code sum
     float* d_out;
     int32_t* xsum_out;
     int total_rb, rb_per_cta;

@@ -37,7 +37,9 @@ __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ 
                                                       double log2_base, __nv_bfloat16* __restrict__ q_out,
                                                       __nv_bfloat16* __restrict__ k_cache, __nv_bfloat16* __restrict__ v_cache,
                                                       int t_max) {
+    // a programmatic dependent of the launch before it (the q/k/v projections) and the primary of the attention launch
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int half = hd / 2;
     const int pairs_per_tok = (n_q + n_kv) * half;
     const int vals_per_tok = n_kv * hd;
@@ -634,11 +636,22 @@ int bitlinear_rope_kv(const float* q, const float* k, const float* v, const int3
     if (M == 0) return BITLINEAR_OK;
     if (!q || !k || !v || !positions || !q_out_bf16 || !k_cache_bf16 || !v_cache_bf16) return BITLINEAR_ERR_NULL;
     const long long work = (long long)M * ((n_q_heads + n_kv_heads) * (head_dim / 2) + n_kv_heads * head_dim);
-    rope_kv_kernel<<<(unsigned)((work + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
-        q, k, v, positions, seq_ids, M, n_q_heads, n_kv_heads, head_dim, n_seq, log2((double)rope_base),
-        static_cast<__nv_bfloat16*>(q_out_bf16), static_cast<__nv_bfloat16*>(k_cache_bf16), static_cast<__nv_bfloat16*>(v_cache_bf16),
-        t_max);
-    return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)((work + 255) / 256));
+    cfg.blockDim = dim3(256);
+    cfg.stream = static_cast<cudaStream_t>(stream);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, rope_kv_kernel, q, k, v, positions, seq_ids, M, n_q_heads, n_kv_heads, head_dim, n_seq,
+                           log2((double)rope_base), static_cast<__nv_bfloat16*>(q_out_bf16), static_cast<__nv_bfloat16*>(k_cache_bf16),
+                           static_cast<__nv_bfloat16*>(v_cache_bf16), t_max) != cudaSuccess) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_CUDA;
+    }
+    return BITLINEAR_OK;
 }
 
 size_t bitlinear_attention_workspace_bytes(int M, int n_q_heads, int n_kv_heads, int head_dim, int t_max) {
