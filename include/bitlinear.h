@@ -263,7 +263,11 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  *              problems of at most 16 tokens.  Problems with M == 0 are skipped.  Outputs must not
  *              alias inputs of other problems of the same call (they run concurrently).
  *   flags    : 0, or an OR of BITLINEAR_BATCH_REUSE_PLAN (the previous call on this workspace had
- *              exactly the same descriptors: skips re-uploading the decode plan) and
+ *              exactly the same descriptors, and the packed weights, their scales and the gains
+ *              have not been written since - the steady state of a decode loop: skips
+ *              re-uploading the decode plan, and a call that is a single launch (one token, one
+ *              shared input row) may begin fetching weights while the launch before it on the
+ *              stream is still running) and
  *              BITLINEAR_BATCH_REUSE_ACT (the inputs are unchanged as well: skips the quantiser
  *              launches and reuses their results in ws), BITLINEAR_BATCH_REUSE_WEIGHTS (same
  *              descriptors and same packed matrices: skips the expansion of the prefill problems).

@@ -290,7 +290,7 @@ int bitlinear_forward(const void* x_bf16, const void* gain, float rms_eps, const
         P.gain = static_cast<const __nv_bfloat16*>(gain); P.eps = rms_eps; P.K = K; P.x_row0 = 0;
         P.total_rb = N / kTileRows;
         P.status_word = device_status_word();
-        return decode_level_forward(P, sm_count, static_cast<cudaStream_t>(stream));
+        return decode_level_forward(P, sm_count, static_cast<cudaStream_t>(stream), /*dependent=*/false);
     }
     int rc = bitlinear_quant_act(x_bf16, gain, rms_eps, M, K, xq, d, xsum, stream);
     if (rc != BITLINEAR_OK) return rc;

@@ -517,7 +517,7 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
 }
 
 template <int kChunkTiles, int FMT, bool FUSE>
-cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
+cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaStream_t st, bool dependent) {
     cudaError_t e = cudaFuncSetAttribute(decode_stream_kernel<kChunkTiles, FMT, FUSE>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -532,7 +532,7 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = dependent ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, decode_stream_kernel<kChunkTiles, FMT, FUSE>, prm);
 }
 
@@ -792,6 +792,9 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
 
     // ... and when the problems are few (a level of a decoder layer) the whole call is one launch that carries its
     // descriptors in its arguments (decode_level.cu); the plan uploaded above stays valid for calls that reuse activations
+    // A fused launch reads weights, scales and gain before it waits for the launch in front of it, which is only safe
+    // when that launch does not write them: the steady state of a decode loop, which BITLINEAR_BATCH_REUSE_PLAN names.
+    const bool static_weights = (flags & BITLINEAR_BATCH_REUSE_PLAN) != 0;
     if (fuse && !dense && decode_level_fits(n_prob, total_rb, max_k, sm_count)) {
         LevelParams P = {};
         P.count = n_prob;
@@ -803,7 +806,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         P.xq_out = dp[0].xq; P.d_out = dp[0].d; P.xsum_out = dp[0].xsum;
         P.total_rb = total_rb;
         P.status_word = device_status_word();
-        return decode_level_forward(P, sm_count, st);
+        return decode_level_forward(P, sm_count, st, static_weights);
     }
 
     // ---- launch 1: quantise every token of every problem ----
@@ -838,10 +841,13 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.arena_bytes = (int)arena_max;
     const size_t smem = ring_bytes(chunk_tiles) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
     prm.fuse_prob = 0;  // the first entry owns the quantised copy of the one row
-    const cudaError_t e = fuse ? (dense ? launch_stream<chunk_tiles, 1, true>(prm, grid, smem, st)
-                                        : launch_stream<chunk_tiles, 0, true>(prm, grid, smem, st))
-                               : (dense ? launch_stream<chunk_tiles, 1, false>(prm, grid, smem, st)
-                                        : launch_stream<chunk_tiles, 0, false>(prm, grid, smem, st));
+    // behind the quantiser launch of this call the stream kernel is always a dependent (that launch writes no weights);
+    // a fused launch only under the promise above
+    const bool dep = !fuse || static_weights;
+    const cudaError_t e = fuse ? (dense ? launch_stream<chunk_tiles, 1, true>(prm, grid, smem, st, dep)
+                                        : launch_stream<chunk_tiles, 0, true>(prm, grid, smem, st, dep))
+                               : (dense ? launch_stream<chunk_tiles, 1, false>(prm, grid, smem, st, dep)
+                                        : launch_stream<chunk_tiles, 0, false>(prm, grid, smem, st, dep));
     return e == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 

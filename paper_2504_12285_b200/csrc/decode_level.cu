@@ -6,8 +6,11 @@
 // Everything the kernel needs is in its parameters.  A CTA takes a contiguous run of 16-row weight blocks and
 //   1. before anything else starts bulk copies of its whole share of the packed weights (11 - 60 KB) into shared memory,
 //      and lets the next launch of the stream begin (programmatic dependent launch): with level kernels back to back the
-//      next level's CTAs sit beside this level's and fetch their weights while this level computes;
-//   2. waits for the launch before it (griddepcontrol.wait) - nothing but weights is read earlier;
+//      next level's CTAs sit beside this level's and fetch their weights while this level computes.  (Only a caller that
+//      vouches that the launch in front does not write weights, scales or gain gets this launch as a dependent; for
+//      everybody else the launch is ordinary and step 2 returns at once.)
+//   2. waits for the launch before it (griddepcontrol.wait) - nothing but weights, their scales and the norm's gain
+//      (all static) is read earlier;
 //   3. quantises the input row itself (fused RMSNorm + absmax int8, the element-wise step in front of it included):
 //      every CTA repeats this, which costs less than a quantiser launch and its round trip through memory;
 //   4. multiplies: a warp takes a slice of the 256-column tiles of one row block (dot-products-of-four on
@@ -36,9 +39,9 @@ __device__ __forceinline__ uint4 lds128(uint32_t addr) {
     return v;
 }
 
-// shared memory: [weights: rb_per_cta x k_tiles KiB][codes of the row: K bytes][partial sums][barrier, abort flag]
+// shared memory: [weights: rb_per_cta x k_tiles KiB][codes of the row: K bytes][gain: 2K bytes][partial sums][barrier, abort flag]
 __host__ __device__ inline size_t level_smem_bytes(int rb_per_cta, int K) {
-    return (size_t)rb_per_cta * (K / kTileCols) * kTileBytes + (size_t)K + (size_t)rb_per_cta * kLevelWarps * 16 * sizeof(int) + 32;
+    return (size_t)rb_per_cta * (K / kTileCols) * kTileBytes + (size_t)3 * K + (size_t)rb_per_cta * kLevelWarps * 16 * sizeof(int) + 32;
 }
 
 template <int VPT>
@@ -53,7 +56,8 @@ __global__ void __launch_bounds__(kLevelThreads) decode_level_kernel(const __gri
     const int R = rb_hi - rb_lo;  // >= 1 by the grid size
     const uint32_t rb_bytes = (uint32_t)k_tiles * kTileBytes;
     uint8_t* arena = smem + (size_t)P.rb_per_cta * rb_bytes;
-    int* part = reinterpret_cast<int*>(arena + P.K);  // [rb][warp slot][16 rows]
+    uint4* gain_s = reinterpret_cast<uint4*>(arena + P.K);  // the norm's gain, copied before the wait (it is static)
+    int* part = reinterpret_cast<int*>(arena + 3 * (size_t)P.K);  // [rb][warp slot][16 rows]
     uint64_t* bar = reinterpret_cast<uint64_t*>(part + P.rb_per_cta * kLevelWarps * 16);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar + 1);
     const uint32_t bar_s = smem_u32(bar), w_s = smem_u32(smem);
@@ -83,16 +87,24 @@ __global__ void __launch_bounds__(kLevelThreads) decode_level_kernel(const __gri
             bulk_load(w_s + (uint32_t)j * rb_bytes, P.prob[i].packed + (size_t)local * rb_bytes, rb_bytes, bar_s);
         }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // what else does not depend on the launch before this one: the gain vector and the weight scales
+    if (P.gain != nullptr)
+        for (int v = threadIdx.x; v < (P.K >> 3); v += kLevelThreads) gain_s[v] = reinterpret_cast<const uint4*>(P.gain)[v];
+    float s_w[kLevelMaxProblems];
+#pragma unroll
+    for (int i = 0; i < kLevelMaxProblems; ++i) s_w[i] = i < P.count ? *P.prob[i].s_w : 0.0f;
 
     // ---- 2. everything else depends on the launch before this one ----
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    __syncthreads();  // the gain copy is complete
 
     // ---- 3. the input row -> int8 codes in shared memory ----
     {
         RowOp op = P.op;
         if (blockIdx.x != 0) op.x_out = nullptr;  // the step's own output (a new hidden state) is written once
         with_row_source(op, P.x, P.x_row0, P.K, [&](auto src) {
-            quant_row_src<VPT, 1, decltype(src), kLevelThreads>(src, P.gain, P.eps, P.K, reinterpret_cast<int8_t*>(arena), &d_s, &xsum_s, qsm);
+            quant_row_src<VPT, 1, decltype(src), kLevelThreads>(src, P.gain ? reinterpret_cast<const __nv_bfloat16*>(gain_s) : nullptr, P.eps,
+                                                                P.K, reinterpret_cast<int8_t*>(arena), &d_s, &xsum_s, qsm);
         });
         __syncthreads();
         if (blockIdx.x == 0 && P.xq_out != nullptr) {
@@ -166,7 +178,10 @@ __global__ void __launch_bounds__(kLevelThreads) decode_level_kernel(const __gri
         int i, local;
         locate(rb_lo + j, i, local);
         const LevelProblem& p = P.prob[i];
-        const float val = __fmul_rn(__fmul_rn((float)v, *p.s_w), d_s);
+        float sw = s_w[0];
+#pragma unroll
+        for (int c = 1; c < kLevelMaxProblems; ++c) sw = i == c ? s_w[c] : sw;
+        const float val = __fmul_rn(__fmul_rn((float)v, sw), d_s);
         const size_t n = (size_t)local * kTileRows + r;
         if (p.acc_out != nullptr) p.acc_out[n] = v;
         if (p.y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(p.y)[n] = __float2bfloat16_rn(val);
@@ -174,8 +189,10 @@ __global__ void __launch_bounds__(kLevelThreads) decode_level_kernel(const __gri
     }
 }
 
+// dependent: launch as a programmatic dependent of the launch before it (the kernel then reads weights, scales and gain
+// while that launch may still be running: only for callers who vouch that it does not write them)
 template <int VPT>
-cudaError_t launch_level(const LevelParams& P, int grid, size_t smem, cudaStream_t st) {
+cudaError_t launch_level(const LevelParams& P, int grid, size_t smem, cudaStream_t st, bool dependent) {
     // the opt-in is per device and cheap: repeated so that every device a process uses gets it
     if (smem > 48 * 1024) {
         const cudaError_t e = cudaFuncSetAttribute(decode_level_kernel<VPT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -190,7 +207,7 @@ cudaError_t launch_level(const LevelParams& P, int grid, size_t smem, cudaStream
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = dependent ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, decode_level_kernel<VPT>, P);
 }
 
@@ -202,11 +219,11 @@ bool decode_level_fits(int count, int total_rb, int K, int sm_count) {
     return level_smem_bytes(rb_per_cta, K) <= 100 * 1024;  // two launches of this kind fit an SM side by side
 }
 
-int decode_level_forward(LevelParams& P, int sm_count, cudaStream_t st) {
+int decode_level_forward(LevelParams& P, int sm_count, cudaStream_t st, bool dependent) {
     P.rb_per_cta = (P.total_rb + sm_count - 1) / sm_count;
     const int grid = (P.total_rb + P.rb_per_cta - 1) / P.rb_per_cta;
     const size_t smem = level_smem_bytes(P.rb_per_cta, P.K);
-    const cudaError_t e = P.K <= 8 * 2 * kLevelThreads ? launch_level<2>(P, grid, smem, st) : launch_level<4>(P, grid, smem, st);
+    const cudaError_t e = P.K <= 8 * 2 * kLevelThreads ? launch_level<2>(P, grid, smem, st, dependent) : launch_level<4>(P, grid, smem, st, dependent);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;

@@ -33,7 +33,8 @@ struct LevelParams {
 // Can this call run as one level launch?  (At most kLevelMaxProblems problems of one token in the 2-bit layout that
 // share their input row, a CTA's share of the weights small enough for two such launches to sit side by side on an SM.)
 bool decode_level_fits(int count, int total_rb, int K, int sm_count);
-// Fills in the split and launches; P.total_rb = sum of N / 16 over the problems.
-int decode_level_forward(LevelParams& P, int sm_count, cudaStream_t st);
+// Fills in the split and launches; P.total_rb = sum of N / 16 over the problems.  dependent: the packed weights, their
+// scales and the gain are not written by the launch before this one on the stream, so the kernel may start beside it.
+int decode_level_forward(LevelParams& P, int sm_count, cudaStream_t st, bool dependent);
 
 }  // namespace bitlinear
