@@ -512,7 +512,7 @@ def run_config1(bl, dev, peaks):
     pb = n * k // 4
     return {"workload": "configs[0]: q projection, M=1, K=N=2560, 1,638,400 packed bytes per forward",
             "isolated_us_per_forward": round(iso_us, 2), "isolated_GBps": round(pb / iso_us / 1e3, 1),
-            "isolated_note": "one bitlinear_forward (quantiser + decode kernel launch) on an idle GPU, weights not in L2: "
+            "isolated_note": "one bitlinear_forward (a single launch that quantises the row and streams the weights) on an idle GPU, weights not in L2: "
                              "latency-bound, a 1.6 MB matmul is far below the bandwidth-delay product of HBM",
             "back_to_back_us_per_forward": round(seq_us, 2), "back_to_back_GBps": round(pb / seq_us / 1e3, 1),
             "steady_us_per_forward": round(ms_b * 1e3 / copies, 3), "steady_GBps": round(pb * copies / ms_b / 1e6, 1),
