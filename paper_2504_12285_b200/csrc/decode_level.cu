@@ -25,7 +25,7 @@ namespace bitlinear {
 
 namespace {
 
-constexpr int kLevelThreads = 256;
+constexpr int kLevelThreads = 512;
 constexpr int kLevelCtasPerSm = 1;  // CTAs per SM the row blocks are dealt to (2 measured slower: 1.13 against 1.07 ms per token)
 constexpr int kLevelWarps = kLevelThreads / 32;
 
@@ -73,7 +73,7 @@ __global__ void __launch_bounds__(kLevelThreads) decode_level_kernel(const __gri
         }
     };
 
-    // ---- 1. the weights of this CTA's row blocks: one bulk copy per row block, issued by eight threads ----
+    // ---- 1. the weights of this CTA's row blocks: one bulk copy per row block, issued by one thread per warp ----
     if (threadIdx.x == 0) {
         *abort_flag = 0;
         mbar_init(bar_s, 1);
@@ -224,7 +224,7 @@ int decode_level_forward(LevelParams& P, int sm_count, cudaStream_t st, bool dep
     P.rb_per_cta = (P.total_rb + kLevelCtasPerSm * sm_count - 1) / (kLevelCtasPerSm * sm_count);
     const int grid = (P.total_rb + P.rb_per_cta - 1) / P.rb_per_cta;
     const size_t smem = level_smem_bytes(P.rb_per_cta, P.K);
-    const cudaError_t e = P.K <= 8 * 2 * kLevelThreads ? launch_level<2>(P, grid, smem, st, dependent) : launch_level<4>(P, grid, smem, st, dependent);
+    const cudaError_t e = P.K <= 8 * kLevelThreads ? launch_level<1>(P, grid, smem, st, dependent) : launch_level<2>(P, grid, smem, st, dependent);
     if (e != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;

@@ -378,6 +378,7 @@ __global__ void __launch_bounds__(128) attn_decode_combine_kernel(const AttnPart
     const size_t mh = blockIdx.x;  // token * n_q + head
     const int m = (int)(mh / n_q);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");  // the o projection may start fetching its weights
     asm volatile("griddepcontrol.wait;" ::: "memory");  // the partial results come from the launch before this one
     const AttnPartial<HD>* p = part + mh * splits;
     // every load of the kernel is issued before the first result is needed, the token's length included: sixteen
