@@ -244,7 +244,11 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  * weight bytes streamed from HBM) take two launches together: one fused RMSNorm+quantiser launch
  * over every token, then one persistent kernel that streams the packed weights of all of them
  * back to back (dot-products-of-four when every such problem has one token; otherwise the tensor
- * cores, with the codes unpacked in registers and handed over in tensor memory).  Problems of 17 to
+ * cores, with the codes unpacked in registers and handed over in tensor memory).  A call whose
+ * problems all have one token and read the same input row the same way - a level of a decoder
+ * layer: q/k/v, o, gate/up or down - is ONE launch: every CTA quantises the row itself while its
+ * share of the packed weights is on its way (up to four problems in the 2-bit layout; otherwise the
+ * streaming kernel without a quantiser launch in front).  Problems of 17 to
  * 96 tokens (K <= 8192) are cut into 16-token problems for that same decode kernel: streaming the
  * packed weights once per 16 tokens is measured faster there than a tensor-core tile that is mostly
  * padding.  Longer problems (prefill; N must be a multiple of 128) take two launches together: the

@@ -442,21 +442,21 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                                 }
                             }
                         }
-                        continue;
-                    }
-                    // the token's codes are stored with the four 16-byte pieces of each lane's 64 columns interleaved
-                    // (piece q of lane t at 64q + 16t inside the tile), so the four t lanes read 64 contiguous bytes
+                    } else {
+                        // the token's codes are stored with the four 16-byte pieces of each lane's 64 columns interleaved
+                        // (piece q of lane t at 64q + 16t inside the tile), so the four t lanes read 64 contiguous bytes
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        uint4 v;
-                        if (XS) v = lds128(xrow_s + xo + 64u * q);
-                        else v = *reinterpret_cast<const uint4*>(xrow_g + xo + 64 * q);
-                        const uint32_t xw[4] = {v.x, v.y, v.z, v.w};
+                        for (int q = 0; q < 4; ++q) {
+                            uint4 v;
+                            if (XS) v = lds128(xrow_s + xo + 64u * q);
+                            else v = *reinterpret_cast<const uint4*>(xrow_g + xo + 64 * q);
+                            const uint32_t xw[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-                        for (int j = 0; j < 4; ++j) {
-                            const uint32_t mask = 0x03030303u << (2 * j);
-                            acc[0][j] = dp4a_u8_s8(w0[q] & mask, xw[j], acc[0][j]);
-                            acc[1][j] = dp4a_u8_s8(w1[q] & mask, xw[j], acc[1][j]);
+                            for (int j = 0; j < 4; ++j) {
+                                const uint32_t mask = 0x03030303u << (2 * j);
+                                acc[0][j] = dp4a_u8_s8(w0[q] & mask, xw[j], acc[0][j]);
+                                acc[1][j] = dp4a_u8_s8(w1[q] & mask, xw[j], acc[1][j]);
+                            }
                         }
                     }
                 }
