@@ -150,6 +150,25 @@ class DecodeStep:
         bl.bitlinear_glue_residual_add(self.h_mid, self.dn)  # the last layer's residual
         return bl.bitlinear_lm_head(self.h_mid, self.table, out=self.logits)
 
+    def capture(self) -> None:
+        """Record the launches of step() once into a CUDA graph; step_graph() then replays them without the host cost of
+        213 calls.  Token ids, positions and lengths are read from device buffers (ids_buf, positions, lengths), so one
+        recording serves every later token: fill ids_buf and call set_positions() before each replay."""
+        self.ids_buf = torch.zeros(self.M, dtype=torch.int32, device=self.h_in.device)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            self.step(self.ids_buf)  # every kernel has run once outside the recording
+            self.graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(self.graph, stream=side):
+                self.step(self.ids_buf)
+        torch.cuda.current_stream().wait_stream(side)
+
+    def step_graph(self) -> torch.Tensor:
+        """Replay the recorded step on the current ids_buf / positions / lengths -> logits fp32 [M, V]."""
+        self.graph.replay()
+        return self.logits
+
 
 class PersistentChain:
     """The same chain at one token through bitlinear_decode_chain: one cooperative kernel per token."""

@@ -220,3 +220,42 @@ def test_whole_decode_step_stage_by_stage():
     ref = ds.lm_head(h_end, bits(table))
     bound = H * 2.0 ** -24 * (np.abs(bf(h_end)) @ np.abs(bf(bits(table))).T)
     assert np.all(np.abs(logits.cpu().numpy().astype(np.float64) - ref) <= bound)
+
+
+def test_recorded_step_replays_with_new_tokens_and_positions():
+    """DecodeStep.capture(): one recording, replayed for two consecutive tokens, gives what the eager calls give."""
+    from paper_2504_12285_b200 import chain as gpu_chain
+
+    H, F, n_q, n_kv, hd, V, M, t_max = 256, 512, 4, 2, 64, 300, 2, 64
+    layers = []
+    for li in range(2):
+        layer = {}
+        for i, (name, n, k) in enumerate((("q", H, H), ("k", n_kv * hd, H), ("v", n_kv * hd, H), ("o", H, H), ("gate", F, H),
+                                          ("up", F, H), ("down", H, F))):
+            packed, s_w = bl.bitlinear_pack_weights(wl.latent_weights(n, k, 8300 + 10 * li + i).to(DEV), wl.WEIGHT_EPS)
+            layer[name] = (packed, s_w, None)
+        layers.append(layer)
+    table = randn((V, H), 60).to(torch.bfloat16).to(DEV)
+
+    def run(recorded):
+        st = gpu_chain.DecodeStep(layers, table, M, t_max, H, F, n_q, n_kv, hd, wl.RMS_EPS, device=DEV)
+        if recorded:
+            st.capture()
+            for c in st.k_cache + st.v_cache:
+                c.zero_()  # the recording's own runs appended rows at position 0
+        outs = []
+        for t, ids in enumerate(([3, 7], [11, 299])):
+            st.set_positions(torch.full((M,), t, dtype=torch.int32, device=DEV))
+            idt = torch.tensor(ids, dtype=torch.int32, device=DEV)
+            if recorded:
+                st.ids_buf.copy_(idt)
+                outs.append(st.step_graph().clone())
+            else:
+                outs.append(st.step(idt).clone())
+        torch.cuda.synchronize()
+        return outs
+
+    eager, replayed = run(False), run(True)
+    for a, b in zip(eager, replayed):
+        assert torch.isfinite(a).all() and torch.equal(a, b)
+    assert bl.bitlinear_poll_status() == 0
