@@ -7,13 +7,16 @@
 //                               in fp64 because positions reach the thousands), writes q as bf16 and appends k, v to
 //                               the bf16 cache of the token's sequence.
 //   attn_decode_partial_kernel: one CTA per (token, KV head, slice of the cache); 64-row tiles of keys and values arrive
-//                               by tensor-map copies, the query heads of the group are the rows of a tensor-core
-//                               operand (mma.sync, bf16 inputs, fp32 accumulation), softmax in fp32; partial
-//                               (max, sum, weighted values) per slice.
+//                               by tensor-map copies issued by a producer warp, the query heads of the group are the
+//                               8-column side of a tensor-core operand (mma.sync, bf16 inputs, fp32 accumulation),
+//                               softmax in fp32; partial (max, sum, weighted values) per slice.
 //   attn_decode_combine_kernel: merges the slices of a (token, query head) and writes bf16.
-//   lm_head_kernel            : logits = x . E^T for up to 16 tokens, one warp per vocabulary row, the table streamed
-//                               once with 128-bit loads (HBM-bound: 657 MB for 128,256 x 2560).
+//   lm_head_kernel            : logits = x . E^T for one token, one warp per vocabulary row, the table streamed once
+//                               with 128-bit loads (HBM-bound: 657 MB for 128,256 x 2560).
+//   lm_head_mma_kernel        : the same for 2 to 16 tokens on the tensor cores (tokens = rows of the A operand).
 //   embed_kernel              : row gather.
+// All of them but the output head and the gather are launched as programmatic dependents of the launch in front of
+// them and read nothing before griddepcontrol.wait.
 #include "common.cuh"
 #include "sm100_sync.cuh"
 #include "tensor_map.cuh"
