@@ -310,6 +310,9 @@ def run_ours(args):
     decode_step = None
     if rank == 0:
         decode_step = run_decode_step(bl, dev, pool, gains, peaks, packed_bytes, reps=max(5, args.steps))
+        # the same with 16 sequences: attention then streams 168 MB per layer and is bound by bandwidth, not latency
+        decode_step["sixteen_sequences"] = run_decode_step(bl, dev, pool, gains, peaks, packed_bytes, reps=5, M=16)
+        torch.cuda.empty_cache()
 
     # ---- prefill: int8 tensor-core path at M = 2048 on the 7 shapes (rank 0 only) ----
     prefill = None
