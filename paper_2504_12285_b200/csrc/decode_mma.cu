@@ -185,6 +185,9 @@ __global__ void __launch_bounds__(kQuantThreads) mma_quant_kernel(const MmaHeade
     // the kernel that follows may start now: it fetches weights first and waits for this grid before it reads
     // anything written here (programmatic dependent launch)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // this launch is itself a programmatic dependent of whatever runs before it on the stream (its launch overlaps that
+    // kernel's tail); nothing is read before that kernel is complete
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (!mma_plan_matches(hdr, count, total_items, grid, rows)) {
         if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
         return;
@@ -598,11 +601,26 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
     // ---- launch 1: quantise every token into the 16-row tile images ----
     if (!(flags & BITLINEAR_BATCH_REUSE_ACT)) {
         const int* rp = reinterpret_cast<const int*>(base + L.row_prob_off);
-        if (rows <= 2 * 8 * sm_count)  // two tokens per CTA, eight CTAs per SM
-            mma_quant_kernel<4><<<(unsigned)((rows + 1) / 2), kQuantThreads, 0, st>>>(hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
-        else
-            mma_quant_kernel<2><<<(unsigned)((rows + 3) / 4), kQuantThreads, 0, st>>>(hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
-        if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+        cudaLaunchConfig_t qcfg = {};
+        qcfg.blockDim = dim3(kQuantThreads);
+        qcfg.stream = st;
+        cudaLaunchAttribute qattr[1];
+        qattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        qattr[0].val.programmaticStreamSerializationAllowed = 1;
+        qcfg.attrs = qattr;
+        qcfg.numAttrs = 1;
+        cudaError_t qe;
+        if (rows <= 2 * 8 * sm_count) {  // two tokens per CTA, eight CTAs per SM
+            qcfg.gridDim = dim3((unsigned)((rows + 1) / 2));
+            qe = cudaLaunchKernelEx(&qcfg, mma_quant_kernel<4>, hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
+        } else {
+            qcfg.gridDim = dim3((unsigned)((rows + 3) / 4));
+            qe = cudaLaunchKernelEx(&qcfg, mma_quant_kernel<2>, hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
+        }
+        if (qe != cudaSuccess) {
+            cudaGetLastError();
+            return BITLINEAR_ERR_CUDA;
+        }
     }
 
     // ---- launch 2: stream the weights through the tensor cores ----
