@@ -448,9 +448,8 @@ int bitlinear_poll_status(void* stream);
  *   A copy that does not land within the wait limit ends the call's kernels and sets BITLINEAR_ERR_TIMEOUT in the
  *   status word (bitlinear_poll_status).
  * bitlinear_lm_head: logits[m][v] = sum_k x[m][k] * table[v][k], x bf16 [M][K] (M <= 16), table bf16 [V][K], fp32
- *   accumulation and output [M][V].  The table is streamed once per call (one token: fp32 FMAs; 2 to 16 tokens: bf16
- *   tensor-core products, which are exact, accumulated in fp32).  K a multiple of 8; x is staged in shared memory, so
- *   K <= 7168 for M > 1 (BITLINEAR_ERR_SHAPE beyond).
+ *   accumulation and output [M][V].  The table is streamed once per call (bf16 tensor-core products, which are exact,
+ *   accumulated in fp32).  K a multiple of 8; x is staged in shared memory, so K <= 7168 (BITLINEAR_ERR_SHAPE beyond).
  * bitlinear_embed: out[m] = table[ids[m]] (bf16 rows; ids outside 0 .. V-1 are clamped).
  */
 int bitlinear_rope_kv(const float* q, const float* k, const float* v, const int32_t* positions, const int32_t* seq_ids, int M,

@@ -11,9 +11,8 @@
 //                               8-column side of a tensor-core operand (mma.sync, bf16 inputs, fp32 accumulation),
 //                               softmax in fp32; partial (max, sum, weighted values) per slice.
 //   attn_decode_combine_kernel: merges the slices of a (token, query head) and writes bf16.
-//   lm_head_kernel            : logits = x . E^T for one token, one warp per vocabulary row, the table streamed once
-//                               with 128-bit loads (HBM-bound: 657 MB for 128,256 x 2560).
-//   lm_head_mma_kernel        : the same for 2 to 16 tokens on the tensor cores (tokens = rows of the A operand).
+//   lm_head_mma_kernel        : logits = x . E^T for up to 16 tokens on the tensor cores (tokens = rows of the A operand),
+//                               the table streamed once with 128-bit loads (HBM-bound: 657 MB for 128,256 x 2560).
 //   embed_kernel              : row gather.
 // All of them but the output head and the gather are launched as programmatic dependents of the launch in front of
 // them and read nothing before griddepcontrol.wait.
@@ -438,58 +437,11 @@ __global__ void __launch_bounds__(128) attn_decode_combine_kernel(const AttnPart
 
 // ---------------------------------------------------------------------------------------------- output head, embedding
 
-template <int MT>
-__global__ void __launch_bounds__(256) lm_head_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ table,
-                                                      int M, int V, int K, float* __restrict__ logits) {
-    extern __shared__ __align__(16) uint8_t xs_raw[];
-    uint4* xs = reinterpret_cast<uint4*>(xs_raw);  // [MT][K] bf16
-    const int n_vec = K / 8;
-    for (int i = threadIdx.x; i < MT * n_vec; i += blockDim.x) {
-        const int m = i / n_vec;
-        xs[i] = m < M ? reinterpret_cast<const uint4*>(x)[(size_t)m * n_vec + (i - m * n_vec)] : make_uint4(0, 0, 0, 0);
-    }
-    __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int warps = gridDim.x * (blockDim.x >> 5);
-    for (int v = blockIdx.x * (blockDim.x >> 5) + warp; v < V; v += warps) {
-        const uint4* row = reinterpret_cast<const uint4*>(table + (size_t)v * K);
-        float acc[MT];
-#pragma unroll
-        for (int m = 0; m < MT; ++m) acc[m] = 0.0f;
-#pragma unroll 4
-        for (int c = lane; c < n_vec; c += 32) {
-            const uint4 u = __ldcs(row + c);  // streamed once
-            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-            float e[8];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) { e[2 * j] = bf16_lo_f(w[j]); e[2 * j + 1] = bf16_hi_f(w[j]); }
-#pragma unroll
-            for (int m = 0; m < MT; ++m) {
-                const uint4 xu = xs[m * n_vec + c];
-                const uint32_t xw[4] = {xu.x, xu.y, xu.z, xu.w};
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    acc[m] = fmaf(bf16_lo_f(xw[j]), e[2 * j], acc[m]);
-                    acc[m] = fmaf(bf16_hi_f(xw[j]), e[2 * j + 1], acc[m]);
-                }
-            }
-        }
-#pragma unroll
-        for (int m = 0; m < MT; ++m) {
-            float a = acc[m];
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-            if (lane == 0 && m < M) logits[(size_t)m * V + v] = a;
-        }
-    }
-}
-
-// The output head for 2 .. 16 tokens on the tensor cores: the tokens are the 16 rows of the A operand (zero rows past M),
+// The output head for 1 .. 16 tokens on the tensor cores: the tokens are the 16 rows of the A operand (zero rows past M),
 // eight vocabulary rows are the columns of B.  A lane loads 16 bytes (eight consecutive k) of its vocabulary row straight
 // from global memory and uses them as the B registers of two mma.sync steps; since a dot product does not care about
 // the order of k, the k-slots of a step are simply those eight values of the four lanes that share a column, and the
 // A operand (x, staged in shared memory) is read with the same assignment.  The table is streamed once.
-template <bool HI_ROWS>  // tokens 8 .. 15 present
 __global__ void __launch_bounds__(512) lm_head_mma_kernel(const __nv_bfloat16* __restrict__ x, const __nv_bfloat16* __restrict__ table,
                                                           int M, int V, int K, int x_stride, float* __restrict__ logits) {
     extern __shared__ __align__(16) uint8_t xs_raw[];  // [16][x_stride bytes]: rows 64 bytes apart modulo 128
@@ -506,41 +458,53 @@ __global__ void __launch_bounds__(512) lm_head_mma_kernel(const __nv_bfloat16* _
     const uint8_t* xa = xs_raw + (size_t)g * x_stride + sq * 16;
     const uint8_t* xb = xa + (size_t)8 * x_stride;
     const int k_blocks = K / 32;  // whole 32-k blocks; K % 32 is handled by the tail below
-    for (int v0 = 8 * (blockIdx.x * (blockDim.x >> 5) + warp); v0 < V; v0 += 8 * warps) {
-        const uint4* row = reinterpret_cast<const uint4*>(table + (size_t)min(v0 + g, V - 1) * K) + sq;
-        float c[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-        auto step = [&](const uint4& b, int kb) {
+    // a warp takes sixteen vocabulary rows per pass - two B operands for every A fragment it reads from shared memory, which
+    // halves the shared-memory traffic per table byte (with sixteen tokens that traffic is what bounds the kernel)
+    for (int v0 = 16 * (blockIdx.x * (blockDim.x >> 5) + warp); v0 < V; v0 += 16 * warps) {
+        const uint4* row0 = reinterpret_cast<const uint4*>(table + (size_t)min(v0 + g, V - 1) * K) + sq;
+        const uint4* row1 = reinterpret_cast<const uint4*>(table + (size_t)min(v0 + 8 + g, V - 1) * K) + sq;
+        float c[2][4] = {{0.0f, 0.0f, 0.0f, 0.0f}, {0.0f, 0.0f, 0.0f, 0.0f}};
+        auto mma2 = [&](float (&d)[4], const uint4& a, const uint4& a8, const uint4& bq) {
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                         : "r"(a.x), "r"(a8.x), "r"(a.y), "r"(a8.y), "r"(bq.x), "r"(bq.y));
+            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+                         : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                         : "r"(a.z), "r"(a8.z), "r"(a.w), "r"(a8.w), "r"(bq.z), "r"(bq.w));
+        };
+        auto step = [&](const uint4& b0, const uint4& b1, int kb) {
             const uint4 a = *reinterpret_cast<const uint4*>(xa + kb * 64);
-            uint4 a8 = make_uint4(0, 0, 0, 0);
-            if constexpr (HI_ROWS) a8 = *reinterpret_cast<const uint4*>(xb + kb * 64);
-            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                         : "r"(a.x), "r"(a8.x), "r"(a.y), "r"(a8.y), "r"(b.x), "r"(b.y));
-            asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
-                         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-                         : "r"(a.z), "r"(a8.z), "r"(a.w), "r"(a8.w), "r"(b.z), "r"(b.w));
+            const uint4 a8 = *reinterpret_cast<const uint4*>(xb + kb * 64);
+            mma2(c[0], a, a8, b0);
+            mma2(c[1], a, a8, b1);
         };
         int kb = 0;
-        for (; kb + 8 <= k_blocks; kb += 8) {  // eight loads in flight per lane
-            uint4 b[8];
+        for (; kb + 4 <= k_blocks; kb += 4) {  // eight loads in flight per lane
+            uint4 b0[4], b1[4];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) b[u] = __ldcs(row + (kb + u) * 4);
+            for (int u = 0; u < 4; ++u) {
+                b0[u] = __ldcs(row0 + (kb + u) * 4);
+                b1[u] = __ldcs(row1 + (kb + u) * 4);
+            }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) step(b[u], kb + u);
+            for (int u = 0; u < 4; ++u) step(b0[u], b1[u], kb + u);
         }
-        for (; kb < k_blocks; ++kb) step(__ldcs(row + kb * 4), kb);
+        for (; kb < k_blocks; ++kb) step(__ldcs(row0 + kb * 4), __ldcs(row1 + kb * 4), kb);
         if (K % 32) {  // 8, 16 or 24 columns left: the lanes whose chunk lies past the end contribute zeros
-            const uint4 b = sq * 8 < K % 32 ? __ldcs(row + kb * 4) : make_uint4(0, 0, 0, 0);
-            step(b, kb);  // the staged x row is zero-padded up to the next 32 columns
-        }
-        const int v = v0 + 2 * sq;
-        if (g < M) {
-            if (v < V) logits[(size_t)g * V + v] = c[0];
-            if (v + 1 < V) logits[(size_t)g * V + v + 1] = c[1];
-        }
-        if (HI_ROWS && g + 8 < M) {
-            if (v < V) logits[(size_t)(g + 8) * V + v] = c[2];
-            if (v + 1 < V) logits[(size_t)(g + 8) * V + v + 1] = c[3];
+            const bool in = sq * 8 < K % 32;
+            step(in ? __ldcs(row0 + kb * 4) : make_uint4(0, 0, 0, 0), in ? __ldcs(row1 + kb * 4) : make_uint4(0, 0, 0, 0), kb);
+        }  // (the staged x row is zero-padded up to the next 32 columns)
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int v = v0 + 8 * h + 2 * sq;
+            if (g < M) {
+                if (v < V) logits[(size_t)g * V + v] = c[h][0];
+                if (v + 1 < V) logits[(size_t)g * V + v + 1] = c[h][1];
+            }
+            if (g + 8 < M) {
+                if (v < V) logits[(size_t)(g + 8) * V + v] = c[h][2];
+                if (v + 1 < V) logits[(size_t)(g + 8) * V + v + 1] = c[h][3];
+            }
         }
     }
 }
@@ -727,22 +691,16 @@ int bitlinear_lm_head(const void* x_bf16, const void* table_bf16, int M, int V, 
     if (const int rc = device_sm_count(&sm_count)) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __nv_bfloat16 *xp = static_cast<const __nv_bfloat16*>(x_bf16), *tp = static_cast<const __nv_bfloat16*>(table_bf16);
-    auto launch = [&](auto kernel, unsigned grid, unsigned threads, size_t smem, auto... args) {
-        if (smem > 48 * 1024 && cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
-            cudaGetLastError();
-            return (int)BITLINEAR_ERR_SHAPE;  // K too large for the staged activations
-        }
-        kernel<<<grid, threads, smem, st>>>(args...);
-        return cudaGetLastError() == cudaSuccess ? (int)BITLINEAR_OK : (int)BITLINEAR_ERR_CUDA;
-    };
-    if (M == 1) return launch(lm_head_kernel<1>, (unsigned)(sm_count * 4), 256u, (size_t)K * 2, xp, tp, M, V, K, logits);
     // rows of the staged x: K rounded up to 32 columns (zero-filled), 64 bytes apart modulo 128 so that the two rows a
     // quarter-warp reads together fall into different halves of the banks
     const int x_stride = ((K + 31) / 32 * 64 + 127) / 128 * 128 + 64;
     const size_t smem = (size_t)16 * x_stride;
-    const unsigned grid = (unsigned)(sm_count * 2);
-    return M <= 8 ? launch(lm_head_mma_kernel<false>, grid, 512u, smem, xp, tp, M, V, K, x_stride, logits)
-                  : launch(lm_head_mma_kernel<true>, grid, 512u, smem, xp, tp, M, V, K, x_stride, logits);
+    if (cudaFuncSetAttribute(lm_head_mma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) {
+        cudaGetLastError();
+        return BITLINEAR_ERR_SHAPE;  // K too large for the staged activations
+    }
+    lm_head_mma_kernel<<<(unsigned)(sm_count * 2), 512, smem, st>>>(xp, tp, M, V, K, x_stride, logits);
+    return cudaGetLastError() == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
 int bitlinear_embed(const int32_t* ids, const void* table_bf16, int M, int V, int K, void* out_bf16, void* stream) {
