@@ -649,6 +649,41 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     char* base = static_cast<char*>(ws);
 
+    // ---- a level of a decoder layer called again (REUSE_PLAN): up to four one-token problems on one input row need no host
+    //      plan at all - the launch carries its descriptors, and the quantised row goes where the plan of the first call put it
+    if ((flags & BITLINEAR_BATCH_REUSE_PLAN) && !(flags & BITLINEAR_BATCH_REUSE_ACT) && !dense && count <= kLevelMaxProblems &&
+        rows == (size_t)count) {
+        const bitlinear_problem& q0 = problems[0];
+        bool one_input = true;
+        int total_rb0 = 0;
+        for (int i = 0; i < count; ++i) {
+            const bitlinear_problem& q = problems[i];
+            one_input = one_input && q.x == q0.x && q.x2 == q0.x2 && q.gain == q0.gain && q.x_out == q0.x_out && q.K == q0.K &&
+                        q.x_op == q0.x_op && q.x_arg0 == q0.x_arg0 && q.x_arg1 == q0.x_arg1 && q.rms_eps == q0.rms_eps;
+            total_rb0 += q.N / kTileRows;
+        }
+        if (one_input && decode_level_fits(count, total_rb0, q0.K, sm_count)) {
+            LevelParams P = {};
+            P.count = count;
+            for (int i = 0; i < count; ++i) {
+                const bitlinear_problem& q = problems[i];
+                P.prob[i].packed = static_cast<const uint8_t*>(q.packed); P.prob[i].s_w = q.s_w; P.prob[i].y = q.y;
+                P.prob[i].acc_out = acc_outs ? acc_outs[i] : nullptr;
+                P.prob[i].N = q.N; P.prob[i].y_dtype = q.y_dtype;
+            }
+            P.x = q0.x;
+            P.op.x2 = q0.x2; P.op.x_out = q0.x_out; P.op.op = q0.x_op; P.op.arg0 = q0.x_arg0; P.op.arg1 = q0.x_arg1; P.op.pad = 0;
+            P.gain = static_cast<const __nv_bfloat16*>(q0.gain); P.eps = q0.rms_eps; P.K = q0.K; P.x_row0 = 0;
+            // the places the plan gives the first entry's quantised row, scale and code sum (see below)
+            P.xq_out = reinterpret_cast<int8_t*>(base + L.xq_off);
+            P.d_out = reinterpret_cast<float*>(base + align_up(L.xq_off + xq_bytes, 256));
+            P.xsum_out = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(P.d_out) + align_up(rows * sizeof(float), 256));
+            P.total_rb = total_rb0;
+            P.status_word = device_status_word();
+            return decode_level_forward(P, sm_count, st, /*dependent=*/true);
+        }
+    }
+
     // ---- host plan: device descriptors, token -> problem table, byte-balanced CTA ranges ----
     std::vector<DevProblem> dp;
     std::vector<int> row_prob;
