@@ -259,3 +259,38 @@ def test_recorded_step_replays_with_new_tokens_and_positions():
     for a, b in zip(eager, replayed):
         assert torch.isfinite(a).all() and torch.equal(a, b)
     assert bl.bitlinear_poll_status() == 0
+
+
+def test_replayed_token_is_deterministic_at_full_layer_shapes():
+    """Every launch of a recorded token is a programmatic dependent of the one before it and starts early (weights, gains
+    and scales are fetched while the predecessor still runs).  A read that came too early would show as a result that
+    changes from replay to replay: 300 replays of one token on two full-size layers must give the same bits, and the
+    same bits as the eager calls."""
+    from paper_2504_12285_b200 import chain as gpu_chain
+
+    H, F, n_q, n_kv, hd, V, t_max = wl.HIDDEN, wl.FFN, wl.N_Q_HEADS, wl.N_KV_HEADS, wl.HEAD_DIM, 4096, 4096
+    layers = []
+    for li in range(2):
+        layer = {}
+        for i, (name, n, k) in enumerate(wl.LAYER_SHAPES):
+            packed, s_w = bl.bitlinear_pack_weights(wl.latent_weights(n, k, 8500 + 10 * li + i).to(DEV), wl.WEIGHT_EPS)
+            layer[name] = (packed, s_w, wl.gain_random(k, 8600 + 10 * li + i).to(DEV))
+        layers.append(layer)
+    table = randn((V, H), 70, 0.05).to(torch.bfloat16).to(DEV)
+    st = gpu_chain.DecodeStep(layers, table, 1, t_max, H, F, n_q, n_kv, hd, wl.RMS_EPS, device=DEV)
+    gen = torch.Generator(device=DEV).manual_seed(71)
+    for c in st.k_cache + st.v_cache:
+        c.copy_(torch.randn(c.shape, generator=gen, device=DEV))
+    st.set_positions(torch.tensor([t_max - 1], dtype=torch.int32, device=DEV))
+    ids = torch.tensor([1234], dtype=torch.int32, device=DEV)
+    want = st.step(ids).clone()
+    assert torch.isfinite(want).all()
+    st.capture()
+    st.ids_buf.copy_(ids)
+    for _ in range(300):
+        got = st.step_graph()
+        assert torch.equal(got, want)  # (the comparison synchronises: replays do not pile up)
+    for _ in range(50):  # and back to back: the first launch of a token overlaps the last launches of the token before
+        st.step_graph()
+    assert torch.equal(st.logits, want)
+    assert bl.bitlinear_poll_status() == 0
