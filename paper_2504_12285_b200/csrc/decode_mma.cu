@@ -172,6 +172,29 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 // D = s32, A = u8 (64 x weight code, tensor memory), B = s8 (activations, K-major shared memory), M = 128, N = 16.
 constexpr uint32_t kIdesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(kTok >> 3) << 17) | ((uint32_t)(kRows >> 4) << 24);
 
+// One CTA per token, the row kept in registers (one read of the input): for calls with so few tokens that they do not
+// even give every SM a CTA - a level of a decoder layer at 2 to 16 tokens - where the latency of a token's chain is all
+// that counts.
+template <int VPT>
+__global__ void __launch_bounds__(kQuantThreads) mma_quant_row_kernel(const MmaHeader* __restrict__ hdr,
+                                                                      const MmaProblem* __restrict__ probs,
+                                                                      const int* __restrict__ row_prob, int count, int total_items,
+                                                                      int grid, int rows, int* status_word) {
+    __shared__ RowReduceSmem sm;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");  // see mma_quant_kernel
+    if (!mma_plan_matches(hdr, count, total_items, grid, rows)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
+        return;
+    }
+    const int row = blockIdx.x;
+    const MmaProblem& p = probs[row_prob[row]];
+    const int m = row - p.row_begin;
+    with_row_source(p.op, p.x, m, p.K, [&](auto src) {
+        quant_row_src<VPT, 3>(src, p.gain, p.eps, p.K, p.xq_out + (size_t)m * 128, p.d_out + m, p.xsum_out + m, sm, m & 7);
+    });
+}
+
 // kQuantGroupWarps warps per token: there are at most a few thousand tokens here, and with one warp per token a
 // 6,912-element token is a serial chain of thousands of instructions for its warp while most of the GPU idles.
 // (Four warps per token while that still fits one wave of CTAs, two beyond.)
@@ -610,7 +633,14 @@ int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, 
         qcfg.attrs = qattr;
         qcfg.numAttrs = 1;
         cudaError_t qe;
-        if (rows <= 2 * 8 * sm_count) {  // two tokens per CTA, eight CTAs per SM
+        if (rows <= sm_count) {  // a CTA per token (K <= 8192: at most four 16-byte vectors per thread)
+            qcfg.gridDim = dim3((unsigned)rows);
+            int max_k = 0;
+            for (const MmaProblem& q : mp) max_k = std::max(max_k, q.K);
+            qe = max_k <= 8 * 2 * kQuantThreads
+                     ? cudaLaunchKernelEx(&qcfg, mma_quant_row_kernel<2>, hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw)
+                     : cudaLaunchKernelEx(&qcfg, mma_quant_row_kernel<4>, hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
+        } else if (rows <= 2 * 8 * sm_count) {  // two tokens per CTA, eight CTAs per SM
             qcfg.gridDim = dim3((unsigned)((rows + 1) / 2));
             qe = cudaLaunchKernelEx(&qcfg, mma_quant_kernel<4>, hdr, probs_dev, rp, n_prob, total_items, grid, rows, sw);
         } else {
