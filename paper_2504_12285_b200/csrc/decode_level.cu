@@ -26,7 +26,10 @@ namespace bitlinear {
 namespace {
 
 constexpr int kLevelThreads = 512;
-constexpr int kLevelCtasPerSm = 1;  // CTAs per SM the row blocks are dealt to (2 measured slower: 1.13 against 1.07 ms per token)
+// CTAs per SM the row blocks are dealt to: with two, a CTA's weight copy and products halve while the quantiser, which every
+// CTA repeats anyway, runs in parallel.  Measured per decoded token of the 2B configuration (CUDA graph): 1.05 ms with
+// one CTA per SM, 1.00 ms with two, 1.11 ms when the largest level is dealt to three (a second wave of CTAs).
+constexpr int kLevelCtasPerSm = 2;
 constexpr int kLevelWarps = kLevelThreads / 32;
 
 __device__ __forceinline__ int dp4a_u8_s8(uint32_t a_u8x4, uint32_t b_s8x4, int c) {
@@ -222,11 +225,6 @@ bool decode_level_fits(int count, int total_rb, int K, int sm_count) {
 
 int decode_level_forward(LevelParams& P, int sm_count, cudaStream_t st, bool dependent) {
     P.rb_per_cta = (P.total_rb + kLevelCtasPerSm * sm_count - 1) / (kLevelCtasPerSm * sm_count);
-    // a level of fewer than two row blocks per SM gets one row block per CTA (up to two CTAs on an SM): the copy and the
-    // products of a CTA halve while the quantiser, which every CTA repeats anyway, runs in parallel - measured on the
-    // q/k/v, o and down levels of the 2B layer: 1.02 ms per decoded token against 1.05 ms; with more row blocks (gate/up)
-    // twice the CTAs were slower
-    if (P.rb_per_cta == 2) P.rb_per_cta = 1;
     const int grid = (P.total_rb + P.rb_per_cta - 1) / P.rb_per_cta;
     const size_t smem = level_smem_bytes(P.rb_per_cta, P.K);
     const cudaError_t e = P.K <= 8 * kLevelThreads ? launch_level<1>(P, grid, smem, st, dependent) : launch_level<2>(P, grid, smem, st, dependent);
