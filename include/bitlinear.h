@@ -447,6 +447,19 @@ int bitlinear_poll_status(void* stream);
  *   partial results per token and query head.
  *   A copy that does not land within the wait limit ends the call's kernels and sets BITLINEAR_ERR_TIMEOUT in the
  *   status word (bitlinear_poll_status).
+ * bitlinear_rope_table: table_out (device, fp32 [t_max][D/2][2], 16-byte aligned) receives (cos, sin) of
+ *   position * rope_base^(-2i/D) for every cache position and pair i, from the same fp64 angle as bitlinear_rope_kv.
+ *   D = 64 or 128.  Built once per (rope_base, D, t_max).
+ * bitlinear_attention_decode_append: bitlinear_rope_kv followed by bitlinear_attention_decode in the attention
+ *   launches themselves (one launch per layer fewer), for the usual decode step in which token m is the newest row
+ *   of its sequence: its position is lengths[m] - 1.  q, k, v fp32 as for bitlinear_rope_kv (16-byte aligned);
+ *   rope_table from bitlinear_rope_table with the same D and a t_max at least this call's; the caches receive the
+ *   rotated k and the unrotated v at row lengths[m] - 1 (the same bits bitlinear_rope_kv stores) and the token
+ *   attends to rows 0 .. lengths[m] - 1, its own included; out as for bitlinear_attention_decode, the same bits as the
+ *   two-call route.  A length outside 1 .. t_max or a sequence outside 0 .. n_seq-1 stores nothing and gives a zero
+ *   row.  The tokens of one call must belong to DIFFERENT sequences (a token does not see rows stored by another
+ *   token of the same call; use the two-call route for that); this is not checked.  Other limits, the workspace and
+ *   the status word as for bitlinear_attention_decode.
  * bitlinear_lm_head: logits[m][v] = sum_k x[m][k] * table[v][k], x bf16 [M][K] (M <= 16), table bf16 [V][K], fp32
  *   accumulation and output [M][V].  The table is streamed once per call (bf16 tensor-core products, which are exact,
  *   accumulated in fp32).  K a multiple of 8; x is staged in shared memory, so K <= 7168 (BITLINEAR_ERR_SHAPE beyond).
@@ -459,6 +472,11 @@ size_t bitlinear_attention_workspace_bytes(int M, int n_q_heads, int n_kv_heads,
 int bitlinear_attention_decode(const void* q_bf16, const void* k_cache_bf16, const void* v_cache_bf16, const int32_t* lengths,
                                const int32_t* seq_ids, int M, int n_q_heads, int n_kv_heads, int head_dim, int n_seq, int t_max,
                                void* out_bf16, void* ws, size_t ws_bytes, void* stream);
+int bitlinear_rope_table(float rope_base, int head_dim, int t_max, float* table_out, void* stream);
+int bitlinear_attention_decode_append(const float* q, const float* k, const float* v, const float* rope_table, void* k_cache_bf16,
+                                      void* v_cache_bf16, const int32_t* lengths, const int32_t* seq_ids, int M, int n_q_heads,
+                                      int n_kv_heads, int head_dim, int n_seq, int t_max, void* out_bf16, void* ws, size_t ws_bytes,
+                                      void* stream);
 int bitlinear_lm_head(const void* x_bf16, const void* table_bf16, int M, int V, int K, float* logits, void* stream);
 int bitlinear_embed(const int32_t* ids, const void* table_bf16, int M, int V, int K, void* out_bf16, void* stream);
 

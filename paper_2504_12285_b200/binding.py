@@ -55,6 +55,10 @@ _SIGNATURES = {
     "bitlinear_attention_workspace_bytes": (_c_size_t, [_c_int, _c_int, _c_int, _c_int, _c_int]),
     "bitlinear_attention_decode": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_int,
                                             _c_int, _c_int, _c_void_p, _c_void_p, _c_size_t, _c_void_p]),
+    "bitlinear_rope_table": (_c_int, [_c_float, _c_int, _c_int, _c_void_p, _c_void_p]),
+    "bitlinear_attention_decode_append": (_c_int, [_c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p, _c_void_p,
+                                                   _c_int, _c_int, _c_int, _c_int, _c_int, _c_int, _c_void_p, _c_void_p, _c_size_t,
+                                                   _c_void_p]),
     "bitlinear_lm_head": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_void_p]),
     "bitlinear_embed": (_c_int, [_c_void_p, _c_void_p, _c_int, _c_int, _c_int, _c_void_p, _c_void_p]),
     "bitlinear_poll_status": (_c_int, [_c_void_p]),
@@ -560,6 +564,37 @@ def bitlinear_attention_decode(q, k_cache, v_cache, lengths, n_q_heads: int, n_k
     rc = lib().bitlinear_attention_decode(_ptr(q), _ptr(k_cache), _ptr(v_cache), _ptr(lengths), _ptr(seq_ids), M, n_q_heads,
                                           n_kv_heads, head_dim, n_seq, t_max, _ptr(out), _ptr(ws), ws.numel(), _stream())
     _check(rc, "bitlinear_attention_decode")
+    return out
+
+
+def bitlinear_rope_table(head_dim: int, t_max: int, rope_base: float = 500000.0, device="cuda:0"):
+    """(cos, sin) of every (position, pair) -> fp32 [t_max, D / 2, 2], for bitlinear_attention_decode_append."""
+    table = torch.empty(t_max, head_dim // 2, 2, dtype=torch.float32, device=device)
+    with torch.cuda.device(table.device):
+        _check(lib().bitlinear_rope_table(rope_base, head_dim, t_max, _ptr(table), _stream()), "bitlinear_rope_table")
+    return table
+
+
+def bitlinear_attention_decode_append(q, k, v, rope_table, k_cache, v_cache, lengths, n_q_heads: int, n_kv_heads: int, head_dim: int,
+                                      seq_ids=None, out=None, ws=None):
+    """Rotary embedding, cache append at row lengths[m] - 1 and attention over rows 0 .. lengths[m] - 1 in the attention
+    launches: q, k, v fp32 projections of one token per (distinct) sequence -> bf16 [M, n_q * D]."""
+    _dev(q, torch.float32, "q"), _dev(k, torch.float32, "k"), _dev(v, torch.float32, "v"), _dev(rope_table, torch.float32, "rope_table")
+    _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache"), _dev(lengths, torch.int32, "lengths")
+    if seq_ids is not None:
+        _dev(seq_ids, torch.int32, "seq_ids")
+    M = q.shape[0]
+    n_seq, t_max = _cache_dims(k_cache, v_cache, n_kv_heads, head_dim)
+    if rope_table.dim() != 3 or rope_table.shape[0] < t_max or tuple(rope_table.shape[1:]) != (head_dim // 2, 2):
+        raise ValueError(f"rope_table must be [>= {t_max}, {head_dim // 2}, 2]")
+    if out is None:
+        out = torch.empty(M, n_q_heads * head_dim, dtype=torch.bfloat16, device=q.device)
+    if ws is None:
+        ws = _workspace(bitlinear_attention_workspace_bytes(M, n_q_heads, n_kv_heads, head_dim, t_max), q.device)
+    rc = lib().bitlinear_attention_decode_append(_ptr(q), _ptr(k), _ptr(v), _ptr(rope_table), _ptr(k_cache), _ptr(v_cache),
+                                                 _ptr(lengths), _ptr(seq_ids), M, n_q_heads, n_kv_heads, head_dim, n_seq, t_max,
+                                                 _ptr(out), _ptr(ws), ws.numel(), _stream())
+    _check(rc, "bitlinear_attention_decode_append")
     return out
 
 

@@ -81,9 +81,14 @@ class DecodeStep:
     every layer's cache."""
 
     def __init__(self, layers, embedding: torch.Tensor, M: int, t_max: int, hidden: int, ffn: int, n_q_heads: int,
-                 n_kv_heads: int, head_dim: int, rms_eps: float = 1e-5, rope_base: float = 500000.0, device="cuda:0"):
-        """layers: as for DecodeChain; embedding: bf16 [V, hidden], used for the gather and as the output head."""
+                 n_kv_heads: int, head_dim: int, rms_eps: float = 1e-5, rope_base: float = 500000.0, device="cuda:0",
+                 append_in_attention: bool = True):
+        """layers: as for DecodeChain; embedding: bf16 [V, hidden], used for the gather and as the output head.
+        append_in_attention: rotary embedding and cache append run inside the attention launches (same bits, one launch
+        per layer fewer); False keeps them a launch of their own, which also leaves the rotated q in q_rot."""
         dev = torch.device(device)
+        self.append_in_attention = append_in_attention
+        self.rope_table = bl.bitlinear_rope_table(head_dim, t_max, rope_base, device=dev) if append_in_attention else None
         self.M, self.dims, self.rope_base, self.table = M, (n_q_heads, n_kv_heads, head_dim), rope_base, embedding
         kv = n_kv_heads * head_dim
         f32 = dict(dtype=torch.float32, device=dev)
@@ -126,9 +131,9 @@ class DecodeStep:
 
     @property
     def launches_per_layer(self) -> int:
-        """Four levels (one launch each at one token, quantiser + weight stream otherwise), rotary/append, attention
-        slices, attention merge."""
-        return (4 if self.M == 1 else 8) + 3
+        """Four levels (one launch each at one token, quantiser + weight stream otherwise), attention slices, attention
+        merge, and rotary/append where that is a launch of its own."""
+        return (4 if self.M == 1 else 8) + (2 if self.append_in_attention else 3)
 
     def set_positions(self, positions: torch.Tensor) -> None:
         """positions: int32 [M] (device): where the next token of each sequence goes; it attends to rows 0 .. position."""
@@ -141,10 +146,14 @@ class DecodeStep:
         bl.bitlinear_embed(ids, self.table, out=self.h_in)
         for li, (qkv, o, gu, down) in enumerate(self.calls):
             bl.bitlinear_forward_batch(*qkv, reuse_plan=True)
-            bl.bitlinear_rope_kv(self.q, self.k, self.v, self.positions, self.k_cache[li], self.v_cache[li], n_q, n_kv, hd,
-                                 rope_base=self.rope_base, seq_ids=self.seq_ids, q_out=self.q_rot)
-            bl.bitlinear_attention_decode(self.q_rot, self.k_cache[li], self.v_cache[li], self.lengths, n_q, n_kv, hd,
-                                          seq_ids=self.seq_ids, out=self.attn, ws=self.attn_ws)
+            if self.append_in_attention:
+                bl.bitlinear_attention_decode_append(self.q, self.k, self.v, self.rope_table, self.k_cache[li], self.v_cache[li],
+                                                     self.lengths, n_q, n_kv, hd, seq_ids=self.seq_ids, out=self.attn, ws=self.attn_ws)
+            else:
+                bl.bitlinear_rope_kv(self.q, self.k, self.v, self.positions, self.k_cache[li], self.v_cache[li], n_q, n_kv, hd,
+                                     rope_base=self.rope_base, seq_ids=self.seq_ids, q_out=self.q_rot)
+                bl.bitlinear_attention_decode(self.q_rot, self.k_cache[li], self.v_cache[li], self.lengths, n_q, n_kv, hd,
+                                              seq_ids=self.seq_ids, out=self.attn, ws=self.attn_ws)
             for batch, ws in (o, gu, down):
                 bl.bitlinear_forward_batch(batch, ws, reuse_plan=True)
         bl.bitlinear_glue_residual_add(self.h_mid, self.dn)  # the last layer's residual
@@ -152,7 +161,7 @@ class DecodeStep:
 
     def capture(self) -> None:
         """Record the launches of step() once into a CUDA graph; step_graph() then replays them without the host cost of
-        213 calls.  Token ids, positions and lengths are read from device buffers (ids_buf, positions, lengths), so one
+        a few hundred calls.  Token ids, positions and lengths are read from device buffers (ids_buf, positions, lengths), so one
         recording serves every later token: fill ids_buf and call set_positions() before each replay."""
         self.ids_buf = torch.zeros(self.M, dtype=torch.int32, device=self.h_in.device)
         side = torch.cuda.Stream()

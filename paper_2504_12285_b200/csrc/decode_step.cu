@@ -33,6 +33,23 @@ __device__ __forceinline__ float bf16_hi_f(uint32_t w) { return __uint_as_float(
 
 // ---------------------------------------------------------------------------------------------- RoPE + cache append
 
+// (cos, sin) of position * base^(-2i / head_dim), formed in fp64 and rounded once: the one place the angle is computed,
+// so the table built from it and the kernel that rotates without a table give the same bits
+__device__ __forceinline__ float2 rope_cos_sin(int pos, int i, int hd, double log2_base) {
+    const double angle = (double)pos * exp2(-2.0 * (double)i / (double)hd * log2_base);
+    double sd, cd;
+    sincos(angle, &sd, &cd);
+    return make_float2((float)cd, (float)sd);
+}
+
+// table[pos][i] = (cos, sin) for every cache position and rotation pair
+__global__ void __launch_bounds__(256) rope_table_kernel(float2* __restrict__ table, int t_max, int hd, double log2_base) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int half = hd / 2;
+    if (idx >= (long long)t_max * half) return;
+    table[idx] = rope_cos_sin((int)(idx / half), (int)(idx % half), hd, log2_base);
+}
+
 __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ q, const float* __restrict__ k,
                                                       const float* __restrict__ v, const int* __restrict__ positions,
                                                       const int* __restrict__ seq_ids, int M, int n_q, int n_kv, int hd, int n_seq,
@@ -51,10 +68,8 @@ __global__ void __launch_bounds__(256) rope_kv_kernel(const float* __restrict__ 
         const int m = (int)(idx / pairs_per_tok), r = (int)(idx - (long long)m * pairs_per_tok);
         const int head = r / half, i = r - head * half;
         const int pos = positions[m];
-        const double angle = (double)pos * exp2(-2.0 * (double)i / (double)hd * log2_base);
-        double sd, cd;
-        sincos(angle, &sd, &cd);
-        const float c = (float)cd, s = (float)sd;
+        const float2 cs = rope_cos_sin(pos, i, hd, log2_base);
+        const float c = cs.x, s = cs.y;
         const bool is_q = head < n_q;
         const float* src = is_q ? q + (size_t)m * n_q * hd + (size_t)head * hd : k + (size_t)m * n_kv * hd + (size_t)(head - n_q) * hd;
         const float lo = src[i], hi = src[i + half];
@@ -138,6 +153,15 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<const uint32_t*>(&v);
 }
 
+// Cache rows token m attends to.  Plain calls clamp the given length to the cache; a call that appends the token's own
+// row (row length - 1) takes a length outside 1 .. t_max as "no token" (nothing stored, a zero result).
+__device__ __forceinline__ int attn_len(const int* __restrict__ lengths, int seq, int m, int n_seq, int t_max, bool own_row) {
+    if (seq < 0 || seq >= n_seq) return 0;
+    const int raw = lengths[m];
+    if (own_row) return (raw >= 1 && raw <= t_max) ? raw : 0;
+    return min(max(raw, 0), t_max);
+}
+
 // One CTA per (slice of the cache, KV head, token): four consumer warps and one producer warp.  A slice is a run of
 // 64-row tiles; each tile's key and value rows of this KV head (64 x HD bf16 each) arrive in shared memory by
 // tensor-map copies of 64 rows x 128 bytes (128-byte swizzle; a head's rows are contiguous in the cache, so a tile is
@@ -156,10 +180,27 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // are not read by the combine kernel.  Rows of a tile past the token's length are copied (they are inside the cache,
 // or zero-filled past its end); their scores are discarded by a select and their value rows are overwritten with zeros
 // before use, so whatever bits they hold never enter a result.
-template <int HD>
+//
+// With OWN (the token's own row is part of the call) the kernel also does the work of the rotary-embedding launch: q, k
+// and v arrive as fp32 projections; every consumer warp rotates the group's query heads itself (cos, sin from a
+// table, the same fp32 operations in the same order as rope_kv_kernel, hence the same bits); the one warp whose keys
+// include row length - 1 rotates k, rounds k and v to bf16, stores them to the cache in global memory and, once the
+// tile has landed, over the row's stale copy in shared memory.  No other CTA reads that row: it lies in one slice of
+// one (token, KV head), and the tokens of such a call belong to different sequences.
+struct AttnOwnRow {
+    const float* q;        // [M][n_q * HD]   fp32, not rotated
+    const float* k;        // [M][n_kv * HD]
+    const float* v;        // [M][n_kv * HD]
+    const float2* table;   // [t_max][HD / 2] (cos, sin)
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+};
+
+template <int HD, bool OWN>
 __global__ void __launch_bounds__(160) attn_decode_partial_kernel(const __grid_constant__ CUtensorMap map_k,
                                                                   const __grid_constant__ CUtensorMap map_v,
-                                                                  const __nv_bfloat16* __restrict__ q, const int* __restrict__ lengths,
+                                                                  const __nv_bfloat16* __restrict__ q, const AttnOwnRow own,
+                                                                  const int* __restrict__ lengths,
                                                                   const int* __restrict__ seq_ids, int n_q, int n_kv, int n_seq, int t_max,
                                                                   int splits, int stages, float scale,
                                                                   AttnPartial<HD>* __restrict__ part, int* __restrict__ status_word) {
@@ -192,7 +233,7 @@ __global__ void __launch_bounds__(160) attn_decode_partial_kernel(const __grid_c
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");  // nothing is read from global memory before this
     const int seq = seq_ids ? seq_ids[m] : 0;
-    const int len = (seq >= 0 && seq < n_seq) ? min(max(lengths[m], 0), t_max) : 0;
+    const int len = attn_len(lengths, seq, m, n_seq, t_max, OWN);
     const AttnSlices sl = attn_slices(len, splits);
     if (split >= sl.live) return;  // the whole CTA: nothing of this slice is live
     const int tile0 = split * sl.per;
@@ -225,15 +266,62 @@ __global__ void __launch_bounds__(160) attn_decode_partial_kernel(const __grid_c
         // ---- consumers
         // Q^T as the B operand: column g = head kvh * group + g (zero columns past the group), two registers per k-step
         uint32_t qb[KS][2];
-        {
+        const int kb = warp * 16;  // this warp's keys of a tile
+        // OWN: the token's own row is row `pos`, in tile `own_tile` of this slice if this CTA has it at all, and among
+        // this warp's keys if own_warp; its new key and value, as bf16 pairs, for dims 2 lane (+ HD / 2) and 4 lane ...
+        const int pos = len - 1;
+        const int own_tile = OWN ? pos / kAttnKeys - tile0 : -1;
+        const bool own_warp = OWN && own_tile >= 0 && own_tile < n_tiles && (pos % kAttnKeys) / 16 == warp;
+        const bool k_lane = 2 * lane < HD / 2, v_lane = 4 * lane < HD;
+        uint32_t k_lo = 0u, k_hi = 0u, v_a = 0u, v_b = 0u;
+        if constexpr (!OWN) {
             const uint32_t* qrow = reinterpret_cast<const uint32_t*>(q + ((size_t)m * n_q + (size_t)kvh * group + min(g, group - 1)) * HD);
 #pragma unroll
             for (int ks = 0; ks < KS; ++ks) {
                 qb[ks][0] = g < group ? qrow[8 * ks + qd] : 0u;
                 qb[ks][1] = g < group ? qrow[8 * ks + 4 + qd] : 0u;
             }
+        } else {
+            // the rotation pairs dim i with dim i + HD / 2: k-step ks with k-step ks + KS / 2, same place in the fragment
+            const float* qrow = own.q + ((size_t)m * n_q + (size_t)kvh * group + min(g, group - 1)) * HD;
+            const float2* trow = own.table + (size_t)pos * (HD / 2);
+#pragma unroll
+            for (int ks = 0; ks < KS / 2; ++ks) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int i = 16 * ks + 8 * h + 2 * qd;
+                    const float2 lo = *reinterpret_cast<const float2*>(qrow + i), hi = *reinterpret_cast<const float2*>(qrow + i + HD / 2);
+                    const float4 cs = *reinterpret_cast<const float4*>(trow + i);  // cos, sin of pair i; cos, sin of pair i + 1
+                    const float lo0 = __fsub_rn(__fmul_rn(lo.x, cs.x), __fmul_rn(hi.x, cs.y));
+                    const float hi0 = __fadd_rn(__fmul_rn(hi.x, cs.x), __fmul_rn(lo.x, cs.y));
+                    const float lo1 = __fsub_rn(__fmul_rn(lo.y, cs.z), __fmul_rn(hi.y, cs.w));
+                    const float hi1 = __fadd_rn(__fmul_rn(hi.y, cs.z), __fmul_rn(lo.y, cs.w));
+                    qb[ks][h] = g < group ? pack_bf16(lo0, lo1) : 0u;
+                    qb[ks + KS / 2][h] = g < group ? pack_bf16(hi0, hi1) : 0u;
+                }
+            }
+            if (own_warp) {
+                const size_t src = ((size_t)m * n_kv + kvh) * HD, dst = (((size_t)seq * n_kv + kvh) * t_max + pos) * HD;
+                if (k_lane) {
+                    const int i = 2 * lane;
+                    const float2 lo = *reinterpret_cast<const float2*>(own.k + src + i);
+                    const float2 hi = *reinterpret_cast<const float2*>(own.k + src + i + HD / 2);
+                    const float4 cs = *reinterpret_cast<const float4*>(trow + i);
+                    k_lo = pack_bf16(__fsub_rn(__fmul_rn(lo.x, cs.x), __fmul_rn(hi.x, cs.y)),
+                                     __fsub_rn(__fmul_rn(lo.y, cs.z), __fmul_rn(hi.y, cs.w)));
+                    k_hi = pack_bf16(__fadd_rn(__fmul_rn(hi.x, cs.x), __fmul_rn(lo.x, cs.y)),
+                                     __fadd_rn(__fmul_rn(hi.y, cs.z), __fmul_rn(lo.y, cs.w)));
+                    *reinterpret_cast<uint32_t*>(own.k_cache + dst + i) = k_lo;
+                    *reinterpret_cast<uint32_t*>(own.k_cache + dst + i + HD / 2) = k_hi;
+                }
+                if (v_lane) {
+                    const float4 t = *reinterpret_cast<const float4*>(own.v + src + 4 * lane);
+                    v_a = pack_bf16(t.x, t.y);
+                    v_b = pack_bf16(t.z, t.w);
+                    *reinterpret_cast<uint2*>(own.v_cache + dst + 4 * lane) = make_uint2(v_a, v_b);
+                }
+            }
         }
-        const int kb = warp * 16;                 // this warp's keys of a tile
         const int mi = lane >> 3, mr = lane & 7;  // the matrix and row this lane addresses for ldmatrix
         for (int i = 0; i < n_tiles; ++i) {
             const uint32_t st = (uint32_t)(i % stages);
@@ -241,6 +329,20 @@ __global__ void __launch_bounds__(160) attn_decode_partial_kernel(const __grid_c
             const int n = min(kAttnKeys, len - (tile0 + i) * kAttnKeys);  // live rows of the tile, >= 1
             if (kb < n) {
                 const uint32_t kbase = ring_s + st * 2u * kTileBytes, vbase = kbase + kTileBytes;
+                if (OWN && own_warp && i == own_tile) {
+                    // the copy of the tile was read from the cache before (or while) the row was stored: put the new
+                    // row over it.  Element d of row r sits in block d / 64 at byte 128 r + 16 ((d % 64) / 8 ^ r % 8) + 2 (d % 8).
+                    const uint32_t r = (uint32_t)(pos % kAttnKeys);
+                    auto at = [&](uint32_t base, int d) {
+                        return base + (uint32_t)(d >> 6) * kHalfBytes + r * 128u + (((((uint32_t)d & 63u) >> 3) ^ (r & 7u)) << 4) + ((uint32_t)d & 7u) * 2u;
+                    };
+                    if (k_lane) {
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(at(kbase, 2 * lane)), "r"(k_lo) : "memory");
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(at(kbase, 2 * lane + HD / 2)), "r"(k_hi) : "memory");
+                    }
+                    if (v_lane) asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(at(vbase, 4 * lane)), "r"(v_a), "r"(v_b) : "memory");
+                    __syncwarp();
+                }
                 if (n < kb + 16) {  // the ragged end: zero this warp's dead value rows
                     for (int idx = lane; idx < (kb + 16 - n) * HALVES * 8; idx += 32) {
                         const int row = n + idx / (HALVES * 8), c = idx % (HALVES * 8);
@@ -374,7 +476,7 @@ __global__ void __launch_bounds__(160) attn_decode_partial_kernel(const __grid_c
 template <int HD>
 __global__ void __launch_bounds__(128) attn_decode_combine_kernel(const AttnPartial<HD>* __restrict__ part, const int* __restrict__ lengths,
                                                                   const int* __restrict__ seq_ids, int n_q, int n_seq, int t_max, int splits,
-                                                                  __nv_bfloat16* __restrict__ out) {
+                                                                  int own_row, __nv_bfloat16* __restrict__ out) {
     constexpr int CPL = HD / 32;
     __shared__ float red[4][HD];
     const size_t mh = blockIdx.x;  // token * n_q + head
@@ -400,8 +502,7 @@ __global__ void __launch_bounds__(128) attn_decode_combine_kernel(const AttnPart
     }
     const float2 ml0 = *reinterpret_cast<const float2*>(&p[min(lane, splits - 1)].m);
     const float2 ml1 = *reinterpret_cast<const float2*>(&p[min(lane + 32, splits - 1)].m);
-    const int seq = seq_ids ? seq_ids[m] : 0;
-    const int len = (seq >= 0 && seq < n_seq) ? min(max(lengths[m], 0), t_max) : 0;
+    const int len = attn_len(lengths, seq_ids ? seq_ids[m] : 0, m, n_seq, t_max, own_row != 0);
     const int live = attn_slices(len, splits).live;  // <= splits <= 64
     if (live == 0) {  // block-uniform
         for (int d = threadIdx.x; d < HD; d += blockDim.x) out[mh * HD + d] = __float2bfloat16_rn(0.0f);
@@ -574,7 +675,9 @@ bool attn_opt_in() {
     }
     std::lock_guard<std::mutex> lock(mu);
     if (!done[dev]) {
-        if (cudaFuncSetAttribute(attn_decode_partial_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        if (cudaFuncSetAttribute(attn_decode_partial_kernel<HD, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 (int)attn_smem_bytes<HD>(kAttnMaxStages)) != cudaSuccess ||
+            cudaFuncSetAttribute(attn_decode_partial_kernel<HD, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)attn_smem_bytes<HD>(kAttnMaxStages)) != cudaSuccess) {
             cudaGetLastError();
             return false;
@@ -586,6 +689,62 @@ bool attn_opt_in() {
 
 bool attn_dims_ok(int M, int n_q, int n_kv, int hd, int t_max) {
     return M >= 0 && M <= 65535 && n_q > 0 && n_kv > 0 && n_q % n_kv == 0 && n_q / n_kv <= 8 && (hd == 64 || hd == 128) && t_max > 0 && t_max <= (1 << 22);
+}
+
+// the two launches of decode attention (slices, merge); arguments already checked for shape and null
+int attn_launch(const __nv_bfloat16* q_bf16, const AttnOwnRow& own, bool own_row, const void* k_cache, const void* v_cache,
+                const int32_t* lengths, const int32_t* seq_ids, int M, int n_q_heads, int n_kv_heads, int head_dim, int n_seq, int t_max,
+                void* out_bf16, void* ws, size_t ws_bytes, void* stream) {
+    if (!aligned16(k_cache) || !aligned16(v_cache) || !aligned16(out_bf16)) return BITLINEAR_ERR_ALIGN;
+    if (!ws || !aligned16(ws) ||
+        ws_bytes < (size_t)M * n_q_heads * attn_splits_max(t_max) * (sizeof(float) * (4 + head_dim)))
+        return BITLINEAR_ERR_WORKSPACE;
+    int sm_count = 0;
+    if (const int rc = device_sm_count(&sm_count)) return rc;
+    CUtensorMap map_k, map_v;
+    if (!make_cache_map(&map_k, k_cache, n_seq, t_max, n_kv_heads, head_dim) ||
+        !make_cache_map(&map_v, v_cache, n_seq, t_max, n_kv_heads, head_dim))
+        return BITLINEAR_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const AttnPlan plan = attn_plan(M, n_kv_heads, t_max, sm_count);
+    const float scale = 1.0f / sqrtf((float)head_dim);
+    int* status = device_status_word();
+    // both kernels are programmatic dependents of the launch before them: they may be scheduled while it drains, and
+    // call griddepcontrol.wait before reading anything
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    auto launch = [&](auto hd_tag, auto own_tag) {
+        constexpr int HD = decltype(hd_tag)::value;
+        constexpr bool OWN = decltype(own_tag)::value;
+        if (!attn_opt_in<HD>()) return (int)BITLINEAR_ERR_CUDA;
+        auto* part = static_cast<AttnPartial<HD>*>(ws);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)plan.splits, (unsigned)n_kv_heads, (unsigned)M);
+        cfg.blockDim = dim3(160);
+        cfg.dynamicSmemBytes = attn_smem_bytes<HD>(plan.stages);
+        cfg.stream = st;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (cudaLaunchKernelEx(&cfg, attn_decode_partial_kernel<HD, OWN>, map_k, map_v, q_bf16, own, lengths, seq_ids, n_q_heads,
+                               n_kv_heads, n_seq, t_max, plan.splits, plan.stages, scale, part, status) != cudaSuccess) {
+            cudaGetLastError();
+            return (int)BITLINEAR_ERR_CUDA;
+        }
+        cfg.gridDim = dim3((unsigned)(M * n_q_heads));
+        cfg.blockDim = dim3(128);
+        cfg.dynamicSmemBytes = 0;
+        if (cudaLaunchKernelEx(&cfg, attn_decode_combine_kernel<HD>, (const AttnPartial<HD>*)part, lengths, seq_ids, n_q_heads, n_seq,
+                               t_max, plan.splits, (int)OWN, static_cast<__nv_bfloat16*>(out_bf16)) != cudaSuccess) {
+            cudaGetLastError();
+            return (int)BITLINEAR_ERR_CUDA;
+        }
+        return (int)BITLINEAR_OK;
+    };
+    using T = std::true_type;
+    using F = std::false_type;
+    if (head_dim == 128) return own_row ? launch(std::integral_constant<int, 128>{}, T{}) : launch(std::integral_constant<int, 128>{}, F{});
+    return own_row ? launch(std::integral_constant<int, 64>{}, T{}) : launch(std::integral_constant<int, 64>{}, F{});
 }
 
 }  // namespace
@@ -634,52 +793,35 @@ int bitlinear_attention_decode(const void* q_bf16, const void* k_cache_bf16, con
         return BITLINEAR_ERR_SHAPE;
     if (M == 0) return BITLINEAR_OK;
     if (!q_bf16 || !k_cache_bf16 || !v_cache_bf16 || !lengths || !out_bf16) return BITLINEAR_ERR_NULL;
-    if (!aligned16(q_bf16) || !aligned16(k_cache_bf16) || !aligned16(v_cache_bf16) || !aligned16(out_bf16)) return BITLINEAR_ERR_ALIGN;
-    if (!ws || !aligned16(ws) || ws_bytes < bitlinear_attention_workspace_bytes(M, n_q_heads, n_kv_heads, head_dim, t_max))
-        return BITLINEAR_ERR_WORKSPACE;
-    int sm_count = 0;
-    if (const int rc = device_sm_count(&sm_count)) return rc;
-    CUtensorMap map_k, map_v;
-    if (!make_cache_map(&map_k, k_cache_bf16, n_seq, t_max, n_kv_heads, head_dim) ||
-        !make_cache_map(&map_v, v_cache_bf16, n_seq, t_max, n_kv_heads, head_dim))
-        return BITLINEAR_ERR_CUDA;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const AttnPlan plan = attn_plan(M, n_kv_heads, t_max, sm_count);
-    const float scale = 1.0f / sqrtf((float)head_dim);
-    const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q_bf16);
-    int* status = device_status_word();
-    // both kernels are programmatic dependents of the launch before them: they may be scheduled while it drains, and
-    // call griddepcontrol.wait before reading anything
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    auto launch = [&](auto hd_tag) {
-        constexpr int HD = decltype(hd_tag)::value;
-        if (!attn_opt_in<HD>()) return (int)BITLINEAR_ERR_CUDA;
-        auto* part = static_cast<AttnPartial<HD>*>(ws);
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)plan.splits, (unsigned)n_kv_heads, (unsigned)M);
-        cfg.blockDim = dim3(160);
-        cfg.dynamicSmemBytes = attn_smem_bytes<HD>(plan.stages);
-        cfg.stream = st;
-        cfg.attrs = attr;
-        cfg.numAttrs = 1;
-        if (cudaLaunchKernelEx(&cfg, attn_decode_partial_kernel<HD>, map_k, map_v, qp, lengths, seq_ids, n_q_heads, n_kv_heads, n_seq,
-                               t_max, plan.splits, plan.stages, scale, part, status) != cudaSuccess) {
-            cudaGetLastError();
-            return (int)BITLINEAR_ERR_CUDA;
-        }
-        cfg.gridDim = dim3((unsigned)(M * n_q_heads));
-        cfg.blockDim = dim3(128);
-        cfg.dynamicSmemBytes = 0;
-        if (cudaLaunchKernelEx(&cfg, attn_decode_combine_kernel<HD>, (const AttnPartial<HD>*)part, lengths, seq_ids, n_q_heads, n_seq,
-                               t_max, plan.splits, static_cast<__nv_bfloat16*>(out_bf16)) != cudaSuccess) {
-            cudaGetLastError();
-            return (int)BITLINEAR_ERR_CUDA;
-        }
-        return (int)BITLINEAR_OK;
-    };
-    return head_dim == 128 ? launch(std::integral_constant<int, 128>{}) : launch(std::integral_constant<int, 64>{});
+    if (!aligned16(q_bf16)) return BITLINEAR_ERR_ALIGN;
+    return attn_launch(static_cast<const __nv_bfloat16*>(q_bf16), AttnOwnRow{}, false, k_cache_bf16, v_cache_bf16, lengths, seq_ids, M,
+                       n_q_heads, n_kv_heads, head_dim, n_seq, t_max, out_bf16, ws, ws_bytes, stream);
+}
+
+int bitlinear_rope_table(float rope_base, int head_dim, int t_max, float* table_out, void* stream) {
+    if ((head_dim != 64 && head_dim != 128) || t_max <= 0 || t_max > (1 << 22) || !(rope_base > 1.0f)) return BITLINEAR_ERR_SHAPE;
+    if (!table_out) return BITLINEAR_ERR_NULL;
+    if (!aligned16(table_out)) return BITLINEAR_ERR_ALIGN;
+    const long long work = (long long)t_max * (head_dim / 2);
+    rope_table_kernel<<<(unsigned)((work + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        reinterpret_cast<float2*>(table_out), t_max, head_dim, log2((double)rope_base));
+    if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    return BITLINEAR_OK;
+}
+
+int bitlinear_attention_decode_append(const float* q, const float* k, const float* v, const float* rope_table, void* k_cache_bf16,
+                                      void* v_cache_bf16, const int32_t* lengths, const int32_t* seq_ids, int M, int n_q_heads,
+                                      int n_kv_heads, int head_dim, int n_seq, int t_max, void* out_bf16, void* ws, size_t ws_bytes,
+                                      void* stream) {
+    if (!attn_dims_ok(M, n_q_heads, n_kv_heads, head_dim, t_max) || n_seq <= 0 || (long long)n_seq * n_kv_heads * t_max > (1ll << 30))
+        return BITLINEAR_ERR_SHAPE;
+    if (M == 0) return BITLINEAR_OK;
+    if (!q || !k || !v || !rope_table || !k_cache_bf16 || !v_cache_bf16 || !lengths || !out_bf16) return BITLINEAR_ERR_NULL;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(rope_table)) return BITLINEAR_ERR_ALIGN;
+    const AttnOwnRow own = {q, k, v, reinterpret_cast<const float2*>(rope_table), static_cast<__nv_bfloat16*>(k_cache_bf16),
+                            static_cast<__nv_bfloat16*>(v_cache_bf16)};
+    return attn_launch(nullptr, own, true, k_cache_bf16, v_cache_bf16, lengths, seq_ids, M, n_q_heads, n_kv_heads, head_dim, n_seq,
+                       t_max, out_bf16, ws, ws_bytes, stream);
 }
 
 int bitlinear_lm_head(const void* x_bf16, const void* table_bf16, int M, int V, int K, float* logits, void* stream) {

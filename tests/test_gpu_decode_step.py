@@ -103,6 +103,52 @@ def test_attention_decode(n_q, n_kv, hd, lengths):
         assert np.all(np.abs(got[m] - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-4 * vmax), m
 
 
+@pytest.mark.parametrize("n_q,n_kv,hd,lengths", [
+    (20, 5, 128, [4096]),                          # the newest row is the last row of a full cache
+    (20, 5, 128, [1, 7, 16, 17, 64, 65, 300, 1000, 0, 1001, 5]),  # every warp and tile boundary; two lengths that are no token
+    (4, 2, 64, [5, 64, 65, 513, 48]),
+    (8, 1, 128, [33]),
+])
+def test_attention_with_append_equals_the_two_call_route(n_q, n_kv, hd, lengths):
+    """Rotary embedding + cache append done inside the attention launches: the caches and the result must carry the bits
+    of bitlinear_rope_kv followed by bitlinear_attention_decode, and the result is checked against the oracle."""
+    M = len(lengths)
+    t_max = max(min(max(lengths), 4096), 16) if max(lengths) != 1001 else 1000
+    n_seq = M + 1
+    q, k, v = randn((M, n_q * hd), 30, 2.0), randn((M, n_kv * hd), 31), randn((M, n_kv * hd), 32)
+    kc0 = cache_to_dev(randn((n_seq, t_max, n_kv * hd), 33).to(torch.bfloat16), n_kv, hd)
+    vc0 = cache_to_dev(randn((n_seq, t_max, n_kv * hd), 34).to(torch.bfloat16), n_kv, hd)
+    seq = np.arange(M, dtype=np.int32)[::-1].copy()  # distinct sequences
+    if M > 4:
+        seq[4] = n_seq + 3  # a sequence that does not exist: nothing stored, a zero row
+    live = [m for m in range(M) if 1 <= lengths[m] <= t_max and seq[m] < n_seq]
+    len_d = torch.tensor(lengths, dtype=torch.int32, device=DEV)
+    seq_d = torch.from_numpy(seq).to(DEV)
+    table = bl.bitlinear_rope_table(hd, t_max + 5, device=DEV)  # a table longer than the cache is fine
+    # the two-call route
+    kc_a, vc_a = kc0.clone(), vc0.clone()
+    q_rot = bl.bitlinear_rope_kv(q.to(DEV), k.to(DEV), v.to(DEV), len_d - 1, kc_a, vc_a, n_q, n_kv, hd, seq_ids=seq_d)
+    out_a = bl.bitlinear_attention_decode(q_rot, kc_a, vc_a, len_d, n_q, n_kv, hd, seq_ids=seq_d)
+    # one call
+    kc_b, vc_b = kc0.clone(), vc0.clone()
+    out_b = bl.bitlinear_attention_decode_append(q.to(DEV), k.to(DEV), v.to(DEV), table, kc_b, vc_b, len_d, n_q, n_kv, hd, seq_ids=seq_d)
+    torch.cuda.synchronize()
+    assert bl.bitlinear_poll_status() == 0
+    assert torch.equal(kc_a, kc_b) and torch.equal(vc_a, vc_b)
+    changed = (kc_b != kc0).any(dim=-1).sum().item()
+    assert changed <= len(live) * n_kv and (not live or changed > 0)
+    for m in range(M):
+        if m in live:
+            assert torch.equal(out_a[m], out_b[m]), m
+        else:
+            assert not out_b[m].any(), m  # a length of t_max + 1 is clamped by the plain call, no token for this one
+    got, kb, vb, qb = bf(bits(out_b)), cache_bits(kc_b), cache_bits(vc_b), bits(q_rot)
+    for m in live:
+        ref = ds.attention_decode(qb[m], kb[seq[m]], vb[seq[m]], lengths[m], n_q, n_kv, hd)
+        vmax = np.abs(bf(vb[seq[m], :lengths[m]])).max()
+        assert np.all(np.abs(got[m] - ref) <= 2.0 ** -8 * np.abs(ref) + 1e-4 * vmax), m
+
+
 def test_attention_hand_cases():
     n_q, n_kv, hd, T = 4, 2, 64, 40
     kc = randn((1, T, n_kv * hd), 20).to(torch.bfloat16)
@@ -159,7 +205,8 @@ def test_argument_checks():
     assert lib.bitlinear_embed(fake, fake, 0, 10, 256, fake, None) == 0
 
 
-def test_whole_decode_step_stage_by_stage():
+@pytest.mark.parametrize("append_in_attention", [False, True])
+def test_whole_decode_step_stage_by_stage(append_in_attention):
     """One decoder layer + embedding + output head through DecodeStep; every stage is checked against the oracle applied
     to the values the GPU fed into that stage (a quantiser between two stages would turn a last-bit difference of an
     earlier floating-point stage into a different code, so the stages are not chained on the oracle side)."""
@@ -176,7 +223,9 @@ def test_whole_decode_step_stage_by_stage():
         layer[name] = (packed, s_w, gain.to(DEV))
         mats[name] = (oracle.quantize_weights(W.numpy(), wl.WEIGHT_EPS), wl.bf16_bits(gain))
     table = randn((V, H), 50).to(torch.bfloat16)
-    st = gpu_chain.DecodeStep([layer], table.to(DEV), M, t_max, H, F, n_q, n_kv, hd, wl.RMS_EPS, device=DEV)
+    st = gpu_chain.DecodeStep([layer], table.to(DEV), M, t_max, H, F, n_q, n_kv, hd, wl.RMS_EPS, device=DEV,
+                              append_in_attention=append_in_attention)
+    assert st.launches_per_layer == (10 if append_in_attention else 11)
     # a context in the caches: sequence m has positions[m] earlier tokens
     pos = np.array([0, 37, 79], np.int32)
     st.k_cache[0].copy_(cache_to_dev(randn((M, t_max, kv), 51).to(torch.bfloat16), n_kv, hd))
@@ -202,6 +251,9 @@ def test_whole_decode_step_stage_by_stage():
     qg, kg, vg = (t.cpu().numpy() for t in (st.q, st.k, st.v))
     q_ref, k_ref = ds.rope(qg, pos, n_q, hd), ds.rope(kg, pos, n_kv, hd)
     slack = 2.0 ** -20 * max(np.abs(qg).max(), np.abs(kg).max()) * 2
+    if append_in_attention:  # the rotated q stays in registers: take it from the rotary launch (same bits, tested above)
+        scratch = torch.zeros_like(st.k_cache[0]), torch.zeros_like(st.v_cache[0])
+        st.q_rot = bl.bitlinear_rope_kv(st.q, st.k, st.v, st.positions, *scratch, n_q, n_kv, hd, seq_ids=st.seq_ids)
     assert np.all(np.abs(bf(bits(st.q_rot)) - q_ref) <= 2.0 ** -8 * np.abs(q_ref) + slack)
     kc, vc = cache_bits(st.k_cache[0]), cache_bits(st.v_cache[0])
     for m in range(M):
