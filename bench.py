@@ -262,10 +262,10 @@ def run_ours(args):
                "h2d_bytes_per_step": int(x_host.numel()), "d2h_bytes_per_step": int(y_host.numel()),
                "api": "bitlinear_forward_batch_host: pinned x arena -> device, 2 launches, y arena -> pinned host, sync"}
 
-    # ---- the same step at M = 4 and M = 16 tokens per forward (rank 0 only): the tensor-core decode kernel ----
+    # ---- the same step at M = 4, 8 and 16 tokens per forward (rank 0 only): the tensor-core decode kernels ----
     decode_m = {}
     if rank == 0:
-        for m in (4, 16):
+        for m in (4, 8, 16):
             its = [(wl.activations_normal(m, p["K"], wl.seed_for(CONFIG_ID, i % 7, m)).to(dev), gains[p["K"]], p["packed"],
                     p["s_w"], torch.empty(m, p["N"], dtype=torch.float32, device=dev)) for i, p in enumerate(pool)]
             bm = bl.ProblemBatch(its, wl.RMS_EPS)
@@ -279,7 +279,8 @@ def run_ours(args):
                                          for _ in range(n_m)]) / n_m
             decode_m[f"M={m}"] = {"ms_per_step": round(ms_m, 4), "value": round(packed_bytes / ms_m / 1e6, 1), "unit": UNIT,
                                   "frac_of_hbm_peak": round(packed_bytes / ms_m / 1e6 / peaks["hbm_gbs"], 4),
-                                  "kernel": "decode_mma_kernel (weights unpacked into tensor memory, tcgen05 kind::i8)",
+                                  "kernel": "decode_stream_mma_kernel (the one-token weight stream feeding int8 mma.sync)" if m <= 8 else
+                                            "decode_mma_kernel (weights unpacked into tensor memory, tcgen05 kind::i8)",
                                   "kernel_alone_ms": round(ms_k, 4),
                                   "kernel_alone_frac_of_hbm_peak": round(packed_bytes / ms_k / 1e6 / peaks["hbm_gbs"], 4)}
             del its, bm, wm
@@ -593,10 +594,10 @@ def run_sweep(bl, dev, peaks, int8_peak):
         n_rep = 5 if M <= 256 else 2
         if M <= 64:
             # decode kernels: one problem per copy and per chunk of at most 16 tokens (M = 1: dot-products-of-four;
-            # 2..16 tokens per problem: tensor-core decode kernel); for M > 16 this is the decode path forced
+            # 2..8 tokens: the same stream feeding mma.sync; 9..16: tcgen05 decode kernel); for M > 16 this is the decode path forced
             chunks = [(c0, min(16, M - c0)) for c0 in range(0, M, 16)]
             items = [(x[c0:c0 + m], gain, packs[j], s_w, y[c0:c0 + m]) for j in range(copies) for c0, m in chunks]
-            steady["streaming_dp4a" if M == 1 else "tensor_core_decode_16_token_chunks"] = batch_us(items, n_rep) / copies
+            steady["streaming_dp4a" if M == 1 else "streaming_mma_sync" if M <= 8 else "tensor_core_decode_16_token_chunks"] = batch_us(items, n_rep) / copies
         if M > 16:
             items = [(x, gain, packs[j], s_w, y) for j in range(copies)]
             steady["grouped_tcgen05_gemm"] = batch_us(items, n_rep) / copies

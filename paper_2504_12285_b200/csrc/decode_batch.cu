@@ -1,5 +1,6 @@
-// Batched decode: many independent BitLinear forwards of ONE token each in two launches (sub-batches in which a
-// problem has 2 to 16 tokens run on the tensor cores instead, decode_mma.cu, which is faster from two tokens on).
+// Batched decode: many independent BitLinear forwards of ONE token each in two launches; with 2 to 8 tokens per
+// problem the same weight stream feeds int8 mma.sync (decode_stream_mma_kernel below), with 9 to 16 tokens the call goes
+// to the tcgen05 kernel of decode_mma.cu.
 // (Paper Section 5.1: the decode cost is the packed weight bytes that must cross HBM; a single
 // decode matmul is smaller than the memory system's bandwidth-delay product, so the weights of a
 // whole batch of matmuls are streamed back to back by one persistent kernel.)
@@ -111,6 +112,13 @@ __device__ __forceinline__ int dp4a_u8_s8(uint32_t a_u8x4, uint32_t b_s8x4, int 
     int d;
     asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a_u8x4), "r"(b_s8x4), "r"(c));
     return d;
+}
+
+// d += a * b, 16 weight rows x 8 tokens x 32 columns: a = unsigned weight codes, b = int8 activations, exact in int32
+__device__ __forceinline__ void mma_u8s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+        : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr) {
@@ -536,6 +544,255 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
     return cudaLaunchKernelEx(&cfg, decode_stream_kernel<kChunkTiles, FMT, FUSE>, prm);
 }
 
+// Ring of the multi-token kernel: two slots of five tiles per warp, as for one token (four slots of two tiles in the same
+// space were 20 % slower: the cost per chunk, not the bytes in flight, is what counts); eight rows of 8,192 columns fit
+// beside it.
+constexpr int kMmaChunk = 5, kMmaRing = 2;
+constexpr size_t mma_bar_bytes(int ring) { return (size_t)kStreamWarps * ring * 2 * 8 + 128; }
+constexpr size_t mma_ring_bytes(int chunk_tiles, int ring) { return (size_t)kStreamWarps * ring * chunk_tiles * kTileBytes + mma_bar_bytes(ring); }
+
+// Problems of 2 to 8 tokens (2-bit layout): the same weight stream, the products on the tensor cores.
+// The tile layout already is the operand layout of an int8 mma.sync of 16 rows x 8 tokens x 32 columns: lane (g, t) holds
+// word q of weight rows g and g + 8 - sixteen codes of columns 64q + 16t + 4j + b - and (word & mask_j) of rows g, g + 8
+// and of two words q, q' are the four registers of the weight operand (the order of the columns inside a dot product is
+// free); the activation operand of lane (g, t) is the matching four bytes of TOKEN g, which the interleaved activation
+// layout puts into one 16-byte load per word.  As in the one-token kernel the codes are not shifted down: mask j leaves
+// 4^j x the code (at most 128, an unsigned byte), one accumulator set per j keeps the scale uniform, and the four are
+// folded once per row block - exact in int32.  Per tile and warp: 32 logic operations, 8 tensor-core instructions,
+// 2 + 4 shared-memory loads; the integer pipe is the busiest unit (about half of its cycles).
+// The arena holds the quantised rows of ONE problem at a time: the CTA goes through its problems in order, all warps meet
+// before the arena is refilled, and the weight ring keeps prefetching across the meeting.  Problems that share their
+// quantised input (q, k, v of a layer) share the copy.  A token's row in the arena is K + 64 bytes long, so that the
+// 64-byte pieces of eight tokens fall into different banks.
+// NT = 8-token groups per problem; only NT = 1 is instantiated (with two groups the kernel spills at its 128-register
+// cap and is slower than the tcgen05 kernel, which therefore keeps 9 to 16 tokens).
+template <int kChunkTiles, int RING, int NT>
+__global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_mma_kernel(const StreamParams prm) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    // [ring: 16 warps x RING slots][full barriers][empty barriers][abort flag][activation arena]
+    constexpr uint32_t kSlotBytes = kChunkTiles * kTileBytes;
+    constexpr int par = kStreamWarps;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + (size_t)par * RING * kSlotBytes);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 2 * kStreamWarps * RING);
+    constexpr size_t kBars = (size_t)kStreamWarps * RING * 2 * 8 + 128;  // as mma_bar_bytes(RING) on the host
+    uint8_t* arena = reinterpret_cast<uint8_t*>(bars) + kBars;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (!plan_matches(prm.hdr, prm.count, prm.total_rb, (int)gridDim.x, prm.rows)) {  // uniform over the grid
+        if (blockIdx.x == 0 && threadIdx.x == 0 && prm.status_word != nullptr)
+            atomicExch(prm.status_word, BITLINEAR_ERR_WORKSPACE);
+        return;
+    }
+    if (lane == 0) {
+        for (int r = 0; r < RING; ++r) {
+            mbar_init(smem_u32(bars + warp * RING + r), 1);                          // full: the copy landed
+            mbar_init(smem_u32(bars + kStreamWarps * RING + warp * RING + r), 1);   // empty: the warp has read it
+        }
+        if (warp == 0) *abort_flag = 0;
+        mbar_init_fence();
+    }
+    __syncthreads();
+    const int4 range = prm.cta_range[blockIdx.x];
+    const int rb_lo = range.x, rb_hi = range.y, p_lo = range.z, p_hi = range.w;
+    const DevProblem* probs = prm.probs;
+    const int rl = warp;
+    const bool mine = rb_lo + rl < rb_hi;
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t ring_s = smem_u32(smem) + (uint32_t)rl * RING * kSlotBytes;
+    const uint32_t bar_s = smem_u32(bars + rl * RING);
+    const uint32_t ebar_s = smem_u32(bars + kStreamWarps * RING + rl * RING);
+    const bool issuer = lane == 0;
+
+    // ---- the weight stream starts before anything else (the plan and the weights are not written by the launch in front)
+    ChunkCursor ld;  // where the next copy comes from
+    ld.rb = rb_lo + rl; ld.c = 0; ld.p = p_lo;
+    ld.rb_begin = 0; ld.rb_end = 0; ld.k_tiles = 1; ld.nc = 1; ld.ct = 1; ld.base = nullptr;
+    bool ld_valid = mine;
+    auto enter_ld = [&]() {
+        while (ld.rb >= probs[ld.p].rb_end) ++ld.p;
+        ld.set_problem(probs[ld.p].rb_begin, probs[ld.p].rb_end, probs[ld.p].k_tiles, probs[ld.p].packed, kChunkTiles);
+    };
+    if (mine) enter_ld();
+    auto issue = [&](int slot) {  // lane 0 only
+        const uint32_t bytes = (uint32_t)ld.tiles() * kTileBytes;
+        mbar_expect_tx(bar_s + 8u * slot, bytes);
+        bulk_load(ring_s + (uint32_t)slot * kSlotBytes, ld.src(), bytes, bar_s + 8u * slot);
+    };
+    auto advance_ld = [&]() {
+        if (++ld.c == ld.nc) {
+            ld.c = 0;
+            ld.rb += par;
+            if (ld.rb >= rb_hi) ld_valid = false;
+            else if (ld.rb >= ld.rb_end) enter_ld();
+        }
+    };
+#pragma unroll
+    for (int r = 0; r < RING; ++r)
+        if (ld_valid) {
+            if (issuer) issue(r);
+            advance_ld();
+        }
+
+    // the quantiser launch that precedes this kernel must be complete before its results are read
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+
+    ChunkCursor cp;  // where the arithmetic is
+    cp.rb = rb_lo + rl; cp.c = 0; cp.p = p_lo;
+    cp.rb_begin = 0; cp.rb_end = 0; cp.k_tiles = 1; cp.nc = 1; cp.ct = 1; cp.base = nullptr;
+    bool done = !mine, ok = true;
+    uint32_t n_chunk = 0;  // chunks consumed: slot = n_chunk % RING, phase = (n_chunk / RING) & 1
+    int macc[NT][4][4];    // [8-token group][scale 4^j][(row g, token 2t), (g, 2t + 1), (g + 8, 2t), (g + 8, 2t + 1)]
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int e = 0; e < 16; ++e) macc[nt][e >> 2][e & 3] = 0;
+    const int8_t* staged_xq = nullptr;  // what the arena holds (uniform over the CTA)
+    int staged_m = 0;
+    const uint32_t arena_s = smem_u32(arena);
+
+    if (rb_lo < rb_hi)
+    for (int pi = p_lo; pi <= p_hi; ++pi) {  // uniform over the CTA
+        const DevProblem& pr = probs[pi];
+        const int M = pr.M, xst = pr.x_stride, pst = xst + 64;
+        const bool fits = M * pst + 128 <= prm.arena_bytes;  // else the rows are read from global memory (slow, rare)
+        if (fits && !(pr.xq == staged_xq && M == staged_m)) {
+            __syncthreads();  // every warp is done with what the arena held
+            const int bytes = M * xst;
+            for (int o = threadIdx.x * 16; o < bytes; o += kStreamThreads * 16) cp_async16(arena_s + o + 64 * (o / xst), pr.xq + o);
+            if ((int)threadIdx.x < M) {
+                float* dx = reinterpret_cast<float*>(arena + M * pst);
+                dx[threadIdx.x] = pr.d[threadIdx.x];
+                reinterpret_cast<int*>(dx)[16 + threadIdx.x] = pr.xsum[threadIdx.x];
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();
+            staged_xq = pr.xq;
+            staged_m = M;
+        }
+        if (done || cp.rb >= pr.rb_end) continue;  // this warp has no row block in the problem
+        cp.p = pi;
+        cp.c = 0;
+        cp.set_problem(pr.rb_begin, pr.rb_end, pr.k_tiles, pr.packed, kChunkTiles);
+        const int y_dtype = pr.y_dtype, n_out = pr.N;
+        void* const y = pr.y;
+        int32_t* const acc_out = pr.acc_out;
+        const float s_w = *pr.s_w;
+        // token 8 nt + g is this lane's column of the activation operand (the last token again where there is none);
+        // the results this lane ends up with are those of tokens 8 nt + 2 t + e
+        uint32_t xtok_s[NT];
+        const int8_t* xtok_g[NT];
+        float d_tok[NT][2];
+        int xs_tok[NT][2];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+            const int tok = min(8 * nt + g, M - 1);
+            xtok_s[nt] = arena_s + (uint32_t)(tok * pst + t * 16);
+            xtok_g[nt] = pr.xq + (size_t)tok * xst + t * 16;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int tk = min(8 * nt + 2 * t + e, M - 1);
+                d_tok[nt][e] = fits ? reinterpret_cast<const float*>(arena + M * pst)[tk] : pr.d[tk];
+                xs_tok[nt][e] = fits ? reinterpret_cast<const int*>(arena + M * pst)[16 + tk] : pr.xsum[tk];
+            }
+        }
+        for (;;) {
+            const uint32_t slot = n_chunk % RING, phase = (n_chunk / RING) & 1u;
+            if (!mbar_wait(bar_s + 8u * slot, phase, abort_flag)) { ok = false; done = true; break; }
+            const int tiles = cp.tiles();
+            auto run_tiles = [&](auto staged) {
+                constexpr bool XS = decltype(staged)::value;  // the problem's activations are in the arena
+                uint32_t wa = ring_s + slot * kSlotBytes + (uint32_t)lane * 16u;
+                uint32_t xo = (uint32_t)(cp.c * cp.ct) * kTileCols;
+                for (int tile = 0; tile < tiles; ++tile, wa += kTileBytes, xo += kTileCols) {
+                    const uint4 w0v = lds128(wa), w1v = lds128(wa + 512);
+                    const uint32_t w0[4] = {w0v.x, w0v.y, w0v.z, w0v.w};  // row g
+                    const uint32_t w1[4] = {w1v.x, w1v.y, w1v.z, w1v.w};  // row g + 8
+#pragma unroll
+                    for (int qp = 0; qp < 2; ++qp) {  // words 2 qp and 2 qp + 1 are the two column halves of an operand
+                        uint32_t xa[NT][4], xb[NT][4];
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            uint4 va, vb;
+                            if (XS) {
+                                va = lds128(xtok_s[nt] + xo + 128u * qp);
+                                vb = lds128(xtok_s[nt] + xo + 128u * qp + 64u);
+                            } else {
+                                va = *reinterpret_cast<const uint4*>(xtok_g[nt] + xo + 128 * qp);
+                                vb = *reinterpret_cast<const uint4*>(xtok_g[nt] + xo + 128 * qp + 64);
+                            }
+                            xa[nt][0] = va.x; xa[nt][1] = va.y; xa[nt][2] = va.z; xa[nt][3] = va.w;
+                            xb[nt][0] = vb.x; xb[nt][1] = vb.y; xb[nt][2] = vb.z; xb[nt][3] = vb.w;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t mask = 0x03030303u << (2 * j);  // codes times 4^j: at most 128, an unsigned byte
+                            const uint32_t a0 = w0[2 * qp] & mask, a1 = w1[2 * qp] & mask;
+                            const uint32_t a2 = w0[2 * qp + 1] & mask, a3 = w1[2 * qp + 1] & mask;
+#pragma unroll
+                            for (int nt = 0; nt < NT; ++nt) mma_u8s8(macc[nt][j], a0, a1, a2, a3, xa[nt][j], xb[nt][j]);
+                        }
+                    }
+                }
+            };
+            if (fits) run_tiles(std::true_type{});
+            else run_tiles(std::false_type{});
+            __syncwarp();  // every lane of this warp has read the slot
+            if (lane == 0) mbar_arrive(ebar_s + 8u * slot);
+            if (ld_valid) {
+                // refill the slot that has just been read
+                if (issuer && mbar_wait(ebar_s + 8u * slot, phase, abort_flag)) issue((int)slot);
+                advance_ld();
+            }
+            ++n_chunk;
+            if (++cp.c == cp.nc) {
+                // ---- end of a row block: fold the two scales, subtract the code offset, dequantise, store ----
+                const int n0 = (cp.rb - cp.rb_begin) * kTileRows + g;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int tok = 8 * nt + 2 * t + (e & 1);
+                        // 64 x the sum, exactly: accumulator j holds 4^j x its share
+                        const int a = ((((macc[nt][0][e] * 4 + macc[nt][1][e]) * 4 + macc[nt][2][e]) * 4 + macc[nt][3][e]) >> 6) - xs_tok[nt][e & 1];
+                        macc[nt][0][e] = macc[nt][1][e] = macc[nt][2][e] = macc[nt][3][e] = 0;
+                        if (tok < M) {
+                            const float val = __fmul_rn(__fmul_rn((float)a, s_w), d_tok[nt][e & 1]);
+                            const size_t idx = (size_t)tok * n_out + (size_t)(n0 + 8 * (e >> 1));
+                            if (acc_out != nullptr) acc_out[idx] = a;
+                            if (y_dtype == BITLINEAR_BF16) reinterpret_cast<__nv_bfloat16*>(y)[idx] = __float2bfloat16_rn(val);
+                            else reinterpret_cast<float*>(y)[idx] = val;
+                        }
+                    }
+                cp.c = 0;
+                cp.rb += par;
+                if (cp.rb >= rb_hi) { done = true; break; }
+                if (cp.rb >= pr.rb_end) break;  // on to the next problem, with everybody else
+            }
+        }
+    }
+    if (!ok) abort_drain();  // copies of this warp may still be in flight
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0 && prm.status_word != nullptr) atomicExch(prm.status_word, BITLINEAR_ERR_TIMEOUT);
+}
+
+template <int kChunkTiles, int RING, int NT>
+cudaError_t launch_stream_mma(const StreamParams& prm, int grid, size_t smem, cudaStream_t st) {
+    cudaError_t e = cudaFuncSetAttribute(decode_stream_mma_kernel<kChunkTiles, RING, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kStreamThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // behind this call's quantiser launch
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, decode_stream_mma_kernel<kChunkTiles, RING, NT>, prm);
+}
+
 struct PlanLayout {
     size_t probs_off, cta_range_off, row_prob_off, xq_off, total;
 };
@@ -568,11 +825,13 @@ namespace bitlinear {
 size_t prefill_group_workspace_bytes(const bitlinear_problem* problems, const int* idx, int n);
 int prefill_group_forward(const bitlinear_problem* problems, const int* idx, int n, void* ws, bool skip_quant,
                           bool skip_unpack, cudaStream_t st);
-// Sub-batches with a problem of more than kDp4aMaxTokens tokens run on the tensor cores (decode_mma.cu): measured on
-// the 210-matmul decode step, 145 us per step there at 2 to 5 tokens against 171 to 174 us for the kernel below.
+// Sub-batches with a problem of more than kStreamMmaMaxTokens tokens run on the tcgen05 decode kernel (decode_mma.cu).
+// Measured on the 210-matmul decode step: 100 to 121 us per step at 2 to 8 tokens through decode_stream_mma_kernel
+// (141 to 153 us through the tcgen05 kernel); at 9 to 16 tokens the stream kernel needs a second accumulator set and twice the
+// activation reads per tile, spills at its 128-register cap and takes 175 to 190 us against 156 to 166 us.
 size_t decode_mma_workspace_bytes(const bitlinear_problem* problems, int count);
 int decode_mma_forward(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes, void* stream);
-constexpr int kDp4aMaxTokens = 1;
+constexpr int kStreamMmaMaxTokens = 8;
 
 namespace {
 
@@ -604,7 +863,7 @@ size_t decode_batch_workspace_bytes(const bitlinear_problem* problems, int count
         rows += (size_t)q.M;
         if (q.M > max_m) max_m = q.M;
     }
-    if (fmt == BITLINEAR_WEIGHTS_2BIT && max_m > kDp4aMaxTokens) return decode_mma_workspace_bytes(problems, count);
+    if (fmt == BITLINEAR_WEIGHTS_2BIT && max_m > kStreamMmaMaxTokens) return decode_mma_workspace_bytes(problems, count);
     // the dense-layout kernel takes one token per problem: a problem of M tokens is planned as M problems
     return plan_layout(fmt == BITLINEAR_WEIGHTS_DENSE5 ? (int)rows : count, kPlanGrid, xq, rows).total;
 }
@@ -636,10 +895,11 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         if (q.M > max_m) max_m = q.M;
         if (q.K > max_k) max_k = q.K;
     }
-    if (!dense && max_m > kDp4aMaxTokens) {
-        if (want_acc) return BITLINEAR_ERR_SHAPE;  // the tensor-core decode kernel has no accumulator output
+    if (!dense && max_m > kStreamMmaMaxTokens) {
+        if (want_acc) return BITLINEAR_ERR_SHAPE;  // the tcgen05 decode kernel has no accumulator output
         return decode_mma_forward(problems, count, flags, ws, ws_bytes, stream);
     }
+    const int nt = dense || max_m <= 1 ? 0 : 1;  // 2 to 8 tokens: the multi-token stream kernel
     const PlanLayout L = plan_layout(dense ? (int)rows : count, kPlanGrid, xq_bytes, rows);
     if (!ws || !aligned16(ws) || ws_bytes < L.total) return BITLINEAR_ERR_WORKSPACE;
     if (rows == 0) return BITLINEAR_OK;
@@ -788,19 +1048,27 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
             if (lo < hi) {
                 if (pl - pf + 1 > table_cap) table_cap = pl - pf + 1;
                 size_t a = 0;
-                for (int i = pf; i <= pl; ++i) a += (size_t)dp[i].M * dp[i].x_stride;
+                for (int i = pf; i <= pl; ++i) {
+                    const size_t one = (size_t)dp[i].M * (dp[i].x_stride + 64) + 128;  // multi-token: one problem at a time, padded rows
+                    if (nt) a = std::max(a, one);
+                    else a += (size_t)dp[i].M * dp[i].x_stride;
+                }
                 if (a > arena_max) arena_max = a;
             }
         }
     }
     // shared memory: chunk ring + descriptor table + activation arena; activations that do not fit the arena are read
     // through L1 instead, and only as many descriptors as fit a quarter of the space are cached
+    // (the multi-token kernel caches no descriptors and keeps the rows of one problem at a time in its arena)
     constexpr int chunk_tiles = 5;
-    const size_t smem_limit = 227 * 1024 - ring_bytes(chunk_tiles) - 128;
+    const size_t ring_total = nt == 0 ? ring_bytes(chunk_tiles) : mma_ring_bytes(kMmaChunk, kMmaRing);
+    const size_t smem_limit = 227 * 1024 - ring_total - 128;
+    if (nt) table_cap = 0;
     const int table_need = table_cap;  // with fewer cached descriptors some problems of a CTA are read from global memory
     if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
     if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
-    arena_max &= ~(size_t)255;
+    if (nt) arena_max = std::min(align_up(arena_max, 256), smem_limit & ~(size_t)255);
+    else arena_max &= ~(size_t)255;
 
     PlanHeader hdr_host;
     hdr_host.magic = kPlanMagic;
@@ -874,8 +1142,12 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     prm.status_word = device_status_word();
     prm.table_cap = table_cap;
     prm.arena_bytes = (int)arena_max;
-    const size_t smem = ring_bytes(chunk_tiles) + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
-    prm.fuse_prob = 0;  // the first entry owns the quantised copy of the one row
+    const size_t smem = ring_total + (size_t)table_cap * sizeof(SProb) + arena_max + 128;
+    prm.fuse_prob = 0;
+    if (nt) {
+        const cudaError_t em = launch_stream_mma<kMmaChunk, kMmaRing, 1>(prm, grid, smem, st);
+        return em == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+    }  // the first entry owns the quantised copy of the one row
     // behind the quantiser launch of this call the stream kernel is always a dependent (that launch writes no weights);
     // a fused launch only under the promise above
     const bool dep = !fuse || static_weights;

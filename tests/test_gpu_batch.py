@@ -84,6 +84,47 @@ def test_batch_several_tokens(ms):
     check(batch, refs)
 
 
+@pytest.mark.parametrize("M", [2, 5, 8])
+def test_batch_several_tokens_accumulators_and_shared_inputs(M):
+    """2 to 8 tokens stream the weights once and multiply with int8 mma.sync: the int32 accumulators must be the oracle's
+    bit for bit.  Three problems share their input (one copy in shared memory), the next has the longest row the call
+    takes (eight tokens of it fill the activation arena), the last has a single token and a single row block."""
+    seed = 4300 + M
+    K = 2560
+    x = wl.activations_student_t(M, K, seed)
+    x_long = wl.activations_normal(M, 8192, seed + 1)
+    x_one = wl.activations_normal(1, 512, seed + 2)
+    gain = wl.gain_random(K, seed + 3)
+    specs = [(x, gain, 640, K), (x, gain, 48, K), (x, gain, 2560, K), (x_long, None, 64, 8192), (x_one, None, 16, 512)]
+    items, refs, accs = [], [], []
+    for i, (xi, gi, N, Ki) in enumerate(specs):
+        W = wl.latent_weights(N, Ki, seed + 10 + i)
+        packed, s_w = bl.bitlinear_pack_weights(W.to(DEV), wl.WEIGHT_EPS)
+        wref = oracle.quantize_weights(W.numpy(), wl.WEIGHT_EPS)
+        refs.append(oracle.bitlinear_forward(wl.bf16_bits(xi), None if gi is None else wl.bf16_bits(gi), wl.RMS_EPS, wref["wq"], wref["s_w"]))
+        y = torch.full((xi.shape[0], N), float("nan"), dtype=torch.bfloat16 if i == 1 else torch.float32, device=DEV)
+        items.append((xi.to(DEV), None if gi is None else gi.to(DEV), packed, s_w, y))
+        accs.append(torch.full((xi.shape[0], N), -7, dtype=torch.int32, device=DEV))
+    items = [(items[0][0], items[0][1]) + it[2:] if i < 3 else it for i, it in enumerate(items)]  # one tensor for the shared input
+    batch = bl.ProblemBatch(items, wl.RMS_EPS)
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    bl.bitlinear_forward_batch_acc(batch, accs, ws)
+    torch.cuda.synchronize()
+    assert bl.bitlinear_poll_status() == 0
+    for acc, ref in zip(accs, refs):
+        assert not ref["fragile"].any()
+        assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+    check(batch, refs)
+    # the same bits when the quantised rows are reused
+    first = [t[4].clone() for t in batch.tensors]
+    for t in batch.tensors:
+        t[4].fill_(float("nan"))
+    bl.bitlinear_forward_batch(batch, ws, reuse_plan=True, reuse_act=True)
+    torch.cuda.synchronize()
+    for a, t in zip(first, batch.tensors):
+        assert torch.equal(a, t[4])
+
+
 def test_batch_bf16_output_and_empty_problem():
     shapes = [(4, 64, 512), (0, 32, 256), (1, 640, 2560)]
     batch, refs = make_case(shapes, 400, y_dtype=torch.bfloat16)
