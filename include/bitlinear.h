@@ -243,8 +243,9 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  * Problems of at most 16 tokens (the decode regime of Section 5.1, where the cost is the packed
  * weight bytes streamed from HBM) take two launches together: one fused RMSNorm+quantiser launch
  * over every token, then one persistent kernel that streams the packed weights of all of them
- * back to back (dot-products-of-four when every such problem has one token; otherwise the tensor
- * cores, with the codes unpacked in registers and handed over in tensor memory).  A call whose
+ * back to back (dot-products-of-four when every such problem has one token; int8 mma.sync fed
+ * from the same stream when none has more than 8; otherwise tcgen05, with the codes unpacked in
+ * registers and handed over in tensor memory).  A call whose
  * problems all have one token and read the same input row the same way - a level of a decoder
  * layer: q/k/v, o, gate/up or down - is ONE launch: every CTA quantises the row itself while its
  * share of the packed weights is on its way (up to four problems in the 2-bit layout; otherwise the
@@ -328,8 +329,9 @@ int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int fl
  * Parity hook: bitlinear_forward_batch that also stores the raw int32 accumulators sum_k xq*Wq of the contraction
  * (Section 5.1: the integer product of unpacked ternary weights and 8-bit activations).
  *   acc_out : HOST array of `count` DEVICE pointers, entry i nullable or [M][N] int32 for problem i.
- * Available where the persistent streaming kernels run the problem: one-token problems in the 2-bit layout and
- * problems of up to 16 tokens in the dense layout; BITLINEAR_ERR_SHAPE for a non-NULL entry anywhere else.
+ * Available where the persistent streaming kernels run the problem: calls in the 2-bit layout whose decode-sized
+ * problems all have at most 8 tokens, and problems of up to 16 tokens in the dense layout; BITLINEAR_ERR_SHAPE for a
+ * non-NULL entry anywhere else.
  */
 int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, int flags, int32_t* const* acc_out,
                                 void* ws, size_t ws_bytes, void* stream);

@@ -71,6 +71,8 @@ __device__ __forceinline__ bool plan_matches(const PlanHeader* h, int count, int
     return h->magic == kPlanMagic && h->count == count && h->total_rb == total_rb && h->grid == grid && h->rows == rows;
 }
 
+constexpr int kDotJ = 2;  // of the four code positions j of a byte, how many the one-token kernel multiplies by dot-product-of-four
+                          // (the rest goes to the tensor cores; 1 and 2 measured the same, 4 - no tensor cores - 3.5 % slower)
 constexpr int kStreamWarps = 16;
 constexpr int kStreamThreads = kStreamWarps * 32;
 constexpr int kRing = 2;  // chunk slots per warp
@@ -409,6 +411,11 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         for (int h = 0; h < 2; ++h)
 #pragma unroll
             for (int j = 0; j < 4; ++j) acc[h][j] = 0;
+        // 2-bit layout: tensor-core accumulators of the codes j = 2, 3: [.][0] row g, [.][2] row g + 8, summed over the four
+        // column lanes already and the same in each of them (every token column of the operand is this token)
+        int macc[4 - kDotJ][4];
+#pragma unroll
+        for (int j = 0; j < 4 - kDotJ; ++j) macc[j][0] = macc[j][1] = macc[j][2] = macc[j][3] = 0;
 
         uint32_t n_chunk = 0;  // chunks consumed: slot = n_chunk % kRing, phase = (n_chunk / kRing) & 1
         bool ok = true;
@@ -453,17 +460,34 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                     } else {
                         // the token's codes are stored with the four 16-byte pieces of each lane's 64 columns interleaved
                         // (piece q of lane t at 64q + 16t inside the tile), so the four t lanes read 64 contiguous bytes
+                        // The products are shared between two units: codes j = 0, 1 of every word go through the
+                        // dot-product-of-four (a quarter-rate instruction of the integer pipe, which also does the masking),
+                        // codes j = 2, 3 through an int8 mma.sync whose 8 token columns all carry this one token - a
+                        // sixteenth of its products are used, and it still costs the integer pipe nothing.
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            uint4 v;
-                            if (XS) v = lds128(xrow_s + xo + 64u * q);
-                            else v = *reinterpret_cast<const uint4*>(xrow_g + xo + 64 * q);
-                            const uint32_t xw[4] = {v.x, v.y, v.z, v.w};
+                        for (int qp = 0; qp < 2; ++qp) {
+                            uint4 va, vb;
+                            if (XS) {
+                                va = lds128(xrow_s + xo + 128u * qp);
+                                vb = lds128(xrow_s + xo + 128u * qp + 64u);
+                            } else {
+                                va = *reinterpret_cast<const uint4*>(xrow_g + xo + 128 * qp);
+                                vb = *reinterpret_cast<const uint4*>(xrow_g + xo + 128 * qp + 64);
+                            }
+                            const uint32_t xa[4] = {va.x, va.y, va.z, va.w}, xb[4] = {vb.x, vb.y, vb.z, vb.w};
 #pragma unroll
-                            for (int j = 0; j < 4; ++j) {
+                            for (int j = 0; j < kDotJ; ++j) {
                                 const uint32_t mask = 0x03030303u << (2 * j);
-                                acc[0][j] = dp4a_u8_s8(w0[q] & mask, xw[j], acc[0][j]);
-                                acc[1][j] = dp4a_u8_s8(w1[q] & mask, xw[j], acc[1][j]);
+                                acc[0][j] = dp4a_u8_s8(w0[2 * qp] & mask, xa[j], acc[0][j]);
+                                acc[1][j] = dp4a_u8_s8(w1[2 * qp] & mask, xa[j], acc[1][j]);
+                                acc[0][j] = dp4a_u8_s8(w0[2 * qp + 1] & mask, xb[j], acc[0][j]);
+                                acc[1][j] = dp4a_u8_s8(w1[2 * qp + 1] & mask, xb[j], acc[1][j]);
+                            }
+#pragma unroll
+                            for (int j = kDotJ; j < 4; ++j) {
+                                const uint32_t mask = 0x03030303u << (2 * j);
+                                mma_u8s8(macc[j - kDotJ], w0[2 * qp] & mask, w1[2 * qp] & mask, w0[2 * qp + 1] & mask, w1[2 * qp + 1] & mask,
+                                         xa[j], xb[j]);
                             }
                         }
                     }
@@ -487,13 +511,20 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
                 for (int h = 0; h < 2; ++h) {
                     // 64 x the sum: ((a0*4 + a1)*4 + a2)*4 + a3; |sum| <= 254*K/4 per lane: no overflow for K <= 8192
                     int sum = acc[h][0];
-                    if constexpr (FMT == 0) {
-                        sum = sum * 4 + acc[h][1];
-                        sum = sum * 4 + acc[h][2];
-                        sum = sum * 4 + acc[h][3];
+                    if constexpr (FMT == 0) {  // the dot-product-of-four part, this lane's share: accumulator j holds 4^j x its sum
+                        sum = 0;
+#pragma unroll
+                        for (int j = 0; j < kDotJ; ++j) sum += acc[h][j] * (1 << (2 * (3 - j)));
                     }
                     sum += __shfl_xor_sync(0xffffffffu, sum, 1);
                     sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                    if constexpr (FMT == 0) {  // the tensor-core part, already summed over the lanes
+#pragma unroll
+                        for (int j = kDotJ; j < 4; ++j) {
+                            sum += macc[j - kDotJ][2 * h] * (1 << (2 * (3 - j)));
+                            macc[j - kDotJ][2 * h] = macc[j - kDotJ][2 * h + 1] = 0;
+                        }
+                    }
                     v[h] = FMT == 0 ? sum >> 6 : sum;  // 2-bit layout: exact, a multiple of 64
 #pragma unroll
                     for (int j = 0; j < 4; ++j) acc[h][j] = 0;
@@ -545,7 +576,7 @@ cudaError_t launch_stream(const StreamParams& prm, int grid, size_t smem, cudaSt
 }
 
 // Ring of the multi-token kernel: two slots of five tiles per warp, as for one token (four slots of two tiles in the same
-// space were 20 % slower: the cost per chunk, not the bytes in flight, is what counts); eight rows of 8,192 columns fit
+// space were 20 % slower and three slots of four tiles 7 % slower: the cost per chunk, not the bytes in flight, is what counts); eight rows of 8,192 columns fit
 // beside it.
 constexpr int kMmaChunk = 5, kMmaRing = 2;
 constexpr size_t mma_bar_bytes(int ring) { return (size_t)kStreamWarps * ring * 2 * 8 + 128; }
