@@ -270,7 +270,10 @@ int bitlinear_forward_host(const void* x_host, const void* gain, float rms_eps, 
  *   flags    : 0, or an OR of BITLINEAR_BATCH_REUSE_PLAN (the previous call on this workspace had
  *              exactly the same descriptors, and the packed weights, their scales and the gains
  *              have not been written since - the steady state of a decode loop: skips
- *              re-uploading the decode plan, and a call that is a single launch (one token, one
+ *              re-uploading the decode plan and, when the library still remembers what it derived
+ *              from these descriptors for this workspace (a small per-process table keyed by the
+ *              workspace address and a hash of the descriptors), planning on the host altogether;
+ *              and a call that is a single launch (one token, one
  *              shared input row) may begin fetching weights while the launch before it on the
  *              stream is still running) and
  *              BITLINEAR_BATCH_REUSE_ACT (the inputs are unchanged as well: skips the quantiser
@@ -341,6 +344,13 @@ int bitlinear_forward_batch_acc(const bitlinear_problem* problems, int count, in
  * descriptors point into one device arena x_dev and the y pointers into one device arena y_dev;
  * the call copies x_host (host, ideally pinned, x_bytes) into x_dev, runs the batch, copies y_dev
  * (y_bytes) into y_host and SYNCHRONISES the stream before returning.
+ * A call of at least 24 decode-sized problems (M <= 16, plain inputs) whose operands lie in both arenas in the order
+ * of the problems runs as three segments of about equal packed bytes, two of them on streams of the library's own
+ * (created on first use, one set per device) that start after the caller's earlier work and that the caller's stream
+ * waits for: one segment's copies then run beside another's kernels.  Every byte of both arenas is still copied
+ * exactly once and the results are those of the unsegmented call.  Each segment keeps its own plan in its slice of ws
+ * (bitlinear_batch_workspace_bytes covers that), so BITLINEAR_BATCH_REUSE_PLAN here refers to an earlier call of
+ * THIS function on the same ws, not to an earlier bitlinear_forward_batch.
  */
 int bitlinear_forward_batch_host(const bitlinear_problem* problems, int count, int flags, const void* x_host,
                                  void* x_dev, size_t x_bytes, const void* y_dev, void* y_host, size_t y_bytes,

@@ -22,7 +22,9 @@
 //             to a dot-product-of-four with the int8 activations; one accumulator per j keeps the
 //             scale uniform and the four are folded once per row block.
 #include <algorithm>
+#include <cstring>
 #include <map>
+#include <mutex>
 #include <tuple>
 #include <type_traits>
 #include <vector>
@@ -899,6 +901,63 @@ size_t decode_batch_workspace_bytes(const bitlinear_problem* problems, int count
     return plan_layout(fmt == BITLINEAR_WEIGHTS_DENSE5 ? (int)rows : count, kPlanGrid, xq, rows).total;
 }
 
+// What the host derives from the problem list of a call (everything the two launches need besides the plan in the
+// workspace).  A call with BITLINEAR_BATCH_REUSE_PLAN whose problem list is the one an earlier call planned into the same
+// workspace takes it from here instead of planning again (a 70-problem plan costs the host about as long as the kernel
+// runs).  Keyed by workspace address and a hash of the descriptors; a few entries, replaced in turn.
+struct PlanShape {
+    int n_prob, total_rb, grid, rows, table_cap, table_need;
+    size_t arena_max;
+};
+struct PlanCacheEntry {
+    const void* ws = nullptr;
+    uint64_t hash = 0;
+    int count = 0;
+    bool has_acc = false;
+    PlanShape shape = {};
+};
+constexpr int kPlanCacheEntries = 16;
+std::mutex g_plan_cache_mu;
+PlanCacheEntry g_plan_cache[kPlanCacheEntries];
+int g_plan_cache_next = 0;
+
+uint64_t hash_problems(const bitlinear_problem* problems, int count) {
+    // the descriptors word by word (their size is a multiple of 8); bytes of padding take part: a list that differs only
+    // there is planned again, which is correct and merely slower
+    static_assert(sizeof(bitlinear_problem) % 8 == 0, "hashed in 8-byte words");
+    uint64_t h = 1469598103934665603ull;
+    const size_t words = (size_t)count * sizeof(bitlinear_problem) / 8;
+    for (size_t i = 0; i < words; ++i) {
+        uint64_t w;
+        memcpy(&w, reinterpret_cast<const char*>(problems) + 8 * i, 8);
+        h = (h ^ w) * 1099511628211ull;
+        h ^= h >> 29;
+    }
+    return h;
+}
+
+bool plan_cache_find(const void* ws, uint64_t hash, int count, bool has_acc, PlanShape* out) {
+    std::lock_guard<std::mutex> lock(g_plan_cache_mu);
+    for (const PlanCacheEntry& e : g_plan_cache)
+        if (e.ws == ws && e.hash == hash && e.count == count && e.has_acc == has_acc) {
+            *out = e.shape;
+            return true;
+        }
+    return false;
+}
+
+void plan_cache_store(const void* ws, uint64_t hash, int count, bool has_acc, const PlanShape& shape) {
+    std::lock_guard<std::mutex> lock(g_plan_cache_mu);
+    PlanCacheEntry* slot = nullptr;
+    for (PlanCacheEntry& e : g_plan_cache)
+        if (e.ws == ws) slot = &e;  // one plan per workspace
+    if (!slot) {
+        slot = &g_plan_cache[g_plan_cache_next];
+        g_plan_cache_next = (g_plan_cache_next + 1) % kPlanCacheEntries;
+    }
+    slot->ws = ws; slot->hash = hash; slot->count = count; slot->has_acc = has_acc; slot->shape = shape;
+}
+
 // acc_outs: nullptr, or one (nullable) device pointer per problem for the raw accumulators.
 int decode_batch_forward(const bitlinear_problem* problems, int count, int flags, int32_t* const* acc_outs, void* ws,
                          size_t ws_bytes, void* stream) {
@@ -975,13 +1034,26 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         }
     }
 
+    // ---- the plan of an earlier call on this workspace, if the caller says it is still there and the problems are the same
+    //      (accumulator pointers are part of the device plan: calls that pass any are always planned)
+    const uint64_t list_hash = want_acc ? 0 : hash_problems(problems, count);
+    PlanShape shape = {};
+    const bool planned = !want_acc && (flags & BITLINEAR_BATCH_REUSE_PLAN) && plan_cache_find(ws, list_hash, count, false, &shape) &&
+                         shape.rows != 1;  // a single input row: the launch is built from the descriptors themselves
+
     // ---- host plan: device descriptors, token -> problem table, byte-balanced CTA ranges ----
     std::vector<DevProblem> dp;
     std::vector<int> row_prob;
     std::map<QuantKey, int> quantised;  // first entry of dp that quantises a given input
+    int total_rb = 0, n_prob = 0, grid = 0, table_cap = 1, table_need = 1;
+    size_t arena_max = 0;  // most activation bytes any CTA needs
+    std::vector<int4> cta_range;
+    if (planned) {
+        n_prob = shape.n_prob; total_rb = shape.total_rb; grid = shape.grid; rows = (size_t)shape.rows;
+        table_cap = shape.table_cap; table_need = shape.table_need; arena_max = shape.arena_max;
+    } else {
     dp.reserve(count);
     row_prob.reserve(rows + 1);
-    int total_rb = 0;
     {
         char* xq_ptr = base + L.xq_off;
         float* d_ptr = reinterpret_cast<float*>(base + align_up(L.xq_off + xq_bytes, 256));
@@ -1045,11 +1117,10 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         rows = (size_t)row;  // tokens actually quantised (shared copies counted once)
         row_prob.push_back(0);
     }
-    const int n_prob = (int)dp.size();
-    const int grid = sm_count < total_rb ? sm_count : total_rb;
-    std::vector<int4> cta_range(grid);
-    int table_cap = 1;     // most problems any CTA touches
-    size_t arena_max = 0;  // most activation bytes any CTA needs
+    n_prob = (int)dp.size();
+    grid = sm_count < total_rb ? sm_count : total_rb;
+    cta_range.resize(grid);
+    table_cap = 1;  // most problems any CTA touches
     {
         std::vector<int> cta_rb(grid + 1);
         double total_tiles = 0.0;
@@ -1091,15 +1162,22 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     // shared memory: chunk ring + descriptor table + activation arena; activations that do not fit the arena are read
     // through L1 instead, and only as many descriptors as fit a quarter of the space are cached
     // (the multi-token kernel caches no descriptors and keeps the rows of one problem at a time in its arena)
+    {
+        const size_t smem_limit = 227 * 1024 - (nt == 0 ? ring_bytes(5) : mma_ring_bytes(kMmaChunk, kMmaRing)) - 128;
+        if (nt) table_cap = 0;
+        table_need = table_cap;  // with fewer cached descriptors some problems of a CTA are read from global memory
+        if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
+        if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
+        if (nt) arena_max = std::min(align_up(arena_max, 256), smem_limit & ~(size_t)255);
+        else arena_max &= ~(size_t)255;
+    }
+    {   // (a call with accumulator pointers leaves no entry: its plan carries them)
+        const PlanShape made = {n_prob, total_rb, grid, (int)rows, table_cap, table_need, arena_max};
+        plan_cache_store(ws, want_acc ? 0 : list_hash, want_acc ? -1 : count, false, made);
+    }
+    }  // planned or not
     constexpr int chunk_tiles = 5;
     const size_t ring_total = nt == 0 ? ring_bytes(chunk_tiles) : mma_ring_bytes(kMmaChunk, kMmaRing);
-    const size_t smem_limit = 227 * 1024 - ring_total - 128;
-    if (nt) table_cap = 0;
-    const int table_need = table_cap;  // with fewer cached descriptors some problems of a CTA are read from global memory
-    if ((size_t)table_cap * sizeof(SProb) > smem_limit / 4) table_cap = (int)(smem_limit / 4 / sizeof(SProb));
-    if (arena_max > smem_limit - (size_t)table_cap * sizeof(SProb)) arena_max = smem_limit - (size_t)table_cap * sizeof(SProb);
-    if (nt) arena_max = std::min(align_up(arena_max, 256), smem_limit & ~(size_t)255);
-    else arena_max &= ~(size_t)255;
 
     PlanHeader hdr_host;
     hdr_host.magic = kPlanMagic;
@@ -1122,7 +1200,7 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
     // One input row in the whole call (a single token, every problem reading it the same way - the usual shape of one level
     // of a decoder layer at one token): no quantiser launch, the stream kernel quantises the row itself (FUSE).
     const bool fuse = rows == 1 && !(flags & BITLINEAR_BATCH_REUSE_ACT) && table_cap == table_need && max_k <= 16 * kStreamThreads;
-    if (fuse) arena_max = std::max(arena_max, align_up((size_t)dp[0].x_stride, 256));
+    if (fuse) arena_max = std::max(arena_max, align_up((size_t)dp[0].x_stride, 256));  // (never with a cached shape: rows != 1)
 
     // ... and when the problems are few (a level of a decoder layer) the whole call is one launch that carries its
     // descriptors in its arguments (decode_level.cu); the plan uploaded above stays valid for calls that reuse activations
@@ -1271,9 +1349,131 @@ int partition_problems(const bitlinear_problem* problems, int count, int32_t* co
 
 }  // namespace
 
-extern "C" {
+namespace {
 
-size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
+// ---- bitlinear_forward_batch_host in segments: while one segment's kernels run, the next one's inputs come in and the
+//      previous one's outputs go out (the copy engines work beside the SMs).
+constexpr int kHostSegments = 3;
+constexpr int kHostSegmentMinProblems = 8;  // per segment; smaller calls are not worth three pairs of launches
+
+struct HostSegments {
+    int cut[kHostSegments + 1];        // problems [cut[s], cut[s + 1])
+    size_t xcut[kHostSegments + 1];    // bytes [xcut[s], xcut[s + 1]) of the x arena belong to segment s
+    size_t ycut[kHostSegments + 1];
+    size_t ws_off[kHostSegments + 1];  // its slice of the workspace
+};
+
+// Decode-sized problems with a plain input whose operands lie in the arenas in the order of the problems: cut where a
+// third and two thirds of the packed bytes have gone by.  A segment's part of an arena begins where its lowest operand
+// begins and ends where the next segment's does, so the parts are disjoint and together the whole arena.  False where
+// any of that does not hold (the call then runs unsegmented).
+size_t batch_workspace_core(const bitlinear_problem* problems, int count);
+
+// which problems go into which segment (by shapes alone, so that the workspace can be sized without the arenas)
+bool host_segment_cuts(const bitlinear_problem* problems, int count, int (&cut)[kHostSegments + 1]) {
+    if (count < kHostSegments * kHostSegmentMinProblems) return false;
+    double total = 0.0;
+    for (int i = 0; i < count; ++i) {
+        const bitlinear_problem& q = problems[i];
+        if (q.M < 1 || q.M > kGemvMaxTokens || q.x_op != BITLINEAR_X_PLAIN || !shape_ok(q.N, q.K)) return false;
+        total += (double)q.N * q.K;
+    }
+    cut[0] = 0;
+    double run = 0.0;
+    int s = 1;
+    for (int i = 0; i < count && s < kHostSegments; ++i) {
+        run += (double)problems[i].N * problems[i].K;
+        if (run >= total * s / kHostSegments) cut[s++] = i + 1;
+    }
+    for (; s <= kHostSegments; ++s) cut[s] = count;
+    for (s = 0; s < kHostSegments; ++s)
+        if (cut[s + 1] - cut[s] < kHostSegmentMinProblems) return false;
+    return true;
+}
+
+// the workspace the segments of a call need together (0: the call is not segmented)
+size_t host_segments_workspace(const bitlinear_problem* problems, int count) {
+    int cut[kHostSegments + 1];
+    if (!problems || !host_segment_cuts(problems, count, cut)) return 0;
+    size_t total = 0;
+    for (int s = 0; s < kHostSegments; ++s) {
+        const size_t need = batch_workspace_core(problems + cut[s], cut[s + 1] - cut[s]);
+        if (need == 0) return 0;
+        total += align_up(need, 1024);
+    }
+    return total;
+}
+
+bool plan_host_segments(const bitlinear_problem* problems, int count, const void* x_dev, size_t x_bytes, const void* y_dev,
+                        size_t y_bytes, size_t ws_bytes, HostSegments* out) {
+    HostSegments sg;
+    if (!host_segment_cuts(problems, count, sg.cut)) return false;
+    const char* xb = static_cast<const char*>(x_dev);
+    const char* yb = static_cast<const char*>(y_dev);
+    for (int i = 0; i < count; ++i)
+        if (!problems[i].x || !problems[i].y) return false;
+    const char *x_lo[kHostSegments], *x_hi[kHostSegments], *y_lo[kHostSegments], *y_hi[kHostSegments];
+    sg.ws_off[0] = 0;
+    for (int s = 0; s < kHostSegments; ++s) {
+        const int n = sg.cut[s + 1] - sg.cut[s];
+        x_lo[s] = x_hi[s] = y_lo[s] = y_hi[s] = nullptr;
+        for (int i = sg.cut[s]; i < sg.cut[s + 1]; ++i) {
+            const bitlinear_problem& q = problems[i];
+            const char* x0 = static_cast<const char*>(q.x);
+            const char* x1 = x0 + (size_t)q.M * q.K * 2;
+            const char* y0 = static_cast<const char*>(q.y);
+            const char* y1 = y0 + (size_t)q.M * q.N * (q.y_dtype == BITLINEAR_BF16 ? 2 : 4);
+            if (x0 < xb || x1 > xb + x_bytes || y0 < yb || y1 > yb + y_bytes) return false;
+            if (!x_lo[s] || x0 < x_lo[s]) x_lo[s] = x0;
+            if (!x_hi[s] || x1 > x_hi[s]) x_hi[s] = x1;
+            if (!y_lo[s] || y0 < y_lo[s]) y_lo[s] = y0;
+            if (!y_hi[s] || y1 > y_hi[s]) y_hi[s] = y1;
+        }
+        if (s > 0 && (x_hi[s - 1] > x_lo[s] || y_hi[s - 1] > y_lo[s])) return false;  // a part reaches into the next one
+        sg.xcut[s] = s == 0 ? 0 : (size_t)(x_lo[s] - xb);
+        sg.ycut[s] = s == 0 ? 0 : (size_t)(y_lo[s] - yb);
+        const size_t need = batch_workspace_core(problems + sg.cut[s], n);
+        if (need == 0) return false;
+        sg.ws_off[s + 1] = sg.ws_off[s] + align_up(need, 1024);
+    }
+    sg.xcut[kHostSegments] = x_bytes;
+    sg.ycut[kHostSegments] = y_bytes;
+    if (sg.ws_off[kHostSegments] > ws_bytes) return false;
+    *out = sg;
+    return true;
+}
+
+struct HostPipe {
+    cudaStream_t side[kHostSegments - 1];
+    cudaEvent_t fork, done[kHostSegments - 1];
+    bool tried = false, ok = false;
+};
+std::mutex g_host_pipe_mu;  // held while a call enqueues its segments: the streams and events are shared per device
+HostPipe g_host_pipe[64];
+
+HostPipe* host_pipe_locked() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    HostPipe& hp = g_host_pipe[dev];
+    if (!hp.tried) {
+        hp.tried = true;
+        bool ok = cudaEventCreateWithFlags(&hp.fork, cudaEventDisableTiming) == cudaSuccess;
+        for (int i = 0; i < kHostSegments - 1 && ok; ++i)
+            ok = cudaStreamCreateWithFlags(&hp.side[i], cudaStreamNonBlocking) == cudaSuccess &&
+                 cudaEventCreateWithFlags(&hp.done[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!ok) cudaGetLastError();
+        hp.ok = ok;
+    }
+    return hp.ok ? &hp : nullptr;
+}
+
+}  // namespace
+
+namespace {
+size_t batch_workspace_core(const bitlinear_problem* problems, int count) {
     if (!problems || count <= 0) return 0;
     std::vector<bitlinear_problem> dec;
     std::vector<int32_t*> dec_acc;
@@ -1283,6 +1483,14 @@ size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int co
     if (!dec.empty()) total += align_up(decode_batch_workspace_bytes(dec.data(), (int)dec.size()), 1024);
     if (!pre.empty()) total += prefill_group_workspace_bytes(problems, pre.data(), (int)pre.size());
     return total;
+}
+}  // namespace
+
+extern "C" {
+
+size_t bitlinear_batch_workspace_bytes(const bitlinear_problem* problems, int count) {
+    // bitlinear_forward_batch_host may run a long decode call as kHostSegments calls with a plan each
+    return std::max(batch_workspace_core(problems, count), host_segments_workspace(problems, count));
 }
 
 int bitlinear_forward_batch(const bitlinear_problem* problems, int count, int flags, void* ws, size_t ws_bytes,
@@ -1330,6 +1538,42 @@ int bitlinear_forward_batch_host(const bitlinear_problem* problems, int count, i
                                  size_t ws_bytes, void* stream) {
     if (count > 0 && (!x_host || !x_dev || !y_dev || !y_host)) return BITLINEAR_ERR_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    HostSegments sg;
+    if (count > 0 && problems && ws && plan_host_segments(problems, count, x_dev, x_bytes, y_dev, y_bytes, ws_bytes, &sg)) {
+        std::unique_lock<std::mutex> lock(g_host_pipe_mu);
+        if (HostPipe* hp = host_pipe_locked()) {
+            // segment 0 runs on the caller's stream, the others on side streams that start after the caller's earlier work
+            // and that the caller's stream waits for at the end
+            bool cuda_ok = cudaEventRecord(hp->fork, st) == cudaSuccess;
+            for (int i = 0; i < kHostSegments - 1 && cuda_ok; ++i) cuda_ok = cudaStreamWaitEvent(hp->side[i], hp->fork, 0) == cudaSuccess;
+            int rc = BITLINEAR_OK;
+            for (int s = 0; s < kHostSegments && cuda_ok && rc == BITLINEAR_OK; ++s) {
+                cudaStream_t ss = s == 0 ? st : hp->side[s - 1];
+                const size_t xn = sg.xcut[s + 1] - sg.xcut[s], yn = sg.ycut[s + 1] - sg.ycut[s];
+                if (xn > 0)
+                    cuda_ok = cudaMemcpyAsync(static_cast<char*>(x_dev) + sg.xcut[s], static_cast<const char*>(x_host) + sg.xcut[s], xn,
+                                              cudaMemcpyHostToDevice, ss) == cudaSuccess;
+                if (cuda_ok)
+                    rc = bitlinear_forward_batch(problems + sg.cut[s], sg.cut[s + 1] - sg.cut[s], flags, static_cast<char*>(ws) + sg.ws_off[s],
+                                                 sg.ws_off[s + 1] - sg.ws_off[s], ss);
+                if (cuda_ok && rc == BITLINEAR_OK && yn > 0)
+                    cuda_ok = cudaMemcpyAsync(static_cast<char*>(y_host) + sg.ycut[s], static_cast<const char*>(y_dev) + sg.ycut[s], yn,
+                                              cudaMemcpyDeviceToHost, ss) == cudaSuccess;
+            }
+            // join whatever was started, also after an error
+            for (int i = 0; i < kHostSegments - 1; ++i)
+                if (cudaEventRecord(hp->done[i], hp->side[i]) != cudaSuccess || cudaStreamWaitEvent(st, hp->done[i], 0) != cudaSuccess)
+                    cuda_ok = false;
+            lock.unlock();
+            if (cudaStreamSynchronize(st) != cudaSuccess) cuda_ok = false;
+            if (rc != BITLINEAR_OK) return rc;
+            if (!cuda_ok) {
+                cudaGetLastError();
+                return BITLINEAR_ERR_CUDA;
+            }
+            return BITLINEAR_OK;
+        }
+    }
     if (count > 0 && x_bytes > 0 && cudaMemcpyAsync(x_dev, x_host, x_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) {
         cudaGetLastError();
         return BITLINEAR_ERR_CUDA;

@@ -125,6 +125,64 @@ def test_batch_several_tokens_accumulators_and_shared_inputs(M):
         assert torch.equal(a, t[4])
 
 
+@pytest.mark.parametrize("n_prob,M,order", [(6, 1, "forward"), (30, 1, "forward"), (27, 3, "forward"), (30, 1, "reversed")])
+def test_batch_host_buffers_match_the_device_call(n_prob, M, order):
+    """bitlinear_forward_batch_host (pinned x arena in, y arena out) against bitlinear_forward_batch on the same
+    descriptors: the same bits, for a call too short to be cut into segments, for calls that are cut into three
+    segments whose copies overlap the kernels, for arenas laid out against the order of the problems (not cut), and for
+    a second call that reuses the plans."""
+    shapes = [(48, 768), (640, 2560), (256, 1024), (128, 256), (2560, 2560), (16, 512)]
+    seed = 5200 + n_prob + M
+    mats = []
+    for i in range(len(shapes)):
+        N, K = shapes[i]
+        W = wl.latent_weights(N, K, seed + i)
+        mats.append(bl.bitlinear_pack_weights(W.to(DEV), wl.WEIGHT_EPS))
+    specs = [shapes[i % len(shapes)] + (i % len(shapes),) for i in range(n_prob)]
+    x_off, y_off, xo, yo = [], [], 0, 0
+    for N, K, _ in specs:
+        x_off.append(xo)
+        y_off.append(yo)
+        xo += (M * K * 2 + 255) // 256 * 256
+        yo += (M * N * 4 + 255) // 256 * 256
+    if order == "reversed":
+        x_off = [xo - o - (M * K * 2 + 255) // 256 * 256 for o, (N, K, _) in zip(x_off, specs)]
+        y_off = [yo - o - (M * N * 4 + 255) // 256 * 256 for o, (N, K, _) in zip(y_off, specs)]
+    x_host = torch.zeros(xo, dtype=torch.uint8).pin_memory()
+    y_host = torch.zeros(yo, dtype=torch.uint8).pin_memory()
+    x_dev = torch.zeros(xo, dtype=torch.uint8, device=DEV)
+    y_dev = torch.zeros(yo, dtype=torch.uint8, device=DEV)
+    gain = {K: wl.gain_random(K, seed + 100 + K).to(DEV) for _, K in shapes}
+    items = []
+    for i, (N, K, mi) in enumerate(specs):
+        x = wl.activations_normal(M, K, seed + 200 + i)
+        nb = M * K * 2
+        x_host[x_off[i]:x_off[i] + nb] = x.view(torch.uint8).reshape(-1)
+        xv = x_dev[x_off[i]:x_off[i] + nb].view(torch.bfloat16).view(M, K)
+        yv = y_dev[y_off[i]:y_off[i] + M * N * 4].view(torch.float32).view(M, N)
+        items.append((xv, gain[K], mats[mi][0], mats[mi][1], yv))
+    batch = bl.ProblemBatch(items, wl.RMS_EPS)
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    # the device call on a copy of the inputs gives the expected bytes
+    x_dev.copy_(x_host)
+    bl.bitlinear_forward_batch(batch, ws)
+    torch.cuda.synchronize()
+    want = y_dev.cpu().clone()
+    for reuse in (False, True):
+        x_dev.zero_()
+        y_dev.fill_(0xEE)
+        y_host.fill_(0x11)
+        bl.bitlinear_forward_batch_host(batch, x_host, x_dev, y_dev, y_host, ws, reuse_plan=reuse)  # synchronises
+        assert bl.bitlinear_poll_status() == 0
+        got = y_host.clone()
+        # bytes between two outputs are padding of the arena: the device call left them as they were (zero), the host call
+        # copies them out as they are now (0xEE); compare the outputs themselves
+        for i, (N, K, _) in enumerate(specs):
+            sl = slice(y_off[i], y_off[i] + M * N * 4)
+            assert torch.equal(got[sl], want[sl]), (i, reuse)
+        assert torch.equal(x_dev.cpu(), x_host)
+
+
 def test_batch_bf16_output_and_empty_problem():
     shapes = [(4, 64, 512), (0, 32, 256), (1, 640, 2560)]
     batch, refs = make_case(shapes, 400, y_dtype=torch.bfloat16)
