@@ -110,6 +110,34 @@ __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHe
         for (int k = p.K + 4 * threadIdx.x; k < p.x_stride; k += 4 * kQuantThreads) *reinterpret_cast<uint32_t*>(xq_row + k) = 0u;
 }
 
+// The same for calls with more tokens than SMs (several tokens per problem): kQuantGroupWarps warps per token and
+// several tokens per CTA, so that a wave of CTAs covers more tokens and a token's chain stays short.  Launched as a
+// programmatic dependent of whatever runs before it (its launch overlaps that kernel's tail); it touches nothing
+// before that kernel is complete.
+template <int kQuantGroupWarps>
+__global__ void __launch_bounds__(kQuantThreads) batch_quant_group_kernel(const PlanHeader* __restrict__ hdr,
+                                                                          const DevProblem* __restrict__ probs,
+                                                                          const int* __restrict__ row_prob, int count, int total_rb,
+                                                                          int grid, int rows, int* status_word) {
+    constexpr int kGroups = kQuantWarps / kQuantGroupWarps;  // tokens per CTA
+    __shared__ GroupReduceSmem sm[kGroups];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!plan_matches(hdr, count, total_rb, grid, rows)) {
+        if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
+        return;
+    }
+    const int group = threadIdx.x / (32 * kQuantGroupWarps);
+    const int row = blockIdx.x * kGroups + group;
+    if (row >= rows) return;  // the whole group leaves: nobody is left waiting at its barrier
+    const DevProblem& p = probs[row_prob[row]];
+    const int m = row - p.row_begin;
+    with_row_source(p.op, p.x, p.x_row0 + m, p.K, [&](auto src) {
+        quant_row_group_src<1, kQuantGroupWarps>(src, p.gain, p.eps, p.K, p.xq + (size_t)m * p.x_stride, p.d + m, p.xsum + m, sm[group],
+                                                 1 + group);
+    });
+}
+
 // ------------------------------------------------------------------------------------ launch 2
 
 __device__ __forceinline__ int dp4a_u8_s8(uint32_t a_u8x4, uint32_t b_s8x4, int c) {
@@ -1228,7 +1256,29 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
         const PlanHeader* h = reinterpret_cast<const PlanHeader*>(base);
         const int* rp = reinterpret_cast<const int*>(base + L.row_prob_off);
         int* sw = device_status_word();
-        if (dense) {
+        if (nt && (int)rows > sm_count) {
+            // more tokens than SMs: groups of warps per token (two tokens per CTA while eight CTAs per SM hold them all)
+            cudaLaunchConfig_t qcfg = {};
+            qcfg.blockDim = dim3(kQuantThreads);
+            qcfg.stream = st;
+            cudaLaunchAttribute qattr[1];
+            qattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            qattr[0].val.programmaticStreamSerializationAllowed = 1;
+            qcfg.attrs = qattr;
+            qcfg.numAttrs = 1;
+            cudaError_t qe;
+            if ((int)rows <= 2 * 8 * sm_count) {
+                qcfg.gridDim = dim3((unsigned)((rows + 1) / 2));
+                qe = cudaLaunchKernelEx(&qcfg, batch_quant_group_kernel<4>, h, probs_dev, rp, n_prob, total_rb, grid, (int)rows, sw);
+            } else {
+                qcfg.gridDim = dim3((unsigned)((rows + 3) / 4));
+                qe = cudaLaunchKernelEx(&qcfg, batch_quant_group_kernel<2>, h, probs_dev, rp, n_prob, total_rb, grid, (int)rows, sw);
+            }
+            if (qe != cudaSuccess) {
+                cudaGetLastError();
+                return BITLINEAR_ERR_CUDA;
+            }
+        } else if (dense) {
             if (vpt <= 1) batch_quant_kernel<1, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
             else if (vpt <= 2) batch_quant_kernel<2, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
             else batch_quant_kernel<4, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);

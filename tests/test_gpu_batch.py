@@ -259,7 +259,7 @@ def test_batch_many_tokens_match_single_forward_bitwise(M):
         assert torch.equal(y, y1)
 
 
-@pytest.mark.parametrize("M", [1, 16])
+@pytest.mark.parametrize("M", [1, 8, 16])  # the three kernels: one token, 2 to 8 tokens (mma.sync stream), 9 to 16 (tcgen05)
 def test_batch_full_decode_step_sampled(M):
     # the launch configuration the benchmark times, with its seeded weights: 30 layers x 7 matmuls in ONE call
     # (210 problems, 521 MB of packed weights), checked on sampled outputs of every problem
