@@ -95,6 +95,10 @@ __global__ void __launch_bounds__(kQuantThreads) batch_quant_kernel(const PlanHe
     // the stream kernel that follows may start now: it fetches weights first and waits for this grid before it reads
     // anything written here (programmatic dependent launch)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    // itself a programmatic dependent of whatever runs before it on the stream (its launch overlaps that kernel's tail -
+    // in a decode loop the previous step's stream kernel, which still reads what this kernel is about to overwrite):
+    // nothing is read or written before that kernel is complete
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (!plan_matches(hdr, count, total_rb, grid, (int)gridDim.x)) {
         if (blockIdx.x == 0 && threadIdx.x == 0 && status_word != nullptr) atomicExch(status_word, BITLINEAR_ERR_WORKSPACE);
         return;
@@ -1278,16 +1282,26 @@ int decode_batch_forward(const bitlinear_problem* problems, int count, int flags
                 cudaGetLastError();
                 return BITLINEAR_ERR_CUDA;
             }
-        } else if (dense) {
-            if (vpt <= 1) batch_quant_kernel<1, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
-            else if (vpt <= 2) batch_quant_kernel<2, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
-            else batch_quant_kernel<4, 0><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
         } else {
-            if (vpt <= 1) batch_quant_kernel<1, 1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
-            else if (vpt <= 2) batch_quant_kernel<2, 1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
-            else batch_quant_kernel<4, 1><<<g, b, 0, st>>>(h, probs_dev, rp, n_prob, total_rb, grid, sw);
+            cudaLaunchConfig_t qcfg = {};
+            qcfg.gridDim = g;
+            qcfg.blockDim = b;
+            qcfg.stream = st;
+            cudaLaunchAttribute qattr[1];
+            qattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+            qattr[0].val.programmaticStreamSerializationAllowed = 1;
+            qcfg.attrs = qattr;
+            qcfg.numAttrs = 1;
+            auto launch_q = [&](auto kernel) { return cudaLaunchKernelEx(&qcfg, kernel, h, probs_dev, rp, n_prob, total_rb, grid, sw); };
+            const cudaError_t qe = dense ? (vpt <= 1 ? launch_q(batch_quant_kernel<1, 0>) : vpt <= 2 ? launch_q(batch_quant_kernel<2, 0>)
+                                                                                                : launch_q(batch_quant_kernel<4, 0>))
+                                         : (vpt <= 1 ? launch_q(batch_quant_kernel<1, 1>) : vpt <= 2 ? launch_q(batch_quant_kernel<2, 1>)
+                                                                                                : launch_q(batch_quant_kernel<4, 1>));
+            if (qe != cudaSuccess) {
+                cudaGetLastError();
+                return BITLINEAR_ERR_CUDA;
+            }
         }
-        if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
 
     // ---- launch 2: stream the weights ----

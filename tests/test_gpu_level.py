@@ -82,6 +82,53 @@ def test_level_launch_matches_oracle(K, shapes, with_gain):
     assert bl.bitlinear_poll_status() == 0
 
 
+@pytest.mark.parametrize("M,K,shapes,with_gain", [
+    (2, 256, (16,), False),                        # one row block, one tile
+    (8, 256, (16, 32, 48, 16), True),              # four problems, eight tokens
+    (3, 2560, (2560, 640, 640), True),             # q, k, v of the 2B layer
+    (8, 2560, (6912, 6912), False),                # gate, up: three row blocks per CTA
+    (5, 6912, (2560,), True),                      # down: 27 tiles per row block
+    (8, 8192, (256, 16), True),                    # the largest K, the largest arena
+    (4, 512, (16 * 700,), False),                  # several row blocks per warp
+])
+def test_level_launch_at_several_tokens_matches_oracle(M, K, shapes, with_gain):
+    """A level at 2 to 8 tokens (a quantiser launch and the multi-token stream kernel on a handful of problems that share
+    their input): int32 accumulators bit for bit, outputs within the suite's bound, the same bits with the plan and then
+    the quantised rows reused."""
+    seed = 7300 + K + len(shapes) + M
+    mats = make_mats(shapes, K, seed)
+    x = wl.activations_student_t(M, K, seed + 50)
+    gain = wl.gain_random(K, seed + 51) if with_gain else None
+    gdev = gain.to(DEV) if with_gain else None
+    ys = [torch.full((M, n), float("nan"), dtype=torch.bfloat16 if i % 2 else torch.float32, device=DEV) for i, (_, _, _, n) in enumerate(mats)]
+    accs = [torch.full((M, n), -1, dtype=torch.int32, device=DEV) for (_, _, _, n) in mats]
+    xd = x.to(DEV)
+    items = [(xd, gdev, packed, s_w, y) for (packed, s_w, _, _), y in zip(mats, ys)]
+    batch = bl.ProblemBatch(items, wl.RMS_EPS)
+    ws = torch.empty(batch.workspace_bytes(), dtype=torch.uint8, device=DEV)
+    refs = [oracle.bitlinear_forward(wl.bf16_bits(x), wl.bf16_bits(gain) if with_gain else None, wl.RMS_EPS, m[2]["wq"], m[2]["s_w"])
+            for m in mats]
+    bl.bitlinear_forward_batch_acc(batch, accs, ws)
+    torch.cuda.synchronize()
+    assert bl.bitlinear_poll_status() == 0
+    for y, acc, ref in zip(ys, accs, refs):
+        ok = ref["fragile"] == 0
+        assert ok.all()
+        assert np.array_equal(acc.cpu().numpy(), ref["acc"])
+        got, want = y.float().cpu().numpy().astype(np.float64), ref["y"].astype(np.float64)
+        tol = 1e-6 if y.dtype == torch.float32 else 2.0 ** -7
+        assert np.all(np.abs(got - want) <= tol * np.abs(want))
+    first = [y.clone() for y in ys]
+    for kwargs in (dict(reuse_plan=True), dict(reuse_plan=True, reuse_act=True)):
+        for y in ys:
+            y.fill_(float("nan"))
+        bl.bitlinear_forward_batch(batch, ws, **kwargs)
+        torch.cuda.synchronize()
+        for a, y in zip(first, ys):
+            assert torch.equal(a, y)
+    assert bl.bitlinear_poll_status() == 0
+
+
 def test_level_launch_with_fused_steps_writes_their_output_once():
     H, F, n_q, n_kv, hd = 2560, 6912, 20, 5, 128
     seed = 7700
