@@ -7,7 +7,8 @@
 //
 //   launch 1  batch_quant_kernel : one CTA per token of every problem - fused RMSNorm + absmax
 //             int8 quantiser into the workspace (codes stored in the lane-interleaved order the
-//             stream kernel reads, see quant_row).
+//             stream kernel reads, see quant_row).  A programmatic dependent of the launch before
+//             it: in a decode loop its launch overlaps the previous step's stream kernel.
 //   launch 2  decode_stream_kernel : one persistent CTA of 16 warps per SM.  The work list is every
 //             block of 16 weight rows of every problem; each CTA owns a contiguous, byte-balanced
 //             range of it.  A row block belongs to ONE warp, so 16 row blocks are in progress per CTA
@@ -19,8 +20,11 @@
 //             Before the stream starts the CTA copies the descriptors of the few problems its range
 //             touches, and their quantised activations, into shared memory once.
 //             Unpack: word & (0x03030303 << 2j) is 4^j x the codes of four consecutive columns, fed
-//             to a dot-product-of-four with the int8 activations; one accumulator per j keeps the
-//             scale uniform and the four are folded once per row block.
+//             to a dot-product-of-four with the int8 activations (j = 0, 1) or, as one of four
+//             operand registers, to an int8 mma.sync whose token columns all carry the one token
+//             (j = 2, 3: the integer pipe, which does the masks and the quarter-rate dot products,
+//             is the busiest unit; the tensor pipe is idle otherwise); one accumulator per j keeps
+//             the scale uniform and the four are folded once per row block.
 #include <algorithm>
 #include <cstring>
 #include <map>
@@ -1428,7 +1432,8 @@ struct HostSegments {
 };
 
 // Decode-sized problems with a plain input whose operands lie in the arenas in the order of the problems: cut where a
-// third and two thirds of the packed bytes have gone by.  A segment's part of an arena begins where its lowest operand
+// third and two thirds of the packed bytes have gone by (cuts at 45 and 80 % measured the same: the call is bound by the
+// host's enqueue time either way).  A segment's part of an arena begins where its lowest operand
 // begins and ends where the next segment's does, so the parts are disjoint and together the whole arena.  False where
 // any of that does not hold (the call then runs unsegmented).
 size_t batch_workspace_core(const bitlinear_problem* problems, int count);
