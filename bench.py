@@ -31,7 +31,7 @@ from paper_2504_12285_b200 import workloads as wl  # noqa: E402
 
 METRIC = "bitlinear_decode_packed_weight_bandwidth_m1"
 UNIT = "GB/s"
-CONFIG_ID = 2  # BASELINE configs[1]: decode step over all 7 BitLinear shapes of one 2B-style layer
+CONFIG_ID = 2  # seed family of the headline workload: a decode step over all 7 BitLinear shapes of a 2B-style layer, 30 layers
 WORKLOAD = ("configs[1] at M=1: decode step over the 7 BitLinear shapes of a 2B-style layer "
             "(q,k,v,o,gate,up,down), rotated over 30 independently seeded layers = 210 forwards, "
             "521,011,200 packed-weight bytes per step")
