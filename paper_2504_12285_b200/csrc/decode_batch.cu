@@ -296,10 +296,11 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_kernel(const 
         ld.set_problem(probs[ld.p].rb_begin, probs[ld.p].rb_end, probs[ld.p].k_tiles, probs[ld.p].packed, kChunkTiles);
     }
     ChunkCursor cp = ld;  // where the arithmetic is
+    const uint64_t once = l2_evict_first_policy();  // the weights pass through L2 once
     auto issue = [&](int slot) {  // lane 0 only
         const uint32_t bytes = (uint32_t)ld.tiles() * kTileBytes;
         mbar_expect_tx(bar_s + 8u * slot, bytes);
-        bulk_load(ring_s + (uint32_t)slot * kSlotBytes, ld.src(), bytes, bar_s + 8u * slot);
+        bulk_load_once(ring_s + (uint32_t)slot * kSlotBytes, ld.src(), bytes, bar_s + 8u * slot, once);
     };
     auto advance_ld = [&](bool may_enter) {
         if (++ld.c == ld.nc) {
@@ -682,10 +683,11 @@ __global__ void __launch_bounds__(kStreamThreads, 1) decode_stream_mma_kernel(co
         ld.set_problem(probs[ld.p].rb_begin, probs[ld.p].rb_end, probs[ld.p].k_tiles, probs[ld.p].packed, kChunkTiles);
     };
     if (mine) enter_ld();
+    const uint64_t once = l2_evict_first_policy();  // the weights pass through L2 once
     auto issue = [&](int slot) {  // lane 0 only
         const uint32_t bytes = (uint32_t)ld.tiles() * kTileBytes;
         mbar_expect_tx(bar_s + 8u * slot, bytes);
-        bulk_load(ring_s + (uint32_t)slot * kSlotBytes, ld.src(), bytes, bar_s + 8u * slot);
+        bulk_load_once(ring_s + (uint32_t)slot * kSlotBytes, ld.src(), bytes, bar_s + 8u * slot, once);
     };
     auto advance_ld = [&]() {
         if (++ld.c == ld.nc) {

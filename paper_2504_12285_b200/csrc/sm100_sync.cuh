@@ -68,6 +68,19 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, ui
                  : "memory");
 }
 
+// The same for data that is read once (a weight stream larger than L2): the lines are marked evict-first, so that they
+// do not push out what is read again (activations, descriptors, the outputs on their way to memory).
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t policy;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(policy));
+    return policy;
+}
+__device__ __forceinline__ void bulk_load_once(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst_smem),
+                 "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+                 : "memory");
+}
+
 // After an abort: give copies that may still be in flight time to land before shared memory goes away.
 __device__ __forceinline__ void abort_drain() {
     const unsigned long long t0 = globaltimer_ns();
