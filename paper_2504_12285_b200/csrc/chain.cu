@@ -239,8 +239,8 @@ __global__ void __launch_bounds__(kChainLaunchThreads, 1) decode_chain_kernel(co
         __syncwarp();
         for (int j = lane; j < n_jobs; j += 32) {
             const Job jb = level_job(level, j, sc, p);
-            bulk_load(smem_u32(wbuf + (size_t)(L & 1) * p.buf_bytes) + (uint32_t)j * rb_bytes,
-                      dsc.packed[jb.mat] + (size_t)jb.rb * rb_bytes, rb_bytes, bar);
+            bulk_load_once(smem_u32(wbuf + (size_t)(L & 1) * p.buf_bytes) + (uint32_t)j * rb_bytes,
+                           dsc.packed[jb.mat] + (size_t)jb.rb * rb_bytes, rb_bytes, bar, l2_evict_first_policy());  // weights: read once
         }
     };
     bool ok = true;

@@ -88,7 +88,8 @@ __global__ void __launch_bounds__(kLevelThreads) decode_level_kernel(const __gri
         for (int j = warp; j < R; j += kLevelWarps) {
             int i, local;
             locate(rb_lo + j, i, local);
-            bulk_load(w_s + (uint32_t)j * rb_bytes, P.prob[i].packed + (size_t)local * rb_bytes, rb_bytes, bar_s);
+            bulk_load_once(w_s + (uint32_t)j * rb_bytes, P.prob[i].packed + (size_t)local * rb_bytes, rb_bytes, bar_s,
+                           l2_evict_first_policy());  // a decode loop's weights pass through L2 once per token
         }
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     // what else does not depend on the launch before this one: the gain vector and the weight scales

@@ -325,8 +325,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) decode_mma_kernel(const MmaPar
                 __syncwarp();
                 if (lane < kCopiesPerWarp) {
                     if (c < n_rb)
-                        bulk_load(p_s + slot * kPackedSlot + c * (kStepTiles * kTileBytes), src_row + (size_t)t0 * kTileBytes,
-                                  (uint32_t)tiles * kTileBytes, pfull + 8 * slot);
+                        bulk_load_once(p_s + slot * kPackedSlot + c * (kStepTiles * kTileBytes), src_row + (size_t)t0 * kTileBytes,
+                                       (uint32_t)tiles * kTileBytes, pfull + 8 * slot, l2_evict_first_policy());  // weights: read once
                     else if (c == kItemRb)
                         bulk_load(x_s + slot * kXSlot, p.x_img + (size_t)t0 * 2 * kTok * 128, (uint32_t)tiles * 2 * kTok * 128,
                                   pfull + 8 * slot);

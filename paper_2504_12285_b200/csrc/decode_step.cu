@@ -120,10 +120,12 @@ __host__ __device__ inline AttnSlices attn_slices(int len, int splits) {
     return {per, (tiles + per - 1) / per};
 }
 
-__device__ __forceinline__ void tma_tile_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+// (cache rows are read once per call: marked evict-first in L2, so that a context longer than L2 does not push out what
+// is read again - the partial results, the projections)
+__device__ __forceinline__ void tma_tile_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar, uint64_t policy) {
     asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
-        "l"(map), "r"(x), "r"(y), "r"(bar)
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst),
+        "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy)
         : "memory");
 }
 // four 8 x 8 matrices of 16-bit elements, row addresses from lanes 8i .. 8i+7 for matrix i
@@ -251,14 +253,15 @@ __global__ void __launch_bounds__(160) attn_decode_partial_kernel(const __grid_c
         // ---- producer: one lane feeds the ring
         if (lane == 0) {
             const int row0 = (seq * n_kv + kvh) * t_max + tile0 * kAttnKeys;  // this head's rows are contiguous
+            const uint64_t once = l2_evict_first_policy();
             for (int i = 0; i < n_tiles; ++i) {
                 const uint32_t st = (uint32_t)(i % stages), dst = ring_s + st * 2u * kTileBytes, bar = full_s + 8u * st;
                 if (i >= stages && !mbar_wait(empty_s + 8u * st, (uint32_t)(i / stages - 1) & 1u, abort_flag)) break;
                 mbar_expect_tx(bar, 2u * kTileBytes);
 #pragma unroll
                 for (int hf = 0; hf < HALVES; ++hf) {
-                    tma_tile_2d(dst + hf * kHalfBytes, &map_k, hf * 64, row0 + i * kAttnKeys, bar);
-                    tma_tile_2d(dst + kTileBytes + hf * kHalfBytes, &map_v, hf * 64, row0 + i * kAttnKeys, bar);
+                    tma_tile_2d(dst + hf * kHalfBytes, &map_k, hf * 64, row0 + i * kAttnKeys, bar, once);
+                    tma_tile_2d(dst + kTileBytes + hf * kHalfBytes, &map_v, hf * 64, row0 + i * kAttnKeys, bar, once);
                 }
             }
         }
