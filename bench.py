@@ -212,9 +212,9 @@ def run_ours(args):
                 "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                 "frac": round(achieved / peaks["hbm_gbs"], 4), "algorithmic_bytes_per_launch": packed_bytes,
                 "avg_launch_us": round(stream_s * 1e6, 2),
-                # dram__bytes_read.sum + dram__bytes_write.sum of this kernel on 10 of the 30 layers (173.96 MB + 4.42 MB,
+                # dram__bytes_read.sum + dram__bytes_write.sum of this kernel on 10 of the 30 layers (173.96 MB + 4.00 MB,
                 # profiles/decode_stream_10layers_m1.md), times 3: it streams every packed byte once
-                "traffic": 3 * (173962240 + 4424960),
+                "traffic": 3 * (173959936 + 4003584),
                 "traffic_source": "ncu capture of a 10-layer launch (profiles/decode_stream_10layers_m1.md) scaled x3, not measured in this run"}
 
     # ---- sustained leg: the same step repeated for at least half a second, with the SM clock sampled meanwhile ----
