@@ -183,6 +183,23 @@ def test_batch_host_buffers_match_the_device_call(n_prob, M, order):
         assert torch.equal(x_dev.cpu(), x_host)
 
 
+def test_batch_one_workspace_serves_different_problem_lists_in_turn():
+    """Calls that reuse their plan skip the host's planning when the library remembers the list it planned for that
+    workspace.  Two different lists (other shapes, other token counts, the same number of problems) take turns on ONE
+    workspace: every call that plans anew must replace what is remembered, every reusing call must run its own list."""
+    batch_a, refs_a = make_case([(1, 48, 768), (1, 640, 2560), (1, 256, 1024), (1, 128, 256), (1, 32, 512)], 5600, gains=True)
+    batch_b, refs_b = make_case([(3, 64, 512), (5, 16, 256), (2, 2560, 2560), (8, 48, 768), (1, 640, 2560)], 5700)
+    ws = torch.empty(max(batch_a.workspace_bytes(), batch_b.workspace_bytes()), dtype=torch.uint8, device=DEV)
+    for batch, refs in ((batch_a, refs_a), (batch_b, refs_b), (batch_a, refs_a), (batch_b, refs_b)):
+        for reuse in (False, True, True):
+            for t in batch.tensors:
+                t[4].fill_(float("nan"))
+            bl.bitlinear_forward_batch(batch, ws, reuse_plan=reuse)
+            torch.cuda.synchronize()
+            assert bl.bitlinear_poll_status() == 0
+            check(batch, refs)
+
+
 def test_batch_bf16_output_and_empty_problem():
     shapes = [(4, 64, 512), (0, 32, 256), (1, 640, 2560)]
     batch, refs = make_case(shapes, 400, y_dtype=torch.bfloat16)
